@@ -1,0 +1,635 @@
+/*
+ * fho.c -- CPU oracle for Channel-wise Mix Compression (FedHybrid, arXiv 2510.11400, Section 4.4.1).
+ *
+ * THIS IS TEST INFRASTRUCTURE.  It is a plain, slow, step-by-step statement of what the codec
+ * computes, written from the paper, and exists only so that tests, the smoke check and the
+ * benchmark's CPU-baseline leg can compare the CUDA library against it.  It shares no code with
+ * the CUDA library and must never be used as a fallback for it.
+ *
+ * The paper fixes the structure of the method (Section 4.4.1):
+ *   - outliers are found with the three-sigma rule and channels are classified into outlier-rich
+ *     ("salient") and normal;
+ *   - normal channels are quantised;
+ *   - a salient channel feature map (h x w) is split, through a non-zero mask that is average-pooled
+ *     with an n x n window and compared with a threshold tau, into sparse blocks (stored in
+ *     Compressed Sparse Row form) and dense blocks (Lorenzo prediction, Eq. 7-8, residuals inside an
+ *     error bound eps are quantised, Eq. 9, unpredictable values are kept verbatim, predictions use
+ *     decompressed values);
+ *   - decompression rebuilds floating-point values from the codes and the prediction.
+ * It fixes none of the constants (bit-width, n, tau, eps, ...), the rounding, or a byte layout.
+ * Those are parameters here, and every such choice is listed next to the code that takes it.
+ *
+ * Parity unpinned: the parameter values themselves (bits, rho, block, tau, eps, code width), the
+ * per-plane scope of mu and sigma, the rounding mode and the container layout are choices the
+ * paper does not fix; tests pin the arithmetic given those choices, not the choices.
+ *
+ * Arithmetic rules: every float operation below is a single IEEE-754 operation with round to
+ * nearest even (compile with -ffp-contract=off, no -ffast-math); fmaf() and fma-free products are
+ * written out where the distinction matters.  No flush-to-zero.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define FHO_OK 0
+#define FHO_ERR_ARG (-1)
+#define FHO_ERR_UNSUPPORTED (-2)
+#define FHO_ERR_CAPACITY (-3)
+#define FHO_ERR_NONFINITE (-4)
+#define FHO_ERR_CORRUPT (-5)
+
+#define FHO_F32 0
+#define FHO_BF16 1
+
+#define CLS_NORMAL 0u
+#define CLS_SALIENT 1u
+#define CLS_RAW 2u
+
+#define MODE_AUTO 0
+#define MODE_OFF 1
+#define MODE_ALL 2
+
+typedef struct {
+  int32_t dtype;
+  int32_t n, c, h, w;
+  uint64_t tensor_id;
+} fho_desc;
+
+typedef struct {
+  int32_t bits;
+  int32_t salient_mode;
+  int32_t rho_num, rho_den;
+  int32_t block;
+  int32_t tau_num, tau_den;
+  float eps;
+  int32_t dense_bits;
+  int32_t rounding;
+  uint64_t seed;
+} fho_params;
+
+static int g_threads = 1;
+
+void fho_set_threads(int t) { g_threads = t < 1 ? 1 : t; }
+int fho_get_threads(void) { return g_threads; }
+int fho_max_threads(void) {
+#ifdef _OPENMP
+  return omp_get_num_procs();
+#else
+  return 1;
+#endif
+}
+
+static size_t a4(size_t x) { return (x + 3) & ~(size_t)3; }
+static size_t a16(size_t x) { return (x + 15) & ~(size_t)15; }
+static size_t esize(int dtype) { return dtype == FHO_F32 ? 4 : 2; }
+
+static float bf16_to_f32(uint16_t h) {
+  uint32_t u = (uint32_t)h << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return f;
+}
+
+/* fp32 -> bf16, round half to even (finite inputs). */
+static uint16_t f32_to_bf16(float f) {
+  uint32_t u;
+  memcpy(&u, &f, 4);
+  uint32_t r = ((u >> 16) & 1u) + 0x7FFFu;
+  return (uint16_t)((u + r) >> 16);
+}
+
+static int check_args(const fho_desc* d, const fho_params* p) {
+  if (!d || !p) return FHO_ERR_ARG;
+  if (d->dtype != FHO_F32 && d->dtype != FHO_BF16) return FHO_ERR_ARG;
+  if (d->n < 1 || d->c < 1 || d->h < 1 || d->w < 1) return FHO_ERR_ARG;
+  if (d->w > 65535) return FHO_ERR_UNSUPPORTED;
+  if (p->bits != 2 && p->bits != 4 && p->bits != 8) return FHO_ERR_UNSUPPORTED;
+  if (p->salient_mode < 0 || p->salient_mode > 2) return FHO_ERR_ARG;
+  if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FHO_ERR_ARG;
+  if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FHO_ERR_ARG;
+  if (p->block != 8) return FHO_ERR_UNSUPPORTED;
+  if (p->dense_bits != 8) return FHO_ERR_UNSUPPORTED;
+  if (p->rounding != 0) return FHO_ERR_UNSUPPORTED;
+  if (!(p->eps >= 1e-30f) || !(p->eps <= 1e30f)) return FHO_ERR_ARG; /* keeps 2*eps and 1/(2*eps) finite */
+  return FHO_OK;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Sizes.  Container (a layout choice; the paper gives none), little-endian:
+ *   [0,64) header | [64, 64+16P) plane table | payloads in plane order, each padded to 16 bytes.
+ * ------------------------------------------------------------------------------------------ */
+static size_t normal_payload(size_t hw, int bits) { return 4 * ((hw * (size_t)bits + 31) / 32); }
+
+size_t fho_compressed_bytes(const fho_desc* d, const fho_params* p, int which) {
+  if (check_args(d, p) != FHO_OK) return 0;
+  size_t P = (size_t)d->n * (size_t)d->c, hw = (size_t)d->h * (size_t)d->w;
+  if (which == 0) return 64 + P * (16 + a16(normal_payload(hw, p->bits)));
+  return 64 + P * (16 + a16(esize(d->dtype) * hw));
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Three-sigma statistics of one plane (Section 4.4.1: "Outliers are identified using the
+ * empirical 3-sigma rule").  mu and sigma are taken over the plane.  To make the result
+ * independent of summation order up to fp64 rounding, sums are formed from fp32 partials of
+ * 4 consecutive elements (tail padded with zeros) that are then added in fp64:
+ *   s_g = (x0+x1)+(x2+x3),  q_g = fma(x1,x1,x0*x0) + fma(x3,x3,x2*x2)        (fp32)
+ *   S = sum s_g, Q = sum q_g                                                  (fp64)
+ *   mu = S/HW, var = max(Q/HW - mu*mu, 0), sigma = sqrt(var)                   (fp64)
+ *   T_hi = (float)(mu + 3 sigma), T_lo = (float)(mu - 3 sigma)
+ *   n_out = #{ x > T_hi or x < T_lo }                                         (fp32 compares)
+ * ------------------------------------------------------------------------------------------ */
+void fho_plane_sigma(const float* x, int64_t hw, double* S_out, double* Q_out, float* t_lo,
+                     float* t_hi, int64_t* n_out) {
+  double S = 0.0, Q = 0.0;
+  for (int64_t g = 0; g < hw; g += 4) {
+    float v[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k = 0; k < 4 && g + k < hw; ++k) v[k] = x[g + k];
+    float s01 = v[0] + v[1], s23 = v[2] + v[3];
+    float sg = s01 + s23;
+    float p0 = v[0] * v[0], p2 = v[2] * v[2];
+    float q01 = fmaf(v[1], v[1], p0), q23 = fmaf(v[3], v[3], p2);
+    float qg = q01 + q23;
+    S += (double)sg;
+    Q += (double)qg;
+  }
+  double mu = S / (double)hw;
+  double ex2 = Q / (double)hw;
+  double mu2 = mu * mu;
+  double var = ex2 - mu2;
+  if (!(var > 0.0)) var = 0.0;
+  double sigma = sqrt(var);
+  double three = 3.0 * sigma;
+  float thi = (float)(mu + three);
+  float tlo = (float)(mu - three);
+  int64_t cnt = 0;
+  for (int64_t i = 0; i < hw; ++i)
+    if (x[i] > thi || x[i] < tlo) ++cnt;
+  *S_out = S;
+  *Q_out = Q;
+  *t_lo = tlo;
+  *t_hi = thi;
+  *n_out = cnt;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Normal planes "undergo quantization" (Section 4.4.1).  Uniform affine quantiser with one group
+ * per plane and the plane's min and max as statistics:
+ *   L = 2^b - 1, range = hi - lo, inv = L / range, scale = range / L          (fp32)
+ *   range == 0 or inv not finite  ->  inv = scale = 0
+ *   q = clamp(round_half_even((x - lo) * inv), 0, L)
+ * where (x - lo) is an fp32 subtraction and its product with inv is taken exactly before the
+ * rounding to an integer (the fp64 product of two fp32 numbers is exact).
+ * ------------------------------------------------------------------------------------------ */
+void fho_quant_params(float lo, float hi, int bits, float* inv, float* scale) {
+  float L = (float)((1 << bits) - 1);
+  float range = hi - lo;
+  float i = L / range, s = range / L;
+  if (range == 0.0f || !isfinite(i)) {
+    i = 0.0f;
+    s = 0.0f;
+  }
+  *inv = i;
+  *scale = s;
+}
+
+uint32_t fho_quant_code(float x, float lo, float inv, int bits) {
+  int L = (1 << bits) - 1;
+  float d = x - lo;
+  double t = (double)d * (double)inv; /* exact */
+  double r = nearbyint(t);            /* default rounding mode: half to even */
+  if (r < 0.0) r = 0.0;
+  if (r > (double)L) r = (double)L;
+  return (uint32_t)r;
+}
+
+float fho_dequant(uint32_t q, float lo, float scale) { return fmaf((float)q, scale, lo); }
+
+/* Pre-quantisation for dense blocks: k = round_half_even(fp32(x * inv2e)), |k| capped at 2^24. */
+static int32_t dense_k(float x, float inv2e, int* big) {
+  float kf = rintf(x * inv2e);
+  *big = fabsf(kf) >= 16777216.0f;
+  if (kf > 16777216.0f) kf = 16777216.0f;
+  if (kf < -16777216.0f) kf = -16777216.0f;
+  return (int32_t)kf;
+}
+
+static void put_u32(uint8_t* p, uint32_t v) { memcpy(p, &v, 4); }
+static void put_u16(uint8_t* p, uint16_t v) { memcpy(p, &v, 2); }
+static uint32_t get_u32(const uint8_t* p) {
+  uint32_t v;
+  memcpy(&v, p, 4);
+  return v;
+}
+static uint16_t get_u16(const uint8_t* p) {
+  uint16_t v;
+  memcpy(&v, p, 2);
+  return v;
+}
+
+typedef struct {
+  uint32_t cls;
+  uint32_t n_out;
+  float lo, scale;
+  uint8_t* payload; /* malloc'd, a16-padded, zero padded */
+  size_t bytes;     /* a16(payload size) */
+  int status;
+} plane_result;
+
+/* Salient plane (Section 4.4.1, block-wise path).  Returns payload size before a16 padding, or
+ * 0 when buf == NULL is used for sizing only.  Layout:
+ *   u32 nnz_s | u32 n_dense | u32 n_out_d | u32 0 | bitmap ceil(nblk/32) u32 (bit=1: dense)
+ *   | row_ptr (H+1) u32 | col nnz_s u16 (pad 4) | val nnz_s elems (pad 4)
+ *   | codes n_dense*64 bytes | outliers n_out_d elems (pad 4)
+ */
+static size_t encode_salient(const float* x, const uint8_t* raw, int dtype, int H, int W,
+                             const fho_params* p, uint8_t** out_buf) {
+  const int B = 8;
+  size_t e = esize(dtype);
+  int nby = (H + B - 1) / B, nbx = (W + B - 1) / B, nblk = nby * nbx;
+  /* mask -> pooled non-zero count per block -> block class.
+   * The paper average-pools the 0/1 mask with an n x n window and compares with tau; the mean of
+   * the mask over a window is nnz/n^2 (divisor n^2 also at ragged edges: zero padding), so the
+   * comparison is nnz/n^2 >= tau, done in integers as nnz * tau_den >= tau_num * n^2. */
+  uint8_t* dense = (uint8_t*)calloc((size_t)nblk, 1);
+  uint32_t n_dense = 0;
+  for (int by = 0; by < nby; ++by)
+    for (int bx = 0; bx < nbx; ++bx) {
+      int nnz = 0;
+      for (int i = 0; i < B; ++i)
+        for (int j = 0; j < B; ++j) {
+          int y = by * B + i, xx = bx * B + j;
+          if (y < H && xx < W && x[(size_t)y * W + xx] != 0.0f) ++nnz;
+        }
+      int is_dense = (int64_t)nnz * p->tau_den >= (int64_t)p->tau_num * (B * B);
+      dense[by * nbx + bx] = (uint8_t)is_dense;
+      n_dense += (uint32_t)is_dense;
+    }
+  /* CSR over non-zeros that lie in sparse blocks. */
+  uint32_t* row_ptr = (uint32_t*)calloc((size_t)H + 1, 4);
+  uint32_t nnz_s = 0;
+  for (int y = 0; y < H; ++y) {
+    row_ptr[y] = nnz_s;
+    for (int xx = 0; xx < W; ++xx)
+      if (x[(size_t)y * W + xx] != 0.0f && !dense[(y / B) * nbx + xx / B]) ++nnz_s;
+  }
+  row_ptr[H] = nnz_s;
+  /* Dense blocks: Lorenzo residuals on pre-quantised integers (Eq. 7-9).
+   * First-order 2-D Lorenzo predictor: pred = up + left - upleft (coefficients sum to one);
+   * neighbours outside the block count as 0.  Because prediction runs on the integers k, the
+   * values the predictor sees are exactly the decoder's reconstruction 2*eps*k. */
+  float two_eps = 2.0f * p->eps;
+  float inv2e = 1.0f / two_eps;
+  uint8_t* codes = (uint8_t*)malloc((size_t)n_dense * 64 + 1);
+  uint8_t* outl = (uint8_t*)malloc((size_t)n_dense * 64 * e + 1);
+  uint32_t n_out_d = 0, di = 0;
+  for (int blk = 0; blk < nblk; ++blk) {
+    if (!dense[blk]) continue;
+    int by = blk / nbx, bx = blk % nbx;
+    int32_t k[8][8];
+    int big[8][8], inpl[8][8];
+    for (int i = 0; i < B; ++i)
+      for (int j = 0; j < B; ++j) {
+        int y = by * B + i, xx = bx * B + j;
+        inpl[i][j] = (y < H && xx < W);
+        float v = inpl[i][j] ? x[(size_t)y * W + xx] : 0.0f;
+        k[i][j] = dense_k(v, inv2e, &big[i][j]);
+      }
+    for (int i = 0; i < B; ++i)
+      for (int j = 0; j < B; ++j) {
+        uint8_t code;
+        if (!inpl[i][j]) {
+          code = 128;
+        } else {
+          int64_t up = i > 0 ? k[i - 1][j] : 0;
+          int64_t left = j > 0 ? k[i][j - 1] : 0;
+          int64_t ul = (i > 0 && j > 0) ? k[i - 1][j - 1] : 0;
+          int64_t delta = (int64_t)k[i][j] - (up + left - ul);
+          if (big[i][j] || delta > 127 || delta < -127) {
+            code = 0;
+            size_t idx = (size_t)(by * B + i) * W + (size_t)(bx * B + j);
+            memcpy(outl + (size_t)n_out_d * e, raw + idx * e, e);
+            ++n_out_d;
+          } else {
+            code = (uint8_t)(delta + 128);
+          }
+        }
+        codes[(size_t)di * 64 + i * 8 + j] = code;
+      }
+    ++di;
+  }
+  size_t nbm = ((size_t)nblk + 31) / 32;
+  size_t size = 16 + 4 * nbm + 4 * ((size_t)H + 1) + a4(2 * (size_t)nnz_s) + a4(e * nnz_s) +
+                64 * (size_t)n_dense + a4(e * n_out_d);
+  uint8_t* buf = (uint8_t*)calloc(a16(size), 1);
+  uint8_t* q = buf;
+  put_u32(q, nnz_s);
+  put_u32(q + 4, n_dense);
+  put_u32(q + 8, n_out_d);
+  put_u32(q + 12, 0);
+  q += 16;
+  for (int blk = 0; blk < nblk; ++blk)
+    if (dense[blk]) {
+      uint32_t wv = get_u32(q + 4 * (blk / 32));
+      put_u32(q + 4 * (blk / 32), wv | (1u << (blk % 32)));
+    }
+  q += 4 * nbm;
+  for (int y = 0; y <= H; ++y) put_u32(q + 4 * y, row_ptr[y]);
+  q += 4 * ((size_t)H + 1);
+  uint8_t* colp = q;
+  uint8_t* valp = q + a4(2 * (size_t)nnz_s);
+  uint32_t t = 0;
+  for (int y = 0; y < H; ++y)
+    for (int xx = 0; xx < W; ++xx)
+      if (x[(size_t)y * W + xx] != 0.0f && !dense[(y / B) * nbx + xx / B]) {
+        put_u16(colp + 2 * (size_t)t, (uint16_t)xx);
+        memcpy(valp + e * t, raw + ((size_t)y * W + xx) * e, e);
+        ++t;
+      }
+  q = valp + a4(e * nnz_s);
+  memcpy(q, codes, (size_t)n_dense * 64);
+  q += (size_t)n_dense * 64;
+  memcpy(q, outl, (size_t)n_out_d * e);
+  free(dense);
+  free(row_ptr);
+  free(codes);
+  free(outl);
+  *out_buf = buf;
+  return size;
+}
+
+static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_params* p,
+                         plane_result* r) {
+  size_t hw = (size_t)H * W, e = esize(dtype);
+  float* x = (float*)malloc(hw * sizeof(float));
+  for (size_t i = 0; i < hw; ++i)
+    x[i] = dtype == FHO_F32 ? ((const float*)raw)[i] : bf16_to_f32(((const uint16_t*)raw)[i]);
+  memset(r, 0, sizeof(*r));
+  float lo = x[0], hi = x[0];
+  int finite = 1;
+  for (size_t i = 0; i < hw; ++i) {
+    if (!isfinite(x[i])) finite = 0;
+    if (x[i] < lo) lo = x[i];
+    if (x[i] > hi) hi = x[i];
+  }
+  if (!finite || !isfinite(hi - lo)) {
+    r->status = FHO_ERR_NONFINITE;
+    free(x);
+    return;
+  }
+  uint32_t cls = CLS_NORMAL, n_out = 0;
+  if (p->salient_mode == MODE_AUTO) {
+    double S, Q;
+    float tlo, thi;
+    int64_t cnt;
+    fho_plane_sigma(x, (int64_t)hw, &S, &Q, &tlo, &thi, &cnt);
+    n_out = (uint32_t)cnt;
+    /* outlier-rich when the three-sigma outliers exceed the fraction rho of the plane */
+    if ((int64_t)cnt * p->rho_den > (int64_t)p->rho_num * (int64_t)hw) cls = CLS_SALIENT;
+  } else if (p->salient_mode == MODE_ALL) {
+    cls = CLS_SALIENT;
+  }
+  if (cls == CLS_SALIENT) {
+    uint8_t* buf = NULL;
+    size_t size = encode_salient(x, raw, dtype, H, W, p, &buf);
+    if (a16(size) >= a16(e * hw)) { /* no gain: keep the plane verbatim */
+      free(buf);
+      cls = CLS_RAW;
+      r->bytes = a16(e * hw);
+      r->payload = (uint8_t*)calloc(r->bytes, 1);
+      memcpy(r->payload, raw, e * hw);
+    } else {
+      r->payload = buf;
+      r->bytes = a16(size);
+    }
+  } else {
+    float inv, scale;
+    fho_quant_params(lo, hi, p->bits, &inv, &scale);
+    size_t size = normal_payload(hw, p->bits);
+    r->bytes = a16(size);
+    r->payload = (uint8_t*)calloc(r->bytes, 1);
+    for (size_t i = 0; i < hw; ++i) {
+      uint32_t qv = fho_quant_code(x[i], lo, inv, p->bits);
+      size_t bit = i * (size_t)p->bits;
+      uint32_t wv = get_u32(r->payload + 4 * (bit / 32));
+      put_u32(r->payload + 4 * (bit / 32), wv | (qv << (bit % 32)));
+    }
+    r->lo = lo;
+    r->scale = scale;
+  }
+  r->cls = cls;
+  r->n_out = n_out;
+  free(x);
+}
+
+/* Compress a whole tensor.  out2[0] = total bytes needed, out2[1] = status (as uint64 of the
+ * negative code, 0 when OK).  Returns the status. */
+int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* dst,
+                 size_t dst_capacity, uint64_t* out2) {
+  int st = check_args(d, p);
+  if (st != FHO_OK) return st;
+  if (!src || !dst) return FHO_ERR_ARG;
+  size_t P = (size_t)d->n * d->c, hw = (size_t)d->h * d->w, e = esize(d->dtype);
+  plane_result* res = (plane_result*)calloc(P, sizeof(plane_result));
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)
+#endif
+  for (int64_t pl = 0; pl < (int64_t)P; ++pl)
+    encode_plane((const uint8_t*)src + (size_t)pl * hw * e, d->dtype, d->h, d->w, p, &res[pl]);
+  size_t total = 64 + 16 * P;
+  uint32_t n_sal = 0, n_raw = 0;
+  for (size_t pl = 0; pl < P; ++pl) {
+    if (res[pl].status != FHO_OK) st = res[pl].status;
+    total += res[pl].bytes;
+    n_sal += res[pl].cls == CLS_SALIENT;
+    n_raw += res[pl].cls == CLS_RAW;
+  }
+  if (st == FHO_OK && total > dst_capacity) st = FHO_ERR_CAPACITY;
+  if (st == FHO_OK && total / 16 > 0xFFFFFFFFull) st = FHO_ERR_UNSUPPORTED;
+  if (st == FHO_OK) {
+    uint8_t* o = (uint8_t*)dst;
+    memset(o, 0, 64);
+    put_u32(o + 0, 0x31434846u); /* 'F','H','C','1' */
+    put_u16(o + 4, 1);
+    o[6] = (uint8_t)d->dtype;
+    o[7] = (uint8_t)p->bits;
+    put_u32(o + 8, (uint32_t)d->n);
+    put_u32(o + 12, (uint32_t)d->c);
+    put_u32(o + 16, (uint32_t)d->h);
+    put_u32(o + 20, (uint32_t)d->w);
+    o[24] = (uint8_t)p->block;
+    o[25] = (uint8_t)p->dense_bits;
+    o[26] = (uint8_t)p->rounding;
+    o[27] = (uint8_t)p->salient_mode;
+    put_u16(o + 28, (uint16_t)p->rho_num);
+    put_u16(o + 30, (uint16_t)p->rho_den);
+    put_u16(o + 32, (uint16_t)p->tau_num);
+    put_u16(o + 34, (uint16_t)p->tau_den);
+    memcpy(o + 36, &p->eps, 4);
+    put_u32(o + 40, n_sal);
+    put_u32(o + 44, n_raw);
+    memcpy(o + 48, &d->tensor_id, 8);
+    uint64_t tb = total;
+    memcpy(o + 56, &tb, 8);
+    size_t off = 64 + 16 * P;
+    for (size_t pl = 0; pl < P; ++pl) {
+      uint8_t* te = o + 64 + 16 * pl;
+      put_u32(te, (uint32_t)(off / 16));
+      put_u32(te + 4, res[pl].cls | (res[pl].n_out << 2));
+      memcpy(te + 8, &res[pl].lo, 4);
+      memcpy(te + 12, &res[pl].scale, 4);
+      memcpy(o + off, res[pl].payload, res[pl].bytes);
+      off += res[pl].bytes;
+    }
+  }
+  for (size_t pl = 0; pl < P; ++pl) free(res[pl].payload);
+  free(res);
+  if (out2) {
+    out2[0] = total;
+    out2[1] = (uint64_t)(int64_t)st;
+  }
+  return st;
+}
+
+static void store_elem(uint8_t* dst, int dtype, size_t i, float v) {
+  if (dtype == FHO_F32)
+    memcpy(dst + 4 * i, &v, 4);
+  else {
+    uint16_t h = f32_to_bf16(v);
+    memcpy(dst + 2 * i, &h, 2);
+  }
+}
+
+static int decode_plane(const uint8_t* src, size_t src_bytes, size_t pl, size_t P, int dtype, int H,
+                        int W, int bits, float eps, uint8_t* out) {
+  size_t hw = (size_t)H * W, e = esize(dtype);
+  const uint8_t* te = src + 64 + 16 * pl;
+  size_t off = (size_t)get_u32(te) * 16;
+  uint32_t meta = get_u32(te + 4);
+  uint32_t cls = meta & 3u;
+  float lo, scale;
+  memcpy(&lo, te + 8, 4);
+  memcpy(&scale, te + 12, 4);
+  if (off < 64 + 16 * P || off > src_bytes) return FHO_ERR_CORRUPT;
+  const uint8_t* pay = src + off;
+  size_t avail = src_bytes - off;
+  if (cls == CLS_NORMAL) {
+    if (normal_payload(hw, bits) > avail) return FHO_ERR_CORRUPT;
+    uint32_t mask = (1u << bits) - 1u;
+    for (size_t i = 0; i < hw; ++i) {
+      size_t bit = i * (size_t)bits;
+      uint32_t q = (get_u32(pay + 4 * (bit / 32)) >> (bit % 32)) & mask;
+      store_elem(out, dtype, i, fho_dequant(q, lo, scale));
+    }
+    return FHO_OK;
+  }
+  if (cls == CLS_RAW) {
+    if (e * hw > avail) return FHO_ERR_CORRUPT;
+    memcpy(out, pay, e * hw);
+    return FHO_OK;
+  }
+  if (cls != CLS_SALIENT) return FHO_ERR_CORRUPT;
+  const int B = 8;
+  int nby = (H + B - 1) / B, nbx = (W + B - 1) / B, nblk = nby * nbx;
+  size_t nbm = ((size_t)nblk + 31) / 32;
+  if (16 > avail) return FHO_ERR_CORRUPT;
+  uint32_t nnz_s = get_u32(pay), n_dense = get_u32(pay + 4), n_out_d = get_u32(pay + 8);
+  size_t size = 16 + 4 * nbm + 4 * ((size_t)H + 1) + a4(2 * (size_t)nnz_s) + a4(e * nnz_s) +
+                64 * (size_t)n_dense + a4(e * n_out_d);
+  if (size > avail) return FHO_ERR_CORRUPT;
+  const uint8_t* bm = pay + 16;
+  const uint8_t* rp = bm + 4 * nbm;
+  const uint8_t* colp = rp + 4 * ((size_t)H + 1);
+  const uint8_t* valp = colp + a4(2 * (size_t)nnz_s);
+  const uint8_t* codes = valp + a4(e * nnz_s);
+  const uint8_t* outl = codes + 64 * (size_t)n_dense;
+  memset(out, 0, e * hw);
+  for (int y = 0; y < H; ++y) {
+    uint32_t a = get_u32(rp + 4 * y), b = get_u32(rp + 4 * (y + 1));
+    if (a > b || b > nnz_s) return FHO_ERR_CORRUPT;
+    for (uint32_t t = a; t < b; ++t) {
+      uint32_t col = get_u16(colp + 2 * (size_t)t);
+      if ((int)col >= W) return FHO_ERR_CORRUPT;
+      memcpy(out + ((size_t)y * W + col) * e, valp + e * t, e);
+    }
+  }
+  float two_eps = 2.0f * eps;
+  float inv2e = 1.0f / two_eps;
+  uint32_t di = 0, oi = 0;
+  for (int blk = 0; blk < nblk; ++blk) {
+    if (!((get_u32(bm + 4 * (blk / 32)) >> (blk % 32)) & 1u)) continue;
+    if (di >= n_dense) return FHO_ERR_CORRUPT;
+    int by = blk / nbx, bx = blk % nbx;
+    int64_t k[8][8];
+    for (int i = 0; i < B; ++i)
+      for (int j = 0; j < B; ++j) {
+        int y = by * B + i, xx = bx * B + j;
+        int64_t up = i > 0 ? k[i - 1][j] : 0;
+        int64_t left = j > 0 ? k[i][j - 1] : 0;
+        int64_t ul = (i > 0 && j > 0) ? k[i - 1][j - 1] : 0;
+        int64_t pred = up + left - ul;
+        uint8_t code = codes[(size_t)di * 64 + i * 8 + j];
+        if (!(y < H && xx < W)) {
+          k[i][j] = pred; /* padding: never read by an in-plane element */
+          continue;
+        }
+        size_t idx = (size_t)y * W + xx;
+        if (code == 0) {
+          if (oi >= n_out_d) return FHO_ERR_CORRUPT;
+          memcpy(out + idx * e, outl + (size_t)oi * e, e);
+          float v;
+          if (dtype == FHO_F32)
+            memcpy(&v, outl + (size_t)oi * e, 4);
+          else
+            v = bf16_to_f32(get_u16(outl + (size_t)oi * e));
+          int big;
+          k[i][j] = dense_k(v, inv2e, &big);
+          ++oi;
+        } else {
+          k[i][j] = pred + ((int64_t)code - 128);
+          float kv = (float)k[i][j];
+          store_elem(out, dtype, idx, kv * two_eps);
+        }
+      }
+    ++di;
+  }
+  return FHO_OK;
+}
+
+int fho_decompress(const void* src, size_t src_bytes, const fho_desc* expect, void* dst) {
+  if (!src || !dst || !expect) return FHO_ERR_ARG;
+  const uint8_t* s = (const uint8_t*)src;
+  if (src_bytes < 64) return FHO_ERR_CORRUPT;
+  if (get_u32(s) != 0x31434846u || get_u16(s + 4) != 1) return FHO_ERR_CORRUPT;
+  int dtype = s[6], bits = s[7];
+  uint32_t N = get_u32(s + 8), C = get_u32(s + 12), H = get_u32(s + 16), W = get_u32(s + 20);
+  if ((int)N != expect->n || (int)C != expect->c || (int)H != expect->h || (int)W != expect->w ||
+      dtype != expect->dtype)
+    return FHO_ERR_CORRUPT;
+  if (bits != 2 && bits != 4 && bits != 8) return FHO_ERR_CORRUPT;
+  if (s[24] != 8 || s[25] != 8) return FHO_ERR_CORRUPT;
+  float eps;
+  memcpy(&eps, s + 36, 4);
+  uint64_t tb;
+  memcpy(&tb, s + 56, 8);
+  size_t P = (size_t)N * C, hw = (size_t)H * W, e = esize(dtype);
+  if (tb > src_bytes || tb < 64 + 16 * P) return FHO_ERR_CORRUPT;
+  int st = FHO_OK;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)
+#endif
+  for (int64_t pl = 0; pl < (int64_t)P; ++pl) {
+    int r = decode_plane(s, (size_t)tb, (size_t)pl, P, dtype, (int)H, (int)W, bits, eps,
+                         (uint8_t*)dst + (size_t)pl * hw * e);
+    if (r != FHO_OK) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+      st = r;
+    }
+  }
+  return st;
+}
