@@ -1,0 +1,197 @@
+/*
+ * fh.h -- C ABI of the B200 activation codec (Channel-wise Mix Compression, FedHybrid,
+ * arXiv 2510.11400, Section 4.4.1).
+ *
+ * Local training compresses the activations its execution plan marks "compress" in the forward
+ * pass and restores them when the backward pass needs them (Section 3.2; Algorithm 1, functions
+ * Compute and Alloc).  This library is that step for one GPU: a dense, contiguous NCHW tensor
+ * goes in, a self-describing packed container comes out, and back.
+ *
+ * Every plane (one (n, c) feature map of h x w elements) is coded independently:
+ *   - three-sigma statistics classify it as normal or outlier-rich (Section 4.4.1);
+ *   - a normal plane is quantised to `bits` bits per element between its own minimum and maximum;
+ *   - an outlier-rich plane is split into 8 x 8 blocks by its pooled non-zero mask; sparse blocks go
+ *     to one CSR structure, dense blocks to 8-bit first-order Lorenzo residual codes within the
+ *     absolute error bound eps, unpredictable values verbatim (Eq. 7-9);
+ *   - a plane that would not shrink is stored verbatim.
+ *
+ * Conventions
+ *   - All functions return FH_OK (0) or a negative fh_status.  Errors that the host can see
+ *     (bad arguments, unsupported shapes) are returned at once and nothing is enqueued.  Errors only
+ *     the device can see (non-finite input, capacity, corrupt container, a wait that gave up) are
+ *     written to the status word the call names.
+ *   - Pointers named d_* are device pointers, h_* host pointers.  The caller owns every buffer.
+ *     Dense and packed device buffers must be 16-byte aligned.
+ *   - fh_compress and fh_decompress only enqueue work on `stream` (a cudaStream_t passed as
+ *     void*; NULL is the legacy default stream) and never synchronise.  Per stream the library keeps
+ *     one small scratch allocation (scan flags) that it creates on first use and frees in
+ *     fh_shutdown(); growing it for a larger tensor synchronises the device once.
+ *   - There is no CPU fallback: without a CUDA device every entry point that does work returns
+ *     FH_ERR_CUDA.
+ *
+ * Container (little-endian; a layout of this library, the paper gives none)
+ *   [0,64)   header: u32 magic "FHC1" | u16 version=1 | u8 dtype | u8 bits | u32 N | u32 C | u32 H |
+ *            u32 W | u8 block | u8 dense_bits | u8 rounding | u8 salient_mode | u16 rho_num |
+ *            u16 rho_den | u16 tau_num | u16 tau_den | f32 eps | u32 n_salient | u32 n_raw |
+ *            u64 tensor_id | u64 total_bytes
+ *   [64,64+16P)  plane table, P = N*C entries: u32 payload offset / 16 | u32 meta (bits 0-1 class:
+ *            0 normal, 1 salient, 2 raw; bits 2-31 three-sigma outlier count) | f32 lo | f32 scale
+ *   payloads in plane order, each zero-padded to a multiple of 16 bytes
+ *     normal : ceil(HW*bits/32) u32 words, element i in bits [(i*bits)%32, +bits) of word i*bits/32
+ *     raw    : HW elements verbatim
+ *     salient: u32 nnz_s | u32 n_dense | u32 n_out_d | u32 0 | block bitmap ceil(nblk/32) u32
+ *              (bit = 1: dense; blocks in raster order) | row_ptr (H+1) u32 | col nnz_s u16 (pad 4) |
+ *              val nnz_s elements (pad 4) | codes n_dense*64 u8 | verbatim values n_out_d elements
+ *              (pad 4)
+ */
+#ifndef FH_H_
+#define FH_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FH_OK = 0,
+  FH_ERR_ARG = -1,         /* null pointer, non-positive extent, misaligned buffer, bad enum        */
+  FH_ERR_UNSUPPORTED = -2, /* valid but outside what the kernels handle (see fh_compress)          */
+  FH_ERR_CAPACITY = -3,    /* packed output does not fit dst_capacity / the arena                  */
+  FH_ERR_NONFINITE = -4,   /* NaN or Inf in the input, or max - min overflows                      */
+  FH_ERR_CORRUPT = -5,     /* container header/table/payload inconsistent with the expectation    */
+  FH_ERR_TIMEOUT = -6,     /* a bounded device-side wait ran out (should never happen)             */
+  FH_ERR_CUDA = -7         /* CUDA runtime error or no device                                       */
+} fh_status;
+
+typedef enum { FH_F32 = 0, FH_BF16 = 1 } fh_dtype;
+
+/* A dense activation: contiguous NCHW, P = n*c planes of h*w elements; w <= 65535. */
+typedef struct {
+  int32_t dtype; /* fh_dtype */
+  int32_t n, c, h, w;
+  uint64_t tensor_id; /* carried in the header; also keys any random rounding */
+} fh_tensor_desc;
+
+typedef enum { FH_SALIENT_AUTO = 0, FH_SALIENT_OFF = 1, FH_SALIENT_ALL = 2 } fh_salient_mode;
+
+/* Codec parameters.  The paper names these quantities but prints no values (Section 4.4.1);
+ * fh_default_params() fills the defaults given beside each field. */
+typedef struct {
+  int32_t bits;             /* code width of normal planes: 2, 4 or 8                      [2]     */
+  int32_t salient_mode;     /* AUTO: three-sigma rule; OFF: every plane normal; ALL: every
+                               plane takes the block-wise path                            [AUTO]  */
+  int32_t rho_num, rho_den; /* plane is outlier-rich iff n_out*rho_den > rho_num*HW        [1/32]  */
+  int32_t block;            /* n: pooling window = block edge; 8 only                      [8]     */
+  int32_t tau_num, tau_den; /* block is dense iff nnz*tau_den >= tau_num*n*n               [1/4]   */
+  float eps;                /* absolute error bound of dense blocks, 1e-30 <= eps <= 1e30  [1/16]  */
+  int32_t dense_bits;       /* residual code width; 8 only                                 [8]     */
+  int32_t rounding;         /* 0 = round half to even; nothing else yet                    [0]     */
+  uint64_t seed;            /* reserved for random rounding                                [0]     */
+} fh_params;
+
+typedef enum { FH_KEEP = 0, FH_COMPRESS = 1, FH_EVICT = 2 } fh_action;
+
+/* One saved activation of a training step, in forward order (Algorithm 1's tensor states). */
+typedef struct {
+  fh_tensor_desc desc;
+  int32_t action;      /* fh_action; KEEP and EVICT entries are skipped by the codec               */
+  const void* d_dense; /* dense input (device)                                                    */
+  void* d_restored;    /* where the backward pass wants it back (device); may equal d_dense       */
+} fh_sched_entry;
+
+typedef struct {
+  uint64_t total_dense_bytes;  /* dense bytes of the COMPRESS entries                              */
+  uint64_t total_packed_bytes; /* sum of their container sizes                                     */
+  uint64_t peak_packed_bytes;  /* arena high-water mark (containers start on 256-byte boundaries)  */
+  float ms_forward, ms_backward;
+  int32_t status; /* first device-side error, FH_OK otherwise */
+} fh_sched_report;
+
+void fh_default_params(fh_params* p);
+
+/* Version of the library (1) -- also proves that the shared object loaded. */
+int fh_version(void);
+
+/* Number of CUDA devices visible, or a negative fh_status. */
+int fh_device_count(void);
+
+/*
+ * Size of the container of a tensor (Section 4.4.1 leaves the layout open; sizes follow the
+ * container described above).
+ *   which = 0: exact size when every plane is normal (always exact for FH_SALIENT_OFF):
+ *              64 + P*(16 + A16(4*ceil(HW*bits/32)))
+ *   which = 1: worst case, every plane verbatim: 64 + P*(16 + A16(esize*HW)); a dst_capacity of
+ *              this many bytes can never overflow.
+ * Returns 0 for invalid arguments.  Host-only, no CUDA call.
+ */
+size_t fh_compressed_bytes(const fh_tensor_desc* desc, const fh_params* params, int which);
+
+/*
+ * Compress one tensor (Section 4.4.1; forward pass of a tensor the plan marks "compress").
+ *   d_src        dense input, n*c*h*w elements of desc->dtype, device, 16-byte aligned
+ *   d_dst        container output, device, 16-byte aligned, dst_capacity bytes; never written past
+ *                dst_capacity.  Must hold at least the header and plane table (64 + 16*P bytes).
+ *   d_out2       optional, two uint64 in device memory (or pinned host memory mapped to the device):
+ *                [0] total container bytes (the size needed, also when it did not fit),
+ *                [1] (uint64)(int64) status: FH_OK, FH_ERR_NONFINITE, FH_ERR_CAPACITY, FH_ERR_TIMEOUT.
+ *                Written by the kernel; valid once `stream` has reached this point.
+ * Limits: one plane plus its working set must fit the shared memory of an SM, i.e. roughly
+ * h*w*esize <= 200 KB; larger planes return FH_ERR_UNSUPPORTED.  The container is limited to
+ * 64 GiB (32-bit offsets in units of 16 bytes).
+ * The packed bytes are a pure function of the input and the parameters.
+ */
+int fh_compress(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
+                size_t dst_capacity, uint64_t* d_out2, void* stream);
+
+/*
+ * Restore a tensor from its container (Section 4.4.1, "Decompression ..."; Algorithm 1, the
+ * COMPRESSED branch of Compute).
+ *   d_src, src_bytes   the container and the number of readable bytes
+ *   expect             shape and dtype the caller expects; a mismatch with the header is
+ *                      FH_ERR_CORRUPT (reported through d_status, the header lives on the device)
+ *   d_dst              dense output, device, 16-byte aligned
+ *   d_status           optional uint64 in device (or mapped pinned) memory: (uint64)(int64) status
+ * Never reads past src_bytes.  Planes whose table entry is corrupt are left unwritten.
+ */
+int fh_decompress(const void* d_src, size_t src_bytes, const fh_tensor_desc* expect, void* d_dst,
+                  uint64_t* d_status, void* stream);
+
+/*
+ * One training step's worth of codec work on one stream (Section 3.2; Algorithm 1): entries with
+ * action FH_COMPRESS are compressed in forward order into d_arena (bump allocation with a
+ * device-side cursor, 256-byte aligned containers, because sizes are only known on the device), then
+ * restored in reverse order into their d_restored buffers.  Forward and backward phases are timed
+ * with CUDA events.  This call synchronises the stream before it returns and fills *report.
+ * An arena too small gives report->status = FH_ERR_CAPACITY (later tensors are skipped, nothing is
+ * written outside the arena).
+ */
+int fh_run_schedule(const fh_sched_entry* entries, int32_t count, const fh_params* params,
+                    void* d_arena, size_t arena_bytes, fh_sched_report* report, void* stream);
+
+/*
+ * Host-buffer variants: the same codec with host memory on both sides.  The library copies
+ * h_src to the device work buffer, runs the kernels, copies the result back and synchronises.
+ *   d_work, work_bytes   caller-owned device workspace, 256-byte aligned, at least
+ *                        fh_host_work_bytes(desc, params) bytes
+ *   h_out2 / h_status    as d_out2 / d_status above, but plain host memory
+ * Pinned host buffers give asynchronous copies; pageable ones work but are slower.
+ */
+size_t fh_host_work_bytes(const fh_tensor_desc* desc, const fh_params* params);
+int fh_compress_host(const fh_tensor_desc* desc, const fh_params* params, const void* h_src,
+                     void* h_dst, size_t dst_capacity, uint64_t* h_out2, void* d_work,
+                     size_t work_bytes, void* stream);
+int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc* expect, void* h_dst,
+                       uint64_t* h_status, void* d_work, size_t work_bytes, void* stream);
+
+/* Number of kernels this library has launched since it was loaded (for launch accounting). */
+uint64_t fh_kernel_launches(void);
+
+/* Free every scratch allocation the library holds on every device.  Synchronises. */
+void fh_shutdown(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FH_H_ */

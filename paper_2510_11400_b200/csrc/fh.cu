@@ -1,0 +1,543 @@
+// Host side of the C ABI declared in include/fh.h: argument checks, size formulas, tiling plans,
+// per-stream scratch, kernel launches, the schedule runner and the host-buffer variants.
+#include "../../include/fh.h"
+
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <utility>
+#include <vector>
+
+#include "fh_compress.cuh"
+#include "fh_decompress.cuh"
+
+namespace {
+
+using fh::Plan;
+
+constexpr size_t kSmemLimit = 227 * 1024 - 1024;  // dynamic shared memory a CTA may ask for
+constexpr size_t kTileTarget = 32 * 1024;         // dense bytes a tile aims for
+constexpr uint32_t kMaxPpt = 2048;
+constexpr uint32_t kSpinLimit = 1u << 20;
+
+std::atomic<uint64_t> g_launches{0};
+
+inline size_t A16(size_t x) { return (x + 15) & ~(size_t)15; }
+inline size_t A256(size_t x) { return (x + 255) & ~(size_t)255; }
+inline size_t esize_of(int dtype) { return dtype == FH_F32 ? 4 : 2; }
+
+int check_desc(const fh_tensor_desc* d) {
+  if (!d) return FH_ERR_ARG;
+  if (d->dtype != FH_F32 && d->dtype != FH_BF16) return FH_ERR_ARG;
+  if (d->n < 1 || d->c < 1 || d->h < 1 || d->w < 1) return FH_ERR_ARG;
+  if (d->w > 65535) return FH_ERR_UNSUPPORTED;
+  return FH_OK;
+}
+
+int check_params(const fh_params* p) {
+  if (!p) return FH_ERR_ARG;
+  if (p->bits != 2 && p->bits != 4 && p->bits != 8) return FH_ERR_UNSUPPORTED;
+  if (p->salient_mode < 0 || p->salient_mode > 2) return FH_ERR_ARG;
+  if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FH_ERR_ARG;
+  if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FH_ERR_ARG;
+  if (p->block != 8 || p->dense_bits != 8 || p->rounding != 0) return FH_ERR_UNSUPPORTED;
+  if (!(p->eps >= 1e-30f) || !(p->eps <= 1e30f)) return FH_ERR_ARG;
+  return FH_OK;
+}
+
+uint32_t pow2_floor(uint32_t x) {
+  uint32_t r = 1;
+  while (r * 2 <= x) r *= 2;
+  return r;
+}
+
+// Tiling and shared-memory layout.  `compress` selects the compress kernel's layout (staged tile,
+// code staging, per-plane records, block-wise scratch); the decompress kernel only needs the
+// block-wise scratch.
+int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* out) {
+  Plan pl;
+  std::memset(&pl, 0, sizeof(pl));
+  pl.dtype = d->dtype;
+  pl.esize = (int)esize_of(d->dtype);
+  pl.H = d->h;
+  pl.W = d->w;
+  pl.N = (uint32_t)d->n;
+  pl.C = (uint32_t)d->c;
+  const uint64_t hw = (uint64_t)d->h * (uint64_t)d->w;
+  if (hw * pl.esize > kSmemLimit) return FH_ERR_UNSUPPORTED;
+  pl.HW = (uint32_t)hw;
+  pl.groups = (pl.HW + 3) / 4;
+  pl.P = (uint64_t)d->n * (uint64_t)d->c;
+  pl.plane_bytes = hw * pl.esize;
+  pl.dense_bytes = pl.P * pl.plane_bytes;
+  pl.bits = p ? p->bits : 2;
+  pl.mode = p ? p->salient_mode : 0;
+  pl.rho_num = p ? p->rho_num : 1;
+  pl.rho_den = p ? p->rho_den : 32;
+  pl.tau_num = p ? p->tau_num : 1;
+  pl.tau_den = p ? p->tau_den : 4;
+  pl.eps = p ? p->eps : 0.0625f;
+  pl.tensor_id = d->tensor_id;
+  pl.npay = (uint32_t)A16(4 * (((uint64_t)pl.HW * pl.bits + 31) / 32));
+  pl.nbx = (uint32_t)(d->w + 7) / 8;
+  pl.nby = (uint32_t)(d->h + 7) / 8;
+  pl.nblk = pl.nbx * pl.nby;
+  pl.nbm = (pl.nblk + 31) / 32;
+  // container offsets are 32-bit counts of 16 bytes
+  const long double worst = 64.0L + (long double)pl.P * (16.0L + (long double)A16(pl.plane_bytes));
+  if (worst / 16.0L >= 4294967295.0L) return FH_ERR_UNSUPPORTED;
+  if (pl.P > 0x7FFFFFFFull) return FH_ERR_UNSUPPORTED;
+
+  if (pl.plane_bytes <= 8192) {
+    uint32_t t = pow2_floor(pl.HW / 8 > 0 ? pl.HW / 8 : 1);
+    pl.team = t > 32 ? 32 : t;
+  } else {
+    pl.team = fh::kThreads;
+  }
+  const uint32_t nteams = pl.team > 32 ? 1 : fh::kThreads / pl.team;
+  const bool need_sal = compress ? (pl.mode != FH_SALIENT_OFF) : true;
+  pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * ((size_t)(compress ? (pl.H + 1 + 3 * pl.nblk) : pl.nblk))) : 0;
+
+  uint64_t ppt = kTileTarget / pl.plane_bytes;
+  if (ppt < 1) ppt = 1;
+  if (ppt > kMaxPpt) ppt = kMaxPpt;
+  if (ppt > pl.P) ppt = pl.P;
+  for (;;) {
+    pl.ppt = (uint32_t)ppt;
+    if (compress) {
+      pl.sm_tile = 0;
+      pl.sm_tile_bytes = (uint32_t)A16(ppt * pl.plane_bytes + 32);
+      pl.sm_out = pl.sm_tile + pl.sm_tile_bytes;
+      pl.sm_rec = pl.sm_out + (uint32_t)(ppt * pl.npay);
+      pl.sm_sal = pl.sm_rec + (uint32_t)A16(20 * ppt);
+      pl.sm_total = pl.sm_sal + nteams * pl.sm_sal_stride;
+    } else {
+      pl.sm_sal = 0;
+      pl.sm_total = nteams * pl.sm_sal_stride;
+    }
+    if (pl.sm_total <= kSmemLimit) break;
+    if (ppt == 1) return FH_ERR_UNSUPPORTED;
+    ppt = ppt / 2;
+  }
+  const uint64_t ntiles = (pl.P + pl.ppt - 1) / pl.ppt;
+  if (ntiles > 0x7FFFFFFFull) return FH_ERR_UNSUPPORTED;
+  pl.ntiles = (uint32_t)ntiles;
+  *out = pl;
+  return FH_OK;
+}
+
+// ---- per-stream scratch ---------------------------------------------------------------------
+struct StreamScratch {
+  fh::Scratch* sc = nullptr;
+  fh::TileState* ts = nullptr;
+  size_t ts_cap = 0;
+  uint32_t epoch = 0;
+  uint64_t ticket_base = 0, done_base = 0;
+  unsigned long long* sched = nullptr;  // schedule runner: offsets, sizes, statuses
+  size_t sched_cap = 0;
+};
+
+std::mutex g_mu;
+std::map<std::pair<int, cudaStream_t>, StreamScratch> g_scratch;
+int g_sm_count[64] = {0};
+
+int get_scratch(cudaStream_t stream, size_t ntiles, StreamScratch** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FH_ERR_CUDA;
+  StreamScratch& s = g_scratch[std::make_pair(dev, stream)];
+  if (!s.sc) {
+    if (cudaMalloc(&s.sc, sizeof(fh::Scratch)) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMemset(s.sc, 0, sizeof(fh::Scratch)) != cudaSuccess) return FH_ERR_CUDA;
+  }
+  if (ntiles > s.ts_cap) {
+    size_t cap = s.ts_cap ? s.ts_cap : 65536;
+    while (cap < ntiles) cap *= 2;
+    if (s.ts) {
+      cudaDeviceSynchronize();
+      cudaFree(s.ts);
+      s.ts = nullptr;
+      s.ts_cap = 0;
+    }
+    if (cudaMalloc(&s.ts, cap * sizeof(fh::TileState)) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMemset(s.ts, 0, cap * sizeof(fh::TileState)) != cudaSuccess) return FH_ERR_CUDA;
+    s.ts_cap = cap;
+  }
+  *out = &s;
+  return FH_OK;
+}
+
+// Advance the epoch; when it would wrap, clear the flags so that stale epochs cannot match.
+int next_epoch(StreamScratch* s, cudaStream_t stream) {
+  if (s->epoch >= 0x7FFFFFF0u) {
+    if (s->ts && cudaMemsetAsync(s->ts, 0, s->ts_cap * sizeof(fh::TileState), stream) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMemsetAsync(&s->sc->status, 0, sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
+    s->epoch = 0;
+  }
+  ++s->epoch;
+  return FH_OK;
+}
+
+int sm_count() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  if (!g_sm_count[dev]) cudaDeviceGetAttribute(&g_sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+  return g_sm_count[dev];
+}
+
+template <typename K>
+int grid_for(K kernel, size_t smem, uint32_t ntiles, int* grid) {
+  static std::map<std::pair<const void*, size_t>, int> cache;  // guarded by g_mu
+  const auto key = std::make_pair((const void*)kernel, smem);
+  auto it = cache.find(key);
+  int per_sm;
+  if (it == cache.end()) {
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
+      return FH_ERR_CUDA;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, fh::kThreads, smem) != cudaSuccess)
+      return FH_ERR_CUDA;
+    if (per_sm < 1) return FH_ERR_UNSUPPORTED;
+    cache[key] = per_sm;
+  } else {
+    per_sm = it->second;
+  }
+  const int sms = sm_count();
+  if (sms < 1) return FH_ERR_CUDA;
+  const uint64_t g = (uint64_t)per_sm * sms;
+  *grid = (int)(ntiles < g ? ntiles : g);
+  return FH_OK;
+}
+
+template <int DT, int BITS>
+int launch_compress_t(const Plan& pl, fh::CompressArgs& a, StreamScratch* s, cudaStream_t stream) {
+  int grid = 0;
+  int rc = grid_for(fh::compress_kernel<DT, BITS>, pl.sm_total, pl.ntiles, &grid);
+  if (rc != FH_OK) return rc;
+  a.ticket_base = s->ticket_base;
+  a.done_base = s->done_base;
+  fh::compress_kernel<DT, BITS><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
+  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  s->ticket_base += (uint64_t)pl.ntiles + (uint64_t)grid;
+  s->done_base += pl.ntiles;
+  g_launches.fetch_add(1);
+  return FH_OK;
+}
+
+int launch_compress(const Plan& pl, fh::CompressArgs& a, StreamScratch* s, cudaStream_t stream) {
+  if (pl.dtype == FH_F32) {
+    if (pl.bits == 2) return launch_compress_t<fh::kF32, 2>(pl, a, s, stream);
+    if (pl.bits == 4) return launch_compress_t<fh::kF32, 4>(pl, a, s, stream);
+    return launch_compress_t<fh::kF32, 8>(pl, a, s, stream);
+  }
+  if (pl.bits == 2) return launch_compress_t<fh::kBF16, 2>(pl, a, s, stream);
+  if (pl.bits == 4) return launch_compress_t<fh::kBF16, 4>(pl, a, s, stream);
+  return launch_compress_t<fh::kBF16, 8>(pl, a, s, stream);
+}
+
+template <int DT>
+int launch_decompress_t(const Plan& pl, fh::DecompressArgs& a, StreamScratch* s, cudaStream_t stream) {
+  int grid = 0;
+  int rc = grid_for(fh::decompress_kernel<DT>, pl.sm_total, pl.ntiles, &grid);
+  if (rc != FH_OK) return rc;
+  a.ticket_base = s->ticket_base;
+  a.done_base = s->done_base;
+  fh::decompress_kernel<DT><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
+  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  s->ticket_base += (uint64_t)pl.ntiles + (uint64_t)grid;
+  s->done_base += pl.ntiles;
+  g_launches.fetch_add(1);
+  return FH_OK;
+}
+
+int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
+                     size_t capacity, const unsigned long long* d_off_in, unsigned long long* d_off_out,
+                     unsigned long long* d_out2, cudaStream_t stream) {
+  Plan pl;
+  int rc = make_plan(desc, params, true, &pl);
+  if (rc != FH_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_mu);
+  StreamScratch* s = nullptr;
+  rc = get_scratch(stream, pl.ntiles, &s);
+  if (rc != FH_OK) return rc;
+  rc = next_epoch(s, stream);
+  if (rc != FH_OK) return rc;
+  fh::CompressArgs a;
+  a.src = (const uint8_t*)d_src;
+  a.dst_base = (uint8_t*)d_dst;
+  a.capacity = capacity;
+  a.d_off_in = d_off_in;
+  a.d_off_out = d_off_out;
+  a.out2 = d_out2;
+  a.sc = s->sc;
+  a.ts = s->ts;
+  a.epoch = s->epoch;
+  a.spin_limit = kSpinLimit;
+  return launch_compress(pl, a, s, stream);
+}
+
+int enqueue_decompress(const void* d_src, size_t src_bytes, const fh_tensor_desc* expect, void* d_dst,
+                       const unsigned long long* d_off_in, unsigned long long* d_status, cudaStream_t stream) {
+  Plan pl;
+  int rc = make_plan(expect, nullptr, false, &pl);
+  if (rc != FH_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_mu);
+  StreamScratch* s = nullptr;
+  rc = get_scratch(stream, 0, &s);
+  if (rc != FH_OK) return rc;
+  rc = next_epoch(s, stream);
+  if (rc != FH_OK) return rc;
+  fh::DecompressArgs a;
+  a.src_base = (const uint8_t*)d_src;
+  a.src_bytes = src_bytes;
+  a.d_off_in = d_off_in;
+  a.dst = (uint8_t*)d_dst;
+  a.d_status = d_status;
+  a.sc = s->sc;
+  a.epoch = s->epoch;
+  if (pl.dtype == FH_F32) return launch_decompress_t<fh::kF32>(pl, a, s, stream);
+  return launch_decompress_t<fh::kBF16>(pl, a, s, stream);
+}
+
+bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) != 0; }
+
+}  // namespace
+
+extern "C" {
+
+void fh_default_params(fh_params* p) {
+  if (!p) return;
+  p->bits = 2;
+  p->salient_mode = FH_SALIENT_AUTO;
+  p->rho_num = 1;
+  p->rho_den = 32;
+  p->block = 8;
+  p->tau_num = 1;
+  p->tau_den = 4;
+  p->eps = 0.0625f;
+  p->dense_bits = 8;
+  p->rounding = 0;
+  p->seed = 0;
+}
+
+int fh_version(void) { return 1; }
+
+int fh_device_count(void) {
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess) return FH_ERR_CUDA;
+  return n;
+}
+
+size_t fh_compressed_bytes(const fh_tensor_desc* desc, const fh_params* params, int which) {
+  if (check_desc(desc) != FH_OK || check_params(params) != FH_OK) return 0;
+  const size_t P = (size_t)desc->n * (size_t)desc->c, hw = (size_t)desc->h * (size_t)desc->w;
+  if (which == 0) return 64 + P * (16 + A16(4 * ((hw * (size_t)params->bits + 31) / 32)));
+  return 64 + P * (16 + A16(esize_of(desc->dtype) * hw));
+}
+
+int fh_compress(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
+                size_t dst_capacity, uint64_t* d_out2, void* stream) {
+  int rc = check_desc(desc);
+  if (rc != FH_OK) return rc;
+  rc = check_params(params);
+  if (rc != FH_OK) return rc;
+  if (!d_src || !d_dst || misaligned(d_src, 16) || misaligned(d_dst, 16) || misaligned(d_out2, 8)) return FH_ERR_ARG;
+  const size_t P = (size_t)desc->n * (size_t)desc->c;
+  if (dst_capacity < 64 + 16 * P) return FH_ERR_CAPACITY;
+  return enqueue_compress(desc, params, d_src, d_dst, dst_capacity, nullptr, nullptr,
+                          (unsigned long long*)d_out2, (cudaStream_t)stream);
+}
+
+int fh_decompress(const void* d_src, size_t src_bytes, const fh_tensor_desc* expect, void* d_dst,
+                  uint64_t* d_status, void* stream) {
+  int rc = check_desc(expect);
+  if (rc != FH_OK) return rc;
+  if (!d_src || !d_dst || misaligned(d_src, 16) || misaligned(d_dst, 16) || misaligned(d_status, 8)) return FH_ERR_ARG;
+  return enqueue_decompress(d_src, src_bytes, expect, d_dst, nullptr, (unsigned long long*)d_status,
+                            (cudaStream_t)stream);
+}
+
+int fh_run_schedule(const fh_sched_entry* entries, int32_t count, const fh_params* params, void* d_arena,
+                    size_t arena_bytes, fh_sched_report* report, void* stream_) {
+  if (!entries || count < 0 || !report || !d_arena || misaligned(d_arena, 256)) return FH_ERR_ARG;
+  int rc = check_params(params);
+  if (rc != FH_OK) return rc;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  std::memset(report, 0, sizeof(*report));
+  std::vector<int> idx;
+  for (int i = 0; i < count; ++i) {
+    if (entries[i].action == FH_COMPRESS) {
+      rc = check_desc(&entries[i].desc);
+      if (rc != FH_OK) return rc;
+      if (!entries[i].d_dense || !entries[i].d_restored || misaligned(entries[i].d_dense, 16) ||
+          misaligned(entries[i].d_restored, 16))
+        return FH_ERR_ARG;
+      Plan pl;
+      rc = make_plan(&entries[i].desc, params, true, &pl);
+      if (rc != FH_OK) return rc;
+      idx.push_back(i);
+      report->total_dense_bytes += pl.dense_bytes;
+    } else if (entries[i].action != FH_KEEP && entries[i].action != FH_EVICT) {
+      return FH_ERR_ARG;
+    }
+  }
+  const size_t k = idx.size();
+  if (k == 0) return FH_OK;
+  // device words: offsets[k+1] | out2[2k] | decode status[k]
+  const size_t words = (k + 1) + 2 * k + k;
+  unsigned long long* d_words = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_mu);
+    StreamScratch* s = nullptr;
+    rc = get_scratch(stream, 0, &s);
+    if (rc != FH_OK) return rc;
+    if (s->sched_cap < words) {
+      if (s->sched) {
+        cudaDeviceSynchronize();
+        cudaFree(s->sched);
+        s->sched = nullptr;
+      }
+      size_t cap = words < 1024 ? 1024 : 2 * words;
+      if (cudaMalloc(&s->sched, cap * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
+      s->sched_cap = cap;
+    }
+    d_words = s->sched;
+  }
+  unsigned long long* d_off = d_words;
+  unsigned long long* d_out2 = d_words + (k + 1);
+  unsigned long long* d_dst = d_out2 + 2 * k;
+  cudaEvent_t e0, e1, e2;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess ||
+      cudaEventCreate(&e2) != cudaSuccess)
+    return FH_ERR_CUDA;
+  rc = FH_OK;
+  if (cudaMemsetAsync(d_words, 0, words * sizeof(unsigned long long), stream) != cudaSuccess) rc = FH_ERR_CUDA;
+  cudaEventRecord(e0, stream);
+  for (size_t j = 0; j < k && rc == FH_OK; ++j) {  // forward order
+    const fh_sched_entry& en = entries[idx[j]];
+    rc = enqueue_compress(&en.desc, params, en.d_dense, d_arena, arena_bytes, d_off + j, d_off + j + 1,
+                          d_out2 + 2 * j, stream);
+  }
+  cudaEventRecord(e1, stream);
+  for (size_t j = k; j-- > 0 && rc == FH_OK;) {  // reverse order
+    const fh_sched_entry& en = entries[idx[j]];
+    rc = enqueue_decompress(d_arena, arena_bytes, &en.desc, en.d_restored, d_off + j, d_dst + j, stream);
+  }
+  cudaEventRecord(e2, stream);
+  if (cudaStreamSynchronize(stream) != cudaSuccess) rc = rc == FH_OK ? FH_ERR_CUDA : rc;
+  if (rc == FH_OK) {
+    std::vector<unsigned long long> h(words);
+    if (cudaMemcpy(h.data(), d_words, words * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess) {
+      rc = FH_ERR_CUDA;
+    } else {
+      cudaEventElapsedTime(&report->ms_forward, e0, e1);
+      cudaEventElapsedTime(&report->ms_backward, e1, e2);
+      int status = FH_OK;
+      uint64_t peak = 0;
+      for (size_t j = 0; j < k; ++j) {
+        const int cs = (int)(long long)h[(k + 1) + 2 * j + 1];
+        if (status == FH_OK && cs != FH_OK) status = cs;
+        if (cs == FH_OK) {
+          report->total_packed_bytes += h[(k + 1) + 2 * j];
+          if (h[j + 1] > peak) peak = h[j + 1];
+        }
+      }
+      for (size_t j = 0; j < k; ++j) {
+        const int ds = (int)(long long)h[(k + 1) + 2 * k + j];
+        if (status == FH_OK && ds != FH_OK) status = ds;
+      }
+      report->peak_packed_bytes = peak;
+      report->status = status;
+    }
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  cudaEventDestroy(e2);
+  return rc;
+}
+
+size_t fh_host_work_bytes(const fh_tensor_desc* desc, const fh_params* params) {
+  fh_params def;
+  fh_default_params(&def);
+  const size_t worst = fh_compressed_bytes(desc, params ? params : &def, 1);
+  if (!worst) return 0;
+  const size_t dense = (size_t)desc->n * desc->c * desc->h * desc->w * esize_of(desc->dtype);
+  return A256(dense) + 256 + A256(worst);
+}
+
+int fh_compress_host(const fh_tensor_desc* desc, const fh_params* params, const void* h_src, void* h_dst,
+                     size_t dst_capacity, uint64_t* h_out2, void* d_work, size_t work_bytes, void* stream_) {
+  int rc = check_desc(desc);
+  if (rc != FH_OK) return rc;
+  rc = check_params(params);
+  if (rc != FH_OK) return rc;
+  if (!h_src || !h_dst || !d_work || misaligned(d_work, 256)) return FH_ERR_ARG;
+  if (work_bytes < fh_host_work_bytes(desc, params)) return FH_ERR_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  const size_t dense = (size_t)desc->n * desc->c * desc->h * desc->w * esize_of(desc->dtype);
+  const size_t worst = fh_compressed_bytes(desc, params, 1);
+  uint8_t* d_dense = (uint8_t*)d_work;
+  unsigned long long* d_out2 = (unsigned long long*)(d_dense + A256(dense));
+  uint8_t* d_pack = (uint8_t*)d_out2 + 256;
+  const size_t cap = dst_capacity < worst ? dst_capacity : worst;
+  if (cudaMemcpyAsync(d_dense, h_src, dense, cudaMemcpyHostToDevice, stream) != cudaSuccess) return FH_ERR_CUDA;
+  rc = fh_compress(desc, params, d_dense, d_pack, cap, (uint64_t*)d_out2, stream_);
+  if (rc != FH_OK) return rc;
+  unsigned long long out2[2] = {0, 0};
+  if (cudaMemcpyAsync(out2, d_out2, 16, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (h_out2) {
+    h_out2[0] = out2[0];
+    h_out2[1] = out2[1];
+  }
+  const int st = (int)(long long)out2[1];
+  if (st != FH_OK) return st;
+  if (cudaMemcpyAsync(h_dst, d_pack, out2[0], cudaMemcpyDeviceToHost, stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return FH_ERR_CUDA;
+  return FH_OK;
+}
+
+int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc* expect, void* h_dst,
+                       uint64_t* h_status, void* d_work, size_t work_bytes, void* stream_) {
+  int rc = check_desc(expect);
+  if (rc != FH_OK) return rc;
+  if (!h_src || !h_dst || !d_work || misaligned(d_work, 256)) return FH_ERR_ARG;
+  const size_t need = fh_host_work_bytes(expect, nullptr);
+  if (work_bytes < need) return FH_ERR_ARG;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  const size_t dense = (size_t)expect->n * expect->c * expect->h * expect->w * esize_of(expect->dtype);
+  uint8_t* d_dense = (uint8_t*)d_work;
+  unsigned long long* d_st = (unsigned long long*)(d_dense + A256(dense));
+  uint8_t* d_pack = (uint8_t*)d_st + 256;
+  if (src_bytes > work_bytes - A256(dense) - 256) return FH_ERR_ARG;
+  if (cudaMemcpyAsync(d_pack, h_src, src_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return FH_ERR_CUDA;
+  rc = fh_decompress(d_pack, src_bytes, expect, d_dense, (uint64_t*)d_st, stream_);
+  if (rc != FH_OK) return rc;
+  unsigned long long st = 0;
+  if (cudaMemcpyAsync(h_dst, d_dense, dense, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (cudaMemcpyAsync(&st, d_st, 8, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (h_status) *h_status = st;
+  return (int)(long long)st;
+}
+
+uint64_t fh_kernel_launches(void) { return g_launches.load(); }
+
+void fh_shutdown(void) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  int cur = 0;
+  cudaGetDevice(&cur);
+  for (auto& kv : g_scratch) {
+    cudaSetDevice(kv.first.first);
+    cudaDeviceSynchronize();
+    if (kv.second.sc) cudaFree(kv.second.sc);
+    if (kv.second.ts) cudaFree(kv.second.ts);
+    if (kv.second.sched) cudaFree(kv.second.sched);
+  }
+  g_scratch.clear();
+  cudaSetDevice(cur);
+}
+
+}  // extern "C"

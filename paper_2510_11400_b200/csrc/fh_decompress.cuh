@@ -1,0 +1,277 @@
+// Decompress kernel: container -> dense tensor, one pass.
+//
+// Tiles of consecutive planes are handed out by a ticket counter; one team of threads restores one
+// plane: unpack-and-dequantise for normal planes, verbatim copy for raw planes, and for outlier-rich
+// planes zero fill + CSR scatter + inverse Lorenzo walk of the dense blocks.  Every read of the
+// container is bounds-checked against src_bytes; a plane whose table entry or payload is
+// inconsistent is left unwritten and the call reports FH_ERR_CORRUPT.
+#pragma once
+
+#include "fh_device.cuh"
+
+namespace fh {
+
+struct DecompressArgs {
+  const uint8_t* src_base;
+  unsigned long long src_bytes;
+  const unsigned long long* d_off_in;  // optional: byte offset of the container in src_base
+  uint8_t* dst;
+  unsigned long long* d_status;        // optional
+  Scratch* sc;
+  uint32_t epoch;
+  unsigned long long ticket_base, done_base;
+};
+
+template <int DT>
+__device__ __forceinline__ void store_elem(uint8_t* plane, uint32_t i, float v) {
+  if (DT == kF32) reinterpret_cast<float*>(plane)[i] = v;
+  else reinterpret_cast<uint16_t*>(plane)[i] = (uint16_t)f32_to_bf16_bits(v);
+}
+
+// x = fma(q, scale, lo); q < 2^23 is turned into a float through its bit pattern.
+__device__ __forceinline__ float dequant(uint32_t q, float scale, float lo) {
+  const float qf = __fsub_rn(__uint_as_float(0x4B000000u | q), 8388608.0f);
+  return __fmaf_rn(qf, scale, lo);
+}
+
+template <int DT, int BITS>
+__device__ __forceinline__ void decode_normal(const Team& t, const Plan& pl, const uint8_t* pay,
+                                              float lo, float scale, uint8_t* out) {
+  constexpr uint32_t L = (1u << BITS) - 1u;
+  const uint32_t HW = pl.HW, groups = pl.groups;
+  const bool vec = (pl.plane_bytes & (DT == kF32 ? 15u : 7u)) == 0u;  // dst base is 16-byte aligned
+  for (uint32_t g = t.lane; g < groups; g += t.size) {
+    uint32_t word;
+    if (BITS == 2) word = __ldg(pay + g);
+    else if (BITS == 4) word = __ldg(reinterpret_cast<const uint16_t*>(pay) + g);
+    else word = __ldg(reinterpret_cast<const uint32_t*>(pay) + g);
+    float v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) v[k] = dequant((word >> (k * BITS)) & L, scale, lo);
+    const uint32_t i0 = g * 4u;
+    if (vec && i0 + 3u < HW) {
+      if (DT == kF32) {
+        reinterpret_cast<float4*>(out)[g] = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
+        uint2 w;
+        w.x = f32_to_bf16_bits(v[0]) | (f32_to_bf16_bits(v[1]) << 16);
+        w.y = f32_to_bf16_bits(v[2]) | (f32_to_bf16_bits(v[3]) << 16);
+        reinterpret_cast<uint2*>(out)[g] = w;
+      }
+    } else {
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (i0 + k < HW) store_elem<DT>(out, i0 + k, v[k]);
+    }
+  }
+}
+
+// Outlier-rich plane.  `scr` is the team's shared scratch: nblk words.
+template <int DT>
+__device__ bool decode_salient(const Team& t, const Plan& pl, const uint8_t* pay, uint64_t avail,
+                               float eps, uint8_t* out, uint32_t* scr) {
+  const int H = pl.H, W = pl.W;
+  const uint32_t nblk = pl.nblk, nbx = pl.nbx, nbm = pl.nbm, e = (uint32_t)pl.esize, HW = pl.HW;
+  if (avail < 16) return false;
+  const uint32_t* p32 = reinterpret_cast<const uint32_t*>(pay);
+  const uint32_t nnz_s = __ldg(p32), n_dense = __ldg(p32 + 1), n_out_d = __ldg(p32 + 2);
+  if (nnz_s > HW || n_dense > nblk || n_out_d > HW) return false;
+  const uint64_t size = 16ull + 4ull * nbm + 4ull * ((uint64_t)H + 1) + a4(2u * nnz_s) + a4(e * nnz_s) +
+                        64ull * n_dense + a4(e * n_out_d);
+  if (size > avail) return false;
+  const uint32_t* g_bm = p32 + 4;
+  const uint32_t* g_rp = g_bm + nbm;
+  const uint8_t* g_col = reinterpret_cast<const uint8_t*>(g_rp + H + 1);
+  const uint8_t* g_val = g_col + a4(2u * nnz_s);
+  const uint8_t* g_codes = g_val + a4(e * nnz_s);
+  const uint8_t* g_outl = g_codes + 64u * n_dense;
+  bool ok = true;
+  // zero fill (16-bit units cover both element sizes)
+  for (uint32_t i = t.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += t.size)
+    reinterpret_cast<uint16_t*>(out)[i] = 0;
+  // verbatim counts of the dense blocks -> first verbatim index of each block
+  for (uint32_t b = t.lane; b < nblk; b += t.size) {
+    uint32_t cnt = 0;
+    if ((__ldg(g_bm + (b >> 5)) >> (b & 31u)) & 1u) {
+      uint32_t rank = 0;
+      for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(__ldg(g_bm + w));
+      rank += __popc(__ldg(g_bm + (b >> 5)) & ((1u << (b & 31u)) - 1u));
+      if (rank < n_dense) {
+        const uint32_t* c32 = reinterpret_cast<const uint32_t*>(g_codes + 64u * rank);
+        for (int k = 0; k < 16; ++k) {
+          const uint32_t w = __ldg(c32 + k);
+          // bytes equal to zero
+          cnt += ((w & 0xFFu) == 0) + ((w & 0xFF00u) == 0) + ((w & 0xFF0000u) == 0) + ((w & 0xFF000000u) == 0);
+        }
+      } else {
+        ok = false;
+      }
+    }
+    scr[b] = cnt;
+  }
+  team_sync(t);
+  const uint32_t tot_out = team_excl_scan(t, scr, nblk);
+  if (tot_out > n_out_d) ok = false;
+  // CSR scatter
+  for (int y = (int)t.lane; y < H; y += (int)t.size) {
+    const uint32_t r0 = __ldg(g_rp + y), r1 = __ldg(g_rp + y + 1);
+    if (r0 > r1 || r1 > nnz_s) { ok = false; continue; }
+    for (uint32_t k = r0; k < r1; ++k) {
+      const uint32_t col = __ldg(reinterpret_cast<const uint16_t*>(g_col) + k);
+      if (col >= (uint32_t)W) { ok = false; continue; }
+      const uint32_t idx = (uint32_t)y * W + col;
+      if (DT == kF32) reinterpret_cast<uint32_t*>(out)[idx] = __ldg(reinterpret_cast<const uint32_t*>(g_val) + k);
+      else reinterpret_cast<uint16_t*>(out)[idx] = __ldg(reinterpret_cast<const uint16_t*>(g_val) + k);
+    }
+  }
+  // dense blocks: raster walk, k = pred + residual (Eq. 7-9), x = k * 2 eps
+  const float two_eps = __fmul_rn(2.0f, eps);
+  const float inv2e = __fdiv_rn(1.0f, two_eps);
+  if (ok && tot_out <= n_out_d) {
+    for (uint32_t b = t.lane; b < nblk; b += t.size) {
+      if (!((__ldg(g_bm + (b >> 5)) >> (b & 31u)) & 1u)) continue;
+      uint32_t rank = 0;
+      for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(__ldg(g_bm + w));
+      rank += __popc(__ldg(g_bm + (b >> 5)) & ((1u << (b & 31u)) - 1u));
+      const uint32_t* c32 = reinterpret_cast<const uint32_t*>(g_codes + 64u * rank);
+      uint32_t oi = scr[b];
+      const int by = (int)(b / nbx), bx = (int)(b % nbx);
+      int32_t prev[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) prev[j] = 0;
+#pragma unroll 1
+      for (int i = 0; i < 8; ++i) {
+        const int y = by * 8 + i;
+        const uint32_t w0 = __ldg(c32 + 2 * i), w1 = __ldg(c32 + 2 * i + 1);
+        int32_t left = 0, ul = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int x = bx * 8 + j;
+          const uint32_t code = ((j < 4 ? w0 : w1) >> (8 * (j & 3))) & 0xFFu;
+          const int32_t up = prev[j];
+          const int32_t pred = up + left - ul;
+          int32_t k = pred;
+          if (y < H && x < W) {
+            const uint32_t idx = (uint32_t)y * W + x;
+            if (code == 0u) {
+              float v;
+              if (DT == kF32) {
+                const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(g_outl) + oi);
+                reinterpret_cast<uint32_t*>(out)[idx] = raw;
+                v = __uint_as_float(raw);
+              } else {
+                const uint32_t raw = __ldg(reinterpret_cast<const uint16_t*>(g_outl) + oi);
+                reinterpret_cast<uint16_t*>(out)[idx] = (uint16_t)raw;
+                v = bf16_bits_to_f32(raw);
+              }
+              bool big;
+              k = dense_k(v, inv2e, &big);
+              ++oi;
+            } else {
+              k = pred + (int32_t)code - 128;
+              store_elem<DT>(out, idx, __fmul_rn((float)k, two_eps));
+            }
+          }
+          ul = up;
+          left = k;
+          prev[j] = k;
+        }
+      }
+    }
+  }
+  return ok;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, const DecompressArgs a) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  __shared__ double s_red[kThreads / 32 * 4 + 8];
+  __shared__ uint32_t s_tile, s_hdr_ok, s_bits;
+  __shared__ float s_eps;
+  __shared__ unsigned long long s_total;
+  const uint32_t tid = threadIdx.x;
+  const unsigned long long off_in = a.d_off_in ? *a.d_off_in : 0ull;
+  const uint8_t* src = a.src_base + off_in;
+  const unsigned long long src_bytes = a.src_bytes > off_in ? a.src_bytes - off_in : 0ull;
+  const unsigned long long epoch_hi = (unsigned long long)a.epoch << 32;
+  const unsigned long long table_end = 64ull + 16ull * pl.P;
+  const Team team = make_team(pl.team, s_red);
+  const uint32_t nteams = team.block ? 1u : kThreads / team.size;
+  const uint32_t my_team = team.block ? 0u : tid / team.size;
+
+  // header check (every CTA, it is 64 bytes)
+  if (tid == 0) {
+    uint32_t ok = src_bytes >= table_end;
+    if (ok) {
+      const uint32_t* h = reinterpret_cast<const uint32_t*>(src);
+      const uint32_t bits = __ldg(h + 1) >> 24;
+      ok = __ldg(h) == kMagic && (__ldg(h + 1) & 0xFFFFu) == 1u && ((__ldg(h + 1) >> 16) & 0xFFu) == (uint32_t)pl.dtype &&
+           (bits == 2u || bits == 4u || bits == 8u) && __ldg(h + 2) == pl.N && __ldg(h + 3) == pl.C &&
+           __ldg(h + 4) == (uint32_t)pl.H && __ldg(h + 5) == (uint32_t)pl.W && (__ldg(h + 6) & 0xFFFFu) == (8u | (8u << 8));
+      const unsigned long long total = (unsigned long long)__ldg(h + 14) | ((unsigned long long)__ldg(h + 15) << 32);
+      const float eps = __uint_as_float(__ldg(h + 9));
+      ok = ok && total <= src_bytes && total >= table_end && eps >= 1e-30f && eps <= 1e30f;
+      s_bits = bits;
+      s_eps = eps;
+      s_total = total;
+    }
+    s_hdr_ok = ok;
+  }
+  __syncthreads();
+  const bool hdr_ok = s_hdr_ok != 0;
+  const uint32_t bits = hdr_ok ? s_bits : 2u;
+  const float eps = s_eps;
+  const unsigned long long total = hdr_ok ? s_total : 0ull;
+  const uint32_t npay_bytes = 4u * ((pl.HW * bits + 31u) / 32u);
+
+  for (;;) {
+    if (tid == 0) s_tile = (uint32_t)(atomicAdd(&a.sc->ticket, 1ull) - a.ticket_base);
+    __syncthreads();
+    const uint32_t tile = s_tile;
+    if (tile >= pl.ntiles) break;
+    const uint64_t p0 = (uint64_t)tile * pl.ppt;
+    const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+    bool bad = !hdr_ok;
+    if (hdr_ok) {
+      for (uint32_t lp = my_team; lp < np; lp += nteams) {
+        const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + (p0 + lp));
+        const unsigned long long off = (unsigned long long)e.x * 16ull;
+        const uint32_t cls = e.y & 3u;
+        uint8_t* out = a.dst + (p0 + lp) * pl.plane_bytes;
+        if (off < table_end || off > total) { bad = true; continue; }
+        const unsigned long long avail = total - off;
+        const uint8_t* pay = src + off;
+        if (cls == kClsNormal) {
+          if (npay_bytes > avail) { bad = true; continue; }
+          const float lo = __uint_as_float(e.z), scale = __uint_as_float(e.w);
+          if (bits == 2u) decode_normal<DT, 2>(team, pl, pay, lo, scale, out);
+          else if (bits == 4u) decode_normal<DT, 4>(team, pl, pay, lo, scale, out);
+          else decode_normal<DT, 8>(team, pl, pay, lo, scale, out);
+        } else if (cls == kClsRaw) {
+          if (pl.plane_bytes > avail) { bad = true; continue; }
+          for (uint32_t i = team.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += team.size)
+            reinterpret_cast<uint16_t*>(out)[i] = __ldg(reinterpret_cast<const uint16_t*>(pay) + i);
+        } else if (cls == kClsSalient) {
+          uint32_t* scr = reinterpret_cast<uint32_t*>(smem) + (uint64_t)my_team * pl.nblk;
+          if (!decode_salient<DT>(team, pl, pay, avail, eps, out, scr)) bad = true;
+        } else {
+          bad = true;
+        }
+      }
+    }
+    if (bad) atomicMax(&a.sc->status, epoch_hi | kErrCorrupt);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      const unsigned long long prev = atomicAdd(&a.sc->done, 1ull) - a.done_base;
+      if (prev == (unsigned long long)pl.ntiles - 1ull) {
+        __threadfence();
+        const unsigned long long st = ld_relaxed(&a.sc->status);
+        const uint32_t code = (st >> 32) == a.epoch ? (uint32_t)st : kErrNone;
+        if (a.d_status) *a.d_status = status_word(code);
+      }
+    }
+  }
+}
+
+}  // namespace fh

@@ -1,0 +1,303 @@
+"""Parity of the CUDA path with the CPU oracle, through the C ABI, on seeded synthetic activations.
+
+Bar: container bytes (header, plane table, payloads) and sizes bit-exact; restored values
+bit-identical (the contract allows 1 ulp; -0.0 and +0.0 compare equal).
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+
+from oracle import fho
+from paper_2510_11400_b200 import api, build, synth
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    api.lib()
+    yield
+    api.shutdown()
+
+
+def to_dev(raw):
+    import torch
+    t = torch.from_numpy(raw.view(np.int16) if raw.dtype == np.uint16 else raw)
+    return t.cuda()
+
+
+def gpu_compress(raw, shape, dtype, **kw):
+    p = api.default_params(**kw)
+    st, packed, total = api.compress_tensor(to_dev(raw), shape, dtype, p)
+    return st, packed, total
+
+
+def oracle_compress(raw, shape, dtype, **kw):
+    d = fho.desc(shape, dtype)
+    p = fho.params(**kw)
+    st, buf, total = fho.compress(raw, d, p)
+    return st, buf, total, d
+
+
+def check_same_values(a, b, dtype):
+    """Bit-identical except that -0.0 == +0.0."""
+    if dtype == synth.F32:
+        a32, b32 = a.view(np.uint32), b.view(np.uint32)
+        diff = (a32 != b32) & ~(((a32 | b32) & 0x7FFFFFFF) == 0)
+    else:
+        diff = (a != b) & ~(((a | b) & 0x7FFF) == 0)
+    assert not diff.any(), f"{int(diff.sum())} values differ, first at {int(np.flatnonzero(diff)[0])}"
+
+
+def full_parity(spec, **kw):
+    raw = synth.make(spec)
+    st_o, buf_o, total_o, d = oracle_compress(raw, spec.shape, spec.dtype, **kw)
+    assert st_o == fho.OK
+    st_g, packed, total_g = gpu_compress(raw, spec.shape, spec.dtype, **kw)
+    assert st_g == api.FH_OK
+    assert total_g == total_o
+    buf_g = packed[:total_g].cpu().numpy()
+    if not np.array_equal(buf_g, buf_o):
+        P = spec.shape[0] * spec.shape[1]
+        tg, to = hp.table(buf_g, P), hp.table(buf_o, P)
+        for key in ("cls", "n_out", "off"):
+            bad = np.flatnonzero(tg[key] != to[key])
+            assert bad.size == 0, f"table field {key} differs at planes {bad[:8]}: gpu {tg[key][bad[:8]]} oracle {to[key][bad[:8]]}"
+        assert np.array_equal(buf_g[:64], buf_o[:64]), "header differs"
+        first = int(np.flatnonzero(buf_g != buf_o)[0])
+        pl = int(np.searchsorted(to["off"], first, side="right") - 1)
+        raise AssertionError(f"payload bytes differ first at byte {first} (plane {pl}, class {to['cls'][pl]})")
+    st_d, out_g = api.decompress_tensor(packed, total_g, spec.shape, spec.dtype)
+    assert st_d == api.FH_OK
+    st_r, out_o = fho.decompress(buf_o, d)
+    assert st_r == fho.OK
+    out_g = out_g.cpu().numpy()
+    if spec.dtype == synth.BF16:
+        out_g = out_g.view(np.uint16)
+    check_same_values(out_g, out_o, spec.dtype)
+    return buf_o
+
+
+def test_config1_round_trip_at_2_bits():
+    buf = full_parity(synth.config1()[0], bits=2)
+    h = fho.parse_header(buf)
+    if h["n_salient"] == 0 and h["n_raw"] == 0:
+        assert buf.size == 139328
+
+
+SHAPES = [
+    (3, 5, 7, 7),      # 49-element planes: unaligned plane starts, tensor size not a multiple of 16 bytes
+    (2, 9, 14, 14),    # sub-warp teams
+    (1, 7, 1, 1),      # single-element planes
+    (2, 3, 3, 1),
+    (1, 5, 5, 7),
+    (2, 6, 33, 17),    # ragged 8x8 blocks in both directions
+    (1, 12, 32, 32),   # one warp per plane, vector loads
+    (2, 8, 28, 28),
+    (1, 6, 56, 56),    # whole-CTA teams, several planes per tile
+    (1, 3, 112, 112),  # whole-CTA teams, one plane per tile
+    (1, 2, 64, 100),
+    (300, 1, 4, 4),    # many tiny planes, several tiles with a ragged last tile
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_parity_auto_mode_mixed_planes(shape, dtype, bits):
+    kind = "spiky_relu" if (shape[1] >= 3) else "relu"
+    spec = synth.TensorSpec("t", shape, dtype, kind, 40 + bits)
+    full_parity(spec, bits=bits)
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+@pytest.mark.parametrize("mode", [api.FH_SALIENT_OFF, api.FH_SALIENT_ALL])
+def test_parity_forced_modes(shape, dtype, mode):
+    spec = synth.TensorSpec("t", shape, dtype, "normal" if mode == api.FH_SALIENT_OFF else "spiky_relu", 90)
+    full_parity(spec, bits=4, salient_mode=mode)
+
+
+@pytest.mark.parametrize("kind", ["relu", "normal", "laplace_ch", "laplace_iid", "spiky_normal"])
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_parity_value_distributions(kind, dtype):
+    spec = synth.TensorSpec("t", (4, 16, 28, 28), dtype, kind, 7)
+    full_parity(spec, bits=2)
+
+
+@pytest.mark.parametrize("eps,tau,rho", [(0.5, (1, 4), (1, 32)), (0.1, (1, 2), (1, 64)), (0.0625, (1, 64), (1, 16)),
+                                         (0.01, (3, 4), (0, 1))])
+def test_parity_other_parameters(eps, tau, rho):
+    spec = synth.TensorSpec("t", (2, 32, 24, 40), synth.F32, "spiky_relu", 11)
+    full_parity(spec, bits=4, eps=eps, tau=tau, rho=rho)
+
+
+def test_parity_multi_tile_scan_with_mixed_sizes():
+    """Many tiles whose sizes differ (salient, raw and normal planes mixed): the plane-ordered offsets
+    come from the look-back scan across tiles."""
+    spec = synth.TensorSpec("t", (64, 48, 14, 14), synth.F32, "spiky_relu", 5)
+    buf = full_parity(spec, bits=2)
+    t = hp.table(buf, 64 * 48)
+    assert (t["cls"] == fho.SALIENT).sum() > 100
+    spec = synth.TensorSpec("t", (16, 32, 56, 56), synth.BF16, "laplace_ch", 6)
+    full_parity(spec, bits=8)
+
+
+def test_special_values_constant_planes_negative_zero_tiny_range():
+    x = synth.normal(8 * 64, 3).reshape(8, 64)
+    x[0] = 2.5                      # constant plane: scale 0, exact
+    x[1] = 0.0
+    x[1, ::3] = -0.0                # signed zeros
+    x[2] = 1e-42                    # denormals, constant
+    x[3, :] = np.float32(1e-40) * np.arange(64)   # denormal range: inv overflows -> all codes 0
+    x[4] *= 1e30                    # huge but finite
+    x[5] = np.arange(64) % 4        # exact codes at 2 bits
+    raw = np.ascontiguousarray(x.reshape(-1), dtype=np.float32)
+    for mode in (api.FH_SALIENT_OFF, api.FH_SALIENT_AUTO, api.FH_SALIENT_ALL):
+        st_o, buf_o, total_o, d = oracle_compress(raw, (1, 8, 8, 8), synth.F32, bits=2, salient_mode=mode)
+        st_g, packed, total_g = gpu_compress(raw, (1, 8, 8, 8), synth.F32, bits=2, salient_mode=mode)
+        assert (st_o, st_g) == (0, 0) and total_o == total_g
+        assert np.array_equal(packed[:total_g].cpu().numpy(), buf_o)
+        st_d, out_g = api.decompress_tensor(packed, total_g, (1, 8, 8, 8), synth.F32)
+        _, out_o = fho.decompress(buf_o, d)
+        check_same_values(out_g.cpu().numpy(), out_o, synth.F32)
+
+
+def test_device_side_errors_nonfinite_capacity_corrupt():
+    import torch
+    shape = (2, 16, 16, 16)
+    raw = synth.relu_normal(2 * 16 * 256, 1)
+    # non-finite input
+    for bad in (np.nan, np.inf, -np.inf):
+        y = raw.copy()
+        y[5000] = bad
+        st, _, _ = gpu_compress(y, shape, synth.F32, bits=2)
+        assert st == api.FH_ERR_NONFINITE
+    y = raw.copy()
+    y[0], y[1] = 3e38, -3e38
+    assert gpu_compress(y, shape, synth.F32, bits=2)[0] == api.FH_ERR_NONFINITE
+    # capacity one byte short: error, needed size reported, nothing written past the capacity
+    p = api.default_params(bits=2, salient_mode=api.FH_SALIENT_OFF)
+    d = api.desc(shape)
+    need = api.compressed_bytes(d, p, 0)
+    x = to_dev(raw)
+    dst = torch.full((need + 64,), 0xAB, dtype=torch.uint8, device="cuda")
+    out2 = torch.zeros(2, dtype=torch.int64, device="cuda")
+    assert api.fh_compress(d, p, x, dst, out2, capacity=need - 1) == api.FH_OK
+    torch.cuda.synchronize()
+    assert out2.tolist() == [need, api.FH_ERR_CAPACITY]
+    assert bool((dst[need - 1:] == 0xAB).all())
+    assert api.fh_compress(d, p, x, dst, out2, capacity=need) == api.FH_OK
+    torch.cuda.synchronize()
+    assert out2.tolist() == [need, api.FH_OK]
+    assert bool((dst[need:] == 0xAB).all())
+    # corrupt container: magic, shape expectation, truncation, table offset
+    good = dst[:need].clone()
+    st, _ = api.decompress_tensor(good, need, shape, synth.F32)
+    assert st == api.FH_OK
+    b = good.clone(); b[0] ^= 1
+    assert api.decompress_tensor(b, need, shape, synth.F32)[0] == api.FH_ERR_CORRUPT
+    assert api.decompress_tensor(good, need, (2, 16, 16, 8), synth.F32)[0] == api.FH_ERR_CORRUPT
+    assert api.decompress_tensor(good, need - 1, shape, synth.F32)[0] == api.FH_ERR_CORRUPT
+    b = good.clone(); b[64 + 16 * 3 + 3] = 0xFF   # plane 3 points far outside the container
+    assert api.decompress_tensor(b, need, shape, synth.F32)[0] == api.FH_ERR_CORRUPT
+
+
+def test_corrupt_salient_payload_is_rejected_without_out_of_bounds_reads():
+    spec = synth.TensorSpec("t", (1, 16, 24, 40), synth.F32, "spiky_relu", 77)
+    raw = synth.make(spec)
+    st, packed, total = gpu_compress(raw, spec.shape, spec.dtype, bits=4)
+    assert st == api.FH_OK
+    buf = packed[:total].cpu().numpy()
+    t = hp.table(buf, 16)
+    pl = int(np.flatnonzero(t["cls"] == fho.SALIENT)[0])
+    off = int(t["off"][pl])
+    for field, val in ((0, 0x7FFFFFFF), (4, 0x7FFFFFFF), (8, 0x7FFFFFFF)):
+        b = packed.clone()
+        b[off + field:off + field + 4] = to_dev(np.frombuffer(np.uint32(val).tobytes(), dtype=np.uint8).copy())
+        assert api.decompress_tensor(b, total, spec.shape, spec.dtype)[0] == api.FH_ERR_CORRUPT
+
+
+def test_repeated_calls_reuse_the_scratch_and_stay_exact():
+    spec = synth.TensorSpec("t", (8, 32, 14, 14), synth.F32, "spiky_relu", 21)
+    raw = synth.make(spec)
+    _, buf_o, total_o, _ = oracle_compress(raw, spec.shape, spec.dtype, bits=2)
+    for _ in range(5):
+        st, packed, total = gpu_compress(raw, spec.shape, spec.dtype, bits=2)
+        assert st == 0 and total == total_o
+        assert np.array_equal(packed[:total].cpu().numpy(), buf_o)
+
+
+def test_schedule_forward_compress_reverse_decompress():
+    import torch
+    specs = [synth.TensorSpec(f"s{i}", s, synth.F32, "spiky_relu" if i == 2 else "relu", 500 + i, compress=(i % 2 == 0))
+             for i, s in enumerate([(4, 16, 32, 32), (4, 16, 32, 32), (4, 32, 16, 16), (4, 32, 16, 16),
+                                    (4, 64, 8, 8), (4, 64, 8, 8), (4, 128, 4, 4)])]
+    p = api.default_params(bits=2)
+    items, raws, restored = [], [], []
+    for s in specs:
+        raw = synth.make(s)
+        raws.append(raw)
+        dense = to_dev(raw)
+        rest = torch.zeros_like(dense)
+        restored.append(rest)
+        items.append(api.SchedItem(api.desc(s.shape, s.dtype, tensor_id=s.seed),
+                                   api.FH_COMPRESS if s.compress else api.FH_KEEP, dense, rest))
+    arena = torch.zeros(8 << 20, dtype=torch.uint8, device="cuda")
+    rep = api.fh_run_schedule(items, p, arena)
+    assert rep.status == api.FH_OK
+    off = 0
+    tot_packed = 0
+    for s, raw, rest in zip(specs, raws, restored):
+        if not s.compress:
+            assert not bool(rest.any())
+            continue
+        d = fho.desc(s.shape, s.dtype, tensor_id=s.seed)
+        st, buf_o, total_o = fho.compress(raw, d, fho.params(bits=2))
+        assert np.array_equal(arena[off:off + total_o].cpu().numpy(), buf_o)
+        _, out_o = fho.decompress(buf_o, d)
+        check_same_values(rest.cpu().numpy(), out_o, s.dtype)
+        tot_packed += total_o
+        off += (total_o + 255) & ~255
+    assert rep.total_packed_bytes == tot_packed
+    assert rep.peak_packed_bytes == off
+    assert rep.total_dense_bytes == sum(s.dense_bytes for s in specs if s.compress)
+    assert rep.ms_forward > 0 and rep.ms_backward > 0
+    # an arena that is too small: error, and the tensors that did not fit are not restored from stale bytes
+    small = arena[:off - 4096]
+    for r in restored:
+        r.zero_()
+    rep = api.fh_run_schedule(items, p, small)
+    assert rep.status == api.FH_ERR_CAPACITY
+    assert not bool(restored[-1].any())          # the last tensor did not fit: left untouched
+    assert bool(restored[0].any())               # the first one did and was restored
+
+
+def test_host_buffer_entry_points():
+    import torch
+    spec = synth.TensorSpec("t", (4, 16, 28, 28), synth.BF16, "laplace_ch", 9)
+    raw = synth.make(spec)
+    d = api.desc(spec.shape, spec.dtype)
+    p = api.default_params(bits=4)
+    work = torch.empty(api.host_work_bytes(d, p), dtype=torch.uint8, device="cuda")
+    h_src = torch.from_numpy(raw.view(np.int16)).pin_memory()
+    h_dst = torch.empty(api.compressed_bytes(d, p, 1), dtype=torch.uint8).pin_memory()
+    st, total = api.fh_compress_host(d, p, h_src, h_dst, work)
+    assert st == api.FH_OK
+    _, buf_o, total_o, od = oracle_compress(raw, spec.shape, spec.dtype, bits=4)
+    assert total == total_o and np.array_equal(h_dst[:total].numpy(), buf_o)
+    h_out = torch.empty_like(h_src)
+    assert api.fh_decompress_host(h_dst, total, d, h_out, work) == api.FH_OK
+    _, out_o = fho.decompress(buf_o, od)
+    check_same_values(h_out.numpy().view(np.uint16), out_o, spec.dtype)
+
+
+def test_launch_counter_counts_our_kernels():
+    before = api.kernel_launches()
+    raw = synth.relu_normal(2 * 4 * 64, 1)
+    st, packed, total = gpu_compress(raw, (2, 4, 8, 8), synth.F32, bits=2)
+    api.decompress_tensor(packed, total, (2, 4, 8, 8), synth.F32)
+    assert api.kernel_launches() == before + 2
