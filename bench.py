@@ -1,0 +1,389 @@
+#!/usr/bin/env python
+"""Benchmark of the activation codec on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one pass of the whole hot path over one batch of synthetic activations: for every code
+width b in {2, 4, 8}, compress every tensor of the workload (forward order), then decompress every
+one (reverse order), salient_mode AUTO.  The headline workload is the ResNet-18-shaped set of saved
+activations at batch 64 (17 fp32 tensors, 563.5 MiB dense).  `value` is dense GB/s: the dense bytes
+that went through compress plus those that came out of decompress, divided by the device time.
+
+One JSON line goes to stdout (rank 0).  With N > 1 (launched by torchrun) every rank runs the
+same workload on its own GPU -- planes and tensors are independent, there is no exchange step --
+and the value is the sum of the dense bytes over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2510_11400_b200 import synth  # noqa: E402
+
+BITS = (2, 4, 8)
+METRIC = "compress+decompress throughput, dense activation bytes"
+UNIT = "GB/s"
+
+
+def workload_specs(name: str):
+    if name == "resnet18_b64":
+        return synth.config2(64), "configs[1]: ResNet-18-shaped saved activations, batch 64, 224x224 input, fp32, " \
+                                  "17 tensors, 563.5 MiB dense; even tensors ReLU(N(0,1)), odd N(0,1)"
+    if name == "mobilenetv2_b128":
+        return synth.config3(128), "configs[2]: MobileNetV2-shaped expanded activations, batch 128, bf16, Laplace(0,1) " \
+                                   "with channel-clustered +-50 outliers"
+    if name == "cifar_schedule":
+        return synth.config5(128), "configs[4]: 20 ResNet-18/CIFAR-shaped tensors, batch 128, fp32 (all compressed here)"
+    if name == "config1":
+        return synth.config1(), "configs[0]: 32x16x32x32 fp32 ReLU(N(0,1))"
+    if name.startswith("sweep_"):          # sweep_<MiB>_<f32|bf16>
+        _, mib, dt = name.split("_")
+        return synth.config4(int(mib), synth.F32 if dt == "f32" else synth.BF16), \
+            f"configs[3]: single {mib} MiB {dt} tensor of 32x32 planes, ReLU(N(0,1))"
+    raise SystemExit(f"unknown workload {name}")
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return float(json.load(open(p))["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown," \
+        "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown," \
+        "clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
+# ------------------------------------------------------------------------------------------------
+
+def oracle_sample(specs, frac_planes: float):
+    """First planes of every tensor of the workload (planes are coded independently, so a prefix of
+    the batch is the same work per byte)."""
+    out = []
+    for s in specs:
+        n, c, h, w = s.shape
+        P = n * c
+        take = max(1, min(P, int(round(P * frac_planes))))
+        sub = synth.TensorSpec(s.name, (1, take, h, w), s.dtype, s.kind, s.seed)
+        out.append((sub, synth.make(sub)))
+    return out
+
+
+def time_oracle(sample, threads: int):
+    from oracle import fho
+    fho.set_threads(threads)
+    dense = 0
+    t0 = time.perf_counter()
+    for b in BITS:
+        p = fho.params(bits=b)
+        packed = []
+        for sub, raw in sample:
+            d = fho.desc(sub.shape, sub.dtype)
+            st, buf, total = fho.compress(raw, d, p)
+            assert st == 0
+            packed.append((d, buf))
+            dense += raw.nbytes
+        for d, buf in reversed(packed):
+            st, out = fho.decompress(buf, d)
+            assert st == 0
+            dense += out.nbytes
+    return dense, time.perf_counter() - t0
+
+
+def cpu_baseline(specs, budget_s: float = 15.0):
+    from oracle import fho
+    cores = fho.max_threads()
+    probe = oracle_sample(specs, 0.01)
+    dense, t = time_oracle(probe, cores)
+    rate = dense / max(t, 1e-6)
+    total_dense = sum(s.dense_bytes for s in specs) * 2 * len(BITS)
+    frac = min(1.0, budget_s * rate / total_dense)
+    sample = oracle_sample(specs, frac)
+    dense, t = time_oracle(sample, cores)
+    return {"value": dense / t / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {frac * 100:.2f}% of the planes of every tensor, bits 2/4/8, compress+decompress, "
+                      f"{dense / 2 / len(BITS) / 2**20:.1f} MiB dense per pass, {t:.1f} s"}
+
+
+def run_reference(args, specs, wl_desc):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import fho
+    cores = fho.max_threads()
+    probe = oracle_sample(specs, 0.01)
+    dense, t = time_oracle(probe, cores)
+    rate = dense / max(t, 1e-6)
+    total_dense = sum(s.dense_bytes for s in specs) * 2 * len(BITS)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    frac = min(1.0, budget * rate / total_dense)
+    sample = oracle_sample(specs, frac)
+    for _ in range(args.warmup):
+        time_oracle(sample, cores)
+    tot_d, tot_t = 0, 0.0
+    for _ in range(args.steps):
+        d, t = time_oracle(sample, cores)
+        tot_d += d
+        tot_t += t
+    val = tot_d / tot_t / 1e9
+    smp = f"first {frac * 100:.3f}% of the planes of every tensor per step ({tot_d / args.steps / 2**20:.1f} MiB dense " \
+          f"through the codec per step)"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": tot_t / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl_desc, "bits": list(BITS), "salient_mode": "AUTO", "sample": smp},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": smp},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+
+def run_ours(args, specs, wl_desc):
+    import torch
+    import torch.distributed as dist
+    from paper_2510_11400_b200 import api, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    build.build()
+    api.lib()
+
+    # the oracle is timed first (rank 0, N = 1 only), before the GPU is busy
+    cpu = cpu_baseline(specs) if (rank == 0 and world == 1 and not args.no_cpu) else None
+
+    dev = torch.device("cuda", local)
+    mode = {"auto": api.FH_SALIENT_AUTO, "off": api.FH_SALIENT_OFF, "all": api.FH_SALIENT_ALL}[args.mode]
+    params = {b: api.default_params(bits=b, salient_mode=mode) for b in BITS}
+    tensors = []
+    for i, s in enumerate(specs):
+        raw = synth.make(s)
+        t = torch.from_numpy(raw.view(np.int16) if raw.dtype == np.uint16 else raw).to(dev)
+        d = api.desc(s.shape, s.dtype, tensor_id=i)
+        cap = api.compressed_bytes(d, params[8], 1)
+        tensors.append(dict(spec=s, desc=d, dense=t, packed=torch.empty(cap, dtype=torch.uint8, device=dev),
+                            restored=torch.empty_like(t), cap=cap,
+                            out2={b: torch.zeros(2, dtype=torch.int64, device=dev) for b in BITS},
+                            st={b: torch.zeros(1, dtype=torch.int64, device=dev) for b in BITS}))
+    dense_bytes = sum(s.dense_bytes for s in specs)
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        for b in BITS:
+            if ev is not None:
+                ev[b][0].record(stream)
+            for t in tensors:
+                rc = api.fh_compress(t["desc"], params[b], t["dense"], t["packed"], t["out2"][b], capacity=t["cap"])
+                assert rc == 0, rc
+            if ev is not None:
+                ev[b][1].record(stream)
+            for t in reversed(tensors):
+                rc = api.fh_decompress(t["packed"], t["cap"], t["desc"], t["restored"], t["st"][b])
+                assert rc == 0, rc
+            if ev is not None:
+                ev[b][2].record(stream)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    packed_bytes = {}
+    for b in BITS:
+        tot = 0
+        for t in tensors:
+            total, st = t["out2"][b].tolist()
+            assert st == 0, f"device status {st}"
+            assert t["st"][b].item() == 0
+            tot += total
+        packed_bytes[b] = tot
+
+    evs = [{b: [torch.cuda.Event(enable_timing=True) for _ in range(3)] for b in BITS} for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = api.kernel_launches()
+    sampler.start()
+    e0.record(stream)
+    for k in range(args.steps):
+        step(evs[k])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    launches = api.kernel_launches() - launches0
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        tt = torch.tensor([ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    t_comp = {b: sum(e[b][0].elapsed_time(e[b][1]) for e in evs) for b in BITS}
+    t_dec = {b: sum(e[b][1].elapsed_time(e[b][2]) for e in evs) for b in BITS}
+
+    # ---- end to end through the host-buffer entry points (pinned host memory on both sides)
+    e2e = None
+    if not args.no_e2e:
+        work = torch.empty(max(api.host_work_bytes(t["desc"], params[8]) for t in tensors), dtype=torch.uint8, device=dev)
+        hosts = []
+        for t in tensors:
+            hosts.append(dict(src=t["dense"].cpu().pin_memory(), pack=torch.empty(t["cap"], dtype=torch.uint8).pin_memory(),
+                              out=torch.empty_like(t["dense"], device="cpu").pin_memory()))
+        def e2e_step():
+            h2d = d2h = 0
+            for b in BITS:
+                sizes = []
+                for t, h in zip(tensors, hosts):
+                    st, total = api.fh_compress_host(t["desc"], params[b], h["src"], h["pack"], work)
+                    assert st == 0, st
+                    sizes.append(total)
+                    h2d += t["spec"].dense_bytes
+                    d2h += total + 16
+                for t, h, total in reversed(list(zip(tensors, hosts, sizes))):
+                    st = api.fh_decompress_host(h["pack"], total, t["desc"], h["out"], work)
+                    assert st == 0, st
+                    h2d += total
+                    d2h += t["spec"].dense_bytes + 8
+            return h2d, d2h
+        e2e_step()
+        ksteps = max(1, min(args.steps, 3))
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(ksteps):
+            h2d, d2h = e2e_step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            tt = torch.tensor([dt], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            dt = float(tt.item())
+        e2e = {"value": world * ksteps * dense_bytes * 2 * len(BITS) / dt / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": ksteps}
+
+    if rank == 0:
+        peak, peak_kind = peaks()
+        n_comp = args.steps * len(BITS) * len(tensors)
+        alg_comp = args.steps * sum(dense_bytes + packed_bytes[b] for b in BITS)
+        comp_s = sum(t_comp.values()) / 1e3
+        achieved = alg_comp / comp_s / 1e9
+        traffic = None
+        value = world * args.steps * dense_bytes * 2 * len(BITS) / (ms / 1e3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32" if specs[0].dtype == synth.F32 else "bf16", "data": "synthetic",
+            "config": {"workload": wl_desc, "bits": list(BITS), "salient_mode": args.mode.upper(),
+                       "tensors": len(tensors), "dense_bytes_per_pass": dense_bytes,
+                       "packed_bytes": {str(b): packed_bytes[b] for b in BITS},
+                       "l2": "inputs larger than L2: every pass streams the whole dense set",
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "compress_gbs": {str(b): args.steps * dense_bytes / t_comp[b] / 1e6 for b in BITS},
+            "decompress_gbs": {str(b): args.steps * dense_bytes / t_dec[b] / 1e6 for b in BITS},
+            "roofline": {"bound": "hbm", "kernel": "compress_kernel", "achieved": achieved, "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
+                         "launches": n_comp, "avg_launch_us": comp_s / n_comp * 1e6,
+                         "algorithmic_bytes_per_launch": alg_comp / n_comp,
+                         "frac_of_nominal_8000": achieved / 8000.0,
+                         "decompress_achieved": args.steps * sum(dense_bytes + packed_bytes[b] for b in BITS)
+                         / (sum(t_dec.values()) / 1e3) / 1e9},
+            "clocks": clocks, "gpu_launches": int(launches),
+        }
+        if e2e is not None:
+            line["e2e"] = e2e
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    api.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18_b64")
+    ap.add_argument("--mode", default="auto", choices=["auto", "off", "all"])
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    specs, wl_desc = workload_specs(args.workload)
+    if args.impl == "reference":
+        run_reference(args, specs, wl_desc)
+    else:
+        run_ours(args, specs, wl_desc)
+
+
+if __name__ == "__main__":
+    main()
