@@ -185,6 +185,37 @@ int fh_compress_host(const fh_tensor_desc* desc, const fh_params* params, const 
 int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc* expect, void* h_dst,
                        uint64_t* h_status, void* d_work, size_t work_bytes, void* stream);
 
+/*
+ * fh_compress without any allocation.  (The paper has no counterpart; this exists for callers of this
+ * library.)
+ *
+ * fh_compress keeps its scan flags in a scratch buffer that it obtains with cudaMalloc on first use
+ * and enlarges when a bigger tensor arrives.  Some callers cannot afford that: the codec is called
+ * exactly when device memory is short (a training engine compresses activations because its budget
+ * is exhausted, so an allocation inside the codec can fail at the worst moment); a process whose
+ * device memory is wholly pre-reserved by a framework pool has nothing left for the driver to hand
+ * out; and a latency-bound training loop cannot take the device-wide synchronisation that
+ * cudaMalloc / cudaFree may imply.  This variant never calls cudaMalloc, cudaFree or any allocating
+ * routine: its scratch is a fixed array compiled into the library's device image
+ * (FH_STATIC_SCRATCH_BYTES bytes, resident on every GPU that loads the library until the process
+ * exits).
+ *
+ * Arguments, output, status reporting and the produced bytes are exactly those of fh_compress.
+ * Differences:
+ *   - the tensor may span at most FH_STATIC_MAX_TILES tiles (a tile is a run of planes of about
+ *     32 KB of dense data, or one plane when a plane is larger; so about 512 MiB of dense data);
+ *     anything larger returns FH_ERR_UNSUPPORTED and enqueues nothing;
+ *   - the first call on a device looks up the device address of the array (once per device, with
+ *     that device current).  Make that first call outside any stream capture;
+ *   - all calls on a device share the one array, which still holds the previous call's flags, so
+ *     each call first clears the part it uses with a memset on `stream`.  Two calls that overlap on
+ *     the GPU (different streams without ordering between them) race on it: order them.
+ */
+#define FH_STATIC_MAX_TILES 16384
+#define FH_STATIC_SCRATCH_BYTES (256 + 32 * FH_STATIC_MAX_TILES)
+int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
+                       size_t dst_capacity, uint64_t* d_out2, void* stream);
+
 /* Number of kernels this library has launched since it was loaded (for launch accounting). */
 uint64_t fh_kernel_launches(void);
 

@@ -18,10 +18,11 @@ FH_OK, FH_ERR_ARG, FH_ERR_UNSUPPORTED, FH_ERR_CAPACITY, FH_ERR_NONFINITE, FH_ERR
 FH_F32, FH_BF16 = 0, 1
 FH_SALIENT_AUTO, FH_SALIENT_OFF, FH_SALIENT_ALL = 0, 1, 2
 FH_KEEP, FH_COMPRESS, FH_EVICT = 0, 1, 2
+FH_STATIC_MAX_TILES = 16384
 
 EXPORTS = ["fh_default_params", "fh_version", "fh_device_count", "fh_compressed_bytes", "fh_compress",
            "fh_decompress", "fh_run_schedule", "fh_host_work_bytes", "fh_compress_host",
-           "fh_decompress_host", "fh_kernel_launches", "fh_shutdown"]
+           "fh_decompress_host", "fh_compress_static", "fh_kernel_launches", "fh_shutdown"]
 
 
 class FhError(RuntimeError):
@@ -87,6 +88,8 @@ def lib() -> C.CDLL:
         L.fh_decompress_host.argtypes = [C.c_void_p, C.c_size_t, D, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_size_t, C.c_void_p]
         L.fh_decompress_host.restype = C.c_int
+        L.fh_compress_static.argtypes = [D, P, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
+        L.fh_compress_static.restype = C.c_int
         L.fh_kernel_launches.restype = C.c_uint64
         L.fh_shutdown.restype = None
         _lib = L
@@ -127,6 +130,15 @@ def fh_compress(d: fh_tensor_desc, p: fh_params, src, dst, out2=None, stream=Non
     cap = dst.numel() * dst.element_size() if capacity is None else capacity
     return int(lib().fh_compress(C.byref(d), C.byref(p), src.data_ptr(), dst.data_ptr(), cap,
                                  out2.data_ptr() if out2 is not None else None, _stream_ptr(stream)))
+
+
+def fh_compress_static(d: fh_tensor_desc, p: fh_params, src, dst, out2=None, stream=None,
+                       capacity: Optional[int] = None) -> int:
+    """fh_compress for callers that must not allocate: same arguments and bytes, scan scratch in a fixed
+    array inside the library (at most FH_STATIC_MAX_TILES tiles; calls sharing a device must not overlap)."""
+    cap = dst.numel() * dst.element_size() if capacity is None else capacity
+    return int(lib().fh_compress_static(C.byref(d), C.byref(p), src.data_ptr(), dst.data_ptr(), cap,
+                                        out2.data_ptr() if out2 is not None else None, _stream_ptr(stream)))
 
 
 def fh_decompress(src, src_bytes: int, d: fh_tensor_desc, dst, status=None, stream=None) -> int:

@@ -523,6 +523,57 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
   return (int)(long long)st;
 }
 
+// ---- allocation-free compress -----------------------------------------------------------------
+// Scan scratch compiled into the device image: a Scratch header (padded to 256 bytes) followed by
+// FH_STATIC_MAX_TILES TileState records.  The name is a device symbol: host code must not pass it to a
+// kernel, it asks the runtime for the symbol's device address instead (once per device).
+static __device__ __align__(256) unsigned char g_static_scratch[FH_STATIC_SCRATCH_BYTES];
+static_assert(sizeof(fh::TileState) == 32 && sizeof(fh::Scratch) <= 256, "static scratch layout");
+
+static std::mutex g_static_mu;
+static unsigned char* g_static_ptr[64] = {nullptr};
+
+int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
+                       size_t dst_capacity, uint64_t* d_out2, void* stream_) {
+  int rc = check_desc(desc);
+  if (rc != FH_OK) return rc;
+  rc = check_params(params);
+  if (rc != FH_OK) return rc;
+  if (!d_src || !d_dst || misaligned(d_src, 16) || misaligned(d_dst, 16) || misaligned(d_out2, 8)) return FH_ERR_ARG;
+  const size_t P = (size_t)desc->n * (size_t)desc->c;
+  if (dst_capacity < 64 + 16 * P) return FH_ERR_CAPACITY;
+  Plan pl;
+  rc = make_plan(desc, params, true, &pl);
+  if (rc != FH_OK) return rc;
+  if (pl.ntiles > FH_STATIC_MAX_TILES) return FH_ERR_UNSUPPORTED;  // beyond the fixed scratch
+  cudaStream_t stream = (cudaStream_t)stream_;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FH_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {  // set-up, once per device, with that device current
+    unsigned char* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_static_scratch) != cudaSuccess || !p) return FH_ERR_CUDA;
+    g_static_ptr[dev] = p;
+  }
+  unsigned char* base = g_static_ptr[dev];
+  // the array keeps the last call's counters and flags: clear the part this call uses
+  if (cudaMemsetAsync(base, 0, 256 + sizeof(fh::TileState) * (size_t)pl.ntiles, stream) != cudaSuccess)
+    return FH_ERR_CUDA;
+  fh::CompressArgs a;
+  a.src = (const uint8_t*)d_src;
+  a.dst_base = (uint8_t*)d_dst;
+  a.capacity = dst_capacity;
+  a.d_off_in = nullptr;
+  a.d_off_out = nullptr;
+  a.out2 = (unsigned long long*)d_out2;
+  a.sc = reinterpret_cast<fh::Scratch*>(base);
+  a.ts = reinterpret_cast<fh::TileState*>(base + 256);
+  a.epoch = 1;
+  a.spin_limit = kSpinLimit;
+  StreamScratch counters;  // tickets and the done count start from zero after the memset
+  return launch_compress(pl, a, &counters, stream);
+}
+
 uint64_t fh_kernel_launches(void) { return g_launches.load(); }
 
 void fh_shutdown(void) {
