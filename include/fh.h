@@ -202,17 +202,17 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
  *
  * Arguments, output, status reporting and the produced bytes are exactly those of fh_compress.
  * Differences:
- *   - the tensor may span at most FH_STATIC_MAX_TILES tiles (a tile is a run of planes of about
- *     32 KB of dense data, or one plane when a plane is larger; so about 512 MiB of dense data);
- *     anything larger returns FH_ERR_UNSUPPORTED and enqueues nothing;
+ *   - the tensor may span at most FH_STATIC_MAX_TILES tiles (a tile is a run of consecutive planes of
+ *     8 to 32 KB of dense data, or a single plane when planes are larger; so roughly 0.5 to 2 GiB of
+ *     dense data); anything larger returns FH_ERR_UNSUPPORTED and enqueues nothing;
  *   - the first call on a device looks up the device address of the array (once per device, with
  *     that device current).  Make that first call outside any stream capture;
  *   - all calls on a device share the one array, which still holds the previous call's flags, so
  *     each call first clears the part it uses with a memset on `stream`.  Two calls that overlap on
  *     the GPU (different streams without ordering between them) race on it: order them.
  */
-#define FH_STATIC_MAX_TILES 16384
-#define FH_STATIC_SCRATCH_BYTES (256 + 32 * FH_STATIC_MAX_TILES)
+#define FH_STATIC_MAX_TILES 65536
+#define FH_STATIC_SCRATCH_BYTES (256 + 8 * FH_STATIC_MAX_TILES)
 int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                        size_t dst_capacity, uint64_t* d_out2, void* stream);
 

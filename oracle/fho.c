@@ -120,7 +120,11 @@ static int check_args(const fho_desc* d, const fho_params* p) {
 
 /* ------------------------------------------------------------------------------------------
  * Sizes.  Container (a layout choice; the paper gives none), little-endian:
- *   [0,64) header | [64, 64+16P) plane table | payloads in plane order, each padded to 16 bytes.
+ *   [0,64) header | [64, 64+16P) plane table | P fixed slots of npay bytes | overflow region.
+ * Every plane owns one slot, npay = A16(4*ceil(HW*bits/32)) bytes, at a closed-form offset.  A
+ * normal plane's codes fill its slot.  The payload of a salient or raw plane is laid through its
+ * slot first and continues, if longer, in the overflow region (plane order, each part padded to
+ * 16 bytes); its table entry holds the offset of that continuation (0 if there is none).
  * ------------------------------------------------------------------------------------------ */
 static size_t normal_payload(size_t hw, int bits) { return 4 * ((hw * (size_t)bits + 31) / 32); }
 
@@ -133,18 +137,57 @@ size_t fho_compressed_bytes(const fho_desc* d, const fho_params* p, int which) {
 
 /* ------------------------------------------------------------------------------------------
  * Three-sigma statistics of one plane (Section 4.4.1: "Outliers are identified using the
- * empirical 3-sigma rule").  mu and sigma are taken over the plane.  To make the result
- * independent of summation order up to fp64 rounding, sums are formed from fp32 partials of
- * 4 consecutive elements (tail padded with zeros) that are then added in fp64:
- *   s_g = (x0+x1)+(x2+x3),  q_g = fma(x1,x1,x0*x0) + fma(x3,x3,x2*x2)        (fp32)
- *   S = sum s_g, Q = sum q_g                                                  (fp64)
- *   mu = S/HW, var = max(Q/HW - mu*mu, 0), sigma = sqrt(var)                   (fp64)
- *   T_hi = (float)(mu + 3 sigma), T_lo = (float)(mu - 3 sigma)
- *   n_out = #{ x > T_hi or x < T_lo }                                         (fp32 compares)
+ * empirical 3-sigma rule").  mu and sigma are taken over the plane.
+ *
+ * The paper does not say how the moments are accumulated.  Here they are accumulated in fixed
+ * point, which makes the result exactly independent of the order of summation (so that any
+ * parallel implementation reproduces it bit for bit):
+ *   A   = max(|min x|, |max x|),  e = unbiased exponent field of A  (2^e <= A < 2^(e+1))
+ *   c_s = 2^k_s, k_s = min(18 - e, 126);   c_q = 2^k_q, k_q = clamp(16 - 2e, -126, 126)
+ *   per group of 4 consecutive elements (tail padded with zeros), in fp32:
+ *     s_g = (x0+x1)+(x2+x3),  q_g = fma(x1,x1,x0*x0) + fma(x3,x3,x2*x2)
+ *     i_s = round_half_even(s_g * c_s),  i_q = round_half_even(q_g * c_q)      (|.| < 2^21)
+ *     taken as the mantissa of fma(s_g, c_s, 1.5*2^23): bits(result) - bits(1.5*2^23)
+ *   I_s = sum i_s, I_q = sum i_q                                                (exact integers)
+ *   r = 1/HW (fp64);  mu = (I_s * 2^-k_s) * r;  m2 = (I_q * 2^-k_q) * r          (fp64)
+ *   var = max(m2 - mu*mu, 0)                                                     (fp64)
+ *   mu_f = (float)mu, sigma_f = sqrtf((float)var)
+ *   T_hi = fma(3, sigma_f, mu_f), T_lo = fma(-3, sigma_f, mu_f)                  (fp32)
+ *   n_out = #{ x > T_hi or x < T_lo }                                           (fp32 compares)
  * ------------------------------------------------------------------------------------------ */
-void fho_plane_sigma(const float* x, int64_t hw, double* S_out, double* Q_out, float* t_lo,
-                     float* t_hi, int64_t* n_out) {
-  double S = 0.0, Q = 0.0;
+static int32_t fixed_point(float v, float c) {
+  const float M = 12582912.0f; /* 1.5 * 2^23: adding it leaves the rounded integer in the mantissa */
+  float r = fmaf(v, c, M);
+  uint32_t rb, mb;
+  memcpy(&rb, &r, 4);
+  memcpy(&mb, &M, 4);
+  return (int32_t)(rb - mb);
+}
+
+static float pow2f(int k) { /* 2^k for -126 <= k <= 127 */
+  uint32_t b = (uint32_t)(k + 127) << 23;
+  float f;
+  memcpy(&f, &b, 4);
+  return f;
+}
+
+void fho_plane_sums(const float* x, int64_t hw, int64_t* Is_out, int64_t* Iq_out, int32_t* ks_out,
+                    int32_t* kq_out) {
+  float lo = x[0], hi = x[0];
+  for (int64_t i = 1; i < hw; ++i) {
+    if (x[i] < lo) lo = x[i];
+    if (x[i] > hi) hi = x[i];
+  }
+  float A = fmaxf(fabsf(lo), fabsf(hi));
+  uint32_t ab;
+  memcpy(&ab, &A, 4);
+  int e = (int)((ab >> 23) & 255u) - 127;
+  int ks = 18 - e, kq = 16 - 2 * e;
+  if (ks > 126) ks = 126;
+  if (kq > 126) kq = 126;
+  if (kq < -126) kq = -126;
+  float cs = pow2f(ks), cq = pow2f(kq);
+  int64_t Is = 0, Iq = 0;
   for (int64_t g = 0; g < hw; g += 4) {
     float v[4] = {0.f, 0.f, 0.f, 0.f};
     for (int k = 0; k < 4 && g + k < hw; ++k) v[k] = x[g + k];
@@ -153,18 +196,31 @@ void fho_plane_sigma(const float* x, int64_t hw, double* S_out, double* Q_out, f
     float p0 = v[0] * v[0], p2 = v[2] * v[2];
     float q01 = fmaf(v[1], v[1], p0), q23 = fmaf(v[3], v[3], p2);
     float qg = q01 + q23;
-    S += (double)sg;
-    Q += (double)qg;
+    Is += fixed_point(sg, cs);
+    Iq += fixed_point(qg, cq);
   }
-  double mu = S / (double)hw;
-  double ex2 = Q / (double)hw;
+  *Is_out = Is;
+  *Iq_out = Iq;
+  *ks_out = ks;
+  *kq_out = kq;
+}
+
+void fho_plane_sigma(const float* x, int64_t hw, double* S_out, double* Q_out, float* t_lo,
+                     float* t_hi, int64_t* n_out) {
+  int64_t Is, Iq;
+  int32_t ks, kq;
+  fho_plane_sums(x, hw, &Is, &Iq, &ks, &kq);
+  double S = ldexp((double)Is, -ks), Q = ldexp((double)Iq, -kq);
+  double r = 1.0 / (double)hw;
+  double mu = S * r;
+  double m2 = Q * r;
   double mu2 = mu * mu;
-  double var = ex2 - mu2;
+  double var = m2 - mu2;
   if (!(var > 0.0)) var = 0.0;
-  double sigma = sqrt(var);
-  double three = 3.0 * sigma;
-  float thi = (float)(mu + three);
-  float tlo = (float)(mu - three);
+  float mu_f = (float)mu;
+  float sigma_f = sqrtf((float)var);
+  float thi = fmaf(3.0f, sigma_f, mu_f);
+  float tlo = fmaf(-3.0f, sigma_f, mu_f);
   int64_t cnt = 0;
   for (int64_t i = 0; i < hw; ++i)
     if (x[i] > thi || x[i] < tlo) ++cnt;
@@ -234,8 +290,9 @@ typedef struct {
   uint32_t cls;
   uint32_t n_out;
   float lo, scale;
-  uint8_t* payload; /* malloc'd, a16-padded, zero padded */
-  size_t bytes;     /* a16(payload size) */
+  uint8_t* payload; /* malloc'd, zero padded to a16(size) */
+  size_t size;      /* payload bytes before padding */
+  size_t bytes;     /* a16(size) */
   int status;
 } plane_result;
 
@@ -398,17 +455,20 @@ static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_
     if (a16(size) >= a16(e * hw)) { /* no gain: keep the plane verbatim */
       free(buf);
       cls = CLS_RAW;
+      r->size = e * hw;
       r->bytes = a16(e * hw);
       r->payload = (uint8_t*)calloc(r->bytes, 1);
       memcpy(r->payload, raw, e * hw);
     } else {
       r->payload = buf;
+      r->size = size;
       r->bytes = a16(size);
     }
   } else {
     float inv, scale;
     fho_quant_params(lo, hi, p->bits, &inv, &scale);
     size_t size = normal_payload(hw, p->bits);
+    r->size = size;
     r->bytes = a16(size);
     r->payload = (uint8_t*)calloc(r->bytes, 1);
     for (size_t i = 0; i < hw; ++i) {
@@ -439,11 +499,12 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
 #endif
   for (int64_t pl = 0; pl < (int64_t)P; ++pl)
     encode_plane((const uint8_t*)src + (size_t)pl * hw * e, d->dtype, d->h, d->w, p, &res[pl]);
-  size_t total = 64 + 16 * P;
+  const size_t npay = a16(normal_payload(hw, p->bits));
+  size_t total = 64 + 16 * P + P * npay;
   uint32_t n_sal = 0, n_raw = 0;
   for (size_t pl = 0; pl < P; ++pl) {
     if (res[pl].status != FHO_OK) st = res[pl].status;
-    total += res[pl].bytes;
+    if (res[pl].bytes > npay) total += res[pl].bytes - npay; /* continuation in the overflow region */
     n_sal += res[pl].cls == CLS_SALIENT;
     n_raw += res[pl].cls == CLS_RAW;
   }
@@ -474,15 +535,26 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
     memcpy(o + 48, &d->tensor_id, 8);
     uint64_t tb = total;
     memcpy(o + 56, &tb, 8);
-    size_t off = 64 + 16 * P;
+    size_t slots = 64 + 16 * P, ovf = slots + P * npay;
+    memset(o + slots, 0, P * npay);
     for (size_t pl = 0; pl < P; ++pl) {
       uint8_t* te = o + 64 + 16 * pl;
-      put_u32(te, (uint32_t)(off / 16));
+      uint8_t* slot = o + slots + pl * npay;
+      size_t in_slot = res[pl].bytes < npay ? res[pl].bytes : npay;
+      memcpy(slot, res[pl].payload, in_slot);
+      uint32_t off16 = (uint32_t)((slots + pl * npay) / 16);
+      if (res[pl].cls != CLS_NORMAL) {
+        off16 = 0;
+        if (res[pl].bytes > npay) {
+          off16 = (uint32_t)(ovf / 16);
+          memcpy(o + ovf, res[pl].payload + npay, res[pl].bytes - npay);
+          ovf += res[pl].bytes - npay;
+        }
+      }
+      put_u32(te, off16);
       put_u32(te + 4, res[pl].cls | (res[pl].n_out << 2));
       memcpy(te + 8, &res[pl].lo, 4);
       memcpy(te + 12, &res[pl].scale, 4);
-      memcpy(o + off, res[pl].payload, res[pl].bytes);
-      off += res[pl].bytes;
     }
   }
   for (size_t pl = 0; pl < P; ++pl) free(res[pl].payload);
@@ -503,6 +575,9 @@ static void store_elem(uint8_t* dst, int dtype, size_t i, float v) {
   }
 }
 
+static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, float eps, uint32_t nnz_s,
+                                  uint32_t n_dense, uint32_t n_out_d, uint8_t* out);
+
 static int decode_plane(const uint8_t* src, size_t src_bytes, size_t pl, size_t P, int dtype, int H,
                         int W, int bits, float eps, uint8_t* out) {
   size_t hw = (size_t)H * W, e = esize(dtype);
@@ -513,33 +588,62 @@ static int decode_plane(const uint8_t* src, size_t src_bytes, size_t pl, size_t 
   float lo, scale;
   memcpy(&lo, te + 8, 4);
   memcpy(&scale, te + 12, 4);
-  if (off < 64 + 16 * P || off > src_bytes) return FHO_ERR_CORRUPT;
-  const uint8_t* pay = src + off;
-  size_t avail = src_bytes - off;
+  const size_t npay = a16(normal_payload(hw, bits));
+  const size_t slots = 64 + 16 * P, ovf0 = slots + P * npay;
+  if (ovf0 > src_bytes) return FHO_ERR_CORRUPT;
+  const uint8_t* slot = src + slots + pl * npay;
   if (cls == CLS_NORMAL) {
-    if (normal_payload(hw, bits) > avail) return FHO_ERR_CORRUPT;
+    if (off != slots + pl * npay) return FHO_ERR_CORRUPT;
     uint32_t mask = (1u << bits) - 1u;
     for (size_t i = 0; i < hw; ++i) {
       size_t bit = i * (size_t)bits;
-      uint32_t q = (get_u32(pay + 4 * (bit / 32)) >> (bit % 32)) & mask;
+      uint32_t q = (get_u32(slot + 4 * (bit / 32)) >> (bit % 32)) & mask;
       store_elem(out, dtype, i, fho_dequant(q, lo, scale));
     }
     return FHO_OK;
   }
-  if (cls == CLS_RAW) {
-    if (e * hw > avail) return FHO_ERR_CORRUPT;
-    memcpy(out, pay, e * hw);
-    return FHO_OK;
-  }
-  if (cls != CLS_SALIENT) return FHO_ERR_CORRUPT;
+  if (cls != CLS_SALIENT && cls != CLS_RAW) return FHO_ERR_CORRUPT;
   const int B = 8;
   int nby = (H + B - 1) / B, nbx = (W + B - 1) / B, nblk = nby * nbx;
   size_t nbm = ((size_t)nblk + 31) / 32;
-  if (16 > avail) return FHO_ERR_CORRUPT;
-  uint32_t nnz_s = get_u32(pay), n_dense = get_u32(pay + 4), n_out_d = get_u32(pay + 8);
-  size_t size = 16 + 4 * nbm + 4 * ((size_t)H + 1) + a4(2 * (size_t)nnz_s) + a4(e * nnz_s) +
-                64 * (size_t)n_dense + a4(e * n_out_d);
-  if (size > avail) return FHO_ERR_CORRUPT;
+  uint32_t nnz_s = 0, n_dense = 0, n_out_d = 0;
+  size_t size;
+  if (cls == CLS_RAW) {
+    size = e * hw;
+  } else {
+    nnz_s = get_u32(slot);
+    n_dense = get_u32(slot + 4);
+    n_out_d = get_u32(slot + 8);
+    if (nnz_s > hw || n_dense > (uint32_t)nblk || n_out_d > hw) return FHO_ERR_CORRUPT;
+    size = 16 + 4 * nbm + 4 * ((size_t)H + 1) + a4(2 * (size_t)nnz_s) + a4(e * nnz_s) +
+           64 * (size_t)n_dense + a4(e * n_out_d);
+  }
+  /* the payload runs through the slot and continues at `off` in the overflow region */
+  uint8_t* pay = (uint8_t*)calloc(a16(size) + 16, 1);
+  memcpy(pay, slot, size < npay ? size : npay);
+  if (size > npay) {
+    if (off < ovf0 || off > src_bytes || size - npay > src_bytes - off) {
+      free(pay);
+      return FHO_ERR_CORRUPT;
+    }
+    memcpy(pay + npay, src + off, size - npay);
+  }
+  if (cls == CLS_RAW) {
+    memcpy(out, pay, e * hw);
+    free(pay);
+    return FHO_OK;
+  }
+  int rc = decode_salient_payload(pay, dtype, H, W, eps, nnz_s, n_dense, n_out_d, out);
+  free(pay);
+  return rc;
+}
+
+static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, float eps, uint32_t nnz_s,
+                                  uint32_t n_dense, uint32_t n_out_d, uint8_t* out) {
+  const int B = 8;
+  size_t hw = (size_t)H * W, e = esize(dtype);
+  int nby = (H + B - 1) / B, nbx = (W + B - 1) / B, nblk = nby * nbx;
+  size_t nbm = ((size_t)nblk + 31) / 32;
   const uint8_t* bm = pay + 16;
   const uint8_t* rp = bm + 4 * nbm;
   const uint8_t* colp = rp + 4 * ((size_t)H + 1);
@@ -616,7 +720,7 @@ int fho_decompress(const void* src, size_t src_bytes, const fho_desc* expect, vo
   uint64_t tb;
   memcpy(&tb, s + 56, 8);
   size_t P = (size_t)N * C, hw = (size_t)H * W, e = esize(dtype);
-  if (tb > src_bytes || tb < 64 + 16 * P) return FHO_ERR_CORRUPT;
+  if (tb > src_bytes || tb < 64 + 16 * P + P * a16(normal_payload(hw, bits))) return FHO_ERR_CORRUPT;
   int st = FHO_OK;
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)

@@ -72,6 +72,9 @@ def lib():
         L.fho_plane_sigma.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_double),
                                       C.POINTER(C.c_double), C.POINTER(C.c_float),
                                       C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+        L.fho_plane_sums.restype = None
+        L.fho_plane_sums.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
+                                     C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         L.fho_quant_params.restype = None
         L.fho_quant_params.argtypes = [C.c_float, C.c_float, C.c_int, C.POINTER(C.c_float),
                                        C.POINTER(C.c_float)]
@@ -127,6 +130,15 @@ def plane_sigma(x: np.ndarray):
     lib().fho_plane_sigma(x.ctypes.data, x.size, C.byref(S), C.byref(Q), C.byref(tlo), C.byref(thi),
                           C.byref(n))
     return S.value, Q.value, tlo.value, thi.value, n.value
+
+
+def plane_sums(x: np.ndarray):
+    """Fixed-point moment sums of a plane: (I_s, I_q, k_s, k_q)."""
+    x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
+    a, b = C.c_int64(), C.c_int64()
+    ks, kq = C.c_int32(), C.c_int32()
+    lib().fho_plane_sums(x.ctypes.data, x.size, C.byref(a), C.byref(b), C.byref(ks), C.byref(kq))
+    return a.value, b.value, ks.value, kq.value
 
 
 def quant_params(lo: float, hi: float, bits: int):

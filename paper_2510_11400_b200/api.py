@@ -18,7 +18,7 @@ FH_OK, FH_ERR_ARG, FH_ERR_UNSUPPORTED, FH_ERR_CAPACITY, FH_ERR_NONFINITE, FH_ERR
 FH_F32, FH_BF16 = 0, 1
 FH_SALIENT_AUTO, FH_SALIENT_OFF, FH_SALIENT_ALL = 0, 1, 2
 FH_KEEP, FH_COMPRESS, FH_EVICT = 0, 1, 2
-FH_STATIC_MAX_TILES = 16384
+FH_STATIC_MAX_TILES = 65536
 
 EXPORTS = ["fh_default_params", "fh_version", "fh_device_count", "fh_compressed_bytes", "fh_compress",
            "fh_decompress", "fh_run_schedule", "fh_host_work_bytes", "fh_compress_host",

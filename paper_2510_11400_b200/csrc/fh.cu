@@ -20,7 +20,8 @@ namespace {
 using fh::Plan;
 
 constexpr size_t kSmemLimit = 227 * 1024 - 1024;  // dynamic shared memory a CTA may ask for
-constexpr size_t kTileTarget = 32 * 1024;         // dense bytes a tile aims for
+constexpr size_t kTileTarget = 32 * 1024;         // dense bytes a tile of the generic kernel aims for
+constexpr size_t kStageTarget = 72 * 1024;        // shared memory the stages of a fast kernel aim for
 constexpr uint32_t kMaxPpt = 2048;
 constexpr uint32_t kSpinLimit = 1u << 20;
 
@@ -55,10 +56,22 @@ uint32_t pow2_floor(uint32_t x) {
   return r;
 }
 
-// Tiling and shared-memory layout.  `compress` selects the compress kernel's layout (staged tile,
-// code staging, per-plane records, block-wise scratch); the decompress kernel only needs the
-// block-wise scratch.
-int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* out) {
+uint32_t pow2_ceil(uint32_t x) {
+  uint32_t r = 1;
+  while (r < x) r *= 2;
+  return r;
+}
+
+// Which kernel a plan runs on.
+struct Variant {
+  bool fast = false;  // compress_fast (register-resident groups, bulk-copy pipeline)
+  bool cta = false;   // fast: one plane per CTA instead of one plane per sub-warp team
+  int G = 0;          // fast: groups per thread
+};
+
+// Tiling and shared-memory layout.  `compress` selects the compress kernels' layout; the decompress
+// kernel only needs the block-wise scratch.
+int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* out, Variant* var) {
   Plan pl;
   std::memset(&pl, 0, sizeof(pl));
   pl.dtype = d->dtype;
@@ -74,6 +87,7 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   pl.P = (uint64_t)d->n * (uint64_t)d->c;
   pl.plane_bytes = hw * pl.esize;
   pl.dense_bytes = pl.P * pl.plane_bytes;
+  pl.inv_hw = 1.0 / (double)hw;
   pl.bits = p ? p->bits : 2;
   pl.mode = p ? p->salient_mode : 0;
   pl.rho_num = p ? p->rho_num : 1;
@@ -83,6 +97,8 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   pl.eps = p ? p->eps : 0.0625f;
   pl.tensor_id = d->tensor_id;
   pl.npay = (uint32_t)A16(4 * (((uint64_t)pl.HW * pl.bits + 31) / 32));
+  pl.slots_off = 64 + 16 * pl.P;
+  pl.ovf_off = pl.slots_off + pl.P * pl.npay;
   pl.nbx = (uint32_t)(d->w + 7) / 8;
   pl.nby = (uint32_t)(d->h + 7) / 8;
   pl.nblk = pl.nbx * pl.nby;
@@ -91,52 +107,91 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   const long double worst = 64.0L + (long double)pl.P * (16.0L + (long double)A16(pl.plane_bytes));
   if (worst / 16.0L >= 4294967295.0L) return FH_ERR_UNSUPPORTED;
   if (pl.P > 0x7FFFFFFFull) return FH_ERR_UNSUPPORTED;
-
-  if (pl.plane_bytes <= 8192) {
-    uint32_t t = pow2_floor(pl.HW / 8 > 0 ? pl.HW / 8 : 1);
-    pl.team = t > 32 ? 32 : t;
-  } else {
-    pl.team = fh::kThreads;
-  }
-  const uint32_t nteams = pl.team > 32 ? 1 : fh::kThreads / pl.team;
   const bool need_sal = compress ? (pl.mode != FH_SALIENT_OFF) : true;
-  pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * ((size_t)(compress ? (pl.H + 1 + 3 * pl.nblk) : pl.nblk))) : 0;
+  const size_t sal_words = compress ? (size_t)(pl.H + 1 + 3 * pl.nblk) : (size_t)pl.nblk;
 
-  uint64_t ppt = kTileTarget / pl.plane_bytes;
-  if (ppt < 1) ppt = 1;
-  if (ppt > kMaxPpt) ppt = kMaxPpt;
-  if (ppt > pl.P) ppt = pl.P;
-  for (;;) {
-    pl.ppt = (uint32_t)ppt;
-    if (compress) {
-      pl.sm_tile = 0;
-      pl.sm_tile_bytes = (uint32_t)A16(ppt * pl.plane_bytes + 32);
-      pl.sm_out = pl.sm_tile + pl.sm_tile_bytes;
-      pl.sm_rec = pl.sm_out + (uint32_t)(ppt * pl.npay);
-      pl.sm_sal = pl.sm_rec + (uint32_t)A16(20 * ppt);
-      pl.sm_total = pl.sm_sal + nteams * pl.sm_sal_stride;
+  Variant v;
+  // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
+  if (compress && pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0 && pl.groups <= 4096) {
+    v.fast = true;
+    if (pl.groups <= 256) {
+      uint32_t t = pow2_ceil((pl.groups + 7) / 8);
+      pl.team = t > 32 ? 32 : t;
+      v.G = (int)pow2_ceil((pl.groups + pl.team - 1) / pl.team);
+      pl.ppt = fh::kThreads / pl.team;
     } else {
-      pl.sm_sal = 0;
-      pl.sm_total = nteams * pl.sm_sal_stride;
+      v.cta = true;
+      pl.team = fh::kThreads;
+      v.G = (int)pow2_ceil((pl.groups + fh::kThreads - 1) / fh::kThreads);
+      pl.ppt = 1;
     }
-    if (pl.sm_total <= kSmemLimit) break;
-    if (ppt == 1) return FH_ERR_UNSUPPORTED;
-    ppt = ppt / 2;
+    if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
+    pl.stage_bytes = (uint32_t)(pl.ppt * pl.plane_bytes);
+    pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * sal_words) : 0;
+    const uint32_t nsal_teams = v.cta ? 1 : fh::kWarps;
+    uint32_t ns = (uint32_t)(kStageTarget / pl.stage_bytes);
+    ns = ns < 2 ? 2 : (ns > (uint32_t)fh::kMaxStages ? (uint32_t)fh::kMaxStages : ns);
+    for (;;) {
+      pl.nstage = ns;
+      pl.sm_tile = 0;
+      pl.sm_rec = (uint32_t)A16((size_t)ns * pl.stage_bytes);
+      pl.sm_sal = pl.sm_rec + (uint32_t)A16(20 * (size_t)pl.ppt);
+      pl.sm_total = pl.sm_sal + nsal_teams * pl.sm_sal_stride;
+      if (pl.sm_total <= kSmemLimit) break;
+      if (ns == 1) {
+        v.fast = false;
+        break;
+      }
+      --ns;
+    }
+  }
+  if (!v.fast) {
+    v = Variant();
+    if (pl.plane_bytes <= 8192) {
+      uint32_t t = pow2_floor(pl.HW / 8 > 0 ? pl.HW / 8 : 1);
+      pl.team = t > 32 ? 32 : t;
+    } else {
+      pl.team = fh::kThreads;
+    }
+    const uint32_t nteams = pl.team > 32 ? 1 : fh::kThreads / pl.team;
+    pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * sal_words) : 0;
+    pl.nstage = 0;
+    pl.stage_bytes = 0;
+    uint64_t ppt = kTileTarget / pl.plane_bytes;
+    if (ppt < 1) ppt = 1;
+    if (ppt > kMaxPpt) ppt = kMaxPpt;
+    if (ppt > pl.P) ppt = pl.P;
+    for (;;) {
+      pl.ppt = (uint32_t)ppt;
+      if (compress) {
+        pl.sm_tile = 0;
+        pl.sm_out = (uint32_t)A16(ppt * pl.plane_bytes + 32);
+        pl.sm_rec = pl.sm_out + (uint32_t)(ppt * pl.npay);
+        pl.sm_sal = pl.sm_rec + (uint32_t)A16(20 * ppt);
+        pl.sm_total = pl.sm_sal + nteams * pl.sm_sal_stride;
+      } else {
+        pl.sm_sal = 0;
+        pl.sm_total = nteams * pl.sm_sal_stride;
+      }
+      if (pl.sm_total <= kSmemLimit) break;
+      if (ppt == 1) return FH_ERR_UNSUPPORTED;
+      ppt = ppt / 2;
+    }
   }
   const uint64_t ntiles = (pl.P + pl.ppt - 1) / pl.ppt;
   if (ntiles > 0x7FFFFFFFull) return FH_ERR_UNSUPPORTED;
   pl.ntiles = (uint32_t)ntiles;
   *out = pl;
+  if (var) *var = v;
   return FH_OK;
 }
 
 // ---- per-stream scratch ---------------------------------------------------------------------
 struct StreamScratch {
   fh::Scratch* sc = nullptr;
-  fh::TileState* ts = nullptr;
+  unsigned long long* ts = nullptr;  // scan words
   size_t ts_cap = 0;
   uint32_t epoch = 0;
-  uint64_t ticket_base = 0, done_base = 0;
   unsigned long long* sched = nullptr;  // schedule runner: offsets, sizes, statuses
   size_t sched_cap = 0;
 };
@@ -162,19 +217,18 @@ int get_scratch(cudaStream_t stream, size_t ntiles, StreamScratch** out) {
       s.ts = nullptr;
       s.ts_cap = 0;
     }
-    if (cudaMalloc(&s.ts, cap * sizeof(fh::TileState)) != cudaSuccess) return FH_ERR_CUDA;
-    if (cudaMemset(s.ts, 0, cap * sizeof(fh::TileState)) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMalloc(&s.ts, cap * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMemset(s.ts, 0, cap * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
     s.ts_cap = cap;
   }
   *out = &s;
   return FH_OK;
 }
 
-// Advance the epoch; when it would wrap, clear the flags so that stale epochs cannot match.
+// Advance the 30-bit epoch; when it would wrap, clear the scan words so that stale epochs cannot match.
 int next_epoch(StreamScratch* s, cudaStream_t stream) {
-  if (s->epoch >= 0x7FFFFFF0u) {
-    if (s->ts && cudaMemsetAsync(s->ts, 0, s->ts_cap * sizeof(fh::TileState), stream) != cudaSuccess) return FH_ERR_CUDA;
-    if (cudaMemsetAsync(&s->sc->status, 0, sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (s->epoch >= 0x3FFFFFF0u) {
+    if (s->ts && cudaMemsetAsync(s->ts, 0, s->ts_cap * sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
     s->epoch = 0;
   }
   ++s->epoch;
@@ -211,43 +265,77 @@ int grid_for(K kernel, size_t smem, uint32_t ntiles, int* grid) {
   return FH_OK;
 }
 
-template <int DT, int BITS>
-int launch_compress_t(const Plan& pl, fh::CompressArgs& a, StreamScratch* s, cudaStream_t stream) {
-  int grid = 0;
-  int rc = grid_for(fh::compress_kernel<DT, BITS>, pl.sm_total, pl.ntiles, &grid);
-  if (rc != FH_OK) return rc;
-  a.ticket_base = s->ticket_base;
-  a.done_base = s->done_base;
-  fh::compress_kernel<DT, BITS><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
-  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
-  s->ticket_base += (uint64_t)pl.ntiles + (uint64_t)grid;
-  s->done_base += pl.ntiles;
-  g_launches.fetch_add(1);
-  return FH_OK;
+template <typename K>
+int launch_on(K kernel, const Plan& pl, cudaStream_t stream, int* grid) {
+  return grid_for(kernel, pl.sm_total, pl.ntiles, grid);
 }
 
-int launch_compress(const Plan& pl, fh::CompressArgs& a, StreamScratch* s, cudaStream_t stream) {
-  if (pl.dtype == FH_F32) {
-    if (pl.bits == 2) return launch_compress_t<fh::kF32, 2>(pl, a, s, stream);
-    if (pl.bits == 4) return launch_compress_t<fh::kF32, 4>(pl, a, s, stream);
-    return launch_compress_t<fh::kF32, 8>(pl, a, s, stream);
+template <int DT, int BITS>
+int launch_generic_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
+  int grid = 0;
+  int rc = grid_for(fh::compress_generic<DT, BITS>, pl.sm_total, pl.ntiles, &grid);
+  if (rc != FH_OK) return rc;
+  fh::compress_generic<DT, BITS><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
+  return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+}
+
+template <int DT, bool SIGMA, int G, bool CTA>
+int launch_fast_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
+  int grid = 0;
+  int rc = grid_for(fh::compress_fast<DT, SIGMA, G, CTA>, pl.sm_total, pl.ntiles, &grid);
+  if (rc != FH_OK) return rc;
+  fh::compress_fast<DT, SIGMA, G, CTA><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
+  return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+}
+
+template <int DT, bool SIGMA>
+int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
+  if (!v.cta) {
+    switch (v.G) {
+      case 1: return launch_fast_t<DT, SIGMA, 1, false>(pl, a, stream);
+      case 2: return launch_fast_t<DT, SIGMA, 2, false>(pl, a, stream);
+      case 4: return launch_fast_t<DT, SIGMA, 4, false>(pl, a, stream);
+      case 8: return launch_fast_t<DT, SIGMA, 8, false>(pl, a, stream);
+    }
+  } else {
+    switch (v.G) {
+      case 2: return launch_fast_t<DT, SIGMA, 2, true>(pl, a, stream);
+      case 4: return launch_fast_t<DT, SIGMA, 4, true>(pl, a, stream);
+      case 8: return launch_fast_t<DT, SIGMA, 8, true>(pl, a, stream);
+      case 16: return launch_fast_t<DT, SIGMA, 16, true>(pl, a, stream);
+    }
   }
-  if (pl.bits == 2) return launch_compress_t<fh::kBF16, 2>(pl, a, s, stream);
-  if (pl.bits == 4) return launch_compress_t<fh::kBF16, 4>(pl, a, s, stream);
-  return launch_compress_t<fh::kBF16, 8>(pl, a, s, stream);
+  return FH_ERR_UNSUPPORTED;
+}
+
+int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
+  int rc;
+  if (v.fast) {
+    const bool sigma = pl.mode == FH_SALIENT_AUTO;
+    if (pl.dtype == FH_F32)
+      rc = sigma ? launch_fast_g<fh::kF32, true>(pl, v, a, stream) : launch_fast_g<fh::kF32, false>(pl, v, a, stream);
+    else
+      rc = sigma ? launch_fast_g<fh::kBF16, true>(pl, v, a, stream) : launch_fast_g<fh::kBF16, false>(pl, v, a, stream);
+  } else if (pl.dtype == FH_F32) {
+    rc = pl.bits == 2   ? launch_generic_t<fh::kF32, 2>(pl, a, stream)
+         : pl.bits == 4 ? launch_generic_t<fh::kF32, 4>(pl, a, stream)
+                        : launch_generic_t<fh::kF32, 8>(pl, a, stream);
+  } else {
+    rc = pl.bits == 2   ? launch_generic_t<fh::kBF16, 2>(pl, a, stream)
+         : pl.bits == 4 ? launch_generic_t<fh::kBF16, 4>(pl, a, stream)
+                        : launch_generic_t<fh::kBF16, 8>(pl, a, stream);
+  }
+  if (rc == FH_OK) g_launches.fetch_add(1);
+  return rc;
 }
 
 template <int DT>
-int launch_decompress_t(const Plan& pl, fh::DecompressArgs& a, StreamScratch* s, cudaStream_t stream) {
+int launch_decompress_t(const Plan& pl, const fh::DecompressArgs& a, cudaStream_t stream) {
   int grid = 0;
   int rc = grid_for(fh::decompress_kernel<DT>, pl.sm_total, pl.ntiles, &grid);
   if (rc != FH_OK) return rc;
-  a.ticket_base = s->ticket_base;
-  a.done_base = s->done_base;
   fh::decompress_kernel<DT><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
   if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
-  s->ticket_base += (uint64_t)pl.ntiles + (uint64_t)grid;
-  s->done_base += pl.ntiles;
   g_launches.fetch_add(1);
   return FH_OK;
 }
@@ -256,7 +344,8 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
                      size_t capacity, const unsigned long long* d_off_in, unsigned long long* d_off_out,
                      unsigned long long* d_out2, cudaStream_t stream) {
   Plan pl;
-  int rc = make_plan(desc, params, true, &pl);
+  Variant v;
+  int rc = make_plan(desc, params, true, &pl, &v);
   if (rc != FH_OK) return rc;
   std::lock_guard<std::mutex> lock(g_mu);
   StreamScratch* s = nullptr;
@@ -275,19 +364,17 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   a.ts = s->ts;
   a.epoch = s->epoch;
   a.spin_limit = kSpinLimit;
-  return launch_compress(pl, a, s, stream);
+  return launch_compress(pl, v, a, stream);
 }
 
 int enqueue_decompress(const void* d_src, size_t src_bytes, const fh_tensor_desc* expect, void* d_dst,
                        const unsigned long long* d_off_in, unsigned long long* d_status, cudaStream_t stream) {
   Plan pl;
-  int rc = make_plan(expect, nullptr, false, &pl);
+  int rc = make_plan(expect, nullptr, false, &pl, nullptr);
   if (rc != FH_OK) return rc;
   std::lock_guard<std::mutex> lock(g_mu);
   StreamScratch* s = nullptr;
   rc = get_scratch(stream, 0, &s);
-  if (rc != FH_OK) return rc;
-  rc = next_epoch(s, stream);
   if (rc != FH_OK) return rc;
   fh::DecompressArgs a;
   a.src_base = (const uint8_t*)d_src;
@@ -296,9 +383,8 @@ int enqueue_decompress(const void* d_src, size_t src_bytes, const fh_tensor_desc
   a.dst = (uint8_t*)d_dst;
   a.d_status = d_status;
   a.sc = s->sc;
-  a.epoch = s->epoch;
-  if (pl.dtype == FH_F32) return launch_decompress_t<fh::kF32>(pl, a, s, stream);
-  return launch_decompress_t<fh::kBF16>(pl, a, s, stream);
+  if (pl.dtype == FH_F32) return launch_decompress_t<fh::kF32>(pl, a, stream);
+  return launch_decompress_t<fh::kBF16>(pl, a, stream);
 }
 
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) != 0; }
@@ -375,7 +461,7 @@ int fh_run_schedule(const fh_sched_entry* entries, int32_t count, const fh_param
           misaligned(entries[i].d_restored, 16))
         return FH_ERR_ARG;
       Plan pl;
-      rc = make_plan(&entries[i].desc, params, true, &pl);
+      rc = make_plan(&entries[i].desc, params, true, &pl, nullptr);
       if (rc != FH_OK) return rc;
       idx.push_back(i);
       report->total_dense_bytes += pl.dense_bytes;
@@ -525,10 +611,10 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
 
 // ---- allocation-free compress -----------------------------------------------------------------
 // Scan scratch compiled into the device image: a Scratch header (padded to 256 bytes) followed by
-// FH_STATIC_MAX_TILES TileState records.  The name is a device symbol: host code must not pass it to a
+// FH_STATIC_MAX_TILES scan words.  The name is a device symbol: host code must not pass it to a
 // kernel, it asks the runtime for the symbol's device address instead (once per device).
 static __device__ __align__(256) unsigned char g_static_scratch[FH_STATIC_SCRATCH_BYTES];
-static_assert(sizeof(fh::TileState) == 32 && sizeof(fh::Scratch) <= 256, "static scratch layout");
+static_assert(sizeof(fh::Scratch) <= 256, "static scratch layout");
 
 static std::mutex g_static_mu;
 static unsigned char* g_static_ptr[64] = {nullptr};
@@ -543,7 +629,8 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   const size_t P = (size_t)desc->n * (size_t)desc->c;
   if (dst_capacity < 64 + 16 * P) return FH_ERR_CAPACITY;
   Plan pl;
-  rc = make_plan(desc, params, true, &pl);
+  Variant v;
+  rc = make_plan(desc, params, true, &pl, &v);
   if (rc != FH_OK) return rc;
   if (pl.ntiles > FH_STATIC_MAX_TILES) return FH_ERR_UNSUPPORTED;  // beyond the fixed scratch
   cudaStream_t stream = (cudaStream_t)stream_;
@@ -556,8 +643,8 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
     g_static_ptr[dev] = p;
   }
   unsigned char* base = g_static_ptr[dev];
-  // the array keeps the last call's counters and flags: clear the part this call uses
-  if (cudaMemsetAsync(base, 0, 256 + sizeof(fh::TileState) * (size_t)pl.ntiles, stream) != cudaSuccess)
+  // the array keeps the last call's counters and scan words: clear the part this call uses
+  if (cudaMemsetAsync(base, 0, 256 + sizeof(unsigned long long) * (size_t)pl.ntiles, stream) != cudaSuccess)
     return FH_ERR_CUDA;
   fh::CompressArgs a;
   a.src = (const uint8_t*)d_src;
@@ -567,11 +654,10 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   a.d_off_out = nullptr;
   a.out2 = (unsigned long long*)d_out2;
   a.sc = reinterpret_cast<fh::Scratch*>(base);
-  a.ts = reinterpret_cast<fh::TileState*>(base + 256);
+  a.ts = reinterpret_cast<unsigned long long*>(base + 256);
   a.epoch = 1;
   a.spin_limit = kSpinLimit;
-  StreamScratch counters;  // tickets and the done count start from zero after the memset
-  return launch_compress(pl, a, &counters, stream);
+  return launch_compress(pl, v, a, stream);
 }
 
 uint64_t fh_kernel_launches(void) { return g_launches.load(); }

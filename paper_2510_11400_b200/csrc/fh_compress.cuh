@@ -1,36 +1,58 @@
-// Compress kernel: one pass over the dense tensor.
+// Compress kernels: one pass over the dense tensor.
 //
-// A persistent grid of CTAs takes tiles (runs of consecutive planes) from a ticket counter.  For
-// each tile the CTA stages the planes in shared memory, and then, entirely on chip,
-//   A. per plane (one team of threads each): min/max and three-sigma statistics, the plane class,
-//      and either the packed codes of a normal plane (into a shared staging buffer) or the size of
-//      the block-wise encoding of an outlier-rich plane;
-//   B. sums the tile's payload sizes, publishes them, and finds the tile's byte offset in the
-//      container by a decoupled look-back over the preceding tiles (bounded wait);
-//   C. writes table entries and payloads.
-// The dense tensor is read from DRAM exactly once and nothing but the container is written.
+// Container recap: every plane owns a slot of npay bytes at a closed-form offset; a normal plane's
+// codes fill its slot; the payload of a salient or raw plane runs through its slot and continues in
+// the overflow region, in plane order.  Normal planes therefore never wait for anything: statistics,
+// class, codes and the stores happen in one sweep.  Only tiles that hold salient or raw planes need
+// their place in the overflow region, which a decoupled look-back over per-tile scan words supplies.
+//
+// Two kernels share this file:
+//   compress_fast<DT, SIGMA, G, CTA>  planes whose size is a multiple of 16 bytes and that fit the
+//       register budget: tiles stream into shared memory through a multi-stage bulk-copy (TMA)
+//       pipeline, every thread keeps its G groups in registers for all passes;
+//   compress_generic<DT, BITS>        everything else (ragged planes, very large planes): staged with
+//       plain loads, passes re-read shared memory.
 #pragma once
 
 #include "fh_device.cuh"
 
 namespace fh {
 
-struct Rec {       // per-plane result of phase A, in shared memory
-  float lo, scale;
-  uint32_t meta;   // class | n_out << 2
-  uint32_t size16; // padded payload size / 16
-};
-
 struct SalientInfo {
   uint32_t nnz_s, n_dense, n_out_d, size;
 };
 
+struct CompressArgs {
+  const uint8_t* src;
+  uint8_t* dst_base;
+  unsigned long long capacity;          // bytes available at dst_base (minus the offset below)
+  const unsigned long long* d_off_in;   // optional: byte offset of the container in dst_base
+  unsigned long long* d_off_out;        // optional: offset for the next container
+  unsigned long long* out2;             // optional: {total bytes, status}
+  Scratch* sc;
+  unsigned long long* ts;               // scan words, one per tile
+  uint32_t epoch;
+  uint32_t spin_limit;
+};
+
+// Where the bytes of a salient / raw payload go: offsets below npay land in the plane's slot, the
+// rest in its overflow part.  Offsets and npay are multiples of the access size.
+struct SplitOut {
+  uint8_t* slot;
+  uint8_t* ovf;
+  uint32_t npay;
+  __device__ __forceinline__ uint8_t* at(uint32_t o) const { return o < npay ? slot + o : ovf + (o - npay); }
+  __device__ __forceinline__ void st32(uint32_t o, uint32_t v) const { *reinterpret_cast<uint32_t*>(at(o)) = v; }
+  __device__ __forceinline__ void st16(uint32_t o, uint32_t v) const { *reinterpret_cast<uint16_t*>(at(o)) = (uint16_t)v; }
+};
+
 // Residual codes of one dense 8x8 block (Eq. 7-9): first-order Lorenzo prediction on the
 // pre-quantised integers k, neighbours outside the block count as 0.  Returns the number of
-// verbatim elements.  WRITE: also emits the 64 code bytes and the verbatim values.
+// verbatim elements.  WRITE: also emits the 64 code bytes (at logical offset o_codes) and the
+// verbatim values (from logical offset o_outl).
 template <int DT, bool WRITE>
-__device__ __forceinline__ uint32_t block_codes(const uint8_t* plane, int H, int W, int by, int bx,
-                                                float inv2e, uint32_t* g_codes, uint8_t* g_outl) {
+__device__ __forceinline__ uint32_t block_codes(const uint8_t* plane, int H, int W, int by, int bx, float inv2e,
+                                                const SplitOut& out, uint32_t o_codes, uint32_t o_outl) {
   int32_t prev[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) prev[j] = 0;
@@ -56,10 +78,8 @@ __device__ __forceinline__ uint32_t block_codes(const uint8_t* plane, int H, int
       } else if (big || delta > 127 || delta < -127) {
         code = 0u;
         if (WRITE) {
-          if (DT == kF32)
-            reinterpret_cast<uint32_t*>(g_outl)[n_out] = reinterpret_cast<const uint32_t*>(plane)[idx];
-          else
-            reinterpret_cast<uint16_t*>(g_outl)[n_out] = reinterpret_cast<const uint16_t*>(plane)[idx];
+          if (DT == kF32) out.st32(o_outl + 4u * n_out, reinterpret_cast<const uint32_t*>(plane)[idx]);
+          else out.st16(o_outl + 2u * n_out, reinterpret_cast<const uint16_t*>(plane)[idx]);
         }
         ++n_out;
       } else {
@@ -72,8 +92,8 @@ __device__ __forceinline__ uint32_t block_codes(const uint8_t* plane, int H, int
       prev[j] = k;
     }
     if (WRITE) {
-      g_codes[2 * i] = w0;
-      g_codes[2 * i + 1] = w1;
+      out.st32(o_codes + 8u * i, w0);
+      out.st32(o_codes + 8u * i + 4u, w1);
     }
   }
   return n_out;
@@ -84,8 +104,11 @@ __device__ __forceinline__ uint32_t block_codes(const uint8_t* plane, int H, int
 // scratch: rowp[0..H] = CSR row pointers, blk_a[b] = 1 for dense blocks, blk_b[b] = rank of block b
 // among the dense blocks, blk_c[b] = index of the block's first verbatim value.
 template <int DT>
-__device__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint8_t* plane,
-                                       uint32_t* rowp, uint32_t* blk_a, uint32_t* blk_b, uint32_t* blk_c) {
+__device__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint8_t* plane, uint32_t* sal) {
+  uint32_t* rowp = sal;
+  uint32_t* blk_a = sal + pl.H + 1;
+  uint32_t* blk_b = blk_a + pl.nblk;
+  uint32_t* blk_c = blk_b + pl.nblk;
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx;
   for (uint32_t b = t.lane; b < nblk; b += t.size) blk_a[b] = 0;
@@ -115,20 +138,17 @@ __device__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint
     uint32_t cnt = 0;
     if (y < H) {
       const uint32_t* brow = blk_a + (uint32_t)(y >> 3) * nbx;
-      for (int x = 0; x < W; ++x)
-        cnt += (load_elem<DT>(plane, (uint32_t)y * W + x) != 0.0f) && !brow[x >> 3];
+      for (int x = 0; x < W; ++x) cnt += (load_elem<DT>(plane, (uint32_t)y * W + x) != 0.0f) && !brow[x >> 3];
     }
     rowp[y] = cnt;
   }
   team_sync(t);
   info.nnz_s = team_excl_scan(t, rowp, (uint32_t)H + 1u);
   // verbatim counts of dense blocks
-  const float two_eps = __fmul_rn(2.0f, pl.eps);
-  const float inv2e = __fdiv_rn(1.0f, two_eps);
+  const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
+  const SplitOut none = {nullptr, nullptr, 0};
   for (uint32_t b = t.lane; b < nblk; b += t.size)
-    blk_c[b] = blk_a[b] ? block_codes<DT, false>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e,
-                                                 nullptr, nullptr)
-                        : 0u;
+    blk_c[b] = blk_a[b] ? block_codes<DT, false>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, none, 0, 0) : 0u;
   team_sync(t);
   info.n_out_d = team_excl_scan(t, blk_c, nblk);
   const uint32_t e = (uint32_t)pl.esize;
@@ -137,97 +157,245 @@ __device__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint
   return info;
 }
 
-// Block-wise path, writing part; the scratch arrays are those salient_measure left.
+// Block-wise path, writing part; `sal` holds what salient_measure left.
 template <int DT>
 __device__ void salient_write(const Team& t, const Plan& pl, const uint8_t* plane, const SalientInfo& info,
-                              const uint32_t* rowp, const uint32_t* blk_a, const uint32_t* blk_b,
-                              const uint32_t* blk_c, uint8_t* g) {
+                              const uint32_t* sal, const SplitOut& out) {
+  const uint32_t* rowp = sal;
+  const uint32_t* blk_a = sal + pl.H + 1;
+  const uint32_t* blk_b = blk_a + pl.nblk;
+  const uint32_t* blk_c = blk_b + pl.nblk;
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx, e = (uint32_t)pl.esize;
-  uint32_t* g32 = reinterpret_cast<uint32_t*>(g);
-  uint32_t* g_bm = g32 + 4;
-  uint32_t* g_rp = g_bm + pl.nbm;
-  uint8_t* g_col = reinterpret_cast<uint8_t*>(g_rp + H + 1);
-  uint8_t* g_val = g_col + a4(2u * info.nnz_s);
-  uint8_t* g_codes = g_val + a4(e * info.nnz_s);
-  uint8_t* g_outl = g_codes + 64u * info.n_dense;
+  const uint32_t o_bm = 16u, o_rp = o_bm + 4u * pl.nbm, o_col = o_rp + 4u * ((uint32_t)H + 1u);
+  const uint32_t o_val = o_col + a4(2u * info.nnz_s), o_codes = o_val + a4(e * info.nnz_s);
+  const uint32_t o_outl = o_codes + 64u * info.n_dense;
   if (t.lane == 0) {
-    g32[0] = info.nnz_s; g32[1] = info.n_dense; g32[2] = info.n_out_d; g32[3] = 0;
-    // zero the pads the section writers leave: col (2 bytes), val / verbatim (bf16: 2 bytes), tail
-    if (info.nnz_s & 1u) reinterpret_cast<uint16_t*>(g_col)[info.nnz_s] = 0;
-    if (DT == kBF16 && (info.nnz_s & 1u)) reinterpret_cast<uint16_t*>(g_val)[info.nnz_s] = 0;
-    if (DT == kBF16 && (info.n_out_d & 1u)) reinterpret_cast<uint16_t*>(g_outl)[info.n_out_d] = 0;
-    for (uint32_t o = info.size; o < a16(info.size); o += 4) g32[o >> 2] = 0;
+    out.st32(0, info.nnz_s);
+    out.st32(4, info.n_dense);
+    out.st32(8, info.n_out_d);
+    out.st32(12, 0);
+    // pads the section writers leave: col (2 bytes), val / verbatim values (bf16: 2 bytes)
+    if (info.nnz_s & 1u) out.st16(o_col + 2u * info.nnz_s, 0);
+    if (DT == kBF16 && (info.nnz_s & 1u)) out.st16(o_val + 2u * info.nnz_s, 0);
+    if (DT == kBF16 && (info.n_out_d & 1u)) out.st16(o_outl + 2u * info.n_out_d, 0);
   }
+  // zero padding up to the end of the slot / of the 16-byte padded overflow part
+  const uint32_t end = max(pl.npay, a16(info.size));
+  for (uint32_t o = info.size + 4u * t.lane; o < end; o += 4u * t.size) out.st32(o, 0);
   for (uint32_t w = t.lane; w < pl.nbm; w += t.size) {
     uint32_t word = 0;
     const uint32_t hi = min(nblk, w * 32u + 32u);
     for (uint32_t b = w * 32u; b < hi; ++b) word |= blk_a[b] << (b & 31u);
-    g_bm[w] = word;
+    out.st32(o_bm + 4u * w, word);
   }
-  for (uint32_t y = t.lane; y <= (uint32_t)H; y += t.size) g_rp[y] = rowp[y];
+  for (uint32_t y = t.lane; y <= (uint32_t)H; y += t.size) out.st32(o_rp + 4u * y, rowp[y]);
   for (int y = (int)t.lane; y < H; y += (int)t.size) {
     uint32_t o = rowp[y];
     const uint32_t* brow = blk_a + (uint32_t)(y >> 3) * nbx;
     for (int x = 0; x < W; ++x) {
       const uint32_t idx = (uint32_t)y * W + x;
       if (load_elem<DT>(plane, idx) != 0.0f && !brow[x >> 3]) {
-        reinterpret_cast<uint16_t*>(g_col)[o] = (uint16_t)x;
-        if (DT == kF32)
-          reinterpret_cast<uint32_t*>(g_val)[o] = reinterpret_cast<const uint32_t*>(plane)[idx];
-        else
-          reinterpret_cast<uint16_t*>(g_val)[o] = reinterpret_cast<const uint16_t*>(plane)[idx];
+        out.st16(o_col + 2u * o, (uint32_t)x);
+        if (DT == kF32) out.st32(o_val + 4u * o, reinterpret_cast<const uint32_t*>(plane)[idx]);
+        else out.st16(o_val + 2u * o, reinterpret_cast<const uint16_t*>(plane)[idx]);
         ++o;
       }
     }
   }
-  const float two_eps = __fmul_rn(2.0f, pl.eps);
-  const float inv2e = __fdiv_rn(1.0f, two_eps);
+  const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
   for (uint32_t b = t.lane; b < nblk; b += t.size)
     if (blk_a[b])
-      block_codes<DT, true>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e,
-                            reinterpret_cast<uint32_t*>(g_codes + 64u * blk_b[b]), g_outl + e * blk_c[b]);
+      block_codes<DT, true>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, out, o_codes + 64u * blk_b[b],
+                            o_outl + e * blk_c[b]);
 }
 
-struct CompressArgs {
-  const uint8_t* src;
-  uint8_t* dst_base;
-  unsigned long long capacity;                 // bytes available at dst_base (+ offset below)
-  const unsigned long long* d_off_in;          // optional: byte offset of the container in dst_base
-  unsigned long long* d_off_out;               // optional: offset for the next container
-  unsigned long long* out2;                    // optional: {total bytes, status}
-  Scratch* sc;
-  TileState* ts;
-  uint32_t epoch;
-  unsigned long long ticket_base, done_base;
-  uint32_t spin_limit;
+// Raw plane: verbatim copy through the slot into the overflow part, zero padded.
+__device__ __forceinline__ void raw_write(const Team& t, const Plan& pl, const uint8_t* plane, const SplitOut& out) {
+  const uint32_t n = (uint32_t)pl.plane_bytes, end = max(pl.npay, a16(n));
+  for (uint32_t o = 2u * t.lane; o < end; o += 2u * t.size)
+    out.st16(o, o < n ? (uint32_t)*reinterpret_cast<const uint16_t*>(plane + o) : 0u);
+}
+
+// Per-plane record kept in shared memory while a tile is processed.
+struct Rec {
+  float lo, scale;
+  uint32_t meta;  // class | n_out << 2
+  uint32_t size;  // payload bytes of a salient / raw plane (before padding)
 };
 
+// What every thread of a CTA knows about the destination.
+struct Dest {
+  uint8_t* dst;
+  unsigned long long capacity, off_in;
+  bool fits;  // header, table and slots fit the capacity
+};
+__device__ __forceinline__ Dest make_dest(const Plan& pl, const CompressArgs& a) {
+  Dest d;
+  d.off_in = a.d_off_in ? *a.d_off_in : 0ull;
+  d.dst = a.dst_base + d.off_in;
+  d.capacity = a.capacity > d.off_in ? a.capacity - d.off_in : 0ull;
+  d.fits = d.capacity >= pl.ovf_off;
+  return d;
+}
+
+// Tile-level placement, executed by warp 0 after the classes and sizes of the tile's planes are in
+// rec[].  Computes each plane's overflow offset (roff[], 16-byte units relative to the tile),
+// publishes the tile's aggregate and, when the tile needs it or is a 32nd tile, resolves the tile's
+// base.  Returns through shared variables: *s_base16 (absolute, 16-byte units), *s_skip.
+__device__ __forceinline__ void tile_place(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
+                                           uint32_t np, const Rec* rec, uint32_t* roff,
+                                           unsigned long long* s_base16, uint32_t* s_skip) {
+  const uint32_t lane = threadIdx.x & 31u;
+  uint32_t carry = 0, nsal = 0, nraw = 0;
+  for (uint32_t base = 0; base < np; base += 32) {
+    const uint32_t i = base + lane;
+    uint32_t v = 0, c = 0;
+    if (i < np) {
+      c = rec[i].meta & 3u;
+      if (c != kClsNormal && a16(rec[i].size) > pl.npay) v = (a16(rec[i].size) - pl.npay) >> 4;
+    }
+    uint32_t incl = v;
+    for (uint32_t o = 1; o < 32; o <<= 1) {
+      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    if (i < np) roff[i] = carry + incl - v;
+    carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    nsal += __popc(__ballot_sync(0xFFFFFFFFu, c == kClsSalient));
+    nraw += __popc(__ballot_sync(0xFFFFFFFFu, c == kClsRaw));
+  }
+  unsigned long long excl = 0;
+  uint32_t skip = d.fits ? 0u : 1u;
+  if (pl.mode != kModeOff) {
+    const bool resolve = carry > 0 || (tile & 31u) == 31u;
+    if (tile == 0) {
+      scan_publish(a.ts, tile, a.epoch, 2u, carry);
+    } else {
+      scan_publish(a.ts, tile, a.epoch, 1u, carry);
+      if (resolve) {
+        if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
+          if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+          skip = 1;
+        }
+        scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)(excl + carry));
+      }
+    }
+    if (lane == 0) {
+      if (carry) atomicAdd(&a.sc->ovf16, (unsigned long long)carry);
+      if (nsal) atomicAdd(&a.sc->nsal, (unsigned long long)nsal);
+      if (nraw) atomicAdd(&a.sc->nraw, (unsigned long long)nraw);
+    }
+  }
+  if (lane == 0) {
+    const unsigned long long base16 = (pl.ovf_off >> 4) + excl;
+    if ((base16 + carry) * 16ull > d.capacity) skip = 1;  // never write past the capacity
+    *s_base16 = base16;
+    *s_skip = skip;
+  }
+}
+
+// Last step of every CTA: count the exit; the last CTA to leave writes the header and the result
+// words and returns the scratch counters to zero for the next call.
+__device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, const Dest& d) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x != 0) return;
+  const unsigned long long prev = atomicAdd(&a.sc->exited, 1ull);
+  if (prev != (unsigned long long)gridDim.x - 1ull) return;
+  __threadfence();
+  const unsigned long long ovf16 = ld_relaxed(&a.sc->ovf16);
+  const unsigned long long nsal = ld_relaxed(&a.sc->nsal), nraw = ld_relaxed(&a.sc->nraw);
+  uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
+  const unsigned long long total = pl.ovf_off + ovf16 * 16ull;
+  if (total > d.capacity && code < kErrCapacity) code = kErrCapacity;
+  if (d.capacity >= 64) {
+    uint32_t h[16];
+    h[0] = code == kErrNone ? kMagic : 0u;  // a failed container must not pass for a valid one
+    h[1] = 1u | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24);
+    h[2] = pl.N;
+    h[3] = pl.C;
+    h[4] = (uint32_t)pl.H;
+    h[5] = (uint32_t)pl.W;
+    h[6] = 8u | (8u << 8) | (0u << 16) | ((uint32_t)pl.mode << 24);
+    h[7] = pl.rho_num | (pl.rho_den << 16);
+    h[8] = pl.tau_num | (pl.tau_den << 16);
+    h[9] = __float_as_uint(pl.eps);
+    h[10] = (uint32_t)nsal;
+    h[11] = (uint32_t)nraw;
+    h[12] = (uint32_t)pl.tensor_id;
+    h[13] = (uint32_t)(pl.tensor_id >> 32);
+    h[14] = (uint32_t)total;
+    h[15] = (uint32_t)(total >> 32);
+    uint32_t* hd = reinterpret_cast<uint32_t*>(d.dst);
+    for (int k = 0; k < 16; ++k) hd[k] = h[k];
+  }
+  if (a.out2) {
+    a.out2[0] = total;
+    a.out2[1] = status_word(code);
+  }
+  if (a.d_off_out) *a.d_off_out = code == kErrNone ? d.off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
+  st_relaxed(&a.sc->ticket, 0ull);
+  st_relaxed(&a.sc->status, 0ull);
+  st_relaxed(&a.sc->ovf16, 0ull);
+  st_relaxed(&a.sc->nsal, 0ull);
+  st_relaxed(&a.sc->nraw, 0ull);
+  st_relaxed(&a.sc->exited, 0ull);
+}
+
+__device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane, uint32_t off16, const Rec& r) {
+  uint4 e;
+  e.x = off16;
+  e.y = r.meta;
+  e.z = __float_as_uint(r.lo);
+  e.w = __float_as_uint(r.scale);
+  reinterpret_cast<uint4*>(d.dst + 64)[plane] = e;
+}
+
+// Writes a salient or raw plane whose record and overflow offset (absolute, 16-byte units) are known.
+template <int DT>
+__device__ __forceinline__ void write_nonnormal(const Team& t, const Plan& pl, const Dest& d, const uint8_t* plane,
+                                                uint64_t gp, const Rec& r, unsigned long long off16, uint32_t* sal) {
+  SplitOut out;
+  out.slot = d.dst + pl.slots_off + gp * pl.npay;
+  out.ovf = d.dst + off16 * 16ull;
+  out.npay = pl.npay;
+  const bool has_ovf = a16(r.size) > pl.npay;
+  if ((r.meta & 3u) == kClsRaw) {
+    raw_write(t, pl, plane, out);
+  } else {
+    const SalientInfo info = salient_measure<DT>(t, pl, plane, sal);
+    salient_write<DT>(t, pl, plane, info, sal, out);
+  }
+  if (t.lane == 0) store_table_entry(d, gp, has_ovf ? (uint32_t)off16 : 0u, r);
+}
+
+// =================================================================================================
+// Generic kernel
+// =================================================================================================
 template <int DT, int BITS>
-__global__ void __launch_bounds__(kThreads) compress_kernel(const Plan pl, const CompressArgs a) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  __shared__ double s_red[kThreads / 32 * 4 + 8];
-  __shared__ uint32_t s_tile;
-  __shared__ unsigned long long s_base16, s_cnt_excl;
-  __shared__ uint32_t s_tile16, s_tile_nsal, s_tile_nraw, s_skip;
+__global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, const CompressArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ double s_red[kWarps * 4];
+  __shared__ uint32_t s_tile, s_skip;
+  __shared__ unsigned long long s_base16;
 
   const uint32_t tid = threadIdx.x;
   uint8_t* tile_buf = smem + pl.sm_tile;
   uint8_t* out_buf = smem + pl.sm_out;
   Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
   uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + 16u * pl.ppt);
-  const unsigned long long off_in = a.d_off_in ? *a.d_off_in : 0ull;
-  uint8_t* dst = a.dst_base + off_in;
-  const unsigned long long capacity = a.capacity > off_in ? a.capacity - off_in : 0ull;
-  const unsigned long long epoch_hi = (unsigned long long)a.epoch << 32;
-  const unsigned long long table_end = 64ull + 16ull * pl.P;
+  const Dest d = make_dest(pl, a);
   const Team team = make_team(pl.team, s_red);
   const uint32_t nteams = team.block ? 1u : kThreads / team.size;
   const uint32_t my_team = team.block ? 0u : tid / team.size;
+  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
   constexpr uint32_t L = (1u << BITS) - 1u;
+  const bool need_sigma = pl.mode == kModeAuto;
+  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
 
   for (;;) {
-    if (tid == 0) s_tile = (uint32_t)(atomicAdd(&a.sc->ticket, 1ull) - a.ticket_base);
+    if (tid == 0) s_tile = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
     __syncthreads();
     const uint32_t tile = s_tile;
     if (tile >= pl.ntiles) break;
@@ -251,56 +419,40 @@ __global__ void __launch_bounds__(kThreads) compress_kernel(const Plan pl, const
     // ---- phase A: per-plane statistics, class, codes / sizes
     for (uint32_t lp = my_team; lp < np; lp += nteams) {
       const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
-      const bool vec = ((uint32_t)__cvta_generic_to_shared(plane) & (DT == kF32 ? 15u : 7u)) == 0u;
+      const bool vec = (smem_u32(plane) & (DT == kF32 ? 15u : 7u)) == 0u;
       const uint32_t HW = pl.HW, nfull = HW >> 2, groups = pl.groups;
-      Stats s;
-      s.lo = __int_as_float(0x7F800000);
-      s.hi = __int_as_float(0xFF800000);
-      s.S = 0.0;
-      s.Q = 0.0;
-      const bool need_sigma = pl.mode == kModeAuto;
+      float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
       for (uint32_t g = team.lane; g < nfull; g += team.size) {
         float v[4];
         load_group<DT>(plane, g, HW, vec, v);
-        s.lo = min_nan(s.lo, min_nan(min_nan(v[0], v[1]), min_nan(v[2], v[3])));
-        s.hi = max_nan(s.hi, max_nan(max_nan(v[0], v[1]), max_nan(v[2], v[3])));
-        if (need_sigma) {
-          const float sg = __fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3]));
-          const float q01 = __fmaf_rn(v[1], v[1], __fmul_rn(v[0], v[0]));
-          const float q23 = __fmaf_rn(v[3], v[3], __fmul_rn(v[2], v[2]));
-          s.S += (double)sg;
-          s.Q += (double)__fadd_rn(q01, q23);
+        lo = min3_nan(lo, min_nan(v[0], v[1]), min_nan(v[2], v[3]));
+        hi = max3_nan(hi, max_nan(v[0], v[1]), max_nan(v[2], v[3]));
+      }
+      if ((HW & 3u) && team.lane == 0) {  // ragged last group
+        for (uint32_t i = nfull * 4u; i < HW; ++i) {
+          const float x = load_elem<DT>(plane, i);
+          lo = min_nan(lo, x);
+          hi = max_nan(hi, x);
         }
       }
-      if ((HW & 3u) && team.lane == 0) {  // ragged last group: zero padded for the sums only
-        float v[4];
-        load_group<DT>(plane, nfull, HW, false, v);
-        for (uint32_t k = 0; k < (HW & 3u); ++k) {
-          s.lo = min_nan(s.lo, v[k]);
-          s.hi = max_nan(s.hi, v[k]);
-        }
-        if (need_sigma) {
-          const float sg = __fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3]));
-          const float q01 = __fmaf_rn(v[1], v[1], __fmul_rn(v[0], v[0]));
-          const float q23 = __fmaf_rn(v[3], v[3], __fmul_rn(v[2], v[2]));
-          s.S += (double)sg;
-          s.Q += (double)__fadd_rn(q01, q23);
-        }
-      }
-      s = team_reduce_stats(team, s);
-      const float range = __fsub_rn(s.hi, s.lo);
-      if (!(fabsf(range) <= 3.402823466e38f) && team.lane == 0)
-        atomicMax(&a.sc->status, epoch_hi | kErrNonfinite);
+      team_minmax(team, lo, hi);
+      if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && team.lane == 0)
+        atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
 
       uint32_t cls = kClsNormal, n_out = 0;
       if (need_sigma) {
-        const double hw = (double)HW;
-        const double mu = __ddiv_rn(s.S, hw);
-        double var = __dsub_rn(__ddiv_rn(s.Q, hw), __dmul_rn(mu, mu));
-        if (!(var > 0.0)) var = 0.0;
-        const double three = __dmul_rn(3.0, __dsqrt_rn(var));
-        const float thi = __double2float_rn(__dadd_rn(mu, three));
-        const float tlo = __double2float_rn(__dsub_rn(mu, three));
+        const SigmaScale sc = sigma_scale(lo, hi);
+        uint32_t as = 0, aq = 0, ng = 0;
+        for (uint32_t g = team.lane; g < groups; g += team.size) {
+          float v[4];
+          load_group<DT>(plane, g, HW, vec, v);
+          sigma_addends(v, sc, as, aq);
+          ++ng;
+        }
+        long long Is, Iq;
+        team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq);
+        float tlo, thi;
+        sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
         uint32_t cnt = 0;
         for (uint32_t g = team.lane; g < groups; g += team.size) {
           float v[4];
@@ -315,27 +467,22 @@ __global__ void __launch_bounds__(kThreads) compress_kernel(const Plan pl, const
         cls = kClsSalient;
       }
 
-      float lo_out = 0.0f, scale_out = 0.0f;
-      uint32_t size = 0;
+      Rec r;
+      r.lo = 0.0f;
+      r.scale = 0.0f;
+      r.size = 0;
       if (cls == kClsSalient) {
-        uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
-        const SalientInfo info =
-            salient_measure<DT>(team, pl, plane, sal, sal + pl.H + 1, sal + pl.H + 1 + pl.nblk,
-                                sal + pl.H + 1 + 2 * pl.nblk);
-        size = info.size;
-        if (a16(size) >= a16((uint32_t)pl.plane_bytes)) {
+        const SalientInfo info = salient_measure<DT>(team, pl, plane, sal);
+        r.size = info.size;
+        if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
           cls = kClsRaw;
-          size = (uint32_t)pl.plane_bytes;
+          r.size = (uint32_t)pl.plane_bytes;
         }
       } else {
-        float inv = __fdiv_rn((float)L, range), scale = __fdiv_rn(range, (float)L);
-        if (range == 0.0f || !(fabsf(inv) <= 3.402823466e38f)) {
-          inv = 0.0f;
-          scale = 0.0f;
-        }
-        lo_out = s.lo;
-        scale_out = scale;
-        size = pl.npay;
+        float inv, scale;
+        quant_params(lo, hi, L, inv, scale);
+        r.lo = lo;
+        r.scale = scale;
         uint8_t* o = out_buf + (uint64_t)lp * pl.npay;
         const uint32_t ogroups = pl.npay * 2u / BITS;
         for (uint32_t g = team.lane; g < ogroups; g += team.size) {
@@ -345,9 +492,7 @@ __global__ void __launch_bounds__(kThreads) compress_kernel(const Plan pl, const
             load_group<DT>(plane, g, HW, vec, v);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              const float d = __fsub_rn(v[k], s.lo);
-              const float r = __fmaf_rn(d, inv, 12582912.0f);  // exact product, rne to an integer
-              uint32_t q = (__float_as_uint(r) - 0x4B400000u) & L;
+              uint32_t q = quant_code(v[k], lo, inv, L);
               if (g * 4u + k >= HW) q = 0;
               word |= q << (k * BITS);
             }
@@ -357,176 +502,281 @@ __global__ void __launch_bounds__(kThreads) compress_kernel(const Plan pl, const
           else reinterpret_cast<uint32_t*>(o)[g] = word;
         }
       }
-      if (team.lane == 0) {
-        Rec r;
-        r.lo = lo_out;
-        r.scale = scale_out;
-        r.meta = cls | (n_out << 2);
-        r.size16 = a16(size) >> 4;
-        rec[lp] = r;
-      }
+      r.meta = cls | (n_out << 2);
+      if (team.lane == 0) rec[lp] = r;
     }
     __syncthreads();
 
-    // ---- phase B: offsets inside the tile, then the tile's offset in the container
-    if (tid < 32) {
-      uint32_t carry = 0, nsal = 0, nraw = 0;
-      for (uint32_t base = 0; base < np; base += 32) {
-        const uint32_t i = base + tid;
-        const uint32_t v = i < np ? rec[i].size16 : 0u;
-        const uint32_t c = i < np ? (rec[i].meta & 3u) : 0u;
-        uint32_t incl = v;
-        for (uint32_t o = 1; o < 32; o <<= 1) {
-          const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-          if (tid >= o) incl += up;
-        }
-        if (i < np) roff[i] = carry + incl - v;
-        carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
-        nsal += __popc(__ballot_sync(0xFFFFFFFFu, c == kClsSalient));
-        nraw += __popc(__ballot_sync(0xFFFFFFFFu, c == kClsRaw));
-      }
-      if (tid == 0) {
-        unsigned long long excl = 0, cnt_excl = 0;
-        uint32_t skip = 0;
-        const unsigned long long my_b = ((unsigned long long)nsal << 32) | nraw;
-        if (pl.mode == kModeOff) {
-          excl = (unsigned long long)tile * pl.ppt * (pl.npay >> 4);
-        } else {
-          TileState* me = a.ts + tile;
-          if (tile > 0) {
-            st_relaxed(&me->agg_b, my_b);
-            st_release(&me->agg_a, epoch_hi | carry);
-            long long j = (long long)tile - 1;
-            uint32_t spins = 0;
-            while (j >= 0) {
-              const TileState* pr = a.ts + j;
-              const unsigned long long ia = ld_acquire(&pr->inc_a);
-              if ((ia >> 32) == a.epoch) {
-                excl += (uint32_t)ia;
-                cnt_excl += ld_relaxed(&pr->inc_b);
-                break;
-              }
-              const unsigned long long aa = ld_acquire(&pr->agg_a);
-              if ((aa >> 32) == a.epoch) {
-                excl += (uint32_t)aa;
-                cnt_excl += ld_relaxed(&pr->agg_b);
-                --j;
-                continue;
-              }
-              if (++spins > a.spin_limit) {  // the predecessor never published: give up cleanly
-                atomicMax(&a.sc->status, epoch_hi | kErrTimeout);
-                skip = 1;
-                break;
-              }
-              __nanosleep(64);
-            }
-          }
-          st_relaxed(&me->inc_b, cnt_excl + my_b);
-          st_release(&me->inc_a, epoch_hi | (uint32_t)(excl + carry));
-        }
-        s_base16 = (table_end >> 4) + excl;
-        s_cnt_excl = cnt_excl;
-        s_tile16 = carry;
-        s_tile_nsal = nsal;
-        s_tile_nraw = nraw;
-        // never write past the capacity
-        if (((table_end >> 4) + excl + carry) * 16ull > capacity) skip = 1;
-        if (64ull + 16ull * (p0 + np) > capacity) skip = 1;
-        s_skip = skip;
-      }
-    }
+    // ---- phase B: placement of the overflow parts
+    if (tid < 32) tile_place(pl, a, d, tile, np, rec, roff, &s_base16, &s_skip);
     __syncthreads();
 
     // ---- phase C: table entries and payloads
     if (!s_skip) {
       const unsigned long long base16 = s_base16;
-      uint4* table = reinterpret_cast<uint4*>(dst + 64) + p0;
-      for (uint32_t i = tid; i < np; i += kThreads) {
-        const Rec r = rec[i];
-        uint4 e;
-        e.x = (uint32_t)(base16 + roff[i]);
-        e.y = r.meta;
-        e.z = __float_as_uint(r.lo);
-        e.w = __float_as_uint(r.scale);
-        table[i] = e;
-      }
-      // normal payloads: straight 16-byte copies out of the staging buffer
       const uint32_t chunks = pl.npay >> 4;
+      uint4* slots = reinterpret_cast<uint4*>(d.dst + pl.slots_off + p0 * pl.npay);
       for (uint32_t i = tid; i < np * chunks; i += kThreads) {
-        const uint32_t lp = i / chunks, c = i - lp * chunks;
-        if ((rec[lp].meta & 3u) == kClsNormal)
-          reinterpret_cast<uint4*>(dst + (base16 + roff[lp]) * 16ull)[c] =
-              reinterpret_cast<const uint4*>(out_buf + (uint64_t)lp * pl.npay)[c];
+        const uint32_t lp = i / chunks;
+        if ((rec[lp].meta & 3u) == kClsNormal) slots[i] = reinterpret_cast<const uint4*>(out_buf)[i];
       }
-      if (s_tile_nsal + s_tile_nraw) {
-        for (uint32_t lp = my_team; lp < np; lp += nteams) {
-          const uint32_t cls = rec[lp].meta & 3u;
-          if (cls == kClsNormal) continue;
-          const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
-          uint8_t* g = dst + (base16 + roff[lp]) * 16ull;
-          if (cls == kClsRaw) {
-            const uint32_t n = (uint32_t)pl.plane_bytes >> 1;  // copy as 16-bit units
-            for (uint32_t i = team.lane; i < (a16((uint32_t)pl.plane_bytes) >> 1); i += team.size)
-              reinterpret_cast<uint16_t*>(g)[i] = i < n ? reinterpret_cast<const uint16_t*>(plane)[i] : (uint16_t)0;
+      for (uint32_t i = tid; i < np; i += kThreads)
+        if ((rec[i].meta & 3u) == kClsNormal)
+          store_table_entry(d, p0 + i, (uint32_t)((pl.slots_off + (p0 + i) * pl.npay) >> 4), rec[i]);
+      for (uint32_t lp = my_team; lp < np; lp += nteams) {
+        if ((rec[lp].meta & 3u) == kClsNormal) continue;
+        const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
+        write_nonnormal<DT>(team, pl, d, plane, p0 + lp, rec[lp], base16 + roff[lp], sal);
+      }
+    }
+    __syncthreads();
+  }
+  cta_exit(pl, a, d);
+}
+
+// =================================================================================================
+// Fast kernel
+// =================================================================================================
+// One plane per team and tile.  Warp-team variant (CTA = false): ppt = kThreads / team planes per
+// tile, each handled by `team` lanes of a warp.  CTA-team variant: one plane per tile, handled by
+// all threads.  Thread t of a team owns groups t, t + team, ..., (G of them), kept in registers.
+template <int DT, int G>
+struct Groups {
+  float v[G][4];
+};
+
+template <int DT, bool SIGMA, int G, bool CTA>
+__global__ void __launch_bounds__(kThreads) compress_fast(const Plan pl, const CompressArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ double s_red[kWarps * 4];
+  __shared__ __align__(8) uint64_t s_full[kMaxStages];
+  __shared__ uint32_t s_tiles[kMaxStages];
+  __shared__ uint32_t s_nonnormal, s_skip, s_abort;
+  __shared__ unsigned long long s_base16;
+
+  const uint32_t tid = threadIdx.x;
+  Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
+  uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + 16u * pl.ppt);
+  const Dest d = make_dest(pl, a);
+  const Team team = make_team(pl.team, s_red);
+  const uint32_t T = CTA ? (uint32_t)kThreads : pl.team;
+  const uint32_t my_team = CTA ? 0u : tid / T;
+  const uint32_t groups = pl.groups, bits = (uint32_t)pl.bits, L = (1u << bits) - 1u;
+  const uint32_t nstage = pl.nstage;
+  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+
+  // ---- pipeline prologue: barriers, first tiles in flight
+  if (tid == 0) {
+    for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
+    fence_mbar_init();
+    s_nonnormal = 0;
+    s_abort = 0;
+  }
+  __syncthreads();
+  auto issue = [&](uint32_t s) {  // thread 0: take a ticket and start its load into stage s
+    const uint32_t t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+    s_tiles[s] = t;
+    if (t < pl.ntiles) {
+      const uint64_t p0 = (uint64_t)t * pl.ppt;
+      const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+      const uint32_t bytes = np * (uint32_t)pl.plane_bytes;
+      fence_proxy_async();
+      mbar_expect_tx(&s_full[s], bytes);
+      bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + p0 * pl.plane_bytes, bytes, &s_full[s]);
+    }
+  };
+  if (tid == 0)
+    for (uint32_t s = 0; s < nstage; ++s) issue(s);
+  __syncthreads();
+
+  for (uint32_t it = 0;; ++it) {
+    const uint32_t s = it % nstage;
+    const uint32_t tile = s_tiles[s];
+    if (tile >= pl.ntiles) break;
+    const uint32_t parity = (it / nstage) & 1u;
+    if (!mbar_wait(&s_full[s], parity, 1u << 22)) s_abort = 1;  // the load never arrived
+    __syncthreads();
+    if (s_abort) break;
+    const uint64_t p0 = (uint64_t)tile * pl.ppt;
+    const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+    const uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+
+    if (CTA || my_team < np) {
+      const uint32_t lp = my_team;
+      const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
+      const uint64_t gp = p0 + lp;
+      // ---- the thread's groups, in registers for every pass
+      Groups<DT, G> x;
+      float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
+      uint32_t ng = 0;
+#pragma unroll
+      for (int k = 0; k < G; ++k) {
+        const uint32_t g = team.lane + (uint32_t)k * T;
+        if (g < groups) {
+          if (DT == kF32) {
+            const float4 t4 = reinterpret_cast<const float4*>(plane)[g];
+            x.v[k][0] = t4.x; x.v[k][1] = t4.y; x.v[k][2] = t4.z; x.v[k][3] = t4.w;
           } else {
-            uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
-            uint32_t* rowp = sal;
-            uint32_t* blk_a = sal + pl.H + 1;
-            uint32_t* blk_b = blk_a + pl.nblk;
-            uint32_t* blk_c = blk_b + pl.nblk;
-            const SalientInfo info = salient_measure<DT>(team, pl, plane, rowp, blk_a, blk_b, blk_c);
-            salient_write<DT>(team, pl, plane, info, rowp, blk_a, blk_b, blk_c, g);
+            const uint2 t2 = reinterpret_cast<const uint2*>(plane)[g];
+            x.v[k][0] = __uint_as_float(t2.x << 16); x.v[k][1] = __uint_as_float(t2.x & 0xFFFF0000u);
+            x.v[k][2] = __uint_as_float(t2.y << 16); x.v[k][3] = __uint_as_float(t2.y & 0xFFFF0000u);
+          }
+          lo = min3_nan(lo, x.v[k][0], x.v[k][1]);
+          lo = min3_nan(lo, x.v[k][2], x.v[k][3]);
+          hi = max3_nan(hi, x.v[k][0], x.v[k][1]);
+          hi = max3_nan(hi, x.v[k][2], x.v[k][3]);
+          ++ng;
+        }
+      }
+      team_minmax(team, lo, hi);
+      if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && team.lane == 0)
+        atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+
+      uint32_t cls = kClsNormal, n_out = 0;
+      if (SIGMA) {
+        const SigmaScale sc = sigma_scale(lo, hi);
+        uint32_t as = 0, aq = 0;
+#pragma unroll
+        for (int k = 0; k < G; ++k)
+          if (team.lane + (uint32_t)k * T < groups) sigma_addends(x.v[k], sc, as, aq);
+        long long Is, Iq;
+        team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq);
+        float tlo, thi;
+        sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
+        uint32_t cnt = 0;
+        if (hi > thi || lo < tlo) {  // otherwise no element can lie outside: the count is zero
+          if (lo >= tlo) {           // nothing below: one compare per element
+#pragma unroll
+            for (int k = 0; k < G; ++k)
+              if (team.lane + (uint32_t)k * T < groups) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) cnt += x.v[k][e] > thi;
+              }
+          } else {
+#pragma unroll
+            for (int k = 0; k < G; ++k)
+              if (team.lane + (uint32_t)k * T < groups) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) cnt += (x.v[k][e] > thi) || (x.v[k][e] < tlo);
+              }
+          }
+          cnt = team_sum_u32(team, cnt);
+        }
+        n_out = cnt;
+        if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
+      } else if (pl.mode == kModeAll) {
+        cls = kClsSalient;
+      }
+
+      Rec r;
+      r.lo = 0.0f;
+      r.scale = 0.0f;
+      r.size = 0;
+      r.meta = cls | (n_out << 2);
+      if (cls == kClsNormal) {
+        float inv, scale;
+        quant_params(lo, hi, L, inv, scale);
+        r.lo = lo;
+        r.scale = scale;
+        if (d.fits) {
+          uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
+#pragma unroll
+          for (int k = 0; k < G; ++k) {
+            const uint32_t g = team.lane + (uint32_t)k * T;
+            if (g < groups) {
+              uint32_t word = 0;
+#pragma unroll
+              for (int e = 0; e < 4; ++e) word |= quant_code(x.v[k][e], lo, inv, L) << (e * bits);
+              if (bits == 2u) slot[g] = (uint8_t)word;
+              else if (bits == 4u) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;
+              else reinterpret_cast<uint32_t*>(slot)[g] = word;
+            }
+          }
+          // zero padding of the slot behind the codes
+          const uint32_t code_bytes = groups * bits / 2u;
+          if (code_bytes < pl.npay) {
+            for (uint32_t o = code_bytes + team.lane; o < a4(code_bytes); o += T) slot[o] = 0;
+            for (uint32_t o = a4(code_bytes) + 4u * team.lane; o < pl.npay; o += 4u * T)
+              *reinterpret_cast<uint32_t*>(slot + o) = 0u;
+          }
+          if (team.lane == 0) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
+        }
+      } else if (team.lane == 0) {
+        atomicAdd(&s_nonnormal, 1u);
+      }
+      if (team.lane == 0) rec[lp] = r;
+    }
+    __syncthreads();
+
+    const uint32_t nonnormal = s_nonnormal;
+    if (nonnormal == 0) {
+      // ---- common case: nothing to place; publish a zero aggregate, every 32nd tile resolves
+      if (pl.mode != kModeOff && tid < 32) {
+        if (tile == 0) {
+          scan_publish(a.ts, tile, a.epoch, 2u, 0u);
+        } else {
+          scan_publish(a.ts, tile, a.epoch, 1u, 0u);
+          if ((tile & 31u) == 31u) {
+            unsigned long long excl = 0;
+            if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
+              if (tid == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+            }
+            scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)excl);
           }
         }
       }
-    }
-    // the tile holding the last planes knows the totals: header
-    if (tile == pl.ntiles - 1 && tid == 0) {
-      const unsigned long long total = (s_base16 + s_tile16) * 16ull;
-      st_relaxed(&a.sc->total, total);
-      if (total > capacity) atomicMax(&a.sc->status, epoch_hi | kErrCapacity);
-      if (!s_skip && capacity >= 64) {
-        const unsigned long long cnt = s_cnt_excl + (((unsigned long long)s_tile_nsal << 32) | s_tile_nraw);
-        uint32_t h[16];
-        h[0] = kMagic;
-        h[1] = 1u | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24);
-        h[2] = pl.N;
-        h[3] = pl.C;
-        h[4] = (uint32_t)pl.H;
-        h[5] = (uint32_t)pl.W;
-        h[6] = 8u | (8u << 8) | (0u << 16) | ((uint32_t)pl.mode << 24);
-        h[7] = pl.rho_num | (pl.rho_den << 16);
-        h[8] = pl.tau_num | (pl.tau_den << 16);
-        h[9] = __float_as_uint(pl.eps);
-        h[10] = (uint32_t)(cnt >> 32);
-        h[11] = (uint32_t)cnt;
-        h[12] = (uint32_t)pl.tensor_id;
-        h[13] = (uint32_t)(pl.tensor_id >> 32);
-        h[14] = (uint32_t)total;
-        h[15] = (uint32_t)(total >> 32);
-        uint32_t* hd = reinterpret_cast<uint32_t*>(dst);
-        for (int k = 0; k < 16; ++k) hd[k] = h[k];
-      }
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-      const unsigned long long prev = atomicAdd(&a.sc->done, 1ull) - a.done_base;
-      if (prev == (unsigned long long)pl.ntiles - 1ull) {  // every tile has finished
-        __threadfence();
-        const unsigned long long total = ld_relaxed(&a.sc->total);
-        const unsigned long long st = ld_relaxed(&a.sc->status);
-        const uint32_t code = (st >> 32) == a.epoch ? (uint32_t)st : kErrNone;
-        if (a.out2) {
-          a.out2[0] = total;
-          a.out2[1] = status_word(code);
+    } else {
+      // ---- block-wise path for the salient planes of this tile (shared-memory resident)
+      const Team wteam = CTA ? team : make_warp_team(s_red);
+      const uint32_t nw = CTA ? 1u : (uint32_t)kWarps, me = CTA ? 0u : tid >> 5;
+      uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)me * pl.sm_sal_stride);
+      uint32_t seen = 0;
+      for (uint32_t lp = 0; lp < np; ++lp) {
+        if ((rec[lp].meta & 3u) == kClsNormal) continue;
+        if (seen++ % nw != me) continue;
+        const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
+        const SalientInfo info = salient_measure<DT>(wteam, pl, plane, sal);
+        if (wteam.lane == 0) {
+          if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
+            rec[lp].meta = (rec[lp].meta & ~3u) | kClsRaw;
+            rec[lp].size = (uint32_t)pl.plane_bytes;
+          } else {
+            rec[lp].size = info.size;
+          }
         }
-        // a failed container must not be mistaken for a valid one, and nothing may follow it
-        if (code != kErrNone && capacity >= 4) *reinterpret_cast<uint32_t*>(dst) = 0u;
-        if (a.d_off_out) *a.d_off_out = code == kErrNone ? off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
       }
+      __syncthreads();
+      if (tid < 32) tile_place(pl, a, d, tile, np, rec, roff, &s_base16, &s_skip);
+      __syncthreads();
+      if (!s_skip) {
+        const unsigned long long base16 = s_base16;
+        seen = 0;
+        for (uint32_t lp = 0; lp < np; ++lp) {
+          if ((rec[lp].meta & 3u) == kClsNormal) continue;
+          if (seen++ % nw != me) continue;
+          const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
+          write_nonnormal<DT>(wteam, pl, d, plane, p0 + lp, rec[lp], base16 + roff[lp], sal);
+        }
+      }
+      __syncthreads();
+      if (tid == 0) s_nonnormal = 0;
+    }
+    // ---- the stage is free: next ticket, next load
+    if (tid == 0) issue(s);
+    __syncthreads();
+  }
+
+  if (s_abort) {  // a load timed out: report, then wait (bounded) for the copies still in flight
+    if (tid == 0) {
+      atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+      for (uint32_t s = 0; s < nstage; ++s)
+        if (s_tiles[s] < pl.ntiles) {
+          mbar_wait(&s_full[s], 0u, 1u << 16);
+          mbar_wait(&s_full[s], 1u, 1u << 16);
+        }
     }
   }
+  cta_exit(pl, a, d);
 }
 
 }  // namespace fh

@@ -18,8 +18,17 @@ struct DecompressArgs {
   uint8_t* dst;
   unsigned long long* d_status;        // optional
   Scratch* sc;
-  uint32_t epoch;
-  unsigned long long ticket_base, done_base;
+};
+
+// Reads of a salient / raw payload: offsets below npay come from the plane's slot, the rest from its
+// overflow part.
+struct SplitIn {
+  const uint8_t* slot;
+  const uint8_t* ovf;
+  uint32_t npay;
+  __device__ __forceinline__ const uint8_t* at(uint32_t o) const { return o < npay ? slot + o : ovf + (o - npay); }
+  __device__ __forceinline__ uint32_t ld32(uint32_t o) const { return __ldg(reinterpret_cast<const uint32_t*>(at(o))); }
+  __device__ __forceinline__ uint32_t ld16(uint32_t o) const { return __ldg(reinterpret_cast<const uint16_t*>(at(o))); }
 };
 
 template <int DT>
@@ -66,41 +75,33 @@ __device__ __forceinline__ void decode_normal(const Team& t, const Plan& pl, con
   }
 }
 
-// Outlier-rich plane.  `scr` is the team's shared scratch: nblk words.
+// Outlier-rich plane.  `scr` is the team's shared scratch: nblk words.  `ovf_avail` is the number of
+// readable bytes behind in.ovf.
 template <int DT>
-__device__ bool decode_salient(const Team& t, const Plan& pl, const uint8_t* pay, uint64_t avail,
-                               float eps, uint8_t* out, uint32_t* scr) {
+__device__ bool decode_salient(const Team& t, const Plan& pl, const SplitIn& in, uint64_t ovf_avail, float eps,
+                               uint8_t* out, uint32_t* scr) {
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx, nbm = pl.nbm, e = (uint32_t)pl.esize, HW = pl.HW;
-  if (avail < 16) return false;
-  const uint32_t* p32 = reinterpret_cast<const uint32_t*>(pay);
-  const uint32_t nnz_s = __ldg(p32), n_dense = __ldg(p32 + 1), n_out_d = __ldg(p32 + 2);
+  const uint32_t nnz_s = in.ld32(0), n_dense = in.ld32(4), n_out_d = in.ld32(8);
   if (nnz_s > HW || n_dense > nblk || n_out_d > HW) return false;
   const uint64_t size = 16ull + 4ull * nbm + 4ull * ((uint64_t)H + 1) + a4(2u * nnz_s) + a4(e * nnz_s) +
                         64ull * n_dense + a4(e * n_out_d);
-  if (size > avail) return false;
-  const uint32_t* g_bm = p32 + 4;
-  const uint32_t* g_rp = g_bm + nbm;
-  const uint8_t* g_col = reinterpret_cast<const uint8_t*>(g_rp + H + 1);
-  const uint8_t* g_val = g_col + a4(2u * nnz_s);
-  const uint8_t* g_codes = g_val + a4(e * nnz_s);
-  const uint8_t* g_outl = g_codes + 64u * n_dense;
+  if (size > in.npay && size - in.npay > ovf_avail) return false;
+  const uint32_t o_bm = 16u, o_rp = o_bm + 4u * nbm, o_col = o_rp + 4u * ((uint32_t)H + 1u);
+  const uint32_t o_val = o_col + a4(2u * nnz_s), o_codes = o_val + a4(e * nnz_s), o_outl = o_codes + 64u * n_dense;
   bool ok = true;
   // zero fill (16-bit units cover both element sizes)
-  for (uint32_t i = t.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += t.size)
-    reinterpret_cast<uint16_t*>(out)[i] = 0;
+  for (uint32_t i = t.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += t.size) reinterpret_cast<uint16_t*>(out)[i] = 0;
   // verbatim counts of the dense blocks -> first verbatim index of each block
   for (uint32_t b = t.lane; b < nblk; b += t.size) {
     uint32_t cnt = 0;
-    if ((__ldg(g_bm + (b >> 5)) >> (b & 31u)) & 1u) {
+    if ((in.ld32(o_bm + 4u * (b >> 5)) >> (b & 31u)) & 1u) {
       uint32_t rank = 0;
-      for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(__ldg(g_bm + w));
-      rank += __popc(__ldg(g_bm + (b >> 5)) & ((1u << (b & 31u)) - 1u));
+      for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(in.ld32(o_bm + 4u * w));
+      rank += __popc(in.ld32(o_bm + 4u * (b >> 5)) & ((1u << (b & 31u)) - 1u));
       if (rank < n_dense) {
-        const uint32_t* c32 = reinterpret_cast<const uint32_t*>(g_codes + 64u * rank);
-        for (int k = 0; k < 16; ++k) {
-          const uint32_t w = __ldg(c32 + k);
-          // bytes equal to zero
+        for (uint32_t k = 0; k < 16; ++k) {
+          const uint32_t w = in.ld32(o_codes + 64u * rank + 4u * k);
           cnt += ((w & 0xFFu) == 0) + ((w & 0xFF00u) == 0) + ((w & 0xFF0000u) == 0) + ((w & 0xFF000000u) == 0);
         }
       } else {
@@ -114,14 +115,14 @@ __device__ bool decode_salient(const Team& t, const Plan& pl, const uint8_t* pay
   if (tot_out > n_out_d) ok = false;
   // CSR scatter
   for (int y = (int)t.lane; y < H; y += (int)t.size) {
-    const uint32_t r0 = __ldg(g_rp + y), r1 = __ldg(g_rp + y + 1);
+    const uint32_t r0 = in.ld32(o_rp + 4u * y), r1 = in.ld32(o_rp + 4u * (y + 1));
     if (r0 > r1 || r1 > nnz_s) { ok = false; continue; }
     for (uint32_t k = r0; k < r1; ++k) {
-      const uint32_t col = __ldg(reinterpret_cast<const uint16_t*>(g_col) + k);
+      const uint32_t col = in.ld16(o_col + 2u * k);
       if (col >= (uint32_t)W) { ok = false; continue; }
       const uint32_t idx = (uint32_t)y * W + col;
-      if (DT == kF32) reinterpret_cast<uint32_t*>(out)[idx] = __ldg(reinterpret_cast<const uint32_t*>(g_val) + k);
-      else reinterpret_cast<uint16_t*>(out)[idx] = __ldg(reinterpret_cast<const uint16_t*>(g_val) + k);
+      if (DT == kF32) reinterpret_cast<uint32_t*>(out)[idx] = in.ld32(o_val + 4u * k);
+      else reinterpret_cast<uint16_t*>(out)[idx] = (uint16_t)in.ld16(o_val + 2u * k);
     }
   }
   // dense blocks: raster walk, k = pred + residual (Eq. 7-9), x = k * 2 eps
@@ -129,11 +130,11 @@ __device__ bool decode_salient(const Team& t, const Plan& pl, const uint8_t* pay
   const float inv2e = __fdiv_rn(1.0f, two_eps);
   if (ok && tot_out <= n_out_d) {
     for (uint32_t b = t.lane; b < nblk; b += t.size) {
-      if (!((__ldg(g_bm + (b >> 5)) >> (b & 31u)) & 1u)) continue;
+      if (!((in.ld32(o_bm + 4u * (b >> 5)) >> (b & 31u)) & 1u)) continue;
       uint32_t rank = 0;
-      for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(__ldg(g_bm + w));
-      rank += __popc(__ldg(g_bm + (b >> 5)) & ((1u << (b & 31u)) - 1u));
-      const uint32_t* c32 = reinterpret_cast<const uint32_t*>(g_codes + 64u * rank);
+      for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(in.ld32(o_bm + 4u * w));
+      rank += __popc(in.ld32(o_bm + 4u * (b >> 5)) & ((1u << (b & 31u)) - 1u));
+      const uint32_t oc = o_codes + 64u * rank;
       uint32_t oi = scr[b];
       const int by = (int)(b / nbx), bx = (int)(b % nbx);
       int32_t prev[8];
@@ -142,7 +143,7 @@ __device__ bool decode_salient(const Team& t, const Plan& pl, const uint8_t* pay
 #pragma unroll 1
       for (int i = 0; i < 8; ++i) {
         const int y = by * 8 + i;
-        const uint32_t w0 = __ldg(c32 + 2 * i), w1 = __ldg(c32 + 2 * i + 1);
+        const uint32_t w0 = in.ld32(oc + 8u * i), w1 = in.ld32(oc + 8u * i + 4u);
         int32_t left = 0, ul = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -156,11 +157,11 @@ __device__ bool decode_salient(const Team& t, const Plan& pl, const uint8_t* pay
             if (code == 0u) {
               float v;
               if (DT == kF32) {
-                const uint32_t raw = __ldg(reinterpret_cast<const uint32_t*>(g_outl) + oi);
+                const uint32_t raw = in.ld32(o_outl + 4u * oi);
                 reinterpret_cast<uint32_t*>(out)[idx] = raw;
                 v = __uint_as_float(raw);
               } else {
-                const uint32_t raw = __ldg(reinterpret_cast<const uint16_t*>(g_outl) + oi);
+                const uint32_t raw = in.ld16(o_outl + 2u * oi);
                 reinterpret_cast<uint16_t*>(out)[idx] = (uint16_t)raw;
                 v = bf16_bits_to_f32(raw);
               }
@@ -184,8 +185,8 @@ __device__ bool decode_salient(const Team& t, const Plan& pl, const uint8_t* pay
 
 template <int DT>
 __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, const DecompressArgs a) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  __shared__ double s_red[kThreads / 32 * 4 + 8];
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ double s_red[kWarps * 4];
   __shared__ uint32_t s_tile, s_hdr_ok, s_bits;
   __shared__ float s_eps;
   __shared__ unsigned long long s_total;
@@ -193,15 +194,13 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
   const unsigned long long off_in = a.d_off_in ? *a.d_off_in : 0ull;
   const uint8_t* src = a.src_base + off_in;
   const unsigned long long src_bytes = a.src_bytes > off_in ? a.src_bytes - off_in : 0ull;
-  const unsigned long long epoch_hi = (unsigned long long)a.epoch << 32;
-  const unsigned long long table_end = 64ull + 16ull * pl.P;
   const Team team = make_team(pl.team, s_red);
   const uint32_t nteams = team.block ? 1u : kThreads / team.size;
   const uint32_t my_team = team.block ? 0u : tid / team.size;
 
   // header check (every CTA, it is 64 bytes)
   if (tid == 0) {
-    uint32_t ok = src_bytes >= table_end;
+    uint32_t ok = src_bytes >= 64ull + 16ull * pl.P;
     if (ok) {
       const uint32_t* h = reinterpret_cast<const uint32_t*>(src);
       const uint32_t bits = __ldg(h + 1) >> 24;
@@ -210,7 +209,8 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
            __ldg(h + 4) == (uint32_t)pl.H && __ldg(h + 5) == (uint32_t)pl.W && (__ldg(h + 6) & 0xFFFFu) == (8u | (8u << 8));
       const unsigned long long total = (unsigned long long)__ldg(h + 14) | ((unsigned long long)__ldg(h + 15) << 32);
       const float eps = __uint_as_float(__ldg(h + 9));
-      ok = ok && total <= src_bytes && total >= table_end && eps >= 1e-30f && eps <= 1e30f;
+      const unsigned long long npay = a16(4u * ((pl.HW * (bits & 15u) + 31u) / 32u));
+      ok = ok && total <= src_bytes && total >= 64ull + 16ull * pl.P + pl.P * npay && eps >= 1e-30f && eps <= 1e30f;
       s_bits = bits;
       s_eps = eps;
       s_total = total;
@@ -222,10 +222,11 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
   const uint32_t bits = hdr_ok ? s_bits : 2u;
   const float eps = s_eps;
   const unsigned long long total = hdr_ok ? s_total : 0ull;
-  const uint32_t npay_bytes = 4u * ((pl.HW * bits + 31u) / 32u);
+  const uint32_t npay = a16(4u * ((pl.HW * bits + 31u) / 32u));
+  const unsigned long long slots_off = 64ull + 16ull * pl.P, ovf_off = slots_off + pl.P * (unsigned long long)npay;
 
   for (;;) {
-    if (tid == 0) s_tile = (uint32_t)(atomicAdd(&a.sc->ticket, 1ull) - a.ticket_base);
+    if (tid == 0) s_tile = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
     __syncthreads();
     const uint32_t tile = s_tile;
     if (tile >= pl.ntiles) break;
@@ -234,42 +235,53 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
     bool bad = !hdr_ok;
     if (hdr_ok) {
       for (uint32_t lp = my_team; lp < np; lp += nteams) {
-        const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + (p0 + lp));
+        const uint64_t gp = p0 + lp;
+        const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + gp);
         const unsigned long long off = (unsigned long long)e.x * 16ull;
         const uint32_t cls = e.y & 3u;
-        uint8_t* out = a.dst + (p0 + lp) * pl.plane_bytes;
-        if (off < table_end || off > total) { bad = true; continue; }
-        const unsigned long long avail = total - off;
-        const uint8_t* pay = src + off;
+        uint8_t* out = a.dst + gp * pl.plane_bytes;
+        const uint8_t* slot = src + slots_off + gp * npay;
         if (cls == kClsNormal) {
-          if (npay_bytes > avail) { bad = true; continue; }
+          if (off != slots_off + gp * npay) { bad = true; continue; }
           const float lo = __uint_as_float(e.z), scale = __uint_as_float(e.w);
-          if (bits == 2u) decode_normal<DT, 2>(team, pl, pay, lo, scale, out);
-          else if (bits == 4u) decode_normal<DT, 4>(team, pl, pay, lo, scale, out);
-          else decode_normal<DT, 8>(team, pl, pay, lo, scale, out);
-        } else if (cls == kClsRaw) {
-          if (pl.plane_bytes > avail) { bad = true; continue; }
-          for (uint32_t i = team.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += team.size)
-            reinterpret_cast<uint16_t*>(out)[i] = __ldg(reinterpret_cast<const uint16_t*>(pay) + i);
-        } else if (cls == kClsSalient) {
-          uint32_t* scr = reinterpret_cast<uint32_t*>(smem) + (uint64_t)my_team * pl.nblk;
-          if (!decode_salient<DT>(team, pl, pay, avail, eps, out, scr)) bad = true;
+          if (bits == 2u) decode_normal<DT, 2>(team, pl, slot, lo, scale, out);
+          else if (bits == 4u) decode_normal<DT, 4>(team, pl, slot, lo, scale, out);
+          else decode_normal<DT, 8>(team, pl, slot, lo, scale, out);
+        } else if (cls == kClsRaw || cls == kClsSalient) {
+          // the continuation, when there is one, lies in the overflow region
+          if (off != 0 && (off < ovf_off || off > total)) { bad = true; continue; }
+          SplitIn in;
+          in.slot = slot;
+          in.ovf = src + off;
+          in.npay = npay;
+          const unsigned long long ovf_avail = off ? total - off : 0ull;
+          if (cls == kClsRaw) {
+            if (pl.plane_bytes > npay && pl.plane_bytes - npay > ovf_avail) { bad = true; continue; }
+            for (uint32_t i = team.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += team.size)
+              reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)in.ld16(2u * i);
+          } else {
+            uint32_t* scr = reinterpret_cast<uint32_t*>(smem) + (uint64_t)my_team * pl.nblk;
+            if (!decode_salient<DT>(team, pl, in, ovf_avail, eps, out, scr)) bad = true;
+          }
         } else {
           bad = true;
         }
       }
     }
-    if (bad) atomicMax(&a.sc->status, epoch_hi | kErrCorrupt);
-    __threadfence();
+    if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
     __syncthreads();
-    if (tid == 0) {
-      const unsigned long long prev = atomicAdd(&a.sc->done, 1ull) - a.done_base;
-      if (prev == (unsigned long long)pl.ntiles - 1ull) {
-        __threadfence();
-        const unsigned long long st = ld_relaxed(&a.sc->status);
-        const uint32_t code = (st >> 32) == a.epoch ? (uint32_t)st : kErrNone;
-        if (a.d_status) *a.d_status = status_word(code);
-      }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned long long prev = atomicAdd(&a.sc->exited, 1ull);
+    if (prev == (unsigned long long)gridDim.x - 1ull) {
+      __threadfence();
+      const uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
+      if (a.d_status) *a.d_status = status_word(code);
+      st_relaxed(&a.sc->ticket, 0ull);
+      st_relaxed(&a.sc->status, 0ull);
+      st_relaxed(&a.sc->exited, 0ull);
     }
   }
 }

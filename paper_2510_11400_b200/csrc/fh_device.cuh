@@ -1,8 +1,9 @@
 // Device-side building blocks shared by the compress and decompress kernels (sm_100a).
 //
-// Terminology: a "plane" is one (n, c) feature map of H x W elements; a "tile" is a run of
-// consecutive planes that one CTA stages in shared memory; a "team" is the group of threads that
-// works on one plane: a power-of-two slice of a warp for small planes, the whole CTA for large ones.
+// Terminology: a "plane" is one (n, c) feature map of H x W elements; a "group" is four consecutive
+// elements of a plane; a "tile" is a run of consecutive planes that one CTA stages in shared memory;
+// a "team" is the set of threads that works on one plane: a power-of-two slice of a warp for small
+// planes, the whole CTA for large ones.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -10,13 +11,17 @@
 
 namespace fh {
 
-constexpr int kThreads = 256;          // CTA size of both kernels
+constexpr int kThreads = 256;             // CTA size of every kernel
+constexpr int kWarps = kThreads / 32;
 constexpr uint32_t kMagic = 0x31434846u;  // "FHC1"
 constexpr uint32_t kClsNormal = 0, kClsSalient = 1, kClsRaw = 2;
 constexpr int kModeAuto = 0, kModeOff = 1, kModeAll = 2;
 constexpr int kF32 = 0, kBF16 = 1;
+constexpr int kMaxStages = 4;
+constexpr float kMagicF = 12582912.0f;    // 1.5 * 2^23: fma(v, c, kMagicF) leaves rne(v*c) in the mantissa
+constexpr uint32_t kMagicBits = 0x4B400000u;
 
-// Device-side error codes (positive, ordered by priority; the host maps them to fh_status).
+// Device-side error codes (positive, ordered by priority; status_word() maps them to fh_status).
 constexpr uint32_t kErrNone = 0, kErrNonfinite = 1, kErrCapacity = 2, kErrCorrupt = 3, kErrTimeout = 4;
 
 // Everything a kernel needs to know about the tensor, the parameters and the tiling.
@@ -24,37 +29,46 @@ struct Plan {
   int32_t dtype, esize, H, W;
   uint32_t N, C;
   uint32_t HW;
-  uint32_t groups;       // ceil(HW / 4): groups of four consecutive elements
+  uint32_t groups;       // ceil(HW / 4)
   uint64_t P;            // planes
   uint64_t plane_bytes;  // HW * esize
   uint64_t dense_bytes;  // P * plane_bytes
+  double inv_hw;         // 1 / HW in fp64
   int32_t bits, mode;
   uint32_t rho_num, rho_den, tau_num, tau_den;
   float eps;
   uint64_t tensor_id;
+  uint32_t npay;         // slot size: A16(bytes of a normal payload)
+  uint64_t slots_off;    // 64 + 16 P
+  uint64_t ovf_off;      // slots_off + P * npay: start of the overflow region
+  uint32_t nbx, nby, nblk, nbm;  // 8x8 blocks per row / column / plane, bitmap words
+  // tiling
   uint32_t ppt;          // planes per tile
   uint32_t ntiles;
   uint32_t team;         // threads per plane: 1..32 (power of two) or kThreads
-  uint32_t npay;         // A16(bytes of a normal payload)
-  uint32_t nbx, nby, nblk, nbm;  // 8x8 blocks per row / column / plane, bitmap words
-  uint32_t sm_tile, sm_tile_bytes;  // shared-memory layout (byte offsets)
-  uint32_t sm_out, sm_rec, sm_sal, sm_sal_stride, sm_total;
+  uint32_t nstage;       // fast kernels: tiles in flight per CTA
+  uint32_t stage_bytes;  // fast kernels: bytes of one stage buffer (ppt * plane_bytes)
+  // shared-memory layout (byte offsets into dynamic shared memory)
+  uint32_t sm_tile, sm_out, sm_rec, sm_sal, sm_sal_stride, sm_total;
 };
 
-// Scan / bookkeeping scratch, one per stream.  Words carry the call's epoch in their upper half so
-// that nothing has to be cleared between calls.
-struct TileState {            // 32 bytes per tile
-  unsigned long long agg_a;   // epoch << 32 | tile size in 16-byte units
-  unsigned long long agg_b;   // n_salient << 32 | n_raw of the tile
-  unsigned long long inc_a;   // epoch << 32 | inclusive prefix of sizes
-  unsigned long long inc_b;   // inclusive prefix of the counts
-};
+// Book-keeping scratch, one per stream: a header of counters followed by one 64-bit scan word per
+// tile.  The scan words carry the call's epoch so that they need no clearing between calls; the
+// counters are returned to zero by the last CTA to leave a kernel.
 struct Scratch {
-  unsigned long long ticket;  // monotonically increasing tile tickets
-  unsigned long long done;    // monotonically increasing count of finished tiles
-  unsigned long long status;  // epoch << 32 | device error code (atomicMax)
-  unsigned long long total;   // container bytes of the current call
+  unsigned long long ticket;  // next tile
+  unsigned long long exited;  // CTAs that have left
+  unsigned long long status;  // device error code (atomicMax)
+  unsigned long long ovf16;   // overflow region size of this call, in 16-byte units
+  unsigned long long nsal, nraw;
+  unsigned long long pad[2];
 };
+static_assert(sizeof(Scratch) == 64, "Scratch layout");
+
+// scan word of a tile: epoch (30 bits) | flag (2 bits: 1 = tile aggregate, 2 = inclusive prefix) | value
+__device__ __forceinline__ unsigned long long scan_word(uint32_t epoch, uint32_t flag, uint32_t value) {
+  return ((unsigned long long)epoch << 34) | ((unsigned long long)flag << 32) | value;
+}
 
 // (uint64)(int64) fh_status of a device error code.
 __device__ __forceinline__ unsigned long long status_word(uint32_t code) {
@@ -65,6 +79,7 @@ __device__ __forceinline__ unsigned long long status_word(uint32_t code) {
 
 __device__ __forceinline__ uint32_t a4(uint32_t x) { return (x + 3u) & ~3u; }
 __device__ __forceinline__ uint32_t a16(uint32_t x) { return (x + 15u) & ~15u; }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ unsigned long long ld_acquire(const unsigned long long* p) {
   unsigned long long v;
@@ -83,8 +98,51 @@ __device__ __forceinline__ void st_relaxed(unsigned long long* p, unsigned long 
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
-// min / max that return NaN when either operand is NaN, so that a NaN anywhere in a plane
-// surfaces in its minimum and maximum.
+// ---- shared-memory barriers and bulk (TMA) copies -------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Bulk copy global -> shared; src, dst and bytes are multiples of 16.  Completion is signalled on `bar`.
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Bulk copy shared -> global (same alignment rules), tracked by bulk async-groups.
+__device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(smem_u32(src)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the phase did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 64) __nanosleep(32);
+  }
+  return false;
+}
+
+// ---- arithmetic helpers --------------------------------------------------------------------------
+// min / max that return NaN when any operand is NaN, so that a NaN anywhere in a plane surfaces in
+// its minimum and maximum.
 __device__ __forceinline__ float min_nan(float a, float b) {
   float r;
   asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
@@ -93,6 +151,16 @@ __device__ __forceinline__ float min_nan(float a, float b) {
 __device__ __forceinline__ float max_nan(float a, float b) {
   float r;
   asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ float min3_nan(float a, float b, float c) {
+  float r;
+  asm("min.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+__device__ __forceinline__ float max3_nan(float a, float b, float c) {
+  float r;
+  asm("max.NaN.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
   return r;
 }
 
@@ -109,11 +177,10 @@ __device__ __forceinline__ float load_elem(const uint8_t* plane, uint32_t i) {
   return bf16_bits_to_f32(reinterpret_cast<const uint16_t*>(plane)[i]);
 }
 
-// Four consecutive elements of a plane (group g), elements past HW read as 0.  `vec` says that the
-// plane starts on a 16-byte (fp32) / 8-byte (bf16) boundary so that a full group is one load.
+// Group g of a plane, elements past HW read as 0.  `vec` says that the plane starts on a 16-byte
+// (fp32) / 8-byte (bf16) boundary so that a full group is one load.
 template <int DT>
-__device__ __forceinline__ void load_group(const uint8_t* plane, uint32_t g, uint32_t HW, bool vec,
-                                           float v[4]) {
+__device__ __forceinline__ void load_group(const uint8_t* plane, uint32_t g, uint32_t HW, bool vec, float v[4]) {
   const uint32_t i0 = g * 4u;
   if (vec && i0 + 3u < HW) {
     if (DT == kF32) {
@@ -130,6 +197,70 @@ __device__ __forceinline__ void load_group(const uint8_t* plane, uint32_t g, uin
   }
 }
 
+// Fixed-point moments of a plane (three-sigma rule): scale factors from the largest magnitude A.
+struct SigmaScale {
+  float cs, cq;    // 2^ks, 2^kq
+  int32_t ks, kq;
+};
+__device__ __forceinline__ SigmaScale sigma_scale(float lo, float hi) {
+  const float A = fmaxf(fabsf(lo), fabsf(hi));
+  const int e = (int)((__float_as_uint(A) >> 23) & 255u) - 127;
+  SigmaScale s;
+  s.ks = min(18 - e, 126);
+  s.kq = max(min(16 - 2 * e, 126), -126);
+  s.cs = __uint_as_float((uint32_t)(s.ks + 127) << 23);
+  s.cq = __uint_as_float((uint32_t)(s.kq + 127) << 23);
+  return s;
+}
+// Raw mantissa images of the two fixed-point addends of one group; the caller sums them with
+// wrap-around arithmetic and subtracts kMagicBits once per group at the end.
+__device__ __forceinline__ void sigma_addends(const float v[4], const SigmaScale& sc, uint32_t& as, uint32_t& aq) {
+  const float sg = __fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3]));
+  const float q01 = __fmaf_rn(v[1], v[1], __fmul_rn(v[0], v[0]));
+  const float q23 = __fmaf_rn(v[3], v[3], __fmul_rn(v[2], v[2]));
+  const float qg = __fadd_rn(q01, q23);
+  as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
+  aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
+}
+// Thresholds mu +- 3 sigma from the exact integer sums.
+__device__ __forceinline__ void sigma_thresholds(long long Is, long long Iq, const SigmaScale& sc, double inv_hw,
+                                                 float& tlo, float& thi) {
+  const double ps = __hiloint2double((1023 - sc.ks) << 20, 0);  // 2^-ks
+  const double pq = __hiloint2double((1023 - sc.kq) << 20, 0);  // 2^-kq
+  const double mu = __dmul_rn(__dmul_rn((double)Is, ps), inv_hw);
+  const double m2 = __dmul_rn(__dmul_rn((double)Iq, pq), inv_hw);
+  double var = __dsub_rn(m2, __dmul_rn(mu, mu));
+  if (!(var > 0.0)) var = 0.0;
+  const float mu_f = __double2float_rn(mu);
+  const float sigma_f = __fsqrt_rn(__double2float_rn(var));
+  thi = __fmaf_rn(3.0f, sigma_f, mu_f);
+  tlo = __fmaf_rn(-3.0f, sigma_f, mu_f);
+}
+
+// Quantiser parameters of a normal plane.
+__device__ __forceinline__ void quant_params(float lo, float hi, uint32_t L, float& inv, float& scale) {
+  const float range = __fsub_rn(hi, lo);
+  inv = __fdiv_rn((float)L, range);
+  scale = __fdiv_rn(range, (float)L);
+  if (range == 0.0f || !(fabsf(inv) <= 3.402823466e38f)) {
+    inv = 0.0f;
+    scale = 0.0f;
+  }
+}
+// Code of one element: rne of the exact product (x - lo) * inv, as an integer in the mantissa.
+__device__ __forceinline__ uint32_t quant_code(float x, float lo, float inv, uint32_t L) {
+  const float r = __fmaf_rn(__fsub_rn(x, lo), inv, kMagicF);
+  return (__float_as_uint(r) - kMagicBits) & L;
+}
+
+// Pre-quantisation of dense-block elements (Eq. 9 on integers): k = rne(fp32(x * inv2e)), |k| <= 2^24.
+__device__ __forceinline__ int32_t dense_k(float x, float inv2e, bool* big) {
+  float kf = rintf(__fmul_rn(x, inv2e));
+  *big = fabsf(kf) >= 16777216.0f;
+  kf = fminf(fmaxf(kf, -16777216.0f), 16777216.0f);
+  return (int32_t)kf;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Teams
 // ------------------------------------------------------------------------------------------------
@@ -138,7 +269,7 @@ struct Team {
   uint32_t lane;   // this thread's index inside the team
   uint32_t mask;   // warp member mask of the team (sub-warp teams)
   bool block;      // the team is the whole CTA
-  double* red;     // shared scratch for CTA-wide reductions: (kThreads/32) * 4 doubles + 8
+  double* red;     // shared scratch for CTA-wide reductions: kWarps * 4 doubles
 };
 
 __device__ __forceinline__ Team make_team(uint32_t team_size, double* red) {
@@ -157,58 +288,89 @@ __device__ __forceinline__ Team make_team(uint32_t team_size, double* red) {
   }
   return t;
 }
+// The warp of this thread as a team (used for the block-wise path of the warp-team kernels).
+__device__ __forceinline__ Team make_warp_team(double* red) {
+  Team t;
+  t.size = 32;
+  t.red = red;
+  t.block = false;
+  t.lane = threadIdx.x & 31u;
+  t.mask = 0xFFFFFFFFu;
+  return t;
+}
 
 __device__ __forceinline__ void team_sync(const Team& t) {
   if (t.block) __syncthreads();
   else __syncwarp(t.mask);
 }
 
-// Plane statistics reduced over the team: lo/hi with NaN propagation, S/Q in fp64.
-struct Stats {
-  float lo, hi;
-  double S, Q;
-};
-
-__device__ __forceinline__ Stats team_reduce_stats(const Team& t, Stats s) {
-  const uint32_t w = t.block ? 32u : t.size;
-  for (uint32_t o = w >> 1; o > 0; o >>= 1) {
-    s.lo = min_nan(s.lo, __shfl_xor_sync(t.mask, s.lo, o));
-    s.hi = max_nan(s.hi, __shfl_xor_sync(t.mask, s.hi, o));
-    s.S += __shfl_xor_sync(t.mask, s.S, o);
-    s.Q += __shfl_xor_sync(t.mask, s.Q, o);
-  }
+// min / max over the team with NaN propagation (hardware warp reduction for fp32).
+__device__ __forceinline__ void team_minmax(const Team& t, float& lo, float& hi) {
+  if (!t.block && t.size == 1u) return;
+  asm volatile("redux.sync.min.NaN.f32 %0, %0, %1;" : "+f"(lo) : "r"(t.mask));
+  asm volatile("redux.sync.max.NaN.f32 %0, %0, %1;" : "+f"(hi) : "r"(t.mask));
   if (t.block) {
-    const uint32_t warp = threadIdx.x >> 5, nw = kThreads / 32;
+    float* r = reinterpret_cast<float*>(t.red);
+    const uint32_t warp = threadIdx.x >> 5;
     __syncthreads();
     if ((threadIdx.x & 31u) == 0) {
-      t.red[warp * 4 + 0] = (double)s.lo;
-      t.red[warp * 4 + 1] = (double)s.hi;
-      t.red[warp * 4 + 2] = s.S;
-      t.red[warp * 4 + 3] = s.Q;
+      r[warp * 2] = lo;
+      r[warp * 2 + 1] = hi;
     }
     __syncthreads();
-    s.lo = (float)t.red[0]; s.hi = (float)t.red[1]; s.S = t.red[2]; s.Q = t.red[3];
-    for (uint32_t k = 1; k < nw; ++k) {
-      s.lo = min_nan(s.lo, (float)t.red[k * 4 + 0]);
-      s.hi = max_nan(s.hi, (float)t.red[k * 4 + 1]);
-      s.S += t.red[k * 4 + 2];
-      s.Q += t.red[k * 4 + 3];
+    lo = r[0];
+    hi = r[1];
+#pragma unroll
+    for (int k = 1; k < kWarps; ++k) {
+      lo = min_nan(lo, r[k * 2]);
+      hi = max_nan(hi, r[k * 2 + 1]);
     }
   }
-  return s;
+}
+
+// Sum of two int32 per thread over the team, returned as 64-bit integers.  Within a warp the sums fit
+// 32 bits (see the callers); warps are combined in 64 bits.
+__device__ __forceinline__ void team_sum2(const Team& t, int32_t a, int32_t b, long long& A, long long& B) {
+  if (!t.block && t.size == 1u) {
+    A = a;
+    B = b;
+    return;
+  }
+  asm volatile("redux.sync.add.s32 %0, %0, %1;" : "+r"(a) : "r"(t.mask));
+  asm volatile("redux.sync.add.s32 %0, %0, %1;" : "+r"(b) : "r"(t.mask));
+  A = a;
+  B = b;
+  if (t.block) {
+    long long* r = reinterpret_cast<long long*>(t.red);
+    const uint32_t warp = threadIdx.x >> 5;
+    __syncthreads();
+    if ((threadIdx.x & 31u) == 0) {
+      r[warp * 2] = a;
+      r[warp * 2 + 1] = b;
+    }
+    __syncthreads();
+    A = 0;
+    B = 0;
+#pragma unroll
+    for (int k = 0; k < kWarps; ++k) {
+      A += r[k * 2];
+      B += r[k * 2 + 1];
+    }
+  }
 }
 
 __device__ __forceinline__ uint32_t team_sum_u32(const Team& t, uint32_t v) {
-  const uint32_t w = t.block ? 32u : t.size;
-  for (uint32_t o = w >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(t.mask, v, o);
+  if (!t.block && t.size == 1u) return v;
+  asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(v) : "r"(t.mask));
   if (t.block) {
     uint32_t* r = reinterpret_cast<uint32_t*>(t.red);
-    const uint32_t warp = threadIdx.x >> 5, nw = kThreads / 32;
+    const uint32_t warp = threadIdx.x >> 5;
     __syncthreads();
     if ((threadIdx.x & 31u) == 0) r[warp] = v;
     __syncthreads();
     v = 0;
-    for (uint32_t k = 0; k < nw; ++k) v += r[k];
+#pragma unroll
+    for (int k = 0; k < kWarps; ++k) v += r[k];
   }
   return v;
 }
@@ -228,8 +390,8 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
     }
     total = __shfl_sync(t.mask, incl, t.size - 1u, t.size);
   } else {
-    uint32_t* r = reinterpret_cast<uint32_t*>(t.red);  // kThreads/32 + 1 words
-    const uint32_t wl = threadIdx.x & 31u, warp = threadIdx.x >> 5, nw = kThreads / 32;
+    uint32_t* r = reinterpret_cast<uint32_t*>(t.red);
+    const uint32_t wl = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     for (uint32_t o = 1; o < 32u; o <<= 1) {
       const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
       if (wl >= o) incl += up;
@@ -239,7 +401,7 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
     __syncthreads();
     uint32_t base = 0;
     total = 0;
-    for (uint32_t k = 0; k < nw; ++k) {
+    for (uint32_t k = 0; k < (uint32_t)kWarps; ++k) {
       if (k < warp) base += r[k];
       total += r[k];
     }
@@ -256,12 +418,50 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
   return total;
 }
 
-// Pre-quantisation of dense-block elements (Eq. 9 on integers): k = rne(fp32(x * inv2e)), |k| <= 2^24.
-__device__ __forceinline__ int32_t dense_k(float x, float inv2e, bool* big) {
-  float kf = rintf(__fmul_rn(x, inv2e));
-  *big = fabsf(kf) >= 16777216.0f;
-  kf = fminf(fmaxf(kf, -16777216.0f), 16777216.0f);
-  return (int32_t)kf;
+// ------------------------------------------------------------------------------------------------
+// Plane-ordered placement of the overflow parts: decoupled look-back over per-tile scan words.
+// Executed by all 32 lanes of warp 0.  Every tile publishes its aggregate (mostly zero); a tile that
+// needs its offset, and every 32nd tile (so that walks stay short), resolves its exclusive prefix
+// and publishes the inclusive one.  The wait is bounded; on expiry the call reports kErrTimeout.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void scan_publish(unsigned long long* ts, uint32_t tile, uint32_t epoch, uint32_t flag,
+                                             uint32_t value) {
+  if ((threadIdx.x & 31u) == 0) st_release(ts + tile, scan_word(epoch, flag, value));
+}
+
+// Returns false on timeout.  *excl receives the sum of the aggregates of tiles [0, tile).
+__device__ __forceinline__ bool scan_resolve(const unsigned long long* ts, uint32_t tile, uint32_t epoch,
+                                             uint32_t spin_limit, const unsigned long long* status,
+                                             unsigned long long* excl) {
+  const uint32_t lane = threadIdx.x & 31u;
+  unsigned long long sum = 0;
+  long long j = (long long)tile - 1;
+  uint32_t spins = 0;
+  while (j >= 0) {
+    const long long idx = j - (long long)lane;
+    // before tile 0 there is nothing: a virtual inclusive prefix of zero
+    const unsigned long long w = idx >= 0 ? ld_acquire(ts + idx) : scan_word(epoch, 2u, 0u);
+    const bool valid = (uint32_t)(w >> 34) == epoch;
+    const uint32_t flag = (uint32_t)(w >> 32) & 3u;
+    const uint32_t inc_mask = __ballot_sync(0xFFFFFFFFu, valid && flag == 2u);
+    const uint32_t inv_mask = __ballot_sync(0xFFFFFFFFu, !valid);
+    const uint32_t first_inc = inc_mask ? (uint32_t)__ffs(inc_mask) - 1u : 32u;
+    const uint32_t first_inv = inv_mask ? (uint32_t)__ffs(inv_mask) - 1u : 32u;
+    const uint32_t need = min(first_inc, 31u);
+    if (first_inv <= need) {  // a predecessor we need has not published yet
+      ++spins;
+      if (spins > spin_limit || ((spins & 63u) == 0 && ld_relaxed(status) == kErrTimeout)) return false;
+      __nanosleep(40);
+      continue;
+    }
+    uint32_t c = lane <= need ? (uint32_t)w : 0u;
+    asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(c) : "r"(0xFFFFFFFFu));
+    sum += c;
+    if (first_inc < 32u) break;
+    j -= 32;
+  }
+  *excl = sum;
+  return true;
 }
 
 }  // namespace fh

@@ -24,8 +24,30 @@ def normal_codes(buf, off, hw, bits):
     return ((w[i // 32] >> (i % 32).astype(np.uint32)) & np.uint32((1 << bits) - 1)).astype(np.int64)
 
 
+def npay_of(buf, hw):
+    """Slot size of a container: A16(4 * ceil(HW * bits / 32)), bits from the header."""
+    bits = int(buf[7])
+    return a16(4 * ((hw * bits + 31) // 32))
+
+
+def logical_payload(buf, P, pl, hw):
+    """Payload bytes of a salient or raw plane: its slot followed by its continuation in the
+    overflow region (returned up to the end of the container; callers parse what they need)."""
+    npay = npay_of(buf, hw)
+    slots = 64 + 16 * P
+    slot = buf[slots + pl * npay: slots + (pl + 1) * npay]
+    off = int(table(buf, P)["off"][pl])
+    if off == 0:
+        return np.concatenate([slot, np.zeros(16, dtype=np.uint8)])
+    return np.concatenate([slot, buf[off:], np.zeros(16, dtype=np.uint8)])
+
+
+def salient_plane(buf, P, pl, H, W, esize):
+    return salient(logical_payload(buf, P, pl, H * W), 0, H, W, esize)
+
+
 def salient(buf, off, H, W, esize):
-    """Split a salient payload into its sections."""
+    """Split a salient payload (contiguous bytes) into its sections."""
     nblk = ((H + 7) // 8) * ((W + 7) // 8)
     nbm = (nblk + 31) // 32
     hdr = np.ascontiguousarray(buf[off:off + 16]).view(np.uint32)

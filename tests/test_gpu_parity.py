@@ -214,11 +214,15 @@ def test_corrupt_salient_payload_is_rejected_without_out_of_bounds_reads():
     buf = packed[:total].cpu().numpy()
     t = hp.table(buf, 16)
     pl = int(np.flatnonzero(t["cls"] == fho.SALIENT)[0])
-    off = int(t["off"][pl])
+    off = 64 + 16 * 16 + pl * hp.npay_of(buf, 24 * 40)     # the payload starts in the plane's slot
     for field, val in ((0, 0x7FFFFFFF), (4, 0x7FFFFFFF), (8, 0x7FFFFFFF)):
         b = packed.clone()
         b[off + field:off + field + 4] = to_dev(np.frombuffer(np.uint32(val).tobytes(), dtype=np.uint8).copy())
         assert api.decompress_tensor(b, total, spec.shape, spec.dtype)[0] == api.FH_ERR_CORRUPT
+    # a continuation offset that points outside the overflow region
+    b = packed.clone()
+    b[64 + 16 * pl:64 + 16 * pl + 4] = to_dev(np.frombuffer(np.uint32(5).tobytes(), dtype=np.uint8).copy())
+    assert api.decompress_tensor(b, total, spec.shape, spec.dtype)[0] == api.FH_ERR_CORRUPT
 
 
 def test_repeated_calls_reuse_the_scratch_and_stay_exact():

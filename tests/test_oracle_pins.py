@@ -239,29 +239,51 @@ def test_config1_size_and_header():
     assert sizes.sum() > 0
 
 
-def test_offsets_are_running_sum_of_padded_payloads_mixed_classes():
+def test_slots_and_overflow_offsets_mixed_classes():
+    """Every plane owns a slot at a closed-form offset; payloads longer than the slot continue in the
+    overflow region in plane order, each continuation padded to 16 bytes; total = fixed part + sum."""
     spec = synth.TensorSpec("s", (2, 32, 24, 40), synth.F32, "spiky_relu", 77)
     x = synth.make(spec)
     d, p, buf = enc(x, spec.shape, bits=4)
     P, H, W = 64, 24, 40
+    npay = hp.a16(4 * ((H * W * 4 + 31) // 32))
+    assert npay == hp.npay_of(buf, H * W)
     t = hp.table(buf, P)
     assert (t["cls"] == fho.SALIENT).sum() >= 4 and (t["cls"] == fho.NORMAL).sum() >= 32
-    off = 64 + 16 * P
+    slots = 64 + 16 * P
+    ovf = slots + P * npay
     for pl in range(P):
-        assert t["off"][pl] == off
         if t["cls"][pl] == fho.NORMAL:
-            sz = 4 * ((H * W * 4 + 31) // 32)
-        elif t["cls"][pl] == fho.RAW:
+            assert t["off"][pl] == slots + pl * npay
+            continue
+        if t["cls"][pl] == fho.RAW:
             sz = 4 * H * W
         else:
-            s = hp.salient(buf, off, H, W, 4)
+            s = hp.salient_plane(buf, P, pl, H, W, 4)
             sz = s["size"]
             assert s["pad"] == 0
             assert sz == 16 + 4 * ((15 + 31) // 32) + 4 * (H + 1) + hp.a4(2 * s["nnz_s"]) + 4 * s["nnz_s"] \
                 + 64 * s["n_dense"] + 4 * s["n_out_d"]
-        assert not buf[off + sz:off + hp.a16(sz)].any()
-        off += hp.a16(sz)
-    assert off == buf.size == fho.parse_header(buf)["total_bytes"]
+        if sz <= npay:
+            assert t["off"][pl] == 0
+            assert not buf[slots + pl * npay + sz: slots + (pl + 1) * npay].any()
+        else:
+            assert t["off"][pl] == ovf
+            assert not buf[ovf + sz - npay: ovf + hp.a16(sz) - npay].any()
+            ovf += hp.a16(sz) - npay
+    assert ovf == buf.size == fho.parse_header(buf)["total_bytes"]
+
+
+def test_short_salient_payload_stays_inside_its_slot():
+    """A salient plane whose payload is no longer than a slot has no continuation (offset 0)."""
+    x = np.zeros(32 * 32, dtype=np.float32)
+    x[5] = 3.0
+    d, p, buf = enc(x, (1, 1, 32, 32), bits=8, salient_mode=fho.ALL)   # slot = 1024 bytes
+    t = hp.table(buf, 1)
+    s = hp.salient_plane(buf, 1, 0, 32, 32, 4)
+    assert t["cls"][0] == fho.SALIENT and t["off"][0] == 0 and s["size"] <= 1024
+    assert buf.size == 64 + 16 + 1024
+    assert np.array_equal(dec(buf, d), x)
 
 
 # ------------------------------------------------------------------------------------------------
@@ -285,20 +307,60 @@ def test_sigma_hand_case_spike():
 @pytest.mark.parametrize("kind,seed", [("normal", 1), ("relu", 2), ("laplace", 3)])
 def test_sigma_count_matches_numpy_float64(kind, seed):
     """mu, sigma are the plain mean and population standard deviation: NumPy float64 agrees on the
-    outlier count whenever no element sits within rounding distance of a threshold."""
+    outlier count whenever no element sits within rounding distance of a threshold.  The fixed-point
+    sums resolve 2^-19 of the largest magnitude per group of four, which bounds the differences."""
     hw = 56 * 56
     x = {"normal": synth.normal, "relu": synth.relu_normal, "laplace": synth.laplace}[kind](8 * hw, seed)
     for pl in range(8):
         xs = x[pl * hw:(pl + 1) * hw]
         S, Q, tlo, thi, n = fho.plane_sigma(xs)
         x64 = xs.astype(np.float64)
+        A = np.abs(x64).max()
+        groups = hw // 4
         mu, sd = x64.mean(), x64.std()
-        assert abs(S - x64.sum()) <= 1e-4 and abs(Q - (x64 ** 2).sum()) <= 1e-3 * hw * 1e-3 + 1e-2
-        assert abs(thi - (mu + 3 * sd)) <= 1e-5 and abs(tlo - (mu - 3 * sd)) <= 1e-5
+        assert abs(S - x64.sum()) <= groups * A * 2.0 ** -18
+        assert abs(Q - (x64 ** 2).sum()) <= groups * A * A * 2.0 ** -15
+        assert abs(thi - (mu + 3 * sd)) <= 1e-4 and abs(tlo - (mu - 3 * sd)) <= 1e-4
         margin = np.minimum(np.abs(x64 - (mu + 3 * sd)), np.abs(x64 - (mu - 3 * sd))).min()
-        if margin > 1e-4:
+        if margin > 1e-3:
             assert n == int(((x64 > mu + 3 * sd) | (x64 < mu - 3 * sd)).sum())
         assert n <= hw / 9  # Chebyshev: P(|x-mu| > 3 sigma) <= 1/9
+
+
+@pytest.mark.parametrize("scale", [1.0, 1e-3, 3e4, 2.0 ** -100, 2.0 ** 40])
+def test_fixed_point_sums_are_exact_integers_of_the_stated_roundings(scale):
+    """I_s and I_q are sums of round-half-even(s_g * 2^k_s) and (q_g * 2^k_q): recomputed here with
+    exact rational arithmetic from fp32 group values, for planes of very different magnitude, and
+    shown to be independent of the order of the groups."""
+    from fractions import Fraction
+    rng = np.random.default_rng(17)
+    x = (rng.standard_normal(203) * scale).astype(np.float32)   # 203: ragged last group
+    Is, Iq, ks, kq = fho.plane_sums(x)
+    A = float(np.abs(x).max())
+    e = int(np.floor(np.log2(A)))
+    assert ks == min(18 - e, 126) and kq == max(min(16 - 2 * e, 126), -126)
+
+    def rne(t):
+        fl = t.numerator // t.denominator
+        rem = t - fl
+        return fl + (1 if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1) else 0)
+    xp = np.concatenate([x, np.zeros(1, np.float32)]).reshape(-1, 4)
+    es = eq = 0
+    for v in xp:
+        sg = np.float32(np.float32(v[0] + v[1]) + np.float32(v[2] + v[3]))
+        f = [Fraction(float(t)) for t in v]
+        q01 = np.float32(float(f[1] * f[1] + Fraction(float(np.float32(v[0] * v[0])))))   # fma: one rounding
+        q23 = np.float32(float(f[3] * f[3] + Fraction(float(np.float32(v[2] * v[2])))))
+        qg = np.float32(q01 + q23)
+        es += rne(Fraction(float(sg)) * Fraction(2) ** ks)
+        eq += rne(Fraction(float(qg)) * Fraction(2) ** kq)
+    assert (Is, Iq) == (es, eq)
+    # a permutation of whole groups leaves the integers unchanged
+    perm = rng.permutation(xp.shape[0])
+    Is2, Iq2, _, _ = fho.plane_sums(xp[perm].reshape(-1))
+    assert (Is2, Iq2) == (Is, Iq)
+    # and the sums are close to the real ones
+    assert abs(Is * 2.0 ** -ks - float(x.astype(np.float64).sum())) <= 51 * A * 2.0 ** -18
 
 
 def test_sigma_tail_group_padding_and_constant_plane():
@@ -356,7 +418,7 @@ def test_block_classes_equal_average_pooled_mask(H, W):
     t = hp.table(buf, 1)
     if t["cls"][0] == fho.RAW:
         pytest.skip("plane stored verbatim")
-    s = hp.salient(buf, int(t["off"][0]), H, W, 4)
+    s = hp.salient_plane(buf, 1, 0, H, W, 4)
     Hp, Wp = 8 * ((H + 7) // 8), 8 * ((W + 7) // 8)
     m = torch.zeros(1, 1, Hp, Wp)
     m[0, 0, :H, :W] = torch.from_numpy((x != 0).astype(np.float32))
@@ -379,7 +441,7 @@ def test_block_threshold_at_15_16_nonzeros():
         d, p, buf = enc(x.reshape(-1), (1, 1, 8, 16), bits=2, salient_mode=fho.ALL)
         t = hp.table(buf, 1)
         assert t["cls"][0] == fho.SALIENT
-        s = hp.salient(buf, int(t["off"][0]), 8, 16, 4)
+        s = hp.salient_plane(buf, 1, 0, 8, 16, 4)
         assert list(s["dense"]) == [0, want]
 
 
@@ -393,7 +455,7 @@ def test_csr_equals_scipy(H, W, dtype):
     d, p, buf = enc(raw, (1, 1, H, W), dtype=dtype, bits=2, salient_mode=fho.ALL)
     t = hp.table(buf, 1)
     assert t["cls"][0] == fho.SALIENT
-    s = hp.salient(buf, int(t["off"][0]), H, W, e)
+    s = hp.salient_plane(buf, 1, 0, H, W, e)
     nbx = (W + 7) // 8
     yy, xx = np.mgrid[0:H, 0:W]
     in_sparse = s["dense"][(yy // 8) * nbx + xx // 8] == 0
@@ -415,7 +477,7 @@ def test_lorenzo_hand_case():
     x[:] = i + j + 1
     d, p, buf = enc(x.reshape(-1), (1, 1, 8, 8), bits=2, salient_mode=fho.ALL, eps=0.5)
     t = hp.table(buf, 1)
-    s = hp.salient(buf, int(t["off"][0]), 8, 8, 4)
+    s = hp.salient_plane(buf, 1, 0, 8, 8, 4)
     assert s["n_dense"] == 1 and s["n_out_d"] == 0 and s["nnz_s"] == 0
     c = s["codes"][0]
     assert list(c[0, :3]) + list(c[1, :3]) == codes
@@ -433,7 +495,7 @@ def test_lorenzo_affine_fields_have_zero_interior_residual(a, b, c):
     x[x == 0] = 2 * eps * 64  # keep blocks dense without breaking integrality much
     d, p, buf = enc(x.reshape(-1), (1, 1, 16, 24), bits=2, salient_mode=fho.ALL, eps=eps)
     t = hp.table(buf, 1)
-    s = hp.salient(buf, int(t["off"][0]), 16, 24, 4)
+    s = hp.salient_plane(buf, 1, 0, 16, 24, 4)
     k = np.rint(x / (2 * eps)).astype(np.int64)
     for bi, blk in enumerate(np.flatnonzero(s["dense"])):
         by, bx = divmod(int(blk), 3)
@@ -457,7 +519,7 @@ def test_dense_blocks_error_bound_outliers_verbatim_zeros_kept(H, W, eps):
     d, p, buf = enc(x, (1, 1, H, W), bits=2, salient_mode=fho.ALL, eps=eps)
     t = hp.table(buf, 1)
     assert t["cls"][0] == fho.SALIENT
-    s = hp.salient(buf, int(t["off"][0]), H, W, 4)
+    s = hp.salient_plane(buf, 1, 0, H, W, 4)
     assert s["n_out_d"] >= 2
     xh = dec(buf, d)
     nbx = (W + 7) // 8
@@ -493,7 +555,7 @@ def test_residual_code_range_is_symmetric_127():
     x[1, 1] = 128   # residuals +127 at (1,1),(2,2) and -127 at (1,2),(2,1): all codable
     x[4, 4] = 129   # residuals +128 at (4,4),(5,5) and -128 at (4,5),(5,4): none codable
     d, p, buf = enc(x.reshape(-1), (1, 1, 8, 8), bits=2, salient_mode=fho.ALL, eps=0.5)
-    s = hp.salient(buf, int(hp.table(buf, 1)["off"][0]), 8, 8, 4)
+    s = hp.salient_plane(buf, 1, 0, 8, 8, 4)
     c = s["codes"][0]
     assert (c[1, 1], c[1, 2], c[2, 1], c[2, 2]) == (255, 1, 1, 255)
     assert (c[4, 4], c[4, 5], c[5, 4], c[5, 5]) == (0, 0, 0, 0)
@@ -508,7 +570,7 @@ def test_predictor_sees_reconstructed_values():
     x = (np.random.default_rng(4).standard_normal(H * W) * 2 + 3).astype(np.float32)
     d, p, buf = enc(x, (1, 1, H, W), bits=2, salient_mode=fho.ALL, eps=eps)
     t = hp.table(buf, 1)
-    s = hp.salient(buf, int(t["off"][0]), H, W, 4)
+    s = hp.salient_plane(buf, 1, 0, H, W, 4)
     assert s["n_dense"] == 4 and s["n_out_d"] == 0
     k_true = np.rint(x.reshape(H, W) / np.float32(2 * eps)).astype(np.int64)
     for bi in range(4):
@@ -530,7 +592,7 @@ def test_raw_rule_when_nothing_is_gained():
     d, p, buf = enc(x, (1, 1, 64, 64), bits=2, salient_mode=fho.ALL, eps=0.0625)
     t = hp.table(buf, 1)
     assert t["cls"][0] == fho.RAW and fho.parse_header(buf)["n_raw"] == 1
-    assert buf.size == 64 + 16 + 4 * 64 * 64
+    assert buf.size == 64 + 16 + 4 * 64 * 64 and hp.table(buf, 1)["off"][0] == 64 + 16 + 1024
     assert np.array_equal(dec(buf, d), x)
 
 
@@ -595,7 +657,7 @@ def test_errors_capacity_nonfinite_corrupt_args():
     z[::3] = -0.0
     z[1] = 5
     dd, pp, bb = enc(z, (1, 1, 8, 8), bits=2, salient_mode=fho.ALL)
-    s = hp.salient(bb, int(hp.table(bb, 1)["off"][0]), 8, 8, 4)
+    s = hp.salient_plane(bb, 1, 0, 8, 8, 4)
     assert s["nnz_s"] == 1 and s["n_dense"] == 0
     out = dec(bb, dd)
     assert out[1] == 5 and np.all(out.view(np.uint32)[np.arange(64) != 1] == 0)
