@@ -21,7 +21,8 @@ using fh::Plan;
 
 constexpr size_t kSmemLimit = 227 * 1024 - 1024;  // dynamic shared memory a CTA may ask for
 constexpr size_t kTileTarget = 32 * 1024;         // dense bytes a tile of the generic kernel aims for
-constexpr size_t kStageTarget = 72 * 1024;        // shared memory the stages of a fast kernel aim for
+constexpr size_t kStageTarget = 72 * 1024;        // shared memory the stages of the CTA-team kernel aim for
+constexpr size_t kWarpStageTarget = 100 * 1024;   // ... and those of the warp-team kernel (two CTAs per SM)
 constexpr uint32_t kMaxPpt = 2048;
 constexpr uint32_t kSpinLimit = 1u << 20;
 
@@ -112,7 +113,8 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
 
   Variant v;
   // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
-  if (compress && pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0 && pl.groups <= 4096) {
+  const bool whole16 = pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0;
+  if (compress && pl.groups <= 4096 && (whole16 || pl.groups <= 256)) {
     v.fast = true;
     if (pl.groups <= 256) {
       uint32_t t = pow2_ceil((pl.groups + 7) / 8);
@@ -126,19 +128,19 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
       pl.ppt = 1;
     }
     if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
-    pl.stage_bytes = (uint32_t)(pl.ppt * pl.plane_bytes);
+    pl.stage_bytes = (uint32_t)((pl.ppt * pl.plane_bytes + 127) & ~(uint64_t)127);
     pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * sal_words) : 0;
-    const uint32_t nsal_teams = v.cta ? 1 : fh::kWarps;
-    uint32_t ns = (uint32_t)(kStageTarget / pl.stage_bytes);
+    const uint32_t nsal_teams = v.cta ? 1 : fh::kThreads / pl.team;
+    uint32_t ns = (uint32_t)((v.cta ? kStageTarget : kWarpStageTarget) / pl.stage_bytes);
     ns = ns < 2 ? 2 : (ns > (uint32_t)fh::kMaxStages ? (uint32_t)fh::kMaxStages : ns);
     for (;;) {
       pl.nstage = ns;
       pl.sm_tile = 0;
       pl.sm_rec = (uint32_t)A16((size_t)ns * pl.stage_bytes);
-      pl.sm_sal = pl.sm_rec + (uint32_t)A16(20 * (size_t)pl.ppt);
+      pl.sm_sal = pl.sm_rec + (v.cta ? 1u : ns) * (uint32_t)A16(20 * (size_t)pl.ppt);
       pl.sm_total = pl.sm_sal + nsal_teams * pl.sm_sal_stride;
       if (pl.sm_total <= kSmemLimit) break;
-      if (ns == 1) {
+      if (ns == 2) {  // the pipeline needs two stages
         v.fast = false;
         break;
       }
@@ -243,7 +245,7 @@ int sm_count() {
 }
 
 template <typename K>
-int grid_for(K kernel, size_t smem, uint32_t ntiles, int* grid) {
+int grid_for(K kernel, size_t smem, uint32_t ntiles, int* grid, int threads = fh::kThreads) {
   static std::map<std::pair<const void*, size_t>, int> cache;  // guarded by g_mu
   const auto key = std::make_pair((const void*)kernel, smem);
   auto it = cache.find(key);
@@ -251,7 +253,7 @@ int grid_for(K kernel, size_t smem, uint32_t ntiles, int* grid) {
   if (it == cache.end()) {
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess)
       return FH_ERR_CUDA;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, fh::kThreads, smem) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem) != cudaSuccess)
       return FH_ERR_CUDA;
     if (per_sm < 1) return FH_ERR_UNSUPPORTED;
     cache[key] = per_sm;
@@ -288,14 +290,23 @@ int launch_fast_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream
   return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
+template <int DT, bool SIGMA, int G>
+int launch_warp_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
+  int grid = 0;
+  int rc = grid_for(fh::compress_warp<DT, SIGMA, G>, pl.sm_total, pl.ntiles, &grid, fh::kWarpKernelThreads);
+  if (rc != FH_OK) return rc;
+  fh::compress_warp<DT, SIGMA, G><<<grid, fh::kWarpKernelThreads, pl.sm_total, stream>>>(pl, a);
+  return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+}
+
 template <int DT, bool SIGMA>
 int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
   if (!v.cta) {
     switch (v.G) {
-      case 1: return launch_fast_t<DT, SIGMA, 1, false>(pl, a, stream);
-      case 2: return launch_fast_t<DT, SIGMA, 2, false>(pl, a, stream);
-      case 4: return launch_fast_t<DT, SIGMA, 4, false>(pl, a, stream);
-      case 8: return launch_fast_t<DT, SIGMA, 8, false>(pl, a, stream);
+      case 1: return launch_warp_t<DT, SIGMA, 1>(pl, a, stream);
+      case 2: return launch_warp_t<DT, SIGMA, 2>(pl, a, stream);
+      case 4: return launch_warp_t<DT, SIGMA, 4>(pl, a, stream);
+      case 8: return launch_warp_t<DT, SIGMA, 8>(pl, a, stream);
     }
   } else {
     switch (v.G) {

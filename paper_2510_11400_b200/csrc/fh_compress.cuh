@@ -376,7 +376,7 @@ __device__ __forceinline__ void write_nonnormal(const Team& t, const Plan& pl, c
 template <int DT, int BITS>
 __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_red[kWarps * 4];
+  __shared__ double s_red[kWarps * 5];
   __shared__ uint32_t s_tile, s_skip;
   __shared__ unsigned long long s_base16;
 
@@ -392,6 +392,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
   uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
   constexpr uint32_t L = (1u << BITS) - 1u;
   const bool need_sigma = pl.mode == kModeAuto;
+  uint32_t rp = 0;  // reduction counter (see red_half)
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
 
   for (;;) {
@@ -435,7 +436,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
           hi = max_nan(hi, x);
         }
       }
-      team_minmax(team, lo, hi);
+      team_minmax(team, lo, hi, rp);
       if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && team.lane == 0)
         atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
 
@@ -450,7 +451,11 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
           ++ng;
         }
         long long Is, Iq;
-        team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq);
+        if (team.block)
+          team_sum2_wide(team, (long long)(int32_t)(as - ng * kMagicBits), (long long)(int32_t)(aq - ng * kMagicBits),
+                         Is, Iq, rp);
+        else
+          team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
         float tlo, thi;
         sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
         uint32_t cnt = 0;
@@ -460,7 +465,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
 #pragma unroll
           for (int k = 0; k < 4; ++k) cnt += (v[k] > thi) || (v[k] < tlo);
         }
-        n_out = team_sum_u32(team, cnt);
+        n_out = team_sum_u32(team, cnt, rp);
         if ((0.0f > thi) || (0.0f < tlo)) n_out -= 4u * groups - HW;  // padded zeros are not elements
         if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * HW) cls = kClsSalient;
       } else if (pl.mode == kModeAll) {
@@ -537,21 +542,347 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
 // =================================================================================================
 // Fast kernel
 // =================================================================================================
-// One plane per team and tile.  Warp-team variant (CTA = false): ppt = kThreads / team planes per
-// tile, each handled by `team` lanes of a warp.  CTA-team variant: one plane per tile, handled by
-// all threads.  Thread t of a team owns groups t, t + team, ..., (G of them), kept in registers.
-template <int DT, int G>
-struct Groups {
-  float v[G][4];
-};
+// One plane per team and tile.  Warp-team variant (CTA = false): kThreads / team planes per tile,
+// each handled by `team` lanes of a warp.  CTA-team variant: one plane per tile, handled by all
+// threads.  Thread t of a team owns groups t, t + team, ... (G of them) and keeps them in registers
+// for every pass.  FULL: groups == G * team, so no group needs a bounds check.
+//
+// One sweep over a plane: min/max -> (fixed-point moments -> thresholds -> count -> class) ->
+// codes, stored straight to the plane's slot together with its table entry.  Salient planes are
+// measured by their team right away; their writes wait for the tile's placement.
+template <int DT, bool SIGMA, int G, bool FULL>
+__device__ __forceinline__ void plane_sweep(const Team& team, uint32_t T, const Plan& pl, const Dest& d,
+                                            const CompressArgs& a, const uint8_t* plane, uint64_t gp, bool vec,
+                                            uint32_t& rp, Rec& r) {
+  const uint32_t groups = pl.groups, bits = (uint32_t)pl.bits, L = (1u << bits) - 1u;
+  float x[G][4];
+  float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
+  uint32_t ng = 0, npad = 0;  // groups of this thread; zero-padded elements among them
+#pragma unroll
+  for (int k = 0; k < G; ++k) {
+    const uint32_t g = team.lane + (uint32_t)k * T;
+    if (FULL || g < groups) {
+      if (vec) {
+        if (DT == kF32) {
+          const float4 t4 = reinterpret_cast<const float4*>(plane)[g];
+          x[k][0] = t4.x; x[k][1] = t4.y; x[k][2] = t4.z; x[k][3] = t4.w;
+        } else {
+          const uint2 t2 = reinterpret_cast<const uint2*>(plane)[g];
+          x[k][0] = __uint_as_float(t2.x << 16); x[k][1] = __uint_as_float(t2.x & 0xFFFF0000u);
+          x[k][2] = __uint_as_float(t2.y << 16); x[k][3] = __uint_as_float(t2.y & 0xFFFF0000u);
+        }
+        lo = min3_nan(lo, x[k][0], x[k][1]);
+        lo = min3_nan(lo, x[k][2], x[k][3]);
+        hi = max3_nan(hi, x[k][0], x[k][1]);
+        hi = max3_nan(hi, x[k][2], x[k][3]);
+      } else {  // plane not on a 16-byte boundary, possibly with a ragged last group
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t i = g * 4u + e;
+          const bool in = i < pl.HW;
+          x[k][e] = in ? load_elem<DT>(plane, i) : 0.0f;
+          if (in) {
+            lo = min_nan(lo, x[k][e]);
+            hi = max_nan(hi, x[k][e]);
+          } else {
+            ++npad;
+          }
+        }
+      }
+      ++ng;
+    }
+  }
+  team_minmax(team, lo, hi, rp);
+  if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && team.lane == 0)
+    atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+
+  uint32_t cls = kClsNormal, n_out = 0;
+  if (SIGMA) {
+    const SigmaScale sc = sigma_scale(lo, hi);
+    uint32_t as = 0, aq = 0;
+#pragma unroll
+    for (int k = 0; k < G; ++k)
+      if (FULL || team.lane + (uint32_t)k * T < groups) sigma_addends(x[k], sc, as, aq);
+    long long Is, Iq;
+    team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
+    float tlo, thi;
+    if (team.block) sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
+    else sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, tlo, thi);
+    uint32_t cnt = 0;
+    if (hi > thi || lo < tlo) {  // otherwise no element can lie outside: the count is zero
+      if (lo >= tlo) {           // nothing below: one compare per element
+#pragma unroll
+        for (int k = 0; k < G; ++k)
+          if (FULL || team.lane + (uint32_t)k * T < groups) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cnt += x[k][e] > thi;
+          }
+        if (0.0f > thi) cnt -= npad;  // padded zeros are not elements
+      } else {
+#pragma unroll
+        for (int k = 0; k < G; ++k)
+          if (FULL || team.lane + (uint32_t)k * T < groups) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) cnt += (x[k][e] > thi) || (x[k][e] < tlo);
+          }
+        if ((0.0f > thi) || (0.0f < tlo)) cnt -= npad;
+      }
+      cnt = team_sum_u32(team, cnt, rp);
+    }
+    n_out = cnt;
+    if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
+  } else if (pl.mode == kModeAll) {
+    cls = kClsSalient;
+  }
+
+  r.lo = 0.0f;
+  r.scale = 0.0f;
+  r.size = 0;
+  r.meta = cls | (n_out << 2);
+  if (cls != kClsNormal) return;
+  float inv, scale;
+  quant_params(lo, hi, L, inv, scale);
+  r.lo = lo;
+  r.scale = scale;
+  if (!d.fits) return;
+  uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
+  // Four codes of a group: sum of (magic + q_e) << (e * bits) minus the magic's contribution.
+  const uint32_t m1 = 1u << bits, m2 = m1 << bits, m3 = m2 << bits;
+  const uint32_t bias = kMagicBits * (1u + m1 + m2 + m3);
+#pragma unroll
+  for (int k = 0; k < G; ++k) {
+    const uint32_t g = team.lane + (uint32_t)k * T;
+    if (FULL || g < groups) {
+      uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF)) * m1;
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF)) * m2;
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF)) * m3;
+      word -= bias;
+      if (!vec) {  // ragged last group: elements past the plane carry no code
+        const uint32_t valid = min(4u, pl.HW - g * 4u);
+        if (valid < 4u) word &= (1u << (valid * bits)) - 1u;
+      }
+      if (bits == 2u) slot[g] = (uint8_t)word;
+      else if (bits == 4u) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;
+      else reinterpret_cast<uint32_t*>(slot)[g] = word;
+    }
+  }
+  // zero padding of the slot behind the codes
+  const uint32_t code_bytes = groups * bits / 2u;
+  if (code_bytes < pl.npay) {
+    for (uint32_t o = code_bytes + team.lane; o < a4(code_bytes); o += T) slot[o] = 0;
+    for (uint32_t o = a4(code_bytes) + 4u * team.lane; o < pl.npay; o += 4u * T)
+      *reinterpret_cast<uint32_t*>(slot + o) = 0u;
+  }
+  if (team.lane == 0) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
+}
+
+// -------------------------------------------------------------------------------------------------
+// Warp-team kernel: planes of at most 256 groups.  Eight consumer warps and one producer warp per
+// CTA.  The producer hands out tiles and streams them into a ring of shared-memory stages with bulk
+// copies; the consumer warps never wait for each other: each sweeps its own planes of a tile and
+// arrives on the stage's "empty" barrier when done.  The warp that finishes a tile last does the
+// tile-level book-keeping (scan word, placement of overflow parts); only warps that hold salient
+// planes wait for that placement.
+// -------------------------------------------------------------------------------------------------
+constexpr int kWarpKernelThreads = kThreads + 32;
+
+template <int DT, bool SIGMA, int G>
+__global__ void __launch_bounds__(kWarpKernelThreads, 2) compress_warp(const Plan pl, const CompressArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ double s_red[kWarps * 5];
+  __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
+  __shared__ uint32_t s_tiles[kMaxStages], s_done[kMaxStages], s_nonnormal[kMaxStages], s_skip[kMaxStages];
+  __shared__ volatile uint32_t s_placed[kMaxStages];  // tile + 1 once the tile's overflow parts are placed
+  __shared__ unsigned long long s_base16[kMaxStages];
+  __shared__ volatile uint32_t s_abort;
+
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+  const Dest d = make_dest(pl, a);
+  const uint32_t nstage = pl.nstage;
+  const uint32_t rec_stride = (20u * pl.ppt + 15u) & ~15u;
+  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+  if (tid == 0) {
+    for (uint32_t s = 0; s < nstage; ++s) {
+      mbar_init(&s_full[s], 1);
+      mbar_init(&s_empty[s], kWarps);
+      s_done[s] = 0;
+      s_nonnormal[s] = 0;
+      s_placed[s] = 0;
+    }
+    fence_mbar_init();
+    s_abort = 0;
+  }
+  __syncthreads();
+
+  if (warp == (uint32_t)kWarps) {
+    // ======================= producer =======================
+    if (lane == 0) {
+      uint32_t s = 0, empty_phase = 0;
+      for (uint32_t n = 0;; ++n) {
+        if (n >= nstage) {  // wait until every consumer warp is done with the previous tile of this stage
+          if (!mbar_wait_abortable(&s_empty[s], (empty_phase >> s) & 1u, 1u << 22, &s_abort)) {
+            s_abort = 1;
+            break;
+          }
+          empty_phase ^= 1u << s;
+        }
+        const uint32_t t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+        s_tiles[s] = t;
+        if (t >= pl.ntiles) {
+          mbar_arrive(&s_full[s]);  // wake the consumers: no more tiles
+          break;
+        }
+        const uint64_t p0 = (uint64_t)t * pl.ppt;
+        const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+        const uint32_t bytes = np * (uint32_t)pl.plane_bytes;
+        uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+        if ((bytes & 15u) == 0u) {
+          fence_proxy_async();
+          mbar_expect_tx(&s_full[s], bytes);
+          bulk_g2s(stage, a.src + p0 * pl.plane_bytes, bytes, &s_full[s]);
+        } else {  // ragged last tile of a tensor of ragged planes: plain loads by this thread
+          const uint16_t* g = reinterpret_cast<const uint16_t*>(a.src + p0 * pl.plane_bytes);
+          for (uint32_t i = 0; i < bytes / 2u; ++i) reinterpret_cast<uint16_t*>(stage)[i] = g[i];
+          mbar_arrive(&s_full[s]);
+        }
+        s = s + 1 == nstage ? 0 : s + 1;
+      }
+      if (s_abort) {  // wait (bounded) for copies still in flight before the CTA may exit
+        atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+        for (uint32_t k = 0; k < nstage; ++k) {
+          mbar_wait(&s_full[k], 0u, 1u << 16);
+          mbar_wait(&s_full[k], 1u, 1u << 16);
+        }
+      }
+    }
+  } else {
+    // ======================= consumers =======================
+    const Team team = make_team(pl.team, s_red);
+    const uint32_t T = pl.team;
+    const uint32_t my_team = tid / T;
+    uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
+    const bool vec = (pl.plane_bytes & 15u) == 0u;
+    const bool full = vec && pl.groups == (uint32_t)G * T;
+    uint32_t rp = 0, s = 0, full_phase = 0;
+    for (;;) {
+      bool ok = mbar_wait_abortable(&s_full[s], (full_phase >> s) & 1u, 1u << 22, &s_abort);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) {
+        s_abort = 1;
+        break;
+      }
+      full_phase ^= 1u << s;
+      const uint32_t tile = s_tiles[s];
+      if (tile >= pl.ntiles) break;
+      const uint64_t p0 = (uint64_t)tile * pl.ppt;
+      const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+      const uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+      Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec + (uint64_t)s * rec_stride);
+      uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + (uint64_t)s * rec_stride + 16u * pl.ppt);
+      const bool active = my_team < np;
+      const uint32_t lp = my_team;
+      const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
+      Rec r;
+      r.meta = kClsNormal;
+      SalientInfo info = {0, 0, 0, 0};
+      if (active) {
+        if (full) plane_sweep<DT, SIGMA, G, true>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
+        else plane_sweep<DT, SIGMA, G, false>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
+        if ((r.meta & 3u) != kClsNormal) {
+          info = salient_measure<DT>(team, pl, plane, sal);
+          r.size = info.size;
+          if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
+            r.meta = (r.meta & ~3u) | kClsRaw;
+            r.size = (uint32_t)pl.plane_bytes;
+          }
+        }
+        if (team.lane == 0) rec[lp] = r;
+      }
+      const bool mine_nonnormal = active && (r.meta & 3u) != kClsNormal;
+      const uint32_t handled = __popc(__ballot_sync(0xFFFFFFFFu, active && team.lane == 0));
+      const uint32_t nn = __popc(__ballot_sync(0xFFFFFFFFu, mine_nonnormal && team.lane == 0));
+      uint32_t last = 0;
+      __syncwarp();  // the records written by this warp's team leaders are ordered before lane 0's signal
+      if (lane == 0 && handled) {
+        if (nn) atomicAdd(&s_nonnormal[s], nn);
+        __threadfence_block();
+        last = (atomicAdd(&s_done[s], handled) + handled == np) ? 1u : 0u;
+      }
+      last = __shfl_sync(0xFFFFFFFFu, last, 0);
+      if (last) {  // this warp finished the tile: tile-level book-keeping
+        __threadfence_block();
+        const uint32_t tile_nn = *reinterpret_cast<volatile uint32_t*>(&s_nonnormal[s]);
+        if (tile_nn == 0) {
+          if (pl.mode != kModeOff) {
+            if (tile == 0) {
+              scan_publish(a.ts, tile, a.epoch, 2u, 0u);
+            } else {
+              scan_publish(a.ts, tile, a.epoch, 1u, 0u);
+              if ((tile & 31u) == 31u) {
+                unsigned long long excl = 0;
+                if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
+                  if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+                }
+                scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)excl);
+              }
+            }
+          }
+        } else {
+          tile_place(pl, a, d, tile, np, rec, roff, &s_base16[s], &s_skip[s]);
+          __threadfence_block();
+          __syncwarp();
+          if (lane == 0) s_placed[s] = tile + 1u;
+        }
+        if (lane == 0) {
+          s_done[s] = 0;
+          s_nonnormal[s] = 0;
+        }
+      }
+      if (nn) {  // teams of this warp hold salient / raw planes: wait for the placement, then write
+        bool placed = false;
+        for (uint32_t i = 0; i < (1u << 22); ++i) {
+          if (s_placed[s] == tile + 1u) {
+            placed = true;
+            break;
+          }
+          if (s_abort) break;
+          __nanosleep(64);
+        }
+        placed = __all_sync(0xFFFFFFFFu, placed);
+        if (!placed) {
+          s_abort = 1;
+          if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+        } else {
+          __threadfence_block();
+          if (mine_nonnormal && !s_skip[s]) {
+            SplitOut out;
+            out.slot = d.dst + pl.slots_off + (p0 + lp) * pl.npay;
+            out.ovf = d.dst + (s_base16[s] + roff[lp]) * 16ull;
+            out.npay = pl.npay;
+            if ((r.meta & 3u) == kClsRaw) raw_write(team, pl, plane, out);
+            else salient_write<DT>(team, pl, plane, info, sal, out);
+            if (team.lane == 0)
+              store_table_entry(d, p0 + lp, a16(r.size) > pl.npay ? (uint32_t)(s_base16[s] + roff[lp]) : 0u, r);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[s]);  // this warp no longer touches the stage or its records
+      if (s_abort) break;
+      s = s + 1 == nstage ? 0 : s + 1;
+    }
+  }
+  cta_exit(pl, a, d);
+}
 
 template <int DT, bool SIGMA, int G, bool CTA>
-__global__ void __launch_bounds__(kThreads) compress_fast(const Plan pl, const CompressArgs a) {
+__global__ void __launch_bounds__(kThreads, (G <= 8 ? 3 : 2)) compress_fast(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_red[kWarps * 4];
+  __shared__ double s_red[kWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
-  __shared__ uint32_t s_nonnormal, s_skip, s_abort;
+  __shared__ uint32_t s_nonnormal[2], s_skip, s_abort;  // s_nonnormal: one slot per tile parity
   __shared__ unsigned long long s_base16;
 
   const uint32_t tid = threadIdx.x;
@@ -561,155 +892,92 @@ __global__ void __launch_bounds__(kThreads) compress_fast(const Plan pl, const C
   const Team team = make_team(pl.team, s_red);
   const uint32_t T = CTA ? (uint32_t)kThreads : pl.team;
   const uint32_t my_team = CTA ? 0u : tid / T;
-  const uint32_t groups = pl.groups, bits = (uint32_t)pl.bits, L = (1u << bits) - 1u;
+  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
   const uint32_t nstage = pl.nstage;
+  const bool vec = (pl.plane_bytes & 15u) == 0u;
+  const bool full = vec && pl.groups == (uint32_t)G * T;
+  uint32_t rp = 0;
+  SalientInfo info = {0, 0, 0, 0};  // measurement of this team's salient plane, kept across the placement
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
 
   // ---- pipeline prologue: barriers, first tiles in flight
   if (tid == 0) {
     for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
     fence_mbar_init();
-    s_nonnormal = 0;
+    s_nonnormal[0] = 0;
+    s_nonnormal[1] = 0;
     s_abort = 0;
   }
   __syncthreads();
-  auto issue = [&](uint32_t s) {  // thread 0: take a ticket and start its load into stage s
+  // thread 0: take a ticket and start its load into stage s.  Tiles whose size is not a multiple of
+  // 16 bytes (only the last tile of a tensor of ragged planes) are not bulk-copied: they are loaded
+  // cooperatively when their turn comes.
+  auto issue = [&](uint32_t s) {
     const uint32_t t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
     s_tiles[s] = t;
     if (t < pl.ntiles) {
       const uint64_t p0 = (uint64_t)t * pl.ppt;
       const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
       const uint32_t bytes = np * (uint32_t)pl.plane_bytes;
-      fence_proxy_async();
-      mbar_expect_tx(&s_full[s], bytes);
-      bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + p0 * pl.plane_bytes, bytes, &s_full[s]);
+      if ((bytes & 15u) == 0u) {
+        fence_proxy_async();
+        mbar_expect_tx(&s_full[s], bytes);
+        bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + p0 * pl.plane_bytes, bytes, &s_full[s]);
+      }
     }
   };
   if (tid == 0)
     for (uint32_t s = 0; s < nstage; ++s) issue(s);
   __syncthreads();
 
+  uint32_t uses[kMaxStages] = {0, 0, 0, 0};  // completed bulk loads per stage (barrier phase)
   for (uint32_t it = 0;; ++it) {
     const uint32_t s = it % nstage;
     const uint32_t tile = s_tiles[s];
     if (tile >= pl.ntiles) break;
-    const uint32_t parity = (it / nstage) & 1u;
-    if (!mbar_wait(&s_full[s], parity, 1u << 22)) s_abort = 1;  // the load never arrived
-    __syncthreads();
-    if (s_abort) break;
     const uint64_t p0 = (uint64_t)tile * pl.ppt;
     const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
-    const uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+    uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+    const uint32_t tile_bytes = np * (uint32_t)pl.plane_bytes;
+    bool ready = true;
+    if ((tile_bytes & 15u) == 0u) {
+      uint32_t u = 0;
+#pragma unroll
+      for (int k = 0; k < kMaxStages; ++k)
+        if (k == (int)s) u = uses[k]++;
+      ready = mbar_wait(&s_full[s], u & 1u, 1u << 22);
+      ready = __all_sync(0xFFFFFFFFu, ready);
+      if (!ready) s_abort = 1;  // the load never arrived
+    } else {
+      __syncthreads();  // ragged last tile: plain loads by everybody
+      for (uint32_t i = tid; i < tile_bytes / 2u; i += kThreads)
+        reinterpret_cast<uint16_t*>(stage)[i] = reinterpret_cast<const uint16_t*>(a.src + p0 * pl.plane_bytes)[i];
+      __syncthreads();
+    }
 
-    if (CTA || my_team < np) {
+    if (ready && (CTA || my_team < np)) {
       const uint32_t lp = my_team;
       const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
-      const uint64_t gp = p0 + lp;
-      // ---- the thread's groups, in registers for every pass
-      Groups<DT, G> x;
-      float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
-      uint32_t ng = 0;
-#pragma unroll
-      for (int k = 0; k < G; ++k) {
-        const uint32_t g = team.lane + (uint32_t)k * T;
-        if (g < groups) {
-          if (DT == kF32) {
-            const float4 t4 = reinterpret_cast<const float4*>(plane)[g];
-            x.v[k][0] = t4.x; x.v[k][1] = t4.y; x.v[k][2] = t4.z; x.v[k][3] = t4.w;
-          } else {
-            const uint2 t2 = reinterpret_cast<const uint2*>(plane)[g];
-            x.v[k][0] = __uint_as_float(t2.x << 16); x.v[k][1] = __uint_as_float(t2.x & 0xFFFF0000u);
-            x.v[k][2] = __uint_as_float(t2.y << 16); x.v[k][3] = __uint_as_float(t2.y & 0xFFFF0000u);
-          }
-          lo = min3_nan(lo, x.v[k][0], x.v[k][1]);
-          lo = min3_nan(lo, x.v[k][2], x.v[k][3]);
-          hi = max3_nan(hi, x.v[k][0], x.v[k][1]);
-          hi = max3_nan(hi, x.v[k][2], x.v[k][3]);
-          ++ng;
-        }
-      }
-      team_minmax(team, lo, hi);
-      if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && team.lane == 0)
-        atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
-
-      uint32_t cls = kClsNormal, n_out = 0;
-      if (SIGMA) {
-        const SigmaScale sc = sigma_scale(lo, hi);
-        uint32_t as = 0, aq = 0;
-#pragma unroll
-        for (int k = 0; k < G; ++k)
-          if (team.lane + (uint32_t)k * T < groups) sigma_addends(x.v[k], sc, as, aq);
-        long long Is, Iq;
-        team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq);
-        float tlo, thi;
-        sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
-        uint32_t cnt = 0;
-        if (hi > thi || lo < tlo) {  // otherwise no element can lie outside: the count is zero
-          if (lo >= tlo) {           // nothing below: one compare per element
-#pragma unroll
-            for (int k = 0; k < G; ++k)
-              if (team.lane + (uint32_t)k * T < groups) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) cnt += x.v[k][e] > thi;
-              }
-          } else {
-#pragma unroll
-            for (int k = 0; k < G; ++k)
-              if (team.lane + (uint32_t)k * T < groups) {
-#pragma unroll
-                for (int e = 0; e < 4; ++e) cnt += (x.v[k][e] > thi) || (x.v[k][e] < tlo);
-              }
-          }
-          cnt = team_sum_u32(team, cnt);
-        }
-        n_out = cnt;
-        if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
-      } else if (pl.mode == kModeAll) {
-        cls = kClsSalient;
-      }
-
       Rec r;
-      r.lo = 0.0f;
-      r.scale = 0.0f;
-      r.size = 0;
-      r.meta = cls | (n_out << 2);
-      if (cls == kClsNormal) {
-        float inv, scale;
-        quant_params(lo, hi, L, inv, scale);
-        r.lo = lo;
-        r.scale = scale;
-        if (d.fits) {
-          uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
-#pragma unroll
-          for (int k = 0; k < G; ++k) {
-            const uint32_t g = team.lane + (uint32_t)k * T;
-            if (g < groups) {
-              uint32_t word = 0;
-#pragma unroll
-              for (int e = 0; e < 4; ++e) word |= quant_code(x.v[k][e], lo, inv, L) << (e * bits);
-              if (bits == 2u) slot[g] = (uint8_t)word;
-              else if (bits == 4u) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;
-              else reinterpret_cast<uint32_t*>(slot)[g] = word;
-            }
-          }
-          // zero padding of the slot behind the codes
-          const uint32_t code_bytes = groups * bits / 2u;
-          if (code_bytes < pl.npay) {
-            for (uint32_t o = code_bytes + team.lane; o < a4(code_bytes); o += T) slot[o] = 0;
-            for (uint32_t o = a4(code_bytes) + 4u * team.lane; o < pl.npay; o += 4u * T)
-              *reinterpret_cast<uint32_t*>(slot + o) = 0u;
-          }
-          if (team.lane == 0) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
+      if (full) plane_sweep<DT, SIGMA, G, true>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
+      else plane_sweep<DT, SIGMA, G, false>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
+      if ((r.meta & 3u) != kClsNormal) {
+        info = salient_measure<DT>(team, pl, plane, sal);
+        r.size = info.size;
+        if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
+          r.meta = (r.meta & ~3u) | kClsRaw;
+          r.size = (uint32_t)pl.plane_bytes;
         }
-      } else if (team.lane == 0) {
-        atomicAdd(&s_nonnormal, 1u);
+        if (team.lane == 0) atomicAdd(&s_nonnormal[it & 1u], 1u);
       }
       if (team.lane == 0) rec[lp] = r;
     }
     __syncthreads();
+    if (s_abort) break;
 
-    const uint32_t nonnormal = s_nonnormal;
-    if (nonnormal == 0) {
+    // Warps may run one tile ahead of each other between barriers, hence the flag per tile parity;
+    // it is cleared only behind the extra barriers of the slow path.
+    if (s_nonnormal[it & 1u] == 0) {
       // ---- common case: nothing to place; publish a zero aggregate, every 32nd tile resolves
       if (pl.mode != kModeOff && tid < 32) {
         if (tile == 0) {
@@ -726,55 +994,41 @@ __global__ void __launch_bounds__(kThreads) compress_fast(const Plan pl, const C
         }
       }
     } else {
-      // ---- block-wise path for the salient planes of this tile (shared-memory resident)
-      const Team wteam = CTA ? team : make_warp_team(s_red);
-      const uint32_t nw = CTA ? 1u : (uint32_t)kWarps, me = CTA ? 0u : tid >> 5;
-      uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)me * pl.sm_sal_stride);
-      uint32_t seen = 0;
-      for (uint32_t lp = 0; lp < np; ++lp) {
-        if ((rec[lp].meta & 3u) == kClsNormal) continue;
-        if (seen++ % nw != me) continue;
-        const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
-        const SalientInfo info = salient_measure<DT>(wteam, pl, plane, sal);
-        if (wteam.lane == 0) {
-          if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
-            rec[lp].meta = (rec[lp].meta & ~3u) | kClsRaw;
-            rec[lp].size = (uint32_t)pl.plane_bytes;
-          } else {
-            rec[lp].size = info.size;
-          }
-        }
-      }
-      __syncthreads();
+      // ---- place the overflow parts of this tile, then the owning teams write their planes
       if (tid < 32) tile_place(pl, a, d, tile, np, rec, roff, &s_base16, &s_skip);
       __syncthreads();
-      if (!s_skip) {
-        const unsigned long long base16 = s_base16;
-        seen = 0;
-        for (uint32_t lp = 0; lp < np; ++lp) {
-          if ((rec[lp].meta & 3u) == kClsNormal) continue;
-          if (seen++ % nw != me) continue;
+      if (!s_skip && (CTA || my_team < np)) {
+        const uint32_t lp = my_team;
+        const Rec r = rec[lp];
+        if ((r.meta & 3u) != kClsNormal) {
           const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
-          write_nonnormal<DT>(wteam, pl, d, plane, p0 + lp, rec[lp], base16 + roff[lp], sal);
+          SplitOut out;
+          out.slot = d.dst + pl.slots_off + (p0 + lp) * pl.npay;
+          out.ovf = d.dst + (s_base16 + roff[lp]) * 16ull;
+          out.npay = pl.npay;
+          if ((r.meta & 3u) == kClsRaw) {
+            raw_write(team, pl, plane, out);
+          } else {  // the team's scratch and `info` still hold the measurement of this plane
+            salient_write<DT>(team, pl, plane, info, sal, out);
+          }
+          if (team.lane == 0)
+            store_table_entry(d, p0 + lp, a16(r.size) > pl.npay ? (uint32_t)(s_base16 + roff[lp]) : 0u, r);
         }
       }
       __syncthreads();
-      if (tid == 0) s_nonnormal = 0;
+      if (tid == 0) s_nonnormal[it & 1u] = 0;
     }
     // ---- the stage is free: next ticket, next load
     if (tid == 0) issue(s);
-    __syncthreads();
   }
 
-  if (s_abort) {  // a load timed out: report, then wait (bounded) for the copies still in flight
-    if (tid == 0) {
-      atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-      for (uint32_t s = 0; s < nstage; ++s)
-        if (s_tiles[s] < pl.ntiles) {
-          mbar_wait(&s_full[s], 0u, 1u << 16);
-          mbar_wait(&s_full[s], 1u, 1u << 16);
-        }
-    }
+  if (s_abort && tid == 0) {  // a load timed out: report, then wait (bounded) for copies still in flight
+    atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+    for (uint32_t s = 0; s < nstage; ++s)
+      if (s_tiles[s] < pl.ntiles) {
+        mbar_wait(&s_full[s], 0u, 1u << 16);
+        mbar_wait(&s_full[s], 1u, 1u << 16);
+      }
   }
   cta_exit(pl, a, d);
 }

@@ -131,6 +131,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait that also gives up when *abort becomes non-zero.
+__device__ __forceinline__ bool mbar_wait_abortable(uint64_t* bar, uint32_t parity, uint32_t limit,
+                                                    const volatile uint32_t* abort) {
+  for (uint32_t i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 32) {
+      if (*abort) return false;
+      __nanosleep(32);
+    }
+  }
+  return false;
+}
 // Bounded wait: false when the phase did not complete within `limit` polls.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit) {
   for (uint32_t i = 0; i < limit; ++i) {
@@ -223,8 +238,9 @@ __device__ __forceinline__ void sigma_addends(const float v[4], const SigmaScale
   aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
 }
 // Thresholds mu +- 3 sigma from the exact integer sums.
-__device__ __forceinline__ void sigma_thresholds(long long Is, long long Iq, const SigmaScale& sc, double inv_hw,
-                                                 float& tlo, float& thi) {
+template <typename I>
+__device__ __forceinline__ void sigma_thresholds(I Is, I Iq, const SigmaScale& sc, double inv_hw, float& tlo,
+                                                 float& thi) {
   const double ps = __hiloint2double((1023 - sc.ks) << 20, 0);  // 2^-ks
   const double pq = __hiloint2double((1023 - sc.kq) << 20, 0);  // 2^-kq
   const double mu = __dmul_rn(__dmul_rn((double)Is, ps), inv_hw);
@@ -269,7 +285,7 @@ struct Team {
   uint32_t lane;   // this thread's index inside the team
   uint32_t mask;   // warp member mask of the team (sub-warp teams)
   bool block;      // the team is the whole CTA
-  double* red;     // shared scratch for CTA-wide reductions: kWarps * 4 doubles
+  double* red;     // shared scratch for CTA-wide reductions: kWarps * 5 doubles (see red_half, team_excl_scan)
 };
 
 __device__ __forceinline__ Team make_team(uint32_t team_size, double* red) {
@@ -304,15 +320,22 @@ __device__ __forceinline__ void team_sync(const Team& t) {
   else __syncwarp(t.mask);
 }
 
+// CTA-wide reductions exchange per-warp partials through t.red, which is split in two halves used
+// alternately (`rp` counts the reductions of this thread), so that one barrier per reduction
+// suffices: a half is rewritten only after the barrier of the reduction in between.
+__device__ __forceinline__ double* red_half(const Team& t, uint32_t& rp) {
+  double* r = t.red + ((rp++) & 1u) * (kWarps * 2);
+  return r;
+}
+
 // min / max over the team with NaN propagation (hardware warp reduction for fp32).
-__device__ __forceinline__ void team_minmax(const Team& t, float& lo, float& hi) {
+__device__ __forceinline__ void team_minmax(const Team& t, float& lo, float& hi, uint32_t& rp) {
   if (!t.block && t.size == 1u) return;
   asm volatile("redux.sync.min.NaN.f32 %0, %0, %1;" : "+f"(lo) : "r"(t.mask));
   asm volatile("redux.sync.max.NaN.f32 %0, %0, %1;" : "+f"(hi) : "r"(t.mask));
   if (t.block) {
-    float* r = reinterpret_cast<float*>(t.red);
+    float* r = reinterpret_cast<float*>(red_half(t, rp));
     const uint32_t warp = threadIdx.x >> 5;
-    __syncthreads();
     if ((threadIdx.x & 31u) == 0) {
       r[warp * 2] = lo;
       r[warp * 2 + 1] = hi;
@@ -328,9 +351,10 @@ __device__ __forceinline__ void team_minmax(const Team& t, float& lo, float& hi)
   }
 }
 
-// Sum of two int32 per thread over the team, returned as 64-bit integers.  Within a warp the sums fit
-// 32 bits (see the callers); warps are combined in 64 bits.
-__device__ __forceinline__ void team_sum2(const Team& t, int32_t a, int32_t b, long long& A, long long& B) {
+// Sum of two int32 per thread over the team, returned as 64-bit integers.  The sums over one warp
+// must fit 32 bits (at most 512 groups per warp, see sigma_addends); warps are combined in 64 bits.
+__device__ __forceinline__ void team_sum2(const Team& t, int32_t a, int32_t b, long long& A, long long& B,
+                                          uint32_t& rp) {
   if (!t.block && t.size == 1u) {
     A = a;
     B = b;
@@ -341,9 +365,8 @@ __device__ __forceinline__ void team_sum2(const Team& t, int32_t a, int32_t b, l
   A = a;
   B = b;
   if (t.block) {
-    long long* r = reinterpret_cast<long long*>(t.red);
+    long long* r = reinterpret_cast<long long*>(red_half(t, rp));
     const uint32_t warp = threadIdx.x >> 5;
-    __syncthreads();
     if ((threadIdx.x & 31u) == 0) {
       r[warp * 2] = a;
       r[warp * 2 + 1] = b;
@@ -359,13 +382,36 @@ __device__ __forceinline__ void team_sum2(const Team& t, int32_t a, int32_t b, l
   }
 }
 
-__device__ __forceinline__ uint32_t team_sum_u32(const Team& t, uint32_t v) {
+// The same for per-thread partial sums that may exceed 32 bits once added over a warp (CTA teams on
+// very large planes): 64-bit shuffles inside the warp.
+__device__ __forceinline__ void team_sum2_wide(const Team& t, long long a, long long b, long long& A, long long& B,
+                                               uint32_t& rp) {
+  for (uint32_t o = 16; o > 0; o >>= 1) {
+    a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
+    b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
+  }
+  long long* r = reinterpret_cast<long long*>(red_half(t, rp));
+  const uint32_t warp = threadIdx.x >> 5;
+  if ((threadIdx.x & 31u) == 0) {
+    r[warp * 2] = a;
+    r[warp * 2 + 1] = b;
+  }
+  __syncthreads();
+  A = 0;
+  B = 0;
+#pragma unroll
+  for (int k = 0; k < kWarps; ++k) {
+    A += r[k * 2];
+    B += r[k * 2 + 1];
+  }
+}
+
+__device__ __forceinline__ uint32_t team_sum_u32(const Team& t, uint32_t v, uint32_t& rp) {
   if (!t.block && t.size == 1u) return v;
   asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(v) : "r"(t.mask));
   if (t.block) {
-    uint32_t* r = reinterpret_cast<uint32_t*>(t.red);
+    uint32_t* r = reinterpret_cast<uint32_t*>(red_half(t, rp));
     const uint32_t warp = threadIdx.x >> 5;
-    __syncthreads();
     if ((threadIdx.x & 31u) == 0) r[warp] = v;
     __syncthreads();
     v = 0;
@@ -390,7 +436,7 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
     }
     total = __shfl_sync(t.mask, incl, t.size - 1u, t.size);
   } else {
-    uint32_t* r = reinterpret_cast<uint32_t*>(t.red);
+    uint32_t* r = reinterpret_cast<uint32_t*>(t.red + kWarps * 4);  // region of its own, behind the two halves
     const uint32_t wl = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     for (uint32_t o = 1; o < 32u; o <<= 1) {
       const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
