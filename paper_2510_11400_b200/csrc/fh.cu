@@ -119,7 +119,7 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     if (pl.groups <= 256) {
       uint32_t t = pow2_ceil((pl.groups + 7) / 8);
       pl.team = t > 32 ? 32 : t;
-      v.G = (int)pow2_ceil((pl.groups + pl.team - 1) / pl.team);
+      v.G = 8;  // the warp-team kernels keep eight groups per thread
       pl.ppt = fh::kThreads / pl.team;
     } else {
       v.cta = true;
@@ -281,40 +281,48 @@ int launch_generic_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t str
   return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
-template <int DT, bool SIGMA, int G, bool CTA>
-int launch_fast_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
+template <int DT, bool SIGMA, int G>
+int launch_cta_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
   int grid = 0;
-  int rc = grid_for(fh::compress_fast<DT, SIGMA, G, CTA>, pl.sm_total, pl.ntiles, &grid);
+  int rc = grid_for(fh::compress_cta<DT, SIGMA, G>, pl.sm_total, pl.ntiles, &grid);
   if (rc != FH_OK) return rc;
-  fh::compress_fast<DT, SIGMA, G, CTA><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
+  fh::compress_cta<DT, SIGMA, G><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
   return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
-template <int DT, bool SIGMA, int G>
+template <int DT, bool SIGMA, int TT, bool FULLVEC>
 int launch_warp_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
   int grid = 0;
-  int rc = grid_for(fh::compress_warp<DT, SIGMA, G>, pl.sm_total, pl.ntiles, &grid, fh::kWarpKernelThreads);
+  int rc = grid_for(fh::compress_warp<DT, SIGMA, TT, FULLVEC>, pl.sm_total, pl.ntiles, &grid, fh::kWarpKernelThreads);
   if (rc != FH_OK) return rc;
-  fh::compress_warp<DT, SIGMA, G><<<grid, fh::kWarpKernelThreads, pl.sm_total, stream>>>(pl, a);
+  fh::compress_warp<DT, SIGMA, TT, FULLVEC><<<grid, fh::kWarpKernelThreads, pl.sm_total, stream>>>(pl, a);
   return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+}
+
+template <int DT, bool SIGMA, bool FULLVEC>
+int launch_warp_tt(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
+  switch (pl.team) {
+    case 1: return launch_warp_t<DT, SIGMA, 1, FULLVEC>(pl, a, stream);
+    case 2: return launch_warp_t<DT, SIGMA, 2, FULLVEC>(pl, a, stream);
+    case 4: return launch_warp_t<DT, SIGMA, 4, FULLVEC>(pl, a, stream);
+    case 8: return launch_warp_t<DT, SIGMA, 8, FULLVEC>(pl, a, stream);
+    case 16: return launch_warp_t<DT, SIGMA, 16, FULLVEC>(pl, a, stream);
+    case 32: return launch_warp_t<DT, SIGMA, 32, FULLVEC>(pl, a, stream);
+  }
+  return FH_ERR_UNSUPPORTED;
 }
 
 template <int DT, bool SIGMA>
 int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
   if (!v.cta) {
-    switch (v.G) {
-      case 1: return launch_warp_t<DT, SIGMA, 1>(pl, a, stream);
-      case 2: return launch_warp_t<DT, SIGMA, 2>(pl, a, stream);
-      case 4: return launch_warp_t<DT, SIGMA, 4>(pl, a, stream);
-      case 8: return launch_warp_t<DT, SIGMA, 8>(pl, a, stream);
-    }
-  } else {
-    switch (v.G) {
-      case 2: return launch_fast_t<DT, SIGMA, 2, true>(pl, a, stream);
-      case 4: return launch_fast_t<DT, SIGMA, 4, true>(pl, a, stream);
-      case 8: return launch_fast_t<DT, SIGMA, 8, true>(pl, a, stream);
-      case 16: return launch_fast_t<DT, SIGMA, 16, true>(pl, a, stream);
-    }
+    const bool fullvec = pl.plane_bytes % 16 == 0 && pl.HW % 4 == 0 && pl.groups == 8u * pl.team;
+    return fullvec ? launch_warp_tt<DT, SIGMA, true>(pl, a, stream) : launch_warp_tt<DT, SIGMA, false>(pl, a, stream);
+  }
+  switch (v.G) {
+    case 2: return launch_cta_t<DT, SIGMA, 2>(pl, a, stream);
+    case 4: return launch_cta_t<DT, SIGMA, 4>(pl, a, stream);
+    case 8: return launch_cta_t<DT, SIGMA, 8>(pl, a, stream);
+    case 16: return launch_cta_t<DT, SIGMA, 16>(pl, a, stream);
   }
   return FH_ERR_UNSUPPORTED;
 }

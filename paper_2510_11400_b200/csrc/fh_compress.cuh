@@ -104,7 +104,7 @@ __device__ __forceinline__ uint32_t block_codes(const uint8_t* plane, int H, int
 // scratch: rowp[0..H] = CSR row pointers, blk_a[b] = 1 for dense blocks, blk_b[b] = rank of block b
 // among the dense blocks, blk_c[b] = index of the block's first verbatim value.
 template <int DT>
-__device__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint8_t* plane, uint32_t* sal) {
+__device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint8_t* plane, uint32_t* sal) {
   uint32_t* rowp = sal;
   uint32_t* blk_a = sal + pl.H + 1;
   uint32_t* blk_b = blk_a + pl.nblk;
@@ -159,7 +159,7 @@ __device__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint
 
 // Block-wise path, writing part; `sal` holds what salient_measure left.
 template <int DT>
-__device__ void salient_write(const Team& t, const Plan& pl, const uint8_t* plane, const SalientInfo& info,
+__device__ __noinline__ void salient_write(const Team& t, const Plan& pl, const uint8_t* plane, const SalientInfo& info,
                               const uint32_t* sal, const SplitOut& out) {
   const uint32_t* rowp = sal;
   const uint32_t* blk_a = sal + pl.H + 1;
@@ -211,7 +211,7 @@ __device__ void salient_write(const Team& t, const Plan& pl, const uint8_t* plan
 }
 
 // Raw plane: verbatim copy through the slot into the overflow part, zero padded.
-__device__ __forceinline__ void raw_write(const Team& t, const Plan& pl, const uint8_t* plane, const SplitOut& out) {
+__device__ __noinline__ void raw_write(const Team& t, const Plan& pl, const uint8_t* plane, const SplitOut& out) {
   const uint32_t n = (uint32_t)pl.plane_bytes, end = max(pl.npay, a16(n));
   for (uint32_t o = 2u * t.lane; o < end; o += 2u * t.size)
     out.st16(o, o < n ? (uint32_t)*reinterpret_cast<const uint16_t*>(plane + o) : 0u);
@@ -243,7 +243,7 @@ __device__ __forceinline__ Dest make_dest(const Plan& pl, const CompressArgs& a)
 // rec[].  Computes each plane's overflow offset (roff[], 16-byte units relative to the tile),
 // publishes the tile's aggregate and, when the tile needs it or is a 32nd tile, resolves the tile's
 // base.  Returns through shared variables: *s_base16 (absolute, 16-byte units), *s_skip.
-__device__ __forceinline__ void tile_place(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
+__device__ __noinline__ void tile_place(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
                                            uint32_t np, const Rec* rec, uint32_t* roff,
                                            unsigned long long* s_base16, uint32_t* s_skip) {
   const uint32_t lane = threadIdx.x & 31u;
@@ -550,24 +550,51 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
 // One sweep over a plane: min/max -> (fixed-point moments -> thresholds -> count -> class) ->
 // codes, stored straight to the plane's slot together with its table entry.  Salient planes are
 // measured by their team right away; their writes wait for the tile's placement.
-template <int DT, bool SIGMA, int G, bool FULL>
-__device__ __forceinline__ void plane_sweep(const Team& team, uint32_t T, const Plan& pl, const Dest& d,
-                                            const CompressArgs& a, const uint8_t* plane, uint64_t gp, bool vec,
-                                            uint32_t& rp, Rec& r) {
-  const uint32_t groups = pl.groups, bits = (uint32_t)pl.bits, L = (1u << bits) - 1u;
+// Codes of the thread's groups, packed and stored to the plane's slot (used inside plane_sweep, on
+// its register-resident groups x[k][e]).  Four codes of a group are the sum of
+// (magic + q_e) << (e * BITS) minus the magic's contribution.
+#define FH_STORE_CODES(BITS)                                                                                  \
+  {                                                                                                           \
+    constexpr uint32_t bias = kMagicBits * (1u + (1u << (BITS)) + (1u << (2 * (BITS))) + (1u << (3 * (BITS)))); \
+    _Pragma("unroll") for (int k = 0; k < G; ++k) {                                                           \
+      const uint32_t g = lane + (uint32_t)(k * TT);                                                           \
+      if (FULL || g < groups) {                                                                               \
+        uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));                     \
+        word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF)) << (BITS);                   \
+        word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF)) << (2 * (BITS));             \
+        word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF)) << (3 * (BITS));             \
+        word -= bias;                                                                                         \
+        if (!VEC) { /* ragged last group: elements past the plane carry no code */                            \
+          const uint32_t valid = min(4u, pl.HW - g * 4u);                                                     \
+          if (valid < 4u) word &= (1u << (valid * (BITS))) - 1u;                                              \
+        }                                                                                                     \
+        if ((BITS) == 2) slot[g] = (uint8_t)word;                                                             \
+        else if ((BITS) == 4) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;                          \
+        else reinterpret_cast<uint32_t*>(slot)[g] = word;                                                     \
+      }                                                                                                       \
+    }                                                                                                         \
+  }
+
+// TT: team size (1..32, or kThreads for the CTA team), a compile-time constant so that the strides
+// between a thread's groups are immediates.  FULL: groups == G * TT.  VEC: planes are whole 16-byte
+// chunks (vector loads, no ragged last group).
+template <int DT, bool SIGMA, int G, int TT, bool FULL, bool VEC>
+__device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, const Dest& d, const CompressArgs& a,
+                                            const uint8_t* plane, uint64_t gp, uint32_t& rp, Rec& r) {
+  const uint32_t groups = pl.groups, lane = team.lane;
   float x[G][4];
   float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
   uint32_t ng = 0, npad = 0;  // groups of this thread; zero-padded elements among them
 #pragma unroll
   for (int k = 0; k < G; ++k) {
-    const uint32_t g = team.lane + (uint32_t)k * T;
+    const uint32_t g = lane + (uint32_t)(k * TT);
     if (FULL || g < groups) {
-      if (vec) {
+      if (VEC) {
         if (DT == kF32) {
-          const float4 t4 = reinterpret_cast<const float4*>(plane)[g];
+          const float4 t4 = (reinterpret_cast<const float4*>(plane) + lane)[k * TT];
           x[k][0] = t4.x; x[k][1] = t4.y; x[k][2] = t4.z; x[k][3] = t4.w;
         } else {
-          const uint2 t2 = reinterpret_cast<const uint2*>(plane)[g];
+          const uint2 t2 = (reinterpret_cast<const uint2*>(plane) + lane)[k * TT];
           x[k][0] = __uint_as_float(t2.x << 16); x[k][1] = __uint_as_float(t2.x & 0xFFFF0000u);
           x[k][2] = __uint_as_float(t2.y << 16); x[k][3] = __uint_as_float(t2.y & 0xFFFF0000u);
         }
@@ -593,7 +620,7 @@ __device__ __forceinline__ void plane_sweep(const Team& team, uint32_t T, const 
     }
   }
   team_minmax(team, lo, hi, rp);
-  if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && team.lane == 0)
+  if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && lane == 0)
     atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
 
   uint32_t cls = kClsNormal, n_out = 0;
@@ -602,30 +629,31 @@ __device__ __forceinline__ void plane_sweep(const Team& team, uint32_t T, const 
     uint32_t as = 0, aq = 0;
 #pragma unroll
     for (int k = 0; k < G; ++k)
-      if (FULL || team.lane + (uint32_t)k * T < groups) sigma_addends(x[k], sc, as, aq);
+      if (FULL || lane + (uint32_t)(k * TT) < groups) sigma_addends4(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
+    if (FULL) ng = G;
     long long Is, Iq;
     team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
     float tlo, thi;
-    if (team.block) sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
+    if (TT > 32) sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
     else sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, tlo, thi);
     uint32_t cnt = 0;
     if (hi > thi || lo < tlo) {  // otherwise no element can lie outside: the count is zero
       if (lo >= tlo) {           // nothing below: one compare per element
 #pragma unroll
         for (int k = 0; k < G; ++k)
-          if (FULL || team.lane + (uint32_t)k * T < groups) {
+          if (FULL || lane + (uint32_t)(k * TT) < groups) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) cnt += x[k][e] > thi;
           }
-        if (0.0f > thi) cnt -= npad;  // padded zeros are not elements
+        if (!VEC && 0.0f > thi) cnt -= npad;  // padded zeros are not elements
       } else {
 #pragma unroll
         for (int k = 0; k < G; ++k)
-          if (FULL || team.lane + (uint32_t)k * T < groups) {
+          if (FULL || lane + (uint32_t)(k * TT) < groups) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) cnt += (x[k][e] > thi) || (x[k][e] < tlo);
           }
-        if ((0.0f > thi) || (0.0f < tlo)) cnt -= npad;
+        if (!VEC && ((0.0f > thi) || (0.0f < tlo))) cnt -= npad;
       }
       cnt = team_sum_u32(team, cnt, rp);
     }
@@ -640,235 +668,318 @@ __device__ __forceinline__ void plane_sweep(const Team& team, uint32_t T, const 
   r.size = 0;
   r.meta = cls | (n_out << 2);
   if (cls != kClsNormal) return;
+  const uint32_t bits = (uint32_t)pl.bits;
   float inv, scale;
-  quant_params(lo, hi, L, inv, scale);
+  quant_params(lo, hi, (1u << bits) - 1u, inv, scale);
   r.lo = lo;
   r.scale = scale;
   if (!d.fits) return;
   uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
-  // Four codes of a group: sum of (magic + q_e) << (e * bits) minus the magic's contribution.
-  const uint32_t m1 = 1u << bits, m2 = m1 << bits, m3 = m2 << bits;
-  const uint32_t bias = kMagicBits * (1u + m1 + m2 + m3);
-#pragma unroll
-  for (int k = 0; k < G; ++k) {
-    const uint32_t g = team.lane + (uint32_t)k * T;
-    if (FULL || g < groups) {
-      uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF)) * m1;
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF)) * m2;
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF)) * m3;
-      word -= bias;
-      if (!vec) {  // ragged last group: elements past the plane carry no code
-        const uint32_t valid = min(4u, pl.HW - g * 4u);
-        if (valid < 4u) word &= (1u << (valid * bits)) - 1u;
-      }
-      if (bits == 2u) slot[g] = (uint8_t)word;
-      else if (bits == 4u) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;
-      else reinterpret_cast<uint32_t*>(slot)[g] = word;
-    }
-  }
+  if (bits == 2u) FH_STORE_CODES(2)
+  else if (bits == 4u) FH_STORE_CODES(4)
+  else FH_STORE_CODES(8)
   // zero padding of the slot behind the codes
   const uint32_t code_bytes = groups * bits / 2u;
   if (code_bytes < pl.npay) {
-    for (uint32_t o = code_bytes + team.lane; o < a4(code_bytes); o += T) slot[o] = 0;
-    for (uint32_t o = a4(code_bytes) + 4u * team.lane; o < pl.npay; o += 4u * T)
+    for (uint32_t o = code_bytes + lane; o < a4(code_bytes); o += TT) slot[o] = 0;
+    for (uint32_t o = a4(code_bytes) + 4u * lane; o < pl.npay; o += 4u * TT)
       *reinterpret_cast<uint32_t*>(slot + o) = 0u;
   }
-  if (team.lane == 0) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
+  if (lane == 0) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
+}
+
+// Picks the specialisation of the sweep.  FULLVEC kernels are launched only for planes of exactly
+// G * TT whole groups, so they carry nothing but the lean variant; the others choose at run time.
+template <int DT, bool SIGMA, int G, int TT, bool FULLVEC>
+__device__ __forceinline__ void plane_sweep_any(const Team& team, const Plan& pl, const Dest& d,
+                                                const CompressArgs& a, const uint8_t* plane, uint64_t gp,
+                                                bool vec, uint32_t& rp, Rec& r) {
+  if (FULLVEC) plane_sweep<DT, SIGMA, G, TT, true, true>(team, pl, d, a, plane, gp, rp, r);
+  else if (vec) plane_sweep<DT, SIGMA, G, TT, false, true>(team, pl, d, a, plane, gp, rp, r);
+  else plane_sweep<DT, SIGMA, G, TT, false, false>(team, pl, d, a, plane, gp, rp, r);
 }
 
 // -------------------------------------------------------------------------------------------------
 // Warp-team kernel: planes of at most 256 groups.  Eight consumer warps and one producer warp per
 // CTA.  The producer hands out tiles and streams them into a ring of shared-memory stages with bulk
-// copies; the consumer warps never wait for each other: each sweeps its own planes of a tile and
-// arrives on the stage's "empty" barrier when done.  The warp that finishes a tile last does the
-// tile-level book-keeping (scan word, placement of overflow parts); only warps that hold salient
-// planes wait for that placement.
+// copies.  The consumer warps never wait for each other on the common path: each sweeps its own
+// planes of a tile (statistics, class, codes, stores) and arrives on the stage's barriers.  When a
+// stage comes back, the producer publishes the tile's (zero) scan word.  Only warps that hold
+// salient or raw planes take the slow path: they wait until the whole tile is classified, one of
+// them places the tile's overflow parts, and they write their planes.
 // -------------------------------------------------------------------------------------------------
 constexpr int kWarpKernelThreads = kThreads + 32;
 
-template <int DT, bool SIGMA, int G>
+// Placement of a tile with salient / raw planes, executed by one warp.  ovf16[i] holds the overflow
+// size of plane i of the tile in 16-byte units (0 for normal planes); on return it holds the
+// plane's offset relative to the tile's base.
+__device__ __noinline__ void tile_place_sparse(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
+                                               uint32_t np, uint32_t* ovf16, unsigned long long* s_base16,
+                                               uint32_t* s_skip) {
+  const uint32_t lane = threadIdx.x & 31u;
+  uint32_t carry = 0;
+  for (uint32_t base = 0; base < np; base += 32) {
+    const uint32_t i = base + lane;
+    const uint32_t v = i < np ? ovf16[i] : 0u;
+    uint32_t incl = v;
+    for (uint32_t o = 1; o < 32; o <<= 1) {
+      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    if (i < np) ovf16[i] = carry + incl - v;
+    carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+  }
+  unsigned long long excl = 0;
+  uint32_t skip = d.fits ? 0u : 1u;
+  if (tile == 0) {
+    scan_publish(a.ts, tile, a.epoch, 2u, carry);
+  } else {
+    scan_publish(a.ts, tile, a.epoch, 1u, carry);
+    if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
+      if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+      skip = 1;
+    }
+    scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)(excl + carry));
+  }
+  if (lane == 0) {
+    if (carry) atomicAdd(&a.sc->ovf16, (unsigned long long)carry);
+    const unsigned long long base16 = (pl.ovf_off >> 4) + excl;
+    if ((base16 + carry) * 16ull > d.capacity) skip = 1;  // never write past the capacity
+    *s_base16 = base16;
+    *s_skip = skip;
+  }
+}
+
+// Scan word of a tile without salient or raw planes (all lanes of the producer warp).  Every 32nd
+// tile also resolves its prefix so that look-backs stay short.
+__device__ __noinline__ void publish_plain_tile(const CompressArgs& a, uint32_t tile) {
+  if (tile == 0) {
+    scan_publish(a.ts, tile, a.epoch, 2u, 0u);
+    return;
+  }
+  scan_publish(a.ts, tile, a.epoch, 1u, 0u);
+  if ((tile & 31u) != 31u) return;
+  unsigned long long excl = 0;
+  if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
+    if ((threadIdx.x & 31u) == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+  }
+  scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)excl);
+}
+
+template <int DT, bool SIGMA, int TT, bool FULLVEC>
 __global__ void __launch_bounds__(kWarpKernelThreads, 2) compress_warp(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kWarps * 5];
-  __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
-  __shared__ uint32_t s_tiles[kMaxStages], s_done[kMaxStages], s_nonnormal[kMaxStages], s_skip[kMaxStages];
+  __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_classified[kMaxStages];
+  __shared__ uint32_t s_tiles[kMaxStages], s_nn[kMaxStages], s_nnmask[kMaxStages], s_skip[kMaxStages];
   __shared__ volatile uint32_t s_placed[kMaxStages];  // tile + 1 once the tile's overflow parts are placed
   __shared__ unsigned long long s_base16[kMaxStages];
   __shared__ volatile uint32_t s_abort;
+  __shared__ Plan s_pl;          // copies for the outlined slow path (salient planes, placement):
+  __shared__ CompressArgs s_a;   // its functions take them by address
 
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const Dest d = make_dest(pl, a);
   const uint32_t nstage = pl.nstage;
-  const uint32_t rec_stride = (20u * pl.ppt + 15u) & ~15u;
+  uint32_t* ovf16_all = reinterpret_cast<uint32_t*>(smem + pl.sm_rec);  // nstage x ppt words, zero when idle
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
   if (tid == 0) {
+    s_pl = pl;
+    s_a = a;
     for (uint32_t s = 0; s < nstage; ++s) {
       mbar_init(&s_full[s], 1);
       mbar_init(&s_empty[s], kWarps);
-      s_done[s] = 0;
-      s_nonnormal[s] = 0;
+      mbar_init(&s_classified[s], kWarps);
+      s_nn[s] = 0;
+      s_nnmask[s] = 0;
       s_placed[s] = 0;
     }
     fence_mbar_init();
     s_abort = 0;
   }
+  for (uint32_t i = tid; i < nstage * pl.ppt; i += kWarpKernelThreads) ovf16_all[i] = 0;
   __syncthreads();
 
   if (warp == (uint32_t)kWarps) {
-    // ======================= producer =======================
-    if (lane == 0) {
-      uint32_t s = 0, empty_phase = 0;
-      for (uint32_t n = 0;; ++n) {
-        if (n >= nstage) {  // wait until every consumer warp is done with the previous tile of this stage
-          if (!mbar_wait_abortable(&s_empty[s], (empty_phase >> s) & 1u, 1u << 22, &s_abort)) {
-            s_abort = 1;
+    // ======================= producer (all 32 lanes walk the loop, lane 0 issues) =======================
+    uint32_t s = 0, empty_phase = 0;
+    bool aborted = false;
+    // Drains stage q: waits until every consumer warp is done with its tile, then gives a tile without
+    // salient planes its scan word (tiles with salient planes were published by their consumers).
+    auto drain = [&](uint32_t q) -> bool {
+      bool ok = mbar_wait_abortable(&s_empty[q], (empty_phase >> q) & 1u, 1u << 20, &s_abort);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) return false;
+      empty_phase ^= 1u << q;
+      if (pl.mode != kModeOff) {
+        const uint32_t nn = *reinterpret_cast<volatile uint32_t*>(&s_nn[q]);
+        if (nn == 0) publish_plain_tile(s_a, s_tiles[q]);
+        __syncwarp();
+        if (lane == 0) {
+          s_nn[q] = 0;
+          s_nnmask[q] = 0;
+        }
+      }
+      return true;
+    };
+    for (uint32_t n = 0;; ++n) {
+      if (n >= nstage && !drain(s)) {
+        aborted = true;
+        break;
+      }
+      uint32_t t = 0;
+      if (lane == 0) t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+      t = __shfl_sync(0xFFFFFFFFu, t, 0);
+      if (t >= pl.ntiles) {
+        // no more tiles: wake the consumers at this stage, then drain the tiles still in the ring
+        const uint32_t first = n >= nstage ? n - nstage + 1u : 0u;
+        uint32_t q = first % nstage;
+        __syncwarp();
+        if (lane == 0) {
+          s_tiles[s] = t;
+          mbar_arrive(&s_full[s]);
+        }
+        for (uint32_t m = first; m < n; ++m) {
+          if (!drain(q)) {
+            aborted = true;
             break;
           }
-          empty_phase ^= 1u << s;
+          q = q + 1 == nstage ? 0 : q + 1;
         }
-        const uint32_t t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+        break;
+      }
+      if (lane == 0) {
         s_tiles[s] = t;
-        if (t >= pl.ntiles) {
-          mbar_arrive(&s_full[s]);  // wake the consumers: no more tiles
-          break;
-        }
-        const uint64_t p0 = (uint64_t)t * pl.ppt;
+        const uint32_t p0 = t * pl.ppt;
         const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
         const uint32_t bytes = np * (uint32_t)pl.plane_bytes;
         uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
         if ((bytes & 15u) == 0u) {
           fence_proxy_async();
           mbar_expect_tx(&s_full[s], bytes);
-          bulk_g2s(stage, a.src + p0 * pl.plane_bytes, bytes, &s_full[s]);
+          bulk_g2s(stage, a.src + (uint64_t)p0 * pl.plane_bytes, bytes, &s_full[s]);
         } else {  // ragged last tile of a tensor of ragged planes: plain loads by this thread
-          const uint16_t* g = reinterpret_cast<const uint16_t*>(a.src + p0 * pl.plane_bytes);
+          const uint16_t* g = reinterpret_cast<const uint16_t*>(a.src + (uint64_t)p0 * pl.plane_bytes);
           for (uint32_t i = 0; i < bytes / 2u; ++i) reinterpret_cast<uint16_t*>(stage)[i] = g[i];
           mbar_arrive(&s_full[s]);
         }
-        s = s + 1 == nstage ? 0 : s + 1;
       }
-      if (s_abort) {  // wait (bounded) for copies still in flight before the CTA may exit
+      __syncwarp();
+      s = s + 1 == nstage ? 0 : s + 1;
+    }
+    if (aborted) {  // wait (bounded) for copies still in flight before the CTA may exit
+      s_abort = 1;
+      if (lane == 0) {
         atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
         for (uint32_t k = 0; k < nstage; ++k) {
-          mbar_wait(&s_full[k], 0u, 1u << 16);
-          mbar_wait(&s_full[k], 1u, 1u << 16);
+          mbar_wait(&s_full[k], 0u, 1u << 10);
+          mbar_wait(&s_full[k], 1u, 1u << 10);
         }
       }
     }
   } else {
     // ======================= consumers =======================
-    const Team team = make_team(pl.team, s_red);
-    const uint32_t T = pl.team;
-    const uint32_t my_team = tid / T;
-    uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
+    constexpr int G = 8;  // groups per thread: a plane has at most 8 * TT groups
+    const Team team = make_team(TT, s_red);
+    const uint32_t my_team = tid / TT;
     const bool vec = (pl.plane_bytes & 15u) == 0u;
-    const bool full = vec && pl.groups == (uint32_t)G * T;
-    uint32_t rp = 0, s = 0, full_phase = 0;
+    uint32_t rp = 0, s = 0, phase = 0;
     for (;;) {
-      bool ok = mbar_wait_abortable(&s_full[s], (full_phase >> s) & 1u, 1u << 22, &s_abort);
+      const uint32_t par = (phase >> s) & 1u;
+      bool ok = mbar_wait_abortable(&s_full[s], par, 1u << 20, &s_abort);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) {
         s_abort = 1;
         break;
       }
-      full_phase ^= 1u << s;
+      phase ^= 1u << s;
       const uint32_t tile = s_tiles[s];
       if (tile >= pl.ntiles) break;
-      const uint64_t p0 = (uint64_t)tile * pl.ppt;
+      const uint32_t p0 = tile * pl.ppt;
       const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
-      const uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
-      Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec + (uint64_t)s * rec_stride);
-      uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + (uint64_t)s * rec_stride + 16u * pl.ppt);
-      const bool active = my_team < np;
       const uint32_t lp = my_team;
-      const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
+      const bool active = lp < np;
+      const uint8_t* plane = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes + (uint64_t)lp * pl.plane_bytes;
       Rec r;
       r.meta = kClsNormal;
-      SalientInfo info = {0, 0, 0, 0};
-      if (active) {
-        if (full) plane_sweep<DT, SIGMA, G, true>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
-        else plane_sweep<DT, SIGMA, G, false>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
-        if ((r.meta & 3u) != kClsNormal) {
-          info = salient_measure<DT>(team, pl, plane, sal);
+      if (active) plane_sweep_any<DT, SIGMA, G, TT, FULLVEC>(team, pl, d, a, plane, (uint64_t)p0 + lp, vec, rp, r);
+      const bool mine_nn = active && (r.meta & 3u) != kClsNormal;
+      if (!__any_sync(0xFFFFFFFFu, mine_nn)) {
+        // ---- common path: this warp is done with the tile
+        if (lane == 0) {
+          mbar_arrive(&s_classified[s]);
+          mbar_arrive(&s_empty[s]);
+        }
+      } else {
+        // ---- slow path: salient / raw planes in this warp
+        uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
+        uint32_t* ovf16 = ovf16_all + s * pl.ppt;
+        SalientInfo info = {0, 0, 0, 0};
+        if (mine_nn) {
+          info = salient_measure<DT>(team, s_pl, plane, sal);
           r.size = info.size;
           if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
             r.meta = (r.meta & ~3u) | kClsRaw;
             r.size = (uint32_t)pl.plane_bytes;
           }
-        }
-        if (team.lane == 0) rec[lp] = r;
-      }
-      const bool mine_nonnormal = active && (r.meta & 3u) != kClsNormal;
-      const uint32_t handled = __popc(__ballot_sync(0xFFFFFFFFu, active && team.lane == 0));
-      const uint32_t nn = __popc(__ballot_sync(0xFFFFFFFFu, mine_nonnormal && team.lane == 0));
-      uint32_t last = 0;
-      __syncwarp();  // the records written by this warp's team leaders are ordered before lane 0's signal
-      if (lane == 0 && handled) {
-        if (nn) atomicAdd(&s_nonnormal[s], nn);
-        __threadfence_block();
-        last = (atomicAdd(&s_done[s], handled) + handled == np) ? 1u : 0u;
-      }
-      last = __shfl_sync(0xFFFFFFFFu, last, 0);
-      if (last) {  // this warp finished the tile: tile-level book-keeping
-        __threadfence_block();
-        const uint32_t tile_nn = *reinterpret_cast<volatile uint32_t*>(&s_nonnormal[s]);
-        if (tile_nn == 0) {
-          if (pl.mode != kModeOff) {
-            if (tile == 0) {
-              scan_publish(a.ts, tile, a.epoch, 2u, 0u);
-            } else {
-              scan_publish(a.ts, tile, a.epoch, 1u, 0u);
-              if ((tile & 31u) == 31u) {
-                unsigned long long excl = 0;
-                if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
-                  if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-                }
-                scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)excl);
-              }
-            }
+          if (team.lane == 0) {
+            ovf16[lp] = a16(r.size) > pl.npay ? (a16(r.size) - pl.npay) >> 4 : 0u;
+            atomicAdd((r.meta & 3u) == kClsRaw ? &a.sc->nraw : &a.sc->nsal, 1ull);
           }
-        } else {
-          tile_place(pl, a, d, tile, np, rec, roff, &s_base16[s], &s_skip[s]);
-          __threadfence_block();
-          __syncwarp();
-          if (lane == 0) s_placed[s] = tile + 1u;
         }
+        __syncwarp();
         if (lane == 0) {
-          s_done[s] = 0;
-          s_nonnormal[s] = 0;
+          atomicAdd(&s_nn[s], 1u);
+          atomicOr(&s_nnmask[s], 1u << warp);
+          __threadfence_block();
+          mbar_arrive(&s_classified[s]);
         }
-      }
-      if (nn) {  // teams of this warp hold salient / raw planes: wait for the placement, then write
-        bool placed = false;
-        for (uint32_t i = 0; i < (1u << 22); ++i) {
-          if (s_placed[s] == tile + 1u) {
-            placed = true;
-            break;
+        bool done = mbar_wait_abortable(&s_classified[s], par, 1u << 20, &s_abort);  // the whole tile is classified
+        done = __all_sync(0xFFFFFFFFu, done);
+        if (done) {
+          __threadfence_block();
+          const uint32_t mask = *reinterpret_cast<volatile uint32_t*>(&s_nnmask[s]);
+          if ((uint32_t)__ffs(mask) - 1u == warp) {  // the first such warp places the tile
+            tile_place_sparse(s_pl, s_a, d, tile, np, ovf16, &s_base16[s], &s_skip[s]);
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) s_placed[s] = tile + 1u;
           }
-          if (s_abort) break;
-          __nanosleep(64);
+          done = false;
+          for (uint32_t i = 0; i < (1u << 22); ++i) {
+            if (s_placed[s] == tile + 1u) {
+              done = true;
+              break;
+            }
+            if (s_abort) break;
+            __nanosleep(64);
+          }
+          done = __all_sync(0xFFFFFFFFu, done);
         }
-        placed = __all_sync(0xFFFFFFFFu, placed);
-        if (!placed) {
+        if (!done) {
           s_abort = 1;
           if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
         } else {
           __threadfence_block();
-          if (mine_nonnormal && !s_skip[s]) {
-            SplitOut out;
-            out.slot = d.dst + pl.slots_off + (p0 + lp) * pl.npay;
-            out.ovf = d.dst + (s_base16[s] + roff[lp]) * 16ull;
-            out.npay = pl.npay;
-            if ((r.meta & 3u) == kClsRaw) raw_write(team, pl, plane, out);
-            else salient_write<DT>(team, pl, plane, info, sal, out);
-            if (team.lane == 0)
-              store_table_entry(d, p0 + lp, a16(r.size) > pl.npay ? (uint32_t)(s_base16[s] + roff[lp]) : 0u, r);
+          if (mine_nn) {
+            const unsigned long long off16 = s_base16[s] + ovf16[lp];
+            if (!s_skip[s]) {
+              SplitOut out;
+              out.slot = d.dst + pl.slots_off + ((uint64_t)p0 + lp) * pl.npay;
+              out.ovf = d.dst + off16 * 16ull;
+              out.npay = pl.npay;
+              if ((r.meta & 3u) == kClsRaw) raw_write(team, s_pl, plane, out);
+              else salient_write<DT>(team, s_pl, plane, info, sal, out);
+              if (team.lane == 0)
+                store_table_entry(d, (uint64_t)p0 + lp, a16(r.size) > pl.npay ? (uint32_t)off16 : 0u, r);
+            }
+            team_sync(team);
+            if (team.lane == 0) ovf16[lp] = 0;  // leave the array clean for the stage's next tile
           }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_empty[s]);
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s_empty[s]);  // this warp no longer touches the stage or its records
       if (s_abort) break;
       s = s + 1 == nstage ? 0 : s + 1;
     }
@@ -876,22 +987,29 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 2) compress_warp(const Pla
   cta_exit(pl, a, d);
 }
 
-template <int DT, bool SIGMA, int G, bool CTA>
-__global__ void __launch_bounds__(kThreads, (G <= 8 ? 3 : 2)) compress_fast(const Plan pl, const CompressArgs a) {
+template <int DT, bool SIGMA, int G>
+__global__ void __launch_bounds__(kThreads, 2) compress_cta(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
   __shared__ uint32_t s_nonnormal[2], s_skip, s_abort;  // s_nonnormal: one slot per tile parity
   __shared__ unsigned long long s_base16;
+  __shared__ Plan s_pl;          // copies for the outlined slow path
+  __shared__ CompressArgs s_a;
 
   const uint32_t tid = threadIdx.x;
+  if (tid == 0) {
+    s_pl = pl;
+    s_a = a;
+  }
   Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
   uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + 16u * pl.ppt);
   const Dest d = make_dest(pl, a);
-  const Team team = make_team(pl.team, s_red);
-  const uint32_t T = CTA ? (uint32_t)kThreads : pl.team;
-  const uint32_t my_team = CTA ? 0u : tid / T;
+  constexpr bool CTA = true;
+  const Team team = make_team(kThreads, s_red);
+  const uint32_t T = kThreads;
+  const uint32_t my_team = 0u;
   uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
   const uint32_t nstage = pl.nstage;
   const bool vec = (pl.plane_bytes & 15u) == 0u;
@@ -945,7 +1063,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 8 ? 3 : 2)) compress_fast(cons
 #pragma unroll
       for (int k = 0; k < kMaxStages; ++k)
         if (k == (int)s) u = uses[k]++;
-      ready = mbar_wait(&s_full[s], u & 1u, 1u << 22);
+      ready = mbar_wait(&s_full[s], u & 1u, 1u << 20);
       ready = __all_sync(0xFFFFFFFFu, ready);
       if (!ready) s_abort = 1;  // the load never arrived
     } else {
@@ -959,10 +1077,9 @@ __global__ void __launch_bounds__(kThreads, (G <= 8 ? 3 : 2)) compress_fast(cons
       const uint32_t lp = my_team;
       const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
       Rec r;
-      if (full) plane_sweep<DT, SIGMA, G, true>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
-      else plane_sweep<DT, SIGMA, G, false>(team, T, pl, d, a, plane, p0 + lp, vec, rp, r);
+      plane_sweep_any<DT, SIGMA, G, kThreads, false>(team, pl, d, a, plane, p0 + lp, vec, rp, r);
       if ((r.meta & 3u) != kClsNormal) {
-        info = salient_measure<DT>(team, pl, plane, sal);
+        info = salient_measure<DT>(team, s_pl, plane, sal);
         r.size = info.size;
         if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
           r.meta = (r.meta & ~3u) | kClsRaw;
@@ -986,7 +1103,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 8 ? 3 : 2)) compress_fast(cons
           scan_publish(a.ts, tile, a.epoch, 1u, 0u);
           if ((tile & 31u) == 31u) {
             unsigned long long excl = 0;
-            if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
+            if (!scan_resolve(s_a.ts, tile, s_a.epoch, s_a.spin_limit, &s_a.sc->status, &excl)) {
               if (tid == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
             }
             scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)excl);
@@ -995,7 +1112,7 @@ __global__ void __launch_bounds__(kThreads, (G <= 8 ? 3 : 2)) compress_fast(cons
       }
     } else {
       // ---- place the overflow parts of this tile, then the owning teams write their planes
-      if (tid < 32) tile_place(pl, a, d, tile, np, rec, roff, &s_base16, &s_skip);
+      if (tid < 32) tile_place(s_pl, s_a, d, tile, np, rec, roff, &s_base16, &s_skip);
       __syncthreads();
       if (!s_skip && (CTA || my_team < np)) {
         const uint32_t lp = my_team;
@@ -1007,9 +1124,9 @@ __global__ void __launch_bounds__(kThreads, (G <= 8 ? 3 : 2)) compress_fast(cons
           out.ovf = d.dst + (s_base16 + roff[lp]) * 16ull;
           out.npay = pl.npay;
           if ((r.meta & 3u) == kClsRaw) {
-            raw_write(team, pl, plane, out);
+            raw_write(team, s_pl, plane, out);
           } else {  // the team's scratch and `info` still hold the measurement of this plane
-            salient_write<DT>(team, pl, plane, info, sal, out);
+            salient_write<DT>(team, s_pl, plane, info, sal, out);
           }
           if (team.lane == 0)
             store_table_entry(d, p0 + lp, a16(r.size) > pl.npay ? (uint32_t)(s_base16 + roff[lp]) : 0u, r);

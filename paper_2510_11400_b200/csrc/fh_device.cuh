@@ -122,12 +122,15 @@ __device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t by
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// One wait attempt: the hardware may suspend the thread for up to about `kSuspendNs` nanoseconds
+// while the phase is incomplete, so that waiting warps do not burn issue slots polling.
+constexpr uint32_t kSuspendNs = 2000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
-      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(kSuspendNs)
       : "memory");
   return ok != 0;
 }
@@ -139,19 +142,14 @@ __device__ __forceinline__ bool mbar_wait_abortable(uint64_t* bar, uint32_t pari
                                                     const volatile uint32_t* abort) {
   for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (i > 32) {
-      if (*abort) return false;
-      __nanosleep(32);
-    }
+    if (*abort) return false;
   }
   return false;
 }
 // Bounded wait: false when the phase did not complete within `limit` polls.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit) {
-  for (uint32_t i = 0; i < limit; ++i) {
+  for (uint32_t i = 0; i < limit; ++i)
     if (mbar_try_wait(bar, parity)) return true;
-    if (i > 64) __nanosleep(32);
-  }
   return false;
 }
 
@@ -233,6 +231,15 @@ __device__ __forceinline__ void sigma_addends(const float v[4], const SigmaScale
   const float sg = __fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3]));
   const float q01 = __fmaf_rn(v[1], v[1], __fmul_rn(v[0], v[0]));
   const float q23 = __fmaf_rn(v[3], v[3], __fmul_rn(v[2], v[2]));
+  const float qg = __fadd_rn(q01, q23);
+  as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
+  aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
+}
+__device__ __forceinline__ void sigma_addends4(float v0, float v1, float v2, float v3, const SigmaScale& sc,
+                                               uint32_t& as, uint32_t& aq) {
+  const float sg = __fadd_rn(__fadd_rn(v0, v1), __fadd_rn(v2, v3));
+  const float q01 = __fmaf_rn(v1, v1, __fmul_rn(v0, v0));
+  const float q23 = __fmaf_rn(v3, v3, __fmul_rn(v2, v2));
   const float qg = __fadd_rn(q01, q23);
   as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
   aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
@@ -476,7 +483,7 @@ __device__ __forceinline__ void scan_publish(unsigned long long* ts, uint32_t ti
 }
 
 // Returns false on timeout.  *excl receives the sum of the aggregates of tiles [0, tile).
-__device__ __forceinline__ bool scan_resolve(const unsigned long long* ts, uint32_t tile, uint32_t epoch,
+__device__ __noinline__ bool scan_resolve(const unsigned long long* ts, uint32_t tile, uint32_t epoch,
                                              uint32_t spin_limit, const unsigned long long* status,
                                              unsigned long long* excl) {
   const uint32_t lane = threadIdx.x & 31u;
