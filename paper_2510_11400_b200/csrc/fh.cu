@@ -22,7 +22,7 @@ using fh::Plan;
 constexpr size_t kSmemLimit = 227 * 1024 - 1024;  // dynamic shared memory a CTA may ask for
 constexpr size_t kTileTarget = 32 * 1024;         // dense bytes a tile of the generic kernel aims for
 constexpr size_t kStageTarget = 72 * 1024;        // shared memory the stages of the CTA-team kernel aim for
-constexpr size_t kWarpStageTarget = 100 * 1024;   // ... and those of the warp-team kernel (two CTAs per SM)
+constexpr size_t kWarpStageTarget = 72 * 1024;    // ... and those of the warp-team kernel (two CTAs per SM)
 constexpr uint32_t kMaxPpt = 2048;
 constexpr uint32_t kSpinLimit = 1u << 20;
 
@@ -219,8 +219,10 @@ int get_scratch(cudaStream_t stream, size_t ntiles, StreamScratch** out) {
       s.ts = nullptr;
       s.ts_cap = 0;
     }
-    if (cudaMalloc(&s.ts, cap * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
-    if (cudaMemset(s.ts, 0, cap * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
+    // tile words | segment counters | segment prefixes (a segment is 32 tiles)
+    const size_t words = cap + 2 * (cap / 32);
+    if (cudaMalloc(&s.ts, words * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMemset(s.ts, 0, words * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
     s.ts_cap = cap;
   }
   *out = &s;
@@ -230,7 +232,8 @@ int get_scratch(cudaStream_t stream, size_t ntiles, StreamScratch** out) {
 // Advance the 30-bit epoch; when it would wrap, clear the scan words so that stale epochs cannot match.
 int next_epoch(StreamScratch* s, cudaStream_t stream) {
   if (s->epoch >= 0x3FFFFFF0u) {
-    if (s->ts && cudaMemsetAsync(s->ts, 0, s->ts_cap * sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
+    if (s->ts && cudaMemsetAsync(s->ts, 0, (s->ts_cap + 2 * (s->ts_cap / 32)) * sizeof(unsigned long long), stream) != cudaSuccess)
+      return FH_ERR_CUDA;
     s->epoch = 0;
   }
   ++s->epoch;
@@ -380,9 +383,12 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   a.d_off_out = d_off_out;
   a.out2 = d_out2;
   a.sc = s->sc;
-  a.ts = s->ts;
-  a.epoch = s->epoch;
-  a.spin_limit = kSpinLimit;
+  a.scan.ts = s->ts;
+  a.scan.seg_cs = s->ts + s->ts_cap;
+  a.scan.seg_inc = s->ts + s->ts_cap + s->ts_cap / 32;
+  a.scan.epoch = s->epoch;
+  a.scan.spin_limit = kSpinLimit;
+  a.nseg = (pl.ntiles + 31) / 32;
   return launch_compress(pl, v, a, stream);
 }
 
@@ -630,7 +636,7 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
 
 // ---- allocation-free compress -----------------------------------------------------------------
 // Scan scratch compiled into the device image: a Scratch header (padded to 256 bytes) followed by
-// FH_STATIC_MAX_TILES scan words.  The name is a device symbol: host code must not pass it to a
+// FH_STATIC_MAX_TILES tile words and 2 * FH_STATIC_MAX_TILES / 32 segment words.  The name is a device symbol: host code must not pass it to a
 // kernel, it asks the runtime for the symbol's device address instead (once per device).
 static __device__ __align__(256) unsigned char g_static_scratch[FH_STATIC_SCRATCH_BYTES];
 static_assert(sizeof(fh::Scratch) <= 256, "static scratch layout");
@@ -662,9 +668,8 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
     g_static_ptr[dev] = p;
   }
   unsigned char* base = g_static_ptr[dev];
-  // the array keeps the last call's counters and scan words: clear the part this call uses
-  if (cudaMemsetAsync(base, 0, 256 + sizeof(unsigned long long) * (size_t)pl.ntiles, stream) != cudaSuccess)
-    return FH_ERR_CUDA;
+  // the array keeps the last call's counters and scan words: clear it (header, tile words, segment words)
+  if (cudaMemsetAsync(base, 0, FH_STATIC_SCRATCH_BYTES, stream) != cudaSuccess) return FH_ERR_CUDA;
   fh::CompressArgs a;
   a.src = (const uint8_t*)d_src;
   a.dst_base = (uint8_t*)d_dst;
@@ -673,9 +678,12 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   a.d_off_out = nullptr;
   a.out2 = (unsigned long long*)d_out2;
   a.sc = reinterpret_cast<fh::Scratch*>(base);
-  a.ts = reinterpret_cast<unsigned long long*>(base + 256);
-  a.epoch = 1;
-  a.spin_limit = kSpinLimit;
+  a.scan.ts = reinterpret_cast<unsigned long long*>(base + 256);
+  a.scan.seg_cs = a.scan.ts + FH_STATIC_MAX_TILES;
+  a.scan.seg_inc = a.scan.seg_cs + FH_STATIC_MAX_TILES / 32;
+  a.scan.epoch = 1;
+  a.scan.spin_limit = kSpinLimit;
+  a.nseg = (pl.ntiles + 31) / 32;
   return launch_compress(pl, v, a, stream);
 }
 

@@ -30,9 +30,8 @@ struct CompressArgs {
   unsigned long long* d_off_out;        // optional: offset for the next container
   unsigned long long* out2;             // optional: {total bytes, status}
   Scratch* sc;
-  unsigned long long* ts;               // scan words, one per tile
-  uint32_t epoch;
-  uint32_t spin_limit;
+  ScanState scan;                       // scan words (tiles, segments), epoch, wait bound
+  uint32_t nseg;                        // segments of this call (for the final clean-up)
 };
 
 // Where the bytes of a salient / raw payload go: offsets below npay land in the plane's slot, the
@@ -241,7 +240,7 @@ __device__ __forceinline__ Dest make_dest(const Plan& pl, const CompressArgs& a)
 
 // Tile-level placement, executed by warp 0 after the classes and sizes of the tile's planes are in
 // rec[].  Computes each plane's overflow offset (roff[], 16-byte units relative to the tile),
-// publishes the tile's aggregate and, when the tile needs it or is a 32nd tile, resolves the tile's
+// publishes the tile's overflow size and, when the tile has overflow parts, resolves the tile's
 // base.  Returns through shared variables: *s_base16 (absolute, 16-byte units), *s_skip.
 __device__ __noinline__ void tile_place(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
                                            uint32_t np, const Rec* rec, uint32_t* roff,
@@ -268,17 +267,11 @@ __device__ __noinline__ void tile_place(const Plan& pl, const CompressArgs& a, c
   unsigned long long excl = 0;
   uint32_t skip = d.fits ? 0u : 1u;
   if (pl.mode != kModeOff) {
-    const bool resolve = carry > 0 || (tile & 31u) == 31u;
-    if (tile == 0) {
-      scan_publish(a.ts, tile, a.epoch, 2u, carry);
-    } else {
-      scan_publish(a.ts, tile, a.epoch, 1u, carry);
-      if (resolve) {
-        if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
-          if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-          skip = 1;
-        }
-        scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)(excl + carry));
+    if (lane == 0) scan_publish(a.scan, tile, carry);
+    if (carry > 0 && tile > 0) {
+      if (!scan_resolve(a.scan, tile, &a.sc->status, &excl)) {
+        if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+        skip = 1;
       }
     }
     if (lane == 0) {
@@ -335,6 +328,8 @@ __device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, 
     a.out2[1] = status_word(code);
   }
   if (a.d_off_out) *a.d_off_out = code == kErrNone ? d.off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
+  if (pl.mode != kModeOff)
+    for (uint32_t k = 0; k < a.nseg; ++k) st_relaxed(a.scan.seg_cs + k, 0ull);  // counters back to zero
   st_relaxed(&a.sc->ticket, 0ull);
   st_relaxed(&a.sc->status, 0ull);
   st_relaxed(&a.sc->ovf16, 0ull);
@@ -583,7 +578,7 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
                                             const uint8_t* plane, uint64_t gp, uint32_t& rp, Rec& r) {
   const uint32_t groups = pl.groups, lane = team.lane;
   float x[G][4];
-  float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
+  float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000), lo1 = lo, hi1 = hi;
   uint32_t ng = 0, npad = 0;  // groups of this thread; zero-padded elements among them
 #pragma unroll
   for (int k = 0; k < G; ++k) {
@@ -598,10 +593,16 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
           x[k][0] = __uint_as_float(t2.x << 16); x[k][1] = __uint_as_float(t2.x & 0xFFFF0000u);
           x[k][2] = __uint_as_float(t2.y << 16); x[k][3] = __uint_as_float(t2.y & 0xFFFF0000u);
         }
-        lo = min3_nan(lo, x[k][0], x[k][1]);
-        lo = min3_nan(lo, x[k][2], x[k][3]);
-        hi = max3_nan(hi, x[k][0], x[k][1]);
-        hi = max3_nan(hi, x[k][2], x[k][3]);
+        // per-group partial results keep the dependency chains short
+        const float gl = min_nan(min3_nan(x[k][0], x[k][1], x[k][2]), x[k][3]);
+        const float gh = max_nan(max3_nan(x[k][0], x[k][1], x[k][2]), x[k][3]);
+        if (k & 1) {
+          lo1 = min_nan(lo1, gl);
+          hi1 = max_nan(hi1, gh);
+        } else {
+          lo = min_nan(lo, gl);
+          hi = max_nan(hi, gh);
+        }
       } else {  // plane not on a 16-byte boundary, possibly with a ragged last group
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -619,6 +620,8 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
       ++ng;
     }
   }
+  lo = min_nan(lo, lo1);
+  hi = max_nan(hi, hi1);
   team_minmax(team, lo, hi, rp);
   if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && lane == 0)
     atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
@@ -638,21 +641,24 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
     else sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, tlo, thi);
     uint32_t cnt = 0;
     if (hi > thi || lo < tlo) {  // otherwise no element can lie outside: the count is zero
-      if (lo >= tlo) {           // nothing below: one compare per element
+      uint32_t c[4] = {0, 0, 0, 0};  // four counters: short dependency chains
+      if (lo >= tlo) {               // nothing below: one compare per element
 #pragma unroll
         for (int k = 0; k < G; ++k)
           if (FULL || lane + (uint32_t)(k * TT) < groups) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) cnt += x[k][e] > thi;
+            for (int e = 0; e < 4; ++e) c[e] += x[k][e] > thi;
           }
+        cnt = (c[0] + c[1]) + (c[2] + c[3]);
         if (!VEC && 0.0f > thi) cnt -= npad;  // padded zeros are not elements
       } else {
 #pragma unroll
         for (int k = 0; k < G; ++k)
           if (FULL || lane + (uint32_t)(k * TT) < groups) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) cnt += (x[k][e] > thi) || (x[k][e] < tlo);
+            for (int e = 0; e < 4; ++e) c[e] += (x[k][e] > thi) || (x[k][e] < tlo);
           }
+        cnt = (c[0] + c[1]) + (c[2] + c[3]);
         if (!VEC && ((0.0f > thi) || (0.0f < tlo))) cnt -= npad;
       }
       cnt = team_sum_u32(team, cnt, rp);
@@ -731,15 +737,12 @@ __device__ __noinline__ void tile_place_sparse(const Plan& pl, const CompressArg
   }
   unsigned long long excl = 0;
   uint32_t skip = d.fits ? 0u : 1u;
-  if (tile == 0) {
-    scan_publish(a.ts, tile, a.epoch, 2u, carry);
-  } else {
-    scan_publish(a.ts, tile, a.epoch, 1u, carry);
-    if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
+  if (lane == 0) scan_publish(a.scan, tile, carry);
+  if (carry > 0 && tile > 0) {
+    if (!scan_resolve(a.scan, tile, &a.sc->status, &excl)) {
       if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
       skip = 1;
     }
-    scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)(excl + carry));
   }
   if (lane == 0) {
     if (carry) atomicAdd(&a.sc->ovf16, (unsigned long long)carry);
@@ -750,24 +753,8 @@ __device__ __noinline__ void tile_place_sparse(const Plan& pl, const CompressArg
   }
 }
 
-// Scan word of a tile without salient or raw planes (all lanes of the producer warp).  Every 32nd
-// tile also resolves its prefix so that look-backs stay short.
-__device__ __noinline__ void publish_plain_tile(const CompressArgs& a, uint32_t tile) {
-  if (tile == 0) {
-    scan_publish(a.ts, tile, a.epoch, 2u, 0u);
-    return;
-  }
-  scan_publish(a.ts, tile, a.epoch, 1u, 0u);
-  if ((tile & 31u) != 31u) return;
-  unsigned long long excl = 0;
-  if (!scan_resolve(a.ts, tile, a.epoch, a.spin_limit, &a.sc->status, &excl)) {
-    if ((threadIdx.x & 31u) == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-  }
-  scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)excl);
-}
-
 template <int DT, bool SIGMA, int TT, bool FULLVEC>
-__global__ void __launch_bounds__(kWarpKernelThreads, 2) compress_warp(const Plan pl, const CompressArgs a) {
+__global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_classified[kMaxStages];
@@ -812,13 +799,12 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 2) compress_warp(const Pla
       if (!ok) return false;
       empty_phase ^= 1u << q;
       if (pl.mode != kModeOff) {
-        const uint32_t nn = *reinterpret_cast<volatile uint32_t*>(&s_nn[q]);
-        if (nn == 0) publish_plain_tile(s_a, s_tiles[q]);
-        __syncwarp();
         if (lane == 0) {
+          if (*reinterpret_cast<volatile uint32_t*>(&s_nn[q]) == 0) scan_publish(a.scan, s_tiles[q], 0u);
           s_nn[q] = 0;
           s_nnmask[q] = 0;
         }
+        __syncwarp();
       }
       return true;
     };
@@ -1095,21 +1081,8 @@ __global__ void __launch_bounds__(kThreads, 2) compress_cta(const Plan pl, const
     // Warps may run one tile ahead of each other between barriers, hence the flag per tile parity;
     // it is cleared only behind the extra barriers of the slow path.
     if (s_nonnormal[it & 1u] == 0) {
-      // ---- common case: nothing to place; publish a zero aggregate, every 32nd tile resolves
-      if (pl.mode != kModeOff && tid < 32) {
-        if (tile == 0) {
-          scan_publish(a.ts, tile, a.epoch, 2u, 0u);
-        } else {
-          scan_publish(a.ts, tile, a.epoch, 1u, 0u);
-          if ((tile & 31u) == 31u) {
-            unsigned long long excl = 0;
-            if (!scan_resolve(s_a.ts, tile, s_a.epoch, s_a.spin_limit, &s_a.sc->status, &excl)) {
-              if (tid == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-            }
-            scan_publish(a.ts, tile, a.epoch, 2u, (uint32_t)excl);
-          }
-        }
-      }
+      // ---- common case: nothing to place; the tile publishes a zero size
+      if (pl.mode != kModeOff && tid == 0) scan_publish(a.scan, tile, 0u);
     } else {
       // ---- place the overflow parts of this tile, then the owning teams write their planes
       if (tid < 32) tile_place(s_pl, s_a, d, tile, np, rec, roff, &s_base16, &s_skip);

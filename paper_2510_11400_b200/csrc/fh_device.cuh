@@ -472,47 +472,79 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
 }
 
 // ------------------------------------------------------------------------------------------------
-// Plane-ordered placement of the overflow parts: decoupled look-back over per-tile scan words.
-// Executed by all 32 lanes of warp 0.  Every tile publishes its aggregate (mostly zero); a tile that
-// needs its offset, and every 32nd tile (so that walks stay short), resolves its exclusive prefix
-// and publishes the inclusive one.  The wait is bounded; on expiry the call reports kErrTimeout.
+// Plane-ordered placement of the overflow parts.
+//
+// Every tile publishes the size of its overflow parts (zero for a tile of normal planes): a word of
+// its own, tagged with the call's epoch, and a fire-and-forget atomic add of (1 << 32 | size) to the
+// counter word of its segment of 32 tiles.  Only tiles that hold salient or raw planes need their
+// offset: such a tile waits until the earlier tiles of its own segment have published and until the
+// earlier segments are complete (count 32), sums them, and leaves the prefix up to its segment in
+// seg_inc so that later walks stop there.  Tensors without salient planes never wait at all.
+// Waits are bounded; on expiry the call reports kErrTimeout.  The counter words are returned to zero
+// by the last CTA of the kernel; tile and seg_inc words carry the epoch and need no clearing.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void scan_publish(unsigned long long* ts, uint32_t tile, uint32_t epoch, uint32_t flag,
-                                             uint32_t value) {
-  if ((threadIdx.x & 31u) == 0) st_release(ts + tile, scan_word(epoch, flag, value));
+struct ScanState {
+  unsigned long long* ts;       // one word per tile
+  unsigned long long* seg_cs;   // per segment: published tiles << 32 | sum of their sizes
+  unsigned long long* seg_inc;  // per segment: epoch-tagged prefix through the end of the segment
+  uint32_t epoch, spin_limit;
+};
+
+// One thread publishes a tile's overflow size (16-byte units).
+__device__ __forceinline__ void scan_publish(const ScanState& sc, uint32_t tile, uint32_t value) {
+  st_relaxed(sc.ts + tile, scan_word(sc.epoch, 1u, value));
+  const unsigned long long add = (1ull << 32) | value;
+  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(sc.seg_cs + (tile >> 5)), "l"(add) : "memory");
 }
 
-// Returns false on timeout.  *excl receives the sum of the aggregates of tiles [0, tile).
-__device__ __noinline__ bool scan_resolve(const unsigned long long* ts, uint32_t tile, uint32_t epoch,
-                                             uint32_t spin_limit, const unsigned long long* status,
-                                             unsigned long long* excl) {
-  const uint32_t lane = threadIdx.x & 31u;
+// All 32 lanes of a warp: sum of the sizes of tiles [0, tile).  Returns false on timeout.
+__device__ __noinline__ bool scan_resolve(const ScanState& sc, uint32_t tile, const unsigned long long* status,
+                                          unsigned long long* excl) {
+  const uint32_t lane = threadIdx.x & 31u, seg = tile >> 5;
   unsigned long long sum = 0;
-  long long j = (long long)tile - 1;
   uint32_t spins = 0;
-  while (j >= 0) {
-    const long long idx = j - (long long)lane;
-    // before tile 0 there is nothing: a virtual inclusive prefix of zero
-    const unsigned long long w = idx >= 0 ? ld_acquire(ts + idx) : scan_word(epoch, 2u, 0u);
-    const bool valid = (uint32_t)(w >> 34) == epoch;
-    const uint32_t flag = (uint32_t)(w >> 32) & 3u;
-    const uint32_t inc_mask = __ballot_sync(0xFFFFFFFFu, valid && flag == 2u);
-    const uint32_t inv_mask = __ballot_sync(0xFFFFFFFFu, !valid);
+  // earlier tiles of the own segment
+  for (;;) {
+    const uint32_t idx = seg * 32u + lane;
+    const bool need = idx < tile;
+    const unsigned long long w = need ? ld_acquire(sc.ts + idx) : 0ull;
+    const bool valid = !need || (uint32_t)(w >> 34) == sc.epoch;
+    if (__all_sync(0xFFFFFFFFu, valid)) {
+      uint32_t c = need ? (uint32_t)w : 0u;
+      asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(c) : "r"(0xFFFFFFFFu));
+      sum = c;
+      break;
+    }
+    ++spins;
+    if (spins > sc.spin_limit || ((spins & 63u) == 0 && ld_relaxed(status) == kErrTimeout)) return false;
+    __nanosleep(40);
+  }
+  const unsigned long long own = sum;
+  // earlier segments, 32 at a time, back to the nearest published prefix
+  long long k = (long long)seg - 1;
+  while (k >= 0) {
+    const long long j = k - (long long)lane;
+    const unsigned long long inc = j >= 0 ? ld_acquire(sc.seg_inc + j) : 0ull;
+    const unsigned long long cs = j >= 0 ? ld_acquire(sc.seg_cs + j) : 0ull;
+    const bool has_inc = j < 0 || (uint32_t)(inc >> 34) == sc.epoch;  // before segment 0: prefix zero
+    const bool complete = j < 0 || (uint32_t)(cs >> 32) == 32u;
+    const uint32_t inc_mask = __ballot_sync(0xFFFFFFFFu, has_inc);
+    const uint32_t bad_mask = __ballot_sync(0xFFFFFFFFu, !complete);
     const uint32_t first_inc = inc_mask ? (uint32_t)__ffs(inc_mask) - 1u : 32u;
-    const uint32_t first_inv = inv_mask ? (uint32_t)__ffs(inv_mask) - 1u : 32u;
-    const uint32_t need = min(first_inc, 31u);
-    if (first_inv <= need) {  // a predecessor we need has not published yet
+    const uint32_t first_bad = bad_mask ? (uint32_t)__ffs(bad_mask) - 1u : 32u;
+    if (first_bad < first_inc) {  // a segment we must add is not complete yet
       ++spins;
-      if (spins > spin_limit || ((spins & 63u) == 0 && ld_relaxed(status) == kErrTimeout)) return false;
+      if (spins > sc.spin_limit || ((spins & 63u) == 0 && ld_relaxed(status) == kErrTimeout)) return false;
       __nanosleep(40);
       continue;
     }
-    uint32_t c = lane <= need ? (uint32_t)w : 0u;
+    uint32_t c = lane < first_inc ? (uint32_t)cs : (lane == first_inc && j >= 0 ? (uint32_t)inc : 0u);
     asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(c) : "r"(0xFFFFFFFFu));
     sum += c;
     if (first_inc < 32u) break;
-    j -= 32;
+    k -= 32;
   }
+  if (lane == 0 && seg > 0) st_relaxed(sc.seg_inc + (seg - 1u), scan_word(sc.epoch, 2u, (uint32_t)(sum - own)));
   *excl = sum;
   return true;
 }
