@@ -19,7 +19,7 @@ namespace {
 
 using fh::Plan;
 
-constexpr size_t kSmemLimit = 227 * 1024 - 1024;  // dynamic shared memory a CTA may ask for
+constexpr size_t kSmemLimit = 227 * 1024 - 4096;  // dynamic shared memory a CTA may ask for
 constexpr size_t kTileTarget = 32 * 1024;         // dense bytes a tile of the generic kernel aims for
 constexpr size_t kStageTarget = 72 * 1024;        // shared memory the stages of the CTA-team kernel aim for
 constexpr size_t kWarpStageTarget = 72 * 1024;    // ... and those of the warp-team kernel (two CTAs per SM)
@@ -114,7 +114,7 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   Variant v;
   // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
   const bool whole16 = pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0;
-  if (compress && pl.groups <= 4096 && (whole16 || pl.groups <= 256)) {
+  if (compress && (pl.groups <= 256 || whole16)) {
     v.fast = true;
     if (pl.groups <= 256) {
       uint32_t t = pow2_ceil((pl.groups + 7) / 8);
@@ -122,9 +122,9 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
       v.G = 8;  // the warp-team kernels keep eight groups per thread
       pl.ppt = fh::kThreads / pl.team;
     } else {
-      v.cta = true;
-      pl.team = fh::kThreads;
-      v.G = (int)pow2_ceil((pl.groups + fh::kThreads - 1) / fh::kThreads);
+      v.cta = true;  // CTA size by plane size: enough work per thread between barriers
+      pl.team = pl.plane_bytes <= 16 * 1024 ? 128 : (pl.plane_bytes <= 32 * 1024 ? 256 : 512);
+      v.G = 0;
       pl.ppt = 1;
     }
     if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
@@ -132,7 +132,8 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * sal_words) : 0;
     const uint32_t nsal_teams = v.cta ? 1 : fh::kThreads / pl.team;
     uint32_t ns = (uint32_t)((v.cta ? kStageTarget : kWarpStageTarget) / pl.stage_bytes);
-    ns = ns < 2 ? 2 : (ns > (uint32_t)fh::kMaxStages ? (uint32_t)fh::kMaxStages : ns);
+    const uint32_t ns_max = v.cta ? 3u : (uint32_t)fh::kMaxStages;
+    ns = ns < 2 ? 2 : (ns > ns_max ? ns_max : ns);
     for (;;) {
       pl.nstage = ns;
       pl.sm_tile = 0;
@@ -284,12 +285,12 @@ int launch_generic_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t str
   return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
-template <int DT, bool SIGMA, int G>
+template <int DT, bool SIGMA, int NT>
 int launch_cta_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
   int grid = 0;
-  int rc = grid_for(fh::compress_cta<DT, SIGMA, G>, pl.sm_total, pl.ntiles, &grid);
+  int rc = grid_for(fh::compress_cta<DT, SIGMA, NT>, pl.sm_total, pl.ntiles, &grid, NT);
   if (rc != FH_OK) return rc;
-  fh::compress_cta<DT, SIGMA, G><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
+  fh::compress_cta<DT, SIGMA, NT><<<grid, NT, pl.sm_total, stream>>>(pl, a);
   return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
@@ -321,11 +322,10 @@ int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, c
     const bool fullvec = pl.plane_bytes % 16 == 0 && pl.HW % 4 == 0 && pl.groups == 8u * pl.team;
     return fullvec ? launch_warp_tt<DT, SIGMA, true>(pl, a, stream) : launch_warp_tt<DT, SIGMA, false>(pl, a, stream);
   }
-  switch (v.G) {
-    case 2: return launch_cta_t<DT, SIGMA, 2>(pl, a, stream);
-    case 4: return launch_cta_t<DT, SIGMA, 4>(pl, a, stream);
-    case 8: return launch_cta_t<DT, SIGMA, 8>(pl, a, stream);
-    case 16: return launch_cta_t<DT, SIGMA, 16>(pl, a, stream);
+  switch (pl.team) {
+    case 128: return launch_cta_t<DT, SIGMA, 128>(pl, a, stream);
+    case 256: return launch_cta_t<DT, SIGMA, 256>(pl, a, stream);
+    case 512: return launch_cta_t<DT, SIGMA, 512>(pl, a, stream);
   }
   return FH_ERR_UNSUPPORTED;
 }

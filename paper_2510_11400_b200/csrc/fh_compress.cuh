@@ -371,7 +371,7 @@ __device__ __forceinline__ void write_nonnormal(const Team& t, const Plan& pl, c
 template <int DT, int BITS>
 __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_red[kWarps * 5];
+  __shared__ double s_red[kMaxWarps * 5];
   __shared__ uint32_t s_tile, s_skip;
   __shared__ unsigned long long s_base16;
 
@@ -756,7 +756,7 @@ __device__ __noinline__ void tile_place_sparse(const Plan& pl, const CompressArg
 template <int DT, bool SIGMA, int TT, bool FULLVEC>
 __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_red[kWarps * 5];
+  __shared__ double s_red[kMaxWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_classified[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages], s_nn[kMaxStages], s_nnmask[kMaxStages], s_skip[kMaxStages];
   __shared__ volatile uint32_t s_placed[kMaxStages];  // tile + 1 once the tile's overflow parts are placed
@@ -973,151 +973,237 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
   cta_exit(pl, a, d);
 }
 
-template <int DT, bool SIGMA, int G>
-__global__ void __launch_bounds__(kThreads, 2) compress_cta(const Plan pl, const CompressArgs a) {
+// -------------------------------------------------------------------------------------------------
+// CTA-team kernel: planes of more than 256 groups (whole 16-byte chunks).  One plane per tile, all
+// NT threads of the CTA work on it.  The plane stays in its shared-memory stage and is swept two or
+// three times (min/max; fixed-point moments; count + codes), so that few registers are needed and
+// several CTAs fit an SM.  Thread 0 keeps the next ticket in flight while the CTA works.
+// -------------------------------------------------------------------------------------------------
+template <int DT>
+__device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, float (&v)[4]) {
+  if (DT == kF32) {
+    const float4 t4 = reinterpret_cast<const float4*>(plane)[g];
+    v[0] = t4.x; v[1] = t4.y; v[2] = t4.z; v[3] = t4.w;
+  } else {
+    const uint2 t2 = reinterpret_cast<const uint2*>(plane)[g];
+    v[0] = __uint_as_float(t2.x << 16); v[1] = __uint_as_float(t2.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(t2.y << 16); v[3] = __uint_as_float(t2.y & 0xFFFF0000u);
+  }
+}
+
+#define FH_CTA_STORE_CODES(BITS)                                                                              \
+  {                                                                                                           \
+    constexpr uint32_t bias = kMagicBits * (1u + (1u << (BITS)) + (1u << (2 * (BITS))) + (1u << (3 * (BITS)))); \
+    _Pragma("unroll 2") for (uint32_t g = tid; g < groups; g += NT) {                                         \
+      float v[4];                                                                                             \
+      lds_group<DT>(plane, g, v);                                                                             \
+      uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(v[0], lo), inv, kMagicF));                          \
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(v[1], lo), inv, kMagicF)) << (BITS);                        \
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(v[2], lo), inv, kMagicF)) << (2 * (BITS));                  \
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(v[3], lo), inv, kMagicF)) << (3 * (BITS));                  \
+      word -= bias;                                                                                           \
+      if ((BITS) == 2) slot[g] = (uint8_t)word;                                                               \
+      else if ((BITS) == 4) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;                            \
+      else reinterpret_cast<uint32_t*>(slot)[g] = word;                                                       \
+      if (COUNT) {                                                                                            \
+        if (one_sided) {                                                                                      \
+          c0 += (v[0] > thi) + (v[2] > thi);                                                                  \
+          c1 += (v[1] > thi) + (v[3] > thi);                                                                  \
+        } else {                                                                                              \
+          c0 += ((v[0] > thi) || (v[0] < tlo)) + ((v[2] > thi) || (v[2] < tlo));                              \
+          c1 += ((v[1] > thi) || (v[1] < tlo)) + ((v[3] > thi) || (v[3] < tlo));                              \
+        }                                                                                                     \
+      }                                                                                                       \
+    }                                                                                                         \
+  }
+
+template <int DT, bool SIGMA, int NT>
+__global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const CompressArgs a) {
+  constexpr int NW = NT / 32;
+  constexpr bool COUNT = SIGMA;
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_red[kWarps * 5];
+  __shared__ double s_red[kMaxWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
-  __shared__ uint32_t s_nonnormal[2], s_skip, s_abort;  // s_nonnormal: one slot per tile parity
+  __shared__ uint32_t s_skip, s_abort;
   __shared__ unsigned long long s_base16;
   __shared__ Plan s_pl;          // copies for the outlined slow path
   __shared__ CompressArgs s_a;
 
-  const uint32_t tid = threadIdx.x;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   if (tid == 0) {
     s_pl = pl;
     s_a = a;
   }
   Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
-  uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + 16u * pl.ppt);
+  uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + 16u);
+  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal);
   const Dest d = make_dest(pl, a);
-  constexpr bool CTA = true;
-  const Team team = make_team(kThreads, s_red);
-  const uint32_t T = kThreads;
-  const uint32_t my_team = 0u;
-  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
-  const uint32_t nstage = pl.nstage;
-  const bool vec = (pl.plane_bytes & 15u) == 0u;
-  const bool full = vec && pl.groups == (uint32_t)G * T;
+  const Team team = make_team(NT, s_red);
+  const uint32_t nstage = pl.nstage, groups = pl.groups, bits = (uint32_t)pl.bits;
   uint32_t rp = 0;
-  SalientInfo info = {0, 0, 0, 0};  // measurement of this team's salient plane, kept across the placement
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
 
-  // ---- pipeline prologue: barriers, first tiles in flight
   if (tid == 0) {
     for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
     fence_mbar_init();
-    s_nonnormal[0] = 0;
-    s_nonnormal[1] = 0;
     s_abort = 0;
   }
   __syncthreads();
-  // thread 0: take a ticket and start its load into stage s.  Tiles whose size is not a multiple of
-  // 16 bytes (only the last tile of a tensor of ragged planes) are not bulk-copied: they are loaded
-  // cooperatively when their turn comes.
+  uint32_t next_ticket = 0;  // thread 0: the ticket for the next load, requested one tile ahead
   auto issue = [&](uint32_t s) {
-    const uint32_t t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+    const uint32_t t = next_ticket;
     s_tiles[s] = t;
     if (t < pl.ntiles) {
-      const uint64_t p0 = (uint64_t)t * pl.ppt;
-      const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
-      const uint32_t bytes = np * (uint32_t)pl.plane_bytes;
-      if ((bytes & 15u) == 0u) {
-        fence_proxy_async();
-        mbar_expect_tx(&s_full[s], bytes);
-        bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + p0 * pl.plane_bytes, bytes, &s_full[s]);
-      }
+      fence_proxy_async();
+      mbar_expect_tx(&s_full[s], (uint32_t)pl.plane_bytes);
+      bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + (uint64_t)t * pl.plane_bytes,
+               (uint32_t)pl.plane_bytes, &s_full[s]);
+      next_ticket = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
     }
   };
-  if (tid == 0)
+  if (tid == 0) {
+    next_ticket = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
     for (uint32_t s = 0; s < nstage; ++s) issue(s);
+  }
   __syncthreads();
 
-  uint32_t uses[kMaxStages] = {0, 0, 0, 0};  // completed bulk loads per stage (barrier phase)
-  for (uint32_t it = 0;; ++it) {
-    const uint32_t s = it % nstage;
+  uint32_t s = 0, phase = 0;
+  for (;;) {
     const uint32_t tile = s_tiles[s];
     if (tile >= pl.ntiles) break;
-    const uint64_t p0 = (uint64_t)tile * pl.ppt;
-    const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
-    uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
-    const uint32_t tile_bytes = np * (uint32_t)pl.plane_bytes;
-    bool ready = true;
-    if ((tile_bytes & 15u) == 0u) {
-      uint32_t u = 0;
-#pragma unroll
-      for (int k = 0; k < kMaxStages; ++k)
-        if (k == (int)s) u = uses[k]++;
-      ready = mbar_wait(&s_full[s], u & 1u, 1u << 20);
-      ready = __all_sync(0xFFFFFFFFu, ready);
-      if (!ready) s_abort = 1;  // the load never arrived
-    } else {
-      __syncthreads();  // ragged last tile: plain loads by everybody
-      for (uint32_t i = tid; i < tile_bytes / 2u; i += kThreads)
-        reinterpret_cast<uint16_t*>(stage)[i] = reinterpret_cast<const uint16_t*>(a.src + p0 * pl.plane_bytes)[i];
-      __syncthreads();
-    }
+    bool ready = mbar_wait(&s_full[s], (phase >> s) & 1u, 1u << 20);
+    ready = __all_sync(0xFFFFFFFFu, ready);
+    phase ^= 1u << s;
+    if (!ready) s_abort = 1;
+    const uint8_t* plane = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+    const uint64_t gp = tile;
 
-    if (ready && (CTA || my_team < np)) {
-      const uint32_t lp = my_team;
-      const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
-      Rec r;
-      plane_sweep_any<DT, SIGMA, G, kThreads, false>(team, pl, d, a, plane, p0 + lp, vec, rp, r);
-      if ((r.meta & 3u) != kClsNormal) {
-        info = salient_measure<DT>(team, s_pl, plane, sal);
-        r.size = info.size;
-        if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
-          r.meta = (r.meta & ~3u) | kClsRaw;
-          r.size = (uint32_t)pl.plane_bytes;
+    // ---- sweep 1: minimum and maximum
+    float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000), lo1 = lo, hi1 = hi;
+    if (ready) {
+#pragma unroll 2
+      for (uint32_t g = tid; g < groups; g += 2 * NT) {
+        float v[4];
+        lds_group<DT>(plane, g, v);
+        lo = min_nan(lo, min_nan(min3_nan(v[0], v[1], v[2]), v[3]));
+        hi = max_nan(hi, max_nan(max3_nan(v[0], v[1], v[2]), v[3]));
+        if (g + NT < groups) {
+          lds_group<DT>(plane, g + NT, v);
+          lo1 = min_nan(lo1, min_nan(min3_nan(v[0], v[1], v[2]), v[3]));
+          hi1 = max_nan(hi1, max_nan(max3_nan(v[0], v[1], v[2]), v[3]));
         }
-        if (team.lane == 0) atomicAdd(&s_nonnormal[it & 1u], 1u);
       }
-      if (team.lane == 0) rec[lp] = r;
     }
-    __syncthreads();
+    lo = min_nan(lo, lo1);
+    hi = max_nan(hi, hi1);
+    team_minmax(team, lo, hi, rp);  // one barrier: also tells every thread about an abort
     if (s_abort) break;
+    if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && tid == 0)
+      atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
 
-    // Warps may run one tile ahead of each other between barriers, hence the flag per tile parity;
-    // it is cleared only behind the extra barriers of the slow path.
-    if (s_nonnormal[it & 1u] == 0) {
-      // ---- common case: nothing to place; the tile publishes a zero size
-      if (pl.mode != kModeOff && tid == 0) scan_publish(a.scan, tile, 0u);
+    // ---- sweep 2: fixed-point moments, thresholds
+    float tlo = 0.0f, thi = 0.0f;
+    bool one_sided = true, need_count = false;
+    if (SIGMA) {
+      const SigmaScale sc = sigma_scale(lo, hi);
+      uint32_t as = 0, aq = 0, ng = 0;
+#pragma unroll 2
+      for (uint32_t g = tid; g < groups; g += NT) {
+        float v[4];
+        lds_group<DT>(plane, g, v);
+        sigma_addends4(v[0], v[1], v[2], v[3], sc, as, aq);
+        ++ng;
+      }
+      long long Is, Iq;
+      team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
+      sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
+      need_count = hi > thi || lo < tlo;  // otherwise no element can lie outside
+      one_sided = lo >= tlo;
+    }
+
+    // ---- sweep 3: codes into the plane's slot (and the outlier count).  A plane that turns out
+    // salient has its slot rewritten by the slow path below.
+    float inv, scale;
+    quant_params(lo, hi, (1u << bits) - 1u, inv, scale);
+    uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
+    uint32_t c0 = 0, c1 = 0;
+    if (d.fits && pl.mode != kModeAll) {
+      if (!need_count) {
+        thi = __int_as_float(0x7F800000);  // nothing is counted
+        one_sided = true;
+      }
+      if (bits == 2u) FH_CTA_STORE_CODES(2)
+      else if (bits == 4u) FH_CTA_STORE_CODES(4)
+      else FH_CTA_STORE_CODES(8)
+      const uint32_t code_bytes = groups * bits / 2u;
+      for (uint32_t o = a4(code_bytes) + 4u * tid; o < pl.npay; o += 4u * NT) *reinterpret_cast<uint32_t*>(slot + o) = 0u;
+      if (tid == 0)
+        for (uint32_t o = code_bytes; o < a4(code_bytes); ++o) slot[o] = 0;
+    } else if (SIGMA && need_count) {  // nothing may be stored: count only
+      for (uint32_t g = tid; g < groups; g += NT) {
+        float v[4];
+        lds_group<DT>(plane, g, v);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) c0 += (v[e] > thi) || (v[e] < tlo);
+      }
+    }
+    uint32_t cls = kClsNormal, n_out = 0;
+    if (SIGMA) {
+      n_out = team_sum_u32(team, c0 + c1, rp);
+      if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
     } else {
-      // ---- place the overflow parts of this tile, then the owning teams write their planes
-      if (tid < 32) tile_place(s_pl, s_a, d, tile, np, rec, roff, &s_base16, &s_skip);
+      if (pl.mode == kModeAll) cls = kClsSalient;
+      __syncthreads();  // every thread is done with the stage
+    }
+
+    Rec r;
+    r.lo = 0.0f;
+    r.scale = 0.0f;
+    r.size = 0;
+    r.meta = cls | (n_out << 2);
+    if (cls == kClsNormal) {
+      r.lo = lo;
+      r.scale = scale;
+      if (tid == 0) {
+        if (d.fits) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
+        if (pl.mode != kModeOff) scan_publish(a.scan, tile, 0u);
+      }
+    } else {
+      // ---- slow path: the block-wise encoding of a salient plane, by the whole CTA
+      const SalientInfo info = salient_measure<DT>(team, s_pl, plane, sal);
+      r.size = info.size;
+      if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
+        r.meta = (r.meta & ~3u) | kClsRaw;
+        r.size = (uint32_t)pl.plane_bytes;
+      }
+      if (tid == 0) rec[0] = r;
       __syncthreads();
-      if (!s_skip && (CTA || my_team < np)) {
-        const uint32_t lp = my_team;
-        const Rec r = rec[lp];
-        if ((r.meta & 3u) != kClsNormal) {
-          const uint8_t* plane = stage + (uint64_t)lp * pl.plane_bytes;
-          SplitOut out;
-          out.slot = d.dst + pl.slots_off + (p0 + lp) * pl.npay;
-          out.ovf = d.dst + (s_base16 + roff[lp]) * 16ull;
-          out.npay = pl.npay;
-          if ((r.meta & 3u) == kClsRaw) {
-            raw_write(team, s_pl, plane, out);
-          } else {  // the team's scratch and `info` still hold the measurement of this plane
-            salient_write<DT>(team, s_pl, plane, info, sal, out);
-          }
-          if (team.lane == 0)
-            store_table_entry(d, p0 + lp, a16(r.size) > pl.npay ? (uint32_t)(s_base16 + roff[lp]) : 0u, r);
-        }
+      if (warp == 0) tile_place(s_pl, s_a, d, tile, 1u, rec, roff, &s_base16, &s_skip);
+      __syncthreads();
+      if (!s_skip) {
+        SplitOut out;
+        out.slot = slot;
+        out.ovf = d.dst + (s_base16 + roff[0]) * 16ull;
+        out.npay = pl.npay;
+        if ((r.meta & 3u) == kClsRaw) raw_write(team, s_pl, plane, out);
+        else salient_write<DT>(team, s_pl, plane, info, sal, out);
+        if (tid == 0) store_table_entry(d, gp, a16(r.size) > pl.npay ? (uint32_t)(s_base16 + roff[0]) : 0u, r);
       }
       __syncthreads();
-      if (tid == 0) s_nonnormal[it & 1u] = 0;
     }
-    // ---- the stage is free: next ticket, next load
+    // ---- the stage is free: next load (thread 0), next stage
     if (tid == 0) issue(s);
+    s = s + 1 == nstage ? 0 : s + 1;
+    // s_tiles[s] for the next iteration was written at least one barrier ago (nstage >= 2)
   }
 
   if (s_abort && tid == 0) {  // a load timed out: report, then wait (bounded) for copies still in flight
     atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-    for (uint32_t s = 0; s < nstage; ++s)
-      if (s_tiles[s] < pl.ntiles) {
-        mbar_wait(&s_full[s], 0u, 1u << 16);
-        mbar_wait(&s_full[s], 1u, 1u << 16);
+    for (uint32_t k = 0; k < nstage; ++k)
+      if (s_tiles[k] < pl.ntiles) {
+        mbar_wait(&s_full[k], 0u, 1u << 10);
+        mbar_wait(&s_full[k], 1u, 1u << 10);
       }
   }
   cta_exit(pl, a, d);

@@ -186,7 +186,7 @@ __device__ bool decode_salient(const Team& t, const Plan& pl, const SplitIn& in,
 template <int DT>
 __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, const DecompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_red[kWarps * 5];
+  __shared__ double s_red[kMaxWarps * 5];
   __shared__ uint32_t s_tile, s_hdr_ok, s_bits;
   __shared__ float s_eps;
   __shared__ unsigned long long s_total;

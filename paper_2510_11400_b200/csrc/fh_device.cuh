@@ -13,6 +13,7 @@ namespace fh {
 
 constexpr int kThreads = 256;             // CTA size of every kernel
 constexpr int kWarps = kThreads / 32;
+constexpr int kMaxWarps = 16;            // largest CTA of any kernel: 512 threads
 constexpr uint32_t kMagic = 0x31434846u;  // "FHC1"
 constexpr uint32_t kClsNormal = 0, kClsSalient = 1, kClsRaw = 2;
 constexpr int kModeAuto = 0, kModeOff = 1, kModeAll = 2;
@@ -292,13 +293,15 @@ struct Team {
   uint32_t lane;   // this thread's index inside the team
   uint32_t mask;   // warp member mask of the team (sub-warp teams)
   bool block;      // the team is the whole CTA
-  double* red;     // shared scratch for CTA-wide reductions: kWarps * 5 doubles (see red_half, team_excl_scan)
+  uint32_t nwarps; // warps of a CTA team
+  double* red;     // shared scratch for CTA-wide reductions: kMaxWarps * 5 doubles (see red_half, team_excl_scan)
 };
 
 __device__ __forceinline__ Team make_team(uint32_t team_size, double* red) {
   Team t;
   t.size = team_size;
   t.red = red;
+  t.nwarps = team_size >> 5;
   if (team_size > 32u) {
     t.block = true;
     t.lane = threadIdx.x;
@@ -315,6 +318,7 @@ __device__ __forceinline__ Team make_team(uint32_t team_size, double* red) {
 __device__ __forceinline__ Team make_warp_team(double* red) {
   Team t;
   t.size = 32;
+  t.nwarps = 1;
   t.red = red;
   t.block = false;
   t.lane = threadIdx.x & 31u;
@@ -331,7 +335,7 @@ __device__ __forceinline__ void team_sync(const Team& t) {
 // alternately (`rp` counts the reductions of this thread), so that one barrier per reduction
 // suffices: a half is rewritten only after the barrier of the reduction in between.
 __device__ __forceinline__ double* red_half(const Team& t, uint32_t& rp) {
-  double* r = t.red + ((rp++) & 1u) * (kWarps * 2);
+  double* r = t.red + ((rp++) & 1u) * (kMaxWarps * 2);
   return r;
 }
 
@@ -350,8 +354,7 @@ __device__ __forceinline__ void team_minmax(const Team& t, float& lo, float& hi,
     __syncthreads();
     lo = r[0];
     hi = r[1];
-#pragma unroll
-    for (int k = 1; k < kWarps; ++k) {
+    for (uint32_t k = 1; k < t.nwarps; ++k) {
       lo = min_nan(lo, r[k * 2]);
       hi = max_nan(hi, r[k * 2 + 1]);
     }
@@ -381,8 +384,7 @@ __device__ __forceinline__ void team_sum2(const Team& t, int32_t a, int32_t b, l
     __syncthreads();
     A = 0;
     B = 0;
-#pragma unroll
-    for (int k = 0; k < kWarps; ++k) {
+    for (uint32_t k = 0; k < t.nwarps; ++k) {
       A += r[k * 2];
       B += r[k * 2 + 1];
     }
@@ -406,8 +408,7 @@ __device__ __forceinline__ void team_sum2_wide(const Team& t, long long a, long 
   __syncthreads();
   A = 0;
   B = 0;
-#pragma unroll
-  for (int k = 0; k < kWarps; ++k) {
+  for (uint32_t k = 0; k < t.nwarps; ++k) {
     A += r[k * 2];
     B += r[k * 2 + 1];
   }
@@ -422,8 +423,7 @@ __device__ __forceinline__ uint32_t team_sum_u32(const Team& t, uint32_t v, uint
     if ((threadIdx.x & 31u) == 0) r[warp] = v;
     __syncthreads();
     v = 0;
-#pragma unroll
-    for (int k = 0; k < kWarps; ++k) v += r[k];
+    for (uint32_t k = 0; k < t.nwarps; ++k) v += r[k];
   }
   return v;
 }
@@ -443,7 +443,7 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
     }
     total = __shfl_sync(t.mask, incl, t.size - 1u, t.size);
   } else {
-    uint32_t* r = reinterpret_cast<uint32_t*>(t.red + kWarps * 4);  // region of its own, behind the two halves
+    uint32_t* r = reinterpret_cast<uint32_t*>(t.red + kMaxWarps * 4);  // region of its own, behind the two halves
     const uint32_t wl = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     for (uint32_t o = 1; o < 32u; o <<= 1) {
       const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
@@ -454,7 +454,7 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
     __syncthreads();
     uint32_t base = 0;
     total = 0;
-    for (uint32_t k = 0; k < (uint32_t)kWarps; ++k) {
+    for (uint32_t k = 0; k < t.nwarps; ++k) {
       if (k < warp) base += r[k];
       total += r[k];
     }
