@@ -148,6 +148,24 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
       --ns;
     }
   }
+  if (!compress) {
+    // decompress: sub-warp teams, planes assigned round-robin (ntiles only bounds the grid)
+    uint32_t t = pow2_ceil((pl.groups + 7) / 8);
+    pl.team = t > 32 ? 32 : t;
+    const uint32_t nteams = fh::kThreads / pl.team;
+    pl.sm_sal_stride = (uint32_t)A16(4 * sal_words);
+    pl.sm_total = nteams * 4 * pl.nblk + 16;
+    if (pl.sm_total > kSmemLimit) return FH_ERR_UNSUPPORTED;
+    pl.ppt = nteams;
+    {
+      const uint64_t chunks = (pl.groups + 8 * pl.team - 1) / (8 * pl.team);
+      const uint64_t ctas = (pl.P * chunks + nteams - 1) / nteams;
+      pl.ntiles = (uint32_t)(ctas > 0x7FFFFFFFull ? 0x7FFFFFFFull : ctas);
+    }
+    *out = pl;
+    if (var) *var = Variant();
+    return FH_OK;
+  }
   if (!v.fast) {
     v = Variant();
     if (pl.plane_bytes <= 8192) {
@@ -351,15 +369,28 @@ int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a,
   return rc;
 }
 
-template <int DT>
+template <int DT, int TT>
 int launch_decompress_t(const Plan& pl, const fh::DecompressArgs& a, cudaStream_t stream) {
   int grid = 0;
-  int rc = grid_for(fh::decompress_kernel<DT>, pl.sm_total, pl.ntiles, &grid);
+  int rc = grid_for(fh::decompress_kernel<DT, TT>, pl.sm_total, pl.ntiles, &grid);
   if (rc != FH_OK) return rc;
-  fh::decompress_kernel<DT><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
+  fh::decompress_kernel<DT, TT><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
   if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
   g_launches.fetch_add(1);
   return FH_OK;
+}
+
+template <int DT>
+int launch_decompress(const Plan& pl, const fh::DecompressArgs& a, cudaStream_t stream) {
+  switch (pl.team) {
+    case 1: return launch_decompress_t<DT, 1>(pl, a, stream);
+    case 2: return launch_decompress_t<DT, 2>(pl, a, stream);
+    case 4: return launch_decompress_t<DT, 4>(pl, a, stream);
+    case 8: return launch_decompress_t<DT, 8>(pl, a, stream);
+    case 16: return launch_decompress_t<DT, 16>(pl, a, stream);
+    case 32: return launch_decompress_t<DT, 32>(pl, a, stream);
+  }
+  return FH_ERR_UNSUPPORTED;
 }
 
 int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
@@ -408,8 +439,8 @@ int enqueue_decompress(const void* d_src, size_t src_bytes, const fh_tensor_desc
   a.dst = (uint8_t*)d_dst;
   a.d_status = d_status;
   a.sc = s->sc;
-  if (pl.dtype == FH_F32) return launch_decompress_t<fh::kF32>(pl, a, stream);
-  return launch_decompress_t<fh::kBF16>(pl, a, stream);
+  if (pl.dtype == FH_F32) return launch_decompress<fh::kF32>(pl, a, stream);
+  return launch_decompress<fh::kBF16>(pl, a, stream);
 }
 
 bool misaligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) != 0; }

@@ -1,10 +1,14 @@
 // Decompress kernel: container -> dense tensor, one pass.
 //
-// Tiles of consecutive planes are handed out by a ticket counter; one team of threads restores one
-// plane: unpack-and-dequantise for normal planes, verbatim copy for raw planes, and for outlier-rich
-// planes zero fill + CSR scatter + inverse Lorenzo walk of the dense blocks.  Every read of the
-// container is bounds-checked against src_bytes; a plane whose table entry or payload is
-// inconsistent is left unwritten and the call reports FH_ERR_CORRUPT.
+// Planes are independent and their slots sit at closed-form offsets, so the kernel needs no
+// hand-out and no barrier: team t of the grid restores planes t, t + teams, ...  A team is a
+// power-of-two slice of a warp (a whole warp for planes of 256 groups and more).  Normal planes are
+// the fused unpack-and-dequantise: code bytes are read straight from the slot (they are 1/16 to 1/4
+// of the output), four values per thread and step go out as one 16-byte (fp32) or 8-byte (bf16)
+// store.  Raw planes are copied; outlier-rich planes take zero fill + CSR scatter + inverse Lorenzo
+// walk of the dense blocks.  Every read of the container is bounds-checked against src_bytes; a
+// plane whose table entry or payload is inconsistent is left unwritten and the call reports
+// FH_ERR_CORRUPT.
 #pragma once
 
 #include "fh_device.cuh"
@@ -43,42 +47,10 @@ __device__ __forceinline__ float dequant(uint32_t q, float scale, float lo) {
   return __fmaf_rn(qf, scale, lo);
 }
 
-template <int DT, int BITS>
-__device__ __forceinline__ void decode_normal(const Team& t, const Plan& pl, const uint8_t* pay,
-                                              float lo, float scale, uint8_t* out) {
-  constexpr uint32_t L = (1u << BITS) - 1u;
-  const uint32_t HW = pl.HW, groups = pl.groups;
-  const bool vec = (pl.plane_bytes & (DT == kF32 ? 15u : 7u)) == 0u;  // dst base is 16-byte aligned
-  for (uint32_t g = t.lane; g < groups; g += t.size) {
-    uint32_t word;
-    if (BITS == 2) word = __ldg(pay + g);
-    else if (BITS == 4) word = __ldg(reinterpret_cast<const uint16_t*>(pay) + g);
-    else word = __ldg(reinterpret_cast<const uint32_t*>(pay) + g);
-    float v[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) v[k] = dequant((word >> (k * BITS)) & L, scale, lo);
-    const uint32_t i0 = g * 4u;
-    if (vec && i0 + 3u < HW) {
-      if (DT == kF32) {
-        reinterpret_cast<float4*>(out)[g] = make_float4(v[0], v[1], v[2], v[3]);
-      } else {
-        uint2 w;
-        w.x = f32_to_bf16_bits(v[0]) | (f32_to_bf16_bits(v[1]) << 16);
-        w.y = f32_to_bf16_bits(v[2]) | (f32_to_bf16_bits(v[3]) << 16);
-        reinterpret_cast<uint2*>(out)[g] = w;
-      }
-    } else {
-#pragma unroll
-      for (int k = 0; k < 4; ++k)
-        if (i0 + k < HW) store_elem<DT>(out, i0 + k, v[k]);
-    }
-  }
-}
-
 // Outlier-rich plane.  `scr` is the team's shared scratch: nblk words.  `ovf_avail` is the number of
 // readable bytes behind in.ovf.
 template <int DT>
-__device__ bool decode_salient(const Team& t, const Plan& pl, const SplitIn& in, uint64_t ovf_avail, float eps,
+__device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const SplitIn& in, uint64_t ovf_avail, float eps,
                                uint8_t* out, uint32_t* scr) {
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx, nbm = pl.nbm, e = (uint32_t)pl.esize, HW = pl.HW;
@@ -183,20 +155,45 @@ __device__ bool decode_salient(const Team& t, const Plan& pl, const SplitIn& in,
   return ok;
 }
 
-template <int DT>
+// Normal plane, whole groups, vector stores.  TT lanes; lane handles groups lane, lane + TT, ...
+#define FH_DECODE_NORMAL(BITS)                                                                             \
+  {                                                                                                        \
+    constexpr uint32_t L = (1u << (BITS)) - 1u;                                                            \
+    _Pragma("unroll 4") for (uint32_t g = g0 + lane; g < g1; g += TT) {                                    \
+      uint32_t word;                                                                                       \
+      if ((BITS) == 2) word = __ldg(slot + g);                                                             \
+      else if ((BITS) == 4) word = __ldg(reinterpret_cast<const uint16_t*>(slot) + g);                     \
+      else word = __ldg(reinterpret_cast<const uint32_t*>(slot) + g);                                      \
+      const float v0 = dequant(word & L, scale, lo), v1 = dequant((word >> (BITS)) & L, scale, lo);        \
+      const float v2 = dequant((word >> (2 * (BITS))) & L, scale, lo);                                     \
+      const float v3 = dequant((word >> (3 * (BITS))) & L, scale, lo);                                     \
+      if (DT == kF32) {                                                                                    \
+        reinterpret_cast<float4*>(out)[g] = make_float4(v0, v1, v2, v3);                                   \
+      } else {                                                                                             \
+        uint2 w;                                                                                           \
+        w.x = f32_to_bf16_bits(v0) | (f32_to_bf16_bits(v1) << 16);                                         \
+        w.y = f32_to_bf16_bits(v2) | (f32_to_bf16_bits(v3) << 16);                                         \
+        reinterpret_cast<uint2*>(out)[g] = w;                                                              \
+      }                                                                                                    \
+    }                                                                                                      \
+  }
+
+template <int DT, int TT>
 __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, const DecompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
-  __shared__ uint32_t s_tile, s_hdr_ok, s_bits;
+  __shared__ uint32_t s_hdr_ok, s_bits;
   __shared__ float s_eps;
   __shared__ unsigned long long s_total;
+  __shared__ Plan s_pl;  // copy for the outlined slow path, which takes it by address
   const uint32_t tid = threadIdx.x;
+  if (tid == 0) s_pl = pl;
   const unsigned long long off_in = a.d_off_in ? *a.d_off_in : 0ull;
   const uint8_t* src = a.src_base + off_in;
   const unsigned long long src_bytes = a.src_bytes > off_in ? a.src_bytes - off_in : 0ull;
-  const Team team = make_team(pl.team, s_red);
-  const uint32_t nteams = team.block ? 1u : kThreads / team.size;
-  const uint32_t my_team = team.block ? 0u : tid / team.size;
+  const Team team = make_team(TT, s_red);
+  constexpr uint32_t kTeams = kThreads / TT;
+  const uint32_t my_team = tid / TT, lane = team.lane;
 
   // header check (every CTA, it is 64 bytes)
   if (tid == 0) {
@@ -219,58 +216,66 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
   }
   __syncthreads();
   const bool hdr_ok = s_hdr_ok != 0;
-  const uint32_t bits = hdr_ok ? s_bits : 2u;
-  const float eps = s_eps;
-  const unsigned long long total = hdr_ok ? s_total : 0ull;
-  const uint32_t npay = a16(4u * ((pl.HW * bits + 31u) / 32u));
-  const unsigned long long slots_off = 64ull + 16ull * pl.P, ovf_off = slots_off + pl.P * (unsigned long long)npay;
-
-  for (;;) {
-    if (tid == 0) s_tile = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
-    __syncthreads();
-    const uint32_t tile = s_tile;
-    if (tile >= pl.ntiles) break;
-    const uint64_t p0 = (uint64_t)tile * pl.ppt;
-    const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
-    bool bad = !hdr_ok;
-    if (hdr_ok) {
-      for (uint32_t lp = my_team; lp < np; lp += nteams) {
-        const uint64_t gp = p0 + lp;
-        const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + gp);
-        const unsigned long long off = (unsigned long long)e.x * 16ull;
-        const uint32_t cls = e.y & 3u;
-        uint8_t* out = a.dst + gp * pl.plane_bytes;
-        const uint8_t* slot = src + slots_off + gp * npay;
-        if (cls == kClsNormal) {
-          if (off != slots_off + gp * npay) { bad = true; continue; }
-          const float lo = __uint_as_float(e.z), scale = __uint_as_float(e.w);
-          if (bits == 2u) decode_normal<DT, 2>(team, pl, slot, lo, scale, out);
-          else if (bits == 4u) decode_normal<DT, 4>(team, pl, slot, lo, scale, out);
-          else decode_normal<DT, 8>(team, pl, slot, lo, scale, out);
-        } else if (cls == kClsRaw || cls == kClsSalient) {
-          // the continuation, when there is one, lies in the overflow region
-          if (off != 0 && (off < ovf_off || off > total)) { bad = true; continue; }
-          SplitIn in;
-          in.slot = slot;
-          in.ovf = src + off;
-          in.npay = npay;
-          const unsigned long long ovf_avail = off ? total - off : 0ull;
-          if (cls == kClsRaw) {
-            if (pl.plane_bytes > npay && pl.plane_bytes - npay > ovf_avail) { bad = true; continue; }
-            for (uint32_t i = team.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += team.size)
-              reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)in.ld16(2u * i);
-          } else {
-            uint32_t* scr = reinterpret_cast<uint32_t*>(smem) + (uint64_t)my_team * pl.nblk;
-            if (!decode_salient<DT>(team, pl, in, ovf_avail, eps, out, scr)) bad = true;
+  bool bad = !hdr_ok;
+  if (hdr_ok) {
+    const uint32_t bits = s_bits;
+    const float eps = s_eps;
+    const unsigned long long total = s_total;
+    const uint32_t npay = a16(4u * ((pl.HW * bits + 31u) / 32u));
+    const unsigned long long slots_off = 64ull + 16ull * pl.P, ovf_off = slots_off + pl.P * (unsigned long long)npay;
+    const bool vec = (pl.plane_bytes & (DT == kF32 ? 15u : 7u)) == 0u;  // dst base is 16-byte aligned
+    const uint32_t nfull = vec ? pl.HW >> 2 : 0u;                       // groups restored with vector stores
+    // Work items are (plane, chunk of 8 * TT groups) pairs so that large planes spread over many
+    // teams; a salient or raw plane is restored as a whole by the team that draws its first chunk.
+    const uint32_t chunk_groups = 8u * TT;
+    const uint32_t chunks = (pl.groups + chunk_groups - 1u) / chunk_groups;
+    const uint64_t items = pl.P * chunks, stride = (uint64_t)gridDim.x * kTeams;
+    for (uint64_t item = (uint64_t)blockIdx.x * kTeams + my_team; item < items; item += stride) {
+      const uint64_t gp = item / chunks;
+      const uint32_t ch = (uint32_t)(item - gp * chunks);
+      const uint32_t g0 = ch * chunk_groups, g1 = min(nfull, g0 + chunk_groups);
+      const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + gp);
+      const unsigned long long off = (unsigned long long)e.x * 16ull;
+      const uint32_t cls = e.y & 3u;
+      uint8_t* out = a.dst + gp * pl.plane_bytes;
+      const uint8_t* slot = src + slots_off + gp * npay;
+      if (cls == kClsNormal) {
+        if (off != slots_off + gp * npay) { bad = true; continue; }
+        const float lo = __uint_as_float(e.z), scale = __uint_as_float(e.w);
+        if (bits == 2u) FH_DECODE_NORMAL(2)
+        else if (bits == 4u) FH_DECODE_NORMAL(4)
+        else FH_DECODE_NORMAL(8)
+        if (ch == chunks - 1u && nfull * 4u < pl.HW) {  // ragged or unaligned rest: element stores
+          const uint32_t L = (1u << bits) - 1u;
+          for (uint32_t i = nfull * 4u + lane; i < pl.HW; i += TT) {
+            const uint32_t bit = i * bits;
+            const uint32_t q = (__ldg(reinterpret_cast<const uint32_t*>(slot) + (bit >> 5)) >> (bit & 31u)) & L;
+            store_elem<DT>(out, i, dequant(q, scale, lo));
           }
-        } else {
-          bad = true;
         }
+      } else if (cls == kClsRaw || cls == kClsSalient) {
+        if (ch != 0) continue;
+        // the continuation, when there is one, lies in the overflow region
+        if (off != 0 && (off < ovf_off || off > total)) { bad = true; continue; }
+        SplitIn in;
+        in.slot = slot;
+        in.ovf = src + off;
+        in.npay = npay;
+        const unsigned long long ovf_avail = off ? total - off : 0ull;
+        if (cls == kClsRaw) {
+          if (pl.plane_bytes > npay && pl.plane_bytes - npay > ovf_avail) { bad = true; continue; }
+          for (uint32_t i = lane; i < (uint32_t)(pl.plane_bytes >> 1); i += TT)
+            reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)in.ld16(2u * i);
+        } else {
+          uint32_t* scr = reinterpret_cast<uint32_t*>(smem) + (uint64_t)my_team * pl.nblk;
+          if (!decode_salient<DT>(team, s_pl, in, ovf_avail, eps, out, scr)) bad = true;
+        }
+      } else {
+        bad = true;
       }
     }
-    if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
-    __syncthreads();
   }
+  if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
   __threadfence();
   __syncthreads();
   if (tid == 0) {
@@ -279,7 +284,6 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
       __threadfence();
       const uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
       if (a.d_status) *a.d_status = status_word(code);
-      st_relaxed(&a.sc->ticket, 0ull);
       st_relaxed(&a.sc->status, 0ull);
       st_relaxed(&a.sc->exited, 0ull);
     }
