@@ -138,7 +138,7 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
       pl.nstage = ns;
       pl.sm_tile = 0;
       pl.sm_rec = (uint32_t)A16((size_t)ns * pl.stage_bytes);
-      pl.sm_sal = pl.sm_rec + (v.cta ? 1u : ns) * (uint32_t)A16(20 * (size_t)pl.ppt);
+      pl.sm_sal = pl.sm_rec + (v.cta ? 1u : ns) * (uint32_t)A16(24 * (size_t)pl.ppt);
       pl.sm_total = pl.sm_sal + nsal_teams * pl.sm_sal_stride;
       if (pl.sm_total <= kSmemLimit) break;
       if (ns == 2) {  // the pipeline needs two stages
@@ -174,6 +174,7 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     } else {
       pl.team = fh::kThreads;
     }
+    if (pl.team < 32) pl.team = 32;  // the block-wise path works with whole warps
     const uint32_t nteams = pl.team > 32 ? 1 : fh::kThreads / pl.team;
     pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * sal_words) : 0;
     pl.nstage = 0;

@@ -45,63 +45,60 @@ struct SplitOut {
   __device__ __forceinline__ void st16(uint32_t o, uint32_t v) const { *reinterpret_cast<uint16_t*>(at(o)) = (uint16_t)v; }
 };
 
-// Residual codes of one dense 8x8 block (Eq. 7-9): first-order Lorenzo prediction on the
-// pre-quantised integers k, neighbours outside the block count as 0.  Returns the number of
-// verbatim elements.  WRITE: also emits the 64 code bytes (at logical offset o_codes) and the
-// verbatim values (from logical offset o_outl).
+// Pre-quantised integer of the element at (y, x); positions outside the plane count as value 0.
+template <int DT>
+__device__ __forceinline__ int32_t plane_k(const uint8_t* plane, int H, int W, int y, int x, float inv2e, bool* big) {
+  const float v = (y < H && x < W) ? load_elem<DT>(plane, (uint32_t)y * (uint32_t)W + (uint32_t)x) : 0.0f;
+  return dense_k(v, inv2e, big);
+}
+
+// Residual codes of one dense 8x8 block (Eq. 7-9), by all 32 lanes of a warp: first-order Lorenzo
+// prediction on the pre-quantised integers k, neighbours outside the block count as 0.  Every element
+// is independent because prediction runs on k, which follows from the input alone.  Lane l takes the
+// elements l and l + 32 of the block's raster order.  Returns the number of verbatim elements.
+// WRITE: also emits the 64 code bytes (logical offset o_codes) and the verbatim values (from logical
+// offset o_outl, raster order).
 template <int DT, bool WRITE>
-__device__ __forceinline__ uint32_t block_codes(const uint8_t* plane, int H, int W, int by, int bx, float inv2e,
-                                                const SplitOut& out, uint32_t o_codes, uint32_t o_outl) {
-  int32_t prev[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) prev[j] = 0;
+__device__ __forceinline__ uint32_t block_codes_warp(const uint8_t* plane, int H, int W, int by, int bx, float inv2e,
+                                                     const SplitOut& out, uint32_t o_codes, uint32_t o_outl) {
+  const uint32_t lane = threadIdx.x & 31u;
+  const int j = (int)(lane & 7u);
   uint32_t n_out = 0;
-#pragma unroll 1
-  for (int i = 0; i < 8; ++i) {
-    const int y = by * 8 + i;
-    int32_t left = 0, ul = 0;
-    uint32_t w0 = 0, w1 = 0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int x = bx * 8 + j;
-      const bool inpl = (y < H) && (x < W);
-      const uint32_t idx = (uint32_t)y * (uint32_t)W + (uint32_t)x;
-      const float v = inpl ? load_elem<DT>(plane, idx) : 0.0f;
-      bool big;
-      const int32_t k = dense_k(v, inv2e, &big);
-      const int32_t up = prev[j];
-      const int32_t delta = k - (up + left - ul);
-      uint32_t code;
-      if (!inpl) {
-        code = 128u;
-      } else if (big || delta > 127 || delta < -127) {
-        code = 0u;
-        if (WRITE) {
-          if (DT == kF32) out.st32(o_outl + 4u * n_out, reinterpret_cast<const uint32_t*>(plane)[idx]);
-          else out.st16(o_outl + 2u * n_out, reinterpret_cast<const uint16_t*>(plane)[idx]);
-        }
-        ++n_out;
-      } else {
-        code = (uint32_t)(delta + 128);
-      }
-      if (j < 4) w0 |= code << (8 * j);
-      else w1 |= code << (8 * (j - 4));
-      ul = up;
-      left = k;
-      prev[j] = k;
-    }
+  for (int half = 0; half < 2; ++half) {
+    const int i = half * 4 + (int)(lane >> 3);
+    const int y = by * 8 + i, x = bx * 8 + j;
+    const bool inpl = (y < H) && (x < W);
+    bool big, nb;
+    const int32_t k = plane_k<DT>(plane, H, W, y, x, inv2e, &big);
+    const int32_t up = i > 0 ? plane_k<DT>(plane, H, W, y - 1, x, inv2e, &nb) : 0;
+    const int32_t left = j > 0 ? plane_k<DT>(plane, H, W, y, x - 1, inv2e, &nb) : 0;
+    const int32_t ul = (i > 0 && j > 0) ? plane_k<DT>(plane, H, W, y - 1, x - 1, inv2e, &nb) : 0;
+    const int32_t delta = k - (up + left - ul);
+    const bool verbatim = inpl && (big || delta > 127 || delta < -127);
+    const uint32_t code = !inpl ? 128u : (verbatim ? 0u : (uint32_t)(delta + 128));
+    const uint32_t m = __ballot_sync(0xFFFFFFFFu, verbatim);
     if (WRITE) {
-      out.st32(o_codes + 8u * i, w0);
-      out.st32(o_codes + 8u * i + 4u, w1);
+      if (verbatim) {
+        const uint32_t rank = n_out + __popc(m & ((1u << lane) - 1u));
+        const uint32_t idx = (uint32_t)y * (uint32_t)W + (uint32_t)x;
+        if (DT == kF32) out.st32(o_outl + 4u * rank, reinterpret_cast<const uint32_t*>(plane)[idx]);
+        else out.st16(o_outl + 2u * rank, reinterpret_cast<const uint16_t*>(plane)[idx]);
+      }
+      uint32_t w = code | (__shfl_down_sync(0xFFFFFFFFu, code, 1) << 8);
+      w |= __shfl_down_sync(0xFFFFFFFFu, w, 2) << 16;
+      if ((lane & 3u) == 0u) out.st32(o_codes + (uint32_t)half * 32u + lane, w);
     }
+    n_out += __popc(m);
   }
   return n_out;
 }
 
 // Block-wise path, measuring part (Section 4.4.1): non-zero mask pooled per 8x8 block against tau,
-// CSR row counts over the sparse blocks, verbatim counts of the dense blocks.  Leaves in shared
-// scratch: rowp[0..H] = CSR row pointers, blk_a[b] = 1 for dense blocks, blk_b[b] = rank of block b
-// among the dense blocks, blk_c[b] = index of the block's first verbatim value.
+// CSR row counts over the sparse blocks, verbatim counts of the dense blocks.  The team is a whole
+// warp or a whole CTA.  Leaves in shared scratch: rowp[0..H] = CSR row pointers, blk_a[b] = 1 for
+// dense blocks, blk_b[b] = rank of block b among the dense blocks, blk_c[b] = index of the block's
+// first verbatim value.
 template <int DT>
 __device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint8_t* plane, uint32_t* sal) {
   uint32_t* rowp = sal;
@@ -110,7 +107,9 @@ __device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& p
   uint32_t* blk_c = blk_b + pl.nblk;
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx;
+  const uint32_t nw = t.block ? t.nwarps : 1u, wid = t.block ? threadIdx.x >> 5 : 0u, lane32 = threadIdx.x & 31u;
   for (uint32_t b = t.lane; b < nblk; b += t.size) blk_a[b] = 0;
+  for (uint32_t y = t.lane; y <= (uint32_t)H; y += t.size) rowp[y] = 0;
   team_sync(t);
   // pooled mask: non-zero count per block, accumulated from (block, row) items
   for (uint32_t r = t.lane; r < nblk * 8u; r += t.size) {
@@ -132,22 +131,27 @@ __device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& p
   team_sync(t);
   SalientInfo info;
   info.n_dense = team_excl_scan(t, blk_b, nblk);
-  // CSR over non-zeros in sparse blocks
-  for (int y = (int)t.lane; y <= H; y += (int)t.size) {
-    uint32_t cnt = 0;
-    if (y < H) {
-      const uint32_t* brow = blk_a + (uint32_t)(y >> 3) * nbx;
-      for (int x = 0; x < W; ++x) cnt += (load_elem<DT>(plane, (uint32_t)y * W + x) != 0.0f) && !brow[x >> 3];
+  // CSR row counts: non-zeros of the sparse blocks, again from (block, row) items
+  for (uint32_t r = t.lane; r < nblk * 8u; r += t.size) {
+    const uint32_t b = r >> 3, i = r & 7u;
+    const int y = (int)(b / nbx) * 8 + (int)i, x0 = (int)(b % nbx) * 8;
+    if (y < H && !blk_a[b]) {
+      uint32_t cnt = 0;
+      const int x1 = min(W, x0 + 8);
+      for (int x = x0; x < x1; ++x) cnt += load_elem<DT>(plane, (uint32_t)y * W + x) != 0.0f;
+      if (cnt) atomicAdd(&rowp[y], cnt);
     }
-    rowp[y] = cnt;
   }
   team_sync(t);
   info.nnz_s = team_excl_scan(t, rowp, (uint32_t)H + 1u);
-  // verbatim counts of dense blocks
+  // verbatim counts of the dense blocks, one warp per block
   const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
   const SplitOut none = {nullptr, nullptr, 0};
-  for (uint32_t b = t.lane; b < nblk; b += t.size)
-    blk_c[b] = blk_a[b] ? block_codes<DT, false>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, none, 0, 0) : 0u;
+  for (uint32_t b = wid; b < nblk; b += nw) {
+    uint32_t n = 0;
+    if (blk_a[b]) n = block_codes_warp<DT, false>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, none, 0, 0);
+    if (lane32 == 0) blk_c[b] = n;
+  }
   team_sync(t);
   info.n_out_d = team_excl_scan(t, blk_c, nblk);
   const uint32_t e = (uint32_t)pl.esize;
@@ -159,13 +163,14 @@ __device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& p
 // Block-wise path, writing part; `sal` holds what salient_measure left.
 template <int DT>
 __device__ __noinline__ void salient_write(const Team& t, const Plan& pl, const uint8_t* plane, const SalientInfo& info,
-                              const uint32_t* sal, const SplitOut& out) {
+                                           const uint32_t* sal, const SplitOut& out) {
   const uint32_t* rowp = sal;
   const uint32_t* blk_a = sal + pl.H + 1;
   const uint32_t* blk_b = blk_a + pl.nblk;
   const uint32_t* blk_c = blk_b + pl.nblk;
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx, e = (uint32_t)pl.esize;
+  const uint32_t nw = t.block ? t.nwarps : 1u, wid = t.block ? threadIdx.x >> 5 : 0u, lane32 = threadIdx.x & 31u;
   const uint32_t o_bm = 16u, o_rp = o_bm + 4u * pl.nbm, o_col = o_rp + 4u * ((uint32_t)H + 1u);
   const uint32_t o_val = o_col + a4(2u * info.nnz_s), o_codes = o_val + a4(e * info.nnz_s);
   const uint32_t o_outl = o_codes + 64u * info.n_dense;
@@ -189,24 +194,29 @@ __device__ __noinline__ void salient_write(const Team& t, const Plan& pl, const 
     out.st32(o_bm + 4u * w, word);
   }
   for (uint32_t y = t.lane; y <= (uint32_t)H; y += t.size) out.st32(o_rp + 4u * y, rowp[y]);
-  for (int y = (int)t.lane; y < H; y += (int)t.size) {
+  // CSR entries: one warp per row, columns in chunks of 32, positions by ballot
+  for (int y = (int)wid; y < H; y += (int)nw) {
     uint32_t o = rowp[y];
     const uint32_t* brow = blk_a + (uint32_t)(y >> 3) * nbx;
-    for (int x = 0; x < W; ++x) {
-      const uint32_t idx = (uint32_t)y * W + x;
-      if (load_elem<DT>(plane, idx) != 0.0f && !brow[x >> 3]) {
-        out.st16(o_col + 2u * o, (uint32_t)x);
-        if (DT == kF32) out.st32(o_val + 4u * o, reinterpret_cast<const uint32_t*>(plane)[idx]);
-        else out.st16(o_val + 2u * o, reinterpret_cast<const uint16_t*>(plane)[idx]);
-        ++o;
+    for (int x0 = 0; x0 < W; x0 += 32) {
+      const int x = x0 + (int)lane32;
+      const uint32_t idx = (uint32_t)y * W + (uint32_t)x;
+      const bool take = x < W && load_elem<DT>(plane, idx) != 0.0f && !brow[x >> 3];
+      const uint32_t m = __ballot_sync(0xFFFFFFFFu, take);
+      if (take) {
+        const uint32_t pos = o + __popc(m & ((1u << lane32) - 1u));
+        out.st16(o_col + 2u * pos, (uint32_t)x);
+        if (DT == kF32) out.st32(o_val + 4u * pos, reinterpret_cast<const uint32_t*>(plane)[idx]);
+        else out.st16(o_val + 2u * pos, reinterpret_cast<const uint16_t*>(plane)[idx]);
       }
+      o += __popc(m);
     }
   }
   const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
-  for (uint32_t b = t.lane; b < nblk; b += t.size)
+  for (uint32_t b = wid; b < nblk; b += nw)
     if (blk_a[b])
-      block_codes<DT, true>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, out, o_codes + 64u * blk_b[b],
-                            o_outl + e * blk_c[b]);
+      block_codes_warp<DT, true>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, out, o_codes + 64u * blk_b[b],
+                                 o_outl + e * blk_c[b]);
 }
 
 // Raw plane: verbatim copy through the slot into the overflow part, zero padded.
@@ -717,11 +727,11 @@ __device__ __forceinline__ void plane_sweep_any(const Team& team, const Plan& pl
 constexpr int kWarpKernelThreads = kThreads + 32;
 
 // Placement of a tile with salient / raw planes, executed by one warp.  ovf16[i] holds the overflow
-// size of plane i of the tile in 16-byte units (0 for normal planes); on return it holds the
-// plane's offset relative to the tile's base.
+// size of plane i of the tile in 16-byte units (0 for normal planes); the
+// sizes are left alone; poff[i] receives the plane's offset relative to the tile's base.
 __device__ __noinline__ void tile_place_sparse(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
-                                               uint32_t np, uint32_t* ovf16, unsigned long long* s_base16,
-                                               uint32_t* s_skip) {
+                                               uint32_t np, const uint32_t* ovf16, uint32_t* poff,
+                                               unsigned long long* s_base16, uint32_t* s_skip) {
   const uint32_t lane = threadIdx.x & 31u;
   uint32_t carry = 0;
   for (uint32_t base = 0; base < np; base += 32) {
@@ -732,7 +742,7 @@ __device__ __noinline__ void tile_place_sparse(const Plan& pl, const CompressArg
       const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
       if (lane >= o) incl += up;
     }
-    if (i < np) ovf16[i] = carry + incl - v;
+    if (i < np) poff[i] = carry + incl - v;
     carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
   }
   unsigned long long excl = 0;
@@ -897,20 +907,32 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
           mbar_arrive(&s_empty[s]);
         }
       } else {
-        // ---- slow path: salient / raw planes in this warp
-        uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
+        // ---- slow path: salient / raw planes in this warp.  Each of them is handled by all 32 lanes.
+        const Team wteam = make_warp_team(s_red);
         uint32_t* ovf16 = ovf16_all + s * pl.ppt;
-        SalientInfo info = {0, 0, 0, 0};
-        if (mine_nn) {
-          info = salient_measure<DT>(team, s_pl, plane, sal);
-          r.size = info.size;
-          if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
-            r.meta = (r.meta & ~3u) | kClsRaw;
-            r.size = (uint32_t)pl.plane_bytes;
+        uint32_t* poff = ovf16_all + nstage * pl.ppt + s * pl.ppt;  // offsets inside the tile, from the placement
+        uint32_t* sinfo = ovf16_all + 2u * nstage * pl.ppt + (s * pl.ppt) * 4u;  // per plane: size, nnz_s, n_dense, n_out_d
+        const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine_nn && team.lane == 0);
+        const uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+        uint32_t raw_mask = 0;  // bit L: the plane led by lane L turned out raw
+        for (uint32_t m = leaders; m; m &= m - 1u) {
+          const uint32_t L = (uint32_t)__ffs(m) - 1u, tlp = (warp * 32u + L) / TT;
+          const uint8_t* tplane = stage + (uint64_t)tlp * pl.plane_bytes;
+          uint32_t* tsal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)tlp * pl.sm_sal_stride);
+          const SalientInfo info = salient_measure<DT>(wteam, s_pl, tplane, tsal);
+          uint32_t size = info.size;
+          const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
+          if (raw) {
+            size = (uint32_t)pl.plane_bytes;
+            raw_mask |= 1u << L;
           }
-          if (team.lane == 0) {
-            ovf16[lp] = a16(r.size) > pl.npay ? (a16(r.size) - pl.npay) >> 4 : 0u;
-            atomicAdd((r.meta & 3u) == kClsRaw ? &a.sc->nraw : &a.sc->nsal, 1ull);
+          if (lane == 0) {
+            ovf16[tlp] = a16(size) > pl.npay ? (a16(size) - pl.npay) >> 4 : 0u;
+            sinfo[tlp * 4u + 0] = size;
+            sinfo[tlp * 4u + 1] = info.nnz_s;
+            sinfo[tlp * 4u + 2] = info.n_dense;
+            sinfo[tlp * 4u + 3] = info.n_out_d;
+            atomicAdd(raw ? &a.sc->nraw : &a.sc->nsal, 1ull);
           }
         }
         __syncwarp();
@@ -926,7 +948,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
           __threadfence_block();
           const uint32_t mask = *reinterpret_cast<volatile uint32_t*>(&s_nnmask[s]);
           if ((uint32_t)__ffs(mask) - 1u == warp) {  // the first such warp places the tile
-            tile_place_sparse(s_pl, s_a, d, tile, np, ovf16, &s_base16[s], &s_skip[s]);
+            tile_place_sparse(s_pl, s_a, d, tile, np, ovf16, poff, &s_base16[s], &s_skip[s]);
             __threadfence_block();
             __syncwarp();
             if (lane == 0) s_placed[s] = tile + 1u;
@@ -947,20 +969,37 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
           if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
         } else {
           __threadfence_block();
-          if (mine_nn) {
-            const unsigned long long off16 = s_base16[s] + ovf16[lp];
-            if (!s_skip[s]) {
+          const bool skip = s_skip[s] != 0;
+          for (uint32_t m = leaders; m; m &= m - 1u) {
+            const uint32_t L = (uint32_t)__ffs(m) - 1u, tlp = (warp * 32u + L) / TT;
+            const uint32_t meta_n = __shfl_sync(0xFFFFFFFFu, r.meta, L);  // the plane's three-sigma count
+            if (!skip) {
+              const uint8_t* tplane = stage + (uint64_t)tlp * pl.plane_bytes;
+              const uint32_t* tsal = reinterpret_cast<const uint32_t*>(smem + pl.sm_sal + (uint64_t)tlp * pl.sm_sal_stride);
+              const unsigned long long off16 = s_base16[s] + poff[tlp];
+              SalientInfo info;
+              info.size = sinfo[tlp * 4u + 0];
+              info.nnz_s = sinfo[tlp * 4u + 1];
+              info.n_dense = sinfo[tlp * 4u + 2];
+              info.n_out_d = sinfo[tlp * 4u + 3];
+              const bool raw = (raw_mask >> L) & 1u;
               SplitOut out;
-              out.slot = d.dst + pl.slots_off + ((uint64_t)p0 + lp) * pl.npay;
+              out.slot = d.dst + pl.slots_off + ((uint64_t)p0 + tlp) * pl.npay;
               out.ovf = d.dst + off16 * 16ull;
               out.npay = pl.npay;
-              if ((r.meta & 3u) == kClsRaw) raw_write(team, s_pl, plane, out);
-              else salient_write<DT>(team, s_pl, plane, info, sal, out);
-              if (team.lane == 0)
-                store_table_entry(d, (uint64_t)p0 + lp, a16(r.size) > pl.npay ? (uint32_t)off16 : 0u, r);
+              if (raw) raw_write(wteam, s_pl, tplane, out);
+              else salient_write<DT>(wteam, s_pl, tplane, info, tsal, out);
+              if (lane == 0) {
+                Rec tr;
+                tr.lo = 0.0f;
+                tr.scale = 0.0f;
+                tr.size = info.size;
+                tr.meta = (meta_n & ~3u) | (raw ? kClsRaw : kClsSalient);
+                store_table_entry(d, (uint64_t)p0 + tlp, a16(info.size) > pl.npay ? (uint32_t)off16 : 0u, tr);
+              }
             }
-            team_sync(team);
-            if (team.lane == 0) ovf16[lp] = 0;  // leave the array clean for the stage's next tile
+            __syncwarp();
+            if (lane == 0) ovf16[tlp] = 0;  // leave the array clean for the stage's next tile
           }
         }
         __syncwarp();
