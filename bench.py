@@ -51,6 +51,11 @@ def workload_specs(name: str):
         _, mib, dt = name.split("_")
         return synth.config4(int(mib), synth.F32 if dt == "f32" else synth.BF16), \
             f"configs[3]: single {mib} MiB {dt} tensor of 32x32 planes, ReLU(N(0,1))"
+    if name.startswith("shape_"):          # shape_<n>x<c>x<h>x<w>_<f32|bf16>_<kind>: one tensor, for profiling
+        _, dims, dt, kind = name.split("_", 3)
+        shape = tuple(int(v) for v in dims.split("x"))
+        return [synth.TensorSpec("shape", shape, synth.F32 if dt == "f32" else synth.BF16, kind, 900)], \
+            f"single {dt} tensor {dims}, {kind}"
     raise SystemExit(f"unknown workload {name}")
 
 

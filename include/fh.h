@@ -24,8 +24,9 @@
  *     Dense and packed device buffers must be 16-byte aligned.
  *   - fh_compress and fh_decompress only enqueue work on `stream` (a cudaStream_t passed as
  *     void*; NULL is the legacy default stream) and never synchronise.  Per stream the library keeps
- *     one small scratch allocation (scan flags) that it creates on first use and frees in
- *     fh_shutdown(); growing it for a larger tensor synchronises the device once.
+ *     one small scratch allocation (counters, and four bytes per plane of the largest tensor seen)
+ *     that it creates on first use and frees in fh_shutdown(); growing it for a tensor with more
+ *     planes synchronises the device once.
  *   - There is no CPU fallback: without a CUDA device every entry point that does work returns
  *     FH_ERR_CUDA.
  *
@@ -34,9 +35,16 @@
  *            u32 W | u8 block | u8 dense_bits | u8 rounding | u8 salient_mode | u16 rho_num |
  *            u16 rho_den | u16 tau_num | u16 tau_den | f32 eps | u32 n_salient | u32 n_raw |
  *            u64 tensor_id | u64 total_bytes
- *   [64,64+16P)  plane table, P = N*C entries: u32 payload offset / 16 | u32 meta (bits 0-1 class:
- *            0 normal, 1 salient, 2 raw; bits 2-31 three-sigma outlier count) | f32 lo | f32 scale
- *   payloads in plane order, each zero-padded to a multiple of 16 bytes
+ *   [64,64+16P)  plane table, P = N*C entries: u32 offset / 16 (see below) | u32 meta (bits 0-1
+ *            class: 0 normal, 1 salient, 2 raw; bits 2-31 three-sigma outlier count) | f32 lo |
+ *            f32 scale (lo = scale = 0 unless normal)
+ *   [64+16P, 64+16P+P*npay)  one slot per plane, npay = A16(4*ceil(HW*bits/32)) bytes, plane order
+ *   [64+16P+P*npay, total)   overflow region
+ *   A normal plane's codes fill its slot (zero padded); its table offset is that of the slot.  The
+ *   payload of a salient or raw plane is laid through its slot first and, if longer, continues in
+ *   the overflow region (continuations in plane order, each zero-padded to a multiple of 16 bytes);
+ *   its table offset is that of the continuation, 0 when there is none.  Slots sit at closed-form
+ *   offsets, so normal planes are written and read without knowing any other plane's size.
  *     normal : ceil(HW*bits/32) u32 words, element i in bits [(i*bits)%32, +bits) of word i*bits/32
  *     raw    : HW elements verbatim
  *     salient: u32 nnz_s | u32 n_dense | u32 n_out_d | u32 0 | block bitmap ceil(nblk/32) u32
@@ -189,8 +197,9 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
  * fh_compress without any allocation.  (The paper has no counterpart; this exists for callers of this
  * library.)
  *
- * fh_compress keeps its scan flags in a scratch buffer that it obtains with cudaMalloc on first use
- * and enlarges when a bigger tensor arrives.  Some callers cannot afford that: the codec is called
+ * fh_compress keeps its book-keeping (counters and the list of planes that take the block-wise
+ * path) in a scratch buffer that it obtains with cudaMalloc on first use and enlarges when a tensor
+ * with more planes arrives.  Some callers cannot afford that: the codec is called
  * exactly when device memory is short (a training engine compresses activations because its budget
  * is exhausted, so an allocation inside the codec can fail at the worst moment); a process whose
  * device memory is wholly pre-reserved by a framework pool has nothing left for the driver to hand
@@ -202,17 +211,16 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
  *
  * Arguments, output, status reporting and the produced bytes are exactly those of fh_compress.
  * Differences:
- *   - the tensor may span at most FH_STATIC_MAX_TILES tiles (a tile is a run of consecutive planes of
- *     8 to 32 KB of dense data, or a single plane when planes are larger; so roughly 0.5 to 2 GiB of
- *     dense data); anything larger returns FH_ERR_UNSUPPORTED and enqueues nothing;
+ *   - the tensor may have at most FH_STATIC_MAX_PLANES planes (n * c); anything larger returns
+ *     FH_ERR_UNSUPPORTED and enqueues nothing;
  *   - the first call on a device looks up the device address of the array (once per device, with
  *     that device current).  Make that first call outside any stream capture;
- *   - all calls on a device share the one array, which still holds the previous call's flags, so
- *     each call first clears the part it uses with a memset on `stream`.  Two calls that overlap on
- *     the GPU (different streams without ordering between them) race on it: order them.
+ *   - all calls on a device share the one array, which still holds the previous call's contents, so
+ *     each call first clears the counters it uses with a memset on `stream`.  Two calls that overlap
+ *     on the GPU (different streams without ordering between them) race on it: order them.
  */
-#define FH_STATIC_MAX_TILES 65536
-#define FH_STATIC_SCRATCH_BYTES (256 + 8 * FH_STATIC_MAX_TILES + 16 * (FH_STATIC_MAX_TILES / 32))
+#define FH_STATIC_MAX_PLANES 131072
+#define FH_STATIC_SCRATCH_BYTES (256 + 4 * 1024 + 4 * FH_STATIC_MAX_PLANES)
 int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                        size_t dst_capacity, uint64_t* d_out2, void* stream);
 

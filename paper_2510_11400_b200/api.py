@@ -18,7 +18,7 @@ FH_OK, FH_ERR_ARG, FH_ERR_UNSUPPORTED, FH_ERR_CAPACITY, FH_ERR_NONFINITE, FH_ERR
 FH_F32, FH_BF16 = 0, 1
 FH_SALIENT_AUTO, FH_SALIENT_OFF, FH_SALIENT_ALL = 0, 1, 2
 FH_KEEP, FH_COMPRESS, FH_EVICT = 0, 1, 2
-FH_STATIC_MAX_TILES = 65536
+FH_STATIC_MAX_PLANES = 131072
 
 EXPORTS = ["fh_default_params", "fh_version", "fh_device_count", "fh_compressed_bytes", "fh_compress",
            "fh_decompress", "fh_run_schedule", "fh_host_work_bytes", "fh_compress_host",
@@ -134,8 +134,9 @@ def fh_compress(d: fh_tensor_desc, p: fh_params, src, dst, out2=None, stream=Non
 
 def fh_compress_static(d: fh_tensor_desc, p: fh_params, src, dst, out2=None, stream=None,
                        capacity: Optional[int] = None) -> int:
-    """fh_compress for callers that must not allocate: same arguments and bytes, scan scratch in a fixed
-    array inside the library (at most FH_STATIC_MAX_TILES tiles; calls sharing a device must not overlap)."""
+    """fh_compress for callers that must not allocate: same arguments and bytes, book-keeping scratch in a
+    fixed array inside the library (at most FH_STATIC_MAX_PLANES planes; calls sharing a device must not
+    overlap)."""
     cap = dst.numel() * dst.element_size() if capacity is None else capacity
     return int(lib().fh_compress_static(C.byref(d), C.byref(p), src.data_ptr(), dst.data_ptr(), cap,
                                         out2.data_ptr() if out2 is not None else None, _stream_ptr(stream)))

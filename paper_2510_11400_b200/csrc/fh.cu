@@ -24,7 +24,6 @@ constexpr size_t kTileTarget = 32 * 1024;         // dense bytes a tile of the g
 constexpr size_t kStageTarget = 72 * 1024;        // shared memory the stages of the CTA-team kernel aim for
 constexpr size_t kWarpStageTarget = 72 * 1024;    // ... and those of the warp-team kernel (two CTAs per SM)
 constexpr uint32_t kMaxPpt = 2048;
-constexpr uint32_t kSpinLimit = 1u << 20;
 
 std::atomic<uint64_t> g_launches{0};
 
@@ -108,8 +107,18 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   const long double worst = 64.0L + (long double)pl.P * (16.0L + (long double)A16(pl.plane_bytes));
   if (worst / 16.0L >= 4294967295.0L) return FH_ERR_UNSUPPORTED;
   if (pl.P > 0x7FFFFFFFull) return FH_ERR_UNSUPPORTED;
-  const bool need_sal = compress ? (pl.mode != FH_SALIENT_OFF) : true;
   const size_t sal_words = compress ? (size_t)(pl.H + 1 + 3 * pl.nblk) : (size_t)pl.nblk;
+  pl.sal_words = (uint32_t)sal_words;
+  if (compress) {
+    // block-wise kernels: one plane per unit (a warp up to 8 KB, the CTA above)
+    pl.sk_cta = pl.plane_bytes > 8192 ? 1u : 0u;
+    pl.sk_threads = pl.sk_cta ? (pl.plane_bytes <= 32 * 1024 ? 256u : 512u) : 256u;
+    pl.sk_sal_off = (uint32_t)A16(pl.plane_bytes + 32);
+    pl.sk_unit_stride = pl.sk_sal_off + (uint32_t)A16(4 * sal_words);
+    pl.sk_pre_off = (pl.sk_cta ? 1u : pl.sk_threads / 32u) * pl.sk_unit_stride;
+    pl.sk_total = pl.sk_pre_off + 4u * fh::kMaxChunks;
+    if (pl.mode != FH_SALIENT_OFF && pl.sk_total > kSmemLimit) return FH_ERR_UNSUPPORTED;
+  }
 
   Variant v;
   // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
@@ -129,17 +138,13 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     }
     if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
     pl.stage_bytes = (uint32_t)((pl.ppt * pl.plane_bytes + 127) & ~(uint64_t)127);
-    pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * sal_words) : 0;
-    const uint32_t nsal_teams = v.cta ? 1 : fh::kThreads / pl.team;
     uint32_t ns = (uint32_t)((v.cta ? kStageTarget : kWarpStageTarget) / pl.stage_bytes);
     const uint32_t ns_max = v.cta ? 3u : (uint32_t)fh::kMaxStages;
     ns = ns < 2 ? 2 : (ns > ns_max ? ns_max : ns);
     for (;;) {
       pl.nstage = ns;
       pl.sm_tile = 0;
-      pl.sm_rec = (uint32_t)A16((size_t)ns * pl.stage_bytes);
-      pl.sm_sal = pl.sm_rec + (v.cta ? 1u : ns) * (uint32_t)A16(24 * (size_t)pl.ppt);
-      pl.sm_total = pl.sm_sal + nsal_teams * pl.sm_sal_stride;
+      pl.sm_total = (uint32_t)A16((size_t)ns * pl.stage_bytes);
       if (pl.sm_total <= kSmemLimit) break;
       if (ns == 2) {  // the pipeline needs two stages
         v.fast = false;
@@ -153,7 +158,6 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     uint32_t t = pow2_ceil((pl.groups + 7) / 8);
     pl.team = t > 32 ? 32 : t;
     const uint32_t nteams = fh::kThreads / pl.team;
-    pl.sm_sal_stride = (uint32_t)A16(4 * sal_words);
     pl.sm_total = nteams * 4 * pl.nblk + 16;
     if (pl.sm_total > kSmemLimit) return FH_ERR_UNSUPPORTED;
     pl.ppt = nteams;
@@ -174,9 +178,6 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     } else {
       pl.team = fh::kThreads;
     }
-    if (pl.team < 32) pl.team = 32;  // the block-wise path works with whole warps
-    const uint32_t nteams = pl.team > 32 ? 1 : fh::kThreads / pl.team;
-    pl.sm_sal_stride = need_sal ? (uint32_t)A16(4 * sal_words) : 0;
     pl.nstage = 0;
     pl.stage_bytes = 0;
     uint64_t ppt = kTileTarget / pl.plane_bytes;
@@ -185,16 +186,10 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     if (ppt > pl.P) ppt = pl.P;
     for (;;) {
       pl.ppt = (uint32_t)ppt;
-      if (compress) {
-        pl.sm_tile = 0;
-        pl.sm_out = (uint32_t)A16(ppt * pl.plane_bytes + 32);
-        pl.sm_rec = pl.sm_out + (uint32_t)(ppt * pl.npay);
-        pl.sm_sal = pl.sm_rec + (uint32_t)A16(20 * ppt);
-        pl.sm_total = pl.sm_sal + nteams * pl.sm_sal_stride;
-      } else {
-        pl.sm_sal = 0;
-        pl.sm_total = nteams * pl.sm_sal_stride;
-      }
+      pl.sm_tile = 0;
+      pl.sm_out = (uint32_t)A16(ppt * pl.plane_bytes + 32);
+      pl.sm_rec = pl.sm_out + (uint32_t)(ppt * pl.npay);
+      pl.sm_total = pl.sm_rec + (uint32_t)A16(16 * ppt);
       if (pl.sm_total <= kSmemLimit) break;
       if (ppt == 1) return FH_ERR_UNSUPPORTED;
       ppt = ppt / 2;
@@ -210,54 +205,48 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
 
 // ---- per-stream scratch ---------------------------------------------------------------------
 struct StreamScratch {
-  fh::Scratch* sc = nullptr;
-  unsigned long long* ts = nullptr;  // scan words
-  size_t ts_cap = 0;
-  uint32_t epoch = 0;
+  fh::Scratch* sc = nullptr;      // counters, followed by kMaxChunks chunk sums
+  uint32_t* worklist = nullptr;   // one word per plane of the largest tensor seen
+  size_t wl_cap = 0;
   unsigned long long* sched = nullptr;  // schedule runner: offsets, sizes, statuses
   size_t sched_cap = 0;
 };
+constexpr size_t kHeadBytes = 256 + 4 * fh::kMaxChunks;  // Scratch (padded) + chunk sums
 
 std::mutex g_mu;
 std::map<std::pair<int, cudaStream_t>, StreamScratch> g_scratch;
 int g_sm_count[64] = {0};
 
-int get_scratch(cudaStream_t stream, size_t ntiles, StreamScratch** out) {
+int get_scratch(cudaStream_t stream, size_t planes, StreamScratch** out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return FH_ERR_CUDA;
   StreamScratch& s = g_scratch[std::make_pair(dev, stream)];
   if (!s.sc) {
-    if (cudaMalloc(&s.sc, sizeof(fh::Scratch)) != cudaSuccess) return FH_ERR_CUDA;
-    if (cudaMemset(s.sc, 0, sizeof(fh::Scratch)) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMalloc(&s.sc, kHeadBytes) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMemset(s.sc, 0, kHeadBytes) != cudaSuccess) return FH_ERR_CUDA;
   }
-  if (ntiles > s.ts_cap) {
-    size_t cap = s.ts_cap ? s.ts_cap : 65536;
-    while (cap < ntiles) cap *= 2;
-    if (s.ts) {
+  if (planes > s.wl_cap) {
+    size_t cap = s.wl_cap ? s.wl_cap : 65536;
+    while (cap < planes) cap *= 2;
+    if (s.worklist) {
       cudaDeviceSynchronize();
-      cudaFree(s.ts);
-      s.ts = nullptr;
-      s.ts_cap = 0;
+      cudaFree(s.worklist);
+      s.worklist = nullptr;
+      s.wl_cap = 0;
     }
-    // tile words | segment counters | segment prefixes (a segment is 32 tiles)
-    const size_t words = cap + 2 * (cap / 32);
-    if (cudaMalloc(&s.ts, words * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
-    if (cudaMemset(s.ts, 0, words * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
-    s.ts_cap = cap;
+    if (cudaMalloc(&s.worklist, cap * sizeof(uint32_t)) != cudaSuccess) return FH_ERR_CUDA;
+    s.wl_cap = cap;
   }
   *out = &s;
   return FH_OK;
 }
 
-// Advance the 30-bit epoch; when it would wrap, clear the scan words so that stale epochs cannot match.
-int next_epoch(StreamScratch* s, cudaStream_t stream) {
-  if (s->epoch >= 0x3FFFFFF0u) {
-    if (s->ts && cudaMemsetAsync(s->ts, 0, (s->ts_cap + 2 * (s->ts_cap / 32)) * sizeof(unsigned long long), stream) != cudaSuccess)
-      return FH_ERR_CUDA;
-    s->epoch = 0;
-  }
-  ++s->epoch;
-  return FH_OK;
+// Chunks of the block-wise kernels: runs of 2^shift consecutive planes, at most kMaxChunks of them.
+void chunking(uint64_t planes, uint32_t* shift, uint32_t* nchunks) {
+  uint32_t sh = 0;
+  while (((planes + ((1ull << sh) - 1)) >> sh) > fh::kMaxChunks) ++sh;
+  *shift = sh;
+  *nchunks = (uint32_t)((planes + ((1ull << sh) - 1)) >> sh);
 }
 
 int sm_count() {
@@ -349,6 +338,22 @@ int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, c
   return FH_ERR_UNSUPPORTED;
 }
 
+template <int DT>
+int launch_blockwise(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
+  int g0 = 0, g1 = 0;
+  int rc = grid_for(fh::blockwise_kernel<DT, false>, pl.sk_total, 0x7FFFFFFFu, &g0, (int)pl.sk_threads);
+  if (rc != FH_OK) return rc;
+  rc = grid_for(fh::blockwise_kernel<DT, true>, pl.sk_total, 0x7FFFFFFFu, &g1, (int)pl.sk_threads);
+  if (rc != FH_OK) return rc;
+  fh::blockwise_kernel<DT, false><<<g0, pl.sk_threads, pl.sk_total, stream>>>(pl, a);
+  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  g_launches.fetch_add(1);
+  fh::blockwise_kernel<DT, true><<<g1, pl.sk_threads, pl.sk_total, stream>>>(pl, a);
+  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return FH_OK;
+}
+
 int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
   int rc;
   if (v.fast) {
@@ -366,7 +371,11 @@ int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a,
          : pl.bits == 4 ? launch_generic_t<fh::kBF16, 4>(pl, a, stream)
                         : launch_generic_t<fh::kBF16, 8>(pl, a, stream);
   }
-  if (rc == FH_OK) g_launches.fetch_add(1);
+  if (rc != FH_OK) return rc;
+  g_launches.fetch_add(1);
+  if (pl.mode == FH_SALIENT_OFF) return FH_OK;
+  // the planes the streaming kernel listed: measure, then place and write
+  rc = pl.dtype == FH_F32 ? launch_blockwise<fh::kF32>(pl, a, stream) : launch_blockwise<fh::kBF16>(pl, a, stream);
   return rc;
 }
 
@@ -403,9 +412,7 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   if (rc != FH_OK) return rc;
   std::lock_guard<std::mutex> lock(g_mu);
   StreamScratch* s = nullptr;
-  rc = get_scratch(stream, pl.ntiles, &s);
-  if (rc != FH_OK) return rc;
-  rc = next_epoch(s, stream);
+  rc = get_scratch(stream, pl.mode == FH_SALIENT_OFF ? 0 : pl.P, &s);
   if (rc != FH_OK) return rc;
   fh::CompressArgs a;
   a.src = (const uint8_t*)d_src;
@@ -415,12 +422,9 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   a.d_off_out = d_off_out;
   a.out2 = d_out2;
   a.sc = s->sc;
-  a.scan.ts = s->ts;
-  a.scan.seg_cs = s->ts + s->ts_cap;
-  a.scan.seg_inc = s->ts + s->ts_cap + s->ts_cap / 32;
-  a.scan.epoch = s->epoch;
-  a.scan.spin_limit = kSpinLimit;
-  a.nseg = (pl.ntiles + 31) / 32;
+  a.worklist = s->worklist;
+  a.chunk_ovf = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(s->sc) + 256);
+  chunking(pl.P, &a.chunk_shift, &a.nchunks);
   return launch_compress(pl, v, a, stream);
 }
 
@@ -667,11 +671,12 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
 }
 
 // ---- allocation-free compress -----------------------------------------------------------------
-// Scan scratch compiled into the device image: a Scratch header (padded to 256 bytes) followed by
-// FH_STATIC_MAX_TILES tile words and 2 * FH_STATIC_MAX_TILES / 32 segment words.  The name is a device symbol: host code must not pass it to a
-// kernel, it asks the runtime for the symbol's device address instead (once per device).
+// Scratch compiled into the device image: the counters (padded to 256 bytes), the chunk sums and a
+// work list of FH_STATIC_MAX_PLANES words.  The name is a device symbol: host code must not pass it
+// to a kernel, it asks the runtime for the symbol's device address instead (once per device).
 static __device__ __align__(256) unsigned char g_static_scratch[FH_STATIC_SCRATCH_BYTES];
 static_assert(sizeof(fh::Scratch) <= 256, "static scratch layout");
+static_assert(FH_STATIC_SCRATCH_BYTES == kHeadBytes + 4 * (size_t)FH_STATIC_MAX_PLANES, "static scratch layout");
 
 static std::mutex g_static_mu;
 static unsigned char* g_static_ptr[64] = {nullptr};
@@ -689,7 +694,7 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   Variant v;
   rc = make_plan(desc, params, true, &pl, &v);
   if (rc != FH_OK) return rc;
-  if (pl.ntiles > FH_STATIC_MAX_TILES) return FH_ERR_UNSUPPORTED;  // beyond the fixed scratch
+  if (pl.P > FH_STATIC_MAX_PLANES) return FH_ERR_UNSUPPORTED;  // beyond the fixed work list
   cudaStream_t stream = (cudaStream_t)stream_;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FH_ERR_CUDA;
@@ -700,8 +705,9 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
     g_static_ptr[dev] = p;
   }
   unsigned char* base = g_static_ptr[dev];
-  // the array keeps the last call's counters and scan words: clear it (header, tile words, segment words)
-  if (cudaMemsetAsync(base, 0, FH_STATIC_SCRATCH_BYTES, stream) != cudaSuccess) return FH_ERR_CUDA;
+  // the array keeps the last call's contents: the counters and chunk sums must start at zero (the
+  // work list is written before it is read)
+  if (cudaMemsetAsync(base, 0, kHeadBytes, stream) != cudaSuccess) return FH_ERR_CUDA;
   fh::CompressArgs a;
   a.src = (const uint8_t*)d_src;
   a.dst_base = (uint8_t*)d_dst;
@@ -710,12 +716,10 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   a.d_off_out = nullptr;
   a.out2 = (unsigned long long*)d_out2;
   a.sc = reinterpret_cast<fh::Scratch*>(base);
-  a.scan.ts = reinterpret_cast<unsigned long long*>(base + 256);
-  a.scan.seg_cs = a.scan.ts + FH_STATIC_MAX_TILES;
-  a.scan.seg_inc = a.scan.seg_cs + FH_STATIC_MAX_TILES / 32;
-  a.scan.epoch = 1;
-  a.scan.spin_limit = kSpinLimit;
-  a.nseg = (pl.ntiles + 31) / 32;
+  a.chunk_ovf = reinterpret_cast<uint32_t*>(base + 256);
+  a.worklist = reinterpret_cast<uint32_t*>(base + kHeadBytes);
+  chunking(pl.P, &a.chunk_shift, &a.nchunks);
+  std::lock_guard<std::mutex> lock2(g_mu);  // the launch helpers keep their occupancy cache under g_mu
   return launch_compress(pl, v, a, stream);
 }
 
@@ -729,7 +733,7 @@ void fh_shutdown(void) {
     cudaSetDevice(kv.first.first);
     cudaDeviceSynchronize();
     if (kv.second.sc) cudaFree(kv.second.sc);
-    if (kv.second.ts) cudaFree(kv.second.ts);
+    if (kv.second.worklist) cudaFree(kv.second.worklist);
     if (kv.second.sched) cudaFree(kv.second.sched);
   }
   g_scratch.clear();

@@ -1,17 +1,24 @@
-// Compress kernels: one pass over the dense tensor.
+// Compress kernels.
 //
 // Container recap: every plane owns a slot of npay bytes at a closed-form offset; a normal plane's
 // codes fill its slot; the payload of a salient or raw plane runs through its slot and continues in
-// the overflow region, in plane order.  Normal planes therefore never wait for anything: statistics,
-// class, codes and the stores happen in one sweep.  Only tiles that hold salient or raw planes need
-// their place in the overflow region, which a decoupled look-back over per-tile scan words supplies.
+// the overflow region, in plane order.
 //
-// Two kernels share this file:
-//   compress_fast<DT, SIGMA, G, CTA>  planes whose size is a multiple of 16 bytes and that fit the
-//       register budget: tiles stream into shared memory through a multi-stage bulk-copy (TMA)
-//       pipeline, every thread keeps its G groups in registers for all passes;
-//   compress_generic<DT, BITS>        everything else (ragged planes, very large planes): staged with
-//       plain loads, passes re-read shared memory.
+// A call runs up to three kernels on its stream:
+//   1. a streaming kernel (one pass over the dense tensor): per-plane statistics, three-sigma class,
+//      and for normal planes the codes and the table entry.  Normal planes depend on nothing but
+//      themselves, so this kernel has no cross-CTA waits.  A plane that takes the block-wise path only
+//      gets a marker in the table and an entry in a work list.  Three variants by plane size:
+//        compress_warp<DT, SIGMA, TT, FULLVEC>  planes of at most 256 groups: bulk-copy (TMA) pipeline,
+//            a sub-warp team per plane, groups kept in registers;
+//        compress_cta<DT, SIGMA, NT>            larger planes of whole 16-byte chunks: one plane per CTA;
+//        compress_generic<DT, BITS>             everything else (ragged large planes);
+//   2. blockwise_kernel<DT, false> measures every plane of the work list (block classes, CSR and code
+//      sizes), decides salient versus raw, records the sizes;
+//   3. blockwise_kernel<DT, true> derives each listed plane's place in the overflow region from the
+//      recorded sizes (plane order, so the bytes do not depend on scheduling) and writes the payloads;
+//      its last CTA writes the header and the result words.
+// With salient_mode OFF only the first kernel runs and finishes the container itself.
 #pragma once
 
 #include "fh_device.cuh"
@@ -22,6 +29,7 @@ struct SalientInfo {
   uint32_t nnz_s, n_dense, n_out_d, size;
 };
 
+
 struct CompressArgs {
   const uint8_t* src;
   uint8_t* dst_base;
@@ -30,9 +38,11 @@ struct CompressArgs {
   unsigned long long* d_off_out;        // optional: offset for the next container
   unsigned long long* out2;             // optional: {total bytes, status}
   Scratch* sc;
-  ScanState scan;                       // scan words (tiles, segments), epoch, wait bound
-  uint32_t nseg;                        // segments of this call (for the final clean-up)
+  uint32_t* worklist;                   // planes that take the block-wise path, in no particular order
+  uint32_t* chunk_ovf;                  // per chunk of 2^chunk_shift planes: overflow size of its planes (16-byte units)
+  uint32_t chunk_shift, nchunks;
 };
+
 
 // Where the bytes of a salient / raw payload go: offsets below npay land in the plane's slot, the
 // rest in its overflow part.  Offsets and npay are multiples of the access size.
@@ -248,58 +258,10 @@ __device__ __forceinline__ Dest make_dest(const Plan& pl, const CompressArgs& a)
   return d;
 }
 
-// Tile-level placement, executed by warp 0 after the classes and sizes of the tile's planes are in
-// rec[].  Computes each plane's overflow offset (roff[], 16-byte units relative to the tile),
-// publishes the tile's overflow size and, when the tile has overflow parts, resolves the tile's
-// base.  Returns through shared variables: *s_base16 (absolute, 16-byte units), *s_skip.
-__device__ __noinline__ void tile_place(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
-                                           uint32_t np, const Rec* rec, uint32_t* roff,
-                                           unsigned long long* s_base16, uint32_t* s_skip) {
-  const uint32_t lane = threadIdx.x & 31u;
-  uint32_t carry = 0, nsal = 0, nraw = 0;
-  for (uint32_t base = 0; base < np; base += 32) {
-    const uint32_t i = base + lane;
-    uint32_t v = 0, c = 0;
-    if (i < np) {
-      c = rec[i].meta & 3u;
-      if (c != kClsNormal && a16(rec[i].size) > pl.npay) v = (a16(rec[i].size) - pl.npay) >> 4;
-    }
-    uint32_t incl = v;
-    for (uint32_t o = 1; o < 32; o <<= 1) {
-      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-      if (lane >= o) incl += up;
-    }
-    if (i < np) roff[i] = carry + incl - v;
-    carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
-    nsal += __popc(__ballot_sync(0xFFFFFFFFu, c == kClsSalient));
-    nraw += __popc(__ballot_sync(0xFFFFFFFFu, c == kClsRaw));
-  }
-  unsigned long long excl = 0;
-  uint32_t skip = d.fits ? 0u : 1u;
-  if (pl.mode != kModeOff) {
-    if (lane == 0) scan_publish(a.scan, tile, carry);
-    if (carry > 0 && tile > 0) {
-      if (!scan_resolve(a.scan, tile, &a.sc->status, &excl)) {
-        if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-        skip = 1;
-      }
-    }
-    if (lane == 0) {
-      if (carry) atomicAdd(&a.sc->ovf16, (unsigned long long)carry);
-      if (nsal) atomicAdd(&a.sc->nsal, (unsigned long long)nsal);
-      if (nraw) atomicAdd(&a.sc->nraw, (unsigned long long)nraw);
-    }
-  }
-  if (lane == 0) {
-    const unsigned long long base16 = (pl.ovf_off >> 4) + excl;
-    if ((base16 + carry) * 16ull > d.capacity) skip = 1;  // never write past the capacity
-    *s_base16 = base16;
-    *s_skip = skip;
-  }
-}
-
-// Last step of every CTA: count the exit; the last CTA to leave writes the header and the result
-// words and returns the scratch counters to zero for the next call.
+// Last step of every CTA of a kernel: count the exit; the last CTA to leave returns the hand-out
+// counters to zero.  FINAL (the call's last kernel): it also writes the header and the result words
+// and clears everything else the call touched.
+template <bool FINAL>
 __device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, const Dest& d) {
   __threadfence();
   __syncthreads();
@@ -307,8 +269,12 @@ __device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, 
   const unsigned long long prev = atomicAdd(&a.sc->exited, 1ull);
   if (prev != (unsigned long long)gridDim.x - 1ull) return;
   __threadfence();
+  st_relaxed(&a.sc->ticket, 0ull);
+  st_relaxed(&a.sc->exited, 0ull);
+  if (!FINAL) return;
   const unsigned long long ovf16 = ld_relaxed(&a.sc->ovf16);
   const unsigned long long nsal = ld_relaxed(&a.sc->nsal), nraw = ld_relaxed(&a.sc->nraw);
+  const unsigned long long listed = ld_relaxed(&a.sc->wl_count);
   uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
   const unsigned long long total = pl.ovf_off + ovf16 * 16ull;
   if (total > d.capacity && code < kErrCapacity) code = kErrCapacity;
@@ -338,14 +304,13 @@ __device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, 
     a.out2[1] = status_word(code);
   }
   if (a.d_off_out) *a.d_off_out = code == kErrNone ? d.off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
-  if (pl.mode != kModeOff)
-    for (uint32_t k = 0; k < a.nseg; ++k) st_relaxed(a.scan.seg_cs + k, 0ull);  // counters back to zero
-  st_relaxed(&a.sc->ticket, 0ull);
+  if (listed)
+    for (uint32_t k = 0; k < a.nchunks; ++k) a.chunk_ovf[k] = 0u;
   st_relaxed(&a.sc->status, 0ull);
   st_relaxed(&a.sc->ovf16, 0ull);
   st_relaxed(&a.sc->nsal, 0ull);
   st_relaxed(&a.sc->nraw, 0ull);
-  st_relaxed(&a.sc->exited, 0ull);
+  st_relaxed(&a.sc->wl_count, 0ull);
 }
 
 __device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane, uint32_t off16, const Rec& r) {
@@ -357,44 +322,39 @@ __device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane,
   reinterpret_cast<uint4*>(d.dst + 64)[plane] = e;
 }
 
-// Writes a salient or raw plane whose record and overflow offset (absolute, 16-byte units) are known.
-template <int DT>
-__device__ __forceinline__ void write_nonnormal(const Team& t, const Plan& pl, const Dest& d, const uint8_t* plane,
-                                                uint64_t gp, const Rec& r, unsigned long long off16, uint32_t* sal) {
-  SplitOut out;
-  out.slot = d.dst + pl.slots_off + gp * pl.npay;
-  out.ovf = d.dst + off16 * 16ull;
-  out.npay = pl.npay;
-  const bool has_ovf = a16(r.size) > pl.npay;
-  if ((r.meta & 3u) == kClsRaw) {
-    raw_write(t, pl, plane, out);
-  } else {
-    const SalientInfo info = salient_measure<DT>(t, pl, plane, sal);
-    salient_write<DT>(t, pl, plane, info, sal, out);
-  }
-  if (t.lane == 0) store_table_entry(d, gp, has_ovf ? (uint32_t)off16 : 0u, r);
+
+// Table marker of a plane that takes the block-wise path: class salient, the three-sigma count, no
+// offset yet.  The block-wise kernels complete the entry.
+__device__ __forceinline__ void store_marker(const Dest& d, uint64_t plane, uint32_t meta) {
+  reinterpret_cast<uint4*>(d.dst + 64)[plane] = make_uint4(0u, (meta & ~3u) | kClsSalient, 0u, 0u);
+}
+
+// Appends plane `gp` to the work list of the block-wise kernels (one thread).
+__device__ __forceinline__ void list_plane(const CompressArgs& a, uint64_t gp) {
+  const unsigned long long at = atomicAdd(&a.sc->wl_count, 1ull);
+  a.worklist[at] = (uint32_t)gp;
 }
 
 // =================================================================================================
-// Generic kernel
+// Generic streaming kernel
 // =================================================================================================
+// Tiles of consecutive planes are staged in shared memory with plain loads (planes need not start
+// on a 16-byte boundary); a team per plane computes statistics and class; the codes of normal planes
+// are staged in shared memory and leave with 16-byte stores.
 template <int DT, int BITS>
 __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
-  __shared__ uint32_t s_tile, s_skip;
-  __shared__ unsigned long long s_base16;
+  __shared__ uint32_t s_tile;
 
   const uint32_t tid = threadIdx.x;
   uint8_t* tile_buf = smem + pl.sm_tile;
   uint8_t* out_buf = smem + pl.sm_out;
   Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
-  uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + 16u * pl.ppt);
   const Dest d = make_dest(pl, a);
   const Team team = make_team(pl.team, s_red);
   const uint32_t nteams = team.block ? 1u : kThreads / team.size;
   const uint32_t my_team = team.block ? 0u : tid / team.size;
-  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)my_team * pl.sm_sal_stride);
   constexpr uint32_t L = (1u << BITS) - 1u;
   const bool need_sigma = pl.mode == kModeAuto;
   uint32_t rp = 0;  // reduction counter (see red_half)
@@ -422,7 +382,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     }
     __syncthreads();
 
-    // ---- phase A: per-plane statistics, class, codes / sizes
+    // ---- phase A: per-plane statistics, class, codes
     for (uint32_t lp = my_team; lp < np; lp += nteams) {
       const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
       const bool vec = (smem_u32(plane) & (DT == kF32 ? 15u : 7u)) == 0u;
@@ -481,14 +441,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
       r.lo = 0.0f;
       r.scale = 0.0f;
       r.size = 0;
-      if (cls == kClsSalient) {
-        const SalientInfo info = salient_measure<DT>(team, pl, plane, sal);
-        r.size = info.size;
-        if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
-          cls = kClsRaw;
-          r.size = (uint32_t)pl.plane_bytes;
-        }
-      } else {
+      if (cls == kClsNormal) {
         float inv, scale;
         quant_params(lo, hi, L, inv, scale);
         r.lo = lo;
@@ -517,31 +470,27 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     }
     __syncthreads();
 
-    // ---- phase B: placement of the overflow parts
-    if (tid < 32) tile_place(pl, a, d, tile, np, rec, roff, &s_base16, &s_skip);
-    __syncthreads();
-
-    // ---- phase C: table entries and payloads
-    if (!s_skip) {
-      const unsigned long long base16 = s_base16;
+    // ---- phase B: table entries and slots of the normal planes; markers and work-list entries of the others
+    if (d.fits) {
       const uint32_t chunks = pl.npay >> 4;
       uint4* slots = reinterpret_cast<uint4*>(d.dst + pl.slots_off + p0 * pl.npay);
       for (uint32_t i = tid; i < np * chunks; i += kThreads) {
         const uint32_t lp = i / chunks;
         if ((rec[lp].meta & 3u) == kClsNormal) slots[i] = reinterpret_cast<const uint4*>(out_buf)[i];
       }
-      for (uint32_t i = tid; i < np; i += kThreads)
-        if ((rec[i].meta & 3u) == kClsNormal)
-          store_table_entry(d, p0 + i, (uint32_t)((pl.slots_off + (p0 + i) * pl.npay) >> 4), rec[i]);
-      for (uint32_t lp = my_team; lp < np; lp += nteams) {
-        if ((rec[lp].meta & 3u) == kClsNormal) continue;
-        const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
-        write_nonnormal<DT>(team, pl, d, plane, p0 + lp, rec[lp], base16 + roff[lp], sal);
+    }
+    for (uint32_t i = tid; i < np; i += kThreads) {
+      if ((rec[i].meta & 3u) == kClsNormal) {
+        if (d.fits) store_table_entry(d, p0 + i, (uint32_t)((pl.slots_off + (p0 + i) * pl.npay) >> 4), rec[i]);
+      } else {
+        if (d.fits) store_marker(d, p0 + i, rec[i].meta);
+        list_plane(a, p0 + i);
       }
     }
     __syncthreads();
   }
-  cta_exit(pl, a, d);
+  if (pl.mode == kModeOff) cta_exit<true>(pl, a, d);
+  else cta_exit<false>(pl, a, d);
 }
 
 // =================================================================================================
@@ -716,107 +665,46 @@ __device__ __forceinline__ void plane_sweep_any(const Team& team, const Plan& pl
 }
 
 // -------------------------------------------------------------------------------------------------
-// Warp-team kernel: planes of at most 256 groups.  Eight consumer warps and one producer warp per
-// CTA.  The producer hands out tiles and streams them into a ring of shared-memory stages with bulk
-// copies.  The consumer warps never wait for each other on the common path: each sweeps its own
-// planes of a tile (statistics, class, codes, stores) and arrives on the stage's barriers.  When a
-// stage comes back, the producer publishes the tile's (zero) scan word.  Only warps that hold
-// salient or raw planes take the slow path: they wait until the whole tile is classified, one of
-// them places the tile's overflow parts, and they write their planes.
+// Warp-team streaming kernel: planes of at most 256 groups.  Eight consumer warps and one producer
+// warp per CTA.  The producer hands out tiles and streams them into a ring of shared-memory stages
+// with bulk copies.  The consumer warps never wait for each other: each sweeps its own planes of a
+// tile (statistics, class, codes, stores), lists the planes that take the block-wise path, and
+// arrives on the stage's barrier.
 // -------------------------------------------------------------------------------------------------
 constexpr int kWarpKernelThreads = kThreads + 32;
-
-// Placement of a tile with salient / raw planes, executed by one warp.  ovf16[i] holds the overflow
-// size of plane i of the tile in 16-byte units (0 for normal planes); the
-// sizes are left alone; poff[i] receives the plane's offset relative to the tile's base.
-__device__ __noinline__ void tile_place_sparse(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t tile,
-                                               uint32_t np, const uint32_t* ovf16, uint32_t* poff,
-                                               unsigned long long* s_base16, uint32_t* s_skip) {
-  const uint32_t lane = threadIdx.x & 31u;
-  uint32_t carry = 0;
-  for (uint32_t base = 0; base < np; base += 32) {
-    const uint32_t i = base + lane;
-    const uint32_t v = i < np ? ovf16[i] : 0u;
-    uint32_t incl = v;
-    for (uint32_t o = 1; o < 32; o <<= 1) {
-      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-      if (lane >= o) incl += up;
-    }
-    if (i < np) poff[i] = carry + incl - v;
-    carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
-  }
-  unsigned long long excl = 0;
-  uint32_t skip = d.fits ? 0u : 1u;
-  if (lane == 0) scan_publish(a.scan, tile, carry);
-  if (carry > 0 && tile > 0) {
-    if (!scan_resolve(a.scan, tile, &a.sc->status, &excl)) {
-      if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-      skip = 1;
-    }
-  }
-  if (lane == 0) {
-    if (carry) atomicAdd(&a.sc->ovf16, (unsigned long long)carry);
-    const unsigned long long base16 = (pl.ovf_off >> 4) + excl;
-    if ((base16 + carry) * 16ull > d.capacity) skip = 1;  // never write past the capacity
-    *s_base16 = base16;
-    *s_skip = skip;
-  }
-}
 
 template <int DT, bool SIGMA, int TT, bool FULLVEC>
 __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
-  __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages], s_classified[kMaxStages];
-  __shared__ uint32_t s_tiles[kMaxStages], s_nn[kMaxStages], s_nnmask[kMaxStages], s_skip[kMaxStages];
-  __shared__ volatile uint32_t s_placed[kMaxStages];  // tile + 1 once the tile's overflow parts are placed
-  __shared__ unsigned long long s_base16[kMaxStages];
+  __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
+  __shared__ uint32_t s_tiles[kMaxStages];
   __shared__ volatile uint32_t s_abort;
-  __shared__ Plan s_pl;          // copies for the outlined slow path (salient planes, placement):
-  __shared__ CompressArgs s_a;   // its functions take them by address
 
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const Dest d = make_dest(pl, a);
   const uint32_t nstage = pl.nstage;
-  uint32_t* ovf16_all = reinterpret_cast<uint32_t*>(smem + pl.sm_rec);  // nstage x ppt words, zero when idle
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
   if (tid == 0) {
-    s_pl = pl;
-    s_a = a;
     for (uint32_t s = 0; s < nstage; ++s) {
       mbar_init(&s_full[s], 1);
       mbar_init(&s_empty[s], kWarps);
-      mbar_init(&s_classified[s], kWarps);
-      s_nn[s] = 0;
-      s_nnmask[s] = 0;
-      s_placed[s] = 0;
     }
     fence_mbar_init();
     s_abort = 0;
   }
-  for (uint32_t i = tid; i < nstage * pl.ppt; i += kWarpKernelThreads) ovf16_all[i] = 0;
   __syncthreads();
 
   if (warp == (uint32_t)kWarps) {
     // ======================= producer (all 32 lanes walk the loop, lane 0 issues) =======================
     uint32_t s = 0, empty_phase = 0;
     bool aborted = false;
-    // Drains stage q: waits until every consumer warp is done with its tile, then gives a tile without
-    // salient planes its scan word (tiles with salient planes were published by their consumers).
+    // Waits until every consumer warp is done with the tile in stage q.
     auto drain = [&](uint32_t q) -> bool {
       bool ok = mbar_wait_abortable(&s_empty[q], (empty_phase >> q) & 1u, 1u << 20, &s_abort);
       ok = __all_sync(0xFFFFFFFFu, ok);
-      if (!ok) return false;
-      empty_phase ^= 1u << q;
-      if (pl.mode != kModeOff) {
-        if (lane == 0) {
-          if (*reinterpret_cast<volatile uint32_t*>(&s_nn[q]) == 0) scan_publish(a.scan, s_tiles[q], 0u);
-          s_nn[q] = 0;
-          s_nnmask[q] = 0;
-        }
-        __syncwarp();
-      }
-      return true;
+      if (ok) empty_phase ^= 1u << q;
+      return ok;
     };
     for (uint32_t n = 0;; ++n) {
       if (n >= nstage && !drain(s)) {
@@ -827,7 +715,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       if (lane == 0) t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
       t = __shfl_sync(0xFFFFFFFFu, t, 0);
       if (t >= pl.ntiles) {
-        // no more tiles: wake the consumers at this stage, then drain the tiles still in the ring
+        // no more tiles: wake the consumers at this stage, then wait for the tiles still in the ring
         const uint32_t first = n >= nstage ? n - nstage + 1u : 0u;
         uint32_t q = first % nstage;
         __syncwarp();
@@ -899,117 +787,26 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       Rec r;
       r.meta = kClsNormal;
       if (active) plane_sweep_any<DT, SIGMA, G, TT, FULLVEC>(team, pl, d, a, plane, (uint64_t)p0 + lp, vec, rp, r);
-      const bool mine_nn = active && (r.meta & 3u) != kClsNormal;
-      if (!__any_sync(0xFFFFFFFFu, mine_nn)) {
-        // ---- common path: this warp is done with the tile
-        if (lane == 0) {
-          mbar_arrive(&s_classified[s]);
-          mbar_arrive(&s_empty[s]);
+      // planes that take the block-wise path: marker in the table, entry in the work list
+      const bool mine = active && (r.meta & 3u) != kClsNormal && team.lane == 0;
+      const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine);
+      if (leaders) {
+        uint32_t base = 0;
+        if (lane == 0) base = (uint32_t)atomicAdd(&a.sc->wl_count, (unsigned long long)__popc(leaders));
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if (mine) {
+          a.worklist[base + __popc(leaders & ((1u << lane) - 1u))] = p0 + lp;
+          if (d.fits) store_marker(d, (uint64_t)p0 + lp, r.meta);
         }
-      } else {
-        // ---- slow path: salient / raw planes in this warp.  Each of them is handled by all 32 lanes.
-        const Team wteam = make_warp_team(s_red);
-        uint32_t* ovf16 = ovf16_all + s * pl.ppt;
-        uint32_t* poff = ovf16_all + nstage * pl.ppt + s * pl.ppt;  // offsets inside the tile, from the placement
-        uint32_t* sinfo = ovf16_all + 2u * nstage * pl.ppt + (s * pl.ppt) * 4u;  // per plane: size, nnz_s, n_dense, n_out_d
-        const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine_nn && team.lane == 0);
-        const uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
-        uint32_t raw_mask = 0;  // bit L: the plane led by lane L turned out raw
-        for (uint32_t m = leaders; m; m &= m - 1u) {
-          const uint32_t L = (uint32_t)__ffs(m) - 1u, tlp = (warp * 32u + L) / TT;
-          const uint8_t* tplane = stage + (uint64_t)tlp * pl.plane_bytes;
-          uint32_t* tsal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + (uint64_t)tlp * pl.sm_sal_stride);
-          const SalientInfo info = salient_measure<DT>(wteam, s_pl, tplane, tsal);
-          uint32_t size = info.size;
-          const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
-          if (raw) {
-            size = (uint32_t)pl.plane_bytes;
-            raw_mask |= 1u << L;
-          }
-          if (lane == 0) {
-            ovf16[tlp] = a16(size) > pl.npay ? (a16(size) - pl.npay) >> 4 : 0u;
-            sinfo[tlp * 4u + 0] = size;
-            sinfo[tlp * 4u + 1] = info.nnz_s;
-            sinfo[tlp * 4u + 2] = info.n_dense;
-            sinfo[tlp * 4u + 3] = info.n_out_d;
-            atomicAdd(raw ? &a.sc->nraw : &a.sc->nsal, 1ull);
-          }
-        }
-        __syncwarp();
-        if (lane == 0) {
-          atomicAdd(&s_nn[s], 1u);
-          atomicOr(&s_nnmask[s], 1u << warp);
-          __threadfence_block();
-          mbar_arrive(&s_classified[s]);
-        }
-        bool done = mbar_wait_abortable(&s_classified[s], par, 1u << 20, &s_abort);  // the whole tile is classified
-        done = __all_sync(0xFFFFFFFFu, done);
-        if (done) {
-          __threadfence_block();
-          const uint32_t mask = *reinterpret_cast<volatile uint32_t*>(&s_nnmask[s]);
-          if ((uint32_t)__ffs(mask) - 1u == warp) {  // the first such warp places the tile
-            tile_place_sparse(s_pl, s_a, d, tile, np, ovf16, poff, &s_base16[s], &s_skip[s]);
-            __threadfence_block();
-            __syncwarp();
-            if (lane == 0) s_placed[s] = tile + 1u;
-          }
-          done = false;
-          for (uint32_t i = 0; i < (1u << 22); ++i) {
-            if (s_placed[s] == tile + 1u) {
-              done = true;
-              break;
-            }
-            if (s_abort) break;
-            __nanosleep(64);
-          }
-          done = __all_sync(0xFFFFFFFFu, done);
-        }
-        if (!done) {
-          s_abort = 1;
-          if (lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-        } else {
-          __threadfence_block();
-          const bool skip = s_skip[s] != 0;
-          for (uint32_t m = leaders; m; m &= m - 1u) {
-            const uint32_t L = (uint32_t)__ffs(m) - 1u, tlp = (warp * 32u + L) / TT;
-            const uint32_t meta_n = __shfl_sync(0xFFFFFFFFu, r.meta, L);  // the plane's three-sigma count
-            if (!skip) {
-              const uint8_t* tplane = stage + (uint64_t)tlp * pl.plane_bytes;
-              const uint32_t* tsal = reinterpret_cast<const uint32_t*>(smem + pl.sm_sal + (uint64_t)tlp * pl.sm_sal_stride);
-              const unsigned long long off16 = s_base16[s] + poff[tlp];
-              SalientInfo info;
-              info.size = sinfo[tlp * 4u + 0];
-              info.nnz_s = sinfo[tlp * 4u + 1];
-              info.n_dense = sinfo[tlp * 4u + 2];
-              info.n_out_d = sinfo[tlp * 4u + 3];
-              const bool raw = (raw_mask >> L) & 1u;
-              SplitOut out;
-              out.slot = d.dst + pl.slots_off + ((uint64_t)p0 + tlp) * pl.npay;
-              out.ovf = d.dst + off16 * 16ull;
-              out.npay = pl.npay;
-              if (raw) raw_write(wteam, s_pl, tplane, out);
-              else salient_write<DT>(wteam, s_pl, tplane, info, tsal, out);
-              if (lane == 0) {
-                Rec tr;
-                tr.lo = 0.0f;
-                tr.scale = 0.0f;
-                tr.size = info.size;
-                tr.meta = (meta_n & ~3u) | (raw ? kClsRaw : kClsSalient);
-                store_table_entry(d, (uint64_t)p0 + tlp, a16(info.size) > pl.npay ? (uint32_t)off16 : 0u, tr);
-              }
-            }
-            __syncwarp();
-            if (lane == 0) ovf16[tlp] = 0;  // leave the array clean for the stage's next tile
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_empty[s]);
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[s]);
       if (s_abort) break;
       s = s + 1 == nstage ? 0 : s + 1;
     }
   }
-  cta_exit(pl, a, d);
+  if (pl.mode == kModeOff) cta_exit<true>(pl, a, d);
+  else cta_exit<false>(pl, a, d);
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -1058,25 +855,14 @@ __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, floa
 
 template <int DT, bool SIGMA, int NT>
 __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const CompressArgs a) {
-  constexpr int NW = NT / 32;
   constexpr bool COUNT = SIGMA;
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
-  __shared__ uint32_t s_skip, s_abort;
-  __shared__ unsigned long long s_base16;
-  __shared__ Plan s_pl;          // copies for the outlined slow path
-  __shared__ CompressArgs s_a;
+  __shared__ uint32_t s_abort;
 
-  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  if (tid == 0) {
-    s_pl = pl;
-    s_a = a;
-  }
-  Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
-  uint32_t* roff = reinterpret_cast<uint32_t*>(smem + pl.sm_rec + 16u);
-  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal);
+  const uint32_t tid = threadIdx.x;
   const Dest d = make_dest(pl, a);
   const Team team = make_team(NT, s_red);
   const uint32_t nstage = pl.nstage, groups = pl.groups, bits = (uint32_t)pl.bits;
@@ -1162,7 +948,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     }
 
     // ---- sweep 3: codes into the plane's slot (and the outlier count).  A plane that turns out
-    // salient has its slot rewritten by the slow path below.
+    // salient has its slot rewritten by the block-wise kernels.
     float inv, scale;
     quant_params(lo, hi, (1u << bits) - 1u, inv, scale);
     uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
@@ -1189,50 +975,26 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     }
     uint32_t cls = kClsNormal, n_out = 0;
     if (SIGMA) {
-      n_out = team_sum_u32(team, c0 + c1, rp);
+      n_out = team_sum_u32(team, c0 + c1, rp);  // its barrier: every thread is done with the stage
       if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
     } else {
       if (pl.mode == kModeAll) cls = kClsSalient;
       __syncthreads();  // every thread is done with the stage
     }
-
-    Rec r;
-    r.lo = 0.0f;
-    r.scale = 0.0f;
-    r.size = 0;
-    r.meta = cls | (n_out << 2);
-    if (cls == kClsNormal) {
-      r.lo = lo;
-      r.scale = scale;
-      if (tid == 0) {
+    if (tid == 0) {
+      Rec r;
+      r.size = 0;
+      r.meta = cls | (n_out << 2);
+      if (cls == kClsNormal) {
+        r.lo = lo;
+        r.scale = scale;
         if (d.fits) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
-        if (pl.mode != kModeOff) scan_publish(a.scan, tile, 0u);
+      } else {
+        if (d.fits) store_marker(d, gp, r.meta);
+        list_plane(a, gp);
       }
-    } else {
-      // ---- slow path: the block-wise encoding of a salient plane, by the whole CTA
-      const SalientInfo info = salient_measure<DT>(team, s_pl, plane, sal);
-      r.size = info.size;
-      if (a16(info.size) >= a16((uint32_t)pl.plane_bytes)) {
-        r.meta = (r.meta & ~3u) | kClsRaw;
-        r.size = (uint32_t)pl.plane_bytes;
-      }
-      if (tid == 0) rec[0] = r;
-      __syncthreads();
-      if (warp == 0) tile_place(s_pl, s_a, d, tile, 1u, rec, roff, &s_base16, &s_skip);
-      __syncthreads();
-      if (!s_skip) {
-        SplitOut out;
-        out.slot = slot;
-        out.ovf = d.dst + (s_base16 + roff[0]) * 16ull;
-        out.npay = pl.npay;
-        if ((r.meta & 3u) == kClsRaw) raw_write(team, s_pl, plane, out);
-        else salient_write<DT>(team, s_pl, plane, info, sal, out);
-        if (tid == 0) store_table_entry(d, gp, a16(r.size) > pl.npay ? (uint32_t)(s_base16 + roff[0]) : 0u, r);
-      }
-      __syncthreads();
+      issue(s);  // the stage is free: next load
     }
-    // ---- the stage is free: next load (thread 0), next stage
-    if (tid == 0) issue(s);
     s = s + 1 == nstage ? 0 : s + 1;
     // s_tiles[s] for the next iteration was written at least one barrier ago (nstage >= 2)
   }
@@ -1245,7 +1007,150 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
         mbar_wait(&s_full[k], 1u, 1u << 10);
       }
   }
-  cta_exit(pl, a, d);
+  if (pl.mode == kModeOff) cta_exit<true>(pl, a, d);
+  else cta_exit<false>(pl, a, d);
+}
+
+// =================================================================================================
+// Block-wise kernels: the planes of the work list
+// =================================================================================================
+// A unit -- one warp for planes up to 8 KB, the whole CTA above -- takes entries i = unit, unit +
+// units, ... of the work list, copies the plane into its shared-memory buffer and runs the
+// measuring part of the block-wise path on it.
+//
+// WRITE = false (measuring kernel): the unit decides salient versus raw, completes the plane's table
+// entry (class; the offset stays 0), leaves the three counts of a salient payload in the first
+// 16 bytes of the plane's slot, and adds the plane's overflow size to the sum of its chunk (a chunk
+// is a run of 2^chunk_shift consecutive planes; there are at most kMaxChunks chunks).
+//
+// WRITE = true (writing kernel): every CTA first turns the chunk sums into chunk offsets.  A plane's
+// place in the overflow region is its chunk's offset plus the overflow sizes of the listed planes
+// before it in the same chunk, which the unit recomputes from their table classes and slot headers
+// (nothing else writes those words while this kernel runs, and every writer stores the value that
+// is already there).  The payload is written and the table offset filled in.  The last CTA to leave
+// writes the header and the result words.
+__device__ __forceinline__ uint32_t salient_size(const Plan& pl, uint32_t nnz_s, uint32_t n_dense, uint32_t n_out_d) {
+  const uint32_t e = (uint32_t)pl.esize;
+  return 16u + 4u * pl.nbm + 4u * ((uint32_t)pl.H + 1u) + a4(2u * nnz_s) + a4(e * nnz_s) + 64u * n_dense +
+         a4(e * n_out_d);
+}
+// Overflow size, in 16-byte units, of a payload of `size` bytes.
+__device__ __forceinline__ uint32_t ovf_units(const Plan& pl, uint32_t size) {
+  return a16(size) > pl.npay ? (a16(size) - pl.npay) >> 4 : 0u;
+}
+
+template <int DT, bool WRITE>
+__global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const CompressArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ double s_red[kMaxWarps * 5];
+  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
+
+  const uint32_t tid = threadIdx.x, lane32 = tid & 31u, warp = tid >> 5;
+  const Dest d = make_dest(pl, a);
+  const uint32_t count = (uint32_t)ld_relaxed(&a.sc->wl_count);
+  if (tid == 0) s_pl = pl;
+  const bool unit_cta = pl.sk_cta != 0u;
+  const uint32_t upc = unit_cta ? 1u : blockDim.x >> 5;
+  const uint32_t unit = unit_cta ? blockIdx.x : blockIdx.x * upc + warp;
+  const uint32_t units = gridDim.x * upc;
+  const Team t = unit_cta ? make_team(blockDim.x, s_red) : make_warp_team(s_red);
+  uint8_t* ubuf = smem + (unit_cta ? 0u : warp * pl.sk_unit_stride);
+  uint32_t* sal = reinterpret_cast<uint32_t*>(ubuf + pl.sk_sal_off);
+  uint32_t* pre = reinterpret_cast<uint32_t*>(smem + pl.sk_pre_off);
+  const uint4* table = reinterpret_cast<const uint4*>(d.dst + 64);
+  const uint32_t raw_units = ovf_units(pl, (uint32_t)pl.plane_bytes);
+
+  if (WRITE && count > 0 && d.fits) {
+    // chunk offsets: exclusive prefix sum of the chunk sums (warp 0: 32 consecutive chunks per lane)
+    for (uint32_t k = tid; k < kMaxChunks; k += blockDim.x) pre[k] = k < a.nchunks ? a.chunk_ovf[k] : 0u;
+    __syncthreads();
+    if (warp == 0) {
+      constexpr uint32_t per = kMaxChunks / 32;
+      uint32_t local = 0;
+      for (uint32_t k = 0; k < per; ++k) local += pre[lane32 * per + k];
+      uint32_t incl = local;
+      for (uint32_t o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane32 >= o) incl += up;
+      }
+      uint32_t run = incl - local;
+      for (uint32_t k = 0; k < per; ++k) {
+        const uint32_t v = pre[lane32 * per + k];
+        pre[lane32 * per + k] = run;
+        run += v;
+      }
+    }
+  }
+  __syncthreads();
+
+  if (WRITE ? d.fits : true) {
+    for (uint32_t i = unit; i < count; i += units) {
+      const uint32_t p = a.worklist[i];
+      // ---- copy the plane: whole 16-byte chunks from the aligned start, the ragged end of the tensor byte-wise
+      const uint64_t start = (uint64_t)p * pl.plane_bytes, end = start + pl.plane_bytes;
+      const uint64_t a0 = start & ~15ull;
+      const uint32_t head = (uint32_t)(start - a0);
+      const uint64_t a1 = min((end + 15ull) & ~15ull, pl.dense_bytes & ~15ull);
+      {
+        const uint4* s16 = reinterpret_cast<const uint4*>(a.src + a0);
+        uint4* t16 = reinterpret_cast<uint4*>(ubuf);
+        const uint32_t n16 = (uint32_t)((a1 - a0) >> 4);
+        for (uint32_t k = t.lane; k < n16; k += t.size) t16[k] = __ldg(s16 + k);
+        for (uint64_t k = a1 + t.lane; k < end; k += t.size) ubuf[k - a0] = a.src[k];
+      }
+      team_sync(t);
+      const uint8_t* plane = ubuf + head;
+      const SalientInfo info = salient_measure<DT>(t, s_pl, plane, sal);
+      const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
+      const uint32_t size = raw ? (uint32_t)pl.plane_bytes : info.size;
+      const uint32_t my_units = ovf_units(pl, size);
+      uint8_t* slot = d.dst + pl.slots_off + (uint64_t)p * pl.npay;
+      if (!WRITE) {
+        if (t.lane == 0) {
+          if (d.fits) {
+            const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(table + p) + 1);  // the streaming kernel's marker
+            reinterpret_cast<uint4*>(d.dst + 64)[p] = make_uint4(0u, (meta & ~3u) | (raw ? kClsRaw : kClsSalient), 0u, 0u);
+            if (!raw) *reinterpret_cast<uint4*>(slot) = make_uint4(info.nnz_s, info.n_dense, info.n_out_d, 0u);
+          }
+          if (my_units) {
+            atomicAdd(&a.chunk_ovf[p >> a.chunk_shift], my_units);
+            atomicAdd(&a.sc->ovf16, (unsigned long long)my_units);
+          }
+          atomicAdd(raw ? &a.sc->nraw : &a.sc->nsal, 1ull);
+        }
+      } else {
+        // ---- overflow units of the listed planes before p in its chunk (every warp of the unit computes them)
+        uint32_t before = 0;
+        for (uint32_t q0 = (p >> a.chunk_shift) << a.chunk_shift; q0 < p; q0 += 32u) {
+          const uint32_t q = q0 + lane32;
+          uint32_t v = 0;
+          if (q < p) {
+            const uint32_t cls = __ldcg(reinterpret_cast<const uint32_t*>(table + q) + 1) & 3u;
+            if (cls == kClsRaw) {
+              v = raw_units;
+            } else if (cls == kClsSalient) {
+              const uint4 h = __ldcg(reinterpret_cast<const uint4*>(d.dst + pl.slots_off + (uint64_t)q * pl.npay));
+              v = ovf_units(pl, salient_size(pl, h.x, h.y, h.z));
+            }
+          }
+          asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(v) : "r"(0xFFFFFFFFu));
+          before += v;
+        }
+        const unsigned long long off16 = (pl.ovf_off >> 4) + pre[p >> a.chunk_shift] + before;
+        if ((off16 + my_units) * 16ull <= d.capacity) {  // never write past the capacity
+          SplitOut out;
+          out.slot = slot;
+          out.ovf = d.dst + off16 * 16ull;
+          out.npay = pl.npay;
+          if (raw) raw_write(t, s_pl, plane, out);
+          else salient_write<DT>(t, s_pl, plane, info, sal, out);
+          if (t.lane == 0) *reinterpret_cast<uint32_t*>(d.dst + 64 + 16ull * p) = my_units ? (uint32_t)off16 : 0u;
+        }
+      }
+      team_sync(t);  // the buffer is reused by the next entry
+    }
+  }
+  if (WRITE) cta_exit<true>(pl, a, d);
 }
 
 }  // namespace fh

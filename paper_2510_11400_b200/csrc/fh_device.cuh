@@ -50,26 +50,31 @@ struct Plan {
   uint32_t nstage;       // fast kernels: tiles in flight per CTA
   uint32_t stage_bytes;  // fast kernels: bytes of one stage buffer (ppt * plane_bytes)
   // shared-memory layout (byte offsets into dynamic shared memory)
-  uint32_t sm_tile, sm_out, sm_rec, sm_sal, sm_sal_stride, sm_total;
+  uint32_t sm_tile, sm_out, sm_rec, sm_total;
+  // block-wise kernels: a unit (one warp, or the whole CTA for large planes) holds one plane
+  uint32_t sk_cta;          // 1: the unit is the CTA
+  uint32_t sk_threads;      // CTA size
+  uint32_t sk_sal_off;      // offset of the unit's measuring scratch behind its plane buffer
+  uint32_t sk_unit_stride;  // bytes of shared memory per unit
+  uint32_t sk_pre_off;      // offset of the chunk prefix array (kMaxChunks words)
+  uint32_t sk_total;
+  uint32_t sal_words;       // words of measuring scratch per plane: H + 1 + 3 * nblk
 };
 
-// Book-keeping scratch, one per stream: a header of counters followed by one 64-bit scan word per
-// tile.  The scan words carry the call's epoch so that they need no clearing between calls; the
-// counters are returned to zero by the last CTA to leave a kernel.
+// Book-keeping scratch, one per stream: a header of counters, kMaxChunks chunk sums (see the
+// block-wise kernels) and the work list of planes that take the block-wise path.  Everything a call
+// changes is returned to zero by the last CTA of its last kernel.
 struct Scratch {
-  unsigned long long ticket;  // next tile
-  unsigned long long exited;  // CTAs that have left
-  unsigned long long status;  // device error code (atomicMax)
-  unsigned long long ovf16;   // overflow region size of this call, in 16-byte units
+  unsigned long long ticket;    // next tile
+  unsigned long long exited;    // CTAs that have left the running kernel
+  unsigned long long status;    // device error code (atomicMax)
+  unsigned long long ovf16;     // overflow region size of this call, in 16-byte units
   unsigned long long nsal, nraw;
-  unsigned long long pad[2];
+  unsigned long long wl_count;  // entries of the work list
+  unsigned long long pad;
 };
 static_assert(sizeof(Scratch) == 64, "Scratch layout");
-
-// scan word of a tile: epoch (30 bits) | flag (2 bits: 1 = tile aggregate, 2 = inclusive prefix) | value
-__device__ __forceinline__ unsigned long long scan_word(uint32_t epoch, uint32_t flag, uint32_t value) {
-  return ((unsigned long long)epoch << 34) | ((unsigned long long)flag << 32) | value;
-}
+constexpr uint32_t kMaxChunks = 1024;
 
 // (uint64)(int64) fh_status of a device error code.
 __device__ __forceinline__ unsigned long long status_word(uint32_t code) {
@@ -469,84 +474,6 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
   }
   team_sync(t);
   return total;
-}
-
-// ------------------------------------------------------------------------------------------------
-// Plane-ordered placement of the overflow parts.
-//
-// Every tile publishes the size of its overflow parts (zero for a tile of normal planes): a word of
-// its own, tagged with the call's epoch, and a fire-and-forget atomic add of (1 << 32 | size) to the
-// counter word of its segment of 32 tiles.  Only tiles that hold salient or raw planes need their
-// offset: such a tile waits until the earlier tiles of its own segment have published and until the
-// earlier segments are complete (count 32), sums them, and leaves the prefix up to its segment in
-// seg_inc so that later walks stop there.  Tensors without salient planes never wait at all.
-// Waits are bounded; on expiry the call reports kErrTimeout.  The counter words are returned to zero
-// by the last CTA of the kernel; tile and seg_inc words carry the epoch and need no clearing.
-// ------------------------------------------------------------------------------------------------
-struct ScanState {
-  unsigned long long* ts;       // one word per tile
-  unsigned long long* seg_cs;   // per segment: published tiles << 32 | sum of their sizes
-  unsigned long long* seg_inc;  // per segment: epoch-tagged prefix through the end of the segment
-  uint32_t epoch, spin_limit;
-};
-
-// One thread publishes a tile's overflow size (16-byte units).
-__device__ __forceinline__ void scan_publish(const ScanState& sc, uint32_t tile, uint32_t value) {
-  st_relaxed(sc.ts + tile, scan_word(sc.epoch, 1u, value));
-  const unsigned long long add = (1ull << 32) | value;
-  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(sc.seg_cs + (tile >> 5)), "l"(add) : "memory");
-}
-
-// All 32 lanes of a warp: sum of the sizes of tiles [0, tile).  Returns false on timeout.
-__device__ __noinline__ bool scan_resolve(const ScanState& sc, uint32_t tile, const unsigned long long* status,
-                                          unsigned long long* excl) {
-  const uint32_t lane = threadIdx.x & 31u, seg = tile >> 5;
-  unsigned long long sum = 0;
-  uint32_t spins = 0;
-  // earlier tiles of the own segment
-  for (;;) {
-    const uint32_t idx = seg * 32u + lane;
-    const bool need = idx < tile;
-    const unsigned long long w = need ? ld_acquire(sc.ts + idx) : 0ull;
-    const bool valid = !need || (uint32_t)(w >> 34) == sc.epoch;
-    if (__all_sync(0xFFFFFFFFu, valid)) {
-      uint32_t c = need ? (uint32_t)w : 0u;
-      asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(c) : "r"(0xFFFFFFFFu));
-      sum = c;
-      break;
-    }
-    ++spins;
-    if (spins > sc.spin_limit || ((spins & 63u) == 0 && ld_relaxed(status) == kErrTimeout)) return false;
-    __nanosleep(40);
-  }
-  const unsigned long long own = sum;
-  // earlier segments, 32 at a time, back to the nearest published prefix
-  long long k = (long long)seg - 1;
-  while (k >= 0) {
-    const long long j = k - (long long)lane;
-    const unsigned long long inc = j >= 0 ? ld_acquire(sc.seg_inc + j) : 0ull;
-    const unsigned long long cs = j >= 0 ? ld_acquire(sc.seg_cs + j) : 0ull;
-    const bool has_inc = j < 0 || (uint32_t)(inc >> 34) == sc.epoch;  // before segment 0: prefix zero
-    const bool complete = j < 0 || (uint32_t)(cs >> 32) == 32u;
-    const uint32_t inc_mask = __ballot_sync(0xFFFFFFFFu, has_inc);
-    const uint32_t bad_mask = __ballot_sync(0xFFFFFFFFu, !complete);
-    const uint32_t first_inc = inc_mask ? (uint32_t)__ffs(inc_mask) - 1u : 32u;
-    const uint32_t first_bad = bad_mask ? (uint32_t)__ffs(bad_mask) - 1u : 32u;
-    if (first_bad < first_inc) {  // a segment we must add is not complete yet
-      ++spins;
-      if (spins > sc.spin_limit || ((spins & 63u) == 0 && ld_relaxed(status) == kErrTimeout)) return false;
-      __nanosleep(40);
-      continue;
-    }
-    uint32_t c = lane < first_inc ? (uint32_t)cs : (lane == first_inc && j >= 0 ? (uint32_t)inc : 0u);
-    asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(c) : "r"(0xFFFFFFFFu));
-    sum += c;
-    if (first_inc < 32u) break;
-    k -= 32;
-  }
-  if (lane == 0 && seg > 0) st_relaxed(sc.seg_inc + (seg - 1u), scan_word(sc.epoch, 2u, (uint32_t)(sum - own)));
-  *excl = sum;
-  return true;
 }
 
 }  // namespace fh

@@ -2,9 +2,9 @@
 
 It serves callers that cannot call cudaMalloc when they need the codec -- an engine that compresses
 because its device-memory budget is already spent, a process whose memory is wholly held by a
-framework pool, a loop that cannot take the synchronisation an allocation may imply.  Its scan
-scratch is a fixed array inside the library, shared by all calls on a device and cleared by each
-call.  The test drives it through the C ABI and requires the same container, byte for byte, as
+framework pool, a loop that cannot take the synchronisation an allocation may imply.  Its
+book-keeping scratch is a fixed array inside the library, shared by all calls on a device and cleared
+by each call.  The test drives it through the C ABI and requires the same container, byte for byte, as
 fh_compress, twice in a row (the second call sees the first call's leftovers in the array), and
 checks that a tensor beyond the fixed limit is refused.
 
@@ -41,11 +41,11 @@ def _compress_both(spec, bits):
 def test_static_scratch_entry_point_matches_fh_compress_on_two_calls_in_a_row():
     build.build()
     api.lib()
-    # first call: many tiles with mixed plane classes, so the look-back scan really uses the flags
+    # first call: many planes of mixed classes, so the work list and the chunk sums are really used
     a = synth.TensorSpec("za", (64, 48, 14, 14), synth.F32, "spiky_relu", 5)
     ref, got = _compress_both(a, 2)
     assert ref.size == got.size and np.array_equal(ref, got)
-    # second call, right after: fewer, differently sized tiles over the same array
+    # second call, right after: fewer, larger planes over the same array
     b = synth.TensorSpec("zb", (8, 24, 56, 56), synth.BF16, "laplace_ch", 6)
     ref, got = _compress_both(b, 8)
     assert ref.size == got.size and np.array_equal(ref, got)
@@ -57,12 +57,11 @@ def test_static_scratch_entry_point_matches_fh_compress_on_two_calls_in_a_row():
 def test_static_scratch_entry_point_refuses_tensors_beyond_its_limit():
     import torch
     build.build()
-    # 4x4 fp32 planes: 512 planes per 32 KB tile -> more than FH_STATIC_MAX_TILES tiles
-    planes = 512 * (api.FH_STATIC_MAX_TILES + 1)
+    planes = api.FH_STATIC_MAX_PLANES + 64           # one batch row more than the fixed work list holds
     d = api.desc((planes // 64, 64, 4, 4), api.FH_F32)
-    p = api.default_params(bits=2, salient_mode=api.FH_SALIENT_OFF)
+    p = api.default_params(bits=2)
     x = torch.zeros(planes * 16, dtype=torch.float32, device="cuda")
-    dst = torch.empty(api.compressed_bytes(d, p, 0), dtype=torch.uint8, device="cuda")
+    dst = torch.empty(api.compressed_bytes(d, p, 1), dtype=torch.uint8, device="cuda")
     assert api.fh_compress_static(d, p, x, dst, None) == api.FH_ERR_UNSUPPORTED
     assert api.fh_compress(d, p, x, dst, None) == api.FH_OK   # the allocating entry point takes it
     torch.cuda.synchronize()
