@@ -284,13 +284,31 @@ int launch_on(K kernel, const Plan& pl, cudaStream_t stream, int* grid) {
   return grid_for(kernel, pl.sm_total, pl.ntiles, grid);
 }
 
+// Launch that may overlap the tail of the previous kernel on the stream: every kernel of this library
+// passes dep_wait() before it touches global memory, so stream order is kept.
+template <typename K, typename A>
+cudaError_t launch_dependent(K kernel, int grid, int threads, size_t smem, cudaStream_t stream, const Plan& pl,
+                             const A& a) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3((unsigned)threads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, pl, a);
+}
+
 template <int DT, int BITS>
 int launch_generic_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
   int grid = 0;
   int rc = grid_for(fh::compress_generic<DT, BITS>, pl.sm_total, pl.ntiles, &grid);
   if (rc != FH_OK) return rc;
-  fh::compress_generic<DT, BITS><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
-  return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+  return launch_dependent(fh::compress_generic<DT, BITS>, grid, fh::kThreads, pl.sm_total, stream, pl, a) == cudaSuccess
+             ? FH_OK : FH_ERR_CUDA;
 }
 
 template <int DT, bool SIGMA, int NT>
@@ -298,8 +316,8 @@ int launch_cta_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream)
   int grid = 0;
   int rc = grid_for(fh::compress_cta<DT, SIGMA, NT>, pl.sm_total, pl.ntiles, &grid, NT);
   if (rc != FH_OK) return rc;
-  fh::compress_cta<DT, SIGMA, NT><<<grid, NT, pl.sm_total, stream>>>(pl, a);
-  return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+  return launch_dependent(fh::compress_cta<DT, SIGMA, NT>, grid, NT, pl.sm_total, stream, pl, a) == cudaSuccess
+             ? FH_OK : FH_ERR_CUDA;
 }
 
 template <int DT, bool SIGMA, int TT, bool FULLVEC>
@@ -307,8 +325,8 @@ int launch_warp_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream
   int grid = 0;
   int rc = grid_for(fh::compress_warp<DT, SIGMA, TT, FULLVEC>, pl.sm_total, pl.ntiles, &grid, fh::kWarpKernelThreads);
   if (rc != FH_OK) return rc;
-  fh::compress_warp<DT, SIGMA, TT, FULLVEC><<<grid, fh::kWarpKernelThreads, pl.sm_total, stream>>>(pl, a);
-  return cudaGetLastError() == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+  return launch_dependent(fh::compress_warp<DT, SIGMA, TT, FULLVEC>, grid, fh::kWarpKernelThreads, pl.sm_total, stream,
+                          pl, a) == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
 template <int DT, bool SIGMA, bool FULLVEC>
@@ -345,11 +363,12 @@ int launch_blockwise(const Plan& pl, const fh::CompressArgs& a, cudaStream_t str
   if (rc != FH_OK) return rc;
   rc = grid_for(fh::blockwise_kernel<DT, true>, pl.sk_total, 0x7FFFFFFFu, &g1, (int)pl.sk_threads);
   if (rc != FH_OK) return rc;
-  fh::blockwise_kernel<DT, false><<<g0, pl.sk_threads, pl.sk_total, stream>>>(pl, a);
-  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  // launched with programmatic serialisation: both may become resident while their predecessor drains
+  if (launch_dependent(fh::blockwise_kernel<DT, false>, g0, (int)pl.sk_threads, pl.sk_total, stream, pl, a) != cudaSuccess)
+    return FH_ERR_CUDA;
   g_launches.fetch_add(1);
-  fh::blockwise_kernel<DT, true><<<g1, pl.sk_threads, pl.sk_total, stream>>>(pl, a);
-  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  if (launch_dependent(fh::blockwise_kernel<DT, true>, g1, (int)pl.sk_threads, pl.sk_total, stream, pl, a) != cudaSuccess)
+    return FH_ERR_CUDA;
   g_launches.fetch_add(1);
   return FH_OK;
 }
@@ -384,8 +403,8 @@ int launch_decompress_t(const Plan& pl, const fh::DecompressArgs& a, cudaStream_
   int grid = 0;
   int rc = grid_for(fh::decompress_kernel<DT, TT>, pl.sm_total, pl.ntiles, &grid);
   if (rc != FH_OK) return rc;
-  fh::decompress_kernel<DT, TT><<<grid, fh::kThreads, pl.sm_total, stream>>>(pl, a);
-  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  if (launch_dependent(fh::decompress_kernel<DT, TT>, grid, fh::kThreads, pl.sm_total, stream, pl, a) != cudaSuccess)
+    return FH_ERR_CUDA;
   g_launches.fetch_add(1);
   return FH_OK;
 }

@@ -346,6 +346,8 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
   __shared__ uint32_t s_tile;
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
+  dep_wait();     // the previous kernel on the stream has completed
 
   const uint32_t tid = threadIdx.x;
   uint8_t* tile_buf = smem + pl.sm_tile;
@@ -682,9 +684,8 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
   __shared__ volatile uint32_t s_abort;
 
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-  const Dest d = make_dest(pl, a);
   const uint32_t nstage = pl.nstage;
-  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
   if (tid == 0) {
     for (uint32_t s = 0; s < nstage; ++s) {
       mbar_init(&s_full[s], 1);
@@ -694,6 +695,9 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     s_abort = 0;
   }
   __syncthreads();
+  dep_wait();  // the previous kernel on the stream has completed; global memory may be touched from here on
+  const Dest d = make_dest(pl, a);
+  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
 
   if (warp == (uint32_t)kWarps) {
     // ======================= producer (all 32 lanes walk the loop, lane 0 issues) =======================
@@ -711,9 +715,12 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
         aborted = true;
         break;
       }
-      uint32_t t = 0;
-      if (lane == 0) t = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
-      t = __shfl_sync(0xFFFFFFFFu, t, 0);
+      // the first tile of every stage follows from the CTA's index; later tiles are handed out
+      uint32_t t = blockIdx.x + n * gridDim.x;
+      if (n >= nstage) {
+        if (lane == 0) t = nstage * gridDim.x + (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+        t = __shfl_sync(0xFFFFFFFFu, t, 0);
+      }
       if (t >= pl.ntiles) {
         // no more tiles: wake the consumers at this stage, then wait for the tiles still in the ring
         const uint32_t first = n >= nstage ? n - nstage + 1u : 0u;
@@ -863,19 +870,21 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
   __shared__ uint32_t s_abort;
 
   const uint32_t tid = threadIdx.x;
-  const Dest d = make_dest(pl, a);
   const Team team = make_team(NT, s_red);
   const uint32_t nstage = pl.nstage, groups = pl.groups, bits = (uint32_t)pl.bits;
   uint32_t rp = 0;
-  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
-
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
   if (tid == 0) {
     for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
     fence_mbar_init();
     s_abort = 0;
   }
-  __syncthreads();
-  uint32_t next_ticket = 0;  // thread 0: the ticket for the next load, requested one tile ahead
+  dep_wait();  // the previous kernel on the stream has completed; global memory may be touched from here on
+  const Dest d = make_dest(pl, a);
+  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+  // Thread 0 issues the loads.  The first tile of every stage follows from the CTA's index; later tiles
+  // are handed out, the request running one tile ahead of its use.
+  uint32_t next_ticket = blockIdx.x, issued = 0;
   auto issue = [&](uint32_t s) {
     const uint32_t t = next_ticket;
     s_tiles[s] = t;
@@ -884,13 +893,13 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
       mbar_expect_tx(&s_full[s], (uint32_t)pl.plane_bytes);
       bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + (uint64_t)t * pl.plane_bytes,
                (uint32_t)pl.plane_bytes, &s_full[s]);
-      next_ticket = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+      ++issued;
+      next_ticket = issued < nstage ? blockIdx.x + issued * gridDim.x
+                                    : nstage * gridDim.x + (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
     }
   };
-  if (tid == 0) {
-    next_ticket = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+  if (tid == 0)
     for (uint32_t s = 0; s < nstage; ++s) issue(s);
-  }
   __syncthreads();
 
   uint32_t s = 0, phase = 0;
@@ -1046,6 +1055,8 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
   __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
 
   const uint32_t tid = threadIdx.x, lane32 = tid & 31u, warp = tid >> 5;
+  dep_trigger();
+  dep_wait();  // the previous kernel of the call has completed: its list, table and counters are visible
   const Dest d = make_dest(pl, a);
   const uint32_t count = (uint32_t)ld_relaxed(&a.sc->wl_count);
   if (tid == 0) s_pl = pl;

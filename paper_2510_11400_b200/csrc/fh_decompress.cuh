@@ -188,6 +188,8 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
   __shared__ Plan s_pl;  // copy for the outlined slow path, which takes it by address
   const uint32_t tid = threadIdx.x;
   if (tid == 0) s_pl = pl;
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
+  dep_wait();     // the previous kernel on the stream (the one that wrote the container) has completed
   const unsigned long long off_in = a.d_off_in ? *a.d_off_in : 0ull;
   const uint8_t* src = a.src_base + off_in;
   const unsigned long long src_bytes = a.src_bytes > off_in ? a.src_bytes - off_in : 0ull;
