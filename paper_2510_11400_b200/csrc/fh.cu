@@ -358,16 +358,11 @@ int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, c
 
 template <int DT>
 int launch_blockwise(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
-  int g0 = 0, g1 = 0;
-  int rc = grid_for(fh::blockwise_kernel<DT, false>, pl.sk_total, 0x7FFFFFFFu, &g0, (int)pl.sk_threads);
+  // the grid must be resident as a whole (the kernel has a barrier over it): what the device holds at once
+  int g = 0;
+  int rc = grid_for(fh::blockwise_kernel<DT>, pl.sk_total, 0x7FFFFFFFu, &g, (int)pl.sk_threads);
   if (rc != FH_OK) return rc;
-  rc = grid_for(fh::blockwise_kernel<DT, true>, pl.sk_total, 0x7FFFFFFFu, &g1, (int)pl.sk_threads);
-  if (rc != FH_OK) return rc;
-  // launched with programmatic serialisation: both may become resident while their predecessor drains
-  if (launch_dependent(fh::blockwise_kernel<DT, false>, g0, (int)pl.sk_threads, pl.sk_total, stream, pl, a) != cudaSuccess)
-    return FH_ERR_CUDA;
-  g_launches.fetch_add(1);
-  if (launch_dependent(fh::blockwise_kernel<DT, true>, g1, (int)pl.sk_threads, pl.sk_total, stream, pl, a) != cudaSuccess)
+  if (launch_dependent(fh::blockwise_kernel<DT>, g, (int)pl.sk_threads, pl.sk_total, stream, pl, a) != cudaSuccess)
     return FH_ERR_CUDA;
   g_launches.fetch_add(1);
   return FH_OK;

@@ -4,7 +4,7 @@
 // codes fill its slot; the payload of a salient or raw plane runs through its slot and continues in
 // the overflow region, in plane order.
 //
-// A call runs up to three kernels on its stream:
+// A call runs one or two kernels on its stream:
 //   1. a streaming kernel (one pass over the dense tensor): per-plane statistics, three-sigma class,
 //      and for normal planes the codes and the table entry.  Normal planes depend on nothing but
 //      themselves, so this kernel has no cross-CTA waits.  A plane that takes the block-wise path only
@@ -13,12 +13,12 @@
 //            a sub-warp team per plane, groups kept in registers;
 //        compress_cta<DT, SIGMA, NT>            larger planes of whole 16-byte chunks: one plane per CTA;
 //        compress_generic<DT, BITS>             everything else (ragged large planes);
-//   2. blockwise_kernel<DT, false> measures every plane of the work list (block classes, CSR and code
-//      sizes), decides salient versus raw, records the sizes;
-//   3. blockwise_kernel<DT, true> derives each listed plane's place in the overflow region from the
-//      recorded sizes (plane order, so the bytes do not depend on scheduling) and writes the payloads;
-//      its last CTA writes the header and the result words.
-// With salient_mode OFF only the first kernel runs and finishes the container itself.
+//   2. blockwise_kernel<DT> (not with salient_mode OFF): measures every plane of the work list (block
+//      classes, CSR and code sizes), decides salient versus raw, and after a barrier over its grid
+//      places the payloads in the overflow region in plane order (so the bytes do not depend on
+//      scheduling) and writes them; its last CTA writes the header and the result words.  With an
+//      empty work list it only writes the header.
+// With salient_mode OFF the streaming kernel finishes the container itself.
 #pragma once
 
 #include "fh_device.cuh"
@@ -55,60 +55,64 @@ struct SplitOut {
   __device__ __forceinline__ void st16(uint32_t o, uint32_t v) const { *reinterpret_cast<uint16_t*>(at(o)) = (uint16_t)v; }
 };
 
-// Pre-quantised integer of the element at (y, x); positions outside the plane count as value 0.
+// One 8x8 block in the registers of a warp: lane l holds the elements (l >> 3, l & 7) and
+// ((l >> 3) + 4, l & 7) of the block, i.e. raster positions l and l + 32.  Positions outside the
+// plane count as value 0.
+struct BlockRegs {
+  float x0, x1;    // values (rows 0-3, rows 4-7)
+  bool in0, in1;   // the positions lie inside the plane
+  uint32_t idx0;   // plane index of the first position; the second is idx0 + 4 W
+};
 template <int DT>
-__device__ __forceinline__ int32_t plane_k(const uint8_t* plane, int H, int W, int y, int x, float inv2e, bool* big) {
-  const float v = (y < H && x < W) ? load_elem<DT>(plane, (uint32_t)y * (uint32_t)W + (uint32_t)x) : 0.0f;
-  return dense_k(v, inv2e, big);
+__device__ __forceinline__ BlockRegs block_load(const uint8_t* plane, int H, int W, int by, int bx, uint32_t lane) {
+  BlockRegs r;
+  const int y0 = by * 8 + (int)(lane >> 3), x = bx * 8 + (int)(lane & 7u);
+  r.in0 = y0 < H && x < W;
+  r.in1 = y0 + 4 < H && x < W;
+  r.idx0 = (uint32_t)y0 * (uint32_t)W + (uint32_t)x;
+  r.x0 = r.in0 ? load_elem<DT>(plane, r.idx0) : 0.0f;
+  r.x1 = r.in1 ? load_elem<DT>(plane, r.idx0 + 4u * (uint32_t)W) : 0.0f;
+  return r;
 }
 
-// Residual codes of one dense 8x8 block (Eq. 7-9), by all 32 lanes of a warp: first-order Lorenzo
-// prediction on the pre-quantised integers k, neighbours outside the block count as 0.  Every element
-// is independent because prediction runs on k, which follows from the input alone.  Lane l takes the
-// elements l and l + 32 of the block's raster order.  Returns the number of verbatim elements.
-// WRITE: also emits the 64 code bytes (logical offset o_codes) and the verbatim values (from logical
-// offset o_outl, raster order).
-template <int DT, bool WRITE>
-__device__ __forceinline__ uint32_t block_codes_warp(const uint8_t* plane, int H, int W, int by, int bx, float inv2e,
-                                                     const SplitOut& out, uint32_t o_codes, uint32_t o_outl) {
-  const uint32_t lane = threadIdx.x & 31u;
-  const int j = (int)(lane & 7u);
-  uint32_t n_out = 0;
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    const int i = half * 4 + (int)(lane >> 3);
-    const int y = by * 8 + i, x = bx * 8 + j;
-    const bool inpl = (y < H) && (x < W);
-    bool big, nb;
-    const int32_t k = plane_k<DT>(plane, H, W, y, x, inv2e, &big);
-    const int32_t up = i > 0 ? plane_k<DT>(plane, H, W, y - 1, x, inv2e, &nb) : 0;
-    const int32_t left = j > 0 ? plane_k<DT>(plane, H, W, y, x - 1, inv2e, &nb) : 0;
-    const int32_t ul = (i > 0 && j > 0) ? plane_k<DT>(plane, H, W, y - 1, x - 1, inv2e, &nb) : 0;
-    const int32_t delta = k - (up + left - ul);
-    const bool verbatim = inpl && (big || delta > 127 || delta < -127);
-    const uint32_t code = !inpl ? 128u : (verbatim ? 0u : (uint32_t)(delta + 128));
-    const uint32_t m = __ballot_sync(0xFFFFFFFFu, verbatim);
-    if (WRITE) {
-      if (verbatim) {
-        const uint32_t rank = n_out + __popc(m & ((1u << lane) - 1u));
-        const uint32_t idx = (uint32_t)y * (uint32_t)W + (uint32_t)x;
-        if (DT == kF32) out.st32(o_outl + 4u * rank, reinterpret_cast<const uint32_t*>(plane)[idx]);
-        else out.st16(o_outl + 2u * rank, reinterpret_cast<const uint16_t*>(plane)[idx]);
-      }
-      uint32_t w = code | (__shfl_down_sync(0xFFFFFFFFu, code, 1) << 8);
-      w |= __shfl_down_sync(0xFFFFFFFFu, w, 2) << 16;
-      if ((lane & 3u) == 0u) out.st32(o_codes + (uint32_t)half * 32u + lane, w);
-    }
-    n_out += __popc(m);
+// Residual codes of a dense block (Eq. 7-9): first-order Lorenzo prediction on the pre-quantised
+// integers k, neighbours outside the block count as 0.  Every element is independent because
+// prediction runs on k, which follows from the input alone; the neighbours' k come from the other
+// lanes by shuffle.  code0/code1: the lane's two code bytes; m0/m1: ballots of the verbatim elements.
+__device__ __forceinline__ void block_codes(const BlockRegs& r, float inv2e, uint32_t lane, uint32_t& code0,
+                                            uint32_t& code1, uint32_t& m0, uint32_t& m1) {
+  const uint32_t full = 0xFFFFFFFFu, c = lane & 7u, r0 = lane >> 3;
+  bool big0, big1;
+  const int32_t k0 = dense_k(r.x0, inv2e, &big0), k1 = dense_k(r.x1, inv2e, &big1);
+  int32_t left0 = __shfl_up_sync(full, k0, 1), up0 = __shfl_up_sync(full, k0, 8), ul0 = __shfl_up_sync(full, k0, 9);
+  int32_t left1 = __shfl_up_sync(full, k1, 1), up1 = __shfl_up_sync(full, k1, 8), ul1 = __shfl_up_sync(full, k1, 9);
+  const int32_t up1r = __shfl_sync(full, k0, 24 + (int)c), ul1r = __shfl_sync(full, k0, 23 + (int)c);  // row 3 feeds row 4
+  if (r0 == 0) {
+    up0 = 0;
+    ul0 = 0;
+    up1 = up1r;
+    ul1 = ul1r;
   }
-  return n_out;
+  if (c == 0) {
+    left0 = 0;
+    ul0 = 0;
+    left1 = 0;
+    ul1 = 0;
+  }
+  const int32_t d0 = k0 - (up0 + left0 - ul0), d1 = k1 - (up1 + left1 - ul1);
+  const bool v0 = r.in0 && (big0 || d0 > 127 || d0 < -127), v1 = r.in1 && (big1 || d1 > 127 || d1 < -127);
+  code0 = !r.in0 ? 128u : (v0 ? 0u : (uint32_t)(d0 + 128));
+  code1 = !r.in1 ? 128u : (v1 ? 0u : (uint32_t)(d1 + 128));
+  m0 = __ballot_sync(full, v0);
+  m1 = __ballot_sync(full, v1);
 }
 
-// Block-wise path, measuring part (Section 4.4.1): non-zero mask pooled per 8x8 block against tau,
-// CSR row counts over the sparse blocks, verbatim counts of the dense blocks.  The team is a whole
-// warp or a whole CTA.  Leaves in shared scratch: rowp[0..H] = CSR row pointers, blk_a[b] = 1 for
-// dense blocks, blk_b[b] = rank of block b among the dense blocks, blk_c[b] = index of the block's
-// first verbatim value.
+// Block-wise path, measuring part (Section 4.4.1): one pass over the plane's 8x8 blocks, a warp per
+// block.  The non-zero mask of a block is two ballots; its pooled density against tau says dense or
+// sparse; a sparse block adds its row counts to the CSR row counters, a dense block is coded once to
+// count its verbatim elements.  The team is a whole warp or a whole CTA.  Leaves in shared scratch:
+// rowp[0..H] = CSR row pointers, blk_a[b] = 1 for dense blocks, blk_b[b] = rank of block b among the
+// dense blocks, blk_c[b] = index of the block's first verbatim value.
 template <int DT>
 __device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& pl, const uint8_t* plane, uint32_t* sal) {
   uint32_t* rowp = sal;
@@ -118,51 +122,34 @@ __device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& p
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx;
   const uint32_t nw = t.block ? t.nwarps : 1u, wid = t.block ? threadIdx.x >> 5 : 0u, lane32 = threadIdx.x & 31u;
-  for (uint32_t b = t.lane; b < nblk; b += t.size) blk_a[b] = 0;
+  const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
   for (uint32_t y = t.lane; y <= (uint32_t)H; y += t.size) rowp[y] = 0;
   team_sync(t);
-  // pooled mask: non-zero count per block, accumulated from (block, row) items
-  for (uint32_t r = t.lane; r < nblk * 8u; r += t.size) {
-    const uint32_t b = r >> 3, i = r & 7u;
-    const int y = (int)(b / nbx) * 8 + (int)i, x0 = (int)(b % nbx) * 8;
-    if (y < H) {
-      uint32_t cnt = 0;
-      const int x1 = min(W, x0 + 8);
-      for (int x = x0; x < x1; ++x) cnt += load_elem<DT>(plane, (uint32_t)y * W + x) != 0.0f;
-      if (cnt) atomicAdd(&blk_a[b], cnt);
+  for (uint32_t b = wid; b < nblk; b += nw) {
+    const uint32_t by = b / nbx, bx = b - by * nbx;
+    const BlockRegs r = block_load<DT>(plane, H, W, (int)by, (int)bx, lane32);
+    const uint32_t z0 = __ballot_sync(0xFFFFFFFFu, r.x0 != 0.0f), z1 = __ballot_sync(0xFFFFFFFFu, r.x1 != 0.0f);
+    const uint32_t nnz = __popc(z0) + __popc(z1);
+    const bool dense = (uint64_t)nnz * pl.tau_den >= (uint64_t)pl.tau_num * 64u;
+    uint32_t n_out = 0;
+    if (dense) {
+      uint32_t c0, c1, m0, m1;
+      block_codes(r, inv2e, lane32, c0, c1, m0, m1);
+      n_out = __popc(m0) + __popc(m1);
+    } else if (lane32 < 8u) {  // lane r: non-zeros of row r of the block
+      const uint32_t cnt = __popc(((lane32 < 4u ? z0 : z1) >> ((lane32 & 3u) * 8u)) & 0xFFu);
+      if (cnt) atomicAdd(&rowp[by * 8u + lane32], cnt);
     }
-  }
-  team_sync(t);
-  for (uint32_t b = t.lane; b < nblk; b += t.size) {
-    const uint32_t dense = (uint64_t)blk_a[b] * pl.tau_den >= (uint64_t)pl.tau_num * 64u;
-    blk_a[b] = dense;
-    blk_b[b] = dense;
+    if (lane32 == 0) {
+      blk_a[b] = dense;
+      blk_b[b] = dense;
+      blk_c[b] = n_out;
+    }
   }
   team_sync(t);
   SalientInfo info;
   info.n_dense = team_excl_scan(t, blk_b, nblk);
-  // CSR row counts: non-zeros of the sparse blocks, again from (block, row) items
-  for (uint32_t r = t.lane; r < nblk * 8u; r += t.size) {
-    const uint32_t b = r >> 3, i = r & 7u;
-    const int y = (int)(b / nbx) * 8 + (int)i, x0 = (int)(b % nbx) * 8;
-    if (y < H && !blk_a[b]) {
-      uint32_t cnt = 0;
-      const int x1 = min(W, x0 + 8);
-      for (int x = x0; x < x1; ++x) cnt += load_elem<DT>(plane, (uint32_t)y * W + x) != 0.0f;
-      if (cnt) atomicAdd(&rowp[y], cnt);
-    }
-  }
-  team_sync(t);
   info.nnz_s = team_excl_scan(t, rowp, (uint32_t)H + 1u);
-  // verbatim counts of the dense blocks, one warp per block
-  const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
-  const SplitOut none = {nullptr, nullptr, 0};
-  for (uint32_t b = wid; b < nblk; b += nw) {
-    uint32_t n = 0;
-    if (blk_a[b]) n = block_codes_warp<DT, false>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, none, 0, 0);
-    if (lane32 == 0) blk_c[b] = n;
-  }
-  team_sync(t);
   info.n_out_d = team_excl_scan(t, blk_c, nblk);
   const uint32_t e = (uint32_t)pl.esize;
   info.size = 16u + 4u * pl.nbm + 4u * ((uint32_t)H + 1u) + a4(2u * info.nnz_s) + a4(e * info.nnz_s) +
@@ -205,28 +192,55 @@ __device__ __noinline__ void salient_write(const Team& t, const Plan& pl, const 
   }
   for (uint32_t y = t.lane; y <= (uint32_t)H; y += t.size) out.st32(o_rp + 4u * y, rowp[y]);
   // CSR entries: one warp per row, columns in chunks of 32, positions by ballot
-  for (int y = (int)wid; y < H; y += (int)nw) {
-    uint32_t o = rowp[y];
-    const uint32_t* brow = blk_a + (uint32_t)(y >> 3) * nbx;
-    for (int x0 = 0; x0 < W; x0 += 32) {
-      const int x = x0 + (int)lane32;
-      const uint32_t idx = (uint32_t)y * W + (uint32_t)x;
-      const bool take = x < W && load_elem<DT>(plane, idx) != 0.0f && !brow[x >> 3];
-      const uint32_t m = __ballot_sync(0xFFFFFFFFu, take);
-      if (take) {
-        const uint32_t pos = o + __popc(m & ((1u << lane32) - 1u));
-        out.st16(o_col + 2u * pos, (uint32_t)x);
-        if (DT == kF32) out.st32(o_val + 4u * pos, reinterpret_cast<const uint32_t*>(plane)[idx]);
-        else out.st16(o_val + 2u * pos, reinterpret_cast<const uint16_t*>(plane)[idx]);
+  if (info.nnz_s) {
+    for (int y = (int)wid; y < H; y += (int)nw) {
+      uint32_t o = rowp[y];
+      if (o == rowp[y + 1]) continue;
+      const uint32_t* brow = blk_a + (uint32_t)(y >> 3) * nbx;
+      for (int x0 = 0; x0 < W; x0 += 32) {
+        const int x = x0 + (int)lane32;
+        const uint32_t idx = (uint32_t)y * W + (uint32_t)x;
+        const bool take = x < W && load_elem<DT>(plane, idx) != 0.0f && !brow[x >> 3];
+        const uint32_t m = __ballot_sync(0xFFFFFFFFu, take);
+        if (take) {
+          const uint32_t pos = o + __popc(m & ((1u << lane32) - 1u));
+          out.st16(o_col + 2u * pos, (uint32_t)x);
+          if (DT == kF32) out.st32(o_val + 4u * pos, reinterpret_cast<const uint32_t*>(plane)[idx]);
+          else out.st16(o_val + 2u * pos, reinterpret_cast<const uint16_t*>(plane)[idx]);
+        }
+        o += __popc(m);
       }
-      o += __popc(m);
     }
   }
+  // dense blocks: 64 code bytes each, verbatim values in raster order
   const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
-  for (uint32_t b = wid; b < nblk; b += nw)
-    if (blk_a[b])
-      block_codes_warp<DT, true>(plane, H, W, (int)(b / nbx), (int)(b % nbx), inv2e, out, o_codes + 64u * blk_b[b],
-                                 o_outl + e * blk_c[b]);
+  const uint32_t lt = (1u << lane32) - 1u;
+  for (uint32_t b = wid; b < nblk; b += nw) {
+    if (!blk_a[b]) continue;
+    const uint32_t by = b / nbx, bx = b - by * nbx;
+    const BlockRegs r = block_load<DT>(plane, H, W, (int)by, (int)bx, lane32);
+    uint32_t c0, c1, m0, m1;
+    block_codes(r, inv2e, lane32, c0, c1, m0, m1);
+    const uint32_t oc = o_codes + 64u * blk_b[b], oo = o_outl + e * blk_c[b];
+    if ((m0 >> lane32) & 1u) {
+      const uint32_t rank = __popc(m0 & lt);
+      if (DT == kF32) out.st32(oo + 4u * rank, reinterpret_cast<const uint32_t*>(plane)[r.idx0]);
+      else out.st16(oo + 2u * rank, reinterpret_cast<const uint16_t*>(plane)[r.idx0]);
+    }
+    if ((m1 >> lane32) & 1u) {
+      const uint32_t rank = __popc(m0) + __popc(m1 & lt), idx1 = r.idx0 + 4u * (uint32_t)W;
+      if (DT == kF32) out.st32(oo + 4u * rank, reinterpret_cast<const uint32_t*>(plane)[idx1]);
+      else out.st16(oo + 2u * rank, reinterpret_cast<const uint16_t*>(plane)[idx1]);
+    }
+    uint32_t w0 = c0 | (__shfl_down_sync(0xFFFFFFFFu, c0, 1) << 8);
+    w0 |= __shfl_down_sync(0xFFFFFFFFu, w0, 2) << 16;
+    uint32_t w1 = c1 | (__shfl_down_sync(0xFFFFFFFFu, c1, 1) << 8);
+    w1 |= __shfl_down_sync(0xFFFFFFFFu, w1, 2) << 16;
+    if ((lane32 & 3u) == 0u) {
+      out.st32(oc + lane32, w0);
+      out.st32(oc + 32u + lane32, w1);
+    }
+  }
 }
 
 // Raw plane: verbatim copy through the slot into the overflow part, zero padded.
@@ -258,9 +272,42 @@ __device__ __forceinline__ Dest make_dest(const Plan& pl, const CompressArgs& a)
   return d;
 }
 
-// Last step of every CTA of a kernel: count the exit; the last CTA to leave returns the hand-out
-// counters to zero.  FINAL (the call's last kernel): it also writes the header and the result words
-// and clears everything else the call touched.
+// One thread, after everything else of the call is done: header, result words, and every counter the
+// call touched back to zero.
+__device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, const Dest& d) {
+  const unsigned long long ovf16 = ld_relaxed(&a.sc->ovf16);
+  const unsigned long long nsal = ld_relaxed(&a.sc->nsal), nraw = ld_relaxed(&a.sc->nraw);
+  const unsigned long long listed = ld_relaxed(&a.sc->wl_count);
+  uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
+  const unsigned long long total = pl.ovf_off + ovf16 * 16ull;
+  if (total > d.capacity && code < kErrCapacity) code = kErrCapacity;
+  if (d.capacity >= 64) {
+    uint4* hd = reinterpret_cast<uint4*>(d.dst);
+    // a failed container must not pass for a valid one: no magic
+    hd[0] = make_uint4(code == kErrNone ? kMagic : 0u, 1u | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24), pl.N, pl.C);
+    hd[1] = make_uint4((uint32_t)pl.H, (uint32_t)pl.W, 8u | (8u << 8) | (0u << 16) | ((uint32_t)pl.mode << 24),
+                       pl.rho_num | (pl.rho_den << 16));
+    hd[2] = make_uint4(pl.tau_num | (pl.tau_den << 16), __float_as_uint(pl.eps), (uint32_t)nsal, (uint32_t)nraw);
+    hd[3] = make_uint4((uint32_t)pl.tensor_id, (uint32_t)(pl.tensor_id >> 32), (uint32_t)total, (uint32_t)(total >> 32));
+  }
+  if (a.out2) {
+    a.out2[0] = total;
+    a.out2[1] = status_word(code);
+  }
+  if (a.d_off_out) *a.d_off_out = code == kErrNone ? d.off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
+  if (listed) {
+    for (uint32_t k = 0; k < a.nchunks; ++k) a.chunk_ovf[k] = 0u;
+    st_relaxed(&a.sc->ovf16, 0ull);
+    st_relaxed(&a.sc->nsal, 0ull);
+    st_relaxed(&a.sc->nraw, 0ull);
+    st_relaxed(&a.sc->wl_count, 0ull);
+    st_relaxed(&a.sc->arrived, 0ull);
+  }
+  if (code) st_relaxed(&a.sc->status, 0ull);
+}
+
+// Last step of every CTA of a kernel that hands out tiles or counts exits: the last CTA to leave
+// returns those counters to zero and, if this is the call's last kernel (FINAL), finishes the call.
 template <bool FINAL>
 __device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, const Dest& d) {
   __threadfence();
@@ -271,46 +318,7 @@ __device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, 
   __threadfence();
   st_relaxed(&a.sc->ticket, 0ull);
   st_relaxed(&a.sc->exited, 0ull);
-  if (!FINAL) return;
-  const unsigned long long ovf16 = ld_relaxed(&a.sc->ovf16);
-  const unsigned long long nsal = ld_relaxed(&a.sc->nsal), nraw = ld_relaxed(&a.sc->nraw);
-  const unsigned long long listed = ld_relaxed(&a.sc->wl_count);
-  uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
-  const unsigned long long total = pl.ovf_off + ovf16 * 16ull;
-  if (total > d.capacity && code < kErrCapacity) code = kErrCapacity;
-  if (d.capacity >= 64) {
-    uint32_t h[16];
-    h[0] = code == kErrNone ? kMagic : 0u;  // a failed container must not pass for a valid one
-    h[1] = 1u | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24);
-    h[2] = pl.N;
-    h[3] = pl.C;
-    h[4] = (uint32_t)pl.H;
-    h[5] = (uint32_t)pl.W;
-    h[6] = 8u | (8u << 8) | (0u << 16) | ((uint32_t)pl.mode << 24);
-    h[7] = pl.rho_num | (pl.rho_den << 16);
-    h[8] = pl.tau_num | (pl.tau_den << 16);
-    h[9] = __float_as_uint(pl.eps);
-    h[10] = (uint32_t)nsal;
-    h[11] = (uint32_t)nraw;
-    h[12] = (uint32_t)pl.tensor_id;
-    h[13] = (uint32_t)(pl.tensor_id >> 32);
-    h[14] = (uint32_t)total;
-    h[15] = (uint32_t)(total >> 32);
-    uint32_t* hd = reinterpret_cast<uint32_t*>(d.dst);
-    for (int k = 0; k < 16; ++k) hd[k] = h[k];
-  }
-  if (a.out2) {
-    a.out2[0] = total;
-    a.out2[1] = status_word(code);
-  }
-  if (a.d_off_out) *a.d_off_out = code == kErrNone ? d.off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
-  if (listed)
-    for (uint32_t k = 0; k < a.nchunks; ++k) a.chunk_ovf[k] = 0u;
-  st_relaxed(&a.sc->status, 0ull);
-  st_relaxed(&a.sc->ovf16, 0ull);
-  st_relaxed(&a.sc->nsal, 0ull);
-  st_relaxed(&a.sc->nraw, 0ull);
-  st_relaxed(&a.sc->wl_count, 0ull);
+  if (FINAL) finalize(pl, a, d);
 }
 
 __device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane, uint32_t off16, const Rec& r) {
@@ -514,12 +522,12 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     constexpr uint32_t bias = kMagicBits * (1u + (1u << (BITS)) + (1u << (2 * (BITS))) + (1u << (3 * (BITS)))); \
     _Pragma("unroll") for (int k = 0; k < G; ++k) {                                                           \
       const uint32_t g = lane + (uint32_t)(k * TT);                                                           \
+      uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));                       \
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF)) << (BITS);                     \
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF)) << (2 * (BITS));               \
+      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF)) << (3 * (BITS));               \
+      word -= bias;                                                                                           \
       if (FULL || g < groups) {                                                                               \
-        uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));                     \
-        word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF)) << (BITS);                   \
-        word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF)) << (2 * (BITS));             \
-        word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF)) << (3 * (BITS));             \
-        word -= bias;                                                                                         \
         if (!VEC) { /* ragged last group: elements past the plane carry no code */                            \
           const uint32_t valid = min(4u, pl.HW - g * 4u);                                                     \
           if (valid < 4u) word &= (1u << (valid * (BITS))) - 1u;                                              \
@@ -537,48 +545,60 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
 template <int DT, bool SIGMA, int G, int TT, bool FULL, bool VEC>
 __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, const Dest& d, const CompressArgs& a,
                                             const uint8_t* plane, uint64_t gp, uint32_t& rp, Rec& r) {
+  // A thread's G group slots that lie past the plane, and the elements past a ragged last group, are
+  // held as zeros: they add exactly nothing to the fixed-point moments, are kept out of minimum and
+  // maximum with neutral values, are subtracted from the outlier count when zero lies outside the
+  // thresholds, and their codes are not stored.  The arithmetic runs unpredicated over all G slots.
   const uint32_t groups = pl.groups, lane = team.lane;
+  const float pinf = __int_as_float(0x7F800000), ninf = __int_as_float(0xFF800000);
   float x[G][4];
-  float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000), lo1 = lo, hi1 = hi;
-  uint32_t ng = 0, npad = 0;  // groups of this thread; zero-padded elements among them
+  float lo = pinf, hi = ninf, lo1 = pinf, hi1 = ninf;
+  uint32_t npad = 0;  // zero-padded elements among this thread's slots
 #pragma unroll
   for (int k = 0; k < G; ++k) {
     const uint32_t g = lane + (uint32_t)(k * TT);
-    if (FULL || g < groups) {
-      if (VEC) {
-        if (DT == kF32) {
-          const float4 t4 = (reinterpret_cast<const float4*>(plane) + lane)[k * TT];
-          x[k][0] = t4.x; x[k][1] = t4.y; x[k][2] = t4.z; x[k][3] = t4.w;
-        } else {
-          const uint2 t2 = (reinterpret_cast<const uint2*>(plane) + lane)[k * TT];
-          x[k][0] = __uint_as_float(t2.x << 16); x[k][1] = __uint_as_float(t2.x & 0xFFFF0000u);
-          x[k][2] = __uint_as_float(t2.y << 16); x[k][3] = __uint_as_float(t2.y & 0xFFFF0000u);
-        }
-        // per-group partial results keep the dependency chains short
-        const float gl = min_nan(min3_nan(x[k][0], x[k][1], x[k][2]), x[k][3]);
-        const float gh = max_nan(max3_nan(x[k][0], x[k][1], x[k][2]), x[k][3]);
-        if (k & 1) {
-          lo1 = min_nan(lo1, gl);
-          hi1 = max_nan(hi1, gh);
-        } else {
-          lo = min_nan(lo, gl);
-          hi = max_nan(hi, gh);
-        }
-      } else {  // plane not on a 16-byte boundary, possibly with a ragged last group
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const uint32_t i = g * 4u + e;
-          const bool in = i < pl.HW;
-          x[k][e] = in ? load_elem<DT>(plane, i) : 0.0f;
-          if (in) {
-            lo = min_nan(lo, x[k][e]);
-            hi = max_nan(hi, x[k][e]);
-          } else {
-            ++npad;
-          }
-        }
+    if (VEC) {
+      const bool act = FULL || g < groups;
+      if (DT == kF32) {
+        float4 t4 = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (act) t4 = (reinterpret_cast<const float4*>(plane) + lane)[k * TT];
+        x[k][0] = t4.x; x[k][1] = t4.y; x[k][2] = t4.z; x[k][3] = t4.w;
+      } else {
+        uint2 t2 = make_uint2(0u, 0u);
+        if (act) t2 = (reinterpret_cast<const uint2*>(plane) + lane)[k * TT];
+        x[k][0] = __uint_as_float(t2.x << 16); x[k][1] = __uint_as_float(t2.x & 0xFFFF0000u);
+        x[k][2] = __uint_as_float(t2.y << 16); x[k][3] = __uint_as_float(t2.y & 0xFFFF0000u);
       }
-      ++ng;
+      // per-group partial results keep the dependency chains short
+      float gl = min_nan(min3_nan(x[k][0], x[k][1], x[k][2]), x[k][3]);
+      float gh = max_nan(max3_nan(x[k][0], x[k][1], x[k][2]), x[k][3]);
+      if (!FULL) {
+        gl = act ? gl : pinf;
+        gh = act ? gh : ninf;
+        npad += act ? 0u : 4u;
+      }
+      if (k & 1) {
+        lo1 = min_nan(lo1, gl);
+        hi1 = max_nan(hi1, gh);
+      } else {
+        lo = min_nan(lo, gl);
+        hi = max_nan(hi, gh);
+      }
+    } else {  // plane not on a 16-byte boundary, possibly with a ragged last group
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const uint32_t i = g * 4u + e;
+        const bool in = i < pl.HW;
+        x[k][e] = in ? load_elem<DT>(plane, i) : 0.0f;
+        if (e & 1) {
+          lo1 = min_nan(lo1, in ? x[k][e] : pinf);
+          hi1 = max_nan(hi1, in ? x[k][e] : ninf);
+        } else {
+          lo = min_nan(lo, in ? x[k][e] : pinf);
+          hi = max_nan(hi, in ? x[k][e] : ninf);
+        }
+        npad += in ? 0u : 1u;
+      }
     }
   }
   lo = min_nan(lo, lo1);
@@ -592,11 +612,9 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
     const SigmaScale sc = sigma_scale(lo, hi);
     uint32_t as = 0, aq = 0;
 #pragma unroll
-    for (int k = 0; k < G; ++k)
-      if (FULL || lane + (uint32_t)(k * TT) < groups) sigma_addends4(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
-    if (FULL) ng = G;
+    for (int k = 0; k < G; ++k) sigma_addends4(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
     long long Is, Iq;
-    team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
+    team_sum2(team, (int32_t)(as - (uint32_t)G * kMagicBits), (int32_t)(aq - (uint32_t)G * kMagicBits), Is, Iq, rp);
     float tlo, thi;
     if (TT > 32) sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
     else sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, tlo, thi);
@@ -605,22 +623,20 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
       uint32_t c[4] = {0, 0, 0, 0};  // four counters: short dependency chains
       if (lo >= tlo) {               // nothing below: one compare per element
 #pragma unroll
-        for (int k = 0; k < G; ++k)
-          if (FULL || lane + (uint32_t)(k * TT) < groups) {
+        for (int k = 0; k < G; ++k) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) c[e] += x[k][e] > thi;
-          }
+          for (int e = 0; e < 4; ++e) c[e] += x[k][e] > thi;
+        }
         cnt = (c[0] + c[1]) + (c[2] + c[3]);
-        if (!VEC && 0.0f > thi) cnt -= npad;  // padded zeros are not elements
+        if (!(FULL && VEC) && 0.0f > thi) cnt -= npad;  // padded zeros are not elements
       } else {
 #pragma unroll
-        for (int k = 0; k < G; ++k)
-          if (FULL || lane + (uint32_t)(k * TT) < groups) {
+        for (int k = 0; k < G; ++k) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) c[e] += (x[k][e] > thi) || (x[k][e] < tlo);
-          }
+          for (int e = 0; e < 4; ++e) c[e] += (x[k][e] > thi) || (x[k][e] < tlo);
+        }
         cnt = (c[0] + c[1]) + (c[2] + c[3]);
-        if (!VEC && ((0.0f > thi) || (0.0f < tlo))) cnt -= npad;
+        if (!(FULL && VEC) && ((0.0f > thi) || (0.0f < tlo))) cnt -= npad;
       }
       cnt = team_sum_u32(team, cnt, rp);
     }
@@ -1021,23 +1037,28 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
 }
 
 // =================================================================================================
-// Block-wise kernels: the planes of the work list
+// Block-wise kernel: the planes of the work list
 // =================================================================================================
-// A unit -- one warp for planes up to 8 KB, the whole CTA above -- takes entries i = unit, unit +
-// units, ... of the work list, copies the plane into its shared-memory buffer and runs the
-// measuring part of the block-wise path on it.
+// Runs after the streaming kernel whenever planes can take the block-wise path.  With an empty work
+// list one thread finishes the container.  Otherwise a unit -- one warp for planes up to 8 KB, the
+// whole CTA above -- takes entries i = unit, unit + units, ... of the list.
 //
-// WRITE = false (measuring kernel): the unit decides salient versus raw, completes the plane's table
-// entry (class; the offset stays 0), leaves the three counts of a salient payload in the first
-// 16 bytes of the plane's slot, and adds the plane's overflow size to the sum of its chunk (a chunk
-// is a run of 2^chunk_shift consecutive planes; there are at most kMaxChunks chunks).
+// Measuring phase: the unit copies the plane into its shared-memory buffer, measures it (block
+// classes, CSR and code sizes), decides salient versus raw, completes the plane's table entry (class;
+// the offset stays 0), leaves the three counts of a salient payload in the first 16 bytes of the
+// plane's slot, and adds the plane's overflow size to the sum of its chunk (a chunk is a run of
+// 2^chunk_shift consecutive planes; there are at most kMaxChunks chunks).
 //
-// WRITE = true (writing kernel): every CTA first turns the chunk sums into chunk offsets.  A plane's
-// place in the overflow region is its chunk's offset plus the overflow sizes of the listed planes
-// before it in the same chunk, which the unit recomputes from their table classes and slot headers
-// (nothing else writes those words while this kernel runs, and every writer stores the value that
-// is already there).  The payload is written and the table offset filled in.  The last CTA to leave
-// writes the header and the result words.
+// A barrier over the grid separates the phases: all CTAs are resident (the grid is sized to what the
+// device holds at once); the wait is bounded, and a wait that runs out ends the call with the
+// time-out status instead of hanging.
+//
+// Writing phase: every CTA turns the chunk sums into chunk offsets.  A plane's place in the overflow
+// region is its chunk's offset plus the overflow sizes of the listed planes before it in the same
+// chunk, recomputed from their table classes and slot headers (nothing changes those words any more:
+// whoever stores to them stores the value that is already there).  The unit walks its entries in
+// reverse so that the plane it measured last is still in its buffer; the others are copied and
+// measured again.  The last CTA to leave finishes the container.
 __device__ __forceinline__ uint32_t salient_size(const Plan& pl, uint32_t nnz_s, uint32_t n_dense, uint32_t n_out_d) {
   const uint32_t e = (uint32_t)pl.esize;
   return 16u + 4u * pl.nbm + 4u * ((uint32_t)pl.H + 1u) + a4(2u * nnz_s) + a4(e * nnz_s) + 64u * n_dense +
@@ -1048,17 +1069,40 @@ __device__ __forceinline__ uint32_t ovf_units(const Plan& pl, uint32_t size) {
   return a16(size) > pl.npay ? (a16(size) - pl.npay) >> 4 : 0u;
 }
 
-template <int DT, bool WRITE>
+// Copies plane p into the unit's buffer (whole 16-byte chunks from the aligned start, the ragged end
+// of the tensor byte-wise) and returns where the plane starts in it.
+__device__ __forceinline__ const uint8_t* fetch_plane(const Team& t, const Plan& pl, const uint8_t* src, uint32_t p,
+                                                      uint8_t* ubuf) {
+  const uint64_t start = (uint64_t)p * pl.plane_bytes, end = start + pl.plane_bytes;
+  const uint64_t a0 = start & ~15ull;
+  const uint64_t a1 = min((end + 15ull) & ~15ull, pl.dense_bytes & ~15ull);
+  const uint4* s16 = reinterpret_cast<const uint4*>(src + a0);
+  uint4* t16 = reinterpret_cast<uint4*>(ubuf);
+  const uint32_t n16 = (uint32_t)((a1 - a0) >> 4);
+  for (uint32_t k = t.lane; k < n16; k += t.size) t16[k] = __ldg(s16 + k);
+  for (uint64_t k = a1 + t.lane; k < end; k += t.size) ubuf[k - a0] = src[k];
+  team_sync(t);
+  return ubuf + (uint32_t)(start - a0);
+}
+
+constexpr uint32_t kGridWaitPolls = 1u << 21;  // about a second
+
+template <int DT>
 __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
   __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
+  __shared__ uint32_t s_ok;
 
   const uint32_t tid = threadIdx.x, lane32 = tid & 31u, warp = tid >> 5;
   dep_trigger();
-  dep_wait();  // the previous kernel of the call has completed: its list, table and counters are visible
+  dep_wait();  // the streaming kernel has completed: its list, table and counters are visible
   const Dest d = make_dest(pl, a);
   const uint32_t count = (uint32_t)ld_relaxed(&a.sc->wl_count);
+  if (count == 0) {  // nothing listed: the container lacks only its header
+    if (blockIdx.x == 0 && tid == 0) finalize(pl, a, d);
+    return;
+  }
   if (tid == 0) s_pl = pl;
   const bool unit_cta = pl.sk_cta != 0u;
   const uint32_t upc = unit_cta ? 1u : blockDim.x >> 5;
@@ -1070,10 +1114,71 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
   uint32_t* pre = reinterpret_cast<uint32_t*>(smem + pl.sk_pre_off);
   const uint4* table = reinterpret_cast<const uint4*>(d.dst + 64);
   const uint32_t raw_units = ovf_units(pl, (uint32_t)pl.plane_bytes);
+  __syncthreads();
 
-  if (WRITE && count > 0 && d.fits) {
-    // chunk offsets: exclusive prefix sum of the chunk sums (warp 0: 32 consecutive chunks per lane)
-    for (uint32_t k = tid; k < kMaxChunks; k += blockDim.x) pre[k] = k < a.nchunks ? a.chunk_ovf[k] : 0u;
+  // ---- measuring phase
+  uint32_t kept = 0xFFFFFFFFu;  // the list entry whose plane and measuring scratch are still in the buffer
+  const uint8_t* plane = ubuf;
+  SalientInfo info;
+  info.nnz_s = info.n_dense = info.n_out_d = info.size = 0;
+  for (uint32_t i = unit; i < count; i += units) {
+    if (kept != 0xFFFFFFFFu) team_sync(t);  // the buffer is reused
+    const uint32_t p = a.worklist[i];
+    plane = fetch_plane(t, pl, a.src, p, ubuf);
+    info = salient_measure<DT>(t, s_pl, plane, sal);
+    kept = i;
+    const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
+    const uint32_t my_units = ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
+    if (t.lane == 0) {
+      if (d.fits) {
+        const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(table + p) + 1);  // the streaming kernel's marker
+        reinterpret_cast<uint4*>(d.dst + 64)[p] = make_uint4(0u, (meta & ~3u) | (raw ? kClsRaw : kClsSalient), 0u, 0u);
+        if (!raw)
+          *reinterpret_cast<uint4*>(d.dst + pl.slots_off + (uint64_t)p * pl.npay) =
+              make_uint4(info.nnz_s, info.n_dense, info.n_out_d, 0u);
+      }
+      if (my_units) {
+        atomicAdd(&a.chunk_ovf[p >> a.chunk_shift], my_units);
+        atomicAdd(&a.sc->ovf16, (unsigned long long)my_units);
+      }
+      atomicAdd(raw ? &a.sc->nraw : &a.sc->nsal, 1ull);
+    }
+  }
+
+  // ---- barrier over the grid (bounded)
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    atomicAdd(&a.sc->arrived, 1ull);
+    uint32_t ok = 0;
+    for (uint32_t k = 0; k < kGridWaitPolls; ++k) {
+      if (ld_acquire(&a.sc->arrived) >= (unsigned long long)gridDim.x) {
+        ok = 1;
+        break;
+      }
+      __nanosleep(200);
+    }
+    if (!ok) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+    s_ok = ok;
+  }
+  __syncthreads();
+
+  // ---- writing phase
+  if (s_ok && d.fits && (unit_cta ? blockIdx.x : blockIdx.x * upc) < count) {  // CTAs without entries are done
+    // chunk offsets: exclusive prefix sum of the chunk sums (warp 0: consecutive chunks per lane)
+    {
+      uint32_t v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t k = tid + (uint32_t)q * blockDim.x;
+        v[q] = k < a.nchunks ? __ldcg(a.chunk_ovf + k) : 0u;
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const uint32_t k = tid + (uint32_t)q * blockDim.x;
+        if (k < kMaxChunks) pre[k] = v[q];
+      }
+    }
     __syncthreads();
     if (warp == 0) {
       constexpr uint32_t per = kMaxChunks / 32;
@@ -1091,46 +1196,18 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
         run += v;
       }
     }
-  }
-  __syncthreads();
-
-  if (WRITE ? d.fits : true) {
-    for (uint32_t i = unit; i < count; i += units) {
-      const uint32_t p = a.worklist[i];
-      // ---- copy the plane: whole 16-byte chunks from the aligned start, the ragged end of the tensor byte-wise
-      const uint64_t start = (uint64_t)p * pl.plane_bytes, end = start + pl.plane_bytes;
-      const uint64_t a0 = start & ~15ull;
-      const uint32_t head = (uint32_t)(start - a0);
-      const uint64_t a1 = min((end + 15ull) & ~15ull, pl.dense_bytes & ~15ull);
-      {
-        const uint4* s16 = reinterpret_cast<const uint4*>(a.src + a0);
-        uint4* t16 = reinterpret_cast<uint4*>(ubuf);
-        const uint32_t n16 = (uint32_t)((a1 - a0) >> 4);
-        for (uint32_t k = t.lane; k < n16; k += t.size) t16[k] = __ldg(s16 + k);
-        for (uint64_t k = a1 + t.lane; k < end; k += t.size) ubuf[k - a0] = a.src[k];
-      }
-      team_sync(t);
-      const uint8_t* plane = ubuf + head;
-      const SalientInfo info = salient_measure<DT>(t, s_pl, plane, sal);
-      const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
-      const uint32_t size = raw ? (uint32_t)pl.plane_bytes : info.size;
-      const uint32_t my_units = ovf_units(pl, size);
-      uint8_t* slot = d.dst + pl.slots_off + (uint64_t)p * pl.npay;
-      if (!WRITE) {
-        if (t.lane == 0) {
-          if (d.fits) {
-            const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(table + p) + 1);  // the streaming kernel's marker
-            reinterpret_cast<uint4*>(d.dst + 64)[p] = make_uint4(0u, (meta & ~3u) | (raw ? kClsRaw : kClsSalient), 0u, 0u);
-            if (!raw) *reinterpret_cast<uint4*>(slot) = make_uint4(info.nnz_s, info.n_dense, info.n_out_d, 0u);
-          }
-          if (my_units) {
-            atomicAdd(&a.chunk_ovf[p >> a.chunk_shift], my_units);
-            atomicAdd(&a.sc->ovf16, (unsigned long long)my_units);
-          }
-          atomicAdd(raw ? &a.sc->nraw : &a.sc->nsal, 1ull);
+    __syncthreads();
+    if (unit < count) {
+      for (uint32_t i = unit + ((count - 1u - unit) / units) * units;; i -= units) {
+        const uint32_t p = a.worklist[i];
+        if (i != kept) {
+          team_sync(t);  // the buffer is reused
+          plane = fetch_plane(t, pl, a.src, p, ubuf);
+          info = salient_measure<DT>(t, s_pl, plane, sal);
         }
-      } else {
-        // ---- overflow units of the listed planes before p in its chunk (every warp of the unit computes them)
+        const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
+        const uint32_t my_units = ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
+        // overflow units of the listed planes before p in its chunk (every warp of the unit computes them)
         uint32_t before = 0;
         for (uint32_t q0 = (p >> a.chunk_shift) << a.chunk_shift; q0 < p; q0 += 32u) {
           const uint32_t q = q0 + lane32;
@@ -1150,18 +1227,18 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
         const unsigned long long off16 = (pl.ovf_off >> 4) + pre[p >> a.chunk_shift] + before;
         if ((off16 + my_units) * 16ull <= d.capacity) {  // never write past the capacity
           SplitOut out;
-          out.slot = slot;
+          out.slot = d.dst + pl.slots_off + (uint64_t)p * pl.npay;
           out.ovf = d.dst + off16 * 16ull;
           out.npay = pl.npay;
           if (raw) raw_write(t, s_pl, plane, out);
           else salient_write<DT>(t, s_pl, plane, info, sal, out);
           if (t.lane == 0) *reinterpret_cast<uint32_t*>(d.dst + 64 + 16ull * p) = my_units ? (uint32_t)off16 : 0u;
         }
+        if (i < units + unit) break;  // that was the unit's first entry
       }
-      team_sync(t);  // the buffer is reused by the next entry
     }
   }
-  if (WRITE) cta_exit<true>(pl, a, d);
+  cta_exit<true>(pl, a, d);
 }
 
 }  // namespace fh

@@ -71,7 +71,7 @@ struct Scratch {
   unsigned long long ovf16;     // overflow region size of this call, in 16-byte units
   unsigned long long nsal, nraw;
   unsigned long long wl_count;  // entries of the work list
-  unsigned long long pad;
+  unsigned long long arrived;   // CTAs of the block-wise kernel that have finished measuring
 };
 static_assert(sizeof(Scratch) == 64, "Scratch layout");
 constexpr uint32_t kMaxChunks = 1024;
