@@ -295,8 +295,7 @@ __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, 
     a.out2[1] = status_word(code);
   }
   if (a.d_off_out) *a.d_off_out = code == kErrNone ? d.off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
-  if (listed) {
-    for (uint32_t k = 0; k < a.nchunks; ++k) a.chunk_ovf[k] = 0u;
+  if (listed) {  // (the chunk sums are cleared by the block-wise kernel's last CTA)
     st_relaxed(&a.sc->ovf16, 0ull);
     st_relaxed(&a.sc->nsal, 0ull);
     st_relaxed(&a.sc->nraw, 0ull);
@@ -1131,9 +1130,10 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
     const uint32_t my_units = ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
     if (t.lane == 0) {
       if (d.fits) {
-        const uint32_t meta = __ldg(reinterpret_cast<const uint32_t*>(table + p) + 1);  // the streaming kernel's marker
-        reinterpret_cast<uint4*>(d.dst + 64)[p] = make_uint4(0u, (meta & ~3u) | (raw ? kClsRaw : kClsSalient), 0u, 0u);
-        if (!raw)
+        // the streaming kernel's marker says salient (class bits 01); a raw plane flips them to 10
+        if (raw)
+          atomicXor(reinterpret_cast<uint32_t*>(d.dst + 64 + 16ull * p) + 1, 3u);
+        else
           *reinterpret_cast<uint4*>(d.dst + pl.slots_off + (uint64_t)p * pl.npay) =
               make_uint4(info.nnz_s, info.n_dense, info.n_out_d, 0u);
       }
@@ -1238,7 +1238,18 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
       }
     }
   }
-  cta_exit<true>(pl, a, d);
+  // last CTA to leave: clear the chunk sums (all threads), then finish the container (one thread)
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_ok = atomicAdd(&a.sc->exited, 1ull) == (unsigned long long)gridDim.x - 1ull;
+  __syncthreads();
+  if (!s_ok) return;
+  for (uint32_t k = tid; k < a.nchunks; k += blockDim.x) a.chunk_ovf[k] = 0u;
+  if (tid == 0) {
+    __threadfence();
+    st_relaxed(&a.sc->exited, 0ull);
+    finalize(pl, a, d);
+  }
 }
 
 }  // namespace fh

@@ -442,6 +442,17 @@ __device__ __forceinline__ uint32_t team_sum_u32(const Team& t, uint32_t v, uint
 // In-place exclusive prefix sum of arr[0..n) (shared memory) by the team; returns the total.
 // Every lane takes a contiguous chunk; chunk sums are scanned across the team.
 __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr, uint32_t n) {
+  if (!t.block && t.size == 32u && n <= 32u) {  // a warp and at most one element per lane: one shuffle scan
+    const uint32_t v = t.lane < n ? arr[t.lane] : 0u;
+    uint32_t incl = v;
+    for (uint32_t o = 1; o < 32u; o <<= 1) {
+      const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (t.lane >= o) incl += up;
+    }
+    if (t.lane < n) arr[t.lane] = incl - v;
+    __syncwarp();
+    return __shfl_sync(0xFFFFFFFFu, incl, 31);
+  }
   const uint32_t chunk = (n + t.size - 1u) / t.size;
   const uint32_t b = min(t.lane * chunk, n), e = min(b + chunk, n);
   uint32_t local = 0;
