@@ -259,7 +259,7 @@ int sm_count() {
 template <typename K>
 int grid_for(K kernel, size_t smem, uint32_t ntiles, int* grid, int threads = fh::kThreads) {
   static std::map<std::pair<const void*, size_t>, int> cache;  // guarded by g_mu
-  const auto key = std::make_pair((const void*)kernel, smem);
+  const auto key = std::make_pair((const void*)kernel, (smem << 12) | (size_t)threads);
   auto it = cache.find(key);
   int per_sm;
   if (it == cache.end()) {

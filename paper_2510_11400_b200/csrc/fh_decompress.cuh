@@ -178,8 +178,48 @@ __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const
     }                                                                                                      \
   }
 
+// Four restored values of one group leave as one 16-byte (fp32) or 8-byte (bf16) store.
+template <int DT>
+__device__ __forceinline__ void store_group(uint8_t* out, uint32_t g, float v0, float v1, float v2, float v3) {
+  if (DT == kF32) {
+    reinterpret_cast<float4*>(out)[g] = make_float4(v0, v1, v2, v3);
+  } else {
+    uint2 w;
+    w.x = f32_to_bf16_bits(v0) | (f32_to_bf16_bits(v1) << 16);
+    w.y = f32_to_bf16_bits(v2) | (f32_to_bf16_bits(v3) << 16);
+    reinterpret_cast<uint2*>(out)[g] = w;
+  }
+}
+
+// Normal plane, whole-warp team, one chunk of up to 256 groups starting at group g0 (a multiple of
+// 256).  The chunk's code bytes are fetched as 32-bit words, one or more coalesced loads per lane
+// issued before anything else, and handed to the lanes that need them by shuffle: lane l restores
+// groups g0 + l, g0 + 32 + l, ...  `w` holds the lane's words: word j*32 + l of the chunk's codes.
+template <int DT, int BITS>
+__device__ __forceinline__ void decode_chunk32(const uint32_t (&w)[8], uint32_t lane, uint32_t g0, uint32_t g1,
+                                               float scale, float lo, uint8_t* out) {
+  constexpr uint32_t L = (1u << BITS) - 1u;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t g = g0 + (uint32_t)k * 32u + lane;
+    uint32_t word;
+    if (BITS == 2) {         // one code byte per group: byte k*32 + l = word k*8 + (l >> 2), byte l & 3
+      const uint32_t src = __shfl_sync(0xFFFFFFFFu, w[k >> 2], (uint32_t)(k & 3) * 8u + (lane >> 2));
+      word = (src >> ((lane & 3u) * 8u)) & 0xFFu;
+    } else if (BITS == 4) {  // two code bytes per group: halfword k*32 + l = word k*16 + (l >> 1)
+      const uint32_t src = __shfl_sync(0xFFFFFFFFu, w[k >> 1], (uint32_t)(k & 1) * 16u + (lane >> 1));
+      word = (src >> ((lane & 1u) * 16u)) & 0xFFFFu;
+    } else {                 // one word per group
+      word = w[k];
+    }
+    if (g < g1)
+      store_group<DT>(out, g, dequant(word & L, scale, lo), dequant((word >> BITS) & L, scale, lo),
+                      dequant((word >> (2 * BITS)) & L, scale, lo), dequant((word >> (3 * BITS)) & L, scale, lo));
+  }
+}
+
 template <int DT, int TT>
-__global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, const DecompressArgs a) {
+__global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, const DecompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
   __shared__ uint32_t s_hdr_ok, s_bits;
@@ -236,6 +276,18 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
       const uint64_t gp = item / chunks;
       const uint32_t ch = (uint32_t)(item - gp * chunks);
       const uint32_t g0 = ch * chunk_groups, g1 = min(nfull, g0 + chunk_groups);
+      // whole-warp teams: the chunk's code words are requested before the table entry is known (the slot
+      // sits at a closed-form offset; what a salient plane keeps there is read and dropped)
+      uint32_t cw[8];
+      if (TT == 32) {
+        const uint32_t* s32 = reinterpret_cast<const uint32_t*>(src + slots_off + gp * npay);
+        const uint32_t nwords = npay >> 2, w0 = (g0 * bits) >> 3, per = bits;  // words per lane: 2, 4 or 8
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const uint32_t i = w0 + (uint32_t)j * 32u + lane;
+          cw[j] = ((uint32_t)j < per && i < nwords) ? __ldg(s32 + i) : 0u;
+        }
+      }
       const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + gp);
       const unsigned long long off = (unsigned long long)e.x * 16ull;
       const uint32_t cls = e.y & 3u;
@@ -244,7 +296,11 @@ __global__ void __launch_bounds__(kThreads) decompress_kernel(const Plan pl, con
       if (cls == kClsNormal) {
         if (off != slots_off + gp * npay) { bad = true; continue; }
         const float lo = __uint_as_float(e.z), scale = __uint_as_float(e.w);
-        if (bits == 2u) FH_DECODE_NORMAL(2)
+        if (TT == 32) {
+          if (bits == 2u) decode_chunk32<DT, 2>(cw, lane, g0, g1, scale, lo, out);
+          else if (bits == 4u) decode_chunk32<DT, 4>(cw, lane, g0, g1, scale, lo, out);
+          else decode_chunk32<DT, 8>(cw, lane, g0, g1, scale, lo, out);
+        } else if (bits == 2u) FH_DECODE_NORMAL(2)
         else if (bits == 4u) FH_DECODE_NORMAL(4)
         else FH_DECODE_NORMAL(8)
         if (ch == chunks - 1u && nfull * 4u < pl.HW) {  // ragged or unaligned rest: element stores

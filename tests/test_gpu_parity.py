@@ -97,9 +97,10 @@ SHAPES = [
     (2, 6, 33, 17),    # ragged 8x8 blocks in both directions
     (1, 12, 32, 32),   # one warp per plane, vector loads
     (2, 8, 28, 28),
-    (1, 6, 56, 56),    # whole-CTA teams, several planes per tile
-    (1, 3, 112, 112),  # whole-CTA teams, one plane per tile
+    (1, 6, 56, 56),    # whole-CTA teams of 128 threads
+    (1, 3, 112, 112),  # whole-CTA teams of 512 threads
     (1, 2, 64, 100),
+    (1, 2, 128, 120),  # 60 KB planes
     (300, 1, 4, 4),    # many tiny planes, several tiles with a ragged last tile
 ]
 
