@@ -393,12 +393,31 @@ int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a,
   return rc;
 }
 
+// Largest prime <= n (n >= 2), or 1.
+uint64_t prime_at_most(uint64_t n) {
+  static std::map<uint64_t, uint64_t> cache;  // guarded by g_mu
+  auto it = cache.find(n);
+  if (it != cache.end()) return it->second;
+  for (uint64_t c = n; c >= 2; --c) {
+    bool prime = true;
+    for (uint64_t f = 2; f * f <= c; ++f)
+      if (c % f == 0) {
+        prime = false;
+        break;
+      }
+    if (prime) return cache[n] = c;
+  }
+  return cache[n] = 1;
+}
+
 template <int DT, int TT>
 int launch_decompress_t(const Plan& pl, const fh::DecompressArgs& a, cudaStream_t stream) {
   int grid = 0;
   int rc = grid_for(fh::decompress_kernel<DT, TT>, pl.sm_total, pl.ntiles, &grid);
   if (rc != FH_OK) return rc;
-  if (launch_dependent(fh::decompress_kernel<DT, TT>, grid, fh::kThreads, pl.sm_total, stream, pl, a) != cudaSuccess)
+  fh::DecompressArgs b = a;
+  b.team_stride = prime_at_most((uint64_t)grid * (fh::kThreads / TT));
+  if (launch_dependent(fh::decompress_kernel<DT, TT>, grid, fh::kThreads, pl.sm_total, stream, pl, b) != cudaSuccess)
     return FH_ERR_CUDA;
   g_launches.fetch_add(1);
   return FH_OK;

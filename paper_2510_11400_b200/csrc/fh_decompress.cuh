@@ -22,6 +22,7 @@ struct DecompressArgs {
   uint8_t* dst;
   unsigned long long* d_status;        // optional
   Scratch* sc;
+  unsigned long long team_stride;      // a prime, at most the number of teams of the grid (see the kernel)
 };
 
 // Reads of a salient / raw payload: offsets below npay come from the plane's slot, the rest from its
@@ -271,8 +272,12 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
     // teams; a salient or raw plane is restored as a whole by the team that draws its first chunk.
     const uint32_t chunk_groups = 8u * TT;
     const uint32_t chunks = (pl.groups + chunk_groups - 1u) / chunk_groups;
-    const uint64_t items = pl.P * chunks, stride = (uint64_t)gridDim.x * kTeams;
-    for (uint64_t item = (uint64_t)blockIdx.x * kTeams + my_team; item < items; item += stride) {
+    // Team t takes items t, t + stride, ...  The stride is a prime (teams beyond it stay idle), so that a
+    // periodic pattern of expensive planes -- every eighth channel outlier-rich, say -- spreads over all
+    // teams instead of landing on the few whose index shares a factor with the period.
+    const uint64_t items = pl.P * chunks, stride = a.team_stride;
+    const uint64_t first = (uint64_t)blockIdx.x * kTeams + my_team;
+    for (uint64_t item = first < stride ? first : items; item < items; item += stride) {
       const uint64_t gp = item / chunks;
       const uint32_t ch = (uint32_t)(item - gp * chunks);
       const uint32_t g0 = ch * chunk_groups, g1 = min(nfull, g0 + chunk_groups);
