@@ -114,7 +114,15 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     pl.sk_cta = pl.plane_bytes > 8192 ? 1u : 0u;
     pl.sk_threads = pl.sk_cta ? (pl.plane_bytes <= 32 * 1024 ? 256u : 512u) : 256u;
     pl.sk_sal_off = (uint32_t)A16(pl.plane_bytes + 32);
-    pl.sk_unit_stride = pl.sk_sal_off + (uint32_t)A16(4 * sal_words);
+    pl.sk_area_words = (uint32_t)(A16(4 * (sal_words + 4)) / 4);
+    {
+      // a few measuring areas per unit, small enough not to cost resident CTAs: 16 KB per CTA unit,
+      // 1 KB per warp unit
+      const size_t budget = pl.sk_cta ? 16 * 1024 : 1024, area = 4 * (size_t)pl.sk_area_words, most = pl.sk_cta ? 8 : 16;
+      const size_t keep = budget / area;
+      pl.sk_keep = (uint32_t)(keep < 1 ? 1 : (keep > most ? most : keep));
+    }
+    pl.sk_unit_stride = pl.sk_sal_off + pl.sk_keep * 4 * pl.sk_area_words;
     pl.sk_pre_off = (pl.sk_cta ? 1u : pl.sk_threads / 32u) * pl.sk_unit_stride;
     pl.sk_total = pl.sk_pre_off + 4u * fh::kMaxChunks;
     if (pl.mode != FH_SALIENT_OFF && pl.sk_total > kSmemLimit) return FH_ERR_UNSUPPORTED;

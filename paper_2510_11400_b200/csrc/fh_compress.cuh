@@ -1109,23 +1109,32 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
   const uint32_t units = gridDim.x * upc;
   const Team t = unit_cta ? make_team(blockDim.x, s_red) : make_warp_team(s_red);
   uint8_t* ubuf = smem + (unit_cta ? 0u : warp * pl.sk_unit_stride);
-  uint32_t* sal = reinterpret_cast<uint32_t*>(ubuf + pl.sk_sal_off);
+  // measuring areas of the unit: the n-th entry it takes uses area min(n, keep - 1); an area starts with
+  // the four sizes of SalientInfo, the measuring scratch follows
+  uint32_t* areas = reinterpret_cast<uint32_t*>(ubuf + pl.sk_sal_off);
+  const uint32_t keep = pl.sk_keep, area_words = pl.sk_area_words;
   uint32_t* pre = reinterpret_cast<uint32_t*>(smem + pl.sk_pre_off);
   const uint4* table = reinterpret_cast<const uint4*>(d.dst + 64);
   const uint32_t raw_units = ovf_units(pl, (uint32_t)pl.plane_bytes);
   __syncthreads();
 
   // ---- measuring phase
-  uint32_t kept = 0xFFFFFFFFu;  // the list entry whose plane and measuring scratch are still in the buffer
+  uint32_t taken = 0;  // entries this unit has measured; the plane of the last one stays in the buffer
   const uint8_t* plane = ubuf;
   SalientInfo info;
   info.nnz_s = info.n_dense = info.n_out_d = info.size = 0;
-  for (uint32_t i = unit; i < count; i += units) {
-    if (kept != 0xFFFFFFFFu) team_sync(t);  // the buffer is reused
+  for (uint32_t i = unit; i < count; i += units, ++taken) {
+    if (taken) team_sync(t);  // the buffer is reused
     const uint32_t p = a.worklist[i];
     plane = fetch_plane(t, pl, a.src, p, ubuf);
-    info = salient_measure<DT>(t, s_pl, plane, sal);
-    kept = i;
+    uint32_t* area = areas + min(taken, keep - 1u) * area_words;
+    info = salient_measure<DT>(t, s_pl, plane, area + 4);
+    if (t.lane == 0) {
+      area[0] = info.nnz_s;
+      area[1] = info.n_dense;
+      area[2] = info.n_out_d;
+      area[3] = info.size;
+    }
     const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
     const uint32_t my_units = ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
     if (t.lane == 0) {
@@ -1197,14 +1206,26 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
       }
     }
     __syncthreads();
-    if (unit < count) {
-      for (uint32_t i = unit + ((count - 1u - unit) / units) * units;; i -= units) {
+    if (taken) {
+      // last entry first: its plane is still in the buffer.  Entries whose area was not reused keep their
+      // measuring results; the others are measured again.
+      team_sync(t);
+      for (uint32_t n = taken; n-- > 0;) {
+        const uint32_t i = unit + n * units;
         const uint32_t p = a.worklist[i];
-        if (i != kept) {
-          team_sync(t);  // the buffer is reused
+        uint32_t* area = areas + min(n, keep - 1u) * area_words;
+        if (n + 1u != taken) {
           plane = fetch_plane(t, pl, a.src, p, ubuf);
-          info = salient_measure<DT>(t, s_pl, plane, sal);
+          if (n >= keep - 1u) {
+            info = salient_measure<DT>(t, s_pl, plane, area + 4);
+          } else {
+            info.nnz_s = area[0];
+            info.n_dense = area[1];
+            info.n_out_d = area[2];
+            info.size = area[3];
+          }
         }
+        const uint32_t* sal = area + 4;
         const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
         const uint32_t my_units = ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
         // overflow units of the listed planes before p in its chunk (every warp of the unit computes them)
@@ -1234,7 +1255,7 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
           else salient_write<DT>(t, s_pl, plane, info, sal, out);
           if (t.lane == 0) *reinterpret_cast<uint32_t*>(d.dst + 64 + 16ull * p) = my_units ? (uint32_t)off16 : 0u;
         }
-        if (i < units + unit) break;  // that was the unit's first entry
+        team_sync(t);  // the buffer is reused
       }
     }
   }

@@ -54,7 +54,9 @@ struct Plan {
   // block-wise kernels: a unit (one warp, or the whole CTA for large planes) holds one plane
   uint32_t sk_cta;          // 1: the unit is the CTA
   uint32_t sk_threads;      // CTA size
-  uint32_t sk_sal_off;      // offset of the unit's measuring scratch behind its plane buffer
+  uint32_t sk_sal_off;      // offset of the unit's measuring areas behind its plane buffer
+  uint32_t sk_keep;         // measuring areas per unit: results of that many planes survive until they are written
+  uint32_t sk_area_words;   // words per area: 4 (sizes) + sal_words
   uint32_t sk_unit_stride;  // bytes of shared memory per unit
   uint32_t sk_pre_off;      // offset of the chunk prefix array (kMaxChunks words)
   uint32_t sk_total;
