@@ -370,8 +370,20 @@ int launch_blockwise(const Plan& pl, const fh::CompressArgs& a, cudaStream_t str
   int g = 0;
   int rc = grid_for(fh::blockwise_kernel<DT>, pl.sk_total, 0x7FFFFFFFu, &g, (int)pl.sk_threads);
   if (rc != FH_OK) return rc;
-  if (launch_dependent(fh::blockwise_kernel<DT>, g, (int)pl.sk_threads, pl.sk_total, stream, pl, a) != cudaSuccess)
-    return FH_ERR_CUDA;
+  // A cooperative launch, and not one that may overlap its predecessor: CTAs that became resident beside
+  // the draining streaming kernel left some SMs unable to take their full share later, and the barrier
+  // then waited for CTAs that could not start.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)g);
+  cfg.blockDim = dim3(pl.sk_threads);
+  cfg.dynamicSmemBytes = pl.sk_total;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, fh::blockwise_kernel<DT>, pl, a) != cudaSuccess) return FH_ERR_CUDA;
   g_launches.fetch_add(1);
   return FH_OK;
 }

@@ -1048,9 +1048,9 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
 // plane's slot, and adds the plane's overflow size to the sum of its chunk (a chunk is a run of
 // 2^chunk_shift consecutive planes; there are at most kMaxChunks chunks).
 //
-// A barrier over the grid separates the phases: all CTAs are resident (the grid is sized to what the
-// device holds at once); the wait is bounded, and a wait that runs out ends the call with the
-// time-out status instead of hanging.
+// A barrier over the grid separates the phases: all CTAs are resident (a cooperative launch of a grid
+// sized to what the device holds at once); the wait is bounded all the same, and a wait that runs out
+// ends the call with the time-out status instead of hanging.
 //
 // Writing phase: every CTA turns the chunk sums into chunk offsets.  A plane's place in the overflow
 // region is its chunk's offset plus the overflow sizes of the listed planes before it in the same
@@ -1094,8 +1094,7 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
   __shared__ uint32_t s_ok;
 
   const uint32_t tid = threadIdx.x, lane32 = tid & 31u, warp = tid >> 5;
-  dep_trigger();
-  dep_wait();  // the streaming kernel has completed: its list, table and counters are visible
+  // (launched in plain stream order: the streaming kernel has completed, its list, table and counters are visible)
   const Dest d = make_dest(pl, a);
   const uint32_t count = (uint32_t)ld_relaxed(&a.sc->wl_count);
   if (count == 0) {  // nothing listed: the container lacks only its header
@@ -1171,6 +1170,9 @@ __global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const Com
     s_ok = ok;
   }
   __syncthreads();
+  // Only now may the next kernel on the stream become resident: before the barrier its CTAs could take
+  // the place of CTAs of this grid that have not started yet, and the barrier would never complete.
+  dep_trigger();
 
   // ---- writing phase
   if (s_ok && d.fits && (unit_cta ? blockIdx.x : blockIdx.x * upc) < count) {  // CTAs without entries are done

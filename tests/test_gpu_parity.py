@@ -311,3 +311,44 @@ def test_launch_counter_counts_our_kernels():
     st, packed, total = gpu_compress(raw, (2, 4, 8, 8), synth.F32, bits=2, salient_mode=api.FH_SALIENT_OFF)
     api.decompress_tensor(packed, total, (2, 4, 8, 8), synth.F32)
     assert api.kernel_launches() == before + 5
+
+
+def test_back_to_back_calls_without_host_synchronisation():
+    """Several tensors with outlier-rich planes, compressed and restored back to back on one stream for
+    three rounds with no host synchronisation in between: kernels of consecutive calls overlap at their
+    edges, and the block-wise kernel's barrier over its grid must still complete (every status word 0);
+    the last round is compared with the oracle."""
+    import torch
+    specs = [synth.TensorSpec("a", (8, 96, 112, 112), synth.BF16, "laplace_ch", 21),
+             synth.TensorSpec("b", (16, 144, 56, 56), synth.BF16, "laplace_ch", 22),
+             synth.TensorSpec("c", (32, 64, 14, 14), synth.F32, "spiky_relu", 23)]
+    ts = []
+    for i, sp in enumerate(specs):
+        raw = synth.make(sp)
+        d = api.desc(sp.shape, sp.dtype)
+        cap = api.compressed_bytes(d, api.default_params(bits=8), 1)
+        x = to_dev(raw)
+        ts.append(dict(sp=sp, raw=raw, d=d, x=x, cap=cap, dst=torch.empty(cap, dtype=torch.uint8, device="cuda"),
+                       out=torch.empty_like(x)))
+    words = []
+    for rnd in range(3):
+        for bits in (2, 4, 8):
+            p = api.default_params(bits=bits)
+            o2 = [torch.zeros(2, dtype=torch.int64, device="cuda") for _ in ts]
+            st = [torch.zeros(1, dtype=torch.int64, device="cuda") for _ in ts]
+            words.append((o2, st))
+            for t, o in zip(ts, o2):
+                assert api.fh_compress(t["d"], p, t["x"], t["dst"], o, capacity=t["cap"]) == api.FH_OK
+            for t, q in zip(reversed(ts), reversed(st)):
+                assert api.fh_decompress(t["dst"], t["cap"], t["d"], t["out"], q) == api.FH_OK
+    torch.cuda.synchronize()
+    for o2, st in words:
+        assert [int(o[1]) for o in o2] == [0] * len(ts)
+        assert [int(q[0]) for q in st] == [0] * len(ts)
+    for t in ts:   # the last round ran at 8 bits
+        st_o, buf_o, total_o, d = oracle_compress(t["raw"], t["sp"].shape, t["sp"].dtype, bits=8)
+        assert st_o == fho.OK
+        assert np.array_equal(t["dst"][:total_o].cpu().numpy(), buf_o)
+        _, out_o = fho.decompress(buf_o, d)
+        got = t["out"].cpu().numpy()
+        check_same_values(got.view(np.uint16) if t["sp"].dtype == synth.BF16 else got, out_o, t["sp"].dtype)
