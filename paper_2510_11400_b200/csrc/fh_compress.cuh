@@ -519,13 +519,20 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
 #define FH_STORE_CODES(BITS)                                                                                  \
   {                                                                                                           \
     constexpr uint32_t bias = kMagicBits * (1u + (1u << (BITS)) + (1u << (2 * (BITS))) + (1u << (3 * (BITS)))); \
+    const f32x2 nlo2 = pack2(-lo, -lo), inv2 = pack2(inv, inv), mag2 = pack2(kMagicF, kMagicF);                 \
     _Pragma("unroll") for (int k = 0; k < G; ++k) {                                                           \
       const uint32_t g = lane + (uint32_t)(k * TT);                                                           \
-      uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));                       \
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF)) << (BITS);                     \
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF)) << (2 * (BITS));               \
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF)) << (3 * (BITS));               \
-      word -= bias;                                                                                           \
+      uint32_t w0, w1, w2, w3;                                                                                \
+      if (DT == kBF16) { /* packed pairs; x - lo is x + (-lo): the same rounding */                          \
+        unpack2u(fma2(add2(pack2(x[k][0], x[k][1]), nlo2), inv2, mag2), w0, w1);                              \
+        unpack2u(fma2(add2(pack2(x[k][2], x[k][3]), nlo2), inv2, mag2), w2, w3);                              \
+      } else {                                                                                                \
+        w0 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));                                \
+        w1 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF));                                \
+        w2 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF));                                \
+        w3 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF));                                \
+      }                                                                                                       \
+      uint32_t word = w0 + (w1 << (BITS)) + (w2 << (2 * (BITS))) + (w3 << (3 * (BITS))) - bias;               \
       if (FULL || g < groups) {                                                                               \
         if (!VEC) { /* ragged last group: elements past the plane carry no code */                            \
           const uint32_t valid = min(4u, pl.HW - g * 4u);                                                     \
@@ -611,7 +618,7 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
     const SigmaScale sc = sigma_scale(lo, hi);
     uint32_t as = 0, aq = 0;
 #pragma unroll
-    for (int k = 0; k < G; ++k) sigma_addends4(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
+    for (int k = 0; k < G; ++k) sigma_addends4<DT == kBF16>(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
     long long Is, Iq;
     team_sum2(team, (int32_t)(as - (uint32_t)G * kMagicBits), (int32_t)(aq - (uint32_t)G * kMagicBits), Is, Iq, rp);
     float tlo, thi;
@@ -852,14 +859,21 @@ __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, floa
 #define FH_CTA_STORE_CODES(BITS)                                                                              \
   {                                                                                                           \
     constexpr uint32_t bias = kMagicBits * (1u + (1u << (BITS)) + (1u << (2 * (BITS))) + (1u << (3 * (BITS)))); \
+    const f32x2 nlo2 = pack2(-lo, -lo), inv2 = pack2(inv, inv), mag2 = pack2(kMagicF, kMagicF);                 \
     _Pragma("unroll 2") for (uint32_t g = tid; g < groups; g += NT) {                                         \
       float v[4];                                                                                             \
       lds_group<DT>(plane, g, v);                                                                             \
-      uint32_t word = __float_as_uint(__fmaf_rn(__fsub_rn(v[0], lo), inv, kMagicF));                          \
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(v[1], lo), inv, kMagicF)) << (BITS);                        \
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(v[2], lo), inv, kMagicF)) << (2 * (BITS));                  \
-      word += __float_as_uint(__fmaf_rn(__fsub_rn(v[3], lo), inv, kMagicF)) << (3 * (BITS));                  \
-      word -= bias;                                                                                           \
+      uint32_t w0, w1, w2, w3;                                                                                \
+      if (DT == kBF16) {                                                                                      \
+        unpack2u(fma2(add2(pack2(v[0], v[1]), nlo2), inv2, mag2), w0, w1);                                    \
+        unpack2u(fma2(add2(pack2(v[2], v[3]), nlo2), inv2, mag2), w2, w3);                                    \
+      } else {                                                                                                \
+        w0 = __float_as_uint(__fmaf_rn(__fsub_rn(v[0], lo), inv, kMagicF));                                   \
+        w1 = __float_as_uint(__fmaf_rn(__fsub_rn(v[1], lo), inv, kMagicF));                                   \
+        w2 = __float_as_uint(__fmaf_rn(__fsub_rn(v[2], lo), inv, kMagicF));                                   \
+        w3 = __float_as_uint(__fmaf_rn(__fsub_rn(v[3], lo), inv, kMagicF));                                   \
+      }                                                                                                       \
+      uint32_t word = w0 + (w1 << (BITS)) + (w2 << (2 * (BITS))) + (w3 << (3 * (BITS))) - bias;               \
       if ((BITS) == 2) slot[g] = (uint8_t)word;                                                               \
       else if ((BITS) == 4) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;                            \
       else reinterpret_cast<uint32_t*>(slot)[g] = word;                                                       \
@@ -961,7 +975,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
       for (uint32_t g = tid; g < groups; g += NT) {
         float v[4];
         lds_group<DT>(plane, g, v);
-        sigma_addends4(v[0], v[1], v[2], v[3], sc, as, aq);
+        sigma_addends4<DT == kBF16>(v[0], v[1], v[2], v[3], sc, as, aq);
         ++ng;
       }
       long long Is, Iq;

@@ -224,6 +224,31 @@ __device__ __forceinline__ void load_group(const uint8_t* plane, uint32_t g, uin
   }
 }
 
+// ---- packed fp32 pairs (sm_100: one instruction, two independent IEEE round-to-nearest results) ----
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ void unpack2u(f32x2 v, uint32_t& a, uint32_t& b) { asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v)); }
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+
 // Fixed-point moments of a plane (three-sigma rule): scale factors from the largest magnitude A.
 struct SigmaScale {
   float cs, cq;    // 2^ks, 2^kq
@@ -249,14 +274,30 @@ __device__ __forceinline__ void sigma_addends(const float v[4], const SigmaScale
   as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
   aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
 }
+// PACKED: the same arithmetic with packed pairs -- (v0, v2) and (v1, v3) give both halves of every step at
+// once.  Used for bf16 input, whose unpacked values can be put in any registers and whose kernels are bound
+// by instruction issue; on fp32 input the repacking costs more than it saves.
+template <bool PACKED>
 __device__ __forceinline__ void sigma_addends4(float v0, float v1, float v2, float v3, const SigmaScale& sc,
                                                uint32_t& as, uint32_t& aq) {
-  const float sg = __fadd_rn(__fadd_rn(v0, v1), __fadd_rn(v2, v3));
-  const float q01 = __fmaf_rn(v1, v1, __fmul_rn(v0, v0));
-  const float q23 = __fmaf_rn(v3, v3, __fmul_rn(v2, v2));
-  const float qg = __fadd_rn(q01, q23);
-  as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
-  aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
+  if (PACKED) {
+    const f32x2 ev = pack2(v0, v2), od = pack2(v1, v3);
+    float s01, s23, q01, q23;
+    unpack2(add2(ev, od), s01, s23);                 // v0 + v1, v2 + v3
+    unpack2(fma2(od, od, mul2(ev, ev)), q01, q23);   // fma(v1, v1, v0 * v0), fma(v3, v3, v2 * v2)
+    const f32x2 fixed = fma2(pack2(__fadd_rn(s01, s23), __fadd_rn(q01, q23)), pack2(sc.cs, sc.cq), pack2(kMagicF, kMagicF));
+    uint32_t is, iq;
+    unpack2u(fixed, is, iq);
+    as += is;
+    aq += iq;
+  } else {
+    const float sg = __fadd_rn(__fadd_rn(v0, v1), __fadd_rn(v2, v3));
+    const float q01 = __fmaf_rn(v1, v1, __fmul_rn(v0, v0));
+    const float q23 = __fmaf_rn(v3, v3, __fmul_rn(v2, v2));
+    const float qg = __fadd_rn(q01, q23);
+    as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
+    aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
+  }
 }
 // Thresholds mu +- 3 sigma from the exact integer sums.
 template <typename I>
