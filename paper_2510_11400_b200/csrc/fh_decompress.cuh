@@ -156,29 +156,6 @@ __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const
   return ok;
 }
 
-// Normal plane, whole groups, vector stores.  TT lanes; lane handles groups lane, lane + TT, ...
-#define FH_DECODE_NORMAL(BITS)                                                                             \
-  {                                                                                                        \
-    constexpr uint32_t L = (1u << (BITS)) - 1u;                                                            \
-    _Pragma("unroll 4") for (uint32_t g = g0 + lane; g < g1; g += TT) {                                    \
-      uint32_t word;                                                                                       \
-      if ((BITS) == 2) word = __ldg(slot + g);                                                             \
-      else if ((BITS) == 4) word = __ldg(reinterpret_cast<const uint16_t*>(slot) + g);                     \
-      else word = __ldg(reinterpret_cast<const uint32_t*>(slot) + g);                                      \
-      const float v0 = dequant(word & L, scale, lo), v1 = dequant((word >> (BITS)) & L, scale, lo);        \
-      const float v2 = dequant((word >> (2 * (BITS))) & L, scale, lo);                                     \
-      const float v3 = dequant((word >> (3 * (BITS))) & L, scale, lo);                                     \
-      if (DT == kF32) {                                                                                    \
-        reinterpret_cast<float4*>(out)[g] = make_float4(v0, v1, v2, v3);                                   \
-      } else {                                                                                             \
-        uint2 w;                                                                                           \
-        w.x = f32_to_bf16_bits(v0) | (f32_to_bf16_bits(v1) << 16);                                         \
-        w.y = f32_to_bf16_bits(v2) | (f32_to_bf16_bits(v3) << 16);                                         \
-        reinterpret_cast<uint2*>(out)[g] = w;                                                              \
-      }                                                                                                    \
-    }                                                                                                      \
-  }
-
 // Four restored values of one group leave as one 16-byte (fp32) or 8-byte (bf16) store.
 template <int DT>
 __device__ __forceinline__ void store_group(uint8_t* out, uint32_t g, float v0, float v1, float v2, float v3) {
@@ -216,6 +193,32 @@ __device__ __forceinline__ void decode_chunk32(const uint32_t (&w)[8], uint32_t 
     if (g < g1)
       store_group<DT>(out, g, dequant(word & L, scale, lo), dequant((word >> BITS) & L, scale, lo),
                       dequant((word >> (2 * BITS)) & L, scale, lo), dequant((word >> (3 * BITS)) & L, scale, lo));
+  }
+}
+
+// Normal plane, sub-warp team of TT lanes (planes of at most 8 * TT groups, one chunk).  cw[k] holds the
+// code word of group lane + k * TT, requested before the table entry was known.  Whole groups of planes
+// that start on a vector boundary leave as one store; everything else (planes that do not, the ragged
+// last group) as element stores.
+template <int DT, int BITS, int TT>
+__device__ __forceinline__ void decode_small(const uint32_t (&cw)[8], uint32_t lane, uint32_t groups, uint32_t nfull,
+                                             uint32_t HW, float scale, float lo, uint8_t* out) {
+  constexpr uint32_t L = (1u << BITS) - 1u;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t g = lane + (uint32_t)k * TT, word = cw[k];
+    if (g >= groups) break;
+    const float v0 = dequant(word & L, scale, lo), v1 = dequant((word >> BITS) & L, scale, lo);
+    const float v2 = dequant((word >> (2 * BITS)) & L, scale, lo), v3 = dequant((word >> (3 * BITS)) & L, scale, lo);
+    if (g < nfull) {
+      store_group<DT>(out, g, v0, v1, v2, v3);
+    } else {
+      const uint32_t i = 4u * g;
+      store_elem<DT>(out, i, v0);
+      if (i + 1u < HW) store_elem<DT>(out, i + 1u, v1);
+      if (i + 2u < HW) store_elem<DT>(out, i + 2u, v2);
+      if (i + 3u < HW) store_elem<DT>(out, i + 3u, v3);
+    }
   }
 }
 
@@ -292,6 +295,18 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
           const uint32_t i = w0 + (uint32_t)j * 32u + lane;
           cw[j] = ((uint32_t)j < per && i < nwords) ? __ldg(s32 + i) : 0u;
         }
+      } else {  // sub-warp teams: one code word (1, 2 or 4 bytes) per group, the plane is one chunk
+        const uint8_t* sl = src + slots_off + gp * npay;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const uint32_t g = lane + (uint32_t)k * TT;
+          uint32_t w = 0;
+          if (g < pl.groups)
+            w = bits == 2u ? (uint32_t)__ldg(sl + g)
+                           : (bits == 4u ? (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(sl) + g)
+                                         : __ldg(reinterpret_cast<const uint32_t*>(sl) + g));
+          cw[k] = w;
+        }
       }
       const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + gp);
       const unsigned long long off = (unsigned long long)e.x * 16ull;
@@ -305,10 +320,10 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
           if (bits == 2u) decode_chunk32<DT, 2>(cw, lane, g0, g1, scale, lo, out);
           else if (bits == 4u) decode_chunk32<DT, 4>(cw, lane, g0, g1, scale, lo, out);
           else decode_chunk32<DT, 8>(cw, lane, g0, g1, scale, lo, out);
-        } else if (bits == 2u) FH_DECODE_NORMAL(2)
-        else if (bits == 4u) FH_DECODE_NORMAL(4)
-        else FH_DECODE_NORMAL(8)
-        if (ch == chunks - 1u && nfull * 4u < pl.HW) {  // ragged or unaligned rest: element stores
+        } else if (bits == 2u) decode_small<DT, 2, TT>(cw, lane, pl.groups, nfull, pl.HW, scale, lo, out);
+        else if (bits == 4u) decode_small<DT, 4, TT>(cw, lane, pl.groups, nfull, pl.HW, scale, lo, out);
+        else decode_small<DT, 8, TT>(cw, lane, pl.groups, nfull, pl.HW, scale, lo, out);
+        if (TT == 32 && ch == chunks - 1u && nfull * 4u < pl.HW) {  // ragged or unaligned rest: element stores
           const uint32_t L = (1u << bits) - 1u;
           for (uint32_t i = nfull * 4u + lane; i < pl.HW; i += TT) {
             const uint32_t bit = i * bits;
