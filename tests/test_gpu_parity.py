@@ -352,3 +352,23 @@ def test_back_to_back_calls_without_host_synchronisation():
         _, out_o = fho.decompress(buf_o, d)
         got = t["out"].cpu().numpy()
         check_same_values(got.view(np.uint16) if t["sp"].dtype == synth.BF16 else got, out_o, t["sp"].dtype)
+
+
+@pytest.mark.parametrize("which", ["c2_112x112_relu", "c2_28x28_normal", "c2_7x7_relu", "c3_56x56_bf16"])
+def test_full_size_tensors_of_the_bench_workloads(which):
+    """Tensors at the sizes the benchmark times (ResNet-18-shaped batch 64, MobileNetV2-shaped batch 128),
+    through the same entry points and launch configuration, compared byte for byte with the oracle."""
+    if which == "c2_112x112_relu":
+        spec = synth.config2(64)[0]
+    elif which == "c2_28x28_normal":
+        spec = synth.config2(64)[5]
+    elif which == "c2_7x7_relu":
+        spec = synth.config2(64)[16]
+    else:
+        spec = synth.config3(128)[1]
+    buf = full_parity(spec, bits=2)
+    P = spec.shape[0] * spec.shape[1]
+    t = hp.table(buf, P)
+    if which == "c3_56x56_bf16":   # every eighth channel carries the +-50 outliers: those planes are not normal
+        ch = np.arange(P) % spec.shape[1]
+        assert (t["cls"][ch % 8 == 0] != fho.NORMAL).all() and (t["cls"][ch % 8 != 0] == fho.NORMAL).mean() > 0.99
