@@ -372,3 +372,51 @@ def test_full_size_tensors_of_the_bench_workloads(which):
     if which == "c3_56x56_bf16":   # every eighth channel carries the +-50 outliers: those planes are not normal
         ch = np.arange(P) % spec.shape[1]
         assert (t["cls"][ch % 8 == 0] != fho.NORMAL).all() and (t["cls"][ch % 8 != 0] == fho.NORMAL).mean() > 0.99
+
+
+def test_tensor_beyond_4_gib_on_sampled_planes():
+    """A tensor a little over 4 GiB (byte offsets past 2^32, 2^30 elements): the oracle cannot take it whole
+    in reasonable time, but planes are coded independently, so sampled planes -- the first, the last 64
+    (which lie beyond 2^32 bytes) and a seeded random hundred -- are compared with the oracle run on just
+    those planes: table entry, slot bytes and restored values.  Input: seeded normal draws on the device,
+    ReLU'd; the oracle sees the very bytes copied back."""
+    import torch
+    P = (1 << 20) + 64
+    shape = (P // 64, 64, 32, 32)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(20251011)
+    x = torch.empty(P * 1024, dtype=torch.float32, device="cuda")
+    x.normal_(generator=gen)
+    x.relu_()
+    d = api.desc(shape, api.FH_F32)
+    p = api.default_params(bits=2)
+    st, packed, total = api.compress_tensor(x, shape, api.FH_F32, p)
+    assert st == api.FH_OK
+    hdr = packed[:64].cpu().numpy()
+    assert int(hdr[56:64].view(np.uint64)[0]) == total
+    npay, slots = 256, 64 + 16 * P
+    assert total >= slots + P * npay
+    rng = np.random.default_rng(7)
+    idx = np.unique(np.concatenate([np.arange(4), np.arange(P - 64, P), rng.integers(0, P, 100)]))
+    sample = x.view(P, 1024)[torch.from_numpy(idx).cuda()].cpu().numpy().reshape(-1)
+    st_o, buf_o, total_o, d_o = oracle_compress(sample, (1, len(idx), 32, 32), synth.F32, bits=2)
+    assert st_o == fho.OK
+    to = hp.table(buf_o, len(idx))
+    tab = packed[64:64 + 16 * P].view(torch.int32).view(P, 4)[torch.from_numpy(idx).cuda()].cpu().numpy().view(np.uint32)
+    assert np.array_equal(tab[:, 1] & 3, to["cls"]) and np.array_equal(tab[:, 1] >> 2, to["n_out"])
+    st_d, out = api.decompress_tensor(packed, total, shape, api.FH_F32)
+    assert st_d == api.FH_OK
+    _, out_o = fho.decompress(buf_o, d_o)
+    got = out.view(P, 1024)[torch.from_numpy(idx).cuda()].cpu().numpy().reshape(-1)
+    check_same_values(got, out_o, synth.F32)
+    slots_o = 64 + 16 * len(idx)
+    for k, pl in enumerate(idx):
+        if to["cls"][k] != fho.NORMAL:
+            continue
+        assert tab[k, 0] * 16 == slots + int(pl) * npay
+        assert np.array_equal(tab[k, 2:4], np.stack([to["lo"][k:k + 1].view(np.uint32), to["scale"][k:k + 1].view(np.uint32)], 1)[0])
+        a0 = slots + int(pl) * npay
+        assert np.array_equal(packed[a0:a0 + npay].cpu().numpy(), buf_o[slots_o + k * npay: slots_o + (k + 1) * npay])
+    # every zero of a post-ReLU plane comes back as zero (normal planes have lo = 0; the block-wise path keeps zeros)
+    probe = torch.from_numpy(idx[:32]).cuda()
+    assert bool(((x.view(P, 1024)[probe] == 0) <= (out.view(P, 1024)[probe] == 0)).all())
