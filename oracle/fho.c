@@ -113,7 +113,7 @@ static int check_args(const fho_desc* d, const fho_params* p) {
   if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FHO_ERR_ARG;
   if (p->block != 8) return FHO_ERR_UNSUPPORTED;
   if (p->dense_bits != 8) return FHO_ERR_UNSUPPORTED;
-  if (p->rounding != 0) return FHO_ERR_UNSUPPORTED;
+  if (p->rounding != 0 && p->rounding != 1) return FHO_ERR_UNSUPPORTED;
   if (!(p->eps >= 1e-30f) || !(p->eps <= 1e30f)) return FHO_ERR_ARG; /* keeps 2*eps and 1/(2*eps) finite */
   return FHO_OK;
 }
@@ -263,6 +263,57 @@ uint32_t fho_quant_code(float x, float lo, float inv, int bits) {
 }
 
 float fho_dequant(uint32_t q, float lo, float scale) { return fmaf((float)q, scale, lo); }
+
+/* ------------------------------------------------------------------------------------------
+ * Random rounding of normal planes (rounding = 1).  The paper is silent on the rounding of its
+ * quantiser; the quantisers it builds on (its Section 2.3 citations) round stochastically so that the
+ * restored value is unbiased.  Here, with 24-bit integers so that nothing depends on floating-point
+ * rounding of a sum:
+ *   t = (x - lo) * inv            (fp32 subtraction, fp32 product; t >= 0)
+ *   n = floor(t),  f = t - n      (exact)
+ *   q = min(n + [ floor(f * 2^24) + r >= 2^24 ], L),   r = a uniform 24-bit integer
+ * so the code goes up with probability floor(f * 2^24) / 2^24 and a position that is already an integer
+ * never moves.
+ *
+ * u comes from the counter-based generator Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw,
+ * "Parallel random numbers: as easy as 1, 2, 3", SC'11): multipliers 0xD2511F53 and 0xCD9E8D57, key
+ * increments 0x9E3779B9 and 0xBB67AE85.  One call per group of four consecutive elements of a plane:
+ *   key     = (seed low word, seed high word)
+ *   counter = (group index within the plane, plane index, tensor_id low word, tensor_id high word)
+ * and element e of the group takes output word e: r = word >> 8.
+ * So the draw of an element depends on (seed, tensor id, element position) and on nothing else.
+ * ------------------------------------------------------------------------------------------ */
+void fho_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+  for (int r = 0; r < 10; ++r) {
+    uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+    uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+    uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+    c0 = n0;
+    c1 = n1;
+    c2 = n2;
+    c3 = n3;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0;
+  out[1] = c1;
+  out[2] = c2;
+  out[3] = c3;
+}
+
+uint32_t fho_quant_code_random(float x, float lo, float inv, int bits, uint32_t word) {
+  uint32_t L = (1u << bits) - 1u;
+  float d = x - lo;
+  float t = d * inv;
+  float nf = floorf(t);
+  float f = t - nf;                               /* exact, 0 <= f < 1 */
+  uint32_t fi = (uint32_t)(f * 16777216.0f);      /* floor(f * 2^24): the scaling is exact */
+  uint32_t up = (fi + (word >> 8)) >> 24;         /* 1 iff fi + r >= 2^24 */
+  uint32_t n = nf >= (float)L ? L : (uint32_t)nf; /* t may exceed L by rounding */
+  uint32_t q = n + up;
+  return q > L ? L : q;
+}
 
 /* Pre-quantisation for dense blocks: k = round_half_even(fp32(x * inv2e)), |k| capped at 2^24. */
 static int32_t dense_k(float x, float inv2e, int* big) {
@@ -419,7 +470,7 @@ static size_t encode_salient(const float* x, const uint8_t* raw, int dtype, int 
 }
 
 static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_params* p,
-                         plane_result* r) {
+                         uint64_t plane_index, uint64_t tensor_id, plane_result* r) {
   size_t hw = (size_t)H * W, e = esize(dtype);
   float* x = (float*)malloc(hw * sizeof(float));
   for (size_t i = 0; i < hw; ++i)
@@ -472,7 +523,15 @@ static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_
     r->bytes = a16(size);
     r->payload = (uint8_t*)calloc(r->bytes, 1);
     for (size_t i = 0; i < hw; ++i) {
-      uint32_t qv = fho_quant_code(x[i], lo, inv, p->bits);
+      uint32_t qv;
+      if (p->rounding == 1) {
+        uint32_t ctr[4] = {(uint32_t)(i / 4), (uint32_t)plane_index, (uint32_t)tensor_id, (uint32_t)(tensor_id >> 32)};
+        uint32_t key[2] = {(uint32_t)p->seed, (uint32_t)(p->seed >> 32)}, rnd[4];
+        fho_philox4x32_10(ctr, key, rnd);
+        qv = fho_quant_code_random(x[i], lo, inv, p->bits, rnd[i % 4]);
+      } else {
+        qv = fho_quant_code(x[i], lo, inv, p->bits);
+      }
       size_t bit = i * (size_t)p->bits;
       uint32_t wv = get_u32(r->payload + 4 * (bit / 32));
       put_u32(r->payload + 4 * (bit / 32), wv | (qv << (bit % 32)));
@@ -498,7 +557,7 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
 #pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)
 #endif
   for (int64_t pl = 0; pl < (int64_t)P; ++pl)
-    encode_plane((const uint8_t*)src + (size_t)pl * hw * e, d->dtype, d->h, d->w, p, &res[pl]);
+    encode_plane((const uint8_t*)src + (size_t)pl * hw * e, d->dtype, d->h, d->w, p, (uint64_t)pl, d->tensor_id, &res[pl]);
   const size_t npay = a16(normal_payload(hw, p->bits));
   size_t total = 64 + 16 * P + P * npay;
   uint32_t n_sal = 0, n_raw = 0;

@@ -82,6 +82,10 @@ def lib():
         L.fho_quant_code.argtypes = [C.c_float, C.c_float, C.c_float, C.c_int]
         L.fho_dequant.restype = C.c_float
         L.fho_dequant.argtypes = [C.c_uint32, C.c_float, C.c_float]
+        L.fho_philox4x32_10.restype = None
+        L.fho_philox4x32_10.argtypes = [C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
+        L.fho_quant_code_random.restype = C.c_uint32
+        L.fho_quant_code_random.argtypes = [C.c_float, C.c_float, C.c_float, C.c_int, C.c_uint32]
         L.fho_set_threads.argtypes = [C.c_int]
         L.fho_max_threads.restype = C.c_int
         L.fho_get_threads.restype = C.c_int
@@ -149,6 +153,18 @@ def quant_params(lo: float, hi: float, bits: int):
 
 def quant_code(x: float, lo: float, inv: float, bits: int) -> int:
     return int(lib().fho_quant_code(x, lo, inv, bits))
+
+
+def philox4x32_10(ctr, key):
+    c = (C.c_uint32 * 4)(*ctr)
+    k = (C.c_uint32 * 2)(*key)
+    o = (C.c_uint32 * 4)()
+    lib().fho_philox4x32_10(c, k, o)
+    return [int(v) for v in o]
+
+
+def quant_code_random(x: float, lo: float, inv: float, bits: int, word: int) -> int:
+    return int(lib().fho_quant_code_random(x, lo, inv, bits, word))
 
 
 def dequant(q: int, lo: float, scale: float) -> float:
