@@ -228,7 +228,7 @@ def run_ours(args, specs, wl_desc):
 
     dev = torch.device("cuda", local)
     mode = {"auto": api.FH_SALIENT_AUTO, "off": api.FH_SALIENT_OFF, "all": api.FH_SALIENT_ALL}[args.mode]
-    params = {b: api.default_params(bits=b, salient_mode=mode) for b in BITS}
+    params = {b: api.default_params(bits=b, salient_mode=mode, rounding=args.rounding, seed=2510_11400) for b in BITS}
     tensors = []
     for i, s in enumerate(specs):
         raw = synth.make(s)
@@ -351,6 +351,7 @@ def run_ours(args, specs, wl_desc):
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32" if specs[0].dtype == synth.F32 else "bf16", "data": "synthetic",
             "config": {"workload": wl_desc, "bits": list(BITS), "salient_mode": args.mode.upper(),
+                       "rounding": "nearest-even" if args.rounding == 0 else "random (Philox-4x32-10)",
                        "tensors": len(tensors), "dense_bytes_per_pass": dense_bytes,
                        "packed_bytes": {str(b): packed_bytes[b] for b in BITS},
                        "l2": "inputs larger than L2: every pass streams the whole dense set",
@@ -387,6 +388,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18_b64")
     ap.add_argument("--mode", default="auto", choices=["auto", "off", "all"])
+    ap.add_argument("--rounding", type=int, default=0, choices=[0, 1],
+                    help="1: random rounding of normal planes (runs on the general-purpose kernel)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     args = ap.parse_args()

@@ -95,8 +95,9 @@ typedef struct {
   int32_t tau_num, tau_den; /* block is dense iff nnz*tau_den >= tau_num*n*n               [1/4]   */
   float eps;                /* absolute error bound of dense blocks, 1e-30 <= eps <= 1e30  [1/16]  */
   int32_t dense_bits;       /* residual code width; 8 only                                 [8]     */
-  int32_t rounding;         /* 0 = round half to even; nothing else yet                    [0]     */
-  uint64_t seed;            /* reserved for random rounding                                [0]     */
+  int32_t rounding;         /* 0 = round half to even; 1 = random rounding of normal planes
+                               (see fh_compress)                                           [0]     */
+  uint64_t seed;            /* key of the random draws (rounding = 1)                      [0]     */
 } fh_params;
 
 typedef enum { FH_KEEP = 0, FH_COMPRESS = 1, FH_EVICT = 2 } fh_action;
@@ -149,6 +150,15 @@ size_t fh_compressed_bytes(const fh_tensor_desc* desc, const fh_params* params, 
  * h*w*esize <= 200 KB; larger planes return FH_ERR_UNSUPPORTED.  The container is limited to
  * 64 GiB (32-bit offsets in units of 16 bytes).
  * The packed bytes are a pure function of the input and the parameters.
+ *
+ * rounding = 1 (the paper does not say how its quantiser rounds; the quantisers it builds on round at
+ * random so that the restored value is unbiased): the code of an element of a normal plane is
+ * floor(t) + [floor(frac(t) * 2^24) + r >= 2^24] with t = (x - lo) * inv in fp32 and r a uniform 24-bit
+ * integer, the top 24 bits of word (i mod 4) of Philox-4x32-10 with key (seed low, seed high) and counter
+ * (i / 4, plane index, tensor_id low, tensor_id high), i the element's index within its plane.  The draw
+ * thus depends on (seed, tensor id, element position) only and results are reproducible.  Dense-block codes
+ * keep round-to-nearest (their error bound needs it).  This mode runs on the general-purpose kernel and is
+ * slower than rounding = 0.
  */
 int fh_compress(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                 size_t dst_capacity, uint64_t* d_out2, void* stream);

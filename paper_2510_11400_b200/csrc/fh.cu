@@ -45,7 +45,7 @@ int check_params(const fh_params* p) {
   if (p->salient_mode < 0 || p->salient_mode > 2) return FH_ERR_ARG;
   if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FH_ERR_ARG;
   if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FH_ERR_ARG;
-  if (p->block != 8 || p->dense_bits != 8 || p->rounding != 0) return FH_ERR_UNSUPPORTED;
+  if (p->block != 8 || p->dense_bits != 8 || (p->rounding != 0 && p->rounding != 1)) return FH_ERR_UNSUPPORTED;
   if (!(p->eps >= 1e-30f) || !(p->eps <= 1e30f)) return FH_ERR_ARG;
   return FH_OK;
 }
@@ -90,6 +90,8 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   pl.inv_hw = 1.0 / (double)hw;
   pl.bits = p ? p->bits : 2;
   pl.mode = p ? p->salient_mode : 0;
+  pl.rounding = p ? p->rounding : 0;
+  pl.seed = p ? p->seed : 0;
   pl.rho_num = p ? p->rho_num : 1;
   pl.rho_den = p ? p->rho_den : 32;
   pl.tau_num = p ? p->tau_num : 1;
@@ -131,7 +133,8 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   Variant v;
   // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
   const bool whole16 = pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0;
-  if (compress && (pl.groups <= 256 || whole16)) {
+  // (random rounding runs on the generic kernel)
+  if (compress && pl.rounding == 0 && (pl.groups <= 256 || whole16)) {
     v.fast = true;
     if (pl.groups <= 256) {
       uint32_t t = pow2_ceil((pl.groups + 7) / 8);

@@ -285,7 +285,7 @@ __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, 
     uint4* hd = reinterpret_cast<uint4*>(d.dst);
     // a failed container must not pass for a valid one: no magic
     hd[0] = make_uint4(code == kErrNone ? kMagic : 0u, 1u | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24), pl.N, pl.C);
-    hd[1] = make_uint4((uint32_t)pl.H, (uint32_t)pl.W, 8u | (8u << 8) | (0u << 16) | ((uint32_t)pl.mode << 24),
+    hd[1] = make_uint4((uint32_t)pl.H, (uint32_t)pl.W, 8u | (8u << 8) | ((uint32_t)pl.rounding << 16) | ((uint32_t)pl.mode << 24),
                        pl.rho_num | (pl.rho_den << 16));
     hd[2] = make_uint4(pl.tau_num | (pl.tau_den << 16), __float_as_uint(pl.eps), (uint32_t)nsal, (uint32_t)nraw);
     hd[3] = make_uint4((uint32_t)pl.tensor_id, (uint32_t)(pl.tensor_id >> 32), (uint32_t)total, (uint32_t)(total >> 32));
@@ -462,9 +462,13 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
           if (g < groups) {
             float v[4];
             load_group<DT>(plane, g, HW, vec, v);
+            uint32_t rnd[4] = {0, 0, 0, 0};
+            if (pl.rounding)  // one generator call per group: counter = (group, plane, tensor id), key = seed
+              philox4x32_10(g, (uint32_t)(p0 + lp), (uint32_t)pl.tensor_id, (uint32_t)(pl.tensor_id >> 32),
+                            (uint32_t)pl.seed, (uint32_t)(pl.seed >> 32), rnd);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              uint32_t q = quant_code(v[k], lo, inv, L);
+              uint32_t q = pl.rounding ? quant_code_random(v[k], lo, inv, L, rnd[k]) : quant_code(v[k], lo, inv, L);
               if (g * 4u + k >= HW) q = 0;
               word |= q << (k * BITS);
             }

@@ -36,6 +36,8 @@ struct Plan {
   uint64_t dense_bytes;  // P * plane_bytes
   double inv_hw;         // 1 / HW in fp64
   int32_t bits, mode;
+  int32_t rounding;      // 0: round half to even; 1: random rounding (Philox draws)
+  uint64_t seed;
   uint32_t rho_num, rho_den, tau_num, tau_den;
   float eps;
   uint64_t tensor_id;
@@ -329,6 +331,38 @@ __device__ __forceinline__ void quant_params(float lo, float hi, uint32_t L, flo
 __device__ __forceinline__ uint32_t quant_code(float x, float lo, float inv, uint32_t L) {
   const float r = __fmaf_rn(__fsub_rn(x, lo), inv, kMagicF);
   return (__float_as_uint(r) - kMagicBits) & L;
+}
+
+// ---- random rounding (rounding = 1) ------------------------------------------------------------------
+// Philox-4x32 with 10 rounds (Salmon et al., SC'11): counter-based, so a draw is a pure function of the
+// key (seed) and the counter (group within the plane, plane, tensor id).
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
+                                              uint32_t (&out)[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+    const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+    c0 = h1 ^ c1 ^ k0;
+    c1 = l1;
+    c2 = h0 ^ c3 ^ k1;
+    c3 = l0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0;
+  out[1] = c1;
+  out[2] = c2;
+  out[3] = c3;
+}
+// Code of one element under random rounding: t = fp32 product (x - lo) * inv, n = floor(t), and the code
+// goes up iff floor(frac(t) * 2^24) + (word >> 8) reaches 2^24.
+__device__ __forceinline__ uint32_t quant_code_random(float x, float lo, float inv, uint32_t L, uint32_t word) {
+  const float t = __fmul_rn(__fsub_rn(x, lo), inv);
+  const float nf = floorf(t);
+  const uint32_t fi = (uint32_t)__fmul_rn(__fsub_rn(t, nf), 16777216.0f);
+  const uint32_t up = (fi + (word >> 8)) >> 24;
+  const uint32_t n = nf >= (float)L ? L : (uint32_t)nf;
+  return min(n + up, L);
 }
 
 // Pre-quantisation of dense-block elements (Eq. 9 on integers): k = rne(fp32(x * inv2e)), |k| <= 2^24.

@@ -62,7 +62,7 @@ def test_argument_errors_are_returned_before_any_cuda_call(lib):
     assert lib.fh_compress(C.byref(d), C.byref(api.default_params(bits=3)), addr, addr, 4096, None, None) == api.FH_ERR_UNSUPPORTED
     assert lib.fh_compress(C.byref(d), C.byref(api.default_params(eps=0.0)), addr, addr, 4096, None, None) == api.FH_ERR_ARG
     assert lib.fh_compress(C.byref(d), C.byref(api.default_params(block=4)), addr, addr, 4096, None, None) == api.FH_ERR_UNSUPPORTED
-    assert lib.fh_compress(C.byref(d), C.byref(api.default_params(rounding=1)), addr, addr, 4096, None, None) == api.FH_ERR_UNSUPPORTED
+    assert lib.fh_compress(C.byref(d), C.byref(api.default_params(rounding=2)), addr, addr, 4096, None, None) == api.FH_ERR_UNSUPPORTED
     # bad tensor
     assert lib.fh_compress(C.byref(api.desc((1, 0, 8, 8))), C.byref(p), addr, addr, 4096, None, None) == api.FH_ERR_ARG
     assert lib.fh_compress(C.byref(api.desc((1, 1, 1, 70000))), C.byref(p), addr, addr, 4096, None, None) == api.FH_ERR_UNSUPPORTED

@@ -420,3 +420,31 @@ def test_tensor_beyond_4_gib_on_sampled_planes():
     # every zero of a post-ReLU plane comes back as zero (normal planes have lo = 0; the block-wise path keeps zeros)
     probe = torch.from_numpy(idx[:32]).cuda()
     assert bool(((x.view(P, 1024)[probe] == 0) <= (out.view(P, 1024)[probe] == 0)).all())
+
+
+@pytest.mark.parametrize("shape", [(3, 5, 7, 7), (2, 9, 14, 14), (1, 12, 32, 32), (2, 8, 28, 28), (1, 6, 56, 56), (1, 3, 112, 112),
+                                   (2, 6, 33, 17), (300, 1, 4, 4)])
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+@pytest.mark.parametrize("bits", [2, 4, 8])
+def test_parity_random_rounding(shape, dtype, bits):
+    """rounding = 1: the draws come from the same counter-based generator on both sides, so the container
+    is still identical byte for byte (normal planes carry randomly rounded codes, outlier-rich planes are
+    coded as before)."""
+    kind = "spiky_relu" if shape[1] >= 3 else "relu"
+    spec = synth.TensorSpec("t", shape, dtype, kind, 60 + bits)
+    raw = synth.make(spec)
+    kw = dict(bits=bits, rounding=1, seed=0x1234567887654321 + bits)
+    st_o, buf_o, total_o = fho.compress(raw, fho.desc(shape, dtype, tensor_id=0xABCDEF0123), fho.params(**kw))
+    assert st_o == fho.OK and fho.parse_header(buf_o)["rounding"] == 1
+    p = api.default_params(**kw)
+    st_g, packed, total_g = api.compress_tensor(to_dev(raw), shape, dtype, p, tensor_id=0xABCDEF0123)
+    assert st_g == api.FH_OK and total_g == total_o
+    assert np.array_equal(packed[:total_g].cpu().numpy(), buf_o)
+    st_d, out_g = api.decompress_tensor(packed, total_g, shape, dtype)
+    assert st_d == api.FH_OK
+    _, out_o = fho.decompress(buf_o, fho.desc(shape, dtype))
+    got = out_g.cpu().numpy()
+    check_same_values(got.view(np.uint16) if dtype == synth.BF16 else got, out_o, dtype)
+    # another seed gives other codes
+    st_2, packed2, _ = api.compress_tensor(to_dev(raw), shape, dtype, api.default_params(bits=bits, rounding=1, seed=5), tensor_id=0xABCDEF0123)
+    assert st_2 == api.FH_OK and not np.array_equal(packed2[:total_g].cpu().numpy(), buf_o)
