@@ -47,7 +47,7 @@ def workload_specs(name: str):
         return synth.config3(128), "configs[2]: MobileNetV2-shaped expanded activations, batch 128, bf16, Laplace(0,1) " \
                                    "with channel-clustered +-50 outliers"
     if name == "cifar_schedule":
-        return synth.config5(128), "configs[4]: 20 ResNet-18/CIFAR-shaped tensors, batch 128, fp32 (all compressed here)"
+        return synth.config5(128), "configs[4]: 20 ResNet-18/CIFAR-shaped tensors, batch 128, fp32"
     if name == "config1":
         return synth.config1(), "configs[0]: 32x16x32x32 fp32 ReLU(N(0,1))"
     if name.startswith("sweep_"):          # sweep_<MiB>_<f32|bf16>
@@ -350,7 +350,8 @@ def run_ours(args, specs, wl_desc):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32" if specs[0].dtype == synth.F32 else "bf16", "data": "synthetic",
-            "config": {"workload": wl_desc, "bits": list(BITS), "salient_mode": args.mode.upper(),
+            "config": {"workload": wl_desc + ("; every tensor compressed" if args.workload == "cifar_schedule" else ""),
+                       "bits": list(BITS), "salient_mode": args.mode.upper(),
                        "rounding": "nearest-even" if args.rounding == 0 else "random (Philox-4x32-10)",
                        "tensors": len(tensors), "dense_bytes_per_pass": dense_bytes,
                        "packed_bytes": {str(b): packed_bytes[b] for b in BITS},
@@ -380,6 +381,63 @@ def run_ours(args, specs, wl_desc):
     api.shutdown()
 
 
+def run_schedule(args, specs, wl_desc):
+    """One training step's worth of codec work through fh_run_schedule: the tensors marked `compress` are
+    compressed in forward order into one arena and restored in reverse order, on one stream.  A step is one
+    call; the library times the two phases with CUDA events and reports the arena's high-water mark."""
+    import torch
+    from paper_2510_11400_b200 import api, build
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    build.build()
+    api.lib()
+    mode = {"auto": api.FH_SALIENT_AUTO, "off": api.FH_SALIENT_OFF, "all": api.FH_SALIENT_ALL}[args.mode]
+    p = api.default_params(bits=2, salient_mode=mode, rounding=args.rounding, seed=2510_11400)
+    items, need = [], 0
+    for i, s in enumerate(specs):
+        raw = synth.make(s)
+        t = torch.from_numpy(raw.view(np.int16) if raw.dtype == np.uint16 else raw).cuda()
+        d = api.desc(s.shape, s.dtype, tensor_id=i)
+        items.append(api.SchedItem(d, api.FH_COMPRESS if s.compress else api.FH_KEEP, t, torch.empty_like(t)))
+        if s.compress:
+            need += (api.compressed_bytes(d, p, 1) + 255) & ~255
+    arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+    sampler = ClockSampler(torch.cuda.current_device())
+    for _ in range(max(3, args.warmup)):
+        rep = api.fh_run_schedule(items, p, arena)
+        assert rep.status == api.FH_OK, rep.status
+    launches0 = api.kernel_launches()
+    sampler.start()
+    fwd = bwd = 0.0
+    for _ in range(args.steps):
+        rep = api.fh_run_schedule(items, p, arena)
+        assert rep.status == api.FH_OK, rep.status
+        fwd += rep.ms_forward
+        bwd += rep.ms_backward
+    clocks = sampler.stop()
+    launches = api.kernel_launches() - launches0
+    dense = int(rep.total_dense_bytes)
+    ms = (fwd + bwd) / args.steps
+    peak, peak_kind = peaks()
+    line = {"metric": METRIC, "value": 2 * dense / (ms / 1e3) / 1e9, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32" if specs[0].dtype == synth.F32 else "bf16", "data": "synthetic",
+            "config": {"workload": wl_desc + "; through fh_run_schedule, tensors with even index compressed, the rest kept",
+                       "bits": [2], "salient_mode": args.mode.upper(), "tensors": len(specs),
+                       "compressed_tensors": sum(1 for s in specs if s.compress)},
+            "schedule": {"ms_forward": fwd / args.steps, "ms_backward": bwd / args.steps, "total_dense_bytes": dense,
+                         "total_packed_bytes": int(rep.total_packed_bytes), "peak_packed_bytes": int(rep.peak_packed_bytes),
+                         "compress_gbs": dense / (fwd / args.steps) / 1e6, "decompress_gbs": dense / (bwd / args.steps) / 1e6},
+            "roofline": {"bound": "hbm", "kernel": "forward phase: every compress call of the schedule",
+                         "achieved": (dense + int(rep.total_packed_bytes)) / (fwd / args.steps) / 1e6, "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                         "frac": (dense + int(rep.total_packed_bytes)) / (fwd / args.steps) / 1e6 / peak, "traffic": None},
+            "clocks": clocks, "gpu_launches": int(launches)}
+    print(json.dumps(line), flush=True)
+    api.shutdown()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -390,6 +448,8 @@ def main():
     ap.add_argument("--mode", default="auto", choices=["auto", "off", "all"])
     ap.add_argument("--rounding", type=int, default=0, choices=[0, 1],
                     help="1: random rounding of normal planes (runs on the general-purpose kernel)")
+    ap.add_argument("--schedule", action="store_true",
+                    help="run the workload through fh_run_schedule (forward-order compress, reverse-order decompress)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     args = ap.parse_args()
@@ -397,6 +457,8 @@ def main():
     specs, wl_desc = workload_specs(args.workload)
     if args.impl == "reference":
         run_reference(args, specs, wl_desc)
+    elif args.schedule:
+        run_schedule(args, specs, wl_desc)
     else:
         run_ours(args, specs, wl_desc)
 
