@@ -69,6 +69,23 @@ def peaks():
     return 6650.0, "fallback"
 
 
+def slowest_rank(value: float, world: int, device=None) -> float:
+    """The timing rule for N replicas: every rank contributes its own device time, the job's time is the
+    slowest rank's.  (One all-reduce(MAX) of a scalar; the data path itself has no collective.)"""
+    if world <= 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(dense_bytes_per_rank: int, world: int, seconds: float) -> float:
+    """Aggregate dense GB/s of N replicas that each pushed `dense_bytes_per_rank` through the codec."""
+    return world * dense_bytes_per_rank / seconds / 1e9
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
     Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown," \
@@ -288,10 +305,7 @@ def run_ours(args, specs, wl_desc):
     clocks = sampler.stop()
     launches = api.kernel_launches() - launches0
     ms = e0.elapsed_time(e1)
-    if world > 1:
-        tt = torch.tensor([ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    ms = slowest_rank(ms, world, dev)
     t_comp = {b: sum(e[b][0].elapsed_time(e[b][1]) for e in evs) for b in BITS}
     t_dec = {b: sum(e[b][1].elapsed_time(e[b][2]) for e in evs) for b in BITS}
 
@@ -329,11 +343,8 @@ def run_ours(args, specs, wl_desc):
             h2d, d2h = e2e_step()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            tt = torch.tensor([dt], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            dt = float(tt.item())
-        e2e = {"value": world * ksteps * dense_bytes * 2 * len(BITS) / dt / 1e9, "unit": UNIT,
+        dt = slowest_rank(dt, world, dev)
+        e2e = {"value": whole_job_value(ksteps * dense_bytes * 2 * len(BITS), world, dt), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": ksteps}
 
     if rank == 0:
@@ -345,7 +356,7 @@ def run_ours(args, specs, wl_desc):
         # DRAM bytes per compress call from the ncu capture summarised under profiles/ (null for any other
         # workload or mode than the one captured)
         traffic = NCU_DRAM_BYTES_PER_COMPRESS_CALL if (args.workload == "resnet18_b64" and args.mode == "auto") else None
-        value = world * args.steps * dense_bytes * 2 * len(BITS) / (ms / 1e3) / 1e9
+        value = whole_job_value(args.steps * dense_bytes * 2 * len(BITS), world, ms / 1e3)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
