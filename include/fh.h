@@ -234,6 +234,61 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
 int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                        size_t dst_capacity, uint64_t* d_out2, void* stream);
 
+/*
+ * Plan generation (Algorithm 1 with the MPS metric of Eq. 5; host only, no CUDA call).
+ *
+ * The computation sequence is walked op by op (Main).  Compute(op) makes the op's inputs resident again --
+ * a COMPRESSED input gets its dense buffer back (decompress), an EVICTED one is recomputed -- and allocates
+ * its outputs.  Every allocation goes through Alloc: while pool_size + size >= memory_budget, the resident
+ * tensor with the largest MPS is purged, evicted if MPS_compute > MPS_compress, compressed otherwise.
+ *   MPS(d) = SM(d) * FLT(d) / (PC(d) + RC(d))                                                  (Eq. 5)
+ *   compress: SM = bytes - packed_bytes, PC = t_compress, RC = t_decompress
+ *   evict   : SM = bytes,                PC = 0,          RC = t_recompute  (Eq. 6, supplied by the caller)
+ *   FLT(d)  = time from the current op's start to the start of the next op that reads d
+ * Readings where the paper is silent: tensors of the current op are locked (never purged); a tensor is
+ * dropped from the pool after its last reader; tensors no op produces are resident from the start; only
+ * resident tensors with a later reader are candidates; ties go to the lower tensor index; a tensor that
+ * cannot shrink (packed_bytes >= bytes) or cannot be recomputed (t_recompute < 0) has MPS 0 for that
+ * technique; when nothing can be purged the allocation proceeds over budget and the report says so.
+ * t_compress / t_decompress are what this library's fh_compress / fh_decompress take on the target device.
+ *
+ * actions[t] receives the last purge decision for tensor t (FH_KEEP, FH_COMPRESS or FH_EVICT) -- the action
+ * of an fh_sched_entry; events (optional, up to max_events) receive every decision in order:
+ * kind FH_COMPRESS / FH_EVICT = purged before op `op`, FH_KEEP = brought back for op `op`.
+ * Returns FH_OK, FH_ERR_ARG (null pointers, tensor ids out of range, negative or all-zero costs), or
+ * FH_ERR_CAPACITY (plan produced, but some allocation could not be brought under the budget).
+ */
+typedef struct {
+  uint64_t bytes;        /* dense size                                                      */
+  uint64_t packed_bytes; /* size once compressed                                            */
+  double t_compress;     /* seconds                                                         */
+  double t_decompress;   /* seconds                                                         */
+  double t_recompute;    /* seconds, Eq. 6; negative: the tensor cannot be recomputed       */
+} fh_plan_tensor;
+
+typedef struct {
+  double time;            /* OpTime, seconds                                                */
+  const int32_t* inputs;  /* tensor ids read                                                */
+  int32_t n_inputs;
+  const int32_t* outputs; /* tensor ids produced                                            */
+  int32_t n_outputs;
+} fh_plan_op;
+
+typedef struct {
+  int32_t op, tensor, kind;
+} fh_plan_event;
+
+typedef struct {
+  uint64_t peak_bytes;     /* largest pool size reached                                     */
+  double overhead_seconds; /* sum of compress, decompress and recompute times the plan adds  */
+  int32_t n_events;        /* decisions taken (may exceed max_events; the rest is not stored) */
+  int32_t n_over_budget;   /* allocations that stayed over budget                            */
+} fh_plan_report;
+
+int fh_plan_generate(const fh_plan_op* ops, int32_t n_ops, const fh_plan_tensor* tensors, int32_t n_tensors,
+                     uint64_t memory_budget, int32_t* actions, fh_plan_event* events, int32_t max_events,
+                     fh_plan_report* report);
+
 /* Number of kernels this library has launched since it was loaded (for launch accounting). */
 uint64_t fh_kernel_launches(void);
 

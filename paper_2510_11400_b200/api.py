@@ -22,7 +22,7 @@ FH_STATIC_MAX_PLANES = 131072
 
 EXPORTS = ["fh_default_params", "fh_version", "fh_device_count", "fh_compressed_bytes", "fh_compress",
            "fh_decompress", "fh_run_schedule", "fh_host_work_bytes", "fh_compress_host",
-           "fh_decompress_host", "fh_compress_static", "fh_kernel_launches", "fh_shutdown"]
+           "fh_decompress_host", "fh_compress_static", "fh_plan_generate", "fh_kernel_launches", "fh_shutdown"]
 
 
 class FhError(RuntimeError):
@@ -52,6 +52,25 @@ class fh_sched_report(C.Structure):
     _fields_ = [("total_dense_bytes", C.c_uint64), ("total_packed_bytes", C.c_uint64),
                 ("peak_packed_bytes", C.c_uint64), ("ms_forward", C.c_float), ("ms_backward", C.c_float),
                 ("status", C.c_int32)]
+
+
+class fh_plan_tensor(C.Structure):
+    _fields_ = [("bytes", C.c_uint64), ("packed_bytes", C.c_uint64), ("t_compress", C.c_double),
+                ("t_decompress", C.c_double), ("t_recompute", C.c_double)]
+
+
+class fh_plan_op(C.Structure):
+    _fields_ = [("time", C.c_double), ("inputs", C.POINTER(C.c_int32)), ("n_inputs", C.c_int32),
+                ("outputs", C.POINTER(C.c_int32)), ("n_outputs", C.c_int32)]
+
+
+class fh_plan_event(C.Structure):
+    _fields_ = [("op", C.c_int32), ("tensor", C.c_int32), ("kind", C.c_int32)]
+
+
+class fh_plan_report(C.Structure):
+    _fields_ = [("peak_bytes", C.c_uint64), ("overhead_seconds", C.c_double), ("n_events", C.c_int32),
+                ("n_over_budget", C.c_int32)]
 
 
 _lib = None
@@ -90,6 +109,10 @@ def lib() -> C.CDLL:
         L.fh_decompress_host.restype = C.c_int
         L.fh_compress_static.argtypes = [D, P, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
         L.fh_compress_static.restype = C.c_int
+        L.fh_plan_generate.argtypes = [C.POINTER(fh_plan_op), C.c_int32, C.POINTER(fh_plan_tensor), C.c_int32, C.c_uint64,
+                                       C.POINTER(C.c_int32), C.POINTER(fh_plan_event), C.c_int32,
+                                       C.POINTER(fh_plan_report)]
+        L.fh_plan_generate.restype = C.c_int
         L.fh_kernel_launches.restype = C.c_uint64
         L.fh_shutdown.restype = None
         _lib = L
@@ -189,6 +212,26 @@ def fh_decompress_host(h_src, src_bytes: int, d: fh_tensor_desc, h_dst, work, st
     rc = lib().fh_decompress_host(h_src.data_ptr(), src_bytes, C.byref(d), h_dst.data_ptr(), C.byref(st),
                                   work.data_ptr(), work.numel() * work.element_size(), _stream_ptr(stream))
     return int(rc)
+
+
+def plan_generate(ops, tensors, memory_budget: int, max_events: int = 4096):
+    """ops: [{time, inputs, outputs}], tensors: [{bytes, packed_bytes, t_compress, t_decompress, t_recompute}].
+    Returns (status, actions, events, report)."""
+    keep = []
+    c_ops = (fh_plan_op * len(ops))()
+    for i, op in enumerate(ops):
+        ins = (C.c_int32 * len(op["inputs"]))(*op["inputs"])
+        outs = (C.c_int32 * len(op["outputs"]))(*op["outputs"])
+        keep += [ins, outs]
+        c_ops[i] = fh_plan_op(op["time"], ins, len(op["inputs"]), outs, len(op["outputs"]))
+    c_t = (fh_plan_tensor * len(tensors))(*[fh_plan_tensor(t["bytes"], t["packed_bytes"], t["t_compress"], t["t_decompress"],
+                                                             t["t_recompute"]) for t in tensors])
+    actions = (C.c_int32 * max(1, len(tensors)))()
+    events = (fh_plan_event * max(1, max_events))()
+    rep = fh_plan_report()
+    rc = lib().fh_plan_generate(c_ops, len(ops), c_t, len(tensors), memory_budget, actions, events, max_events, C.byref(rep))
+    n = min(rep.n_events, max_events)
+    return int(rc), [int(a) for a in actions[:len(tensors)]], [(e.op, e.tensor, e.kind) for e in events[:n]], rep
 
 
 def kernel_launches() -> int:

@@ -448,3 +448,45 @@ def test_parity_random_rounding(shape, dtype, bits):
     # another seed gives other codes
     st_2, packed2, _ = api.compress_tensor(to_dev(raw), shape, dtype, api.default_params(bits=bits, rounding=1, seed=5), tensor_id=0xABCDEF0123)
     assert st_2 == api.FH_OK and not np.array_equal(packed2[:total_g].cpu().numpy(), buf_o)
+
+
+def test_generated_plan_drives_the_schedule():
+    """Algorithm 1 end to end: a plan is generated for one training step under a memory budget (costs of
+    compression as this library delivers them on a B200-class device, recomputation costs made up), and its
+    per-tensor actions are what fh_run_schedule executes."""
+    import torch
+    shapes = [(8, 32, 32, 32), (8, 32, 32, 32), (8, 64, 16, 16), (8, 64, 16, 16), (8, 128, 8, 8), (8, 128, 8, 8)]
+    specs = [synth.TensorSpec(f"p{i}", sh, synth.F32, "relu", 700 + i) for i, sh in enumerate(shapes)]
+    n = len(specs)
+    p = api.default_params(bits=2)
+    tensors = []
+    for i, sp in enumerate(specs):
+        b = sp.dense_bytes
+        packed = api.compressed_bytes(api.desc(sp.shape, sp.dtype), p, 0)
+        tensors.append(dict(bytes=b, packed_bytes=packed, t_compress=20e-6 + b / 3e12, t_decompress=12e-6 + b / 4e12,
+                            t_recompute=(30e-6 if i % 3 == 2 else 400e-6)))
+    ops = [dict(time=100e-6, inputs=[k - 1] if k else [], outputs=[k]) for k in range(n)]
+    ops += [dict(time=200e-6, inputs=[k], outputs=[]) for k in reversed(range(n))]
+    budget = int(0.5 * sum(t["bytes"] for t in tensors))
+    rc, actions, events, rep = api.plan_generate(ops, tensors, budget)
+    assert rc == api.FH_OK and rep.peak_bytes < budget
+    assert api.FH_COMPRESS in actions and api.FH_EVICT in actions       # the hybrid: both techniques get used
+    items, raws, rest = [], [], []
+    for sp, act in zip(specs, actions):
+        raw = synth.make(sp)
+        raws.append(raw)
+        dense = to_dev(raw)
+        out = torch.zeros_like(dense)
+        rest.append(out)
+        items.append(api.SchedItem(api.desc(sp.shape, sp.dtype, tensor_id=sp.seed), act, dense, out))
+    arena = torch.zeros(4 << 20, dtype=torch.uint8, device="cuda")
+    srep = api.fh_run_schedule(items, p, arena)
+    assert srep.status == api.FH_OK
+    assert srep.total_dense_bytes == sum(t["bytes"] for t, a in zip(tensors, actions) if a == api.FH_COMPRESS)
+    for sp, raw, out, act in zip(specs, raws, rest, actions):
+        if act != api.FH_COMPRESS:
+            assert not bool(out.any())
+            continue
+        d = fho.desc(sp.shape, sp.dtype, tensor_id=sp.seed)
+        _, buf_o, _ = fho.compress(raw, d, fho.params(bits=2))
+        check_same_values(out.cpu().numpy(), fho.decompress(buf_o, d)[1], sp.dtype)
