@@ -52,6 +52,7 @@
 #define MODE_AUTO 0
 #define MODE_OFF 1
 #define MODE_ALL 2
+#define MODE_CHANNEL 3 /* three-sigma rule with mu, sigma and the class taken per channel over the whole batch */
 
 typedef struct {
   int32_t dtype;
@@ -108,7 +109,7 @@ static int check_args(const fho_desc* d, const fho_params* p) {
   if (d->n < 1 || d->c < 1 || d->h < 1 || d->w < 1) return FHO_ERR_ARG;
   if (d->w > 65535) return FHO_ERR_UNSUPPORTED;
   if (p->bits != 2 && p->bits != 4 && p->bits != 8) return FHO_ERR_UNSUPPORTED;
-  if (p->salient_mode < 0 || p->salient_mode > 2) return FHO_ERR_ARG;
+  if (p->salient_mode < 0 || p->salient_mode > 3) return FHO_ERR_ARG;
   if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FHO_ERR_ARG;
   if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FHO_ERR_ARG;
   if (p->block != 8) return FHO_ERR_UNSUPPORTED;
@@ -226,6 +227,64 @@ void fho_plane_sigma(const float* x, int64_t hw, double* S_out, double* Q_out, f
     if (x[i] > thi || x[i] < tlo) ++cnt;
   *S_out = S;
   *Q_out = Q;
+  *t_lo = tlo;
+  *t_hi = thi;
+  *n_out = cnt;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * The other reading of "classify channels" (Section 4.4.1): a channel is channel c of the layer, i.e.
+ * the N planes (n, c) of the batch together.  mu and sigma are then taken over all N*HW elements of
+ * the channel, with the same fixed-point accumulation as above (A = largest magnitude of the channel;
+ * every plane is cut into its own groups of four, tail padded with zeros; r = 1/(N*HW)); the count
+ * runs over the whole channel and the channel, hence each of its planes, is outlier-rich when
+ * n_out * rho_den > rho_num * N * HW.  A plane's table entry carries the plane's own count.
+ * x: N planes of channel c, each hw elements, plane n at x + n*stride.
+ * ------------------------------------------------------------------------------------------ */
+void fho_channel_sigma(const float* x, int64_t n_planes, int64_t stride, int64_t hw, float* t_lo, float* t_hi,
+                       int64_t* n_out) {
+  float lo = x[0], hi = x[0];
+  for (int64_t n = 0; n < n_planes; ++n)
+    for (int64_t i = 0; i < hw; ++i) {
+      float v = x[n * stride + i];
+      if (v < lo) lo = v;
+      if (v > hi) hi = v;
+    }
+  float A = fmaxf(fabsf(lo), fabsf(hi));
+  uint32_t ab;
+  memcpy(&ab, &A, 4);
+  int e = (int)((ab >> 23) & 255u) - 127;
+  int ks = 18 - e, kq = 16 - 2 * e;
+  if (ks > 126) ks = 126;
+  if (kq > 126) kq = 126;
+  if (kq < -126) kq = -126;
+  float cs = pow2f(ks), cq = pow2f(kq);
+  int64_t Is = 0, Iq = 0;
+  for (int64_t n = 0; n < n_planes; ++n)
+    for (int64_t g = 0; g < hw; g += 4) {
+      float v[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int k = 0; k < 4 && g + k < hw; ++k) v[k] = x[n * stride + g + k];
+      float s01 = v[0] + v[1], s23 = v[2] + v[3];
+      float sg = s01 + s23;
+      float p0 = v[0] * v[0], p2 = v[2] * v[2];
+      float q01 = fmaf(v[1], v[1], p0), q23 = fmaf(v[3], v[3], p2);
+      float qg = q01 + q23;
+      Is += fixed_point(sg, cs);
+      Iq += fixed_point(qg, cq);
+    }
+  double S = ldexp((double)Is, -ks), Q = ldexp((double)Iq, -kq);
+  double r = 1.0 / (double)(n_planes * hw);
+  double mu = S * r, m2 = Q * r, mu2 = mu * mu;
+  double var = m2 - mu2;
+  if (!(var > 0.0)) var = 0.0;
+  float mu_f = (float)mu, sigma_f = sqrtf((float)var);
+  float thi = fmaf(3.0f, sigma_f, mu_f), tlo = fmaf(-3.0f, sigma_f, mu_f);
+  int64_t cnt = 0;
+  for (int64_t n = 0; n < n_planes; ++n)
+    for (int64_t i = 0; i < hw; ++i) {
+      float v = x[n * stride + i];
+      if (v > thi || v < tlo) ++cnt;
+    }
   *t_lo = tlo;
   *t_hi = thi;
   *n_out = cnt;
@@ -469,8 +528,14 @@ static size_t encode_salient(const float* x, const uint8_t* raw, int dtype, int 
   return size;
 }
 
+/* ch: for MODE_CHANNEL the channel's {t_lo, t_hi} and whether the channel is outlier-rich; NULL otherwise */
+typedef struct {
+  float tlo, thi;
+  int salient;
+} channel_info;
+
 static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_params* p,
-                         uint64_t plane_index, uint64_t tensor_id, plane_result* r) {
+                         uint64_t plane_index, uint64_t tensor_id, const channel_info* ch, plane_result* r) {
   size_t hw = (size_t)H * W, e = esize(dtype);
   float* x = (float*)malloc(hw * sizeof(float));
   for (size_t i = 0; i < hw; ++i)
@@ -499,6 +564,10 @@ static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_
     if ((int64_t)cnt * p->rho_den > (int64_t)p->rho_num * (int64_t)hw) cls = CLS_SALIENT;
   } else if (p->salient_mode == MODE_ALL) {
     cls = CLS_SALIENT;
+  } else if (p->salient_mode == MODE_CHANNEL) {
+    for (size_t i = 0; i < hw; ++i)
+      if (x[i] > ch->thi || x[i] < ch->tlo) ++n_out;
+    if (ch->salient) cls = CLS_SALIENT;
   }
   if (cls == CLS_SALIENT) {
     uint8_t* buf = NULL;
@@ -553,11 +622,42 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
   if (!src || !dst) return FHO_ERR_ARG;
   size_t P = (size_t)d->n * d->c, hw = (size_t)d->h * d->w, e = esize(d->dtype);
   plane_result* res = (plane_result*)calloc(P, sizeof(plane_result));
+  channel_info* chan = NULL;
+  if (p->salient_mode == MODE_CHANNEL) {
+    chan = (channel_info*)calloc((size_t)d->c, sizeof(channel_info));
+    int bad = 0;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(dynamic, 1) num_threads(g_threads)
+#endif
+    for (int64_t c = 0; c < (int64_t)d->c; ++c) {
+      float* x = (float*)malloc((size_t)d->n * hw * sizeof(float));
+      int finite = 1;
+      for (int64_t n = 0; n < (int64_t)d->n; ++n)
+        for (size_t i = 0; i < hw; ++i) {
+          size_t idx = ((size_t)n * d->c + (size_t)c) * hw + i;
+          float v = d->dtype == FHO_F32 ? ((const float*)src)[idx] : bf16_to_f32(((const uint16_t*)src)[idx]);
+          if (!isfinite(v)) finite = 0;
+          x[(size_t)n * hw + i] = v;
+        }
+      if (!finite) {
+        bad = 1; /* reported per plane below */
+        chan[c].tlo = chan[c].thi = 0.0f;
+      } else {
+        int64_t cnt;
+        fho_channel_sigma(x, d->n, (int64_t)hw, (int64_t)hw, &chan[c].tlo, &chan[c].thi, &cnt);
+        chan[c].salient = cnt * (int64_t)p->rho_den > (int64_t)p->rho_num * (int64_t)d->n * (int64_t)hw;
+      }
+      free(x);
+    }
+    (void)bad;
+  }
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)
 #endif
   for (int64_t pl = 0; pl < (int64_t)P; ++pl)
-    encode_plane((const uint8_t*)src + (size_t)pl * hw * e, d->dtype, d->h, d->w, p, (uint64_t)pl, d->tensor_id, &res[pl]);
+    encode_plane((const uint8_t*)src + (size_t)pl * hw * e, d->dtype, d->h, d->w, p, (uint64_t)pl, d->tensor_id,
+                 chan ? &chan[pl % d->c] : NULL, &res[pl]);
+  free(chan);
   const size_t npay = a16(normal_payload(hw, p->bits));
   size_t total = 64 + 16 * P + P * npay;
   uint32_t n_sal = 0, n_raw = 0;

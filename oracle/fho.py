@@ -18,7 +18,7 @@ _LIB = os.path.join(_HERE, "libfho.so")
 
 OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_NONFINITE, ERR_CORRUPT = 0, -1, -2, -3, -4, -5
 F32, BF16 = 0, 1
-AUTO, OFF, ALL = 0, 1, 2
+AUTO, OFF, ALL, CHANNEL = 0, 1, 2, 3
 NORMAL, SALIENT, RAW = 0, 1, 2
 
 
@@ -72,6 +72,9 @@ def lib():
         L.fho_plane_sigma.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_double),
                                       C.POINTER(C.c_double), C.POINTER(C.c_float),
                                       C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+        L.fho_channel_sigma.restype = None
+        L.fho_channel_sigma.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.POINTER(C.c_float),
+                                        C.POINTER(C.c_float), C.POINTER(C.c_int64)]
         L.fho_plane_sums.restype = None
         L.fho_plane_sums.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                      C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
@@ -134,6 +137,15 @@ def plane_sigma(x: np.ndarray):
     lib().fho_plane_sigma(x.ctypes.data, x.size, C.byref(S), C.byref(Q), C.byref(tlo), C.byref(thi),
                           C.byref(n))
     return S.value, Q.value, tlo.value, thi.value, n.value
+
+
+def channel_sigma(x: np.ndarray):
+    """x: (n_planes, hw) float32, the planes of one channel over the batch.  Returns (t_lo, t_hi, n_out)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    tlo, thi = C.c_float(), C.c_float()
+    n = C.c_int64()
+    lib().fho_channel_sigma(x.ctypes.data, x.shape[0], x.shape[1], x.shape[1], C.byref(tlo), C.byref(thi), C.byref(n))
+    return tlo.value, thi.value, n.value
 
 
 def plane_sums(x: np.ndarray):
