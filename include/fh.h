@@ -82,14 +82,19 @@ typedef struct {
   uint64_t tensor_id; /* carried in the header; also keys any random rounding */
 } fh_tensor_desc;
 
-typedef enum { FH_SALIENT_AUTO = 0, FH_SALIENT_OFF = 1, FH_SALIENT_ALL = 2 } fh_salient_mode;
+/* AUTO: three-sigma rule per plane.  OFF: every plane normal.  ALL: every plane takes the block-wise path.
+ * CHANNEL: the other reading of "classify channels" (Section 4.4.1) -- mu, sigma and the outlier count are
+ * taken over the N planes of channel c together (same fixed-point sums, r = 1/(N*HW)) and the channel as a
+ * whole, hence each of its planes, is normal or outlier-rich (n_out*rho_den > rho_num*N*HW); a plane's table
+ * entry carries the plane's own count.  It costs three more passes over the tensor and is not available
+ * through fh_compress_static. */
+typedef enum { FH_SALIENT_AUTO = 0, FH_SALIENT_OFF = 1, FH_SALIENT_ALL = 2, FH_SALIENT_CHANNEL = 3 } fh_salient_mode;
 
 /* Codec parameters.  The paper names these quantities but prints no values (Section 4.4.1);
  * fh_default_params() fills the defaults given beside each field. */
 typedef struct {
   int32_t bits;             /* code width of normal planes: 2, 4 or 8                      [2]     */
-  int32_t salient_mode;     /* AUTO: three-sigma rule; OFF: every plane normal; ALL: every
-                               plane takes the block-wise path                            [AUTO]  */
+  int32_t salient_mode;     /* fh_salient_mode                                            [AUTO]  */
   int32_t rho_num, rho_den; /* plane is outlier-rich iff n_out*rho_den > rho_num*HW        [1/32]  */
   int32_t block;            /* n: pooling window = block edge; 8 only                      [8]     */
   int32_t tau_num, tau_den; /* block is dense iff nnz*tau_den >= tau_num*n*n               [1/4]   */

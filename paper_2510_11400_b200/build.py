@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfh_sm100a.so")
 SOURCES = [os.path.join(CSRC, "fh.cu"), os.path.join(CSRC, "fh_plan.cpp")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("fh_device.cuh", "fh_compress.cuh", "fh_decompress.cuh")] + \
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("fh_device.cuh", "fh_channel.cuh", "fh_compress.cuh", "fh_decompress.cuh")] + \
     [os.path.join(os.path.dirname(HERE), "include", "fh.h")]
 
 

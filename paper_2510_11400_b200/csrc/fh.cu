@@ -12,6 +12,7 @@
 #include <utility>
 #include <vector>
 
+#include "fh_channel.cuh"
 #include "fh_compress.cuh"
 #include "fh_decompress.cuh"
 
@@ -42,7 +43,7 @@ int check_desc(const fh_tensor_desc* d) {
 int check_params(const fh_params* p) {
   if (!p) return FH_ERR_ARG;
   if (p->bits != 2 && p->bits != 4 && p->bits != 8) return FH_ERR_UNSUPPORTED;
-  if (p->salient_mode < 0 || p->salient_mode > 2) return FH_ERR_ARG;
+  if (p->salient_mode < 0 || p->salient_mode > 3) return FH_ERR_ARG;
   if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FH_ERR_ARG;
   if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FH_ERR_ARG;
   if (p->block != 8 || p->dense_bits != 8 || (p->rounding != 0 && p->rounding != 1)) return FH_ERR_UNSUPPORTED;
@@ -219,6 +220,10 @@ struct StreamScratch {
   fh::Scratch* sc = nullptr;      // counters, followed by kMaxChunks chunk sums
   uint32_t* worklist = nullptr;   // one word per plane of the largest tensor seen
   size_t wl_cap = 0;
+  uint32_t* plane_nout = nullptr;  // channel-wide three-sigma mode: per-plane counts ...
+  size_t pn_cap = 0;
+  fh::ChanStat* chan = nullptr;    // ... and per-channel statistics
+  size_t chan_cap = 0;
   unsigned long long* sched = nullptr;  // schedule runner: offsets, sizes, statuses
   size_t sched_cap = 0;
 };
@@ -249,6 +254,52 @@ int get_scratch(cudaStream_t stream, size_t planes, StreamScratch** out) {
     s.wl_cap = cap;
   }
   *out = &s;
+  return FH_OK;
+}
+
+int sm_count();
+
+// Scratch of the channel-wide three-sigma mode (grown like the work list).
+int get_channel_scratch(StreamScratch* s, size_t planes, size_t channels) {
+  if (planes > s->pn_cap) {
+    size_t cap = s->pn_cap ? s->pn_cap : 65536;
+    while (cap < planes) cap *= 2;
+    if (s->plane_nout) {
+      cudaDeviceSynchronize();
+      cudaFree(s->plane_nout);
+      s->plane_nout = nullptr;
+      s->pn_cap = 0;
+    }
+    if (cudaMalloc(&s->plane_nout, cap * sizeof(uint32_t)) != cudaSuccess) return FH_ERR_CUDA;
+    s->pn_cap = cap;
+  }
+  if (channels > s->chan_cap) {
+    size_t cap = s->chan_cap ? s->chan_cap : 4096;
+    while (cap < channels) cap *= 2;
+    if (s->chan) {
+      cudaDeviceSynchronize();
+      cudaFree(s->chan);
+      s->chan = nullptr;
+      s->chan_cap = 0;
+    }
+    if (cudaMalloc(&s->chan, cap * sizeof(fh::ChanStat)) != cudaSuccess) return FH_ERR_CUDA;
+    s->chan_cap = cap;
+  }
+  return FH_OK;
+}
+
+template <int DT>
+int launch_channel_passes(const Plan& pl, const fh::ChannelArgs& ca, cudaStream_t stream) {
+  const int sms = sm_count();
+  if (sms < 1) return FH_ERR_CUDA;
+  const uint64_t want = (pl.P + fh::kWarps - 1) / fh::kWarps, most = (uint64_t)sms * 8;
+  const int grid = (int)(want < most ? want : most);
+  if (cudaMemsetAsync(ca.chan, 0, pl.C * sizeof(fh::ChanStat), stream) != cudaSuccess) return FH_ERR_CUDA;
+  fh::channel_pass<DT, 0><<<grid, fh::kThreads, 0, stream>>>(pl, ca);
+  fh::channel_pass<DT, 1><<<grid, fh::kThreads, 0, stream>>>(pl, ca);
+  fh::channel_pass<DT, 2><<<grid, fh::kThreads, 0, stream>>>(pl, ca);
+  if (cudaGetLastError() != cudaSuccess) return FH_ERR_CUDA;
+  g_launches.fetch_add(3);
   return FH_OK;
 }
 
@@ -481,6 +532,21 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   a.worklist = s->worklist;
   a.chunk_ovf = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(s->sc) + 256);
   chunking(pl.P, &a.chunk_shift, &a.nchunks);
+  a.chan_nout = nullptr;
+  a.plane_nout = nullptr;
+  if (pl.mode == fh::kModeChannel) {  // statistics per channel over the batch: three passes ahead of the streaming kernel
+    rc = get_channel_scratch(s, pl.P, pl.C);
+    if (rc != FH_OK) return rc;
+    fh::ChannelArgs ca;
+    ca.src = (const uint8_t*)d_src;
+    ca.chan = s->chan;
+    ca.plane_nout = s->plane_nout;
+    ca.inv_nhw = 1.0 / ((double)pl.N * (double)pl.HW);
+    rc = pl.dtype == FH_F32 ? launch_channel_passes<fh::kF32>(pl, ca, stream) : launch_channel_passes<fh::kBF16>(pl, ca, stream);
+    if (rc != FH_OK) return rc;
+    a.chan_nout = reinterpret_cast<const unsigned long long*>(s->chan) + 3;
+    a.plane_nout = s->plane_nout;
+  }
   return launch_compress(pl, v, a, stream);
 }
 
@@ -751,6 +817,7 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   rc = make_plan(desc, params, true, &pl, &v);
   if (rc != FH_OK) return rc;
   if (pl.P > FH_STATIC_MAX_PLANES) return FH_ERR_UNSUPPORTED;  // beyond the fixed work list
+  if (pl.mode == fh::kModeChannel) return FH_ERR_UNSUPPORTED;  // its statistics need scratch the fixed array does not hold
   cudaStream_t stream = (cudaStream_t)stream_;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FH_ERR_CUDA;
@@ -774,6 +841,8 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   a.sc = reinterpret_cast<fh::Scratch*>(base);
   a.chunk_ovf = reinterpret_cast<uint32_t*>(base + 256);
   a.worklist = reinterpret_cast<uint32_t*>(base + kHeadBytes);
+  a.chan_nout = nullptr;
+  a.plane_nout = nullptr;
   chunking(pl.P, &a.chunk_shift, &a.nchunks);
   std::lock_guard<std::mutex> lock2(g_mu);  // the launch helpers keep their occupancy cache under g_mu
   return launch_compress(pl, v, a, stream);
@@ -790,6 +859,8 @@ void fh_shutdown(void) {
     cudaDeviceSynchronize();
     if (kv.second.sc) cudaFree(kv.second.sc);
     if (kv.second.worklist) cudaFree(kv.second.worklist);
+    if (kv.second.plane_nout) cudaFree(kv.second.plane_nout);
+    if (kv.second.chan) cudaFree(kv.second.chan);
     if (kv.second.sched) cudaFree(kv.second.sched);
   }
   g_scratch.clear();

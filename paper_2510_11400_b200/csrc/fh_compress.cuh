@@ -41,7 +41,17 @@ struct CompressArgs {
   uint32_t* worklist;                   // planes that take the block-wise path, in no particular order
   uint32_t* chunk_ovf;                  // per chunk of 2^chunk_shift planes: overflow size of its planes (16-byte units)
   uint32_t chunk_shift, nchunks;
+  // channel-wide three-sigma mode: per-channel outlier counts and per-plane counts from the statistics passes
+  const unsigned long long* chan_nout;  // stride: 4 words (see ChanStat)
+  const uint32_t* plane_nout;
 };
+
+// Class and outlier count of plane gp when mu and sigma are taken per channel over the batch.
+__device__ __forceinline__ uint32_t channel_class(const Plan& pl, const CompressArgs& a, uint64_t gp, uint32_t& n_out) {
+  n_out = a.plane_nout[gp];
+  const unsigned long long total = a.chan_nout[(gp % pl.C) * 4ull];
+  return total * pl.rho_den > (unsigned long long)pl.rho_num * pl.N * pl.HW ? kClsSalient : kClsNormal;
+}
 
 
 // Where the bytes of a salient / raw payload go: offsets below npay land in the plane's slot, the
@@ -444,6 +454,8 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
         if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * HW) cls = kClsSalient;
       } else if (pl.mode == kModeAll) {
         cls = kClsSalient;
+      } else if (pl.mode == kModeChannel) {
+        cls = channel_class(pl, a, p0 + lp, n_out);
       }
 
       Rec r;
@@ -654,6 +666,8 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
     if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
   } else if (pl.mode == kModeAll) {
     cls = kClsSalient;
+  } else if (pl.mode == kModeChannel) {
+    cls = channel_class(pl, a, gp, n_out);
   }
 
   r.lo = 0.0f;
@@ -1021,6 +1035,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
       if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
     } else {
       if (pl.mode == kModeAll) cls = kClsSalient;
+      if (pl.mode == kModeChannel) cls = channel_class(pl, a, gp, n_out);
       __syncthreads();  // every thread is done with the stage
     }
     if (tid == 0) {

@@ -490,3 +490,17 @@ def test_generated_plan_drives_the_schedule():
         d = fho.desc(sp.shape, sp.dtype, tensor_id=sp.seed)
         _, buf_o, _ = fho.compress(raw, d, fho.params(bits=2))
         check_same_values(out.cpu().numpy(), fho.decompress(buf_o, d)[1], sp.dtype)
+
+
+@pytest.mark.parametrize("shape", [(6, 20, 14, 14), (3, 5, 7, 7), (4, 12, 32, 32), (5, 8, 28, 28), (3, 6, 56, 56), (2, 3, 112, 112),
+                                   (4, 6, 33, 17), (40, 7, 4, 4)])
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_parity_channel_wide_three_sigma(shape, dtype):
+    """salient_mode = CHANNEL: statistics and class per channel over the batch; container identical to the
+    oracle's, and every channel is normal or outlier-rich as a whole."""
+    for kind, bits in (("spiky_relu", 2), ("laplace_ch", 8)):
+        spec = synth.TensorSpec("t", shape, dtype, kind, 83)
+        buf = full_parity(spec, bits=bits, salient_mode=api.FH_SALIENT_CHANNEL)
+        cls = hp.table(buf, shape[0] * shape[1])["cls"].reshape(shape[0], shape[1])
+        assert ((cls != fho.NORMAL).all(0) | (cls == fho.NORMAL).all(0)).all()
+    assert fho.parse_header(buf)["salient_mode"] == fho.CHANNEL
