@@ -53,6 +53,7 @@
 #define MODE_OFF 1
 #define MODE_ALL 2
 #define MODE_CHANNEL 3 /* three-sigma rule with mu, sigma and the class taken per channel over the whole batch */
+#define MODE_TENSOR 4  /* three-sigma thresholds from mu, sigma of the whole tensor; the class per plane */
 
 typedef struct {
   int32_t dtype;
@@ -109,7 +110,7 @@ static int check_args(const fho_desc* d, const fho_params* p) {
   if (d->n < 1 || d->c < 1 || d->h < 1 || d->w < 1) return FHO_ERR_ARG;
   if (d->w > 65535) return FHO_ERR_UNSUPPORTED;
   if (p->bits != 2 && p->bits != 4 && p->bits != 8) return FHO_ERR_UNSUPPORTED;
-  if (p->salient_mode < 0 || p->salient_mode > 3) return FHO_ERR_ARG;
+  if (p->salient_mode < 0 || p->salient_mode > 4) return FHO_ERR_ARG;
   if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FHO_ERR_ARG;
   if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FHO_ERR_ARG;
   if (p->block != 8) return FHO_ERR_UNSUPPORTED;
@@ -528,7 +529,8 @@ static size_t encode_salient(const float* x, const uint8_t* raw, int dtype, int 
   return size;
 }
 
-/* ch: for MODE_CHANNEL the channel's {t_lo, t_hi} and whether the channel is outlier-rich; NULL otherwise */
+/* ch: for MODE_CHANNEL the channel's {t_lo, t_hi} and whether the channel is outlier-rich; for MODE_TENSOR the
+ * tensor's {t_lo, t_hi} (a plane is then outlier-rich by its own count against these); NULL otherwise */
 typedef struct {
   float tlo, thi;
   int salient;
@@ -568,6 +570,14 @@ static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_
     for (size_t i = 0; i < hw; ++i)
       if (x[i] > ch->thi || x[i] < ch->tlo) ++n_out;
     if (ch->salient) cls = CLS_SALIENT;
+  } else if (p->salient_mode == MODE_TENSOR) {
+    /* Third reading of the three-sigma rule (Section 4.4.1): what counts as an outlier is fixed once for the
+     * layer's whole activation tensor (mu and sigma over all N*C*HW elements, same fixed-point sums with
+     * A = the tensor's largest magnitude and r = 1/(N*C*HW)); a plane is outlier-rich when its own share of
+     * such outliers exceeds rho. */
+    for (size_t i = 0; i < hw; ++i)
+      if (x[i] > ch->thi || x[i] < ch->tlo) ++n_out;
+    if ((int64_t)n_out * p->rho_den > (int64_t)p->rho_num * (int64_t)hw) cls = CLS_SALIENT;
   }
   if (cls == CLS_SALIENT) {
     uint8_t* buf = NULL;
@@ -650,13 +660,26 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
       free(x);
     }
     (void)bad;
+  } else if (p->salient_mode == MODE_TENSOR) {
+    chan = (channel_info*)calloc(1, sizeof(channel_info));
+    float* x = (float*)malloc(P * hw * sizeof(float));
+    int finite = 1;
+    for (size_t i = 0; i < P * hw; ++i) {
+      x[i] = d->dtype == FHO_F32 ? ((const float*)src)[i] : bf16_to_f32(((const uint16_t*)src)[i]);
+      if (!isfinite(x[i])) finite = 0;
+    }
+    if (finite) { /* otherwise the planes report the error below */
+      int64_t cnt;
+      fho_channel_sigma(x, (int64_t)P, (int64_t)hw, (int64_t)hw, &chan[0].tlo, &chan[0].thi, &cnt);
+    }
+    free(x);
   }
 #ifdef _OPENMP
 #pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)
 #endif
   for (int64_t pl = 0; pl < (int64_t)P; ++pl)
     encode_plane((const uint8_t*)src + (size_t)pl * hw * e, d->dtype, d->h, d->w, p, (uint64_t)pl, d->tensor_id,
-                 chan ? &chan[pl % d->c] : NULL, &res[pl]);
+                 chan ? &chan[p->salient_mode == MODE_TENSOR ? 0 : pl % d->c] : NULL, &res[pl]);
   free(chan);
   const size_t npay = a16(normal_payload(hw, p->bits));
   size_t total = 64 + 16 * P + P * npay;

@@ -18,7 +18,7 @@ _LIB = os.path.join(_HERE, "libfho.so")
 
 OK, ERR_ARG, ERR_UNSUPPORTED, ERR_CAPACITY, ERR_NONFINITE, ERR_CORRUPT = 0, -1, -2, -3, -4, -5
 F32, BF16 = 0, 1
-AUTO, OFF, ALL, CHANNEL = 0, 1, 2, 3
+AUTO, OFF, ALL, CHANNEL, TENSOR = 0, 1, 2, 3, 4
 NORMAL, SALIENT, RAW = 0, 1, 2
 
 
