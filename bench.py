@@ -245,7 +245,7 @@ def run_ours(args, specs, wl_desc):
 
     dev = torch.device("cuda", local)
     mode = {"auto": api.FH_SALIENT_AUTO, "off": api.FH_SALIENT_OFF, "all": api.FH_SALIENT_ALL,
-            "channel": api.FH_SALIENT_CHANNEL}[args.mode]
+            "channel": api.FH_SALIENT_CHANNEL, "tensor": api.FH_SALIENT_TENSOR}[args.mode]
     params = {b: api.default_params(bits=b, salient_mode=mode, rounding=args.rounding, seed=2510_11400) for b in BITS}
     tensors = []
     for i, s in enumerate(specs):
@@ -405,7 +405,7 @@ def run_schedule(args, specs, wl_desc):
     build.build()
     api.lib()
     mode = {"auto": api.FH_SALIENT_AUTO, "off": api.FH_SALIENT_OFF, "all": api.FH_SALIENT_ALL,
-            "channel": api.FH_SALIENT_CHANNEL}[args.mode]
+            "channel": api.FH_SALIENT_CHANNEL, "tensor": api.FH_SALIENT_TENSOR}[args.mode]
     p = api.default_params(bits=2, salient_mode=mode, rounding=args.rounding, seed=2510_11400)
     items, need = [], 0
     for i, s in enumerate(specs):
@@ -458,7 +458,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet18_b64")
-    ap.add_argument("--mode", default="auto", choices=["auto", "off", "all", "channel"])
+    ap.add_argument("--mode", default="auto", choices=["auto", "off", "all", "channel", "tensor"])
     ap.add_argument("--rounding", type=int, default=0, choices=[0, 1],
                     help="1: random rounding of normal planes (runs on the general-purpose kernel)")
     ap.add_argument("--schedule", action="store_true",

@@ -86,9 +86,15 @@ typedef struct {
  * CHANNEL: the other reading of "classify channels" (Section 4.4.1) -- mu, sigma and the outlier count are
  * taken over the N planes of channel c together (same fixed-point sums, r = 1/(N*HW)) and the channel as a
  * whole, hence each of its planes, is normal or outlier-rich (n_out*rho_den > rho_num*N*HW); a plane's table
- * entry carries the plane's own count.  It costs three more passes over the tensor and is not available
- * through fh_compress_static. */
-typedef enum { FH_SALIENT_AUTO = 0, FH_SALIENT_OFF = 1, FH_SALIENT_ALL = 2, FH_SALIENT_CHANNEL = 3 } fh_salient_mode;
+ * entry carries the plane's own count.
+ * TENSOR: a third reading -- what counts as an outlier is fixed once for the whole tensor (mu and sigma over
+ * all N*C*HW elements, same fixed-point sums, r = 1/(N*C*HW)); a plane is outlier-rich when its own count of
+ * such outliers satisfies n_out*rho_den > rho_num*HW.
+ * CHANNEL and TENSOR cost three more passes over the tensor and are not available through
+ * fh_compress_static. */
+typedef enum {
+  FH_SALIENT_AUTO = 0, FH_SALIENT_OFF = 1, FH_SALIENT_ALL = 2, FH_SALIENT_CHANNEL = 3, FH_SALIENT_TENSOR = 4
+} fh_salient_mode;
 
 /* Codec parameters.  The paper names these quantities but prints no values (Section 4.4.1);
  * fh_default_params() fills the defaults given beside each field. */

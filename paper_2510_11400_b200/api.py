@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libfh_sm100a.so")
 FH_OK, FH_ERR_ARG, FH_ERR_UNSUPPORTED, FH_ERR_CAPACITY, FH_ERR_NONFINITE, FH_ERR_CORRUPT, \
     FH_ERR_TIMEOUT, FH_ERR_CUDA = 0, -1, -2, -3, -4, -5, -6, -7
 FH_F32, FH_BF16 = 0, 1
-FH_SALIENT_AUTO, FH_SALIENT_OFF, FH_SALIENT_ALL, FH_SALIENT_CHANNEL = 0, 1, 2, 3
+FH_SALIENT_AUTO, FH_SALIENT_OFF, FH_SALIENT_ALL, FH_SALIENT_CHANNEL, FH_SALIENT_TENSOR = 0, 1, 2, 3, 4
 FH_KEEP, FH_COMPRESS, FH_EVICT = 0, 1, 2
 FH_STATIC_MAX_PLANES = 131072
 

@@ -43,7 +43,7 @@ int check_desc(const fh_tensor_desc* d) {
 int check_params(const fh_params* p) {
   if (!p) return FH_ERR_ARG;
   if (p->bits != 2 && p->bits != 4 && p->bits != 8) return FH_ERR_UNSUPPORTED;
-  if (p->salient_mode < 0 || p->salient_mode > 3) return FH_ERR_ARG;
+  if (p->salient_mode < 0 || p->salient_mode > 4) return FH_ERR_ARG;
   if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FH_ERR_ARG;
   if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FH_ERR_ARG;
   if (p->block != 8 || p->dense_bits != 8 || (p->rounding != 0 && p->rounding != 1)) return FH_ERR_UNSUPPORTED;
@@ -534,14 +534,14 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   chunking(pl.P, &a.chunk_shift, &a.nchunks);
   a.chan_nout = nullptr;
   a.plane_nout = nullptr;
-  if (pl.mode == fh::kModeChannel) {  // statistics per channel over the batch: three passes ahead of the streaming kernel
+  if (pl.mode >= fh::kModeChannel) {  // statistics per channel over the batch, or over the tensor: three passes ahead of the streaming kernel
     rc = get_channel_scratch(s, pl.P, pl.C);
     if (rc != FH_OK) return rc;
     fh::ChannelArgs ca;
     ca.src = (const uint8_t*)d_src;
     ca.chan = s->chan;
     ca.plane_nout = s->plane_nout;
-    ca.inv_nhw = 1.0 / ((double)pl.N * (double)pl.HW);
+    ca.inv_nhw = 1.0 / ((double)(pl.mode == fh::kModeTensor ? pl.P : pl.N) * (double)pl.HW);
     rc = pl.dtype == FH_F32 ? launch_channel_passes<fh::kF32>(pl, ca, stream) : launch_channel_passes<fh::kBF16>(pl, ca, stream);
     if (rc != FH_OK) return rc;
     a.chan_nout = reinterpret_cast<const unsigned long long*>(s->chan) + 3;
@@ -817,7 +817,7 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   rc = make_plan(desc, params, true, &pl, &v);
   if (rc != FH_OK) return rc;
   if (pl.P > FH_STATIC_MAX_PLANES) return FH_ERR_UNSUPPORTED;  // beyond the fixed work list
-  if (pl.mode == fh::kModeChannel) return FH_ERR_UNSUPPORTED;  // its statistics need scratch the fixed array does not hold
+  if (pl.mode >= fh::kModeChannel) return FH_ERR_UNSUPPORTED;  // its statistics need scratch the fixed array does not hold
   cudaStream_t stream = (cudaStream_t)stream_;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FH_ERR_CUDA;

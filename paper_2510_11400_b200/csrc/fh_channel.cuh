@@ -1,5 +1,7 @@
 // Channel-wide three-sigma statistics (salient_mode = CHANNEL): mu, sigma and the outlier count are taken
 // over the N planes (n, c) of a channel c together, and the channel as a whole is normal or outlier-rich.
+// Tensor-wide statistics (salient_mode = TENSOR) run through the same passes with the whole tensor as the
+// one "channel"; a plane's class then follows from its own count.
 // Three passes over the tensor, a warp per plane, results gathered per channel with atomics:
 //   pass 0: minimum and maximum of the channel (they fix the fixed-point scale of the moment sums);
 //   pass 1: fixed-point moment sums of the channel (exact integers, so the order of the atomics is immaterial);
@@ -32,9 +34,9 @@ __device__ __forceinline__ float key_float(unsigned int k) {
 
 struct ChannelArgs {
   const uint8_t* src;
-  ChanStat* chan;        // C entries, zeroed before pass 0
+  ChanStat* chan;        // C entries (one in the tensor-wide mode), zeroed before pass 0
   uint32_t* plane_nout;  // P entries, written by pass 2
-  double inv_nhw;        // 1 / (N * HW)
+  double inv_nhw;        // 1 / (N * HW); tensor-wide: 1 / (N * C * HW)
 };
 
 template <int DT>
@@ -53,9 +55,16 @@ template <int DT, int PASS>
 __global__ void __launch_bounds__(kThreads) channel_pass(const Plan pl, const ChannelArgs a) {
   const uint32_t lane = threadIdx.x & 31u;
   const uint64_t warps = (uint64_t)gridDim.x * kWarps, first = (uint64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
+  // Tensor-wide statistics have a single destination: a warp gathers over its planes, the CTA's warps are
+  // combined in shared memory, and one thread per CTA issues the atomics.
+  const bool whole = pl.mode == kModeTensor;
+  __shared__ float s_lo[kWarps], s_hi[kWarps];
+  __shared__ long long s_s[kWarps], s_q[kWarps];
+  float wlo = __int_as_float(0x7F800000), whi = __int_as_float(0xFF800000);
+  long long ws = 0, wq = 0;
   for (uint64_t p = first; p < pl.P; p += warps) {
     const uint8_t* plane = a.src + p * pl.plane_bytes;
-    ChanStat* cs = a.chan + (p % pl.C);
+    ChanStat* cs = a.chan + (pl.mode == kModeTensor ? 0ull : p % pl.C);
     if (PASS == 0) {
       float lo = __int_as_float(0x7F800000), hi = __int_as_float(0xFF800000);
       for (uint32_t i = lane; i < pl.HW; i += 32u) {
@@ -68,7 +77,10 @@ __global__ void __launch_bounds__(kThreads) channel_pass(const Plan pl, const Ch
         lo = fminf(lo, __shfl_xor_sync(0xFFFFFFFFu, lo, o));
         hi = fmaxf(hi, __shfl_xor_sync(0xFFFFFFFFu, hi, o));
       }
-      if (lane == 0) {
+      if (whole) {
+        wlo = fminf(wlo, lo);
+        whi = fmaxf(whi, hi);
+      } else if (lane == 0) {
         atomicMax(&cs->lo_inv, ~float_key(lo));
         atomicMax(&cs->hi_key, float_key(hi));
       }
@@ -89,7 +101,10 @@ __global__ void __launch_bounds__(kThreads) channel_pass(const Plan pl, const Ch
           s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
           q += __shfl_xor_sync(0xFFFFFFFFu, q, o);
         }
-        if (lane == 0) {
+        if (whole) {
+          ws += s;
+          wq += q;
+        } else if (lane == 0) {
           atomicAdd(&cs->Is, (unsigned long long)s);
           atomicAdd(&cs->Iq, (unsigned long long)q);
         }
@@ -105,8 +120,33 @@ __global__ void __launch_bounds__(kThreads) channel_pass(const Plan pl, const Ch
         asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(cnt) : "r"(0xFFFFFFFFu));
         if (lane == 0) {
           a.plane_nout[p] = cnt;
-          if (cnt) atomicAdd(&cs->nout, (unsigned long long)cnt);
+          if (cnt && !whole) atomicAdd(&cs->nout, (unsigned long long)cnt);  // the tensor-wide mode classifies by the plane's count
         }
+      }
+    }
+  }
+  if (whole && PASS < 2) {
+    const uint32_t warp = threadIdx.x >> 5;
+    if (lane == 0) {
+      s_lo[warp] = wlo;
+      s_hi[warp] = whi;
+      s_s[warp] = ws;
+      s_q[warp] = wq;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (uint32_t k = 1; k < (uint32_t)kWarps; ++k) {
+        wlo = fminf(wlo, s_lo[k]);
+        whi = fmaxf(whi, s_hi[k]);
+        ws += s_s[k];
+        wq += s_q[k];
+      }
+      if (PASS == 0) {  // (every CTA of the grid owns at least one plane, so both values are finite numbers of the input)
+        atomicMax(&a.chan->lo_inv, ~float_key(wlo));
+        atomicMax(&a.chan->hi_key, float_key(whi));
+      } else {
+        atomicAdd(&a.chan->Is, (unsigned long long)ws);
+        atomicAdd(&a.chan->Iq, (unsigned long long)wq);
       }
     }
   }

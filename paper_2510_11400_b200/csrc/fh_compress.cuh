@@ -46,9 +46,12 @@ struct CompressArgs {
   const uint32_t* plane_nout;
 };
 
-// Class and outlier count of plane gp when mu and sigma are taken per channel over the batch.
+// Class and outlier count of plane gp when mu and sigma are taken per channel over the batch (the class is
+// the channel's) or over the whole tensor (the class follows from the plane's own count).
 __device__ __forceinline__ uint32_t channel_class(const Plan& pl, const CompressArgs& a, uint64_t gp, uint32_t& n_out) {
   n_out = a.plane_nout[gp];
+  if (pl.mode == kModeTensor)
+    return (uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW ? kClsSalient : kClsNormal;
   const unsigned long long total = a.chan_nout[(gp % pl.C) * 4ull];
   return total * pl.rho_den > (unsigned long long)pl.rho_num * pl.N * pl.HW ? kClsSalient : kClsNormal;
 }
@@ -454,7 +457,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
         if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * HW) cls = kClsSalient;
       } else if (pl.mode == kModeAll) {
         cls = kClsSalient;
-      } else if (pl.mode == kModeChannel) {
+      } else if (pl.mode >= kModeChannel) {
         cls = channel_class(pl, a, p0 + lp, n_out);
       }
 
@@ -666,7 +669,7 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
     if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
   } else if (pl.mode == kModeAll) {
     cls = kClsSalient;
-  } else if (pl.mode == kModeChannel) {
+  } else if (pl.mode >= kModeChannel) {
     cls = channel_class(pl, a, gp, n_out);
   }
 
@@ -1035,7 +1038,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
       if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
     } else {
       if (pl.mode == kModeAll) cls = kClsSalient;
-      if (pl.mode == kModeChannel) cls = channel_class(pl, a, gp, n_out);
+      if (pl.mode >= kModeChannel) cls = channel_class(pl, a, gp, n_out);
       __syncthreads();  // every thread is done with the stage
     }
     if (tid == 0) {

@@ -16,7 +16,7 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kMaxWarps = 16;            // largest CTA of any kernel: 512 threads
 constexpr uint32_t kMagic = 0x31434846u;  // "FHC1"
 constexpr uint32_t kClsNormal = 0, kClsSalient = 1, kClsRaw = 2;
-constexpr int kModeAuto = 0, kModeOff = 1, kModeAll = 2, kModeChannel = 3;
+constexpr int kModeAuto = 0, kModeOff = 1, kModeAll = 2, kModeChannel = 3, kModeTensor = 4;
 constexpr int kF32 = 0, kBF16 = 1;
 constexpr int kMaxStages = 4;
 constexpr float kMagicF = 12582912.0f;    // 1.5 * 2^23: fma(v, c, kMagicF) leaves rne(v*c) in the mantissa

@@ -504,3 +504,17 @@ def test_parity_channel_wide_three_sigma(shape, dtype):
         cls = hp.table(buf, shape[0] * shape[1])["cls"].reshape(shape[0], shape[1])
         assert ((cls != fho.NORMAL).all(0) | (cls == fho.NORMAL).all(0)).all()
     assert fho.parse_header(buf)["salient_mode"] == fho.CHANNEL
+
+
+@pytest.mark.parametrize("shape", [(6, 20, 14, 14), (3, 5, 7, 7), (4, 12, 32, 32), (5, 8, 28, 28), (3, 6, 56, 56), (2, 3, 112, 112),
+                                   (4, 6, 33, 17), (40, 7, 4, 4)])
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_parity_tensor_wide_three_sigma(shape, dtype):
+    """salient_mode = TENSOR: thresholds from the whole tensor's mu and sigma, class by each plane's own count;
+    container identical to the oracle's, both classes present on the spiky data."""
+    for kind, bits in (("spiky_relu", 2), ("laplace_ch", 8)):
+        spec = synth.TensorSpec("t", shape, dtype, kind, 84)
+        buf = full_parity(spec, bits=bits, salient_mode=api.FH_SALIENT_TENSOR)
+        t = hp.table(buf, shape[0] * shape[1])
+        assert ((t["cls"] != fho.NORMAL) == (t["n_out"].astype(np.int64) * 32 > shape[2] * shape[3])).all()
+    assert fho.parse_header(buf)["salient_mode"] == fho.TENSOR
