@@ -144,7 +144,9 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
       pl.ppt = fh::kThreads / pl.team;
     } else {
       v.cta = true;  // CTA size by plane size: enough work per thread between barriers
-      pl.team = pl.plane_bytes <= 16 * 1024 ? 128 : (pl.plane_bytes <= 32 * 1024 ? 256 : 512);
+      // (the per-plane reductions and scalar steps cost every warp the same, whatever its share of the plane:
+      // fewer, busier threads win as long as enough warps stay resident)
+      pl.team = pl.plane_bytes <= 16 * 1024 ? 128 : (pl.plane_bytes <= 64 * 1024 ? 256 : 512);
       v.G = 0;
       pl.ppt = 1;
     }

@@ -440,13 +440,25 @@ __device__ __forceinline__ void team_minmax(const Team& t, float& lo, float& hi,
       r[warp * 2 + 1] = hi;
     }
     __syncthreads();
-    lo = r[0];
-    hi = r[1];
-    for (uint32_t k = 1; k < t.nwarps; ++k) {
-      lo = min_nan(lo, r[k * 2]);
-      hi = max_nan(hi, r[k * 2 + 1]);
-    }
+    // second stage, lane k takes warp k's pair (a CTA has at most 32 warps): two more warp reductions
+    // instead of a walk over all pairs by every thread
+    const uint32_t k = min(threadIdx.x & 31u, t.nwarps - 1u);
+    const float2 pr = reinterpret_cast<const float2*>(r)[k];
+    lo = pr.x;
+    hi = pr.y;
+    asm volatile("redux.sync.min.NaN.f32 %0, %0, %1;" : "+f"(lo) : "r"(0xFFFFFFFFu));
+    asm volatile("redux.sync.max.NaN.f32 %0, %0, %1;" : "+f"(hi) : "r"(0xFFFFFFFFu));
   }
+}
+
+// Exact 64-bit sum over the warp of one int32 per lane: high and low halves are summed apart (neither sum
+// can overflow 32 bits) and put together again.
+__device__ __forceinline__ long long warp_sum_s32_wide(int32_t v) {
+  int32_t h = v >> 16;
+  uint32_t l = (uint32_t)v & 0xFFFFu;
+  asm volatile("redux.sync.add.s32 %0, %0, %1;" : "+r"(h) : "r"(0xFFFFFFFFu));
+  asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(l) : "r"(0xFFFFFFFFu));
+  return (long long)h * 65536ll + (long long)l;
 }
 
 // Sum of two int32 per thread over the team, returned as 64-bit integers.  The sums over one warp
@@ -463,19 +475,14 @@ __device__ __forceinline__ void team_sum2(const Team& t, int32_t a, int32_t b, l
   A = a;
   B = b;
   if (t.block) {
-    long long* r = reinterpret_cast<long long*>(red_half(t, rp));
-    const uint32_t warp = threadIdx.x >> 5;
-    if ((threadIdx.x & 31u) == 0) {
-      r[warp * 2] = a;
-      r[warp * 2 + 1] = b;
-    }
+    int2* r = reinterpret_cast<int2*>(red_half(t, rp));
+    const uint32_t warp = threadIdx.x >> 5, wl = threadIdx.x & 31u;
+    if (wl == 0) r[warp] = make_int2(a, b);
     __syncthreads();
-    A = 0;
-    B = 0;
-    for (uint32_t k = 0; k < t.nwarps; ++k) {
-      A += r[k * 2];
-      B += r[k * 2 + 1];
-    }
+    // second stage: lane k takes warp k's pair, the warp adds them up in 64 bits
+    const int2 pr = wl < t.nwarps ? r[wl] : make_int2(0, 0);
+    A = warp_sum_s32_wide(pr.x);
+    B = warp_sum_s32_wide(pr.y);
   }
 }
 
@@ -510,8 +517,8 @@ __device__ __forceinline__ uint32_t team_sum_u32(const Team& t, uint32_t v, uint
     const uint32_t warp = threadIdx.x >> 5;
     if ((threadIdx.x & 31u) == 0) r[warp] = v;
     __syncthreads();
-    v = 0;
-    for (uint32_t k = 0; k < t.nwarps; ++k) v += r[k];
+    v = (threadIdx.x & 31u) < t.nwarps ? r[threadIdx.x & 31u] : 0u;  // second stage: lane k takes warp k's sum
+    asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(v) : "r"(0xFFFFFFFFu));
   }
   return v;
 }
