@@ -153,7 +153,8 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
     pl.stage_bytes = (uint32_t)((pl.ppt * pl.plane_bytes + 127) & ~(uint64_t)127);
     uint32_t ns = (uint32_t)((v.cta ? kStageTarget : kWarpStageTarget) / pl.stage_bytes);
-    const uint32_t ns_max = v.cta ? 3u : (uint32_t)fh::kMaxStages;
+    // (CTA-team kernel: two stages; a third buys nothing that more resident CTAs do not give)
+    const uint32_t ns_max = v.cta ? 2u : (uint32_t)fh::kMaxStages;
     ns = ns < 2 ? 2 : (ns > ns_max ? ns_max : ns);
     for (;;) {
       pl.nstage = ns;
