@@ -487,14 +487,15 @@ uint64_t prime_at_most(uint64_t n) {
   return cache[n] = 1;
 }
 
-template <int DT, int TT>
+template <int DT, int TT, bool DEFER = false>
 int launch_decompress_t(const Plan& pl, const fh::DecompressArgs& a, cudaStream_t stream) {
+  if (TT == 32 && !DEFER && pl.nblk >= fh::kDeferBlocks) return launch_decompress_t<DT, TT, TT == 32>(pl, a, stream);
   int grid = 0;
-  int rc = grid_for(fh::decompress_kernel<DT, TT>, pl.sm_total, pl.ntiles, &grid);
+  int rc = grid_for(fh::decompress_kernel<DT, TT, DEFER>, pl.sm_total, pl.ntiles, &grid);
   if (rc != FH_OK) return rc;
   fh::DecompressArgs b = a;
   b.team_stride = prime_at_most((uint64_t)grid * (fh::kThreads / TT));
-  if (launch_dependent(fh::decompress_kernel<DT, TT>, grid, fh::kThreads, pl.sm_total, stream, pl, b) != cudaSuccess)
+  if (launch_dependent(fh::decompress_kernel<DT, TT, DEFER>, grid, fh::kThreads, pl.sm_total, stream, pl, b) != cudaSuccess)
     return FH_ERR_CUDA;
   g_launches.fetch_add(1);
   return FH_OK;

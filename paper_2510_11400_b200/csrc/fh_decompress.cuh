@@ -222,7 +222,10 @@ __device__ __forceinline__ void decode_small(const uint32_t (&cw)[8], uint32_t l
   }
 }
 
-template <int DT, int TT>
+constexpr uint32_t kDeferBlocks = 128;  // planes of at least this many 8x8 blocks: outlier-rich ones go to the whole CTA
+
+// DEFER: instantiated for whole-warp teams on planes of at least kDeferBlocks blocks.
+template <int DT, int TT, bool DEFER>
 __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, const DecompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
@@ -230,8 +233,17 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
   __shared__ float s_eps;
   __shared__ unsigned long long s_total;
   __shared__ Plan s_pl;  // copy for the outlined slow path, which takes it by address
+  // Outlier-rich planes of many blocks are not restored by the warp that meets them (one lane per block:
+  // nblk / 32 rounds of a long serial walk while the CTA's other warps wait at the exit) but put on this list
+  // and restored afterwards by the whole CTA, one lane per block.
+  constexpr uint32_t kDeferCap = 64;
+  __shared__ uint32_t s_defer[kDeferCap];
+  __shared__ uint32_t s_ndefer;
   const uint32_t tid = threadIdx.x;
-  if (tid == 0) s_pl = pl;
+  if (tid == 0) {
+    s_pl = pl;
+    s_ndefer = 0;
+  }
   dep_trigger();  // the next kernel on the stream may become resident as this one drains
   dep_wait();     // the previous kernel on the stream (the one that wrote the container) has completed
   const unsigned long long off_in = a.d_off_in ? *a.d_off_in : 0ull;
@@ -345,12 +357,47 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
           for (uint32_t i = lane; i < (uint32_t)(pl.plane_bytes >> 1); i += TT)
             reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)in.ld16(2u * i);
         } else {
+          if (DEFER) {
+            uint32_t at = 0;
+            if (lane == 0) at = atomicAdd(&s_ndefer, 1u);
+            at = __shfl_sync(0xFFFFFFFFu, at, 0);
+            if (at < kDeferCap) {
+              if (lane == 0) s_defer[at] = (uint32_t)gp;
+              continue;
+            }
+          }
           uint32_t* scr = reinterpret_cast<uint32_t*>(smem) + (uint64_t)my_team * pl.nblk;
           if (!decode_salient<DT>(team, s_pl, in, ovf_avail, eps, out, scr)) bad = true;
         }
       } else {
         bad = true;
       }
+    }
+  }
+  if (DEFER && hdr_ok) {  // (uniform over the CTA)
+    __syncthreads();
+    const uint32_t n = min(s_ndefer, kDeferCap);
+    const Team cta = make_team(kThreads, s_red);
+    const uint32_t bits = s_bits;
+    const uint32_t npay = a16(4u * ((pl.HW * bits + 31u) / 32u));
+    const unsigned long long total = s_total;
+    const unsigned long long slots_off = 64ull + 16ull * pl.P, ovf_off = slots_off + pl.P * (unsigned long long)npay;
+    for (uint32_t q = 0; q < n; ++q) {
+      const uint64_t gp = s_defer[q];
+      const uint4 e = __ldg(reinterpret_cast<const uint4*>(src + 64) + gp);
+      const unsigned long long off = (unsigned long long)e.x * 16ull;
+      if (off != 0 && (off < ovf_off || off > total)) {  // (the same for every thread)
+        bad = true;
+        continue;
+      }
+      SplitIn in;
+      in.slot = src + slots_off + gp * npay;
+      in.ovf = src + off;
+      in.npay = npay;
+      if (!decode_salient<DT>(cta, s_pl, in, off ? total - off : 0ull, s_eps, a.dst + gp * pl.plane_bytes,
+                              reinterpret_cast<uint32_t*>(smem)))
+        bad = true;
+      __syncthreads();  // the scratch is reused
     }
   }
   if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
