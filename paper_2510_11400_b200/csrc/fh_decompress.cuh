@@ -163,8 +163,8 @@ __device__ __forceinline__ void store_group(uint8_t* out, uint32_t g, float v0, 
     reinterpret_cast<float4*>(out)[g] = make_float4(v0, v1, v2, v3);
   } else {
     uint2 w;
-    w.x = f32_to_bf16_bits(v0) | (f32_to_bf16_bits(v1) << 16);
-    w.y = f32_to_bf16_bits(v2) | (f32_to_bf16_bits(v3) << 16);
+    w.x = f32x2_to_bf16x2(v0, v1);
+    w.y = f32x2_to_bf16x2(v2, v3);
     reinterpret_cast<uint2*>(out)[g] = w;
   }
 }

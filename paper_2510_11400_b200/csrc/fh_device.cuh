@@ -195,9 +195,17 @@ __device__ __forceinline__ float max3_nan(float a, float b, float c) {
 
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h) { return __uint_as_float(h << 16); }
 // fp32 -> bf16 bits, round half to even (finite inputs).
+// fp32 -> bf16, round to nearest even (the hardware conversion; the values converted here are never NaN).
 __device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
-  uint32_t u = __float_as_uint(f);
-  return (u + (((u >> 16) & 1u) + 0x7FFFu)) >> 16;
+  uint16_t r;
+  asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(f));
+  return r;
+}
+// Two at once: `lo` lands in the low half of the word.
+__device__ __forceinline__ uint32_t f32x2_to_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
 }
 
 template <int DT>
