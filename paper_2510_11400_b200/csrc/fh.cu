@@ -65,8 +65,8 @@ uint32_t pow2_ceil(uint32_t x) {
 
 // Which kernel a plan runs on.
 struct Variant {
-  bool fast = false;  // compress_fast (register-resident groups, bulk-copy pipeline)
-  bool cta = false;   // fast: one plane per CTA instead of one plane per sub-warp team
+  bool fast = false;  // compress_warp / compress_cta (bulk-copy pipeline) instead of compress_generic
+  bool cta = false;   // fast: compress_cta (one plane per CTA) instead of compress_warp (one plane per team of lanes)
   int G = 0;          // fast: groups per thread
 };
 

@@ -863,7 +863,9 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
 // CTA-team kernel: planes of more than 256 groups (whole 16-byte chunks).  One plane per tile, all
 // NT threads of the CTA work on it.  The plane stays in its shared-memory stage and is swept two or
 // three times (min/max; fixed-point moments; count + codes), so that few registers are needed and
-// several CTAs fit an SM.  Thread 0 keeps the next ticket in flight while the CTA works.
+// shared memory alone limits how many CTAs fit an SM (two stages each).  What every warp repeats per
+// plane -- reductions, thresholds, quantiser parameters -- does not shrink with the warp's share of the
+// plane, so NT is kept small for small planes.  Thread 0 keeps the next ticket in flight while the CTA works.
 // -------------------------------------------------------------------------------------------------
 template <int DT>
 __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, float (&v)[4]) {
