@@ -138,112 +138,44 @@ size_t fho_compressed_bytes(const fho_desc* d, const fho_params* p, int which) {
 }
 
 /* ------------------------------------------------------------------------------------------
- * Three-sigma statistics of one plane (Section 4.4.1: "Outliers are identified using the
- * empirical 3-sigma rule").  mu and sigma are taken over the plane.
+ * Three-sigma statistics (Section 4.4.1: outliers are found with the empirical three-sigma rule).
+ * mu and sigma are the mean and the population standard deviation of the elements in scope (a plane;
+ * a channel over the batch; the whole tensor).
  *
- * The paper does not say how the moments are accumulated.  Here they are accumulated in fixed
- * point, which makes the result exactly independent of the order of summation (so that any
- * parallel implementation reproduces it bit for bit):
- *   A   = max(|min x|, |max x|),  e = unbiased exponent field of A  (2^e <= A < 2^(e+1))
- *   c_s = 2^k_s, k_s = min(18 - e, 126);   c_q = 2^k_q, k_q = clamp(16 - 2e, -126, 126)
- *   per group of 4 consecutive elements (tail padded with zeros), in fp32:
- *     s_g = (x0+x1)+(x2+x3),  q_g = fma(x1,x1,x0*x0) + fma(x3,x3,x2*x2)
- *     i_s = round_half_even(s_g * c_s),  i_q = round_half_even(q_g * c_q)      (|.| < 2^21)
- *     taken as the mantissa of fma(s_g, c_s, 1.5*2^23): bits(result) - bits(1.5*2^23)
- *   I_s = sum i_s, I_q = sum i_q                                                (exact integers)
- *   r = 1/HW (fp64);  mu = (I_s * 2^-k_s) * r;  m2 = (I_q * 2^-k_q) * r          (fp64)
- *   var = max(m2 - mu*mu, 0)                                                     (fp64)
- *   mu_f = (float)mu, sigma_f = sqrtf((float)var)
- *   T_hi = fma(3, sigma_f, mu_f), T_lo = fma(-3, sigma_f, mu_f)                  (fp32)
- *   n_out = #{ x > T_hi or x < T_lo }                                           (fp32 compares)
+ * The paper does not say how the moments are accumulated.  Two requirements shape the reading taken
+ * here: the rule must hold on data with an offset (|mu| much larger than sigma, e.g. a biased
+ * pre-activation), so the moments are taken of the distances d = x - lo from the smallest element
+ * and never of x itself; and the result must not depend on the order of summation (so that a parallel
+ * implementation reproduces it bit for bit), so the sums run over integers:
+ *   lo = min x, hi = max x, range = hi - lo (fp32), e = floor(log2(range))
+ *   range == 0 (constant data): no outliers.
+ *   e < -40 or e > 60 (range below 2^-40 or from 2^61 up): the rule is not applied, no outliers are
+ *       counted -- inside [-40, 60] neither d*d nor the scalings below can overflow or underflow.
+ *   d_i = x_i - lo (fp32, >= 0); elements are taken in consecutive groups of 4 per plane, the last
+ *       group of a plane padded with d = 0; per group, in fp32:
+ *     s_g = (d0 + d1) + (d2 + d3),   q_g = fma(d1, d1, d0*d0) + fma(d3, d3, d2*d2)
+ *     i_s = round_half_even(s_g * 2^(18-e)),  i_q = round_half_even(q_g * 2^(16-2e))   (exact products,
+ *       integers below 2^22: the sums resolve 2^-18 of the range and 2^-16 of its square per group)
+ *   I_s = sum i_s, I_q = sum i_q                                          (exact integers, any order)
+ *   r = 1/count (fp64);  m1 = (I_s * 2^(e-18)) * r;  m2 = (I_q * 2^(2e-16)) * r            (fp64)
+ *   var = max(m2 - m1*m1, 0) (fp64);  m_f = (float)m1;  sigma_f = sqrtf((float)var)
+ *   D_hi = fma(3, sigma_f, m_f),  D_lo = fma(-3, sigma_f, m_f)                             (fp32)
+ *   element i is an outlier iff d_i > D_hi or d_i < D_lo                           (fp32 compares)
+ * i.e. x_i > mu + 3 sigma or x_i < mu - 3 sigma with mu = lo + m1, written in distances from lo.
  * ------------------------------------------------------------------------------------------ */
-static int32_t fixed_point(float v, float c) {
-  const float M = 12582912.0f; /* 1.5 * 2^23: adding it leaves the rounded integer in the mantissa */
-  float r = fmaf(v, c, M);
-  uint32_t rb, mb;
-  memcpy(&rb, &r, 4);
-  memcpy(&mb, &M, 4);
-  return (int32_t)(rb - mb);
-}
+typedef struct {
+  float lo, range;
+  int applies;    /* 0: constant data or range outside [2^-40, 2^61): no outliers are counted */
+  int e;
+  int64_t Is, Iq; /* the integer sums */
+  float d_lo, d_hi;
+} sigma_stats;
 
-static float pow2f(int k) { /* 2^k for -126 <= k <= 127 */
-  uint32_t b = (uint32_t)(k + 127) << 23;
-  float f;
-  memcpy(&f, &b, 4);
-  return f;
-}
+/* round_half_even(v * 2^k) as an integer; the product of a float with a power of two is exact in fp64 */
+static int64_t fixed_point(float v, int k) { return (int64_t)nearbyint(ldexp((double)v, k)); }
 
-void fho_plane_sums(const float* x, int64_t hw, int64_t* Is_out, int64_t* Iq_out, int32_t* ks_out,
-                    int32_t* kq_out) {
-  float lo = x[0], hi = x[0];
-  for (int64_t i = 1; i < hw; ++i) {
-    if (x[i] < lo) lo = x[i];
-    if (x[i] > hi) hi = x[i];
-  }
-  float A = fmaxf(fabsf(lo), fabsf(hi));
-  uint32_t ab;
-  memcpy(&ab, &A, 4);
-  int e = (int)((ab >> 23) & 255u) - 127;
-  int ks = 18 - e, kq = 16 - 2 * e;
-  if (ks > 126) ks = 126;
-  if (kq > 126) kq = 126;
-  if (kq < -126) kq = -126;
-  float cs = pow2f(ks), cq = pow2f(kq);
-  int64_t Is = 0, Iq = 0;
-  for (int64_t g = 0; g < hw; g += 4) {
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int k = 0; k < 4 && g + k < hw; ++k) v[k] = x[g + k];
-    float s01 = v[0] + v[1], s23 = v[2] + v[3];
-    float sg = s01 + s23;
-    float p0 = v[0] * v[0], p2 = v[2] * v[2];
-    float q01 = fmaf(v[1], v[1], p0), q23 = fmaf(v[3], v[3], p2);
-    float qg = q01 + q23;
-    Is += fixed_point(sg, cs);
-    Iq += fixed_point(qg, cq);
-  }
-  *Is_out = Is;
-  *Iq_out = Iq;
-  *ks_out = ks;
-  *kq_out = kq;
-}
-
-void fho_plane_sigma(const float* x, int64_t hw, double* S_out, double* Q_out, float* t_lo,
-                     float* t_hi, int64_t* n_out) {
-  int64_t Is, Iq;
-  int32_t ks, kq;
-  fho_plane_sums(x, hw, &Is, &Iq, &ks, &kq);
-  double S = ldexp((double)Is, -ks), Q = ldexp((double)Iq, -kq);
-  double r = 1.0 / (double)hw;
-  double mu = S * r;
-  double m2 = Q * r;
-  double mu2 = mu * mu;
-  double var = m2 - mu2;
-  if (!(var > 0.0)) var = 0.0;
-  float mu_f = (float)mu;
-  float sigma_f = sqrtf((float)var);
-  float thi = fmaf(3.0f, sigma_f, mu_f);
-  float tlo = fmaf(-3.0f, sigma_f, mu_f);
-  int64_t cnt = 0;
-  for (int64_t i = 0; i < hw; ++i)
-    if (x[i] > thi || x[i] < tlo) ++cnt;
-  *S_out = S;
-  *Q_out = Q;
-  *t_lo = tlo;
-  *t_hi = thi;
-  *n_out = cnt;
-}
-
-/* ------------------------------------------------------------------------------------------
- * The other reading of "classify channels" (Section 4.4.1): a channel is channel c of the layer, i.e.
- * the N planes (n, c) of the batch together.  mu and sigma are then taken over all N*HW elements of
- * the channel, with the same fixed-point accumulation as above (A = largest magnitude of the channel;
- * every plane is cut into its own groups of four, tail padded with zeros; r = 1/(N*HW)); the count
- * runs over the whole channel and the channel, hence each of its planes, is outlier-rich when
- * n_out * rho_den > rho_num * N * HW.  A plane's table entry carries the plane's own count.
- * x: N planes of channel c, each hw elements, plane n at x + n*stride.
- * ------------------------------------------------------------------------------------------ */
-void fho_channel_sigma(const float* x, int64_t n_planes, int64_t stride, int64_t hw, float* t_lo, float* t_hi,
-                       int64_t* n_out) {
+/* Integer sums of the distances from lo of n_planes planes of hw elements (plane n at x + n*stride). */
+static void sigma_sums(const float* x, int64_t n_planes, int64_t stride, int64_t hw, sigma_stats* st) {
   float lo = x[0], hi = x[0];
   for (int64_t n = 0; n < n_planes; ++n)
     for (int64_t i = 0; i < hw; ++i) {
@@ -251,43 +183,94 @@ void fho_channel_sigma(const float* x, int64_t n_planes, int64_t stride, int64_t
       if (v < lo) lo = v;
       if (v > hi) hi = v;
     }
-  float A = fmaxf(fabsf(lo), fabsf(hi));
-  uint32_t ab;
-  memcpy(&ab, &A, 4);
-  int e = (int)((ab >> 23) & 255u) - 127;
-  int ks = 18 - e, kq = 16 - 2 * e;
-  if (ks > 126) ks = 126;
-  if (kq > 126) kq = 126;
-  if (kq < -126) kq = -126;
-  float cs = pow2f(ks), cq = pow2f(kq);
-  int64_t Is = 0, Iq = 0;
+  memset(st, 0, sizeof(*st));
+  st->lo = lo;
+  st->range = hi - lo;
+  if (!(st->range > 0.0f)) return;
+  st->e = ilogbf(st->range);
+  if (st->e < -40 || st->e > 60) return;
+  st->applies = 1;
   for (int64_t n = 0; n < n_planes; ++n)
     for (int64_t g = 0; g < hw; g += 4) {
-      float v[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int k = 0; k < 4 && g + k < hw; ++k) v[k] = x[n * stride + g + k];
-      float s01 = v[0] + v[1], s23 = v[2] + v[3];
+      float d[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int k = 0; k < 4 && g + k < hw; ++k) d[k] = x[n * stride + g + k] - lo;
+      float s01 = d[0] + d[1], s23 = d[2] + d[3];
       float sg = s01 + s23;
-      float p0 = v[0] * v[0], p2 = v[2] * v[2];
-      float q01 = fmaf(v[1], v[1], p0), q23 = fmaf(v[3], v[3], p2);
+      float p0 = d[0] * d[0], p2 = d[2] * d[2];
+      float q01 = fmaf(d[1], d[1], p0), q23 = fmaf(d[3], d[3], p2);
       float qg = q01 + q23;
-      Is += fixed_point(sg, cs);
-      Iq += fixed_point(qg, cq);
+      st->Is += fixed_point(sg, 18 - st->e);
+      st->Iq += fixed_point(qg, 16 - 2 * st->e);
     }
-  double S = ldexp((double)Is, -ks), Q = ldexp((double)Iq, -kq);
-  double r = 1.0 / (double)(n_planes * hw);
-  double mu = S * r, m2 = Q * r, mu2 = mu * mu;
-  double var = m2 - mu2;
+}
+
+static void sigma_thresholds(sigma_stats* st, int64_t count) {
+  double S = ldexp((double)st->Is, st->e - 18), Q = ldexp((double)st->Iq, 2 * st->e - 16);
+  double r = 1.0 / (double)count;
+  double m1 = S * r;
+  double m2 = Q * r;
+  double m1sq = m1 * m1;
+  double var = m2 - m1sq;
   if (!(var > 0.0)) var = 0.0;
-  float mu_f = (float)mu, sigma_f = sqrtf((float)var);
-  float thi = fmaf(3.0f, sigma_f, mu_f), tlo = fmaf(-3.0f, sigma_f, mu_f);
+  float m_f = (float)m1;
+  float sigma_f = sqrtf((float)var);
+  st->d_hi = fmaf(3.0f, sigma_f, m_f);
+  st->d_lo = fmaf(-3.0f, sigma_f, m_f);
+}
+
+static int64_t sigma_count(const float* x, int64_t hw, const sigma_stats* st) {
+  if (!st->applies) return 0;
   int64_t cnt = 0;
-  for (int64_t n = 0; n < n_planes; ++n)
-    for (int64_t i = 0; i < hw; ++i) {
-      float v = x[n * stride + i];
-      if (v > thi || v < tlo) ++cnt;
-    }
-  *t_lo = tlo;
-  *t_hi = thi;
+  for (int64_t i = 0; i < hw; ++i) {
+    float d = x[i] - st->lo;
+    if (d > st->d_hi || d < st->d_lo) ++cnt;
+  }
+  return cnt;
+}
+
+/* Exposed for the tests: the integer sums of one plane and the exponent they are scaled by. */
+void fho_plane_sums(const float* x, int64_t hw, int64_t* Is_out, int64_t* Iq_out, int32_t* e_out,
+                    int32_t* applies_out) {
+  sigma_stats st;
+  sigma_sums(x, 1, hw, hw, &st);
+  *Is_out = st.Is;
+  *Iq_out = st.Iq;
+  *e_out = st.e;
+  *applies_out = st.applies;
+}
+
+/* One plane: lo, the thresholds as distances from lo, and the outlier count. */
+void fho_plane_sigma(const float* x, int64_t hw, float* lo_out, float* d_lo, float* d_hi, int64_t* n_out) {
+  sigma_stats st;
+  sigma_sums(x, 1, hw, hw, &st);
+  if (st.applies) sigma_thresholds(&st, hw);
+  *lo_out = st.lo;
+  *d_lo = st.d_lo;
+  *d_hi = st.d_hi;
+  *n_out = sigma_count(x, hw, &st);
+}
+
+/* ------------------------------------------------------------------------------------------
+ * The other readings of "classify channels" (Section 4.4.1): a channel is channel c of the layer, i.e.
+ * the N planes (n, c) of the batch together (salient_mode CHANNEL), or what counts as an outlier is
+ * fixed once for the whole tensor (TENSOR).  lo, range, the integer sums (every plane cut into its own
+ * groups of four) and the divisor then run over all planes in scope.
+ * x: n_planes planes, each hw elements, plane n at x + n*stride.
+ * ------------------------------------------------------------------------------------------ */
+static void scope_sigma(const float* x, int64_t n_planes, int64_t stride, int64_t hw, sigma_stats* st) {
+  sigma_sums(x, n_planes, stride, hw, st);
+  if (st->applies) sigma_thresholds(st, n_planes * hw);
+}
+
+void fho_channel_sigma(const float* x, int64_t n_planes, int64_t stride, int64_t hw, float* lo_out, float* d_lo,
+                       float* d_hi, int64_t* n_out) {
+  sigma_stats st;
+  scope_sigma(x, n_planes, stride, hw, &st);
+  int64_t cnt = 0;
+  for (int64_t n = 0; n < n_planes; ++n) cnt += sigma_count(x + n * stride, hw, &st);
+  *lo_out = st.lo;
+  *d_lo = st.d_lo;
+  *d_hi = st.d_hi;
   *n_out = cnt;
 }
 
@@ -529,10 +512,10 @@ static size_t encode_salient(const float* x, const uint8_t* raw, int dtype, int 
   return size;
 }
 
-/* ch: for MODE_CHANNEL the channel's {t_lo, t_hi} and whether the channel is outlier-rich; for MODE_TENSOR the
+/* ch: for MODE_CHANNEL the channel's statistics and whether the channel is outlier-rich; for MODE_TENSOR the
  * tensor's {t_lo, t_hi} (a plane is then outlier-rich by its own count against these); NULL otherwise */
 typedef struct {
-  float tlo, thi;
+  sigma_stats st;
   int salient;
 } channel_info;
 
@@ -557,26 +540,23 @@ static void encode_plane(const uint8_t* raw, int dtype, int H, int W, const fho_
   }
   uint32_t cls = CLS_NORMAL, n_out = 0;
   if (p->salient_mode == MODE_AUTO) {
-    double S, Q;
-    float tlo, thi;
+    float plo, dlo, dhi;
     int64_t cnt;
-    fho_plane_sigma(x, (int64_t)hw, &S, &Q, &tlo, &thi, &cnt);
+    fho_plane_sigma(x, (int64_t)hw, &plo, &dlo, &dhi, &cnt);
     n_out = (uint32_t)cnt;
     /* outlier-rich when the three-sigma outliers exceed the fraction rho of the plane */
     if ((int64_t)cnt * p->rho_den > (int64_t)p->rho_num * (int64_t)hw) cls = CLS_SALIENT;
   } else if (p->salient_mode == MODE_ALL) {
     cls = CLS_SALIENT;
   } else if (p->salient_mode == MODE_CHANNEL) {
-    for (size_t i = 0; i < hw; ++i)
-      if (x[i] > ch->thi || x[i] < ch->tlo) ++n_out;
+    n_out = (uint32_t)sigma_count(x, (int64_t)hw, &ch->st);
     if (ch->salient) cls = CLS_SALIENT;
   } else if (p->salient_mode == MODE_TENSOR) {
     /* Third reading of the three-sigma rule (Section 4.4.1): what counts as an outlier is fixed once for the
-     * layer's whole activation tensor (mu and sigma over all N*C*HW elements, same fixed-point sums with
-     * A = the tensor's largest magnitude and r = 1/(N*C*HW)); a plane is outlier-rich when its own share of
+     * layer's whole activation tensor (mu and sigma over all N*C*HW elements, the same integer sums with lo and range
+     * of the tensor and r = 1/(N*C*HW)); a plane is outlier-rich when its own share of
      * such outliers exceeds rho. */
-    for (size_t i = 0; i < hw; ++i)
-      if (x[i] > ch->thi || x[i] < ch->tlo) ++n_out;
+    n_out = (uint32_t)sigma_count(x, (int64_t)hw, &ch->st);
     if ((int64_t)n_out * p->rho_den > (int64_t)p->rho_num * (int64_t)hw) cls = CLS_SALIENT;
   }
   if (cls == CLS_SALIENT) {
@@ -651,10 +631,10 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
         }
       if (!finite) {
         bad = 1; /* reported per plane below */
-        chan[c].tlo = chan[c].thi = 0.0f;
       } else {
-        int64_t cnt;
-        fho_channel_sigma(x, d->n, (int64_t)hw, (int64_t)hw, &chan[c].tlo, &chan[c].thi, &cnt);
+        scope_sigma(x, d->n, (int64_t)hw, (int64_t)hw, &chan[c].st);
+        int64_t cnt = 0;
+        for (int64_t n = 0; n < (int64_t)d->n; ++n) cnt += sigma_count(x + (size_t)n * hw, (int64_t)hw, &chan[c].st);
         chan[c].salient = cnt * (int64_t)p->rho_den > (int64_t)p->rho_num * (int64_t)d->n * (int64_t)hw;
       }
       free(x);
@@ -668,10 +648,8 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
       x[i] = d->dtype == FHO_F32 ? ((const float*)src)[i] : bf16_to_f32(((const uint16_t*)src)[i]);
       if (!isfinite(x[i])) finite = 0;
     }
-    if (finite) { /* otherwise the planes report the error below */
-      int64_t cnt;
-      fho_channel_sigma(x, (int64_t)P, (int64_t)hw, (int64_t)hw, &chan[0].tlo, &chan[0].thi, &cnt);
-    }
+    if (finite) /* otherwise the planes report the error below */
+      scope_sigma(x, (int64_t)P, (int64_t)hw, (int64_t)hw, &chan[0].st);
     free(x);
   }
 #ifdef _OPENMP

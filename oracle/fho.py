@@ -69,12 +69,11 @@ def lib():
         L.fho_decompress.restype = C.c_int
         L.fho_decompress.argtypes = [C.c_void_p, C.c_size_t, C.POINTER(Desc), C.c_void_p]
         L.fho_plane_sigma.restype = None
-        L.fho_plane_sigma.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_double),
-                                      C.POINTER(C.c_double), C.POINTER(C.c_float),
+        L.fho_plane_sigma.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_float), C.POINTER(C.c_float),
                                       C.POINTER(C.c_float), C.POINTER(C.c_int64)]
         L.fho_channel_sigma.restype = None
         L.fho_channel_sigma.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.POINTER(C.c_float),
-                                        C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+                                        C.POINTER(C.c_float), C.POINTER(C.c_float), C.POINTER(C.c_int64)]
         L.fho_plane_sums.restype = None
         L.fho_plane_sums.argtypes = [C.c_void_p, C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int64),
                                      C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
@@ -130,31 +129,33 @@ def decompress(packed: np.ndarray, d: Desc, nbytes: int | None = None) -> Tuple[
 
 
 def plane_sigma(x: np.ndarray):
+    """Three-sigma statistics of one plane: (lo, d_lo, d_hi, n_out) -- the smallest element, the two
+    thresholds as fp32 distances from it, and the number of elements outside them."""
     x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
-    S, Q = C.c_double(), C.c_double()
-    tlo, thi = C.c_float(), C.c_float()
+    lo, dlo, dhi = C.c_float(), C.c_float(), C.c_float()
     n = C.c_int64()
-    lib().fho_plane_sigma(x.ctypes.data, x.size, C.byref(S), C.byref(Q), C.byref(tlo), C.byref(thi),
-                          C.byref(n))
-    return S.value, Q.value, tlo.value, thi.value, n.value
+    lib().fho_plane_sigma(x.ctypes.data, x.size, C.byref(lo), C.byref(dlo), C.byref(dhi), C.byref(n))
+    return lo.value, dlo.value, dhi.value, n.value
 
 
 def channel_sigma(x: np.ndarray):
-    """x: (n_planes, hw) float32, the planes of one channel over the batch.  Returns (t_lo, t_hi, n_out)."""
+    """x: (n_planes, hw) float32, the planes in scope (a channel over the batch, or a whole tensor).
+    Returns (lo, d_lo, d_hi, n_out)."""
     x = np.ascontiguousarray(x, dtype=np.float32)
-    tlo, thi = C.c_float(), C.c_float()
+    lo, dlo, dhi = C.c_float(), C.c_float(), C.c_float()
     n = C.c_int64()
-    lib().fho_channel_sigma(x.ctypes.data, x.shape[0], x.shape[1], x.shape[1], C.byref(tlo), C.byref(thi), C.byref(n))
-    return tlo.value, thi.value, n.value
+    lib().fho_channel_sigma(x.ctypes.data, x.shape[0], x.shape[1], x.shape[1], C.byref(lo), C.byref(dlo), C.byref(dhi),
+                            C.byref(n))
+    return lo.value, dlo.value, dhi.value, n.value
 
 
 def plane_sums(x: np.ndarray):
-    """Fixed-point moment sums of a plane: (I_s, I_q, k_s, k_q)."""
+    """Integer moment sums of a plane's distances from its minimum: (I_s, I_q, e, applies)."""
     x = np.ascontiguousarray(x, dtype=np.float32).reshape(-1)
     a, b = C.c_int64(), C.c_int64()
-    ks, kq = C.c_int32(), C.c_int32()
-    lib().fho_plane_sums(x.ctypes.data, x.size, C.byref(a), C.byref(b), C.byref(ks), C.byref(kq))
-    return a.value, b.value, ks.value, kq.value
+    e, ap = C.c_int32(), C.c_int32()
+    lib().fho_plane_sums(x.ctypes.data, x.size, C.byref(a), C.byref(b), C.byref(e), C.byref(ap))
+    return a.value, b.value, e.value, ap.value
 
 
 def quant_params(lo: float, hi: float, bits: int):

@@ -12,18 +12,28 @@ def test_channel_thresholds_and_count_against_numpy_float64():
     for n, hw in ((4, 49), (8, 196), (3, 1024), (16, 16)):
         x = rng.standard_normal((n, hw)).astype(np.float32)
         x[rng.random((n, hw)) < 0.02] *= 6.0
-        tlo, thi, cnt = fho.channel_sigma(x)
+        lo, dlo, dhi, cnt = fho.channel_sigma(x)
+        tlo, thi = float(lo) + dlo, float(lo) + dhi
         mu, sd = x.astype(np.float64).mean(), x.astype(np.float64).std()
-        assert abs(thi - (mu + 3 * sd)) < 1e-5 * max(1.0, abs(thi)) and abs(tlo - (mu - 3 * sd)) < 1e-5 * max(1.0, abs(tlo))
-        margin = 1e-5 * max(abs(tlo), abs(thi))
+        span = float(x.max()) - float(x.min())
+        assert abs(thi - (mu + 3 * sd)) < 1e-5 * span and abs(tlo - (mu - 3 * sd)) < 1e-5 * span
+        margin = 2e-5 * span
         near = ((np.abs(x - thi) < margin) | (np.abs(x - tlo) < margin)).sum()
         want = int(((x > mu + 3 * sd) | (x < mu - 3 * sd)).sum())
         assert abs(cnt - want) <= near
         assert cnt <= x.size / 9          # Chebyshev
     # one plane: the channel is the plane
     x = rng.standard_normal((1, 256)).astype(np.float32)
-    _, _, tlo_p, thi_p, cnt_p = fho.plane_sigma(x[0])
-    assert fho.channel_sigma(x) == (tlo_p, thi_p, cnt_p)
+    assert fho.channel_sigma(x) == fho.plane_sigma(x[0])
+    # a channel far from zero: the same plain answer (moments of the distances from the channel's minimum)
+    x = (500.0 + 0.05 * rng.standard_normal((8, 196))).astype(np.float32)
+    x[rng.random((8, 196)) < 0.02] += 1.0
+    lo, dlo, dhi, cnt = fho.channel_sigma(x)
+    mu, sd = x.astype(np.float64).mean(), x.astype(np.float64).std()
+    span = float(x.max()) - float(x.min())
+    assert abs(float(lo) + dhi - (mu + 3 * sd)) < 1e-5 * span and abs(float(lo) + dlo - (mu - 3 * sd)) < 1e-5 * span
+    near = ((np.abs(x - (mu + 3 * sd)) < 2e-5 * span) | (np.abs(x - (mu - 3 * sd)) < 2e-5 * span)).sum()
+    assert abs(cnt - int(((x > mu + 3 * sd) | (x < mu - 3 * sd)).sum())) <= near and cnt > 0
 
 
 def test_batch_of_one_reduces_to_the_per_plane_mode():
@@ -50,7 +60,7 @@ def test_one_class_per_channel_and_counts_add_up():
     x = raw.reshape(6, 20, 196)
     for c in range(20):
         assert len(set((cls[:, c] != fho.NORMAL).tolist())) == 1          # the whole channel or none of it
-        tlo, thi, cnt = fho.channel_sigma(x[:, c])
+        cnt = fho.channel_sigma(x[:, c])[3]
         assert int(t["n_out"].reshape(6, 20)[:, c].sum()) == cnt
         assert (cls[0, c] != fho.NORMAL) == (cnt * 32 > 6 * 196)
     assert (cls[:, 0] != fho.NORMAL).all() and (cls[:, 16] != fho.NORMAL).all() and (cls[:, 1:16] == fho.NORMAL).all()

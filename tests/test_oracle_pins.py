@@ -294,84 +294,151 @@ def test_sigma_hand_case_spike():
     exp = golden()["sigma_spike"][1].split()
     x = np.zeros(16, dtype=np.float32)
     x[5] = 16
-    S, Q, tlo, thi, n = fho.plane_sigma(x)
-    assert (S, Q) == (16.0, 256.0)
+    lo, dlo, dhi, n = fho.plane_sigma(x)
+    Is, Iq, e, applies = fho.plane_sums(x)
+    assert (lo, e, applies) == (0.0, 4, 1)
+    assert (Is * 2.0 ** (e - 18), Iq * 2.0 ** (2 * e - 16)) == (16.0, 256.0)     # sum d, sum d^2
     assert n == int(exp[1])
-    assert abs(thi - float(exp[5])) < 1e-5 and abs(tlo - float(exp[7])) < 1e-5
+    assert abs(lo + dhi - float(exp[5])) < 1e-5 and abs(lo + dlo - float(exp[7])) < 1e-5
     d, p, buf = enc(x, (1, 1, 4, 4), bits=2, eps=0.0625)
     t = hp.table(buf, 1)
     assert t["n_out"][0] == 1
     assert t["cls"][0] in (fho.SALIENT, fho.RAW)  # outlier-rich; RAW only because a 4x4 plane cannot gain
 
 
+def _numpy_three_sigma(xs):
+    """The rule in float64: thresholds, outlier count, and the distance of the closest element to a threshold."""
+    x64 = xs.astype(np.float64)
+    mu, sd = x64.mean(), x64.std()
+    thi, tlo = mu + 3 * sd, mu - 3 * sd
+    margin = np.minimum(np.abs(x64 - thi), np.abs(x64 - tlo)).min()
+    return mu, sd, tlo, thi, int(((x64 > thi) | (x64 < tlo)).sum()), margin
+
+
 @pytest.mark.parametrize("kind,seed", [("normal", 1), ("relu", 2), ("laplace", 3)])
 def test_sigma_count_matches_numpy_float64(kind, seed):
     """mu, sigma are the plain mean and population standard deviation: NumPy float64 agrees on the
-    outlier count whenever no element sits within rounding distance of a threshold.  The fixed-point
-    sums resolve 2^-19 of the largest magnitude per group of four, which bounds the differences."""
+    thresholds to 1e-5 of the range and on the outlier count whenever no element sits that close to a
+    threshold.  (The integer sums resolve 2^-18 of the range per group of four.)"""
     hw = 56 * 56
     x = {"normal": synth.normal, "relu": synth.relu_normal, "laplace": synth.laplace}[kind](8 * hw, seed)
     for pl in range(8):
         xs = x[pl * hw:(pl + 1) * hw]
-        S, Q, tlo, thi, n = fho.plane_sigma(xs)
-        x64 = xs.astype(np.float64)
-        A = np.abs(x64).max()
-        groups = hw // 4
-        mu, sd = x64.mean(), x64.std()
-        assert abs(S - x64.sum()) <= groups * A * 2.0 ** -18
-        assert abs(Q - (x64 ** 2).sum()) <= groups * A * A * 2.0 ** -15
-        assert abs(thi - (mu + 3 * sd)) <= 1e-4 and abs(tlo - (mu - 3 * sd)) <= 1e-4
-        margin = np.minimum(np.abs(x64 - (mu + 3 * sd)), np.abs(x64 - (mu - 3 * sd))).min()
-        if margin > 1e-3:
-            assert n == int(((x64 > mu + 3 * sd) | (x64 < mu - 3 * sd)).sum())
+        lo, dlo, dhi, n = fho.plane_sigma(xs)
+        mu, sd, tlo, thi, want, margin = _numpy_three_sigma(xs)
+        rng_ = float(xs.max()) - float(xs.min())
+        assert abs(float(lo) + dhi - thi) <= 1e-5 * rng_ and abs(float(lo) + dlo - tlo) <= 1e-5 * rng_
+        if margin > 2e-5 * rng_:
+            assert n == want
         assert n <= hw / 9  # Chebyshev: P(|x-mu| > 3 sigma) <= 1/9
 
 
-@pytest.mark.parametrize("scale", [1.0, 1e-3, 3e4, 2.0 ** -100, 2.0 ** 40])
-def test_fixed_point_sums_are_exact_integers_of_the_stated_roundings(scale):
-    """I_s and I_q are sums of round-half-even(s_g * 2^k_s) and (q_g * 2^k_q): recomputed here with
-    exact rational arithmetic from fp32 group values, for planes of very different magnitude, and
-    shown to be independent of the order of the groups."""
+@pytest.mark.parametrize("offset,sigma", [(1000.0, 0.01), (-37.0, 1.0), (3.0e4, 0.5), (-1.0e6, 2.0), (255.0, 1e-3)])
+@pytest.mark.parametrize("kind", ["normal", "relu", "spiky"])
+def test_sigma_rule_on_planes_with_an_offset(offset, sigma, kind):
+    """|mu| up to 10^5..10^6 sigma (a biased pre-activation, a plane far from zero): the rule has the same plain
+    answer as for centred data, because the moments are taken of the distances from the plane's minimum.
+    One-pass raw moments E[x^2] - mu^2 would be rounding noise here."""
+    rng = np.random.default_rng(int(abs(offset)) + len(kind))
+    hw = 28 * 28
+    for _ in range(6):
+        z = rng.standard_normal(hw)
+        if kind == "relu":
+            z = np.maximum(z, 0.0)
+        elif kind == "spiky":                       # 6 % far outliers: the plane must come out outlier-rich
+            z = np.where(rng.random(hw) < 0.06, 12.0 + np.abs(z), np.maximum(z, 0.0) * 0.2)
+        xs = (offset + sigma * z).astype(np.float32)
+        lo, dlo, dhi, n = fho.plane_sigma(xs)
+        mu, sd, tlo, thi, want, margin = _numpy_three_sigma(xs)
+        rng_ = float(xs.max()) - float(xs.min())
+        assert abs(float(lo) + dhi - thi) <= 1e-5 * rng_ and abs(float(lo) + dlo - tlo) <= 1e-5 * rng_
+        if margin > 2e-5 * rng_:
+            assert n == want
+        if kind == "spiky":
+            assert n * 32 > hw
+        else:
+            assert n * 32 <= hw
+    # the container carries the same count and class
+    d, p, buf = enc(xs, (1, 1, 28, 28), bits=4)
+    t = hp.table(buf, 1)
+    assert t["n_out"][0] == n and (t["cls"][0] != fho.NORMAL) == (n * 32 > hw)
+
+
+def test_sigma_rule_on_bf16_planes_with_an_offset():
+    """bf16 activations around 100 with a spread of a few units (8 mantissa bits: steps of 0.5): widened exactly,
+    then the same rule."""
+    rng = np.random.default_rng(5)
+    hw = 32 * 32
+    xs = synth.bf16_bits_to_f32(synth.to_bf16_bits((100.0 + 3.0 * rng.standard_normal(hw)).astype(np.float32)))
+    lo, dlo, dhi, n = fho.plane_sigma(xs)
+    mu, sd, tlo, thi, want, margin = _numpy_three_sigma(xs)
+    assert abs(float(lo) + dhi - thi) <= 1e-4 and abs(float(lo) + dlo - tlo) <= 1e-4
+    assert margin > 1e-3 and n == want
+    d, p, buf = enc(synth.to_bf16_bits(xs), (1, 1, 32, 32), dtype=fho.BF16, bits=2)
+    assert hp.table(buf, 1)["n_out"][0] == n
+
+
+@pytest.mark.parametrize("scale,offset", [(1.0, 0.0), (1e-3, 0.0), (3e4, 7e5), (2.0 ** -38, 0.0), (2.0 ** 55, 0.0), (0.25, -1e3)])
+def test_fixed_point_sums_are_exact_integers_of_the_stated_roundings(scale, offset):
+    """I_s and I_q are sums of round-half-even(s_g * 2^(18-e)) and (q_g * 2^(16-2e)) over the distances from
+    the minimum: recomputed here with exact rational arithmetic from fp32 group values, for planes of very
+    different magnitude and offset, and shown to be independent of the order of the groups."""
     from fractions import Fraction
     rng = np.random.default_rng(17)
-    x = (rng.standard_normal(203) * scale).astype(np.float32)   # 203: ragged last group
-    Is, Iq, ks, kq = fho.plane_sums(x)
-    A = float(np.abs(x).max())
-    e = int(np.floor(np.log2(A)))
-    assert ks == min(18 - e, 126) and kq == max(min(16 - 2 * e, 126), -126)
+    x = (offset + rng.standard_normal(203) * scale).astype(np.float32)   # 203: ragged last group
+    Is, Iq, e, applies = fho.plane_sums(x)
+    lo = x.min()
+    span = float(np.float32(x.max() - lo))
+    assert applies == 1 and e == int(np.floor(np.log2(span)))
 
     def rne(t):
         fl = t.numerator // t.denominator
         rem = t - fl
         return fl + (1 if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1) else 0)
-    xp = np.concatenate([x, np.zeros(1, np.float32)]).reshape(-1, 4)
+    dd = (x - lo).astype(np.float32)                                     # fp32 subtraction, element by element
+    assert (dd >= 0).all()
+    dp = np.concatenate([dd, np.zeros(1, np.float32)]).reshape(-1, 4)
     es = eq = 0
-    for v in xp:
+    for v in dp:
         sg = np.float32(np.float32(v[0] + v[1]) + np.float32(v[2] + v[3]))
         f = [Fraction(float(t)) for t in v]
         q01 = np.float32(float(f[1] * f[1] + Fraction(float(np.float32(v[0] * v[0])))))   # fma: one rounding
         q23 = np.float32(float(f[3] * f[3] + Fraction(float(np.float32(v[2] * v[2])))))
         qg = np.float32(q01 + q23)
-        es += rne(Fraction(float(sg)) * Fraction(2) ** ks)
-        eq += rne(Fraction(float(qg)) * Fraction(2) ** kq)
+        es += rne(Fraction(float(sg)) * Fraction(2) ** (18 - e))
+        eq += rne(Fraction(float(qg)) * Fraction(2) ** (16 - 2 * e))
     assert (Is, Iq) == (es, eq)
     # a permutation of whole groups leaves the integers unchanged
+    xp = np.concatenate([x, np.full(1, lo, np.float32)]).reshape(-1, 4)
     perm = rng.permutation(xp.shape[0])
     Is2, Iq2, _, _ = fho.plane_sums(xp[perm].reshape(-1))
     assert (Is2, Iq2) == (Is, Iq)
     # and the sums are close to the real ones
-    assert abs(Is * 2.0 ** -ks - float(x.astype(np.float64).sum())) <= 51 * A * 2.0 ** -18
+    d64 = x.astype(np.float64) - float(lo)
+    assert abs(Is * 2.0 ** (e - 18) - d64.sum()) <= 51 * span * 2.0 ** -18
+    assert abs(Iq * 2.0 ** (2 * e - 16) - (d64 ** 2).sum()) <= 51 * span * span * 2.0 ** -15
 
 
-def test_sigma_tail_group_padding_and_constant_plane():
-    # HW not a multiple of 4: the padded zeros must not change S, Q, and the divisor is HW
+def test_sigma_tail_group_padding_constant_plane_and_domain():
+    # HW not a multiple of 4: the padded group members add nothing, and the divisor is HW
     x = np.array([1, 2, 3, 4, 5, 6, 7], dtype=np.float32)
-    S, Q, tlo, thi, n = fho.plane_sigma(x)
-    assert S == 28.0 and Q == 140.0
+    lo, dlo, dhi, n = fho.plane_sigma(x)
+    Is, Iq, e, applies = fho.plane_sums(x)
+    assert (Is * 2.0 ** (e - 18), Iq * 2.0 ** (2 * e - 16)) == (21.0, 91.0)          # distances 0..6
     mu, sd = 4.0, 2.0
-    assert thi == np.float32(mu + 3 * sd) and tlo == np.float32(mu - 3 * sd) and n == 0
-    S, Q, tlo, thi, n = fho.plane_sigma(np.full(10, -2.5, dtype=np.float32))
-    assert n == 0 and tlo == thi == np.float32(-2.5)
+    assert lo == 1.0 and lo + dhi == np.float32(mu + 3 * sd) and lo + dlo == np.float32(mu - 3 * sd) and n == 0
+    # constant plane: no spread, no outliers
+    lo, dlo, dhi, n = fho.plane_sigma(np.full(10, -2.5, dtype=np.float32))
+    assert (lo, n) == (-2.5, 0) and fho.plane_sums(np.full(10, -2.5, dtype=np.float32))[3] == 0
+    # the rule is applied for ranges in [2^-40, 2^61) and for no other
+    spike = np.zeros(64, dtype=np.float32)
+    spike[:3] = 1.0                                  # 3 of 64 elements far out: outlier-rich wherever the rule applies
+    for k, want in ((-41, 0), (-40, 1), (0, 1), (60, 1), (61, 0)):
+        xs = spike * np.float32(2.0 ** k)
+        assert fho.plane_sums(xs)[3] == want
+        assert fho.plane_sigma(xs)[3] == (3 if want else 0)
+        d, p, buf = enc(xs, (1, 1, 8, 8), bits=2)
+        assert (hp.table(buf, 1)["cls"][0] != fho.NORMAL) == bool(want)
 
 
 def test_classification_threshold_is_strict_fraction():

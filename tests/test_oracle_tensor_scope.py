@@ -32,7 +32,7 @@ def test_counts_follow_the_tensor_wide_thresholds_and_classes_the_planes_own_sha
     x64 = x.astype(np.float64)
     mu, sd = x64.mean(), x64.std()
     thi, tlo = mu + 3 * sd, mu - 3 * sd
-    margin = 1e-5 * max(abs(thi), abs(tlo))
+    margin = 2e-5 * (float(x.max()) - float(x.min()))
     flat = x.reshape(n * c, h * w)
     want = ((flat > thi) | (flat < tlo)).sum(axis=1)
     near = ((np.abs(flat - thi) < margin) | (np.abs(flat - tlo) < margin)).sum(axis=1)
@@ -40,7 +40,7 @@ def test_counts_follow_the_tensor_wide_thresholds_and_classes_the_planes_own_sha
     assert want.sum() > 0
     assert ((t["cls"] != fho.NORMAL) == (t["n_out"].astype(np.int64) * 32 > h * w)).all()
     # the oracle's own statistic over all planes gives the same total
-    assert int(t["n_out"].sum()) == fho.channel_sigma(flat)[2]
+    assert int(t["n_out"].sum()) == fho.channel_sigma(flat)[3]
     cls = t["cls"].reshape(n, c)
     assert (cls[:, 3] != fho.NORMAL).all()                 # sigma of the tensor is ~1.5: a third of 4 N(0,1) lies outside
     assert cls[2, 7] == fho.NORMAL                         # 3 of 196 elements: below 1/32
