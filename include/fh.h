@@ -241,7 +241,7 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
  *     on the GPU (different streams without ordering between them) race on it: order them.
  */
 #define FH_STATIC_MAX_PLANES 131072
-#define FH_STATIC_SCRATCH_BYTES (256 + 4 * 1024 + 4 * FH_STATIC_MAX_PLANES)
+#define FH_STATIC_SCRATCH_BYTES (256 + 8 * (FH_STATIC_MAX_PLANES + 2 * (FH_STATIC_MAX_PLANES / 32)))
 int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                        size_t dst_capacity, uint64_t* d_out2, void* stream);
 
@@ -299,6 +299,19 @@ typedef struct {
 int fh_plan_generate(const fh_plan_op* ops, int32_t n_ops, const fh_plan_tensor* tensors, int32_t n_tensors,
                      uint64_t memory_budget, int32_t* actions, fh_plan_event* events, int32_t max_events,
                      fh_plan_report* report);
+
+/*
+ * Fault injection on the host side, for tests of the error path of the device-side waits.  (The paper has no
+ * counterpart.)  Compressing places the overflow parts of outlier-rich planes in plane order: a tile of
+ * planes waits, with a limit, until every earlier tile has published its size; a wait that runs out ends the
+ * call with FH_ERR_TIMEOUT in its status word (no magic in the header) and leaves the library usable.
+ *   FH_DEBUG_WAIT_POLLS   limit of those waits in polls of about 0.1 us (default 2^22)
+ *   FH_DEBUG_SILENT_TILE  index of a tile that never publishes its size, so that every later tile with
+ *                         an outlier-rich plane runs into the limit; UINT64_MAX: none (default)
+ * Both apply to calls enqueued afterwards, process-wide.  Returns FH_OK or FH_ERR_ARG.
+ */
+enum { FH_DEBUG_WAIT_POLLS = 0, FH_DEBUG_SILENT_TILE = 1 };
+int fh_debug_set(int what, uint64_t value);
 
 /* Number of kernels this library has launched since it was loaded (for launch accounting). */
 uint64_t fh_kernel_launches(void);

@@ -19,10 +19,12 @@ FH_F32, FH_BF16 = 0, 1
 FH_SALIENT_AUTO, FH_SALIENT_OFF, FH_SALIENT_ALL, FH_SALIENT_CHANNEL, FH_SALIENT_TENSOR = 0, 1, 2, 3, 4
 FH_KEEP, FH_COMPRESS, FH_EVICT = 0, 1, 2
 FH_STATIC_MAX_PLANES = 131072
+FH_DEBUG_WAIT_POLLS, FH_DEBUG_SILENT_TILE = 0, 1
 
 EXPORTS = ["fh_default_params", "fh_version", "fh_device_count", "fh_compressed_bytes", "fh_compress",
            "fh_decompress", "fh_run_schedule", "fh_host_work_bytes", "fh_compress_host",
-           "fh_decompress_host", "fh_compress_static", "fh_plan_generate", "fh_kernel_launches", "fh_shutdown"]
+           "fh_decompress_host", "fh_compress_static", "fh_plan_generate", "fh_debug_set", "fh_kernel_launches",
+           "fh_shutdown"]
 
 
 class FhError(RuntimeError):
@@ -113,6 +115,8 @@ def lib() -> C.CDLL:
                                        C.POINTER(C.c_int32), C.POINTER(fh_plan_event), C.c_int32,
                                        C.POINTER(fh_plan_report)]
         L.fh_plan_generate.restype = C.c_int
+        L.fh_debug_set.argtypes = [C.c_int, C.c_uint64]
+        L.fh_debug_set.restype = C.c_int
         L.fh_kernel_launches.restype = C.c_uint64
         L.fh_shutdown.restype = None
         _lib = L
@@ -232,6 +236,11 @@ def plan_generate(ops, tensors, memory_budget: int, max_events: int = 4096):
     rc = lib().fh_plan_generate(c_ops, len(ops), c_t, len(tensors), memory_budget, actions, events, max_events, C.byref(rep))
     n = min(rep.n_events, max_events)
     return int(rc), [int(a) for a in actions[:len(tensors)]], [(e.op, e.tensor, e.kind) for e in events[:n]], rep
+
+
+def debug_set(what: int, value: int) -> int:
+    """Host-side fault injection for the time-out test (see fh_debug_set in include/fh.h)."""
+    return int(lib().fh_debug_set(what, value & 0xFFFFFFFFFFFFFFFF))
 
 
 def kernel_launches() -> int:

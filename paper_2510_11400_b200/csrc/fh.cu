@@ -9,6 +9,7 @@
 #include <cstring>
 #include <map>
 #include <mutex>
+#include <tuple>
 #include <utility>
 #include <vector>
 
@@ -112,30 +113,16 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   if (pl.P > 0x7FFFFFFFull) return FH_ERR_UNSUPPORTED;
   const size_t sal_words = compress ? (size_t)(pl.H + 1 + 3 * pl.nblk) : (size_t)pl.nblk;
   pl.sal_words = (uint32_t)sal_words;
-  if (compress) {
-    // block-wise kernels: one plane per unit (a warp up to 8 KB, the CTA above)
-    pl.sk_cta = pl.plane_bytes > 8192 ? 1u : 0u;
-    pl.sk_threads = pl.sk_cta ? (pl.plane_bytes <= 32 * 1024 ? 256u : 512u) : 256u;
-    pl.sk_sal_off = (uint32_t)A16(pl.plane_bytes + 32);
-    pl.sk_area_words = (uint32_t)(A16(4 * (sal_words + 4)) / 4);
-    {
-      // a few measuring areas per unit, small enough not to cost resident CTAs: 16 KB per CTA unit,
-      // 1 KB per warp unit
-      const size_t budget = pl.sk_cta ? 16 * 1024 : 1024, area = 4 * (size_t)pl.sk_area_words, most = pl.sk_cta ? 8 : 16;
-      const size_t keep = budget / area;
-      pl.sk_keep = (uint32_t)(keep < 1 ? 1 : (keep > most ? most : keep));
-    }
-    pl.sk_unit_stride = pl.sk_sal_off + pl.sk_keep * 4 * pl.sk_area_words;
-    pl.sk_pre_off = (pl.sk_cta ? 1u : pl.sk_threads / 32u) * pl.sk_unit_stride;
-    pl.sk_total = pl.sk_pre_off + 4u * fh::kMaxChunks;
-    if (pl.mode != FH_SALIENT_OFF && pl.sk_total > kSmemLimit) return FH_ERR_UNSUPPORTED;
-  }
+  const uint32_t sal_bytes = (uint32_t)A16(4 * sal_words + 16);  // one measuring area of the block-wise path
+  const bool blockwise = compress && pl.mode != FH_SALIENT_OFF;
 
   Variant v;
   // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
   const bool whole16 = pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0;
   // (random rounding runs on the generic kernel)
-  if (compress && pl.rounding == 0 && (pl.groups <= 256 || whole16)) {
+  // (a warp-team kernel keeps one measuring area per warp: planes whose area is large -- very tall, narrow
+  // ones -- go to the general-purpose kernel)
+  if (compress && pl.rounding == 0 && ((pl.groups <= 256 && (!blockwise || sal_bytes <= 1024)) || (pl.groups > 256 && whole16))) {
     v.fast = true;
     if (pl.groups <= 256) {
       uint32_t t = pow2_ceil((pl.groups + 7) / 8);
@@ -156,10 +143,13 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     // (CTA-team kernel: two stages; a third buys nothing that more resident CTAs do not give)
     const uint32_t ns_max = v.cta ? 2u : (uint32_t)fh::kMaxStages;
     ns = ns < 2 ? 2 : (ns > ns_max ? ns_max : ns);
+    const uint32_t areas = blockwise ? (v.cta ? 1u : (uint32_t)fh::kWarps) : 0u;
     for (;;) {
       pl.nstage = ns;
       pl.sm_tile = 0;
-      pl.sm_total = (uint32_t)A16((size_t)ns * pl.stage_bytes);
+      pl.sm_sal = (uint32_t)A16((size_t)ns * pl.stage_bytes);
+      pl.sal_stride = sal_bytes;
+      pl.sm_total = pl.sm_sal + areas * sal_bytes;
       if (pl.sm_total <= kSmemLimit) break;
       if (ns == 2) {  // the pipeline needs two stages
         v.fast = false;
@@ -204,7 +194,9 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
       pl.sm_tile = 0;
       pl.sm_out = (uint32_t)A16(ppt * pl.plane_bytes + 32);
       pl.sm_rec = pl.sm_out + (uint32_t)(ppt * pl.npay);
-      pl.sm_total = pl.sm_rec + (uint32_t)A16(16 * ppt);
+      pl.sm_sal = pl.sm_rec + (uint32_t)A16(16 * ppt);
+      pl.sal_stride = sal_bytes;
+      pl.sm_total = pl.sm_sal + (blockwise ? sal_bytes : 0u);
       if (pl.sm_total <= kSmemLimit) break;
       if (ppt == 1) return FH_ERR_UNSUPPORTED;
       ppt = ppt / 2;
@@ -220,43 +212,73 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
 
 // ---- per-stream scratch ---------------------------------------------------------------------
 struct StreamScratch {
-  fh::Scratch* sc = nullptr;      // counters, followed by kMaxChunks chunk sums
-  uint32_t* worklist = nullptr;   // one word per plane of the largest tensor seen
-  size_t wl_cap = 0;
-  uint32_t* plane_nout = nullptr;  // channel-wide three-sigma mode: per-plane counts ...
+  fh::Scratch* sc = nullptr;             // counters
+  unsigned long long* scan = nullptr;    // placement scan: tile words, then group sums, then group prefixes
+  size_t tile_cap = 0;                   // tiles the scan arrays hold (groups: tile_cap / 32)
+  uint32_t calls = 0;                    // compress calls so far: parity of the ticket counter, epoch of the scan
+  uint32_t* plane_nout = nullptr;        // channel-wide three-sigma mode: per-plane counts ...
   size_t pn_cap = 0;
-  fh::ChanStat* chan = nullptr;    // ... and per-channel statistics
+  fh::ChanStat* chan = nullptr;          // ... and per-channel statistics
   size_t chan_cap = 0;
-  unsigned long long* sched = nullptr;  // schedule runner: offsets, sizes, statuses
+  unsigned long long* sched = nullptr;   // schedule runner: offsets, sizes, statuses
   size_t sched_cap = 0;
 };
-constexpr size_t kHeadBytes = 256 + 4 * fh::kMaxChunks;  // Scratch (padded) + chunk sums
+inline size_t scan_words(size_t tile_cap) { return tile_cap + 2 * (tile_cap / 32); }
 
 std::mutex g_mu;
 std::map<std::pair<int, cudaStream_t>, StreamScratch> g_scratch;
 int g_sm_count[64] = {0};
 
-int get_scratch(cudaStream_t stream, size_t planes, StreamScratch** out) {
+// Fault injection for the time-out test (see fh_debug_set in the header): limit of the device-side waits
+// of the placement scan, and a tile that never publishes.
+uint32_t g_scan_polls = 1u << 22;
+uint32_t g_skip_tile = 0xFFFFFFFFu;
+
+// `tiles`: tiles of the compress call that is about to be enqueued (0: none, e.g. for decompress).
+int get_scratch(cudaStream_t stream, size_t tiles, StreamScratch** out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return FH_ERR_CUDA;
   StreamScratch& s = g_scratch[std::make_pair(dev, stream)];
   if (!s.sc) {
-    if (cudaMalloc(&s.sc, kHeadBytes) != cudaSuccess) return FH_ERR_CUDA;
-    if (cudaMemset(s.sc, 0, kHeadBytes) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMalloc(&s.sc, fh::kScratchHeadBytes) != cudaSuccess) return FH_ERR_CUDA;
+    // cleared in the order of the stream that will use it (a non-blocking stream is not ordered with
+    // the legacy default stream)
+    if (cudaMemsetAsync(s.sc, 0, fh::kScratchHeadBytes, stream) != cudaSuccess) return FH_ERR_CUDA;
   }
-  if (planes > s.wl_cap) {
-    size_t cap = s.wl_cap ? s.wl_cap : 65536;
-    while (cap < planes) cap *= 2;
-    if (s.worklist) {
+  if (tiles > s.tile_cap) {
+    size_t cap = s.tile_cap ? s.tile_cap : 16384;
+    while (cap < tiles) cap *= 2;
+    if (s.scan) {
       cudaDeviceSynchronize();
-      cudaFree(s.worklist);
-      s.worklist = nullptr;
-      s.wl_cap = 0;
+      cudaFree(s.scan);
+      s.scan = nullptr;
+      s.tile_cap = 0;
     }
-    if (cudaMalloc(&s.worklist, cap * sizeof(uint32_t)) != cudaSuccess) return FH_ERR_CUDA;
-    s.wl_cap = cap;
+    if (cudaMalloc(&s.scan, scan_words(cap) * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
+    if (cudaMemsetAsync(s.scan, 0, scan_words(cap) * sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
+    s.tile_cap = cap;
   }
   *out = &s;
+  return FH_OK;
+}
+
+// Parity, epoch and scan pointers of the next compress call on a scratch (`scan` may be null when the call
+// places nothing).  The epoch never is 0; when the counter wraps, the tagged arrays are cleared.
+int next_call(uint32_t* calls, unsigned long long* scan, size_t tile_cap, cudaStream_t stream, fh::CompressArgs* a) {
+  ++*calls;
+  if ((*calls & 0x7FFFFFFFu) == 0u) {  // 2^31 calls later an old tag could pass for a new one: start afresh
+    if (scan && cudaMemsetAsync(scan, 0, scan_words(tile_cap) * sizeof(unsigned long long), stream) != cudaSuccess)
+      return FH_ERR_CUDA;
+    ++*calls;
+  }
+  a->parity = *calls & 1u;
+  a->scan.tile = scan;
+  a->scan.grp = scan ? scan + tile_cap : nullptr;
+  a->scan.gpre = scan ? scan + tile_cap + tile_cap / 32 : nullptr;
+  a->scan.epoch = *calls & 0x7FFFFFFFu;
+  a->scan.polls = g_scan_polls;
+  a->scan.skip_tile = g_skip_tile;
+  a->scan.reserved = 0;
   return FH_OK;
 }
 
@@ -306,14 +328,6 @@ int launch_channel_passes(const Plan& pl, const fh::ChannelArgs& ca, cudaStream_
   return FH_OK;
 }
 
-// Chunks of the block-wise kernels: runs of 2^shift consecutive planes, at most kMaxChunks of them.
-void chunking(uint64_t planes, uint32_t* shift, uint32_t* nchunks) {
-  uint32_t sh = 0;
-  while (((planes + ((1ull << sh) - 1)) >> sh) > fh::kMaxChunks) ++sh;
-  *shift = sh;
-  *nchunks = (uint32_t)((planes + ((1ull << sh) - 1)) >> sh);
-}
-
 int sm_count() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
@@ -323,8 +337,10 @@ int sm_count() {
 
 template <typename K>
 int grid_for(K kernel, size_t smem, uint32_t ntiles, int* grid, int threads = fh::kThreads) {
-  static std::map<std::pair<const void*, size_t>, int> cache;  // guarded by g_mu
-  const auto key = std::make_pair((const void*)kernel, (smem << 12) | (size_t)threads);
+  static std::map<std::tuple<int, const void*, size_t>, int> cache;  // guarded by g_mu; per device: the attribute is
+  int dev = 0;                                                        // set once for every device that runs the kernel
+  if (cudaGetDevice(&dev) != cudaSuccess) return FH_ERR_CUDA;
+  const auto key = std::make_tuple(dev, (const void*)kernel, (smem << 12) | (size_t)threads);
   auto it = cache.find(key);
   int per_sm;
   if (it == cache.end()) {
@@ -421,30 +437,6 @@ int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, c
   return FH_ERR_UNSUPPORTED;
 }
 
-template <int DT>
-int launch_blockwise(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
-  // the grid must be resident as a whole (the kernel has a barrier over it): what the device holds at once
-  int g = 0;
-  int rc = grid_for(fh::blockwise_kernel<DT>, pl.sk_total, 0x7FFFFFFFu, &g, (int)pl.sk_threads);
-  if (rc != FH_OK) return rc;
-  // A cooperative launch, and not one that may overlap its predecessor: CTAs that became resident beside
-  // the draining streaming kernel left some SMs unable to take their full share later, and the barrier
-  // then waited for CTAs that could not start.
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)g);
-  cfg.blockDim = dim3(pl.sk_threads);
-  cfg.dynamicSmemBytes = pl.sk_total;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeCooperative;
-  attr[0].val.cooperative = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, fh::blockwise_kernel<DT>, pl, a) != cudaSuccess) return FH_ERR_CUDA;
-  g_launches.fetch_add(1);
-  return FH_OK;
-}
-
 int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
   int rc;
   if (v.fast) {
@@ -464,10 +456,7 @@ int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a,
   }
   if (rc != FH_OK) return rc;
   g_launches.fetch_add(1);
-  if (pl.mode == FH_SALIENT_OFF) return FH_OK;
-  // the planes the streaming kernel listed: measure, then place and write
-  rc = pl.dtype == FH_F32 ? launch_blockwise<fh::kF32>(pl, a, stream) : launch_blockwise<fh::kBF16>(pl, a, stream);
-  return rc;
+  return FH_OK;
 }
 
 // Largest prime <= n (n >= 2), or 1.
@@ -523,7 +512,7 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   if (rc != FH_OK) return rc;
   std::lock_guard<std::mutex> lock(g_mu);
   StreamScratch* s = nullptr;
-  rc = get_scratch(stream, pl.mode == FH_SALIENT_OFF ? 0 : pl.P, &s);
+  rc = get_scratch(stream, pl.mode == FH_SALIENT_OFF ? 0 : pl.ntiles, &s);
   if (rc != FH_OK) return rc;
   fh::CompressArgs a;
   a.src = (const uint8_t*)d_src;
@@ -533,9 +522,9 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   a.d_off_out = d_off_out;
   a.out2 = d_out2;
   a.sc = s->sc;
-  a.worklist = s->worklist;
-  a.chunk_ovf = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(s->sc) + 256);
-  chunking(pl.P, &a.chunk_shift, &a.nchunks);
+  a.early_ticket = 1;
+  rc = next_call(&s->calls, s->scan, s->tile_cap, stream, &a);
+  if (rc != FH_OK) return rc;
   a.chan_nout = nullptr;
   a.plane_nout = nullptr;
   if (pl.mode >= fh::kModeChannel) {  // statistics per channel over the batch, or over the tensor: three passes ahead of the streaming kernel
@@ -797,15 +786,18 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
 }
 
 // ---- allocation-free compress -----------------------------------------------------------------
-// Scratch compiled into the device image: the counters (padded to 256 bytes), the chunk sums and a
-// work list of FH_STATIC_MAX_PLANES words.  The name is a device symbol: host code must not pass it
-// to a kernel, it asks the runtime for the symbol's device address instead (once per device).
+// Scratch compiled into the device image: the counters (padded to 256 bytes) and the placement scan's
+// arrays for FH_STATIC_MAX_PLANES tiles (a tile is at least one plane).  The name is a device symbol: host
+// code must not pass it to a kernel, it asks the runtime for the symbol's device address instead (once per
+// device).
 static __device__ __align__(256) unsigned char g_static_scratch[FH_STATIC_SCRATCH_BYTES];
-static_assert(sizeof(fh::Scratch) <= 256, "static scratch layout");
-static_assert(FH_STATIC_SCRATCH_BYTES == kHeadBytes + 4 * (size_t)FH_STATIC_MAX_PLANES, "static scratch layout");
+static_assert(sizeof(fh::Scratch) <= fh::kScratchHeadBytes, "static scratch layout");
+static_assert(FH_STATIC_SCRATCH_BYTES == fh::kScratchHeadBytes + 8 * (FH_STATIC_MAX_PLANES + 2 * (FH_STATIC_MAX_PLANES / 32)),
+              "static scratch layout");
 
 static std::mutex g_static_mu;
 static unsigned char* g_static_ptr[64] = {nullptr};
+static uint32_t g_static_calls[64] = {0};
 
 int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                        size_t dst_capacity, uint64_t* d_out2, void* stream_) {
@@ -820,7 +812,7 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   Variant v;
   rc = make_plan(desc, params, true, &pl, &v);
   if (rc != FH_OK) return rc;
-  if (pl.P > FH_STATIC_MAX_PLANES) return FH_ERR_UNSUPPORTED;  // beyond the fixed work list
+  if (pl.P > FH_STATIC_MAX_PLANES) return FH_ERR_UNSUPPORTED;  // beyond the fixed arrays
   if (pl.mode >= fh::kModeChannel) return FH_ERR_UNSUPPORTED;  // its statistics need scratch the fixed array does not hold
   cudaStream_t stream = (cudaStream_t)stream_;
   int dev = 0;
@@ -832,9 +824,12 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
     g_static_ptr[dev] = p;
   }
   unsigned char* base = g_static_ptr[dev];
-  // the array keeps the last call's contents: the counters and chunk sums must start at zero (the
-  // work list is written before it is read)
-  if (cudaMemsetAsync(base, 0, kHeadBytes, stream) != cudaSuccess) return FH_ERR_CUDA;
+  // The array keeps the last call's contents.  The counters and the scan's group sums must start at zero;
+  // the scan's other words carry the number of the call that wrote them and need no clearing.
+  unsigned long long* scan = reinterpret_cast<unsigned long long*>(base + fh::kScratchHeadBytes);
+  const size_t cap = FH_STATIC_MAX_PLANES;
+  if (cudaMemsetAsync(base, 0, fh::kScratchHeadBytes, stream) != cudaSuccess) return FH_ERR_CUDA;
+  if (cudaMemsetAsync(scan + cap, 0, (cap / 32) * sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
   fh::CompressArgs a;
   a.src = (const uint8_t*)d_src;
   a.dst_base = (uint8_t*)d_dst;
@@ -843,13 +838,26 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   a.d_off_out = nullptr;
   a.out2 = (unsigned long long*)d_out2;
   a.sc = reinterpret_cast<fh::Scratch*>(base);
-  a.chunk_ovf = reinterpret_cast<uint32_t*>(base + 256);
-  a.worklist = reinterpret_cast<uint32_t*>(base + kHeadBytes);
+  a.early_ticket = 0;  // the counters are cleared by the memset just enqueued: nothing may touch them before it
+  rc = next_call(&g_static_calls[dev], scan, cap, stream, &a);
+  if (rc != FH_OK) return rc;
   a.chan_nout = nullptr;
   a.plane_nout = nullptr;
-  chunking(pl.P, &a.chunk_shift, &a.nchunks);
   std::lock_guard<std::mutex> lock2(g_mu);  // the launch helpers keep their occupancy cache under g_mu
   return launch_compress(pl, v, a, stream);
+}
+
+int fh_debug_set(int what, uint64_t value) {
+  std::lock_guard<std::mutex> lock(g_mu);
+  if (what == FH_DEBUG_WAIT_POLLS) {
+    if (value < 1 || value > 0xFFFFFFFFull) return FH_ERR_ARG;
+    g_scan_polls = (uint32_t)value;
+  } else if (what == FH_DEBUG_SILENT_TILE) {
+    g_skip_tile = value > 0xFFFFFFFEull ? 0xFFFFFFFFu : (uint32_t)value;
+  } else {
+    return FH_ERR_ARG;
+  }
+  return FH_OK;
 }
 
 uint64_t fh_kernel_launches(void) { return g_launches.load(); }
@@ -862,7 +870,7 @@ void fh_shutdown(void) {
     cudaSetDevice(kv.first.first);
     cudaDeviceSynchronize();
     if (kv.second.sc) cudaFree(kv.second.sc);
-    if (kv.second.worklist) cudaFree(kv.second.worklist);
+    if (kv.second.scan) cudaFree(kv.second.scan);
     if (kv.second.plane_nout) cudaFree(kv.second.plane_nout);
     if (kv.second.chan) cudaFree(kv.second.chan);
     if (kv.second.sched) cudaFree(kv.second.sched);

@@ -3,8 +3,9 @@
 // Tensor-wide statistics (salient_mode = TENSOR) run through the same passes with the whole tensor as the
 // one "channel"; a plane's class then follows from its own count.
 // Three passes over the tensor, a warp per plane, results gathered per channel with atomics:
-//   pass 0: minimum and maximum of the channel (they fix the fixed-point scale of the moment sums);
-//   pass 1: fixed-point moment sums of the channel (exact integers, so the order of the atomics is immaterial);
+//   pass 0: minimum and maximum of the channel (the moments are taken of the distances from the minimum, and the
+//           range fixes the scale of the integer sums);
+//   pass 1: integer moment sums of the channel (exact, so the order of the atomics is immaterial);
 //   pass 2: thresholds from the sums; outliers per plane (kept for the plane table) and per channel.
 // The streaming kernel then reads a plane's class from its channel's count.  This mode is not tuned: it
 // reads the tensor four times where the per-plane mode reads it once.
@@ -22,8 +23,8 @@ struct ChanStat {
 };
 static_assert(sizeof(ChanStat) == 32, "ChanStat layout");
 
-// Order-preserving map float -> unsigned (finite values; -0.0 < +0.0, which min/max may not distinguish:
-// the key is only used to find the largest magnitude's exponent).
+// Order-preserving map float -> unsigned (finite values; -0.0 sorts below +0.0, and a distance from either is
+// the same number).
 __device__ __forceinline__ unsigned int float_key(float f) {
   const unsigned int b = __float_as_uint(f);
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
@@ -86,12 +87,18 @@ __global__ void __launch_bounds__(kThreads) channel_pass(const Plan pl, const Ch
       }
     } else {
       const float clo = key_float(~cs->lo_inv), chi = key_float(cs->hi_key);
-      const SigmaScale sc = sigma_scale(clo, chi);
+      const SigmaScale sc = sigma_scale(__fsub_rn(chi, clo));
+      if (!sc.applies) {  // constant channel, or a range outside the rule's domain: no outliers
+        if (PASS == 2 && lane == 0) a.plane_nout[p] = 0;
+        continue;
+      }
       if (PASS == 1) {
         long long s = 0, q = 0;
         for (uint32_t g = lane; g < pl.groups; g += 32u) {
           float v[4];
           load_group_global<DT>(plane, g, pl.HW, v);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) v[k] = (g * 4u + k < pl.HW) ? __fsub_rn(v[k], clo) : 0.0f;
           uint32_t as = 0, aq = 0;
           sigma_addends(v, sc, as, aq);
           s += (int32_t)(as - kMagicBits);
@@ -109,13 +116,14 @@ __global__ void __launch_bounds__(kThreads) channel_pass(const Plan pl, const Ch
           atomicAdd(&cs->Iq, (unsigned long long)q);
         }
       } else {
-        float tlo, thi;
-        sigma_thresholds((long long)cs->Is, (long long)cs->Iq, sc, a.inv_nhw, tlo, thi);
+        float dlo, dhi;
+        sigma_thresholds((long long)cs->Is, (long long)cs->Iq, sc, a.inv_nhw, dlo, dhi);
         uint32_t cnt = 0;
         for (uint32_t i = lane; i < pl.HW; i += 32u) {
           const float x = DT == kF32 ? __ldg(reinterpret_cast<const float*>(plane) + i)
                                      : bf16_bits_to_f32(__ldg(reinterpret_cast<const uint16_t*>(plane) + i));
-          cnt += (x > thi) || (x < tlo);
+          const float dd = __fsub_rn(x, clo);
+          cnt += (dd > dhi) || (dd < dlo);
         }
         asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(cnt) : "r"(0xFFFFFFFFu));
         if (lane == 0) {

@@ -1,24 +1,21 @@
 // Compress kernels.
 //
 // Container recap: every plane owns a slot of npay bytes at a closed-form offset; a normal plane's
-// codes fill its slot; the payload of a salient or raw plane runs through its slot and continues in
-// the overflow region, in plane order.
+// codes fill its slot; the payload of an outlier-rich (salient) or raw plane runs through its slot and
+// continues in the overflow region, in plane order.
 //
-// A call runs one or two kernels on its stream:
-//   1. a streaming kernel (one pass over the dense tensor): per-plane statistics, three-sigma class,
-//      and for normal planes the codes and the table entry.  Normal planes depend on nothing but
-//      themselves, so this kernel has no cross-CTA waits.  A plane that takes the block-wise path only
-//      gets a marker in the table and an entry in a work list.  Three variants by plane size:
-//        compress_warp<DT, SIGMA, TT, FULLVEC>  planes of at most 256 groups: bulk-copy (TMA) pipeline,
-//            a sub-warp team per plane, groups kept in registers;
-//        compress_cta<DT, SIGMA, NT>            larger planes of whole 16-byte chunks: one plane per CTA;
-//        compress_generic<DT, BITS>             everything else (ragged large planes);
-//   2. blockwise_kernel<DT> (not with salient_mode OFF): measures every plane of the work list (block
-//      classes, CSR and code sizes), decides salient versus raw, and after a barrier over its grid
-//      places the payloads in the overflow region in plane order (so the bytes do not depend on
-//      scheduling) and writes them; its last CTA writes the header and the result words.  With an
-//      empty work list it only writes the header.
-// With salient_mode OFF the streaming kernel finishes the container itself.
+// A call is ONE kernel, one pass over the dense tensor.  Tiles (runs of consecutive planes) are handed
+// out in order by a ticket.  Per plane: statistics, three-sigma class, and
+//   normal plane:   codes and table entry, written at once (the slot's offset is closed-form);
+//   other planes:   measured at once while they lie in shared memory (block classes, CSR and code sizes,
+//                   salient versus raw); the tile publishes the overflow size of its planes, obtains the sum
+//                   over all earlier tiles from the placement scan (fh_device.cuh) and writes the payloads.
+// Three variants by plane size:
+//   compress_warp<DT, SIGMA, TT, FULLVEC>  planes of at most 256 groups: bulk-copy (TMA) pipeline, a sub-warp
+//       team per plane, groups kept in registers; a warp handles the outlier-rich planes of its slice;
+//   compress_cta<DT, SIGMA, NT>            larger planes of whole 16-byte chunks: one plane per CTA and tile;
+//   compress_generic<DT, BITS>             everything else (ragged large planes, random rounding).
+// The kernel's last CTA writes the header and the result words and returns the scratch to its idle state.
 #pragma once
 
 #include "fh_device.cuh"
@@ -29,7 +26,6 @@ struct SalientInfo {
   uint32_t nnz_s, n_dense, n_out_d, size;
 };
 
-
 struct CompressArgs {
   const uint8_t* src;
   uint8_t* dst_base;
@@ -38,9 +34,9 @@ struct CompressArgs {
   unsigned long long* d_off_out;        // optional: offset for the next container
   unsigned long long* out2;             // optional: {total bytes, status}
   Scratch* sc;
-  uint32_t* worklist;                   // planes that take the block-wise path, in no particular order
-  uint32_t* chunk_ovf;                  // per chunk of 2^chunk_shift planes: overflow size of its planes (16-byte units)
-  uint32_t chunk_shift, nchunks;
+  Scan scan;                            // placement of overflow parts (unused with salient_mode OFF)
+  uint32_t parity;                      // which of the two ticket counters this call uses
+  uint32_t early_ticket;                // 1: tiles may be requested before the previous kernel on the stream has completed
   // channel-wide three-sigma mode: per-channel outlier counts and per-plane counts from the statistics passes
   const unsigned long long* chan_nout;  // stride: 4 words (see ChanStat)
   const uint32_t* plane_nout;
@@ -55,7 +51,6 @@ __device__ __forceinline__ uint32_t channel_class(const Plan& pl, const Compress
   const unsigned long long total = a.chan_nout[(gp % pl.C) * 4ull];
   return total * pl.rho_den > (unsigned long long)pl.rho_num * pl.N * pl.HW ? kClsSalient : kClsNormal;
 }
-
 
 // Where the bytes of a salient / raw payload go: offsets below npay land in the plane's slot, the
 // rest in its overflow part.  Offsets and npay are multiples of the access size.
@@ -263,13 +258,6 @@ __device__ __noinline__ void raw_write(const Team& t, const Plan& pl, const uint
     out.st16(o, o < n ? (uint32_t)*reinterpret_cast<const uint16_t*>(plane + o) : 0u);
 }
 
-// Per-plane record kept in shared memory while a tile is processed.
-struct Rec {
-  float lo, scale;
-  uint32_t meta;  // class | n_out << 2
-  uint32_t size;  // payload bytes of a salient / raw plane (before padding)
-};
-
 // What every thread of a CTA knows about the destination.
 struct Dest {
   uint8_t* dst;
@@ -285,12 +273,54 @@ __device__ __forceinline__ Dest make_dest(const Plan& pl, const CompressArgs& a)
   return d;
 }
 
+__device__ __forceinline__ uint32_t salient_size(const Plan& pl, uint32_t nnz_s, uint32_t n_dense, uint32_t n_out_d) {
+  const uint32_t e = (uint32_t)pl.esize;
+  return 16u + 4u * pl.nbm + 4u * ((uint32_t)pl.H + 1u) + a4(2u * nnz_s) + a4(e * nnz_s) + 64u * n_dense +
+         a4(e * n_out_d);
+}
+// Overflow size, in 16-byte units, of a payload of `size` bytes.
+__device__ __forceinline__ uint32_t ovf_units(const Plan& pl, uint32_t size) {
+  return a16(size) > pl.npay ? (a16(size) - pl.npay) >> 4 : 0u;
+}
+// A measured plane is stored salient, or raw when that would not be smaller; returns its overflow units.
+__device__ __forceinline__ uint32_t plane_units(const Plan& pl, const SalientInfo& info, bool& raw) {
+  raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
+  return ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
+}
+
+// Per-call counters of a tile's outlier-rich planes (one thread): nsal and nraw share a word.
+__device__ __forceinline__ void count_blockwise(const CompressArgs& a, uint32_t units, uint32_t nsal, uint32_t nraw) {
+  if (units) atomicAdd(&a.sc->ovf16, (unsigned long long)units);
+  if (nsal | nraw) atomicAdd(&a.sc->nsal, (unsigned long long)nsal | ((unsigned long long)nraw << 32));
+}
+
+// Writes the payload of the measured plane gp (`plane` in shared memory, `info` and `sal` from
+// salient_measure) with its overflow part `at` units into the overflow region, and its table entry.
+template <int DT>
+__device__ __forceinline__ void write_blockwise(const Team& t, const Plan& pl, const Dest& d, uint64_t gp,
+                                                const uint8_t* plane, const SalientInfo& info, const uint32_t* sal,
+                                                uint32_t n_out, uint32_t at) {
+  bool raw;
+  const uint32_t my_units = plane_units(pl, info, raw);
+  const unsigned long long off16 = (pl.ovf_off >> 4) + at;
+  if (!d.fits || (off16 + my_units) * 16ull > d.capacity) return;  // never write past the capacity
+  SplitOut out;
+  out.slot = d.dst + pl.slots_off + gp * pl.npay;
+  out.ovf = d.dst + off16 * 16ull;
+  out.npay = pl.npay;
+  if (raw) raw_write(t, pl, plane, out);
+  else salient_write<DT>(t, pl, plane, info, sal, out);
+  if (t.lane == 0)
+    reinterpret_cast<uint4*>(d.dst + 64)[gp] =
+        make_uint4(my_units ? (uint32_t)off16 : 0u, (raw ? kClsRaw : kClsSalient) | (n_out << 2), 0u, 0u);
+}
+
 // One thread, after everything else of the call is done: header, result words, and every counter the
 // call touched back to zero.
 __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, const Dest& d) {
   const unsigned long long ovf16 = ld_relaxed(&a.sc->ovf16);
-  const unsigned long long nsal = ld_relaxed(&a.sc->nsal), nraw = ld_relaxed(&a.sc->nraw);
-  const unsigned long long listed = ld_relaxed(&a.sc->wl_count);
+  const unsigned long long cnt = ld_relaxed(&a.sc->nsal);
+  const uint32_t nsal = (uint32_t)cnt, nraw = (uint32_t)(cnt >> 32);
   uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
   const unsigned long long total = pl.ovf_off + ovf16 * 16ull;
   if (total > d.capacity && code < kErrCapacity) code = kErrCapacity;
@@ -300,7 +330,7 @@ __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, 
     hd[0] = make_uint4(code == kErrNone ? kMagic : 0u, 1u | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24), pl.N, pl.C);
     hd[1] = make_uint4((uint32_t)pl.H, (uint32_t)pl.W, 8u | (8u << 8) | ((uint32_t)pl.rounding << 16) | ((uint32_t)pl.mode << 24),
                        pl.rho_num | (pl.rho_den << 16));
-    hd[2] = make_uint4(pl.tau_num | (pl.tau_den << 16), __float_as_uint(pl.eps), (uint32_t)nsal, (uint32_t)nraw);
+    hd[2] = make_uint4(pl.tau_num | (pl.tau_den << 16), __float_as_uint(pl.eps), nsal, nraw);
     hd[3] = make_uint4((uint32_t)pl.tensor_id, (uint32_t)(pl.tensor_id >> 32), (uint32_t)total, (uint32_t)(total >> 32));
   }
   if (a.out2) {
@@ -308,73 +338,78 @@ __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, 
     a.out2[1] = status_word(code);
   }
   if (a.d_off_out) *a.d_off_out = code == kErrNone ? d.off_in + ((total + 255ull) & ~255ull) : (~0ull >> 1);
-  if (listed) {  // (the chunk sums are cleared by the block-wise kernel's last CTA)
-    st_relaxed(&a.sc->ovf16, 0ull);
-    st_relaxed(&a.sc->nsal, 0ull);
-    st_relaxed(&a.sc->nraw, 0ull);
-    st_relaxed(&a.sc->wl_count, 0ull);
-    st_relaxed(&a.sc->arrived, 0ull);
-  }
+  if (ovf16) st_relaxed(&a.sc->ovf16, 0ull);
+  if (cnt) st_relaxed(&a.sc->nsal, 0ull);
   if (code) st_relaxed(&a.sc->status, 0ull);
 }
 
-// Last step of every CTA of a kernel that hands out tiles or counts exits: the last CTA to leave
-// returns those counters to zero and, if this is the call's last kernel (FINAL), finishes the call.
-template <bool FINAL>
-__device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, const Dest& d) {
+// Last step of every CTA: the last CTA to leave returns the scan's group counters and the hand-out
+// counters to zero and finishes the container.
+__device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t* s_last) {
   __threadfence();
   __syncthreads();
+  if (threadIdx.x == 0) *s_last = atomicAdd(&a.sc->exited, 1ull) == (unsigned long long)gridDim.x - 1ull;
+  __syncthreads();
+  if (!*s_last) return;
+  if (pl.mode != kModeOff)
+    for (uint32_t k = threadIdx.x; k < ((pl.ntiles + 31u) >> 5); k += blockDim.x) a.scan.grp[k] = 0ull;
   if (threadIdx.x != 0) return;
-  const unsigned long long prev = atomicAdd(&a.sc->exited, 1ull);
-  if (prev != (unsigned long long)gridDim.x - 1ull) return;
   __threadfence();
-  st_relaxed(&a.sc->ticket, 0ull);
+  st_relaxed(&a.sc->ticket[a.parity], 0ull);
   st_relaxed(&a.sc->exited, 0ull);
-  if (FINAL) finalize(pl, a, d);
+  finalize(pl, a, d);
 }
 
-__device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane, uint32_t off16, const Rec& r) {
-  uint4 e;
-  e.x = off16;
-  e.y = r.meta;
-  e.z = __float_as_uint(r.lo);
-  e.w = __float_as_uint(r.scale);
-  reinterpret_cast<uint4*>(d.dst + 64)[plane] = e;
+__device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane, uint32_t off16, uint32_t meta, float lo,
+                                                  float scale) {
+  reinterpret_cast<uint4*>(d.dst + 64)[plane] = make_uint4(off16, meta, __float_as_uint(lo), __float_as_uint(scale));
 }
 
-
-// Table marker of a plane that takes the block-wise path: class salient, the three-sigma count, no
-// offset yet.  The block-wise kernels complete the entry.
-__device__ __forceinline__ void store_marker(const Dest& d, uint64_t plane, uint32_t meta) {
-  reinterpret_cast<uint4*>(d.dst + 64)[plane] = make_uint4(0u, (meta & ~3u) | kClsSalient, 0u, 0u);
+// Distances d = x - lo of group g of a plane; positions past HW read as 0.
+template <int DT>
+__device__ __forceinline__ void load_dist(const uint8_t* plane, uint32_t g, uint32_t HW, bool vec, float lo, float d[4]) {
+  float v[4];
+  load_group<DT>(plane, g, HW, vec, v);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) d[k] = (g * 4u + k < HW) ? __fsub_rn(v[k], lo) : 0.0f;
 }
 
-// Appends plane `gp` to the work list of the block-wise kernels (one thread).
-__device__ __forceinline__ void list_plane(const CompressArgs& a, uint64_t gp) {
-  const unsigned long long at = atomicAdd(&a.sc->wl_count, 1ull);
-  a.worklist[at] = (uint32_t)gp;
-}
+// Per-plane record kept in shared memory while a tile of the generic kernel is processed.
+struct Rec {
+  float lo, scale;
+  uint32_t meta;   // class | n_out << 2
+  uint32_t units;  // overflow units of a salient / raw plane
+};
 
 // =================================================================================================
 // Generic streaming kernel
 // =================================================================================================
 // Tiles of consecutive planes are staged in shared memory with plain loads (planes need not start
 // on a 16-byte boundary); a team per plane computes statistics and class; the codes of normal planes
-// are staged in shared memory and leave with 16-byte stores.
+// are staged in shared memory and leave with 16-byte stores.  Outlier-rich planes of the tile are then
+// taken one after the other by the whole CTA: measured, placed through the scan, measured again and
+// written (this kernel serves the odd shapes; the fast kernels below do not measure twice).
 template <int DT, int BITS>
 __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
-  __shared__ uint32_t s_tile;
-  dep_trigger();  // the next kernel on the stream may become resident as this one drains
-  dep_wait();     // the previous kernel on the stream has completed
+  __shared__ uint32_t s_tile, s_last, s_base, s_ok;
+  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
 
   const uint32_t tid = threadIdx.x;
+  if (tid == 0) {
+    s_pl = pl;
+    if (a.early_ticket) s_tile = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
+  }
+  dep_wait();     // the previous kernel on the stream has completed
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
   uint8_t* tile_buf = smem + pl.sm_tile;
   uint8_t* out_buf = smem + pl.sm_out;
   Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
+  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal);
   const Dest d = make_dest(pl, a);
   const Team team = make_team(pl.team, s_red);
+  const Team cta = make_team(kThreads, s_red);
   const uint32_t nteams = team.block ? 1u : kThreads / team.size;
   const uint32_t my_team = team.block ? 0u : tid / team.size;
   constexpr uint32_t L = (1u << BITS) - 1u;
@@ -382,8 +417,8 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
   uint32_t rp = 0;  // reduction counter (see red_half)
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
 
-  for (;;) {
-    if (tid == 0) s_tile = (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+  for (bool first = true;; first = false) {
+    if (tid == 0 && !(first && a.early_ticket)) s_tile = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
     __syncthreads();
     const uint32_t tile = s_tile;
     if (tile >= pl.ntiles) break;
@@ -424,37 +459,39 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
         }
       }
       team_minmax(team, lo, hi, rp);
-      if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && team.lane == 0)
+      const float range = __fsub_rn(hi, lo);
+      if (!(fabsf(range) <= 3.402823466e38f) && team.lane == 0)
         atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
 
       uint32_t cls = kClsNormal, n_out = 0;
       if (need_sigma) {
-        const SigmaScale sc = sigma_scale(lo, hi);
-        uint32_t as = 0, aq = 0, ng = 0;
-        for (uint32_t g = team.lane; g < groups; g += team.size) {
-          float v[4];
-          load_group<DT>(plane, g, HW, vec, v);
-          sigma_addends(v, sc, as, aq);
-          ++ng;
-        }
-        long long Is, Iq;
-        if (team.block)
-          team_sum2_wide(team, (long long)(int32_t)(as - ng * kMagicBits), (long long)(int32_t)(aq - ng * kMagicBits),
-                         Is, Iq, rp);
-        else
-          team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
-        float tlo, thi;
-        sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
-        uint32_t cnt = 0;
-        for (uint32_t g = team.lane; g < groups; g += team.size) {
-          float v[4];
-          load_group<DT>(plane, g, HW, vec, v);
+        const SigmaScale sc = sigma_scale(range);
+        if (sc.applies) {  // (the same for every thread of the team)
+          uint32_t as = 0, aq = 0, ng = 0;
+          for (uint32_t g = team.lane; g < groups; g += team.size) {
+            float dd[4];
+            load_dist<DT>(plane, g, HW, vec, lo, dd);
+            sigma_addends(dd, sc, as, aq);
+            ++ng;
+          }
+          long long Is, Iq;
+          if (team.block)
+            team_sum2_wide(team, (long long)(int32_t)(as - ng * kMagicBits), (long long)(int32_t)(aq - ng * kMagicBits),
+                           Is, Iq, rp);
+          else
+            team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
+          float dlo, dhi;
+          sigma_thresholds(Is, Iq, sc, pl.inv_hw, dlo, dhi);
+          uint32_t cnt = 0;
+          for (uint32_t g = team.lane; g < groups; g += team.size) {
+            float dd[4];
+            load_dist<DT>(plane, g, HW, vec, lo, dd);
 #pragma unroll
-          for (int k = 0; k < 4; ++k) cnt += (v[k] > thi) || (v[k] < tlo);
+            for (int k = 0; k < 4; ++k) cnt += (g * 4u + k < HW) && ((dd[k] > dhi) || (dd[k] < dlo));
+          }
+          n_out = team_sum_u32(team, cnt, rp);
+          if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * HW) cls = kClsSalient;
         }
-        n_out = team_sum_u32(team, cnt, rp);
-        if ((0.0f > thi) || (0.0f < tlo)) n_out -= 4u * groups - HW;  // padded zeros are not elements
-        if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * HW) cls = kClsSalient;
       } else if (pl.mode == kModeAll) {
         cls = kClsSalient;
       } else if (pl.mode >= kModeChannel) {
@@ -464,10 +501,10 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
       Rec r;
       r.lo = 0.0f;
       r.scale = 0.0f;
-      r.size = 0;
+      r.units = 0;
       if (cls == kClsNormal) {
         float inv, scale;
-        quant_params(lo, hi, L, inv, scale);
+        quant_params(range, L, inv, scale);
         r.lo = lo;
         r.scale = scale;
         uint8_t* o = out_buf + (uint64_t)lp * pl.npay;
@@ -475,15 +512,15 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
         for (uint32_t g = team.lane; g < ogroups; g += team.size) {
           uint32_t word = 0;
           if (g < groups) {
-            float v[4];
-            load_group<DT>(plane, g, HW, vec, v);
+            float dd[4];
+            load_dist<DT>(plane, g, HW, vec, lo, dd);
             uint32_t rnd[4] = {0, 0, 0, 0};
             if (pl.rounding)  // one generator call per group: counter = (group, plane, tensor id), key = seed
               philox4x32_10(g, (uint32_t)(p0 + lp), (uint32_t)pl.tensor_id, (uint32_t)(pl.tensor_id >> 32),
                             (uint32_t)pl.seed, (uint32_t)(pl.seed >> 32), rnd);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              uint32_t q = pl.rounding ? quant_code_random(v[k], lo, inv, L, rnd[k]) : quant_code(v[k], lo, inv, L);
+              uint32_t q = pl.rounding ? quant_code_random(dd[k], inv, L, rnd[k]) : quant_code(dd[k], inv, L);
               if (g * 4u + k >= HW) q = 0;
               word |= q << (k * BITS);
             }
@@ -498,7 +535,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     }
     __syncthreads();
 
-    // ---- phase B: table entries and slots of the normal planes; markers and work-list entries of the others
+    // ---- phase B: table entries and slots of the normal planes
     if (d.fits) {
       const uint32_t chunks = pl.npay >> 4;
       uint4* slots = reinterpret_cast<uint4*>(d.dst + pl.slots_off + p0 * pl.npay);
@@ -506,57 +543,89 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
         const uint32_t lp = i / chunks;
         if ((rec[lp].meta & 3u) == kClsNormal) slots[i] = reinterpret_cast<const uint4*>(out_buf)[i];
       }
+      for (uint32_t i = tid; i < np; i += kThreads)
+        if ((rec[i].meta & 3u) == kClsNormal)
+          store_table_entry(d, p0 + i, (uint32_t)((pl.slots_off + (p0 + i) * pl.npay) >> 4), rec[i].meta, rec[i].lo,
+                            rec[i].scale);
     }
-    for (uint32_t i = tid; i < np; i += kThreads) {
-      if ((rec[i].meta & 3u) == kClsNormal) {
-        if (d.fits) store_table_entry(d, p0 + i, (uint32_t)((pl.slots_off + (p0 + i) * pl.npay) >> 4), rec[i]);
-      } else {
-        if (d.fits) store_marker(d, p0 + i, rec[i].meta);
-        list_plane(a, p0 + i);
+
+    // ---- phase C: the other planes, one after the other by the whole CTA
+    if (pl.mode != kModeOff) {
+      uint32_t U = 0, nsal = 0, nraw = 0;  // (every thread keeps the same figures)
+      for (uint32_t lp = 0; lp < np; ++lp) {
+        if ((rec[lp].meta & 3u) == kClsNormal) continue;
+        const SalientInfo info = salient_measure<DT>(cta, s_pl, tile_buf + head + (uint64_t)lp * pl.plane_bytes, sal);
+        bool raw;
+        const uint32_t u = plane_units(pl, info, raw);
+        if (tid == 0) rec[lp].units = u;
+        U += u;
+        nsal += raw ? 0u : 1u;
+        nraw += raw ? 1u : 0u;
+        __syncthreads();  // the measuring scratch is reused
+      }
+      if (tid < 32u) {
+        bool ok = true;
+        uint32_t base = 0;
+        if (tid == 0) {
+          scan_publish(a.scan, tile, U);
+          count_blockwise(a, U, nsal, nraw);
+        }
+        if (U) ok = scan_prefix(a.scan, tile, base);
+        if (tid == 0) {
+          if (!ok) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+          s_base = base;
+          s_ok = ok;
+        }
+      }
+      __syncthreads();
+      if ((nsal | nraw) && s_ok) {
+        uint32_t at = s_base;
+        for (uint32_t lp = 0; lp < np; ++lp) {
+          if ((rec[lp].meta & 3u) == kClsNormal) continue;
+          const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
+          const SalientInfo info = salient_measure<DT>(cta, s_pl, plane, sal);
+          write_blockwise<DT>(cta, s_pl, d, p0 + lp, plane, info, sal, rec[lp].meta >> 2, at);
+          at += rec[lp].units;
+          __syncthreads();
+        }
       }
     }
     __syncthreads();
   }
-  if (pl.mode == kModeOff) cta_exit<true>(pl, a, d);
-  else cta_exit<false>(pl, a, d);
+  cta_exit(pl, a, d, &s_last);
 }
 
 // =================================================================================================
-// Fast kernel
+// Fast kernels
 // =================================================================================================
-// One plane per team and tile.  Warp-team variant (CTA = false): kThreads / team planes per tile,
-// each handled by `team` lanes of a warp.  CTA-team variant: one plane per tile, handled by all
-// threads.  Thread t of a team owns groups t, t + team, ... (G of them) and keeps them in registers
-// for every pass.  FULL: groups == G * team, so no group needs a bounds check.
+// One plane per team.  Warp-team variant: kThreads / team planes per tile, each handled by `team` lanes of a
+// warp; thread t of a team owns groups t, t + team, ... (G of them) and keeps them in registers for every
+// pass.  FULL: groups == G * team, so no group needs a bounds check.
 //
-// One sweep over a plane: min/max -> (fixed-point moments -> thresholds -> count -> class) ->
-// codes, stored straight to the plane's slot together with its table entry.  Salient planes are
-// measured by their team right away; their writes wait for the tile's placement.
-// Codes of the thread's groups, packed and stored to the plane's slot (used inside plane_sweep, on
-// its register-resident groups x[k][e]).  Four codes of a group are the sum of
-// (magic + q_e) << (e * BITS) minus the magic's contribution.
+// One sweep over a plane: min/max -> distances from the minimum -> (integer moments -> thresholds -> count
+// -> class) -> codes, stored straight to the plane's slot together with its table entry.
+//
+// Codes of the thread's groups, packed and stored to the plane's slot (used inside plane_sweep, on its
+// register-resident distances x[k][e]).  Four codes of a group are the sum of (magic + q_e) << (e * BITS)
+// minus the magic's contribution.
 #define FH_STORE_CODES(BITS)                                                                                  \
   {                                                                                                           \
     constexpr uint32_t bias = kMagicBits * (1u + (1u << (BITS)) + (1u << (2 * (BITS))) + (1u << (3 * (BITS)))); \
-    const f32x2 nlo2 = pack2(-lo, -lo), inv2 = pack2(inv, inv), mag2 = pack2(kMagicF, kMagicF);                 \
+    const f32x2 inv2 = pack2(inv, inv), mag2 = pack2(kMagicF, kMagicF);                                         \
     _Pragma("unroll") for (int k = 0; k < G; ++k) {                                                           \
       const uint32_t g = lane + (uint32_t)(k * TT);                                                           \
       uint32_t w0, w1, w2, w3;                                                                                \
-      if (DT == kBF16) { /* packed pairs; x - lo is x + (-lo): the same rounding */                          \
-        unpack2u(fma2(add2(pack2(x[k][0], x[k][1]), nlo2), inv2, mag2), w0, w1);                              \
-        unpack2u(fma2(add2(pack2(x[k][2], x[k][3]), nlo2), inv2, mag2), w2, w3);                              \
+      if (DT == kBF16) { /* packed pairs */                                                                  \
+        unpack2u(fma2(pack2(x[k][0], x[k][1]), inv2, mag2), w0, w1);                                          \
+        unpack2u(fma2(pack2(x[k][2], x[k][3]), inv2, mag2), w2, w3);                                          \
       } else {                                                                                                \
-        w0 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][0], lo), inv, kMagicF));                                \
-        w1 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][1], lo), inv, kMagicF));                                \
-        w2 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][2], lo), inv, kMagicF));                                \
-        w3 = __float_as_uint(__fmaf_rn(__fsub_rn(x[k][3], lo), inv, kMagicF));                                \
+        w0 = __float_as_uint(__fmaf_rn(x[k][0], inv, kMagicF));                                               \
+        w1 = __float_as_uint(__fmaf_rn(x[k][1], inv, kMagicF));                                               \
+        w2 = __float_as_uint(__fmaf_rn(x[k][2], inv, kMagicF));                                               \
+        w3 = __float_as_uint(__fmaf_rn(x[k][3], inv, kMagicF));                                               \
       }                                                                                                       \
       uint32_t word = w0 + (w1 << (BITS)) + (w2 << (2 * (BITS))) + (w3 << (3 * (BITS))) - bias;               \
       if (FULL || g < groups) {                                                                               \
-        if (!VEC) { /* ragged last group: elements past the plane carry no code */                            \
-          const uint32_t valid = min(4u, pl.HW - g * 4u);                                                     \
-          if (valid < 4u) word &= (1u << (valid * (BITS))) - 1u;                                              \
-        }                                                                                                     \
         if ((BITS) == 2) slot[g] = (uint8_t)word;                                                             \
         else if ((BITS) == 4) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;                          \
         else reinterpret_cast<uint32_t*>(slot)[g] = word;                                                     \
@@ -564,21 +633,22 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     }                                                                                                         \
   }
 
-// TT: team size (1..32, or kThreads for the CTA team), a compile-time constant so that the strides
-// between a thread's groups are immediates.  FULL: groups == G * TT.  VEC: planes are whole 16-byte
-// chunks (vector loads, no ragged last group).
+// TT: team size (1..32), a compile-time constant so that the strides between a thread's groups are
+// immediates.  FULL: groups == G * TT.  VEC: planes are whole 16-byte chunks (vector loads, no ragged last
+// group).  Returns class | n_out << 2; a normal plane is complete when the function returns.
 template <int DT, bool SIGMA, int G, int TT, bool FULL, bool VEC>
-__device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, const Dest& d, const CompressArgs& a,
-                                            const uint8_t* plane, uint64_t gp, uint32_t& rp, Rec& r) {
+__device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl, const Dest& d, const CompressArgs& a,
+                                                const uint8_t* plane, uint64_t gp, uint32_t& rp) {
   // A thread's G group slots that lie past the plane, and the elements past a ragged last group, are
-  // held as zeros: they add exactly nothing to the fixed-point moments, are kept out of minimum and
-  // maximum with neutral values, are subtracted from the outlier count when zero lies outside the
-  // thresholds, and their codes are not stored.  The arithmetic runs unpredicated over all G slots.
+  // kept out of minimum and maximum with neutral values and then held as distance 0: they add exactly
+  // nothing to the moments, are subtracted from the outlier count when 0 lies outside the thresholds, and
+  // carry code 0 (a ragged last group) or are not stored at all.  The arithmetic runs unpredicated over all
+  // G slots.
   const uint32_t groups = pl.groups, lane = team.lane;
   const float pinf = __int_as_float(0x7F800000), ninf = __int_as_float(0xFF800000);
   float x[G][4];
   float lo = pinf, hi = ninf, lo1 = pinf, hi1 = ninf;
-  uint32_t npad = 0;  // zero-padded elements among this thread's slots
+  uint32_t npad = 0;  // padded elements among this thread's slots
 #pragma unroll
   for (int k = 0; k < G; ++k) {
     const uint32_t g = lane + (uint32_t)(k * TT);
@@ -629,61 +699,79 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
   lo = min_nan(lo, lo1);
   hi = max_nan(hi, hi1);
   team_minmax(team, lo, hi, rp);
-  if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && lane == 0)
-    atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+  const float range = __fsub_rn(hi, lo);
+  if (!(fabsf(range) <= 3.402823466e38f) && lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+
+  // distances from the minimum, in place (x - lo is x + (-lo): the same rounding)
+  {
+    const float nlo = -lo;
+    const f32x2 nlo2 = pack2(nlo, nlo);
+#pragma unroll
+    for (int k = 0; k < G; ++k) {
+      if (DT == kBF16) {
+        unpack2(add2(pack2(x[k][0], x[k][1]), nlo2), x[k][0], x[k][1]);
+        unpack2(add2(pack2(x[k][2], x[k][3]), nlo2), x[k][2], x[k][3]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) x[k][e] = __fadd_rn(x[k][e], nlo);
+      }
+      if (!(FULL && VEC)) {
+        const uint32_t g = lane + (uint32_t)(k * TT);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const bool in = VEC ? g < groups : g * 4u + e < pl.HW;
+          x[k][e] = in ? x[k][e] : 0.0f;
+        }
+      }
+    }
+  }
 
   uint32_t cls = kClsNormal, n_out = 0;
   if (SIGMA) {
-    const SigmaScale sc = sigma_scale(lo, hi);
-    uint32_t as = 0, aq = 0;
+    const SigmaScale sc = sigma_scale(range);
+    if (sc.applies) {  // (the same for every thread of the team)
+      uint32_t as = 0, aq = 0;
 #pragma unroll
-    for (int k = 0; k < G; ++k) sigma_addends4<DT == kBF16>(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
-    long long Is, Iq;
-    team_sum2(team, (int32_t)(as - (uint32_t)G * kMagicBits), (int32_t)(aq - (uint32_t)G * kMagicBits), Is, Iq, rp);
-    float tlo, thi;
-    if (TT > 32) sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
-    else sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, tlo, thi);
-    uint32_t cnt = 0;
-    if (hi > thi || lo < tlo) {  // otherwise no element can lie outside: the count is zero
-      uint32_t c[4] = {0, 0, 0, 0};  // four counters: short dependency chains
-      if (lo >= tlo) {               // nothing below: one compare per element
+      for (int k = 0; k < G; ++k) sigma_addends4<DT == kBF16>(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
+      long long Is, Iq;
+      team_sum2(team, (int32_t)(as - (uint32_t)G * kMagicBits), (int32_t)(aq - (uint32_t)G * kMagicBits), Is, Iq, rp);
+      float dlo, dhi;
+      sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, dlo, dhi);
+      uint32_t cnt = 0;
+      if (range > dhi || 0.0f < dlo) {  // otherwise no element can lie outside: the count is zero
+        uint32_t c[4] = {0, 0, 0, 0};  // four counters: short dependency chains
+        if (!(0.0f < dlo)) {           // nothing below: one compare per element
 #pragma unroll
-        for (int k = 0; k < G; ++k) {
+          for (int k = 0; k < G; ++k) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) c[e] += x[k][e] > thi;
+            for (int e = 0; e < 4; ++e) c[e] += x[k][e] > dhi;
+          }
+          cnt = (c[0] + c[1]) + (c[2] + c[3]);
+        } else {
+#pragma unroll
+          for (int k = 0; k < G; ++k) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) c[e] += (x[k][e] > dhi) || (x[k][e] < dlo);
+          }
+          cnt = (c[0] + c[1]) + (c[2] + c[3]);
+          if (!(FULL && VEC)) cnt -= npad;  // padded positions (distance 0, below the lower threshold) are not elements
         }
-        cnt = (c[0] + c[1]) + (c[2] + c[3]);
-        if (!(FULL && VEC) && 0.0f > thi) cnt -= npad;  // padded zeros are not elements
-      } else {
-#pragma unroll
-        for (int k = 0; k < G; ++k) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) c[e] += (x[k][e] > thi) || (x[k][e] < tlo);
-        }
-        cnt = (c[0] + c[1]) + (c[2] + c[3]);
-        if (!(FULL && VEC) && ((0.0f > thi) || (0.0f < tlo))) cnt -= npad;
+        cnt = team_sum_u32(team, cnt, rp);
       }
-      cnt = team_sum_u32(team, cnt, rp);
+      n_out = cnt;
+      if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
     }
-    n_out = cnt;
-    if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
   } else if (pl.mode == kModeAll) {
     cls = kClsSalient;
   } else if (pl.mode >= kModeChannel) {
     cls = channel_class(pl, a, gp, n_out);
   }
 
-  r.lo = 0.0f;
-  r.scale = 0.0f;
-  r.size = 0;
-  r.meta = cls | (n_out << 2);
-  if (cls != kClsNormal) return;
+  const uint32_t meta = cls | (n_out << 2);
+  if (cls != kClsNormal || !d.fits) return meta;
   const uint32_t bits = (uint32_t)pl.bits;
   float inv, scale;
-  quant_params(lo, hi, (1u << bits) - 1u, inv, scale);
-  r.lo = lo;
-  r.scale = scale;
-  if (!d.fits) return;
+  quant_params(range, (1u << bits) - 1u, inv, scale);
   uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
   if (bits == 2u) FH_STORE_CODES(2)
   else if (bits == 4u) FH_STORE_CODES(4)
@@ -695,28 +783,94 @@ __device__ __forceinline__ void plane_sweep(const Team& team, const Plan& pl, co
     for (uint32_t o = a4(code_bytes) + 4u * lane; o < pl.npay; o += 4u * TT)
       *reinterpret_cast<uint32_t*>(slot + o) = 0u;
   }
-  if (lane == 0) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
+  if (lane == 0) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), meta, lo, scale);
+  return meta;
 }
 
 // Picks the specialisation of the sweep.  FULLVEC kernels are launched only for planes of exactly
 // G * TT whole groups, so they carry nothing but the lean variant; the others choose at run time.
 template <int DT, bool SIGMA, int G, int TT, bool FULLVEC>
-__device__ __forceinline__ void plane_sweep_any(const Team& team, const Plan& pl, const Dest& d,
-                                                const CompressArgs& a, const uint8_t* plane, uint64_t gp,
-                                                bool vec, uint32_t& rp, Rec& r) {
-  if (FULLVEC) plane_sweep<DT, SIGMA, G, TT, true, true>(team, pl, d, a, plane, gp, rp, r);
-  else if (vec) plane_sweep<DT, SIGMA, G, TT, false, true>(team, pl, d, a, plane, gp, rp, r);
-  else plane_sweep<DT, SIGMA, G, TT, false, false>(team, pl, d, a, plane, gp, rp, r);
+__device__ __forceinline__ uint32_t plane_sweep_any(const Team& team, const Plan& pl, const Dest& d,
+                                                    const CompressArgs& a, const uint8_t* plane, uint64_t gp,
+                                                    bool vec, uint32_t& rp) {
+  if (FULLVEC) return plane_sweep<DT, SIGMA, G, TT, true, true>(team, pl, d, a, plane, gp, rp);
+  if (vec) return plane_sweep<DT, SIGMA, G, TT, false, true>(team, pl, d, a, plane, gp, rp);
+  return plane_sweep<DT, SIGMA, G, TT, false, false>(team, pl, d, a, plane, gp, rp);
 }
 
 // -------------------------------------------------------------------------------------------------
 // Warp-team streaming kernel: planes of at most 256 groups.  Eight consumer warps and one producer
-// warp per CTA.  The producer hands out tiles and streams them into a ring of shared-memory stages
-// with bulk copies.  The consumer warps never wait for each other: each sweeps its own planes of a
-// tile (statistics, class, codes, stores), lists the planes that take the block-wise path, and
-// arrives on the stage's barrier.
+// warp per CTA.  The producer requests tiles and streams them into a ring of shared-memory stages
+// with bulk copies.  A consumer warp sweeps its own planes of a tile (statistics, class, codes, stores).
+// Outlier-rich planes are rare: a warp that has some in its slice measures them, the tile's eight
+// warps add up their overflow sizes in shared memory, the last of them to get there publishes the
+// tile's total and obtains the tile's place from the scan, and the warps that need it wait for that one
+// word before they write.  Warps without such planes wait for nobody.
 // -------------------------------------------------------------------------------------------------
 constexpr int kWarpKernelThreads = kThreads + 32;
+
+// What a warp knows about the outlier-rich planes of its slice after measuring them.
+struct WarpSal {
+  uint32_t units;      // lane j: overflow units of the slice's j-th such plane ...
+  uint32_t excl;       // ... and of those before it
+  uint32_t raw;        // ... 1: stored raw
+  uint32_t total;      // of the slice
+  uint32_t nsal, nraw;
+  uint32_t last_j;     // the plane whose measuring results still lie in the warp's area
+  SalientInfo last_info;
+};
+
+template <int DT, int TT>
+__device__ __noinline__ void warp_measure(const Plan& spl, const uint8_t* stage, uint32_t lp0, uint32_t leaders,
+                                          uint32_t* sal, WarpSal& ws) {
+  const Team team = make_warp_team(nullptr);
+  const uint32_t lane = team.lane;
+  ws.units = 0;
+  ws.raw = 0;
+  uint32_t j = 0;
+  for (uint32_t m = leaders; m; m &= m - 1u, ++j) {
+    const uint32_t lp = lp0 + ((uint32_t)__ffs((int)m) - 1u) / TT;
+    if (j) __syncwarp();
+    const SalientInfo info = salient_measure<DT>(team, spl, stage + (uint64_t)lp * spl.plane_bytes, sal);
+    bool raw;
+    const uint32_t u = plane_units(spl, info, raw);
+    if (lane == j) {
+      ws.units = u;
+      ws.raw = raw;
+    }
+    ws.last_info = info;
+    ws.last_j = j;
+  }
+  uint32_t incl = ws.units;
+  for (uint32_t o = 1; o < 32u; o <<= 1) {
+    const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  ws.excl = incl - ws.units;
+  ws.total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+  ws.nraw = __popc(__ballot_sync(0xFFFFFFFFu, ws.raw != 0u));
+  ws.nsal = j - ws.nraw;
+}
+
+template <int DT, int TT>
+__device__ __noinline__ void warp_write(const Plan& spl, const Dest d, const uint8_t* stage, uint64_t p0, uint32_t lp0,
+                                        uint32_t leaders, uint32_t meta, uint32_t* sal, const WarpSal& ws, uint32_t base) {
+  const Team team = make_warp_team(nullptr);
+  for (uint32_t j = (uint32_t)__popc(leaders); j-- > 0;) {  // the plane measured last comes first: its results are still there
+    const uint32_t src = __fns(leaders, 0u, (int)j + 1);
+    const uint32_t lp = lp0 + src / TT;
+    const uint8_t* plane = stage + (uint64_t)lp * spl.plane_bytes;
+    SalientInfo info = ws.last_info;
+    if (j != ws.last_j) {
+      __syncwarp();
+      info = salient_measure<DT>(team, spl, plane, sal);
+    }
+    const uint32_t n_out = __shfl_sync(0xFFFFFFFFu, meta, (int)src) >> 2;
+    const uint32_t at = base + __shfl_sync(0xFFFFFFFFu, ws.excl, (int)j);
+    write_blockwise<DT>(team, spl, d, p0 + lp, plane, info, sal, n_out, at);
+    __syncwarp();
+  }
+}
 
 template <int DT, bool SIGMA, int TT, bool FULLVEC>
 __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Plan pl, const CompressArgs a) {
@@ -725,20 +879,34 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
   __shared__ __align__(8) uint64_t s_full[kMaxStages], s_empty[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
   __shared__ volatile uint32_t s_abort;
+  __shared__ uint32_t s_last;
+  // placement of the outlier-rich planes of a tile (see above)
+  __shared__ uint32_t s_wu[kMaxStages][kWarps], s_wc[kMaxStages][kWarps], s_arr[kMaxStages], s_base[kMaxStages];
+  __shared__ volatile uint32_t s_ready[kMaxStages];
+  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
 
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const uint32_t nstage = pl.nstage;
-  dep_trigger();  // the next kernel on the stream may become resident as this one drains
+  const bool scan_on = pl.mode != kModeOff;
+  uint32_t first_ticket = 0;
   if (tid == 0) {
     for (uint32_t s = 0; s < nstage; ++s) {
       mbar_init(&s_full[s], 1);
       mbar_init(&s_empty[s], kWarps);
+      s_arr[s] = 0;
+      s_ready[s] = 0;
     }
     fence_mbar_init();
     s_abort = 0;
+    if (scan_on) s_pl = pl;
   }
+  // (the ticket counter of this call was returned to zero by the call before the previous one, which had
+  // completed before the previous kernel let this one start)
+  if (tid == (uint32_t)kThreads && a.early_ticket)
+    first_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
   __syncthreads();
-  dep_wait();  // the previous kernel on the stream has completed; global memory may be touched from here on
+  dep_wait();     // the previous kernel on the stream has completed; global memory may be touched from here on
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
   const Dest d = make_dest(pl, a);
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
 
@@ -746,6 +914,9 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     // ======================= producer (all 32 lanes walk the loop, lane 0 issues) =======================
     uint32_t s = 0, empty_phase = 0;
     bool aborted = false;
+    if (!a.early_ticket && lane == 0)
+      first_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
+    first_ticket = __shfl_sync(0xFFFFFFFFu, first_ticket, 0);
     // Waits until every consumer warp is done with the tile in stage q.
     auto drain = [&](uint32_t q) -> bool {
       bool ok = mbar_wait_abortable(&s_empty[q], (empty_phase >> q) & 1u, 1u << 20, &s_abort);
@@ -758,10 +929,10 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
         aborted = true;
         break;
       }
-      // the first tile of every stage follows from the CTA's index; later tiles are handed out
-      uint32_t t = blockIdx.x + n * gridDim.x;
+      // tiles come in ticket order: the first nstage of them in one request, then one at a time
+      uint32_t t = first_ticket + n;
       if (n >= nstage) {
-        if (lane == 0) t = nstage * gridDim.x + (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+        if (lane == 0) t = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
         t = __shfl_sync(0xFFFFFFFFu, t, 0);
       }
       if (t >= pl.ntiles) {
@@ -770,7 +941,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
         uint32_t q = first % nstage;
         __syncwarp();
         if (lane == 0) {
-          s_tiles[s] = t;
+          s_tiles[s] = 0xFFFFFFFFu;
           mbar_arrive(&s_full[s]);
         }
         for (uint32_t m = first; m < n; ++m) {
@@ -815,9 +986,10 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     // ======================= consumers =======================
     constexpr int G = 8;  // groups per thread: a plane has at most 8 * TT groups
     const Team team = make_team(TT, s_red);
-    const uint32_t my_team = tid / TT;
+    const uint32_t my_team = tid / TT, lp0 = (warp * 32u) / TT;
     const bool vec = (pl.plane_bytes & 15u) == 0u;
-    uint32_t rp = 0, s = 0, phase = 0;
+    uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + warp * pl.sal_stride);
+    uint32_t rp = 0, s = 0, phase = 0, seq = 0;
     for (;;) {
       const uint32_t par = (phase >> s) & 1u;
       bool ok = mbar_wait_abortable(&s_full[s], par, 1u << 20, &s_abort);
@@ -829,24 +1001,65 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       phase ^= 1u << s;
       const uint32_t tile = s_tiles[s];
       if (tile >= pl.ntiles) break;
+      ++seq;
       const uint32_t p0 = tile * pl.ppt;
       const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
       const uint32_t lp = my_team;
       const bool active = lp < np;
-      const uint8_t* plane = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes + (uint64_t)lp * pl.plane_bytes;
-      Rec r;
-      r.meta = kClsNormal;
-      if (active) plane_sweep_any<DT, SIGMA, G, TT, FULLVEC>(team, pl, d, a, plane, (uint64_t)p0 + lp, vec, rp, r);
-      // planes that take the block-wise path: marker in the table, entry in the work list
-      const bool mine = active && (r.meta & 3u) != kClsNormal && team.lane == 0;
-      const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine);
-      if (leaders) {
-        uint32_t base = 0;
-        if (lane == 0) base = (uint32_t)atomicAdd(&a.sc->wl_count, (unsigned long long)__popc(leaders));
-        base = __shfl_sync(0xFFFFFFFFu, base, 0);
-        if (mine) {
-          a.worklist[base + __popc(leaders & ((1u << lane) - 1u))] = p0 + lp;
-          if (d.fits) store_marker(d, (uint64_t)p0 + lp, r.meta);
+      const uint8_t* stage = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+      uint32_t meta = kClsNormal;
+      if (active)
+        meta = plane_sweep_any<DT, SIGMA, G, TT, FULLVEC>(team, pl, d, a, stage + (uint64_t)lp * pl.plane_bytes,
+                                                          (uint64_t)p0 + lp, vec, rp);
+      if (scan_on) {
+        const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, active && (meta & 3u) != kClsNormal && team.lane == 0);
+        WarpSal ws;
+        ws.total = ws.nsal = ws.nraw = 0;
+        if (leaders) warp_measure<DT, TT>(s_pl, stage, lp0, leaders, sal, ws);
+        uint32_t old = 0;
+        if (lane == 0) {
+          s_wu[s][warp] = ws.total;
+          s_wc[s][warp] = ws.nsal | (ws.nraw << 16);
+          __threadfence_block();
+          old = atomicAdd(&s_arr[s], 1u);
+        }
+        old = __shfl_sync(0xFFFFFFFFu, old, 0);
+        if ((old & 7u) == 7u) {  // the last of the tile's eight warps: publish the tile, obtain its place
+          __threadfence_block();
+          uint32_t U = lane < (uint32_t)kWarps ? s_wu[s][lane] : 0u, C = lane < (uint32_t)kWarps ? s_wc[s][lane] : 0u;
+          asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(U) : "r"(0xFFFFFFFFu));
+          asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(C) : "r"(0xFFFFFFFFu));
+          if (lane == 0) {
+            scan_publish(a.scan, tile, U);
+            count_blockwise(a, U, C & 0xFFFFu, C >> 16);
+          }
+          if (U) {
+            uint32_t base = 0;
+            const bool got = scan_prefix(a.scan, tile, base);
+            if (lane == 0) {
+              if (!got) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+              s_base[s] = base;
+              __threadfence_block();
+              s_ready[s] = got ? seq : (seq | 0x80000000u);
+            }
+          }
+        }
+        if (leaders) {
+          uint32_t base = 0;
+          bool placed = true;
+          if (ws.total) {  // wait (bounded) for the tile's place
+            uint32_t v = 0;
+            for (uint32_t k = 0; k < a.scan.polls; ++k) {
+              v = s_ready[s];
+              if ((v & 0x7FFFFFFFu) == seq) break;
+              __nanosleep(64);
+            }
+            placed = v == seq;
+            __threadfence_block();
+            base = s_base[s];
+            for (uint32_t w = 0; w < warp; ++w) base += s_wu[s][w];
+          }
+          if (placed) warp_write<DT, TT>(s_pl, d, stage, (uint64_t)p0, lp0, leaders, meta, sal, ws, base);
         }
       }
       __syncwarp();
@@ -855,17 +1068,17 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       s = s + 1 == nstage ? 0 : s + 1;
     }
   }
-  if (pl.mode == kModeOff) cta_exit<true>(pl, a, d);
-  else cta_exit<false>(pl, a, d);
+  cta_exit(pl, a, d, &s_last);
 }
 
 // -------------------------------------------------------------------------------------------------
 // CTA-team kernel: planes of more than 256 groups (whole 16-byte chunks).  One plane per tile, all
 // NT threads of the CTA work on it.  The plane stays in its shared-memory stage and is swept two or
-// three times (min/max; fixed-point moments; count + codes), so that few registers are needed and
+// three times (min/max; integer moments; count + codes), so that few registers are needed and
 // shared memory alone limits how many CTAs fit an SM (two stages each).  What every warp repeats per
 // plane -- reductions, thresholds, quantiser parameters -- does not shrink with the warp's share of the
 // plane, so NT is kept small for small planes.  Thread 0 keeps the next ticket in flight while the CTA works.
+// An outlier-rich plane is measured and written by the whole CTA while it lies in its stage.
 // -------------------------------------------------------------------------------------------------
 template <int DT>
 __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, float (&v)[4]) {
@@ -878,23 +1091,36 @@ __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, floa
     v[2] = __uint_as_float(t2.y << 16); v[3] = __uint_as_float(t2.y & 0xFFFF0000u);
   }
 }
+// The group's distances from lo (x - lo is x + (-lo): the same rounding).
+template <int DT>
+__device__ __forceinline__ void lds_dist(const uint8_t* plane, uint32_t g, float nlo, float (&v)[4]) {
+  lds_group<DT>(plane, g, v);
+  if (DT == kBF16) {
+    const f32x2 nlo2 = pack2(nlo, nlo);
+    unpack2(add2(pack2(v[0], v[1]), nlo2), v[0], v[1]);
+    unpack2(add2(pack2(v[2], v[3]), nlo2), v[2], v[3]);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) v[e] = __fadd_rn(v[e], nlo);
+  }
+}
 
 #define FH_CTA_STORE_CODES(BITS)                                                                              \
   {                                                                                                           \
     constexpr uint32_t bias = kMagicBits * (1u + (1u << (BITS)) + (1u << (2 * (BITS))) + (1u << (3 * (BITS)))); \
-    const f32x2 nlo2 = pack2(-lo, -lo), inv2 = pack2(inv, inv), mag2 = pack2(kMagicF, kMagicF);                 \
+    const f32x2 inv2 = pack2(inv, inv), mag2 = pack2(kMagicF, kMagicF);                                         \
     _Pragma("unroll 2") for (uint32_t g = tid; g < groups; g += NT) {                                         \
       float v[4];                                                                                             \
-      lds_group<DT>(plane, g, v);                                                                             \
+      lds_dist<DT>(plane, g, nlo, v);                                                                         \
       uint32_t w0, w1, w2, w3;                                                                                \
       if (DT == kBF16) {                                                                                      \
-        unpack2u(fma2(add2(pack2(v[0], v[1]), nlo2), inv2, mag2), w0, w1);                                    \
-        unpack2u(fma2(add2(pack2(v[2], v[3]), nlo2), inv2, mag2), w2, w3);                                    \
+        unpack2u(fma2(pack2(v[0], v[1]), inv2, mag2), w0, w1);                                                \
+        unpack2u(fma2(pack2(v[2], v[3]), inv2, mag2), w2, w3);                                                \
       } else {                                                                                                \
-        w0 = __float_as_uint(__fmaf_rn(__fsub_rn(v[0], lo), inv, kMagicF));                                   \
-        w1 = __float_as_uint(__fmaf_rn(__fsub_rn(v[1], lo), inv, kMagicF));                                   \
-        w2 = __float_as_uint(__fmaf_rn(__fsub_rn(v[2], lo), inv, kMagicF));                                   \
-        w3 = __float_as_uint(__fmaf_rn(__fsub_rn(v[3], lo), inv, kMagicF));                                   \
+        w0 = __float_as_uint(__fmaf_rn(v[0], inv, kMagicF));                                                  \
+        w1 = __float_as_uint(__fmaf_rn(v[1], inv, kMagicF));                                                  \
+        w2 = __float_as_uint(__fmaf_rn(v[2], inv, kMagicF));                                                  \
+        w3 = __float_as_uint(__fmaf_rn(v[3], inv, kMagicF));                                                  \
       }                                                                                                       \
       uint32_t word = w0 + (w1 << (BITS)) + (w2 << (2 * (BITS))) + (w3 << (3 * (BITS))) - bias;               \
       if ((BITS) == 2) slot[g] = (uint8_t)word;                                                               \
@@ -902,11 +1128,11 @@ __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, floa
       else reinterpret_cast<uint32_t*>(slot)[g] = word;                                                       \
       if (COUNT) {                                                                                            \
         if (one_sided) {                                                                                      \
-          c0 += (v[0] > thi) + (v[2] > thi);                                                                  \
-          c1 += (v[1] > thi) + (v[3] > thi);                                                                  \
+          c0 += (v[0] > dhi) + (v[2] > dhi);                                                                  \
+          c1 += (v[1] > dhi) + (v[3] > dhi);                                                                  \
         } else {                                                                                              \
-          c0 += ((v[0] > thi) || (v[0] < tlo)) + ((v[2] > thi) || (v[2] < tlo));                              \
-          c1 += ((v[1] > thi) || (v[1] < tlo)) + ((v[3] > thi) || (v[3] < tlo));                              \
+          c0 += ((v[0] > dhi) || (v[0] < dlo)) + ((v[2] > dhi) || (v[2] < dlo));                              \
+          c1 += ((v[1] > dhi) || (v[1] < dlo)) + ((v[3] > dhi) || (v[3] < dlo));                              \
         }                                                                                                     \
       }                                                                                                       \
     }                                                                                                         \
@@ -919,24 +1145,31 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
   __shared__ double s_red[kMaxWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
-  __shared__ uint32_t s_abort;
+  __shared__ uint32_t s_abort, s_last, s_base, s_ok;
+  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
 
   const uint32_t tid = threadIdx.x;
   const Team team = make_team(NT, s_red);
   const uint32_t nstage = pl.nstage, groups = pl.groups, bits = (uint32_t)pl.bits;
+  const bool scan_on = pl.mode != kModeOff;
+  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal);
   uint32_t rp = 0;
-  dep_trigger();  // the next kernel on the stream may become resident as this one drains
+  // Thread 0 requests the tiles and issues the loads: the first nstage tiles in one request, later ones one
+  // at a time, the request running one tile ahead of its use.  Tiles come in ticket order.
+  uint32_t next_ticket = 0, issued = 0;
   if (tid == 0) {
     for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
     fence_mbar_init();
     s_abort = 0;
+    if (scan_on) s_pl = pl;
+    // (the ticket counter of this call was returned to zero by the call before the previous one, which had
+    // completed before the previous kernel let this one start)
+    if (a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
   }
-  dep_wait();  // the previous kernel on the stream has completed; global memory may be touched from here on
+  dep_wait();     // the previous kernel on the stream has completed; global memory may be touched from here on
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
   const Dest d = make_dest(pl, a);
   if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
-  // Thread 0 issues the loads.  The first tile of every stage follows from the CTA's index; later tiles
-  // are handed out, the request running one tile ahead of its use.
-  uint32_t next_ticket = blockIdx.x, issued = 0;
   auto issue = [&](uint32_t s) {
     const uint32_t t = next_ticket;
     s_tiles[s] = t;
@@ -946,12 +1179,13 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
       bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + (uint64_t)t * pl.plane_bytes,
                (uint32_t)pl.plane_bytes, &s_full[s]);
       ++issued;
-      next_ticket = issued < nstage ? blockIdx.x + issued * gridDim.x
-                                    : nstage * gridDim.x + (uint32_t)atomicAdd(&a.sc->ticket, 1ull);
+      next_ticket = issued < nstage ? t + 1u : (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
     }
   };
-  if (tid == 0)
+  if (tid == 0) {
+    if (!a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
     for (uint32_t s = 0; s < nstage; ++s) issue(s);
+  }
   __syncthreads();
 
   uint32_t s = 0, phase = 0;
@@ -985,38 +1219,40 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     hi = max_nan(hi, hi1);
     team_minmax(team, lo, hi, rp);  // one barrier: also tells every thread about an abort
     if (s_abort) break;
-    if (!(fabsf(__fsub_rn(hi, lo)) <= 3.402823466e38f) && tid == 0)
-      atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+    const float range = __fsub_rn(hi, lo), nlo = -lo;
+    if (!(fabsf(range) <= 3.402823466e38f) && tid == 0) atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
 
-    // ---- sweep 2: fixed-point moments, thresholds
-    float tlo = 0.0f, thi = 0.0f;
+    // ---- sweep 2: integer moments of the distances from lo, thresholds
+    float dlo = 0.0f, dhi = 0.0f;
     bool one_sided = true, need_count = false;
     if (SIGMA) {
-      const SigmaScale sc = sigma_scale(lo, hi);
-      uint32_t as = 0, aq = 0, ng = 0;
+      const SigmaScale sc = sigma_scale(range);
+      if (sc.applies) {  // (the same for every thread)
+        uint32_t as = 0, aq = 0, ng = 0;
 #pragma unroll 2
-      for (uint32_t g = tid; g < groups; g += NT) {
-        float v[4];
-        lds_group<DT>(plane, g, v);
-        sigma_addends4<DT == kBF16>(v[0], v[1], v[2], v[3], sc, as, aq);
-        ++ng;
+        for (uint32_t g = tid; g < groups; g += NT) {
+          float v[4];
+          lds_dist<DT>(plane, g, nlo, v);
+          sigma_addends4<DT == kBF16>(v[0], v[1], v[2], v[3], sc, as, aq);
+          ++ng;
+        }
+        long long Is, Iq;
+        team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
+        sigma_thresholds(Is, Iq, sc, pl.inv_hw, dlo, dhi);
+        need_count = range > dhi || 0.0f < dlo;  // otherwise no element can lie outside
+        one_sided = !(0.0f < dlo);
       }
-      long long Is, Iq;
-      team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
-      sigma_thresholds(Is, Iq, sc, pl.inv_hw, tlo, thi);
-      need_count = hi > thi || lo < tlo;  // otherwise no element can lie outside
-      one_sided = lo >= tlo;
     }
 
     // ---- sweep 3: codes into the plane's slot (and the outlier count).  A plane that turns out
-    // salient has its slot rewritten by the block-wise kernels.
+    // outlier-rich has its slot rewritten below.
     float inv, scale;
-    quant_params(lo, hi, (1u << bits) - 1u, inv, scale);
+    quant_params(range, (1u << bits) - 1u, inv, scale);
     uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
     uint32_t c0 = 0, c1 = 0;
     if (d.fits && pl.mode != kModeAll) {
       if (!need_count) {
-        thi = __int_as_float(0x7F800000);  // nothing is counted
+        dhi = __int_as_float(0x7F800000);  // nothing is counted
         one_sided = true;
       }
       if (bits == 2u) FH_CTA_STORE_CODES(2)
@@ -1029,33 +1265,48 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     } else if (SIGMA && need_count) {  // nothing may be stored: count only
       for (uint32_t g = tid; g < groups; g += NT) {
         float v[4];
-        lds_group<DT>(plane, g, v);
+        lds_dist<DT>(plane, g, nlo, v);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) c0 += (v[e] > thi) || (v[e] < tlo);
+        for (int e = 0; e < 4; ++e) c0 += (v[e] > dhi) || (v[e] < dlo);
       }
     }
     uint32_t cls = kClsNormal, n_out = 0;
     if (SIGMA) {
-      n_out = team_sum_u32(team, c0 + c1, rp);  // its barrier: every thread is done with the stage
+      n_out = team_sum_u32(team, c0 + c1, rp);  // its barrier: every thread is done with the sweeps
       if ((uint64_t)n_out * pl.rho_den > (uint64_t)pl.rho_num * pl.HW) cls = kClsSalient;
     } else {
       if (pl.mode == kModeAll) cls = kClsSalient;
       if (pl.mode >= kModeChannel) cls = channel_class(pl, a, gp, n_out);
-      __syncthreads();  // every thread is done with the stage
+      __syncthreads();  // every thread is done with the sweeps
     }
-    if (tid == 0) {
-      Rec r;
-      r.size = 0;
-      r.meta = cls | (n_out << 2);
-      if (cls == kClsNormal) {
-        r.lo = lo;
-        r.scale = scale;
-        if (d.fits) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), r);
-      } else {
-        if (d.fits) store_marker(d, gp, r.meta);
-        list_plane(a, gp);
+    if (cls == kClsNormal) {
+      if (tid == 0) {
+        if (d.fits) store_table_entry(d, gp, (uint32_t)((pl.slots_off + gp * pl.npay) >> 4), cls | (n_out << 2), lo, scale);
+        if (scan_on) scan_publish(a.scan, tile, 0u);
+        issue(s);  // the stage is free: next load
       }
-      issue(s);  // the stage is free: next load
+    } else {  // (the same for every thread) measured, placed and written while the plane lies in its stage
+      const SalientInfo info = salient_measure<DT>(team, s_pl, plane, sal);
+      bool raw;
+      const uint32_t my_units = plane_units(pl, info, raw);
+      if (tid < 32u) {
+        bool got = true;
+        uint32_t base = 0;
+        if (tid == 0) {
+          scan_publish(a.scan, tile, my_units);
+          count_blockwise(a, my_units, raw ? 0u : 1u, raw ? 1u : 0u);
+        }
+        if (my_units) got = scan_prefix(a.scan, tile, base);
+        if (tid == 0) {
+          if (!got) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+          s_base = base;
+          s_ok = got;
+        }
+      }
+      __syncthreads();
+      if (s_ok) write_blockwise<DT>(team, s_pl, d, gp, plane, info, sal, n_out, s_base);
+      __syncthreads();  // every thread is done with the stage
+      if (tid == 0) issue(s);
     }
     s = s + 1 == nstage ? 0 : s + 1;
     // s_tiles[s] for the next iteration was written at least one barrier ago (nstage >= 2)
@@ -1069,248 +1320,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
         mbar_wait(&s_full[k], 1u, 1u << 10);
       }
   }
-  if (pl.mode == kModeOff) cta_exit<true>(pl, a, d);
-  else cta_exit<false>(pl, a, d);
-}
-
-// =================================================================================================
-// Block-wise kernel: the planes of the work list
-// =================================================================================================
-// Runs after the streaming kernel whenever planes can take the block-wise path.  With an empty work
-// list one thread finishes the container.  Otherwise a unit -- one warp for planes up to 8 KB, the
-// whole CTA above -- takes entries i = unit, unit + units, ... of the list.
-//
-// Measuring phase: the unit copies the plane into its shared-memory buffer, measures it (block
-// classes, CSR and code sizes), decides salient versus raw, completes the plane's table entry (class;
-// the offset stays 0), leaves the three counts of a salient payload in the first 16 bytes of the
-// plane's slot, and adds the plane's overflow size to the sum of its chunk (a chunk is a run of
-// 2^chunk_shift consecutive planes; there are at most kMaxChunks chunks).
-//
-// A barrier over the grid separates the phases: all CTAs are resident (a cooperative launch of a grid
-// sized to what the device holds at once); the wait is bounded all the same, and a wait that runs out
-// ends the call with the time-out status instead of hanging.
-//
-// Writing phase: every CTA turns the chunk sums into chunk offsets.  A plane's place in the overflow
-// region is its chunk's offset plus the overflow sizes of the listed planes before it in the same
-// chunk, recomputed from their table classes and slot headers (nothing changes those words any more:
-// whoever stores to them stores the value that is already there).  The unit walks its entries in
-// reverse so that the plane it measured last is still in its buffer; the others are copied and
-// measured again.  The last CTA to leave finishes the container.
-__device__ __forceinline__ uint32_t salient_size(const Plan& pl, uint32_t nnz_s, uint32_t n_dense, uint32_t n_out_d) {
-  const uint32_t e = (uint32_t)pl.esize;
-  return 16u + 4u * pl.nbm + 4u * ((uint32_t)pl.H + 1u) + a4(2u * nnz_s) + a4(e * nnz_s) + 64u * n_dense +
-         a4(e * n_out_d);
-}
-// Overflow size, in 16-byte units, of a payload of `size` bytes.
-__device__ __forceinline__ uint32_t ovf_units(const Plan& pl, uint32_t size) {
-  return a16(size) > pl.npay ? (a16(size) - pl.npay) >> 4 : 0u;
-}
-
-// Copies plane p into the unit's buffer (whole 16-byte chunks from the aligned start, the ragged end
-// of the tensor byte-wise) and returns where the plane starts in it.
-__device__ __forceinline__ const uint8_t* fetch_plane(const Team& t, const Plan& pl, const uint8_t* src, uint32_t p,
-                                                      uint8_t* ubuf) {
-  const uint64_t start = (uint64_t)p * pl.plane_bytes, end = start + pl.plane_bytes;
-  const uint64_t a0 = start & ~15ull;
-  const uint64_t a1 = min((end + 15ull) & ~15ull, pl.dense_bytes & ~15ull);
-  const uint4* s16 = reinterpret_cast<const uint4*>(src + a0);
-  uint4* t16 = reinterpret_cast<uint4*>(ubuf);
-  const uint32_t n16 = (uint32_t)((a1 - a0) >> 4);
-  for (uint32_t k = t.lane; k < n16; k += t.size) t16[k] = __ldg(s16 + k);
-  for (uint64_t k = a1 + t.lane; k < end; k += t.size) ubuf[k - a0] = src[k];
-  team_sync(t);
-  return ubuf + (uint32_t)(start - a0);
-}
-
-constexpr uint32_t kGridWaitPolls = 1u << 21;  // about a second
-
-template <int DT>
-__global__ void __launch_bounds__(512) blockwise_kernel(const Plan pl, const CompressArgs a) {
-  extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ double s_red[kMaxWarps * 5];
-  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
-  __shared__ uint32_t s_ok;
-
-  const uint32_t tid = threadIdx.x, lane32 = tid & 31u, warp = tid >> 5;
-  // (launched in plain stream order: the streaming kernel has completed, its list, table and counters are visible)
-  const Dest d = make_dest(pl, a);
-  const uint32_t count = (uint32_t)ld_relaxed(&a.sc->wl_count);
-  if (count == 0) {  // nothing listed: the container lacks only its header
-    if (blockIdx.x == 0 && tid == 0) finalize(pl, a, d);
-    return;
-  }
-  if (tid == 0) s_pl = pl;
-  const bool unit_cta = pl.sk_cta != 0u;
-  const uint32_t upc = unit_cta ? 1u : blockDim.x >> 5;
-  const uint32_t unit = unit_cta ? blockIdx.x : blockIdx.x * upc + warp;
-  const uint32_t units = gridDim.x * upc;
-  const Team t = unit_cta ? make_team(blockDim.x, s_red) : make_warp_team(s_red);
-  uint8_t* ubuf = smem + (unit_cta ? 0u : warp * pl.sk_unit_stride);
-  // measuring areas of the unit: the n-th entry it takes uses area min(n, keep - 1); an area starts with
-  // the four sizes of SalientInfo, the measuring scratch follows
-  uint32_t* areas = reinterpret_cast<uint32_t*>(ubuf + pl.sk_sal_off);
-  const uint32_t keep = pl.sk_keep, area_words = pl.sk_area_words;
-  uint32_t* pre = reinterpret_cast<uint32_t*>(smem + pl.sk_pre_off);
-  const uint4* table = reinterpret_cast<const uint4*>(d.dst + 64);
-  const uint32_t raw_units = ovf_units(pl, (uint32_t)pl.plane_bytes);
-  __syncthreads();
-
-  // ---- measuring phase
-  uint32_t taken = 0;  // entries this unit has measured; the plane of the last one stays in the buffer
-  const uint8_t* plane = ubuf;
-  SalientInfo info;
-  info.nnz_s = info.n_dense = info.n_out_d = info.size = 0;
-  for (uint32_t i = unit; i < count; i += units, ++taken) {
-    if (taken) team_sync(t);  // the buffer is reused
-    const uint32_t p = a.worklist[i];
-    plane = fetch_plane(t, pl, a.src, p, ubuf);
-    uint32_t* area = areas + min(taken, keep - 1u) * area_words;
-    info = salient_measure<DT>(t, s_pl, plane, area + 4);
-    if (t.lane == 0) {
-      area[0] = info.nnz_s;
-      area[1] = info.n_dense;
-      area[2] = info.n_out_d;
-      area[3] = info.size;
-    }
-    const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
-    const uint32_t my_units = ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
-    if (t.lane == 0) {
-      if (d.fits) {
-        // the streaming kernel's marker says salient (class bits 01); a raw plane flips them to 10
-        if (raw)
-          atomicXor(reinterpret_cast<uint32_t*>(d.dst + 64 + 16ull * p) + 1, 3u);
-        else
-          *reinterpret_cast<uint4*>(d.dst + pl.slots_off + (uint64_t)p * pl.npay) =
-              make_uint4(info.nnz_s, info.n_dense, info.n_out_d, 0u);
-      }
-      if (my_units) {
-        atomicAdd(&a.chunk_ovf[p >> a.chunk_shift], my_units);
-        atomicAdd(&a.sc->ovf16, (unsigned long long)my_units);
-      }
-      atomicAdd(raw ? &a.sc->nraw : &a.sc->nsal, 1ull);
-    }
-  }
-
-  // ---- barrier over the grid (bounded)
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    atomicAdd(&a.sc->arrived, 1ull);
-    uint32_t ok = 0;
-    for (uint32_t k = 0; k < kGridWaitPolls; ++k) {
-      if (ld_acquire(&a.sc->arrived) >= (unsigned long long)gridDim.x) {
-        ok = 1;
-        break;
-      }
-      __nanosleep(200);
-    }
-    if (!ok) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-    s_ok = ok;
-  }
-  __syncthreads();
-  // Only now may the next kernel on the stream become resident: before the barrier its CTAs could take
-  // the place of CTAs of this grid that have not started yet, and the barrier would never complete.
-  dep_trigger();
-
-  // ---- writing phase
-  if (s_ok && d.fits && (unit_cta ? blockIdx.x : blockIdx.x * upc) < count) {  // CTAs without entries are done
-    // chunk offsets: exclusive prefix sum of the chunk sums (warp 0: consecutive chunks per lane)
-    {
-      uint32_t v[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint32_t k = tid + (uint32_t)q * blockDim.x;
-        v[q] = k < a.nchunks ? __ldcg(a.chunk_ovf + k) : 0u;
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const uint32_t k = tid + (uint32_t)q * blockDim.x;
-        if (k < kMaxChunks) pre[k] = v[q];
-      }
-    }
-    __syncthreads();
-    if (warp == 0) {
-      constexpr uint32_t per = kMaxChunks / 32;
-      uint32_t local = 0;
-      for (uint32_t k = 0; k < per; ++k) local += pre[lane32 * per + k];
-      uint32_t incl = local;
-      for (uint32_t o = 1; o < 32; o <<= 1) {
-        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane32 >= o) incl += up;
-      }
-      uint32_t run = incl - local;
-      for (uint32_t k = 0; k < per; ++k) {
-        const uint32_t v = pre[lane32 * per + k];
-        pre[lane32 * per + k] = run;
-        run += v;
-      }
-    }
-    __syncthreads();
-    if (taken) {
-      // last entry first: its plane is still in the buffer.  Entries whose area was not reused keep their
-      // measuring results; the others are measured again.
-      team_sync(t);
-      for (uint32_t n = taken; n-- > 0;) {
-        const uint32_t i = unit + n * units;
-        const uint32_t p = a.worklist[i];
-        uint32_t* area = areas + min(n, keep - 1u) * area_words;
-        if (n + 1u != taken) {
-          plane = fetch_plane(t, pl, a.src, p, ubuf);
-          if (n >= keep - 1u) {
-            info = salient_measure<DT>(t, s_pl, plane, area + 4);
-          } else {
-            info.nnz_s = area[0];
-            info.n_dense = area[1];
-            info.n_out_d = area[2];
-            info.size = area[3];
-          }
-        }
-        const uint32_t* sal = area + 4;
-        const bool raw = a16(info.size) >= a16((uint32_t)pl.plane_bytes);
-        const uint32_t my_units = ovf_units(pl, raw ? (uint32_t)pl.plane_bytes : info.size);
-        // overflow units of the listed planes before p in its chunk (every warp of the unit computes them)
-        uint32_t before = 0;
-        for (uint32_t q0 = (p >> a.chunk_shift) << a.chunk_shift; q0 < p; q0 += 32u) {
-          const uint32_t q = q0 + lane32;
-          uint32_t v = 0;
-          if (q < p) {
-            const uint32_t cls = __ldcg(reinterpret_cast<const uint32_t*>(table + q) + 1) & 3u;
-            if (cls == kClsRaw) {
-              v = raw_units;
-            } else if (cls == kClsSalient) {
-              const uint4 h = __ldcg(reinterpret_cast<const uint4*>(d.dst + pl.slots_off + (uint64_t)q * pl.npay));
-              v = ovf_units(pl, salient_size(pl, h.x, h.y, h.z));
-            }
-          }
-          asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(v) : "r"(0xFFFFFFFFu));
-          before += v;
-        }
-        const unsigned long long off16 = (pl.ovf_off >> 4) + pre[p >> a.chunk_shift] + before;
-        if ((off16 + my_units) * 16ull <= d.capacity) {  // never write past the capacity
-          SplitOut out;
-          out.slot = d.dst + pl.slots_off + (uint64_t)p * pl.npay;
-          out.ovf = d.dst + off16 * 16ull;
-          out.npay = pl.npay;
-          if (raw) raw_write(t, s_pl, plane, out);
-          else salient_write<DT>(t, s_pl, plane, info, sal, out);
-          if (t.lane == 0) *reinterpret_cast<uint32_t*>(d.dst + 64 + 16ull * p) = my_units ? (uint32_t)off16 : 0u;
-        }
-        team_sync(t);  // the buffer is reused
-      }
-    }
-  }
-  // last CTA to leave: clear the chunk sums (all threads), then finish the container (one thread)
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_ok = atomicAdd(&a.sc->exited, 1ull) == (unsigned long long)gridDim.x - 1ull;
-  __syncthreads();
-  if (!s_ok) return;
-  for (uint32_t k = tid; k < a.nchunks; k += blockDim.x) a.chunk_ovf[k] = 0u;
-  if (tid == 0) {
-    __threadfence();
-    st_relaxed(&a.sc->exited, 0ull);
-    finalize(pl, a, d);
-  }
+  cta_exit(pl, a, d, &s_last);
 }
 
 }  // namespace fh

@@ -53,32 +53,25 @@ struct Plan {
   uint32_t stage_bytes;  // fast kernels: bytes of one stage buffer (ppt * plane_bytes)
   // shared-memory layout (byte offsets into dynamic shared memory)
   uint32_t sm_tile, sm_out, sm_rec, sm_total;
-  // block-wise kernels: a unit (one warp, or the whole CTA for large planes) holds one plane
-  uint32_t sk_cta;          // 1: the unit is the CTA
-  uint32_t sk_threads;      // CTA size
-  uint32_t sk_sal_off;      // offset of the unit's measuring areas behind its plane buffer
-  uint32_t sk_keep;         // measuring areas per unit: results of that many planes survive until they are written
-  uint32_t sk_area_words;   // words per area: 4 (sizes) + sal_words
-  uint32_t sk_unit_stride;  // bytes of shared memory per unit
-  uint32_t sk_pre_off;      // offset of the chunk prefix array (kMaxChunks words)
-  uint32_t sk_total;
+  // block-wise path (outlier-rich planes): measuring scratch of one unit (a warp, or the whole CTA)
   uint32_t sal_words;       // words of measuring scratch per plane: H + 1 + 3 * nblk
+  uint32_t sm_sal;          // byte offset of the first measuring area in dynamic shared memory
+  uint32_t sal_stride;      // bytes between the areas of consecutive units
 };
 
-// Book-keeping scratch, one per stream: a header of counters, kMaxChunks chunk sums (see the
-// block-wise kernels) and the work list of planes that take the block-wise path.  Everything a call
-// changes is returned to zero by the last CTA of its last kernel.
+// Book-keeping scratch, one per stream: a header of counters and three arrays for the plane-ordered
+// placement of overflow parts (see "Placement scan" below).  Everything in the header that a call changes
+// is returned to zero by the last CTA of its kernel.
 struct Scratch {
-  unsigned long long ticket;    // next tile
-  unsigned long long exited;    // CTAs that have left the running kernel
-  unsigned long long status;    // device error code (atomicMax)
-  unsigned long long ovf16;     // overflow region size of this call, in 16-byte units
+  unsigned long long ticket[2];  // next tile; consecutive compress calls on a stream alternate between the two
+  unsigned long long exited;     // CTAs that have left the running kernel
+  unsigned long long status;     // device error code (atomicMax)
+  unsigned long long ovf16;      // overflow region size of this call, in 16-byte units
   unsigned long long nsal, nraw;
-  unsigned long long wl_count;  // entries of the work list
-  unsigned long long arrived;   // CTAs of the block-wise kernel that have finished measuring
+  unsigned long long reserved;
 };
 static_assert(sizeof(Scratch) == 64, "Scratch layout");
-constexpr uint32_t kMaxChunks = 1024;
+constexpr uint32_t kScratchHeadBytes = 256;  // the header, padded
 
 // (uint64)(int64) fh_status of a device error code.
 __device__ __forceinline__ unsigned long long status_word(uint32_t code) {
@@ -259,32 +252,35 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
   return r;
 }
 
-// Fixed-point moments of a plane (three-sigma rule): scale factors from the largest magnitude A.
+// Three-sigma rule: integer moment sums of the distances d = x - lo from the smallest element, scaled by
+// the exponent e of the range (2^e <= range < 2^(e+1)): a group of four contributes rne(s * 2^(18-e)) and
+// rne(q * 2^(16-2e)), both below 2^22.  The rule is applied for -40 <= e <= 60 only (no product can over-
+// or underflow there); a constant plane (range 0, exponent field 0) falls outside like any other.
 struct SigmaScale {
-  float cs, cq;    // 2^ks, 2^kq
-  int32_t ks, kq;
+  float cs, cq;   // 2^(18-e), 2^(16-2e)
+  int32_t e;
+  bool applies;
 };
-__device__ __forceinline__ SigmaScale sigma_scale(float lo, float hi) {
-  const float A = fmaxf(fabsf(lo), fabsf(hi));
-  const int e = (int)((__float_as_uint(A) >> 23) & 255u) - 127;
+__device__ __forceinline__ SigmaScale sigma_scale(float range) {
   SigmaScale s;
-  s.ks = min(18 - e, 126);
-  s.kq = max(min(16 - 2 * e, 126), -126);
-  s.cs = __uint_as_float((uint32_t)(s.ks + 127) << 23);
-  s.cq = __uint_as_float((uint32_t)(s.kq + 127) << 23);
+  s.e = (int)((__float_as_uint(range) >> 23) & 255u) - 127;
+  s.applies = s.e >= -40 && s.e <= 60;
+  const int32_t e = s.applies ? s.e : 0;
+  s.cs = __uint_as_float((uint32_t)(18 - e + 127) << 23);
+  s.cq = __uint_as_float((uint32_t)(16 - 2 * e + 127) << 23);
   return s;
 }
-// Raw mantissa images of the two fixed-point addends of one group; the caller sums them with
-// wrap-around arithmetic and subtracts kMagicBits once per group at the end.
-__device__ __forceinline__ void sigma_addends(const float v[4], const SigmaScale& sc, uint32_t& as, uint32_t& aq) {
-  const float sg = __fadd_rn(__fadd_rn(v[0], v[1]), __fadd_rn(v[2], v[3]));
-  const float q01 = __fmaf_rn(v[1], v[1], __fmul_rn(v[0], v[0]));
-  const float q23 = __fmaf_rn(v[3], v[3], __fmul_rn(v[2], v[2]));
+// Raw mantissa images of the two addends of one group of distances; the caller sums them with wrap-around
+// arithmetic and subtracts kMagicBits once per group at the end.
+__device__ __forceinline__ void sigma_addends(const float d[4], const SigmaScale& sc, uint32_t& as, uint32_t& aq) {
+  const float sg = __fadd_rn(__fadd_rn(d[0], d[1]), __fadd_rn(d[2], d[3]));
+  const float q01 = __fmaf_rn(d[1], d[1], __fmul_rn(d[0], d[0]));
+  const float q23 = __fmaf_rn(d[3], d[3], __fmul_rn(d[2], d[2]));
   const float qg = __fadd_rn(q01, q23);
   as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
   aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
 }
-// PACKED: the same arithmetic with packed pairs -- (v0, v2) and (v1, v3) give both halves of every step at
+// PACKED: the same arithmetic with packed pairs -- (d0, d2) and (d1, d3) give both halves of every step at
 // once.  Used for bf16 input, whose unpacked values can be put in any registers and whose kernels are bound
 // by instruction issue; on fp32 input the repacking costs more than it saves.
 template <bool PACKED>
@@ -293,8 +289,8 @@ __device__ __forceinline__ void sigma_addends4(float v0, float v1, float v2, flo
   if (PACKED) {
     const f32x2 ev = pack2(v0, v2), od = pack2(v1, v3);
     float s01, s23, q01, q23;
-    unpack2(add2(ev, od), s01, s23);                 // v0 + v1, v2 + v3
-    unpack2(fma2(od, od, mul2(ev, ev)), q01, q23);   // fma(v1, v1, v0 * v0), fma(v3, v3, v2 * v2)
+    unpack2(add2(ev, od), s01, s23);                 // d0 + d1, d2 + d3
+    unpack2(fma2(od, od, mul2(ev, ev)), q01, q23);   // fma(d1, d1, d0 * d0), fma(d3, d3, d2 * d2)
     const f32x2 fixed = fma2(pack2(__fadd_rn(s01, s23), __fadd_rn(q01, q23)), pack2(sc.cs, sc.cq), pack2(kMagicF, kMagicF));
     uint32_t is, iq;
     unpack2u(fixed, is, iq);
@@ -309,25 +305,24 @@ __device__ __forceinline__ void sigma_addends4(float v0, float v1, float v2, flo
     aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
   }
 }
-// Thresholds mu +- 3 sigma from the exact integer sums.
+// Thresholds, as distances from lo, from the exact integer sums: m1 +- 3 sigma.
 template <typename I>
-__device__ __forceinline__ void sigma_thresholds(I Is, I Iq, const SigmaScale& sc, double inv_hw, float& tlo,
-                                                 float& thi) {
-  const double ps = __hiloint2double((1023 - sc.ks) << 20, 0);  // 2^-ks
-  const double pq = __hiloint2double((1023 - sc.kq) << 20, 0);  // 2^-kq
-  const double mu = __dmul_rn(__dmul_rn((double)Is, ps), inv_hw);
-  const double m2 = __dmul_rn(__dmul_rn((double)Iq, pq), inv_hw);
-  double var = __dsub_rn(m2, __dmul_rn(mu, mu));
+__device__ __forceinline__ void sigma_thresholds(I Is, I Iq, const SigmaScale& sc, double inv_count, float& dlo,
+                                                 float& dhi) {
+  const double ps = __hiloint2double((1023 + sc.e - 18) << 20, 0);      // 2^(e-18)
+  const double pq = __hiloint2double((1023 + 2 * sc.e - 16) << 20, 0);  // 2^(2e-16)
+  const double m1 = __dmul_rn(__dmul_rn((double)Is, ps), inv_count);
+  const double m2 = __dmul_rn(__dmul_rn((double)Iq, pq), inv_count);
+  double var = __dsub_rn(m2, __dmul_rn(m1, m1));
   if (!(var > 0.0)) var = 0.0;
-  const float mu_f = __double2float_rn(mu);
+  const float m_f = __double2float_rn(m1);
   const float sigma_f = __fsqrt_rn(__double2float_rn(var));
-  thi = __fmaf_rn(3.0f, sigma_f, mu_f);
-  tlo = __fmaf_rn(-3.0f, sigma_f, mu_f);
+  dhi = __fmaf_rn(3.0f, sigma_f, m_f);
+  dlo = __fmaf_rn(-3.0f, sigma_f, m_f);
 }
 
 // Quantiser parameters of a normal plane.
-__device__ __forceinline__ void quant_params(float lo, float hi, uint32_t L, float& inv, float& scale) {
-  const float range = __fsub_rn(hi, lo);
+__device__ __forceinline__ void quant_params(float range, uint32_t L, float& inv, float& scale) {
   inv = __fdiv_rn((float)L, range);
   scale = __fdiv_rn(range, (float)L);
   if (range == 0.0f || !(fabsf(inv) <= 3.402823466e38f)) {
@@ -335,9 +330,10 @@ __device__ __forceinline__ void quant_params(float lo, float hi, uint32_t L, flo
     scale = 0.0f;
   }
 }
-// Code of one element: rne of the exact product (x - lo) * inv, as an integer in the mantissa.
-__device__ __forceinline__ uint32_t quant_code(float x, float lo, float inv, uint32_t L) {
-  const float r = __fmaf_rn(__fsub_rn(x, lo), inv, kMagicF);
+// Code of one element from its distance d = x - lo: rne of the exact product d * inv, as an integer in the
+// mantissa.
+__device__ __forceinline__ uint32_t quant_code(float d, float inv, uint32_t L) {
+  const float r = __fmaf_rn(d, inv, kMagicF);
   return (__float_as_uint(r) - kMagicBits) & L;
 }
 
@@ -362,10 +358,10 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
   out[2] = c2;
   out[3] = c3;
 }
-// Code of one element under random rounding: t = fp32 product (x - lo) * inv, n = floor(t), and the code
+// Code of one element (distance d = x - lo) under random rounding: t = fp32 product d * inv, n = floor(t), and the code
 // goes up iff floor(frac(t) * 2^24) + (word >> 8) reaches 2^24.
-__device__ __forceinline__ uint32_t quant_code_random(float x, float lo, float inv, uint32_t L, uint32_t word) {
-  const float t = __fmul_rn(__fsub_rn(x, lo), inv);
+__device__ __forceinline__ uint32_t quant_code_random(float d, float inv, uint32_t L, uint32_t word) {
+  const float t = __fmul_rn(d, inv);
   const float nf = floorf(t);
   const uint32_t fi = (uint32_t)__fmul_rn(__fsub_rn(t, nf), 16777216.0f);
   const uint32_t up = (fi + (word >> 8)) >> 24;
@@ -583,6 +579,107 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
   }
   team_sync(t);
   return total;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Placement scan
+// ------------------------------------------------------------------------------------------------
+// The overflow parts of outlier-rich and raw planes lie in plane order, so a plane's place is the sum of
+// the overflow sizes of all planes before it.  A tile (a run of consecutive planes, handed out in order by
+// a ticket) publishes the total U of its planes' overflow sizes as soon as it has measured them -- before
+// it waits for anything -- and a tile with U > 0 then needs the sum over all earlier tiles.  Two levels
+// keep that look-back short (sizes in units of 16 bytes):
+//   tile[t] = epoch << 32 | U_t          written once per call; an entry of another epoch reads as "not yet"
+//   grp[g]  = count << 40 | sum of U     over the tiles of group g = t >> 5 that have published (atomic adds;
+//                                        returned to zero by the call's last CTA)
+//   gpre[g] = epoch << 32 | sum of U     over all tiles of groups 0..g, published by whoever has worked it out
+// Progress: tiles are taken in ticket order by CTAs that are running, a CTA works through its tiles in
+// increasing order, and a tile publishes before it waits; so the smallest tile that has not published is
+// never waiting.  Every wait is bounded all the same and reports a time-out instead of hanging.
+struct Scan {
+  unsigned long long* tile;
+  unsigned long long* grp;
+  unsigned long long* gpre;
+  uint32_t epoch;      // of this call (never 0)
+  uint32_t polls;      // limit of every wait, in polls of about 0.1 us
+  uint32_t skip_tile;  // this tile never publishes (fault injection for the time-out test; 0xFFFFFFFF: none)
+  uint32_t reserved;
+};
+
+// One thread: tile t has measured its planes.
+__device__ __forceinline__ void scan_publish(const Scan& s, uint32_t t, uint32_t U) {
+  if (t == s.skip_tile) return;
+  st_relaxed(&s.tile[t], ((unsigned long long)s.epoch << 32) | U);
+  atomicAdd(&s.grp[t >> 5], (1ull << 40) | (unsigned long long)U);
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+  for (uint32_t o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// A whole warp: sum of U over the tiles before t.  False when a wait ran out.
+__device__ __noinline__ bool scan_prefix(const Scan& s, uint32_t t, uint32_t& prefix) {
+  const uint32_t lane = threadIdx.x & 31u, full = 0xFFFFFFFFu;
+  const uint32_t g = t >> 5, within = t & 31u;
+  // tiles of the own group before t
+  unsigned long long u = 0;
+  {
+    bool ok = lane >= within;
+    for (uint32_t k = 0; k < s.polls; ++k) {
+      if (!ok) {
+        const unsigned long long v = ld_relaxed(&s.tile[g * 32u + lane]);
+        if ((uint32_t)(v >> 32) == s.epoch) {
+          u = v & 0xFFFFFFFFull;
+          ok = true;
+        }
+      }
+      if (__all_sync(full, ok)) break;
+      __nanosleep(100);
+    }
+    if (!__all_sync(full, ok)) return false;
+  }
+  unsigned long long acc = warp_sum_u64(u);
+  // earlier groups, the nearest first, 32 at a time, until a group whose prefix somebody has published
+  unsigned long long gsum = 0;
+  uint32_t hi = g;
+  while (hi > 0) {
+    const bool act = lane < hi;
+    const uint32_t j = act ? hi - 1u - lane : 0u;
+    bool have_pre = false, done = !act;
+    unsigned long long val = 0;
+    uint32_t first = 32, need = full, dm = 0;
+    for (uint32_t k = 0; k < s.polls; ++k) {
+      if (act && !have_pre) {
+        const unsigned long long v = ld_relaxed(&s.gpre[j]);
+        if ((uint32_t)(v >> 32) == s.epoch) {
+          have_pre = true;
+          done = true;
+          val = v & 0xFFFFFFFFull;
+        }
+      }
+      if (act && !done) {
+        const unsigned long long v = ld_relaxed(&s.grp[j]);
+        if ((v >> 40) == 32ull) {  // every group before another one is a whole group of 32 tiles
+          done = true;
+          val = v & ((1ull << 40) - 1ull);
+        }
+      }
+      const uint32_t pm = __ballot_sync(full, have_pre);
+      first = pm ? (uint32_t)__ffs((int)pm) - 1u : 32u;
+      need = first >= 31u ? full : ((2u << first) - 1u);  // lanes 0..first
+      dm = __ballot_sync(full, done);
+      if ((dm & need) == need) break;
+      __nanosleep(100);
+    }
+    if ((dm & need) != need) return false;
+    gsum += warp_sum_u64(lane <= first ? val : 0ull);
+    if (first < 32u) break;
+    hi = hi > 32u ? hi - 32u : 0u;
+  }
+  if (g > 0 && lane == 0) st_relaxed(&s.gpre[g - 1u], ((unsigned long long)s.epoch << 32) | (gsum & 0xFFFFFFFFull));
+  prefix = (uint32_t)(gsum + acc);
+  return true;
 }
 
 }  // namespace fh

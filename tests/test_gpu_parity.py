@@ -303,14 +303,16 @@ def test_host_buffer_entry_points():
 def test_launch_counter_counts_our_kernels():
     before = api.kernel_launches()
     raw = synth.relu_normal(2 * 4 * 64, 1)
-    # three-sigma mode: streaming kernel + block-wise kernel, then one decompress kernel
+    # a compress call is one kernel, a decompress call is one kernel, whatever the mode
     st, packed, total = gpu_compress(raw, (2, 4, 8, 8), synth.F32, bits=2)
     api.decompress_tensor(packed, total, (2, 4, 8, 8), synth.F32)
-    assert api.kernel_launches() == before + 3
-    # every plane normal: the streaming kernel alone
+    assert api.kernel_launches() == before + 2
     st, packed, total = gpu_compress(raw, (2, 4, 8, 8), synth.F32, bits=2, salient_mode=api.FH_SALIENT_OFF)
     api.decompress_tensor(packed, total, (2, 4, 8, 8), synth.F32)
-    assert api.kernel_launches() == before + 5
+    assert api.kernel_launches() == before + 4
+    # the channel-wide mode adds its three statistics passes
+    st, packed, total = gpu_compress(raw, (2, 4, 8, 8), synth.F32, bits=2, salient_mode=api.FH_SALIENT_CHANNEL)
+    assert api.kernel_launches() == before + 8
 
 
 def test_back_to_back_calls_without_host_synchronisation():
