@@ -241,7 +241,7 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
  *     on the GPU (different streams without ordering between them) race on it: order them.
  */
 #define FH_STATIC_MAX_PLANES 131072
-#define FH_STATIC_SCRATCH_BYTES (256 + 8 * (FH_STATIC_MAX_PLANES + 2 * (FH_STATIC_MAX_PLANES / 32)))
+#define FH_STATIC_SCRATCH_BYTES (256 + 8 * (FH_STATIC_MAX_PLANES + 2 * (FH_STATIC_MAX_PLANES / 32)) + 4 * FH_STATIC_MAX_PLANES)
 int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                        size_t dst_capacity, uint64_t* d_out2, void* stream);
 

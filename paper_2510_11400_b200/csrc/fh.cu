@@ -213,7 +213,7 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
 // ---- per-stream scratch ---------------------------------------------------------------------
 struct StreamScratch {
   fh::Scratch* sc = nullptr;             // counters
-  unsigned long long* scan = nullptr;    // placement scan: tile words, then group sums, then group prefixes
+  unsigned long long* scan = nullptr;    // placement scan: tile words, group sums, group prefixes; then the tile links
   size_t tile_cap = 0;                   // tiles the scan arrays hold (groups: tile_cap / 32)
   uint32_t calls = 0;                    // compress calls so far: parity of the ticket counter, epoch of the scan
   uint32_t* plane_nout = nullptr;        // channel-wide three-sigma mode: per-plane counts ...
@@ -223,7 +223,7 @@ struct StreamScratch {
   unsigned long long* sched = nullptr;   // schedule runner: offsets, sizes, statuses
   size_t sched_cap = 0;
 };
-inline size_t scan_words(size_t tile_cap) { return tile_cap + 2 * (tile_cap / 32); }
+inline size_t scan_words(size_t tile_cap) { return tile_cap + 2 * (tile_cap / 32) + tile_cap / 2; }
 
 std::mutex g_mu;
 std::map<std::pair<int, cudaStream_t>, StreamScratch> g_scratch;
@@ -275,6 +275,7 @@ int next_call(uint32_t* calls, unsigned long long* scan, size_t tile_cap, cudaSt
   a->scan.tile = scan;
   a->scan.grp = scan ? scan + tile_cap : nullptr;
   a->scan.gpre = scan ? scan + tile_cap + tile_cap / 32 : nullptr;
+  a->defer_next = scan ? reinterpret_cast<uint32_t*>(scan + tile_cap + 2 * (tile_cap / 32)) : nullptr;
   a->scan.epoch = *calls & 0x7FFFFFFFu;
   a->scan.polls = g_scan_polls;
   a->scan.skip_tile = g_skip_tile;
@@ -786,13 +787,14 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
 }
 
 // ---- allocation-free compress -----------------------------------------------------------------
-// Scratch compiled into the device image: the counters (padded to 256 bytes) and the placement scan's
-// arrays for FH_STATIC_MAX_PLANES tiles (a tile is at least one plane).  The name is a device symbol: host
+// Scratch compiled into the device image: the counters (padded to 256 bytes), the placement scan's arrays
+// and the tile links for FH_STATIC_MAX_PLANES tiles (a tile is at least one plane).  The name is a device symbol: host
 // code must not pass it to a kernel, it asks the runtime for the symbol's device address instead (once per
 // device).
 static __device__ __align__(256) unsigned char g_static_scratch[FH_STATIC_SCRATCH_BYTES];
 static_assert(sizeof(fh::Scratch) <= fh::kScratchHeadBytes, "static scratch layout");
-static_assert(FH_STATIC_SCRATCH_BYTES == fh::kScratchHeadBytes + 8 * (FH_STATIC_MAX_PLANES + 2 * (FH_STATIC_MAX_PLANES / 32)),
+static_assert(FH_STATIC_SCRATCH_BYTES ==
+                  fh::kScratchHeadBytes + 8 * (FH_STATIC_MAX_PLANES + 2 * (FH_STATIC_MAX_PLANES / 32)) + 4 * FH_STATIC_MAX_PLANES,
               "static scratch layout");
 
 static std::mutex g_static_mu;

@@ -35,6 +35,7 @@ struct CompressArgs {
   unsigned long long* out2;             // optional: {total bytes, status}
   Scratch* sc;
   Scan scan;                            // placement of overflow parts (unused with salient_mode OFF)
+  uint32_t* defer_next;                 // one word per tile: links the tiles a CTA has put off (see BlockCtl)
   uint32_t parity;                      // which of the two ticket counters this call uses
   uint32_t early_ticket;                // 1: tiles may be requested before the previous kernel on the stream has completed
   // channel-wide three-sigma mode: per-channel outlier counts and per-plane counts from the statistics passes
@@ -365,6 +366,56 @@ __device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane,
   reinterpret_cast<uint4*>(d.dst + 64)[plane] = make_uint4(off16, meta, __float_as_uint(lo), __float_as_uint(scale));
 }
 
+// Table entry of a plane that takes the block-wise path, until its payload is written: class salient, the
+// three-sigma count, no offset.
+__device__ __forceinline__ void store_marker(const Dest& d, uint64_t plane, uint32_t meta) {
+  reinterpret_cast<uint4*>(d.dst + 64)[plane] = make_uint4(0u, (meta & ~3u) | kClsSalient, 0u, 0u);
+}
+
+// The block-wise path runs in two phases so that nothing in the streaming phase ever waits for another CTA.
+// Phase 1, while a tile lies in shared memory: its outlier-rich planes are measured, the tile publishes the
+// overflow size of its planes to the scan, and the CTA links the tile into its own list (newest first;
+// `defer_next[tile]` holds the tile listed before it).  Phase 2, when the CTA has run out of tiles: it takes
+// its listed tiles again (they come from the L2 cache when the tensor is small), obtains each tile's place
+// from the scan -- every tile before it has been published, or is about to be, by a CTA in phase 1 -- and
+// writes the payloads.  This block sits in shared memory: what the outlined functions of both phases need.
+constexpr uint32_t kNoTile = 0xFFFFFFFFu;
+struct BlockCtl {
+  Plan pl;
+  CompressArgs a;
+  Dest d;
+  uint32_t U[kMaxStages], C[kMaxStages], arr[kMaxStages];  // warp-team kernel, per stage: units, counts, warps done
+  uint32_t wu[kMaxWarps];                                  // phase 2: overflow units per warp
+  uint32_t base, ok;
+  uint32_t head;                                           // the tile this CTA listed last
+};
+
+// One thread: tile `tile` has `units` of overflow in `nsal` salient and `nraw` raw planes.
+__device__ __forceinline__ void publish_tile(BlockCtl* c, uint32_t tile, uint32_t units, uint32_t nsal, uint32_t nraw) {
+  scan_publish(c->a.scan, tile, units);
+  count_blockwise(c->a, units, nsal, nraw);
+  if ((nsal | nraw) && c->d.fits) c->a.defer_next[tile] = atomicExch(&c->head, tile);
+}
+
+// Copies planes [p0, p0 + np) into `buf` (whole 16-byte chunks from the aligned start, the ragged end of the
+// tensor byte-wise; all threads of the CTA) and returns the offset of plane p0 in it.
+__device__ __forceinline__ uint32_t stage_planes(const Plan& pl, const uint8_t* src, uint64_t p0, uint32_t np, uint8_t* buf) {
+  const uint64_t start = p0 * pl.plane_bytes, end = start + (uint64_t)np * pl.plane_bytes;
+  const uint64_t a0 = start & ~15ull;
+  const uint64_t a1 = min((end + 15ull) & ~15ull, pl.dense_bytes & ~15ull);
+  const uint4* s16 = reinterpret_cast<const uint4*>(src + a0);
+  uint4* t16 = reinterpret_cast<uint4*>(buf);
+  const uint32_t n16 = (uint32_t)((a1 - a0) >> 4);
+  for (uint32_t i = threadIdx.x; i < n16; i += blockDim.x) t16[i] = __ldg(s16 + i);
+  for (uint64_t i = a1 + threadIdx.x; i < end; i += blockDim.x) buf[i - a0] = src[i];
+  return (uint32_t)(start - a0);
+}
+
+// Class bits and three-sigma count a plane's table entry carries.
+__device__ __forceinline__ uint32_t table_meta(const Dest& d, uint64_t plane) {
+  return reinterpret_cast<const volatile uint32_t*>(d.dst + 64 + 16ull * plane)[1];
+}
+
 // Distances d = x - lo of group g of a plane; positions past HW read as 0.
 template <int DT>
 __device__ __forceinline__ void load_dist(const uint8_t* plane, uint32_t g, uint32_t HW, bool vec, float lo, float d[4]) {
@@ -387,20 +438,17 @@ struct Rec {
 // Tiles of consecutive planes are staged in shared memory with plain loads (planes need not start
 // on a 16-byte boundary); a team per plane computes statistics and class; the codes of normal planes
 // are staged in shared memory and leave with 16-byte stores.  Outlier-rich planes of the tile are then
-// taken one after the other by the whole CTA: measured, placed through the scan, measured again and
-// written (this kernel serves the odd shapes; the fast kernels below do not measure twice).
+// measured one after the other by the whole CTA, and written the same way in phase 2 (this kernel serves the
+// odd shapes and is not tuned).
 template <int DT, int BITS>
 __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
-  __shared__ uint32_t s_tile, s_last, s_base, s_ok;
-  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
+  __shared__ uint32_t s_tile, s_last;
+  __shared__ BlockCtl s_ctl;
 
   const uint32_t tid = threadIdx.x;
-  if (tid == 0) {
-    s_pl = pl;
-    if (a.early_ticket) s_tile = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
-  }
+  if (tid == 0 && a.early_ticket) s_tile = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
   dep_wait();     // the previous kernel on the stream has completed
   dep_trigger();  // the next kernel on the stream may become resident as this one drains
   uint8_t* tile_buf = smem + pl.sm_tile;
@@ -408,6 +456,12 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
   Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
   uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal);
   const Dest d = make_dest(pl, a);
+  if (tid == 0 && pl.mode != kModeOff) {
+    s_ctl.pl = pl;
+    s_ctl.a = a;
+    s_ctl.d = d;
+    s_ctl.head = kNoTile;
+  }
   const Team team = make_team(pl.team, s_red);
   const Team cta = make_team(kThreads, s_red);
   const uint32_t nteams = team.block ? 1u : kThreads / team.size;
@@ -425,18 +479,8 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     const uint64_t p0 = (uint64_t)tile * pl.ppt;
     const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
 
-    // ---- stage the tile: whole 16-byte chunks, then the ragged end of the tensor byte by byte
-    const uint64_t start = p0 * pl.plane_bytes, end = start + (uint64_t)np * pl.plane_bytes;
-    const uint64_t a0 = start & ~15ull;
-    const uint32_t head = (uint32_t)(start - a0);
-    const uint64_t a1 = min((end + 15ull) & ~15ull, pl.dense_bytes & ~15ull);
-    {
-      const uint4* s16 = reinterpret_cast<const uint4*>(a.src + a0);
-      uint4* t16 = reinterpret_cast<uint4*>(tile_buf);
-      const uint32_t n16 = (uint32_t)((a1 - a0) >> 4);
-      for (uint32_t i = tid; i < n16; i += kThreads) t16[i] = __ldg(s16 + i);
-      for (uint64_t i = a1 + tid; i < end; i += kThreads) tile_buf[i - a0] = a.src[i];
-    }
+    // ---- stage the tile
+    const uint32_t head = stage_planes(pl, a.src, p0, np, tile_buf);
     __syncthreads();
 
     // ---- phase A: per-plane statistics, class, codes
@@ -549,48 +593,68 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
                             rec[i].scale);
     }
 
-    // ---- phase C: the other planes, one after the other by the whole CTA
+    // ---- phase C: the other planes are measured, one after the other by the whole CTA; the tile publishes
+    // their overflow size and is put off until the CTA has run out of tiles
     if (pl.mode != kModeOff) {
       uint32_t U = 0, nsal = 0, nraw = 0;  // (every thread keeps the same figures)
       for (uint32_t lp = 0; lp < np; ++lp) {
         if ((rec[lp].meta & 3u) == kClsNormal) continue;
-        const SalientInfo info = salient_measure<DT>(cta, s_pl, tile_buf + head + (uint64_t)lp * pl.plane_bytes, sal);
+        if (tid == 0 && d.fits) store_marker(d, p0 + lp, rec[lp].meta);
+        const SalientInfo info = salient_measure<DT>(cta, s_ctl.pl, tile_buf + head + (uint64_t)lp * pl.plane_bytes, sal);
         bool raw;
-        const uint32_t u = plane_units(pl, info, raw);
-        if (tid == 0) rec[lp].units = u;
-        U += u;
+        U += plane_units(pl, info, raw);
         nsal += raw ? 0u : 1u;
         nraw += raw ? 1u : 0u;
         __syncthreads();  // the measuring scratch is reused
       }
-      if (tid < 32u) {
-        bool ok = true;
-        uint32_t base = 0;
-        if (tid == 0) {
-          scan_publish(a.scan, tile, U);
-          count_blockwise(a, U, nsal, nraw);
-        }
-        if (U) ok = scan_prefix(a.scan, tile, base);
-        if (tid == 0) {
-          if (!ok) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-          s_base = base;
-          s_ok = ok;
-        }
-      }
+      if (tid == 0) publish_tile(&s_ctl, tile, U, nsal, nraw);
+    }
+    __syncthreads();
+  }
+
+  // ---- phase 2: the tiles put off, newest first
+  __syncthreads();
+  for (uint32_t tile = pl.mode != kModeOff ? s_ctl.head : kNoTile; tile != kNoTile;) {
+    const uint32_t next = a.defer_next[tile];
+    const uint64_t p0 = (uint64_t)tile * pl.ppt;
+    const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+    const uint32_t head = stage_planes(pl, a.src, p0, np, tile_buf);
+    for (uint32_t i = tid; i < np; i += kThreads) rec[i].meta = table_meta(d, p0 + i);
+    __syncthreads();
+    uint32_t U = 0;
+    for (uint32_t lp = 0; lp < np; ++lp) {
+      if ((rec[lp].meta & 3u) == kClsNormal) continue;
+      const SalientInfo info = salient_measure<DT>(cta, s_ctl.pl, tile_buf + head + (uint64_t)lp * pl.plane_bytes, sal);
+      bool raw;
+      const uint32_t u = plane_units(pl, info, raw);
+      if (tid == 0) rec[lp].units = u;
+      U += u;
       __syncthreads();
-      if ((nsal | nraw) && s_ok) {
-        uint32_t at = s_base;
-        for (uint32_t lp = 0; lp < np; ++lp) {
-          if ((rec[lp].meta & 3u) == kClsNormal) continue;
-          const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
-          const SalientInfo info = salient_measure<DT>(cta, s_pl, plane, sal);
-          write_blockwise<DT>(cta, s_pl, d, p0 + lp, plane, info, sal, rec[lp].meta >> 2, at);
-          at += rec[lp].units;
-          __syncthreads();
-        }
+    }
+    if (tid < 32u) {
+      bool ok = true;
+      uint32_t base = 0;
+      if (U) ok = scan_prefix(a.scan, tile, base);
+      if (tid == 0) {
+        if (!ok) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+        s_ctl.base = base;
+        s_ctl.ok = ok;
       }
     }
     __syncthreads();
+    if (s_ctl.ok) {
+      uint32_t at = s_ctl.base;
+      for (uint32_t lp = 0; lp < np; ++lp) {
+        if ((rec[lp].meta & 3u) == kClsNormal) continue;
+        const uint8_t* plane = tile_buf + head + (uint64_t)lp * pl.plane_bytes;
+        const SalientInfo info = salient_measure<DT>(cta, s_ctl.pl, plane, sal);
+        write_blockwise<DT>(cta, s_ctl.pl, d, p0 + lp, plane, info, sal, rec[lp].meta >> 2, at);
+        at += rec[lp].units;
+        __syncthreads();
+      }
+    }
+    __syncthreads();
+    tile = next;
   }
   cta_exit(pl, a, d, &s_last);
 }
@@ -768,7 +832,11 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
   }
 
   const uint32_t meta = cls | (n_out << 2);
-  if (cls != kClsNormal || !d.fits) return meta;
+  if (!d.fits) return meta;
+  if (cls != kClsNormal) {
+    if (lane == 0) store_marker(d, gp, meta);
+    return meta;
+  }
   const uint32_t bits = (uint32_t)pl.bits;
   float inv, scale;
   quant_params(range, (1u << bits) - 1u, inv, scale);
@@ -801,11 +869,10 @@ __device__ __forceinline__ uint32_t plane_sweep_any(const Team& team, const Plan
 // -------------------------------------------------------------------------------------------------
 // Warp-team streaming kernel: planes of at most 256 groups.  Eight consumer warps and one producer
 // warp per CTA.  The producer requests tiles and streams them into a ring of shared-memory stages
-// with bulk copies.  A consumer warp sweeps its own planes of a tile (statistics, class, codes, stores).
-// Outlier-rich planes are rare: a warp that has some in its slice measures them, the tile's eight
-// warps add up their overflow sizes in shared memory, the last of them to get there publishes the
-// tile's total and obtains the tile's place from the scan, and the warps that need it wait for that one
-// word before they write.  Warps without such planes wait for nobody.
+// with bulk copies.  A consumer warp sweeps its own planes of a tile (statistics, class, codes, stores)
+// and never waits for another warp.  Outlier-rich planes are rare: a warp that has some in its slice
+// measures them and adds their overflow size to the tile's sum in shared memory; the last of the tile's
+// eight warps to get there publishes the tile and puts it on the CTA's list for phase 2.
 // -------------------------------------------------------------------------------------------------
 constexpr int kWarpKernelThreads = kThreads + 32;
 
@@ -820,9 +887,10 @@ struct WarpSal {
   SalientInfo last_info;
 };
 
+// `leaders`: the lanes (first lane of a team) whose plane is outlier-rich; lp0: first plane of the warp's slice.
 template <int DT, int TT>
-__device__ __noinline__ void warp_measure(const Plan& spl, const uint8_t* stage, uint32_t lp0, uint32_t leaders,
-                                          uint32_t* sal, WarpSal& ws) {
+__device__ __forceinline__ void warp_measure(const Plan& spl, const uint8_t* tbuf, uint32_t lp0, uint32_t leaders,
+                                             uint32_t* sal, WarpSal& ws) {
   const Team team = make_warp_team(nullptr);
   const uint32_t lane = team.lane;
   ws.units = 0;
@@ -831,7 +899,7 @@ __device__ __noinline__ void warp_measure(const Plan& spl, const uint8_t* stage,
   for (uint32_t m = leaders; m; m &= m - 1u, ++j) {
     const uint32_t lp = lp0 + ((uint32_t)__ffs((int)m) - 1u) / TT;
     if (j) __syncwarp();
-    const SalientInfo info = salient_measure<DT>(team, spl, stage + (uint64_t)lp * spl.plane_bytes, sal);
+    const SalientInfo info = salient_measure<DT>(team, spl, tbuf + (uint64_t)lp * spl.plane_bytes, sal);
     bool raw;
     const uint32_t u = plane_units(spl, info, raw);
     if (lane == j) {
@@ -852,23 +920,88 @@ __device__ __noinline__ void warp_measure(const Plan& spl, const uint8_t* stage,
   ws.nsal = j - ws.nraw;
 }
 
+// Phase 1, a warp with outlier-rich planes in its slice: their sizes go into the sums of the tile in stage s.
 template <int DT, int TT>
-__device__ __noinline__ void warp_write(const Plan& spl, const Dest d, const uint8_t* stage, uint64_t p0, uint32_t lp0,
-                                        uint32_t leaders, uint32_t meta, uint32_t* sal, const WarpSal& ws, uint32_t base) {
+__device__ __noinline__ void warp_tile_measure(BlockCtl* c, const uint8_t* tbuf, uint32_t s, uint32_t lp0,
+                                               uint32_t leaders, uint32_t* sal) {
+  WarpSal ws;
+  warp_measure<DT, TT>(c->pl, tbuf, lp0, leaders, sal, ws);
+  if ((threadIdx.x & 31u) == 0) {
+    if (ws.total) atomicAdd(&c->U[s], ws.total);
+    atomicAdd(&c->C[s], ws.nsal | (ws.nraw << 16));
+  }
+}
+
+// Phase 1, the last of a tile's eight warps (one thread): the tile's sums are complete.
+__device__ __noinline__ void warp_tile_publish(BlockCtl* c, uint32_t s, uint32_t tile) {
+  const uint32_t U = c->U[s], C = c->C[s];
+  c->U[s] = 0;
+  c->C[s] = 0;
+  publish_tile(c, tile, U, C & 0xFFFFu, C >> 16);
+}
+
+// Phase 2 of the warp-team kernel: every tile the CTA has put off, newest first, by all warps as in phase 1.
+template <int DT, int TT>
+__device__ __noinline__ void warp_phase2(BlockCtl* c, uint8_t* tbuf, uint8_t* sal_base) {
+  const Plan& pl = c->pl;
+  const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const Team team = make_warp_team(nullptr);
-  for (uint32_t j = (uint32_t)__popc(leaders); j-- > 0;) {  // the plane measured last comes first: its results are still there
-    const uint32_t src = __fns(leaders, 0u, (int)j + 1);
-    const uint32_t lp = lp0 + src / TT;
-    const uint8_t* plane = stage + (uint64_t)lp * spl.plane_bytes;
-    SalientInfo info = ws.last_info;
-    if (j != ws.last_j) {
-      __syncwarp();
-      info = salient_measure<DT>(team, spl, plane, sal);
+  const uint32_t lp0 = (warp * 32u) / TT;
+  uint32_t* sal = reinterpret_cast<uint32_t*>(sal_base + warp * pl.sal_stride);
+  for (uint32_t tile = c->head; tile != kNoTile;) {
+    const uint32_t next = c->a.defer_next[tile];
+    const uint32_t p0 = tile * pl.ppt;
+    const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+    stage_planes(pl, c->a.src, p0, np, tbuf);  // (tiles of this kernel start on 16-byte boundaries)
+    __syncthreads();
+    uint32_t meta = 0;
+    bool mine = false;
+    if (warp < (uint32_t)kWarps) {
+      const uint32_t lp = tid / TT;
+      if (lp < np && (tid % TT) == 0u) {
+        meta = table_meta(c->d, (uint64_t)p0 + lp);
+        mine = (meta & 3u) != kClsNormal;
+      }
     }
-    const uint32_t n_out = __shfl_sync(0xFFFFFFFFu, meta, (int)src) >> 2;
-    const uint32_t at = base + __shfl_sync(0xFFFFFFFFu, ws.excl, (int)j);
-    write_blockwise<DT>(team, spl, d, p0 + lp, plane, info, sal, n_out, at);
-    __syncwarp();
+    const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine);
+    WarpSal ws;
+    ws.total = ws.excl = ws.last_j = 0;
+    if (leaders) warp_measure<DT, TT>(pl, tbuf, lp0, leaders, sal, ws);
+    if (lane == 0 && warp < (uint32_t)kWarps) c->wu[warp] = ws.total;
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t U = lane < (uint32_t)kWarps ? c->wu[lane] : 0u;
+      asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(U) : "r"(0xFFFFFFFFu));
+      bool ok = true;
+      uint32_t base = 0;
+      if (U) ok = scan_prefix(c->a.scan, tile, base);
+      if (lane == 0) {
+        if (!ok) atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
+        c->base = base;
+        c->ok = ok;
+      }
+    }
+    __syncthreads();
+    if (leaders && c->ok) {
+      uint32_t base = c->base;
+      for (uint32_t w = 0; w < warp; ++w) base += c->wu[w];
+      for (uint32_t j = (uint32_t)__popc(leaders); j-- > 0;) {  // the plane measured last comes first: its results are still there
+        const uint32_t src = __fns(leaders, 0u, (int)j + 1);
+        const uint32_t lp = lp0 + src / TT;
+        const uint8_t* plane = tbuf + (uint64_t)lp * pl.plane_bytes;
+        SalientInfo info = ws.last_info;
+        if (j != ws.last_j) {
+          __syncwarp();
+          info = salient_measure<DT>(team, pl, plane, sal);
+        }
+        const uint32_t n_out = __shfl_sync(0xFFFFFFFFu, meta, (int)src) >> 2;
+        const uint32_t at = base + __shfl_sync(0xFFFFFFFFu, ws.excl, (int)j);
+        write_blockwise<DT>(team, pl, c->d, (uint64_t)p0 + lp, plane, info, sal, n_out, at);
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    tile = next;
   }
 }
 
@@ -880,10 +1013,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
   __shared__ uint32_t s_tiles[kMaxStages];
   __shared__ volatile uint32_t s_abort;
   __shared__ uint32_t s_last;
-  // placement of the outlier-rich planes of a tile (see above)
-  __shared__ uint32_t s_wu[kMaxStages][kWarps], s_wc[kMaxStages][kWarps], s_arr[kMaxStages], s_base[kMaxStages];
-  __shared__ volatile uint32_t s_ready[kMaxStages];
-  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
+  __shared__ BlockCtl s_ctl;
 
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const uint32_t nstage = pl.nstage;
@@ -893,22 +1023,28 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     for (uint32_t s = 0; s < nstage; ++s) {
       mbar_init(&s_full[s], 1);
       mbar_init(&s_empty[s], kWarps);
-      s_arr[s] = 0;
-      s_ready[s] = 0;
     }
     fence_mbar_init();
     s_abort = 0;
-    if (scan_on) s_pl = pl;
   }
   // (the ticket counter of this call was returned to zero by the call before the previous one, which had
   // completed before the previous kernel let this one start)
   if (tid == (uint32_t)kThreads && a.early_ticket)
     first_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
-  __syncthreads();
   dep_wait();     // the previous kernel on the stream has completed; global memory may be touched from here on
   dep_trigger();  // the next kernel on the stream may become resident as this one drains
   const Dest d = make_dest(pl, a);
-  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+  if (tid == 0) {
+    if (!d.fits && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+    if (scan_on) {
+      s_ctl.pl = pl;
+      s_ctl.a = a;
+      s_ctl.d = d;
+      s_ctl.head = kNoTile;
+      for (uint32_t s = 0; s < nstage; ++s) s_ctl.U[s] = s_ctl.C[s] = s_ctl.arr[s] = 0;
+    }
+  }
+  __syncthreads();
 
   if (warp == (uint32_t)kWarps) {
     // ======================= producer (all 32 lanes walk the loop, lane 0 issues) =======================
@@ -941,7 +1077,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
         uint32_t q = first % nstage;
         __syncwarp();
         if (lane == 0) {
-          s_tiles[s] = 0xFFFFFFFFu;
+          s_tiles[s] = kNoTile;
           mbar_arrive(&s_full[s]);
         }
         for (uint32_t m = first; m < n; ++m) {
@@ -986,10 +1122,9 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     // ======================= consumers =======================
     constexpr int G = 8;  // groups per thread: a plane has at most 8 * TT groups
     const Team team = make_team(TT, s_red);
-    const uint32_t my_team = tid / TT, lp0 = (warp * 32u) / TT;
+    const uint32_t my_team = tid / TT;
     const bool vec = (pl.plane_bytes & 15u) == 0u;
-    uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal + warp * pl.sal_stride);
-    uint32_t rp = 0, s = 0, phase = 0, seq = 0;
+    uint32_t rp = 0, s = 0, phase = 0;
     for (;;) {
       const uint32_t par = (phase >> s) & 1u;
       bool ok = mbar_wait_abortable(&s_full[s], par, 1u << 20, &s_abort);
@@ -1001,7 +1136,6 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       phase ^= 1u << s;
       const uint32_t tile = s_tiles[s];
       if (tile >= pl.ntiles) break;
-      ++seq;
       const uint32_t p0 = tile * pl.ppt;
       const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
       const uint32_t lp = my_team;
@@ -1011,55 +1145,14 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       if (active)
         meta = plane_sweep_any<DT, SIGMA, G, TT, FULLVEC>(team, pl, d, a, stage + (uint64_t)lp * pl.plane_bytes,
                                                           (uint64_t)p0 + lp, vec, rp);
-      if (scan_on) {
+      if (scan_on) {  // phase 1 of the block-wise path
         const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, active && (meta & 3u) != kClsNormal && team.lane == 0);
-        WarpSal ws;
-        ws.total = ws.nsal = ws.nraw = 0;
-        if (leaders) warp_measure<DT, TT>(s_pl, stage, lp0, leaders, sal, ws);
-        uint32_t old = 0;
+        if (leaders)
+          warp_tile_measure<DT, TT>(&s_ctl, stage, s, (warp * 32u) / TT, leaders,
+                                    reinterpret_cast<uint32_t*>(smem + pl.sm_sal + warp * pl.sal_stride));
         if (lane == 0) {
-          s_wu[s][warp] = ws.total;
-          s_wc[s][warp] = ws.nsal | (ws.nraw << 16);
           __threadfence_block();
-          old = atomicAdd(&s_arr[s], 1u);
-        }
-        old = __shfl_sync(0xFFFFFFFFu, old, 0);
-        if ((old & 7u) == 7u) {  // the last of the tile's eight warps: publish the tile, obtain its place
-          __threadfence_block();
-          uint32_t U = lane < (uint32_t)kWarps ? s_wu[s][lane] : 0u, C = lane < (uint32_t)kWarps ? s_wc[s][lane] : 0u;
-          asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(U) : "r"(0xFFFFFFFFu));
-          asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(C) : "r"(0xFFFFFFFFu));
-          if (lane == 0) {
-            scan_publish(a.scan, tile, U);
-            count_blockwise(a, U, C & 0xFFFFu, C >> 16);
-          }
-          if (U) {
-            uint32_t base = 0;
-            const bool got = scan_prefix(a.scan, tile, base);
-            if (lane == 0) {
-              if (!got) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-              s_base[s] = base;
-              __threadfence_block();
-              s_ready[s] = got ? seq : (seq | 0x80000000u);
-            }
-          }
-        }
-        if (leaders) {
-          uint32_t base = 0;
-          bool placed = true;
-          if (ws.total) {  // wait (bounded) for the tile's place
-            uint32_t v = 0;
-            for (uint32_t k = 0; k < a.scan.polls; ++k) {
-              v = s_ready[s];
-              if ((v & 0x7FFFFFFFu) == seq) break;
-              __nanosleep(64);
-            }
-            placed = v == seq;
-            __threadfence_block();
-            base = s_base[s];
-            for (uint32_t w = 0; w < warp; ++w) base += s_wu[s][w];
-          }
-          if (placed) warp_write<DT, TT>(s_pl, d, stage, (uint64_t)p0, lp0, leaders, meta, sal, ws, base);
+          if ((atomicAdd(&s_ctl.arr[s], 1u) & 7u) == 7u) warp_tile_publish(&s_ctl, s, tile);
         }
       }
       __syncwarp();
@@ -1067,6 +1160,10 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       if (s_abort) break;
       s = s + 1 == nstage ? 0 : s + 1;
     }
+  }
+  if (scan_on) {
+    __syncthreads();
+    if (s_ctl.head != kNoTile && !s_abort) warp_phase2<DT, TT>(&s_ctl, smem + pl.sm_tile, smem + pl.sm_sal);
   }
   cta_exit(pl, a, d, &s_last);
 }
@@ -1078,8 +1175,61 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
 // shared memory alone limits how many CTAs fit an SM (two stages each).  What every warp repeats per
 // plane -- reductions, thresholds, quantiser parameters -- does not shrink with the warp's share of the
 // plane, so NT is kept small for small planes.  Thread 0 keeps the next ticket in flight while the CTA works.
-// An outlier-rich plane is measured and written by the whole CTA while it lies in its stage.
+// An outlier-rich plane is measured by the whole CTA while it lies in its stage and written in phase 2.
 // -------------------------------------------------------------------------------------------------
+// Phase 1: the plane in `plane` is measured, tile (= plane) `tile` published and put on the CTA's list.
+template <int DT, int NT>
+__device__ __noinline__ void cta_tile_measure(BlockCtl* c, double* red, const uint8_t* plane, uint32_t* sal, uint32_t tile) {
+  const Team team = make_team(NT, red);
+  const SalientInfo info = salient_measure<DT>(team, c->pl, plane, sal);
+  bool raw;
+  const uint32_t units = plane_units(c->pl, info, raw);
+  if (threadIdx.x == 0) publish_tile(c, tile, units, raw ? 0u : 1u, raw ? 1u : 0u);
+}
+
+// Phase 2 of the CTA-team kernel: every plane the CTA has put off, newest first.
+template <int DT, int NT>
+__device__ __noinline__ void cta_phase2(BlockCtl* c, double* red, uint8_t* stage, uint32_t* sal, uint64_t* bar, uint32_t parity) {
+  const Plan& pl = c->pl;
+  const Team team = make_team(NT, red);
+  const uint32_t tid = threadIdx.x;
+  for (uint32_t tile = c->head; tile != kNoTile;) {
+    const uint32_t next = c->a.defer_next[tile];
+    if (tid == 0) {
+      fence_proxy_async();
+      mbar_expect_tx(bar, (uint32_t)pl.plane_bytes);
+      bulk_g2s(stage, c->a.src + (uint64_t)tile * pl.plane_bytes, (uint32_t)pl.plane_bytes, bar);
+    }
+    bool ready = mbar_wait(bar, parity, 1u << 20);
+    ready = __syncthreads_and(ready);
+    parity ^= 1u;
+    if (!ready) {  // the load timed out: report, wait (bounded) for the copy, give up
+      if (tid == 0) {
+        atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
+        mbar_wait(bar, parity ^ 1u, 1u << 10);
+      }
+      return;
+    }
+    const SalientInfo info = salient_measure<DT>(team, pl, stage, sal);
+    bool raw;
+    const uint32_t units = plane_units(pl, info, raw);
+    if (tid < 32u) {
+      bool ok = true;
+      uint32_t base = 0;
+      if (units) ok = scan_prefix(c->a.scan, tile, base);
+      if (tid == 0) {
+        if (!ok) atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
+        c->base = base;
+        c->ok = ok;
+      }
+    }
+    __syncthreads();
+    if (c->ok) write_blockwise<DT>(team, pl, c->d, (uint64_t)tile, stage, info, sal, table_meta(c->d, tile) >> 2, c->base);
+    __syncthreads();
+    tile = next;
+  }
+}
+
 template <int DT>
 __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, float (&v)[4]) {
   if (DT == kF32) {
@@ -1145,8 +1295,8 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
   __shared__ double s_red[kMaxWarps * 5];
   __shared__ __align__(8) uint64_t s_full[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
-  __shared__ uint32_t s_abort, s_last, s_base, s_ok;
-  __shared__ Plan s_pl;  // copy for the outlined measuring / writing functions, which take it by address
+  __shared__ uint32_t s_abort, s_last;
+  __shared__ BlockCtl s_ctl;
 
   const uint32_t tid = threadIdx.x;
   const Team team = make_team(NT, s_red);
@@ -1161,7 +1311,6 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
     fence_mbar_init();
     s_abort = 0;
-    if (scan_on) s_pl = pl;
     // (the ticket counter of this call was returned to zero by the call before the previous one, which had
     // completed before the previous kernel let this one start)
     if (a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
@@ -1183,6 +1332,12 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     }
   };
   if (tid == 0) {
+    if (scan_on) {
+      s_ctl.pl = pl;
+      s_ctl.a = a;
+      s_ctl.d = d;
+      s_ctl.head = kNoTile;
+    }
     if (!a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
     for (uint32_t s = 0; s < nstage; ++s) issue(s);
   }
@@ -1285,26 +1440,9 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
         if (scan_on) scan_publish(a.scan, tile, 0u);
         issue(s);  // the stage is free: next load
       }
-    } else {  // (the same for every thread) measured, placed and written while the plane lies in its stage
-      const SalientInfo info = salient_measure<DT>(team, s_pl, plane, sal);
-      bool raw;
-      const uint32_t my_units = plane_units(pl, info, raw);
-      if (tid < 32u) {
-        bool got = true;
-        uint32_t base = 0;
-        if (tid == 0) {
-          scan_publish(a.scan, tile, my_units);
-          count_blockwise(a, my_units, raw ? 0u : 1u, raw ? 1u : 0u);
-        }
-        if (my_units) got = scan_prefix(a.scan, tile, base);
-        if (tid == 0) {
-          if (!got) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
-          s_base = base;
-          s_ok = got;
-        }
-      }
-      __syncthreads();
-      if (s_ok) write_blockwise<DT>(team, s_pl, d, gp, plane, info, sal, n_out, s_base);
+    } else {  // (the same for every thread) phase 1 of the block-wise path
+      if (tid == 0 && d.fits) store_marker(d, gp, cls | (n_out << 2));
+      cta_tile_measure<DT, NT>(&s_ctl, s_red, plane, sal, tile);
       __syncthreads();  // every thread is done with the stage
       if (tid == 0) issue(s);
     }
@@ -1319,6 +1457,11 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
         mbar_wait(&s_full[k], 0u, 1u << 10);
         mbar_wait(&s_full[k], 1u, 1u << 10);
       }
+  }
+  if (scan_on) {
+    __syncthreads();
+    if (s_ctl.head != kNoTile && !s_abort)
+      cta_phase2<DT, NT>(&s_ctl, s_red, smem + pl.sm_tile, sal, &s_full[0], phase & 1u);
   }
   cta_exit(pl, a, d, &s_last);
 }
