@@ -259,6 +259,164 @@ __device__ __noinline__ void raw_write(const Team& t, const Plan& pl, const uint
     out.st16(o, o < n ? (uint32_t)*reinterpret_cast<const uint16_t*>(plane + o) : 0u);
 }
 
+// -------------------------------------------------------------------------------------------------
+// Small planes (at most kSmallBlocks blocks and fewer than 32 rows: 7x7, 8x8, 14x14, 16x16, ...) take the
+// block-wise path in the registers of one warp: no measuring scratch, no second look at the plane.  The
+// results are those of salient_measure / salient_write.
+// -------------------------------------------------------------------------------------------------
+constexpr uint32_t kSmallBlocks = 4;
+__device__ __forceinline__ bool is_small_plane(const Plan& pl) { return pl.nblk <= kSmallBlocks && pl.H < 32; }
+
+struct SmallBlocks {
+  uint32_t z0[kSmallBlocks], z1[kSmallBlocks];  // non-zero masks of the block's two halves (ballots)
+  uint32_t m0[kSmallBlocks], m1[kSmallBlocks];  // verbatim elements of a dense block (ballots)
+  uint32_t c0[kSmallBlocks], c1[kSmallBlocks];  // this lane's two residual codes
+  uint32_t w0[kSmallBlocks], w1[kSmallBlocks];  // this lane's two elements, verbatim bits
+  uint32_t dense;                               // bit b: block b is dense
+  uint32_t rowp;                                // lane y: CSR row pointer of row y; lane H: nnz_s
+  SalientInfo info;
+};
+// Non-zero bits of row rr (0..7) of a block.
+__device__ __forceinline__ uint32_t block_row_bits(uint32_t z0, uint32_t z1, uint32_t rr) {
+  return ((rr < 4u ? z0 : z1) >> ((rr & 3u) * 8u)) & 0xFFu;
+}
+
+template <int DT>
+__device__ __forceinline__ void small_blocks(const Plan& pl, const uint8_t* plane, SmallBlocks& sb) {
+  const uint32_t lane = threadIdx.x & 31u, full = 0xFFFFFFFFu;
+  const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
+  sb.dense = 0;
+  uint32_t n_dense = 0, n_out_d = 0;
+#pragma unroll
+  for (uint32_t b = 0; b < kSmallBlocks; ++b) {
+    sb.z0[b] = sb.z1[b] = sb.m0[b] = sb.m1[b] = 0;
+    sb.c0[b] = sb.c1[b] = 128u;
+    sb.w0[b] = sb.w1[b] = 0;
+    if (b < pl.nblk) {
+      const uint32_t by = b / pl.nbx, bx = b - by * pl.nbx;
+      const BlockRegs r = block_load<DT>(plane, pl.H, pl.W, (int)by, (int)bx, lane);
+      sb.w0[b] = DT == kF32 ? __float_as_uint(r.x0) : __float_as_uint(r.x0) >> 16;
+      sb.w1[b] = DT == kF32 ? __float_as_uint(r.x1) : __float_as_uint(r.x1) >> 16;
+      sb.z0[b] = __ballot_sync(full, r.x0 != 0.0f);
+      sb.z1[b] = __ballot_sync(full, r.x1 != 0.0f);
+      const uint32_t nnz = __popc(sb.z0[b]) + __popc(sb.z1[b]);
+      if ((uint64_t)nnz * pl.tau_den >= (uint64_t)pl.tau_num * 64u) {  // (the same for every lane)
+        sb.dense |= 1u << b;
+        ++n_dense;
+        block_codes(r, inv2e, lane, sb.c0[b], sb.c1[b], sb.m0[b], sb.m1[b]);
+        n_out_d += __popc(sb.m0[b]) + __popc(sb.m1[b]);
+      }
+    }
+  }
+  // CSR row pointers: lane y counts the non-zeros of row y that lie in sparse blocks
+  uint32_t cnt = 0;
+  {
+    const uint32_t by = lane >> 3, rr = lane & 7u;
+#pragma unroll
+    for (uint32_t b = 0; b < kSmallBlocks; ++b)
+      if (b < pl.nblk && !((sb.dense >> b) & 1u) && b / pl.nbx == by && lane < (uint32_t)pl.H)
+        cnt += __popc(block_row_bits(sb.z0[b], sb.z1[b], rr));
+  }
+  uint32_t incl = cnt;
+  for (uint32_t o = 1; o < 32u; o <<= 1) {
+    const uint32_t up = __shfl_up_sync(full, incl, o);
+    if (lane >= o) incl += up;
+  }
+  sb.rowp = incl - cnt;
+  const uint32_t nnz_s = __shfl_sync(full, incl, 31), e = (uint32_t)pl.esize;
+  sb.info.nnz_s = nnz_s;
+  sb.info.n_dense = n_dense;
+  sb.info.n_out_d = n_out_d;
+  sb.info.size = 16u + 4u * pl.nbm + 4u * ((uint32_t)pl.H + 1u) + a4(2u * nnz_s) + a4(e * nnz_s) + 64u * n_dense +
+                 a4(e * n_out_d);
+}
+
+template <int DT>
+__device__ __forceinline__ void small_write(const Plan& pl, const SmallBlocks& sb, const SplitOut& out) {
+  const uint32_t lane = threadIdx.x & 31u, full = 0xFFFFFFFFu, e = (uint32_t)pl.esize, H = (uint32_t)pl.H;
+  const SalientInfo& info = sb.info;
+  const uint32_t o_bm = 16u, o_rp = o_bm + 4u * pl.nbm, o_col = o_rp + 4u * (H + 1u);
+  const uint32_t o_val = o_col + a4(2u * info.nnz_s), o_codes = o_val + a4(e * info.nnz_s);
+  const uint32_t o_outl = o_codes + 64u * info.n_dense;
+  if (lane == 0) {
+    out.st32(0, info.nnz_s);
+    out.st32(4, info.n_dense);
+    out.st32(8, info.n_out_d);
+    out.st32(12, 0);
+    out.st32(o_bm, sb.dense);  // (at most kSmallBlocks blocks: one bitmap word)
+    // pads the section writers leave: col (2 bytes), val / verbatim values (bf16: 2 bytes)
+    if (info.nnz_s & 1u) out.st16(o_col + 2u * info.nnz_s, 0);
+    if (DT == kBF16 && (info.nnz_s & 1u)) out.st16(o_val + 2u * info.nnz_s, 0);
+    if (DT == kBF16 && (info.n_out_d & 1u)) out.st16(o_outl + 2u * info.n_out_d, 0);
+  }
+  // zero padding up to the end of the slot / of the 16-byte padded overflow part
+  const uint32_t end = max(pl.npay, a16(info.size));
+  for (uint32_t o = info.size + 4u * lane; o < end; o += 128u) out.st32(o, 0);
+  if (lane <= H) out.st32(o_rp + 4u * lane, sb.rowp);
+  const uint32_t lt = (1u << lane) - 1u, c = lane & 7u, r0 = lane >> 3;
+  uint32_t dense_rank = 0, outl_at = 0;
+#pragma unroll
+  for (uint32_t b = 0; b < kSmallBlocks; ++b) {
+    if (b >= pl.nblk) continue;
+    const uint32_t by = b / pl.nbx, bx = b - by * pl.nbx;
+    if ((sb.dense >> b) & 1u) {
+      const uint32_t oc = o_codes + 64u * dense_rank, oo = o_outl + e * outl_at;
+      if ((sb.m0[b] >> lane) & 1u) {
+        const uint32_t rank = __popc(sb.m0[b] & lt);
+        if (DT == kF32) out.st32(oo + 4u * rank, sb.w0[b]);
+        else out.st16(oo + 2u * rank, sb.w0[b]);
+      }
+      if ((sb.m1[b] >> lane) & 1u) {
+        const uint32_t rank = __popc(sb.m0[b]) + __popc(sb.m1[b] & lt);
+        if (DT == kF32) out.st32(oo + 4u * rank, sb.w1[b]);
+        else out.st16(oo + 2u * rank, sb.w1[b]);
+      }
+      uint32_t v0 = sb.c0[b] | (__shfl_down_sync(full, sb.c0[b], 1) << 8);
+      v0 |= __shfl_down_sync(full, v0, 2) << 16;
+      uint32_t v1 = sb.c1[b] | (__shfl_down_sync(full, sb.c1[b], 1) << 8);
+      v1 |= __shfl_down_sync(full, v1, 2) << 16;
+      if ((lane & 3u) == 0u) {
+        out.st32(oc + lane, v0);
+        out.st32(oc + 32u + lane, v1);
+      }
+      ++dense_rank;
+      outl_at += __popc(sb.m0[b]) + __popc(sb.m1[b]);
+    } else {
+      // CSR entries of the block's two halves: row pointer of the element's row, plus the non-zeros of that
+      // row in sparse blocks to the left, plus those before it in the block's row
+#pragma unroll
+      for (uint32_t half = 0; half < 2u; ++half) {
+        const uint32_t rr = r0 + 4u * half, y = by * 8u + rr;
+        uint32_t pos = __shfl_sync(full, sb.rowp, (int)(y & 31u));
+#pragma unroll
+        for (uint32_t bl = 0; bl < kSmallBlocks; ++bl)
+          if (bl < b && bl / pl.nbx == by && !((sb.dense >> bl) & 1u)) pos += __popc(block_row_bits(sb.z0[bl], sb.z1[bl], rr));
+        const uint32_t bits = block_row_bits(sb.z0[b], sb.z1[b], rr);
+        pos += __popc(bits & ((1u << c) - 1u));
+        if ((bits >> c) & 1u) {
+          out.st16(o_col + 2u * pos, bx * 8u + c);
+          const uint32_t w = half ? sb.w1[b] : sb.w0[b];
+          if (DT == kF32) out.st32(o_val + 4u * pos, w);
+          else out.st16(o_val + 2u * pos, w);
+        }
+      }
+    }
+  }
+}
+
+// A warp measures an outlier-rich plane that lies in shared memory: small planes in registers, others through
+// the measuring scratch `sal`.
+template <int DT>
+__device__ __forceinline__ SalientInfo warp_plane_measure(const Team& warp_team, const Plan& pl, const uint8_t* plane,
+                                                          uint32_t* sal) {
+  if (is_small_plane(pl)) {
+    SmallBlocks sb;
+    small_blocks<DT>(pl, plane, sb);
+    return sb.info;
+  }
+  return salient_measure<DT>(warp_team, pl, plane, sal);
+}
+
 // What every thread of a CTA knows about the destination.
 struct Dest {
   uint8_t* dst;
@@ -316,6 +474,33 @@ __device__ __forceinline__ void write_blockwise(const Team& t, const Plan& pl, c
         make_uint4(my_units ? (uint32_t)off16 : 0u, (raw ? kClsRaw : kClsSalient) | (n_out << 2), 0u, 0u);
 }
 
+// A warp measures the outlier-rich plane gp (in shared memory) and writes it with its overflow part `at` units
+// into the overflow region: small planes in registers, others through the measuring scratch `sal`.
+template <int DT>
+__device__ __forceinline__ void warp_plane_write(const Team& warp_team, const Plan& pl, const Dest& d, uint64_t gp,
+                                                 const uint8_t* plane, uint32_t* sal, uint32_t n_out, uint32_t at) {
+  if (!is_small_plane(pl)) {
+    const SalientInfo info = salient_measure<DT>(warp_team, pl, plane, sal);
+    write_blockwise<DT>(warp_team, pl, d, gp, plane, info, sal, n_out, at);
+    return;
+  }
+  SmallBlocks sb;
+  small_blocks<DT>(pl, plane, sb);
+  bool raw;
+  const uint32_t my_units = plane_units(pl, sb.info, raw);
+  const unsigned long long off16 = (pl.ovf_off >> 4) + at;
+  if (!d.fits || (off16 + my_units) * 16ull > d.capacity) return;  // never write past the capacity
+  SplitOut out;
+  out.slot = d.dst + pl.slots_off + gp * pl.npay;
+  out.ovf = d.dst + off16 * 16ull;
+  out.npay = pl.npay;
+  if (raw) raw_write(warp_team, pl, plane, out);
+  else small_write<DT>(pl, sb, out);
+  if (warp_team.lane == 0)
+    reinterpret_cast<uint4*>(d.dst + 64)[gp] =
+        make_uint4(my_units ? (uint32_t)off16 : 0u, (raw ? kClsRaw : kClsSalient) | (n_out << 2), 0u, 0u);
+}
+
 // One thread, after everything else of the call is done: header, result words, and every counter the
 // call touched back to zero.
 __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, const Dest& d) {
@@ -367,9 +552,13 @@ __device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane,
 }
 
 // Table entry of a plane that takes the block-wise path, until its payload is written: class salient, the
-// three-sigma count, no offset.
-__device__ __forceinline__ void store_marker(const Dest& d, uint64_t plane, uint32_t meta) {
-  reinterpret_cast<uint4*>(d.dst + 64)[plane] = make_uint4(0u, (meta & ~3u) | kClsSalient, 0u, 0u);
+// three-sigma count; phase 1 leaves the plane's overflow size (16-byte units) where the offset will go.
+__device__ __forceinline__ void store_marker(const Dest& d, uint64_t plane, uint32_t meta, uint32_t units) {
+  reinterpret_cast<uint4*>(d.dst + 64)[plane] = make_uint4(units, (meta & ~3u) | kClsSalient, 0u, 0u);
+}
+__device__ __forceinline__ uint2 load_marker(const Dest& d, uint64_t plane) {
+  const volatile uint32_t* e = reinterpret_cast<const volatile uint32_t*>(d.dst + 64 + 16ull * plane);
+  return make_uint2(e[0], e[1]);
 }
 
 // The block-wise path runs in two phases so that nothing in the streaming phase ever waits for another CTA.
@@ -385,9 +574,13 @@ struct BlockCtl {
   CompressArgs a;
   Dest d;
   uint32_t U[kMaxStages], C[kMaxStages], arr[kMaxStages];  // warp-team kernel, per stage: units, counts, warps done
-  uint32_t wu[kMaxWarps];                                  // phase 2: overflow units per warp
+  uint32_t wcnt[kMaxWarps];                                // phase 2: outlier-rich planes per warp's slice
   uint32_t base, ok;
   uint32_t head;                                           // the tile this CTA listed last
+  // phase 2 of the warp-team kernel: the outlier-rich planes of the tile in hand, in plane order
+  uint32_t list_at[256];                                   // overflow units, then (scanned) the place within the tile's part
+  uint32_t list_meta[256];
+  uint16_t list_lp[256];
 };
 
 // One thread: tile `tile` has `units` of overflow in `nsal` salient and `nraw` raw planes.
@@ -409,11 +602,6 @@ __device__ __forceinline__ uint32_t stage_planes(const Plan& pl, const uint8_t* 
   for (uint32_t i = threadIdx.x; i < n16; i += blockDim.x) t16[i] = __ldg(s16 + i);
   for (uint64_t i = a1 + threadIdx.x; i < end; i += blockDim.x) buf[i - a0] = src[i];
   return (uint32_t)(start - a0);
-}
-
-// Class bits and three-sigma count a plane's table entry carries.
-__device__ __forceinline__ uint32_t table_meta(const Dest& d, uint64_t plane) {
-  return reinterpret_cast<const volatile uint32_t*>(d.dst + 64 + 16ull * plane)[1];
 }
 
 // Distances d = x - lo of group g of a plane; positions past HW read as 0.
@@ -599,10 +787,11 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
       uint32_t U = 0, nsal = 0, nraw = 0;  // (every thread keeps the same figures)
       for (uint32_t lp = 0; lp < np; ++lp) {
         if ((rec[lp].meta & 3u) == kClsNormal) continue;
-        if (tid == 0 && d.fits) store_marker(d, p0 + lp, rec[lp].meta);
         const SalientInfo info = salient_measure<DT>(cta, s_ctl.pl, tile_buf + head + (uint64_t)lp * pl.plane_bytes, sal);
         bool raw;
-        U += plane_units(pl, info, raw);
+        const uint32_t u = plane_units(pl, info, raw);
+        if (tid == 0 && d.fits) store_marker(d, p0 + lp, rec[lp].meta, u);
+        U += u;
         nsal += raw ? 0u : 1u;
         nraw += raw ? 1u : 0u;
         __syncthreads();  // the measuring scratch is reused
@@ -619,18 +808,14 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     const uint64_t p0 = (uint64_t)tile * pl.ppt;
     const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
     const uint32_t head = stage_planes(pl, a.src, p0, np, tile_buf);
-    for (uint32_t i = tid; i < np; i += kThreads) rec[i].meta = table_meta(d, p0 + i);
-    __syncthreads();
     uint32_t U = 0;
-    for (uint32_t lp = 0; lp < np; ++lp) {
-      if ((rec[lp].meta & 3u) == kClsNormal) continue;
-      const SalientInfo info = salient_measure<DT>(cta, s_ctl.pl, tile_buf + head + (uint64_t)lp * pl.plane_bytes, sal);
-      bool raw;
-      const uint32_t u = plane_units(pl, info, raw);
-      if (tid == 0) rec[lp].units = u;
-      U += u;
-      __syncthreads();
+    for (uint32_t i = tid; i < np; i += kThreads) {
+      const uint2 m = load_marker(d, p0 + i);
+      rec[i].meta = m.y;
+      rec[i].units = (m.y & 3u) != kClsNormal ? m.x : 0u;
+      U += rec[i].units;
     }
+    U = __syncthreads_or(U);  // (only whether the tile has any overflow matters here)
     if (tid < 32u) {
       bool ok = true;
       uint32_t base = 0;
@@ -832,11 +1017,7 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
   }
 
   const uint32_t meta = cls | (n_out << 2);
-  if (!d.fits) return meta;
-  if (cls != kClsNormal) {
-    if (lane == 0) store_marker(d, gp, meta);
-    return meta;
-  }
+  if (cls != kClsNormal || !d.fits) return meta;  // (the caller sees to a plane that is not normal)
   const uint32_t bits = (uint32_t)pl.bits;
   float inv, scale;
   quant_params(range, (1u << bits) - 1u, inv, scale);
@@ -876,59 +1057,29 @@ __device__ __forceinline__ uint32_t plane_sweep_any(const Team& team, const Plan
 // -------------------------------------------------------------------------------------------------
 constexpr int kWarpKernelThreads = kThreads + 32;
 
-// What a warp knows about the outlier-rich planes of its slice after measuring them.
-struct WarpSal {
-  uint32_t units;      // lane j: overflow units of the slice's j-th such plane ...
-  uint32_t excl;       // ... and of those before it
-  uint32_t raw;        // ... 1: stored raw
-  uint32_t total;      // of the slice
-  uint32_t nsal, nraw;
-  uint32_t last_j;     // the plane whose measuring results still lie in the warp's area
-  SalientInfo last_info;
-};
-
-// `leaders`: the lanes (first lane of a team) whose plane is outlier-rich; lp0: first plane of the warp's slice.
+// Phase 1, a warp with outlier-rich planes in its slice (`leaders`: the first lanes of their teams; lp0: first
+// plane of the warp's slice): they are measured, their sizes go into the sums of the tile in stage s and into
+// their table markers.
 template <int DT, int TT>
-__device__ __forceinline__ void warp_measure(const Plan& spl, const uint8_t* tbuf, uint32_t lp0, uint32_t leaders,
-                                             uint32_t* sal, WarpSal& ws) {
+__device__ __noinline__ void warp_tile_measure(BlockCtl* c, const uint8_t* tbuf, uint64_t p0, uint32_t s, uint32_t lp0,
+                                               uint32_t leaders, uint32_t meta, uint32_t* sal) {
   const Team team = make_warp_team(nullptr);
-  const uint32_t lane = team.lane;
-  ws.units = 0;
-  ws.raw = 0;
-  uint32_t j = 0;
-  for (uint32_t m = leaders; m; m &= m - 1u, ++j) {
-    const uint32_t lp = lp0 + ((uint32_t)__ffs((int)m) - 1u) / TT;
-    if (j) __syncwarp();
-    const SalientInfo info = salient_measure<DT>(team, spl, tbuf + (uint64_t)lp * spl.plane_bytes, sal);
+  const Plan& pl = c->pl;
+  uint32_t total = 0, nraw = 0, n = 0;
+  for (uint32_t m = leaders; m; m &= m - 1u, ++n) {
+    const uint32_t src = (uint32_t)__ffs((int)m) - 1u, lp = lp0 + src / TT;
+    if (n) __syncwarp();
+    const SalientInfo info = warp_plane_measure<DT>(team, pl, tbuf + (uint64_t)lp * pl.plane_bytes, sal);
     bool raw;
-    const uint32_t u = plane_units(spl, info, raw);
-    if (lane == j) {
-      ws.units = u;
-      ws.raw = raw;
-    }
-    ws.last_info = info;
-    ws.last_j = j;
+    const uint32_t u = plane_units(pl, info, raw);
+    total += u;
+    nraw += raw ? 1u : 0u;
+    const uint32_t mt = __shfl_sync(0xFFFFFFFFu, meta, (int)src);
+    if (team.lane == 0 && c->d.fits) store_marker(c->d, p0 + lp, mt, u);
   }
-  uint32_t incl = ws.units;
-  for (uint32_t o = 1; o < 32u; o <<= 1) {
-    const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-    if (lane >= o) incl += up;
-  }
-  ws.excl = incl - ws.units;
-  ws.total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-  ws.nraw = __popc(__ballot_sync(0xFFFFFFFFu, ws.raw != 0u));
-  ws.nsal = j - ws.nraw;
-}
-
-// Phase 1, a warp with outlier-rich planes in its slice: their sizes go into the sums of the tile in stage s.
-template <int DT, int TT>
-__device__ __noinline__ void warp_tile_measure(BlockCtl* c, const uint8_t* tbuf, uint32_t s, uint32_t lp0,
-                                               uint32_t leaders, uint32_t* sal) {
-  WarpSal ws;
-  warp_measure<DT, TT>(c->pl, tbuf, lp0, leaders, sal, ws);
-  if ((threadIdx.x & 31u) == 0) {
-    if (ws.total) atomicAdd(&c->U[s], ws.total);
-    atomicAdd(&c->C[s], ws.nsal | (ws.nraw << 16));
+  if (team.lane == 0) {
+    if (total) atomicAdd(&c->U[s], total);
+    atomicAdd(&c->C[s], (n - nraw) | (nraw << 16));
   }
 }
 
@@ -940,41 +1091,57 @@ __device__ __noinline__ void warp_tile_publish(BlockCtl* c, uint32_t s, uint32_t
   publish_tile(c, tile, U, C & 0xFFFFu, C >> 16);
 }
 
-// Phase 2 of the warp-team kernel: every tile the CTA has put off, newest first, by all warps as in phase 1.
+// Phase 2 of the warp-team kernel: every tile the CTA has put off, newest first.  The tile's outlier-rich
+// planes are listed in plane order (their markers carry class, count and size), placed by one scan over
+// the list, and dealt out to the warps in turn.
 template <int DT, int TT>
 __device__ __noinline__ void warp_phase2(BlockCtl* c, uint8_t* tbuf, uint8_t* sal_base) {
   const Plan& pl = c->pl;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const Team team = make_warp_team(nullptr);
-  const uint32_t lp0 = (warp * 32u) / TT;
-  uint32_t* sal = reinterpret_cast<uint32_t*>(sal_base + warp * pl.sal_stride);
+  uint32_t* sal = reinterpret_cast<uint32_t*>(sal_base + min(warp, (uint32_t)kWarps - 1u) * pl.sal_stride);
   for (uint32_t tile = c->head; tile != kNoTile;) {
     const uint32_t next = c->a.defer_next[tile];
     const uint32_t p0 = tile * pl.ppt;
     const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
     stage_planes(pl, c->a.src, p0, np, tbuf);  // (tiles of this kernel start on 16-byte boundaries)
-    __syncthreads();
-    uint32_t meta = 0;
+    uint2 mk = make_uint2(0u, 0u);
     bool mine = false;
-    if (warp < (uint32_t)kWarps) {
-      const uint32_t lp = tid / TT;
-      if (lp < np && (tid % TT) == 0u) {
-        meta = table_meta(c->d, (uint64_t)p0 + lp);
-        mine = (meta & 3u) != kClsNormal;
-      }
+    const uint32_t lp = tid / TT;
+    if (warp < (uint32_t)kWarps && lp < np && (tid % TT) == 0u) {
+      mk = load_marker(c->d, (uint64_t)p0 + lp);
+      mine = (mk.y & 3u) != kClsNormal;
     }
     const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine);
-    WarpSal ws;
-    ws.total = ws.excl = ws.last_j = 0;
-    if (leaders) warp_measure<DT, TT>(pl, tbuf, lp0, leaders, sal, ws);
-    if (lane == 0 && warp < (uint32_t)kWarps) c->wu[warp] = ws.total;
+    if (lane == 0 && warp < (uint32_t)kWarps) c->wcnt[warp] = __popc(leaders);
     __syncthreads();
-    if (warp == 0) {
-      uint32_t U = lane < (uint32_t)kWarps ? c->wu[lane] : 0u;
-      asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(U) : "r"(0xFFFFFFFFu));
+    uint32_t before = 0, total = 0;
+    for (uint32_t w = 0; w < (uint32_t)kWarps; ++w) {
+      before += w < warp ? c->wcnt[w] : 0u;
+      total += c->wcnt[w];
+    }
+    if (mine) {
+      const uint32_t r = before + __popc(leaders & ((1u << lane) - 1u));
+      c->list_at[r] = mk.x;
+      c->list_meta[r] = mk.y;
+      c->list_lp[r] = (uint16_t)lp;
+    }
+    __syncthreads();
+    if (warp == 0) {  // places within the tile's part of the overflow region, and the tile's place
+      uint32_t run = 0;
+      for (uint32_t r0 = 0; r0 < total; r0 += 32u) {
+        const uint32_t v = r0 + lane < total ? c->list_at[r0 + lane] : 0u;
+        uint32_t incl = v;
+        for (uint32_t o = 1; o < 32u; o <<= 1) {
+          const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= o) incl += up;
+        }
+        if (r0 + lane < total) c->list_at[r0 + lane] = run + incl - v;
+        run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+      }
       bool ok = true;
       uint32_t base = 0;
-      if (U) ok = scan_prefix(c->a.scan, tile, base);
+      if (run) ok = scan_prefix(c->a.scan, tile, base);
       if (lane == 0) {
         if (!ok) atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
         c->base = base;
@@ -982,24 +1149,13 @@ __device__ __noinline__ void warp_phase2(BlockCtl* c, uint8_t* tbuf, uint8_t* sa
       }
     }
     __syncthreads();
-    if (leaders && c->ok) {
-      uint32_t base = c->base;
-      for (uint32_t w = 0; w < warp; ++w) base += c->wu[w];
-      for (uint32_t j = (uint32_t)__popc(leaders); j-- > 0;) {  // the plane measured last comes first: its results are still there
-        const uint32_t src = __fns(leaders, 0u, (int)j + 1);
-        const uint32_t lp = lp0 + src / TT;
-        const uint8_t* plane = tbuf + (uint64_t)lp * pl.plane_bytes;
-        SalientInfo info = ws.last_info;
-        if (j != ws.last_j) {
-          __syncwarp();
-          info = salient_measure<DT>(team, pl, plane, sal);
-        }
-        const uint32_t n_out = __shfl_sync(0xFFFFFFFFu, meta, (int)src) >> 2;
-        const uint32_t at = base + __shfl_sync(0xFFFFFFFFu, ws.excl, (int)j);
-        write_blockwise<DT>(team, pl, c->d, (uint64_t)p0 + lp, plane, info, sal, n_out, at);
+    if (c->ok && warp < (uint32_t)kWarps)
+      for (uint32_t r = warp; r < total; r += (uint32_t)kWarps) {
+        const uint32_t pl_lp = c->list_lp[r];
+        warp_plane_write<DT>(team, pl, c->d, (uint64_t)p0 + pl_lp, tbuf + (uint64_t)pl_lp * pl.plane_bytes, sal,
+                             c->list_meta[r] >> 2, c->base + c->list_at[r]);
         __syncwarp();
       }
-    }
     __syncthreads();
     tile = next;
   }
@@ -1148,7 +1304,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       if (scan_on) {  // phase 1 of the block-wise path
         const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, active && (meta & 3u) != kClsNormal && team.lane == 0);
         if (leaders)
-          warp_tile_measure<DT, TT>(&s_ctl, stage, s, (warp * 32u) / TT, leaders,
+          warp_tile_measure<DT, TT>(&s_ctl, stage, (uint64_t)p0, s, (warp * 32u) / TT, leaders, meta,
                                     reinterpret_cast<uint32_t*>(smem + pl.sm_sal + warp * pl.sal_stride));
         if (lane == 0) {
           __threadfence_block();
@@ -1179,12 +1335,16 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
 // -------------------------------------------------------------------------------------------------
 // Phase 1: the plane in `plane` is measured, tile (= plane) `tile` published and put on the CTA's list.
 template <int DT, int NT>
-__device__ __noinline__ void cta_tile_measure(BlockCtl* c, double* red, const uint8_t* plane, uint32_t* sal, uint32_t tile) {
+__device__ __noinline__ void cta_tile_measure(BlockCtl* c, double* red, const uint8_t* plane, uint32_t* sal, uint32_t tile,
+                                              uint32_t meta) {
   const Team team = make_team(NT, red);
   const SalientInfo info = salient_measure<DT>(team, c->pl, plane, sal);
   bool raw;
   const uint32_t units = plane_units(c->pl, info, raw);
-  if (threadIdx.x == 0) publish_tile(c, tile, units, raw ? 0u : 1u, raw ? 1u : 0u);
+  if (threadIdx.x == 0) {
+    if (c->d.fits) store_marker(c->d, tile, meta, units);
+    publish_tile(c, tile, units, raw ? 0u : 1u, raw ? 1u : 0u);
+  }
 }
 
 // Phase 2 of the CTA-team kernel: every plane the CTA has put off, newest first.
@@ -1224,7 +1384,7 @@ __device__ __noinline__ void cta_phase2(BlockCtl* c, double* red, uint8_t* stage
       }
     }
     __syncthreads();
-    if (c->ok) write_blockwise<DT>(team, pl, c->d, (uint64_t)tile, stage, info, sal, table_meta(c->d, tile) >> 2, c->base);
+    if (c->ok) write_blockwise<DT>(team, pl, c->d, (uint64_t)tile, stage, info, sal, load_marker(c->d, tile).y >> 2, c->base);
     __syncthreads();
     tile = next;
   }
@@ -1441,8 +1601,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
         issue(s);  // the stage is free: next load
       }
     } else {  // (the same for every thread) phase 1 of the block-wise path
-      if (tid == 0 && d.fits) store_marker(d, gp, cls | (n_out << 2));
-      cta_tile_measure<DT, NT>(&s_ctl, s_red, plane, sal, tile);
+      cta_tile_measure<DT, NT>(&s_ctl, s_red, plane, sal, tile, cls | (n_out << 2));
       __syncthreads();  // every thread is done with the stage
       if (tid == 0) issue(s);
     }
