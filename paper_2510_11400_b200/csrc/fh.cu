@@ -368,6 +368,15 @@ int launch_on(K kernel, const Plan& pl, cudaStream_t stream, int* grid) {
 
 // Launch that may overlap the tail of the previous kernel on the stream: every kernel of this library
 // passes dep_wait() before it touches global memory, so stream order is kept.
+// Tiles a CTA requests at once when it starts: all its stages when every CTA of the grid gets that many, fewer
+// when the tensor is small, so that the tiles spread over all CTAs before any CTA takes a second one.
+Plan with_first_request(const Plan& pl, int grid, uint32_t least) {
+  Plan q = pl;
+  const uint32_t each = pl.ntiles / (uint32_t)(grid > 0 ? grid : 1);
+  q.nstage = each < least ? least : (each > pl.nstage ? pl.nstage : each);
+  return q;
+}
+
 template <typename K, typename A>
 cudaError_t launch_dependent(K kernel, int grid, int threads, size_t smem, cudaStream_t stream, const Plan& pl,
                              const A& a) {
@@ -398,7 +407,7 @@ int launch_cta_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream)
   int grid = 0;
   int rc = grid_for(fh::compress_cta<DT, SIGMA, NT>, pl.sm_total, pl.ntiles, &grid, NT);
   if (rc != FH_OK) return rc;
-  return launch_dependent(fh::compress_cta<DT, SIGMA, NT>, grid, NT, pl.sm_total, stream, pl, a) == cudaSuccess
+  return launch_dependent(fh::compress_cta<DT, SIGMA, NT>, grid, NT, pl.sm_total, stream, with_first_request(pl, grid, 2), a) == cudaSuccess
              ? FH_OK : FH_ERR_CUDA;
 }
 
@@ -408,7 +417,7 @@ int launch_warp_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream
   int rc = grid_for(fh::compress_warp<DT, SIGMA, TT, FULLVEC>, pl.sm_total, pl.ntiles, &grid, fh::kWarpKernelThreads);
   if (rc != FH_OK) return rc;
   return launch_dependent(fh::compress_warp<DT, SIGMA, TT, FULLVEC>, grid, fh::kWarpKernelThreads, pl.sm_total, stream,
-                          pl, a) == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+                          with_first_request(pl, grid, 1), a) == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
 template <int DT, bool SIGMA, bool FULLVEC>

@@ -577,6 +577,7 @@ struct BlockCtl {
   uint32_t wcnt[kMaxWarps];                                // phase 2: outlier-rich planes per warp's slice
   uint32_t base, ok;
   uint32_t head;                                           // the tile this CTA listed last
+  uint32_t held[kMaxStages];                               // warp-team kernel: the tile each stage buffer holds
   // phase 2 of the warp-team kernel: the outlier-rich planes of the tile in hand, in plane order
   uint32_t list_at[256];                                   // overflow units, then (scanned) the place within the tile's part
   uint32_t list_meta[256];
@@ -1095,69 +1096,81 @@ __device__ __noinline__ void warp_tile_publish(BlockCtl* c, uint32_t s, uint32_t
 // planes are listed in plane order (their markers carry class, count and size), placed by one scan over
 // the list, and dealt out to the warps in turn.
 template <int DT, int TT>
-__device__ __noinline__ void warp_phase2(BlockCtl* c, uint8_t* tbuf, uint8_t* sal_base) {
+__device__ __noinline__ void warp_phase2(BlockCtl* c, uint8_t* stages, uint8_t* sal_base) {
   const Plan& pl = c->pl;
   const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
   const Team team = make_warp_team(nullptr);
   uint32_t* sal = reinterpret_cast<uint32_t*>(sal_base + min(warp, (uint32_t)kWarps - 1u) * pl.sal_stride);
-  for (uint32_t tile = c->head; tile != kNoTile;) {
-    const uint32_t next = c->a.defer_next[tile];
-    const uint32_t p0 = tile * pl.ppt;
-    const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
-    stage_planes(pl, c->a.src, p0, np, tbuf);  // (tiles of this kernel start on 16-byte boundaries)
-    uint2 mk = make_uint2(0u, 0u);
-    bool mine = false;
-    const uint32_t lp = tid / TT;
-    if (warp < (uint32_t)kWarps && lp < np && (tid % TT) == 0u) {
-      mk = load_marker(c->d, (uint64_t)p0 + lp);
-      mine = (mk.y & 3u) != kClsNormal;
-    }
-    const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine);
-    if (lane == 0 && warp < (uint32_t)kWarps) c->wcnt[warp] = __popc(leaders);
-    __syncthreads();
-    uint32_t before = 0, total = 0;
-    for (uint32_t w = 0; w < (uint32_t)kWarps; ++w) {
-      before += w < warp ? c->wcnt[w] : 0u;
-      total += c->wcnt[w];
-    }
-    if (mine) {
-      const uint32_t r = before + __popc(leaders & ((1u << lane) - 1u));
-      c->list_at[r] = mk.x;
-      c->list_meta[r] = mk.y;
-      c->list_lp[r] = (uint16_t)lp;
-    }
-    __syncthreads();
-    if (warp == 0) {  // places within the tile's part of the overflow region, and the tile's place
-      uint32_t run = 0;
-      for (uint32_t r0 = 0; r0 < total; r0 += 32u) {
-        const uint32_t v = r0 + lane < total ? c->list_at[r0 + lane] : 0u;
-        uint32_t incl = v;
-        for (uint32_t o = 1; o < 32u; o <<= 1) {
-          const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-          if (lane >= o) incl += up;
+  // Two walks over the list: first the tiles that still lie in a stage buffer (the last ones the CTA streamed:
+  // all of them when the tensor is small), then the others, fetched again into the first buffer.
+  for (uint32_t walk = 0; walk < 2u; ++walk) {
+    for (uint32_t tile = c->head; tile != kNoTile;) {
+      const uint32_t next = c->a.defer_next[tile];
+      uint32_t at_stage = kMaxStages;
+      for (uint32_t s = 0; s < pl.nstage; ++s)
+        if (c->held[s] == tile) at_stage = s;
+      if ((at_stage < (uint32_t)kMaxStages) != (walk == 0u)) {  // (the same for every thread)
+        tile = next;
+        continue;
+      }
+      const uint32_t p0 = tile * pl.ppt;
+      const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+      uint8_t* tbuf = stages + (uint64_t)(walk == 0u ? at_stage : 0u) * pl.stage_bytes;
+      if (walk) stage_planes(pl, c->a.src, p0, np, tbuf);  // (tiles of this kernel start on 16-byte boundaries)
+      uint2 mk = make_uint2(0u, 0u);
+      bool mine = false;
+      const uint32_t lp = tid / TT;
+      if (warp < (uint32_t)kWarps && lp < np && (tid % TT) == 0u) {
+        mk = load_marker(c->d, (uint64_t)p0 + lp);
+        mine = (mk.y & 3u) != kClsNormal;
+      }
+      const uint32_t leaders = __ballot_sync(0xFFFFFFFFu, mine);
+      if (lane == 0 && warp < (uint32_t)kWarps) c->wcnt[warp] = __popc(leaders);
+      __syncthreads();
+      uint32_t before = 0, total = 0;
+      for (uint32_t w = 0; w < (uint32_t)kWarps; ++w) {
+        before += w < warp ? c->wcnt[w] : 0u;
+        total += c->wcnt[w];
+      }
+      if (mine) {
+        const uint32_t r = before + __popc(leaders & ((1u << lane) - 1u));
+        c->list_at[r] = mk.x;
+        c->list_meta[r] = mk.y;
+        c->list_lp[r] = (uint16_t)lp;
+      }
+      __syncthreads();
+      if (warp == 0) {  // places within the tile's part of the overflow region, and the tile's place
+        uint32_t run = 0;
+        for (uint32_t r0 = 0; r0 < total; r0 += 32u) {
+          const uint32_t v = r0 + lane < total ? c->list_at[r0 + lane] : 0u;
+          uint32_t incl = v;
+          for (uint32_t o = 1; o < 32u; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += up;
+          }
+          if (r0 + lane < total) c->list_at[r0 + lane] = run + incl - v;
+          run += __shfl_sync(0xFFFFFFFFu, incl, 31);
         }
-        if (r0 + lane < total) c->list_at[r0 + lane] = run + incl - v;
-        run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        bool ok = true;
+        uint32_t base = 0;
+        if (run) ok = scan_prefix(c->a.scan, tile, base);
+        if (lane == 0) {
+          if (!ok) atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
+          c->base = base;
+          c->ok = ok;
+        }
       }
-      bool ok = true;
-      uint32_t base = 0;
-      if (run) ok = scan_prefix(c->a.scan, tile, base);
-      if (lane == 0) {
-        if (!ok) atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
-        c->base = base;
-        c->ok = ok;
-      }
+      __syncthreads();
+      if (c->ok && warp < (uint32_t)kWarps)
+        for (uint32_t r = warp; r < total; r += (uint32_t)kWarps) {
+          const uint32_t pl_lp = c->list_lp[r];
+          warp_plane_write<DT>(team, pl, c->d, (uint64_t)p0 + pl_lp, tbuf + (uint64_t)pl_lp * pl.plane_bytes, sal,
+                               c->list_meta[r] >> 2, c->base + c->list_at[r]);
+          __syncwarp();
+        }
+      __syncthreads();
+      tile = next;
     }
-    __syncthreads();
-    if (c->ok && warp < (uint32_t)kWarps)
-      for (uint32_t r = warp; r < total; r += (uint32_t)kWarps) {
-        const uint32_t pl_lp = c->list_lp[r];
-        warp_plane_write<DT>(team, pl, c->d, (uint64_t)p0 + pl_lp, tbuf + (uint64_t)pl_lp * pl.plane_bytes, sal,
-                             c->list_meta[r] >> 2, c->base + c->list_at[r]);
-        __syncwarp();
-      }
-    __syncthreads();
-    tile = next;
   }
 }
 
@@ -1197,7 +1210,10 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       s_ctl.a = a;
       s_ctl.d = d;
       s_ctl.head = kNoTile;
-      for (uint32_t s = 0; s < nstage; ++s) s_ctl.U[s] = s_ctl.C[s] = s_ctl.arr[s] = 0;
+      for (uint32_t s = 0; s < nstage; ++s) {
+        s_ctl.U[s] = s_ctl.C[s] = s_ctl.arr[s] = 0;
+        s_ctl.held[s] = kNoTile;
+      }
     }
   }
   __syncthreads();
@@ -1247,6 +1263,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       }
       if (lane == 0) {
         s_tiles[s] = t;
+        if (scan_on) s_ctl.held[s] = t;
         const uint32_t p0 = t * pl.ppt;
         const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
         const uint32_t bytes = np * (uint32_t)pl.plane_bytes;
