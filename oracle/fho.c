@@ -153,7 +153,8 @@ size_t fho_compressed_bytes(const fho_desc* d, const fho_params* p, int which) {
  *       counted -- inside [-40, 60] neither d*d nor the scalings below can overflow or underflow.
  *   d_i = x_i - lo (fp32, >= 0); elements are taken in consecutive groups of 4 per plane, the last
  *       group of a plane padded with d = 0; per group, in fp32:
- *     s_g = (d0 + d1) + (d2 + d3),   q_g = fma(d1, d1, d0*d0) + fma(d3, d3, d2*d2)
+ *     s_g = (d0 + d2) + (d1 + d3),   q_g = fma(d2, d2, d0*d0) + fma(d3, d3, d1*d1)
+ *       (elements 0,1 and 2,3 of a group are treated as two pairs that are combined position by position)
  *     i_s = round_half_even(s_g * 2^(18-e)),  i_q = round_half_even(q_g * 2^(16-2e))   (exact products,
  *       integers below 2^22: the sums resolve 2^-18 of the range and 2^-16 of its square per group)
  *   I_s = sum i_s, I_q = sum i_q                                          (exact integers, any order)
@@ -194,11 +195,11 @@ static void sigma_sums(const float* x, int64_t n_planes, int64_t stride, int64_t
     for (int64_t g = 0; g < hw; g += 4) {
       float d[4] = {0.f, 0.f, 0.f, 0.f};
       for (int k = 0; k < 4 && g + k < hw; ++k) d[k] = x[n * stride + g + k] - lo;
-      float s01 = d[0] + d[1], s23 = d[2] + d[3];
-      float sg = s01 + s23;
-      float p0 = d[0] * d[0], p2 = d[2] * d[2];
-      float q01 = fmaf(d[1], d[1], p0), q23 = fmaf(d[3], d[3], p2);
-      float qg = q01 + q23;
+      float s02 = d[0] + d[2], s13 = d[1] + d[3];
+      float sg = s02 + s13;
+      float p0 = d[0] * d[0], p1 = d[1] * d[1];
+      float q02 = fmaf(d[2], d[2], p0), q13 = fmaf(d[3], d[3], p1);
+      float qg = q02 + q13;
       st->Is += fixed_point(sg, 18 - st->e);
       st->Iq += fixed_point(qg, 16 - 2 * st->e);
     }

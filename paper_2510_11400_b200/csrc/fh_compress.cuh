@@ -865,15 +865,8 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
     _Pragma("unroll") for (int k = 0; k < G; ++k) {                                                           \
       const uint32_t g = lane + (uint32_t)(k * TT);                                                           \
       uint32_t w0, w1, w2, w3;                                                                                \
-      if (DT == kBF16) { /* packed pairs */                                                                  \
-        unpack2u(fma2(pack2(x[k][0], x[k][1]), inv2, mag2), w0, w1);                                          \
-        unpack2u(fma2(pack2(x[k][2], x[k][3]), inv2, mag2), w2, w3);                                          \
-      } else {                                                                                                \
-        w0 = __float_as_uint(__fmaf_rn(x[k][0], inv, kMagicF));                                               \
-        w1 = __float_as_uint(__fmaf_rn(x[k][1], inv, kMagicF));                                               \
-        w2 = __float_as_uint(__fmaf_rn(x[k][2], inv, kMagicF));                                               \
-        w3 = __float_as_uint(__fmaf_rn(x[k][3], inv, kMagicF));                                               \
-      }                                                                                                       \
+      unpack2u(fma2(pack2(x[k][0], x[k][1]), inv2, mag2), w0, w1); /* packed pairs */                         \
+      unpack2u(fma2(pack2(x[k][2], x[k][3]), inv2, mag2), w2, w3);                                            \
       uint32_t word = w0 + (w1 << (BITS)) + (w2 << (2 * (BITS))) + (w3 << (3 * (BITS))) - bias;               \
       if (FULL || g < groups) {                                                                               \
         if ((BITS) == 2) slot[g] = (uint8_t)word;                                                             \
@@ -958,13 +951,8 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
     const f32x2 nlo2 = pack2(nlo, nlo);
 #pragma unroll
     for (int k = 0; k < G; ++k) {
-      if (DT == kBF16) {
-        unpack2(add2(pack2(x[k][0], x[k][1]), nlo2), x[k][0], x[k][1]);
-        unpack2(add2(pack2(x[k][2], x[k][3]), nlo2), x[k][2], x[k][3]);
-      } else {
-#pragma unroll
-        for (int e = 0; e < 4; ++e) x[k][e] = __fadd_rn(x[k][e], nlo);
-      }
+      unpack2(add2(pack2(x[k][0], x[k][1]), nlo2), x[k][0], x[k][1]);
+      unpack2(add2(pack2(x[k][2], x[k][3]), nlo2), x[k][2], x[k][3]);
       if (!(FULL && VEC)) {
         const uint32_t g = lane + (uint32_t)(k * TT);
 #pragma unroll
@@ -982,7 +970,7 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
     if (sc.applies) {  // (the same for every thread of the team)
       uint32_t as = 0, aq = 0;
 #pragma unroll
-      for (int k = 0; k < G; ++k) sigma_addends4<DT == kBF16>(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
+      for (int k = 0; k < G; ++k) sigma_addends4(x[k][0], x[k][1], x[k][2], x[k][3], sc, as, aq);
       long long Is, Iq;
       team_sum2(team, (int32_t)(as - (uint32_t)G * kMagicBits), (int32_t)(aq - (uint32_t)G * kMagicBits), Is, Iq, rp);
       float dlo, dhi;
@@ -1422,14 +1410,9 @@ __device__ __forceinline__ void lds_group(const uint8_t* plane, uint32_t g, floa
 template <int DT>
 __device__ __forceinline__ void lds_dist(const uint8_t* plane, uint32_t g, float nlo, float (&v)[4]) {
   lds_group<DT>(plane, g, v);
-  if (DT == kBF16) {
-    const f32x2 nlo2 = pack2(nlo, nlo);
-    unpack2(add2(pack2(v[0], v[1]), nlo2), v[0], v[1]);
-    unpack2(add2(pack2(v[2], v[3]), nlo2), v[2], v[3]);
-  } else {
-#pragma unroll
-    for (int e = 0; e < 4; ++e) v[e] = __fadd_rn(v[e], nlo);
-  }
+  const f32x2 nlo2 = pack2(nlo, nlo);
+  unpack2(add2(pack2(v[0], v[1]), nlo2), v[0], v[1]);
+  unpack2(add2(pack2(v[2], v[3]), nlo2), v[2], v[3]);
 }
 
 #define FH_CTA_STORE_CODES(BITS)                                                                              \
@@ -1440,15 +1423,8 @@ __device__ __forceinline__ void lds_dist(const uint8_t* plane, uint32_t g, float
       float v[4];                                                                                             \
       lds_dist<DT>(plane, g, nlo, v);                                                                         \
       uint32_t w0, w1, w2, w3;                                                                                \
-      if (DT == kBF16) {                                                                                      \
-        unpack2u(fma2(pack2(v[0], v[1]), inv2, mag2), w0, w1);                                                \
-        unpack2u(fma2(pack2(v[2], v[3]), inv2, mag2), w2, w3);                                                \
-      } else {                                                                                                \
-        w0 = __float_as_uint(__fmaf_rn(v[0], inv, kMagicF));                                                  \
-        w1 = __float_as_uint(__fmaf_rn(v[1], inv, kMagicF));                                                  \
-        w2 = __float_as_uint(__fmaf_rn(v[2], inv, kMagicF));                                                  \
-        w3 = __float_as_uint(__fmaf_rn(v[3], inv, kMagicF));                                                  \
-      }                                                                                                       \
+      unpack2u(fma2(pack2(v[0], v[1]), inv2, mag2), w0, w1);                                                  \
+      unpack2u(fma2(pack2(v[2], v[3]), inv2, mag2), w2, w3);                                                  \
       uint32_t word = w0 + (w1 << (BITS)) + (w2 << (2 * (BITS))) + (w3 << (3 * (BITS))) - bias;               \
       if ((BITS) == 2) slot[g] = (uint8_t)word;                                                               \
       else if ((BITS) == 4) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;                            \
@@ -1565,7 +1541,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
         for (uint32_t g = tid; g < groups; g += NT) {
           float v[4];
           lds_dist<DT>(plane, g, nlo, v);
-          sigma_addends4<DT == kBF16>(v[0], v[1], v[2], v[3], sc, as, aq);
+          sigma_addends4(v[0], v[1], v[2], v[3], sc, as, aq);
           ++ng;
         }
         long long Is, Iq;

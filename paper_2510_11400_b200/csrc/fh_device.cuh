@@ -270,40 +270,27 @@ __device__ __forceinline__ SigmaScale sigma_scale(float range) {
   s.cq = __uint_as_float((uint32_t)(16 - 2 * e + 127) << 23);
   return s;
 }
-// Raw mantissa images of the two addends of one group of distances; the caller sums them with wrap-around
-// arithmetic and subtracts kMagicBits once per group at the end.
-__device__ __forceinline__ void sigma_addends(const float d[4], const SigmaScale& sc, uint32_t& as, uint32_t& aq) {
-  const float sg = __fadd_rn(__fadd_rn(d[0], d[1]), __fadd_rn(d[2], d[3]));
-  const float q01 = __fmaf_rn(d[1], d[1], __fmul_rn(d[0], d[0]));
-  const float q23 = __fmaf_rn(d[3], d[3], __fmul_rn(d[2], d[2]));
-  const float qg = __fadd_rn(q01, q23);
-  as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
-  aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
+// Raw mantissa images of the two addends of one group of distances (d0, d1, d2, d3); the caller sums them
+// with wrap-around arithmetic and subtracts kMagicBits once per group at the end.  The group's two pairs
+// (d0, d1) and (d2, d3) are combined position by position, s = (d0 + d2) + (d1 + d3) and
+// q = fma(d2, d2, d0 * d0) + fma(d3, d3, d1 * d1): with packed two-wide instructions that is one add, one
+// multiply and one multiply-add on the pairs as they come out of a 16-byte load, then one add of the halves each.
+__device__ __forceinline__ void sigma_addends2(f32x2 p, f32x2 q, const SigmaScale& sc, uint32_t& as, uint32_t& aq) {
+  float sa, sb, qa, qb;
+  unpack2(add2(p, q), sa, sb);                 // d0 + d2, d1 + d3
+  unpack2(fma2(q, q, mul2(p, p)), qa, qb);     // fma(d2, d2, d0 * d0), fma(d3, d3, d1 * d1)
+  const f32x2 fixed = fma2(pack2(__fadd_rn(sa, sb), __fadd_rn(qa, qb)), pack2(sc.cs, sc.cq), pack2(kMagicF, kMagicF));
+  uint32_t is, iq;
+  unpack2u(fixed, is, iq);
+  as += is;
+  aq += iq;
 }
-// PACKED: the same arithmetic with packed pairs -- (d0, d2) and (d1, d3) give both halves of every step at
-// once.  Used for bf16 input, whose unpacked values can be put in any registers and whose kernels are bound
-// by instruction issue; on fp32 input the repacking costs more than it saves.
-template <bool PACKED>
-__device__ __forceinline__ void sigma_addends4(float v0, float v1, float v2, float v3, const SigmaScale& sc,
+__device__ __forceinline__ void sigma_addends4(float d0, float d1, float d2, float d3, const SigmaScale& sc,
                                                uint32_t& as, uint32_t& aq) {
-  if (PACKED) {
-    const f32x2 ev = pack2(v0, v2), od = pack2(v1, v3);
-    float s01, s23, q01, q23;
-    unpack2(add2(ev, od), s01, s23);                 // d0 + d1, d2 + d3
-    unpack2(fma2(od, od, mul2(ev, ev)), q01, q23);   // fma(d1, d1, d0 * d0), fma(d3, d3, d2 * d2)
-    const f32x2 fixed = fma2(pack2(__fadd_rn(s01, s23), __fadd_rn(q01, q23)), pack2(sc.cs, sc.cq), pack2(kMagicF, kMagicF));
-    uint32_t is, iq;
-    unpack2u(fixed, is, iq);
-    as += is;
-    aq += iq;
-  } else {
-    const float sg = __fadd_rn(__fadd_rn(v0, v1), __fadd_rn(v2, v3));
-    const float q01 = __fmaf_rn(v1, v1, __fmul_rn(v0, v0));
-    const float q23 = __fmaf_rn(v3, v3, __fmul_rn(v2, v2));
-    const float qg = __fadd_rn(q01, q23);
-    as += __float_as_uint(__fmaf_rn(sg, sc.cs, kMagicF));
-    aq += __float_as_uint(__fmaf_rn(qg, sc.cq, kMagicF));
-  }
+  sigma_addends2(pack2(d0, d1), pack2(d2, d3), sc, as, aq);
+}
+__device__ __forceinline__ void sigma_addends(const float d[4], const SigmaScale& sc, uint32_t& as, uint32_t& aq) {
+  sigma_addends2(pack2(d[0], d[1]), pack2(d[2], d[3]), sc, as, aq);
 }
 // Thresholds, as distances from lo, from the exact integer sums: m1 +- 3 sigma.
 template <typename I>

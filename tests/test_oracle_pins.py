@@ -400,11 +400,11 @@ def test_fixed_point_sums_are_exact_integers_of_the_stated_roundings(scale, offs
     dp = np.concatenate([dd, np.zeros(1, np.float32)]).reshape(-1, 4)
     es = eq = 0
     for v in dp:
-        sg = np.float32(np.float32(v[0] + v[1]) + np.float32(v[2] + v[3]))
+        sg = np.float32(np.float32(v[0] + v[2]) + np.float32(v[1] + v[3]))
         f = [Fraction(float(t)) for t in v]
-        q01 = np.float32(float(f[1] * f[1] + Fraction(float(np.float32(v[0] * v[0])))))   # fma: one rounding
-        q23 = np.float32(float(f[3] * f[3] + Fraction(float(np.float32(v[2] * v[2])))))
-        qg = np.float32(q01 + q23)
+        q02 = np.float32(float(f[2] * f[2] + Fraction(float(np.float32(v[0] * v[0])))))   # fma: one rounding
+        q13 = np.float32(float(f[3] * f[3] + Fraction(float(np.float32(v[1] * v[1])))))
+        qg = np.float32(q02 + q13)
         es += rne(Fraction(float(sg)) * Fraction(2) ** (18 - e))
         eq += rne(Fraction(float(qg)) * Fraction(2) ** (16 - 2 * e))
     assert (Is, Iq) == (es, eq)
