@@ -1074,6 +1074,7 @@ __device__ __noinline__ void warp_tile_measure(BlockCtl* c, const uint8_t* tbuf,
 
 // Phase 1, the last of a tile's eight warps (one thread): the tile's sums are complete.
 __device__ __noinline__ void warp_tile_publish(BlockCtl* c, uint32_t s, uint32_t tile) {
+  __threadfence_block();  // the other warps' sums after their arrivals
   const uint32_t U = c->U[s], C = c->C[s];
   c->U[s] = 0;
   c->C[s] = 0;
@@ -1312,7 +1313,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
           warp_tile_measure<DT, TT>(&s_ctl, stage, (uint64_t)p0, s, (warp * 32u) / TT, leaders, meta,
                                     reinterpret_cast<uint32_t*>(smem + pl.sm_sal + warp * pl.sal_stride));
         if (lane == 0) {
-          __threadfence_block();
+          if (leaders) __threadfence_block();  // the warp's sums before its arrival
           if ((atomicAdd(&s_ctl.arr[s], 1u) & 7u) == 7u) warp_tile_publish(&s_ctl, s, tile);
         }
       }
@@ -1449,6 +1450,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
   __shared__ __align__(8) uint64_t s_full[kMaxStages];
   __shared__ uint32_t s_tiles[kMaxStages];
   __shared__ uint32_t s_abort, s_last;
+  __shared__ float2 s_thr;
   __shared__ BlockCtl s_ctl;
 
   const uint32_t tid = threadIdx.x;
@@ -1544,9 +1546,25 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
           sigma_addends4(v[0], v[1], v[2], v[3], sc, as, aq);
           ++ng;
         }
-        long long Is, Iq;
-        team_sum2(team, (int32_t)(as - ng * kMagicBits), (int32_t)(aq - ng * kMagicBits), Is, Iq, rp);
-        sigma_thresholds(Is, Iq, sc, pl.inv_hw, dlo, dhi);
+        {  // the first warp adds up the warps' sums and works out what depends on them, for all
+          int32_t pa = (int32_t)(as - ng * kMagicBits), pb = (int32_t)(aq - ng * kMagicBits);
+          asm volatile("redux.sync.add.s32 %0, %0, %1;" : "+r"(pa) : "r"(0xFFFFFFFFu));
+          asm volatile("redux.sync.add.s32 %0, %0, %1;" : "+r"(pb) : "r"(0xFFFFFFFFu));
+          int2* r = reinterpret_cast<int2*>(red_half(team, rp));
+          const uint32_t wl = tid & 31u;
+          if (wl == 0) r[tid >> 5] = make_int2(pa, pb);
+          __syncthreads();
+          if (tid < 32u) {
+            const int2 pr = wl < team.nwarps ? r[wl] : make_int2(0, 0);
+            const long long Is = warp_sum_s32_wide(pr.x), Iq = warp_sum_s32_wide(pr.y);
+            float tl, th;
+            sigma_thresholds(Is, Iq, sc, pl.inv_hw, tl, th);
+            if (tid == 0) s_thr = make_float2(tl, th);
+          }
+          __syncthreads();
+          dlo = s_thr.x;
+          dhi = s_thr.y;
+        }
         need_count = range > dhi || 0.0f < dlo;  // otherwise no element can lie outside
         one_sided = !(0.0f < dlo);
       }
