@@ -500,8 +500,29 @@ int launch_decompress_t(const Plan& pl, const fh::DecompressArgs& a, cudaStream_
   return FH_OK;
 }
 
+// Planes of at most 128 groups: tiles of 256 / team planes restored in shared memory, one bulk store per tile.
+template <int DT>
+int launch_decompress_small(const Plan& pl0, const fh::DecompressArgs& a, cudaStream_t stream) {
+  Plan pl = pl0;
+  pl.ppt = fh::kThreads / pl.team;
+  if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
+  pl.stage_bytes = (uint32_t)((pl.ppt * pl.plane_bytes + 127) & ~(uint64_t)127);
+  pl.ntiles = (uint32_t)((pl.P + pl.ppt - 1) / pl.ppt);
+  // two tile buffers, then per warp: scratch for a small plane's payload, or the block-wise scratch of a larger one
+  pl.sm_total = 2u * pl.stage_bytes + (uint32_t)fh::kWarps * (uint32_t)(A16(pl.plane_bytes) + 16 + 4u * pl.nblk);
+  if (pl.sm_total > kSmemLimit) return FH_ERR_UNSUPPORTED;
+  int grid = 0;
+  int rc = grid_for(fh::decompress_small<DT>, pl.sm_total, pl.ntiles, &grid);
+  if (rc != FH_OK) return rc;
+  if (launch_dependent(fh::decompress_small<DT>, grid, fh::kThreads, pl.sm_total, stream, pl, a) != cudaSuccess)
+    return FH_ERR_CUDA;
+  g_launches.fetch_add(1);
+  return FH_OK;
+}
+
 template <int DT>
 int launch_decompress(const Plan& pl, const fh::DecompressArgs& a, cudaStream_t stream) {
+  if (pl.groups <= 128 && pl.P <= 0x7FFFFFFFull) return launch_decompress_small<DT>(pl, a, stream);
   switch (pl.team) {
     case 1: return launch_decompress_t<DT, 1>(pl, a, stream);
     case 2: return launch_decompress_t<DT, 2>(pl, a, stream);

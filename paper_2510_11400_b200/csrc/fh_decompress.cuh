@@ -156,6 +156,22 @@ __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const
   return ok;
 }
 
+// Header of a container against what the caller expects; also returns code width, eps and total size.
+__device__ __forceinline__ uint32_t check_header(const Plan& pl, const uint8_t* src, unsigned long long src_bytes, uint32_t& bits,
+                                                 float& eps, unsigned long long& total) {
+  if (src_bytes < 64ull + 16ull * pl.P) return 0u;
+  const uint32_t* h = reinterpret_cast<const uint32_t*>(src);
+  bits = __ldg(h + 1) >> 24;
+  bool ok = __ldg(h) == kMagic && (__ldg(h + 1) & 0xFFFFu) == 1u && ((__ldg(h + 1) >> 16) & 0xFFu) == (uint32_t)pl.dtype &&
+            (bits == 2u || bits == 4u || bits == 8u) && __ldg(h + 2) == pl.N && __ldg(h + 3) == pl.C &&
+            __ldg(h + 4) == (uint32_t)pl.H && __ldg(h + 5) == (uint32_t)pl.W && (__ldg(h + 6) & 0xFFFFu) == (8u | (8u << 8));
+  total = (unsigned long long)__ldg(h + 14) | ((unsigned long long)__ldg(h + 15) << 32);
+  eps = __uint_as_float(__ldg(h + 9));
+  const unsigned long long npay = a16(4u * ((pl.HW * (bits & 15u) + 31u) / 32u));
+  ok = ok && total <= src_bytes && total >= 64ull + 16ull * pl.P + pl.P * npay && eps >= 1e-30f && eps <= 1e30f;
+  return ok ? 1u : 0u;
+}
+
 // Four restored values of one group leave as one 16-byte (fp32) or 8-byte (bf16) store.
 template <int DT>
 __device__ __forceinline__ void store_group(uint8_t* out, uint32_t g, float v0, float v1, float v2, float v3) {
@@ -255,22 +271,13 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
 
   // header check (every CTA, it is 64 bytes)
   if (tid == 0) {
-    uint32_t ok = src_bytes >= 64ull + 16ull * pl.P;
-    if (ok) {
-      const uint32_t* h = reinterpret_cast<const uint32_t*>(src);
-      const uint32_t bits = __ldg(h + 1) >> 24;
-      ok = __ldg(h) == kMagic && (__ldg(h + 1) & 0xFFFFu) == 1u && ((__ldg(h + 1) >> 16) & 0xFFu) == (uint32_t)pl.dtype &&
-           (bits == 2u || bits == 4u || bits == 8u) && __ldg(h + 2) == pl.N && __ldg(h + 3) == pl.C &&
-           __ldg(h + 4) == (uint32_t)pl.H && __ldg(h + 5) == (uint32_t)pl.W && (__ldg(h + 6) & 0xFFFFu) == (8u | (8u << 8));
-      const unsigned long long total = (unsigned long long)__ldg(h + 14) | ((unsigned long long)__ldg(h + 15) << 32);
-      const float eps = __uint_as_float(__ldg(h + 9));
-      const unsigned long long npay = a16(4u * ((pl.HW * (bits & 15u) + 31u) / 32u));
-      ok = ok && total <= src_bytes && total >= 64ull + 16ull * pl.P + pl.P * npay && eps >= 1e-30f && eps <= 1e30f;
-      s_bits = bits;
-      s_eps = eps;
-      s_total = total;
-    }
-    s_hdr_ok = ok;
+    uint32_t bits = 0;
+    float eps = 0.0f;
+    unsigned long long total = 0;
+    s_hdr_ok = check_header(pl, src, src_bytes, bits, eps, total);
+    s_bits = bits;
+    s_eps = eps;
+    s_total = total;
   }
   __syncthreads();
   const bool hdr_ok = s_hdr_ok != 0;
@@ -399,6 +406,311 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
         bad = true;
       __syncthreads();  // the scratch is reused
     }
+  }
+  if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const unsigned long long prev = atomicAdd(&a.sc->exited, 1ull);
+    if (prev == (unsigned long long)gridDim.x - 1ull) {
+      __threadfence();
+      const uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
+      if (a.d_status) *a.d_status = status_word(code);
+      st_relaxed(&a.sc->status, 0ull);
+      st_relaxed(&a.sc->exited, 0ull);
+    }
+  }
+}
+
+// -------------------------------------------------------------------------------------------------
+// Small planes (at most 128 groups: 7x7, 14x14, 16x16, ...).  Such planes rarely start on 16-byte boundaries,
+// and a team of a few lanes that stores its plane element by element scatters 4-byte stores over many
+// sectors.  Here a CTA restores a tile of consecutive planes into shared memory -- a team of lanes per
+// normal plane, the whole warp for an outlier-rich one -- and the tile leaves as one bulk (TMA) store.
+// Tiles (256 / team planes) start on 16-byte boundaries; two buffers alternate.
+// -------------------------------------------------------------------------------------------------
+
+// Outlier-rich plane of at most four blocks and fewer than 32 rows, restored by one warp: CSR scatter, then per
+// dense block the inverse of the Lorenzo prediction as a two-dimensional prefix sum of the residuals over the
+// warp's lanes (lane l holds raster positions l and l + 32), corrected in raster order for every verbatim
+// element, whose k follows from its stored value.  The result is that of the raster walk in decode_salient.
+// A payload copied to shared memory as one piece.
+struct FlatIn {
+  const uint8_t* p;
+  uint32_t npay;  // (kept for the size check: bytes of the payload that came from the slot)
+  __device__ __forceinline__ uint32_t ld32(uint32_t o) const { return *reinterpret_cast<const uint32_t*>(p + o); }
+  __device__ __forceinline__ uint32_t ld16(uint32_t o) const { return *reinterpret_cast<const uint16_t*>(p + o); }
+};
+
+template <int DT, typename In>
+__device__ __forceinline__ bool small_decode(const Plan& pl, const In& in, uint64_t ovf_avail, float eps, uint8_t* out) {
+  const uint32_t lane = threadIdx.x & 31u, full = 0xFFFFFFFFu;
+  const uint32_t H = (uint32_t)pl.H, W = (uint32_t)pl.W, nblk = pl.nblk, nbx = pl.nbx, e = (uint32_t)pl.esize, HW = pl.HW;
+  const uint32_t nnz_s = in.ld32(0), n_dense = in.ld32(4), n_out_d = in.ld32(8);
+  if (nnz_s > HW || n_dense > nblk || n_out_d > HW) return false;
+  const uint64_t size = 16ull + 4ull * pl.nbm + 4ull * ((uint64_t)H + 1) + a4(2u * nnz_s) + a4(e * nnz_s) +
+                        64ull * n_dense + a4(e * n_out_d);
+  if (size > in.npay && size - in.npay > ovf_avail) return false;
+  const uint32_t o_bm = 16u, o_rp = o_bm + 4u * pl.nbm, o_col = o_rp + 4u * (H + 1u);
+  const uint32_t o_val = o_col + a4(2u * nnz_s), o_codes = o_val + a4(e * nnz_s), o_outl = o_codes + 64u * n_dense;
+  const uint32_t bitmap = in.ld32(o_bm) & ((1u << nblk) - 1u);
+  if ((uint32_t)__popc(bitmap) != n_dense) return false;
+  bool ok = true;
+  for (uint32_t i = lane; i < (uint32_t)(pl.plane_bytes >> 1); i += 32u) reinterpret_cast<uint16_t*>(out)[i] = 0;
+  __syncwarp();
+  if (lane < H) {  // CSR scatter, a lane per row
+    const uint32_t r0 = in.ld32(o_rp + 4u * lane), r1 = in.ld32(o_rp + 4u * lane + 4u);
+    if (r0 > r1 || r1 > nnz_s) {
+      ok = false;
+    } else {
+      for (uint32_t k = r0; k < r1; ++k) {
+        const uint32_t col = in.ld16(o_col + 2u * k);
+        if (col >= W) {
+          ok = false;
+          continue;
+        }
+        const uint32_t idx = lane * W + col;
+        if (DT == kF32) reinterpret_cast<uint32_t*>(out)[idx] = in.ld32(o_val + 4u * k);
+        else reinterpret_cast<uint16_t*>(out)[idx] = (uint16_t)in.ld16(o_val + 2u * k);
+      }
+    }
+  }
+  const float two_eps = __fmul_rn(2.0f, eps), inv2e = __fdiv_rn(1.0f, two_eps);
+  const uint32_t c = lane & 7u, r0 = lane >> 3, lt = (1u << lane) - 1u;
+  uint32_t oi = 0, rank = 0;
+#pragma unroll 1
+  for (uint32_t b = 0; b < nblk; ++b) {
+    if (!((bitmap >> b) & 1u)) continue;
+    const uint32_t oc = o_codes + 64u * rank;
+    const uint32_t code0 = (in.ld32(oc + (lane & ~3u)) >> (8u * (lane & 3u))) & 0xFFu;
+    const uint32_t code1 = (in.ld32(oc + 32u + (lane & ~3u)) >> (8u * (lane & 3u))) & 0xFFu;
+    const uint32_t by = b / nbx, bx = b - by * nbx;
+    const uint32_t y0 = by * 8u + r0, x = bx * 8u + c;
+    const bool in0 = y0 < H && x < W, in1 = y0 + 4u < H && x < W;
+    const bool v0 = in0 && code0 == 0u, v1 = in1 && code1 == 0u;
+    int32_t k0 = (in0 && !v0) ? (int32_t)code0 - 128 : 0, k1 = (in1 && !v1) ? (int32_t)code1 - 128 : 0;
+#pragma unroll
+    for (uint32_t o = 1; o < 8u; o <<= 1) {  // along the rows
+      const int32_t t0 = __shfl_up_sync(full, k0, o), t1 = __shfl_up_sync(full, k1, o);
+      if (c >= o) {
+        k0 += t0;
+        k1 += t1;
+      }
+    }
+#pragma unroll
+    for (uint32_t o = 8; o < 32u; o <<= 1) {  // down the columns, within each half
+      const int32_t t0 = __shfl_up_sync(full, k0, o), t1 = __shfl_up_sync(full, k1, o);
+      if (lane >= o) {
+        k0 += t0;
+        k1 += t1;
+      }
+    }
+    k1 += __shfl_sync(full, k0, 24 + (int)c);  // rows 4-7 continue below row 3
+    const uint32_t m0 = __ballot_sync(full, v0), m1 = __ballot_sync(full, v1);
+    const uint32_t nv = (uint32_t)(__popc(m0) + __popc(m1));
+    if (oi + nv > n_out_d) return false;  // (the same for every lane)
+    uint32_t raw0 = 0, raw1 = 0;
+    int32_t kv0 = 0, kv1 = 0;
+    if (v0) {
+      const uint32_t at = oi + (uint32_t)__popc(m0 & lt);
+      raw0 = DT == kF32 ? in.ld32(o_outl + 4u * at) : in.ld16(o_outl + 2u * at);
+      bool big;
+      kv0 = dense_k(DT == kF32 ? __uint_as_float(raw0) : bf16_bits_to_f32(raw0), inv2e, &big);
+    }
+    if (v1) {
+      const uint32_t at = oi + (uint32_t)__popc(m0) + (uint32_t)__popc(m1 & lt);
+      raw1 = DT == kF32 ? in.ld32(o_outl + 4u * at) : in.ld16(o_outl + 2u * at);
+      bool big;
+      kv1 = dense_k(DT == kF32 ? __uint_as_float(raw1) : bf16_bits_to_f32(raw1), inv2e, &big);
+    }
+    // a verbatim element replaces its k: the difference moves every k below and to the right of it
+    for (uint32_t mm = m0; mm; mm &= mm - 1u) {
+      const uint32_t src = (uint32_t)__ffs((int)mm) - 1u, i = src >> 3, j = src & 7u;
+      const int32_t diff = __shfl_sync(full, kv0 - k0, (int)src);
+      if (c >= j) {
+        if (r0 >= i) k0 += diff;
+        k1 += diff;
+      }
+    }
+    for (uint32_t mm = m1; mm; mm &= mm - 1u) {
+      const uint32_t src = (uint32_t)__ffs((int)mm) - 1u, i = src >> 3, j = src & 7u;
+      const int32_t diff = __shfl_sync(full, kv1 - k1, (int)src);
+      if (c >= j && r0 >= i) k1 += diff;
+    }
+    if (in0) {
+      const uint32_t idx = y0 * W + x;
+      if (v0) {
+        if (DT == kF32) reinterpret_cast<uint32_t*>(out)[idx] = raw0;
+        else reinterpret_cast<uint16_t*>(out)[idx] = (uint16_t)raw0;
+      } else {
+        store_elem<DT>(out, idx, __fmul_rn((float)k0, two_eps));
+      }
+    }
+    if (in1) {
+      const uint32_t idx = (y0 + 4u) * W + x;
+      if (v1) {
+        if (DT == kF32) reinterpret_cast<uint32_t*>(out)[idx] = raw1;
+        else reinterpret_cast<uint16_t*>(out)[idx] = (uint16_t)raw1;
+      } else {
+        store_elem<DT>(out, idx, __fmul_rn((float)k1, two_eps));
+      }
+    }
+    oi += nv;
+    ++rank;
+  }
+  return __all_sync(full, ok);
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 4) decompress_small(const Plan pl, const DecompressArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ double s_red[kMaxWarps * 5];
+  __shared__ uint32_t s_hdr_ok, s_bits;
+  __shared__ float s_eps;
+  __shared__ unsigned long long s_total;
+  __shared__ Plan s_pl;  // copy for the outlined slow path, which takes it by address
+  const uint32_t tid = threadIdx.x, wlane = tid & 31u;
+  if (tid == 0) s_pl = pl;
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
+  dep_wait();     // the previous kernel on the stream (the one that wrote the container) has completed
+  const unsigned long long off_in = a.d_off_in ? *a.d_off_in : 0ull;
+  const uint8_t* src = a.src_base + off_in;
+  const unsigned long long src_bytes = a.src_bytes > off_in ? a.src_bytes - off_in : 0ull;
+  if (tid == 0) {
+    uint32_t bits = 0;
+    float eps = 0.0f;
+    unsigned long long total = 0;
+    s_hdr_ok = check_header(pl, src, src_bytes, bits, eps, total);
+    s_bits = bits;
+    s_eps = eps;
+    s_total = total;
+  }
+  __syncthreads();
+  bool bad = s_hdr_ok == 0;
+  if (!bad) {
+    const uint32_t bits = s_bits, L = (1u << bits) - 1u;
+    const float eps = s_eps;
+    const unsigned long long total = s_total;
+    const uint32_t npay = a16(4u * ((pl.HW * bits + 31u) / 32u));
+    const unsigned long long slots_off = 64ull + 16ull * pl.P, ovf_off = slots_off + pl.P * (unsigned long long)npay;
+    const uint32_t tt = pl.team, lane = tid & (tt - 1u), my_team = tid / tt;
+    const Team warp_team = make_warp_team(s_red);
+    const bool vec = (pl.plane_bytes & (DT == kF32 ? 15u : 7u)) == 0u;  // planes start on vector boundaries in the tile buffer
+    const uint32_t tile_bytes_max = pl.stage_bytes;
+    const uint32_t pay_stride = a16((uint32_t)pl.plane_bytes) + 16u;  // per-warp scratch for a small plane's payload
+    uint32_t buf = 0;
+    for (uint32_t tile = blockIdx.x; tile < pl.ntiles; tile += gridDim.x, buf ^= 1u) {
+      uint8_t* tbuf = smem + (uint64_t)buf * tile_bytes_max;
+      if (tid == 0) bulk_wait_read<1>();  // the store that left this buffer two tiles ago has read it
+      __syncthreads();
+      const uint64_t p0 = (uint64_t)tile * pl.ppt;
+      const uint32_t np = (uint32_t)min((uint64_t)pl.ppt, pl.P - p0);
+      const uint32_t lp = my_team;
+      bool salient = false;
+      if (lp < np) {
+        const uint64_t gp = p0 + lp;
+        const uint4 en = __ldg(reinterpret_cast<const uint4*>(src + 64) + gp);
+        const unsigned long long off = (unsigned long long)en.x * 16ull;
+        const uint32_t cls = en.y & 3u;
+        uint8_t* out = tbuf + (uint64_t)lp * pl.plane_bytes;
+        const uint8_t* slot = src + slots_off + gp * npay;
+        if (cls == kClsNormal) {
+          if (off != slots_off + gp * npay) {
+            bad = true;
+          } else {
+            const float lo = __uint_as_float(en.z), scale = __uint_as_float(en.w);
+            for (uint32_t g = lane; g < pl.groups; g += tt) {
+              const uint32_t word = bits == 2u ? (uint32_t)__ldg(slot + g)
+                                               : (bits == 4u ? (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(slot) + g)
+                                                             : __ldg(reinterpret_cast<const uint32_t*>(slot) + g));
+              const uint32_t i = 4u * g;
+              if (vec && i + 3u < pl.HW) {  // whole group of a plane on a vector boundary: one store
+                store_group<DT>(out, g, dequant(word & L, scale, lo), dequant((word >> bits) & L, scale, lo),
+                                dequant((word >> (2u * bits)) & L, scale, lo), dequant((word >> (3u * bits)) & L, scale, lo));
+              } else {
+#pragma unroll
+                for (uint32_t k = 0; k < 4u; ++k)
+                  if (i + k < pl.HW) store_elem<DT>(out, i + k, dequant((word >> (k * bits)) & L, scale, lo));
+              }
+            }
+          }
+        } else if (cls == kClsRaw) {
+          if (off != 0 && (off < ovf_off || off > total)) {
+            bad = true;
+          } else {
+            SplitIn in;
+            in.slot = slot;
+            in.ovf = src + off;
+            in.npay = npay;
+            const unsigned long long ovf_avail = off ? total - off : 0ull;
+            if (pl.plane_bytes > npay && pl.plane_bytes - npay > ovf_avail) bad = true;
+            else
+              for (uint32_t i = lane; i < (uint32_t)(pl.plane_bytes >> 1); i += tt)
+                reinterpret_cast<uint16_t*>(out)[i] = (uint16_t)in.ld16(2u * i);
+          }
+        } else if (cls == kClsSalient) {
+          salient = true;
+        } else {
+          bad = true;
+        }
+      }
+      // outlier-rich planes of the warp's slice: the whole warp restores them one after the other
+      for (uint32_t m = __ballot_sync(0xFFFFFFFFu, salient && lane == 0); m; m &= m - 1u) {
+        const uint32_t slp = (tid & ~31u) / tt + ((uint32_t)__ffs((int)m) - 1u) / tt;
+        const uint64_t gp = p0 + slp;
+        const unsigned long long off = (unsigned long long)__ldg(reinterpret_cast<const uint32_t*>(src + 64 + 16ull * gp)) * 16ull;
+        if (off != 0 && (off < ovf_off || off > total)) {
+          bad = true;
+          continue;
+        }
+        SplitIn in;
+        in.slot = src + slots_off + gp * npay;
+        in.ovf = src + off;
+        in.npay = npay;
+        uint8_t* out = tbuf + (uint64_t)slp * pl.plane_bytes;
+        const unsigned long long ovf_avail = off ? total - off : 0ull;
+        __syncwarp();
+        bool good;
+        if (pl.nblk <= 4u && pl.H < 32) {
+          // the payload (shorter than the plane, or it would have been stored raw) is fetched in one go into the
+          // warp's scratch and decoded from there
+          uint8_t* pay = smem + 2ull * tile_bytes_max + (uint64_t)(tid >> 5) * pay_stride;
+          const uint32_t nnz_s = in.ld32(0), n_dense = in.ld32(4), n_out_d = in.ld32(8), es = (uint32_t)pl.esize;
+          const uint64_t size = 16ull + 4ull * pl.nbm + 4ull * ((uint64_t)pl.H + 1) + a4(2u * nnz_s) + a4(es * nnz_s) +
+                                64ull * n_dense + a4(es * n_out_d);
+          good = nnz_s <= pl.HW && n_dense <= pl.nblk && n_out_d <= pl.HW && size <= pay_stride &&
+                 !(size > npay && size - npay > ovf_avail);
+          if (good) {
+            for (uint32_t o = 4u * wlane; o < (uint32_t)size; o += 128u) *reinterpret_cast<uint32_t*>(pay + o) = in.ld32(o);
+            __syncwarp();
+            FlatIn flat;
+            flat.p = pay;
+            flat.npay = npay;
+            good = small_decode<DT>(s_pl, flat, ovf_avail, eps, out);
+          }
+        } else {
+          good = decode_salient<DT>(warp_team, s_pl, in, ovf_avail, eps, out,
+                                    reinterpret_cast<uint32_t*>(smem + 2ull * tile_bytes_max) + (tid >> 5) * pl.nblk);
+        }
+        if (!good) bad = true;
+        __syncwarp();
+      }
+      __syncthreads();
+      // the tile leaves: one bulk store when it is whole 16-byte chunks, plain stores otherwise
+      const uint32_t bytes = np * (uint32_t)pl.plane_bytes;
+      uint8_t* dst = a.dst + p0 * pl.plane_bytes;
+      if ((bytes & 15u) == 0u) {
+        if (tid == 0) {
+          fence_proxy_async();
+          bulk_s2g(dst, tbuf, bytes);
+          bulk_commit();
+        }
+      } else {
+        for (uint32_t i = tid; i < (bytes >> 1); i += kThreads)
+          reinterpret_cast<uint16_t*>(dst)[i] = reinterpret_cast<const uint16_t*>(tbuf)[i];
+      }
+    }
+    if (tid == 0) bulk_wait<0>();  // every store of this CTA is complete
   }
   if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
   __threadfence();

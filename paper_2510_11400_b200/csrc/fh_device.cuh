@@ -131,6 +131,9 @@ __device__ __forceinline__ void bulk_s2g(void* dst, const void* src, uint32_t by
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// ... until all but the N most recent groups are complete (their writes performed).
+template <int N>
+__device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
 // One wait attempt: the hardware may suspend the thread for up to about `kSuspendNs` nanoseconds
 // while the phase is incomplete, so that waiting warps do not burn issue slots polling.
 constexpr uint32_t kSuspendNs = 2000;
