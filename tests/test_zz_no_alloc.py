@@ -5,8 +5,8 @@ because its device-memory budget is already spent, a process whose memory is who
 framework pool, a loop that cannot take the synchronisation an allocation may imply.  Its
 book-keeping scratch is a fixed array inside the library, shared by all calls on a device and cleared
 by each call.  The test drives it through the C ABI and requires the same container, byte for byte, as
-fh_compress, twice in a row (the second call sees the first call's leftovers in the array), and
-checks that a tensor beyond the fixed limit is refused.
+fh_compress and as the CPU oracle, twice in a row (the second call sees the first call's leftovers in
+the array), and checks that a tensor beyond the fixed limit is refused.
 
 Collected last on purpose, and self-contained: it must pass alone in a fresh process and after the
 other GPU tests.
@@ -14,6 +14,7 @@ other GPU tests.
 import numpy as np
 import pytest
 
+from oracle import fho
 from paper_2510_11400_b200 import api, build, synth
 
 pytestmark = pytest.mark.gpu
@@ -35,6 +36,8 @@ def _compress_both(spec, bits):
         total, st = out2.tolist()
         assert st == api.FH_OK
         outs.append(dst[:total].cpu().numpy())
+    st_o, buf_o, total_o = fho.compress(raw, fho.desc(spec.shape, spec.dtype, tensor_id=7), fho.params(bits=bits))
+    assert st_o == fho.OK and np.array_equal(outs[1], buf_o), "fh_compress_static differs from the oracle"
     return outs
 
 
