@@ -301,6 +301,22 @@ int fh_plan_generate(const fh_plan_op* ops, int32_t n_ops, const fh_plan_tensor*
                      fh_plan_report* report);
 
 /*
+ * Costs of compression as this library delivers them on the current device, measured: the quantities PC(d)
+ * and RC(d) of the compression technique in Eq. 5 and the space it frees (SM(d)), for fh_plan_generate.
+ * For every tensor i the call compresses d_dense[i] into the work buffer and restores it again, `repeats`
+ * times each after one untimed run, timed with CUDA events on `stream`, and fills
+ *   out[i].bytes, out[i].packed_bytes (the container's size), out[i].t_compress, out[i].t_decompress
+ * (seconds, mean of the repeats).  out[i].t_recompute is left as the caller set it (Eq. 6 is the caller's).
+ *   descs, d_dense   n tensor descriptions and their dense device buffers (16-byte aligned)
+ *   d_work           caller-owned device workspace, 256-byte aligned, at least fh_host_work_bytes(desc, params)
+ *                    bytes for the largest tensor (it holds the container and the restored copy)
+ *   repeats          1..1000
+ * The call synchronises the stream.  Returns FH_OK, an argument error, or the first device-side status.
+ */
+int fh_plan_measure(const fh_tensor_desc* descs, int32_t n, const fh_params* params, const void* const* d_dense,
+                    void* d_work, size_t work_bytes, int32_t repeats, fh_plan_tensor* out, void* stream);
+
+/*
  * Fault injection on the host side, for tests of the error path of the device-side waits.  (The paper has no
  * counterpart.)  Compressing places the overflow parts of outlier-rich planes in plane order: a tile of
  * planes waits, with a limit, until every earlier tile has published its size; a wait that runs out ends the

@@ -23,7 +23,8 @@ FH_DEBUG_WAIT_POLLS, FH_DEBUG_SILENT_TILE = 0, 1
 
 EXPORTS = ["fh_default_params", "fh_version", "fh_device_count", "fh_compressed_bytes", "fh_compress",
            "fh_decompress", "fh_run_schedule", "fh_host_work_bytes", "fh_compress_host",
-           "fh_decompress_host", "fh_compress_static", "fh_plan_generate", "fh_debug_set", "fh_kernel_launches",
+           "fh_decompress_host", "fh_compress_static", "fh_plan_generate", "fh_plan_measure", "fh_debug_set",
+           "fh_kernel_launches",
            "fh_shutdown"]
 
 
@@ -115,6 +116,9 @@ def lib() -> C.CDLL:
                                        C.POINTER(C.c_int32), C.POINTER(fh_plan_event), C.c_int32,
                                        C.POINTER(fh_plan_report)]
         L.fh_plan_generate.restype = C.c_int
+        L.fh_plan_measure.argtypes = [D, C.c_int32, P, C.POINTER(C.c_void_p), C.c_void_p, C.c_size_t, C.c_int32,
+                                      C.POINTER(fh_plan_tensor), C.c_void_p]
+        L.fh_plan_measure.restype = C.c_int
         L.fh_debug_set.argtypes = [C.c_int, C.c_uint64]
         L.fh_debug_set.restype = C.c_int
         L.fh_kernel_launches.restype = C.c_uint64
@@ -236,6 +240,22 @@ def plan_generate(ops, tensors, memory_budget: int, max_events: int = 4096):
     rc = lib().fh_plan_generate(c_ops, len(ops), c_t, len(tensors), memory_budget, actions, events, max_events, C.byref(rep))
     n = min(rep.n_events, max_events)
     return int(rc), [int(a) for a in actions[:len(tensors)]], [(e.op, e.tensor, e.kind) for e in events[:n]], rep
+
+
+def plan_measure(descs, p: fh_params, dense, work, repeats: int = 5, t_recompute=None, stream=None):
+    """Measured costs of compression for plan generation: descs and dense are matching lists (descriptions, torch
+    CUDA tensors); work is a uint8 CUDA tensor of at least host_work_bytes of the largest tensor.  Returns
+    (status, list of dicts in the form plan_generate takes); t_recompute (list, seconds) is passed through."""
+    n = len(descs)
+    c_d = (fh_tensor_desc * n)(*descs)
+    ptrs = (C.c_void_p * n)(*[t.data_ptr() for t in dense])
+    out = (fh_plan_tensor * n)()
+    for i in range(n):
+        out[i].t_recompute = -1.0 if t_recompute is None else t_recompute[i]
+    rc = lib().fh_plan_measure(c_d, n, C.byref(p), ptrs, work.data_ptr(), work.numel() * work.element_size(), repeats, out,
+                               _stream_ptr(stream))
+    return int(rc), [dict(bytes=int(o.bytes), packed_bytes=int(o.packed_bytes), t_compress=float(o.t_compress),
+                          t_decompress=float(o.t_decompress), t_recompute=float(o.t_recompute)) for o in out]
 
 
 def debug_set(what: int, value: int) -> int:

@@ -816,6 +816,66 @@ int fh_decompress_host(const void* h_src, size_t src_bytes, const fh_tensor_desc
   return (int)(long long)st;
 }
 
+int fh_plan_measure(const fh_tensor_desc* descs, int32_t n, const fh_params* params, const void* const* d_dense,
+                    void* d_work, size_t work_bytes, int32_t repeats, fh_plan_tensor* out, void* stream_) {
+  if (!descs || !d_dense || !out || n < 0 || !d_work || misaligned(d_work, 256) || repeats < 1 || repeats > 1000)
+    return FH_ERR_ARG;
+  int rc = check_params(params);
+  if (rc != FH_OK) return rc;
+  for (int32_t i = 0; i < n; ++i) {
+    rc = check_desc(&descs[i]);
+    if (rc != FH_OK) return rc;
+    if (!d_dense[i] || misaligned(d_dense[i], 16)) return FH_ERR_ARG;
+    if (work_bytes < fh_host_work_bytes(&descs[i], params)) return FH_ERR_ARG;
+  }
+  cudaStream_t stream = (cudaStream_t)stream_;
+  cudaEvent_t e0, e1, e2;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess || cudaEventCreate(&e2) != cudaSuccess)
+    return FH_ERR_CUDA;
+  rc = FH_OK;
+  for (int32_t i = 0; i < n && rc == FH_OK; ++i) {
+    const fh_tensor_desc& d = descs[i];
+    const size_t dense = (size_t)d.n * d.c * d.h * d.w * esize_of(d.dtype);
+    const size_t worst = fh_compressed_bytes(&d, params, 1);
+    // work buffer: restored copy | result words | container (the layout of the host-buffer entry points)
+    uint8_t* d_rest = (uint8_t*)d_work;
+    unsigned long long* d_words = (unsigned long long*)(d_rest + A256(dense));
+    uint8_t* d_pack = (uint8_t*)d_words + 256;
+    for (int pass = 0; pass < 2 && rc == FH_OK; ++pass) {  // pass 0: the untimed run
+      const int reps = pass ? repeats : 1;
+      cudaEventRecord(e0, stream);
+      for (int r = 0; r < reps && rc == FH_OK; ++r)
+        rc = fh_compress(&d, params, d_dense[i], d_pack, worst, (uint64_t*)d_words, stream_);
+      cudaEventRecord(e1, stream);
+      for (int r = 0; r < reps && rc == FH_OK; ++r)
+        rc = fh_decompress(d_pack, worst, &d, d_rest, (uint64_t*)(d_words + 2), stream_);
+      cudaEventRecord(e2, stream);
+      if (cudaStreamSynchronize(stream) != cudaSuccess) rc = rc == FH_OK ? FH_ERR_CUDA : rc;
+      if (rc != FH_OK) break;
+      unsigned long long h[3] = {0, 0, 0};
+      if (cudaMemcpy(h, d_words, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        rc = FH_ERR_CUDA;
+        break;
+      }
+      if ((int)(long long)h[1] != FH_OK) rc = (int)(long long)h[1];
+      else if ((int)(long long)h[2] != FH_OK) rc = (int)(long long)h[2];
+      if (pass && rc == FH_OK) {
+        float ms_c = 0.0f, ms_d = 0.0f;
+        cudaEventElapsedTime(&ms_c, e0, e1);
+        cudaEventElapsedTime(&ms_d, e1, e2);
+        out[i].bytes = dense;
+        out[i].packed_bytes = h[0];
+        out[i].t_compress = (double)ms_c * 1e-3 / repeats;
+        out[i].t_decompress = (double)ms_d * 1e-3 / repeats;
+      }
+    }
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  cudaEventDestroy(e2);
+  return rc;
+}
+
 // ---- allocation-free compress -----------------------------------------------------------------
 // Scratch compiled into the device image: the counters (padded to 256 bytes), the placement scan's arrays
 // and the tile links for FH_STATIC_MAX_PLANES tiles (a tile is at least one plane).  The name is a device symbol: host

@@ -572,34 +572,35 @@ def test_parity_random_rounding(shape, dtype, bits):
 
 
 def test_generated_plan_drives_the_schedule():
-    """Algorithm 1 end to end: a plan is generated for one training step under a memory budget (costs of
-    compression as this library delivers them on a B200-class device, recomputation costs made up), and its
-    per-tensor actions are what fh_run_schedule executes."""
+    """Algorithm 1 end to end: the costs of compression are measured from this library on this device
+    (fh_plan_measure: PC, RC and the freed space of Eq. 5), a plan is generated for one training step under a
+    memory budget (recomputation costs made up), and its per-tensor actions are what fh_run_schedule executes."""
     import torch
     shapes = [(8, 32, 32, 32), (8, 32, 32, 32), (8, 64, 16, 16), (8, 64, 16, 16), (8, 128, 8, 8), (8, 128, 8, 8)]
     specs = [synth.TensorSpec(f"p{i}", sh, synth.F32, "relu", 700 + i) for i, sh in enumerate(shapes)]
     n = len(specs)
     p = api.default_params(bits=2)
-    tensors = []
-    for i, sp in enumerate(specs):
-        b = sp.dense_bytes
-        packed = api.compressed_bytes(api.desc(sp.shape, sp.dtype), p, 0)
-        tensors.append(dict(bytes=b, packed_bytes=packed, t_compress=20e-6 + b / 3e12, t_decompress=12e-6 + b / 4e12,
-                            t_recompute=(10e-6 if i == 1 else 400e-6)))
+    raws = [synth.make(sp) for sp in specs]
+    dense = [to_dev(r) for r in raws]
+    descs = [api.desc(sp.shape, sp.dtype, tensor_id=sp.seed) for sp in specs]
+    work = torch.empty(max(api.host_work_bytes(d, p) for d in descs), dtype=torch.uint8, device="cuda")
+    rc, tensors = api.plan_measure(descs, p, dense, work, repeats=5, t_recompute=[(10e-6 if i == 1 else 400e-6) for i in range(n)])
+    assert rc == api.FH_OK
+    for t, sp, d in zip(tensors, specs, descs):
+        st_o, _, total_o = fho.compress(synth.make(sp), fho.desc(sp.shape, sp.dtype, tensor_id=sp.seed), fho.params(bits=2))
+        assert st_o == fho.OK and t["bytes"] == sp.dense_bytes and t["packed_bytes"] == total_o
+        assert 1e-6 < t["t_compress"] < 1e-3 and 1e-6 < t["t_decompress"] < 1e-3
     ops = [dict(time=100e-6, inputs=[k - 1] if k else [], outputs=[k]) for k in range(n)]
     ops += [dict(time=200e-6, inputs=[k], outputs=[]) for k in reversed(range(n))]
     budget = int(0.6 * sum(t["bytes"] for t in tensors))
     rc, actions, events, rep = api.plan_generate(ops, tensors, budget)
     assert rc == api.FH_OK and rep.peak_bytes < budget
     assert api.FH_COMPRESS in actions and api.FH_EVICT in actions       # the hybrid: both techniques get used
-    items, raws, rest = [], [], []
-    for sp, act in zip(specs, actions):
-        raw = synth.make(sp)
-        raws.append(raw)
-        dense = to_dev(raw)
-        out = torch.zeros_like(dense)
+    items, rest = [], []
+    for sp, act, dn, dsc in zip(specs, actions, dense, descs):
+        out = torch.zeros_like(dn)
         rest.append(out)
-        items.append(api.SchedItem(api.desc(sp.shape, sp.dtype, tensor_id=sp.seed), act, dense, out))
+        items.append(api.SchedItem(dsc, act, dn, out))
     arena = torch.zeros(4 << 20, dtype=torch.uint8, device="cuda")
     srep = api.fh_run_schedule(items, p, arena)
     assert srep.status == api.FH_OK

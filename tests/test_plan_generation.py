@@ -64,6 +64,58 @@ def test_longer_freed_lifetime_wins():
     assert purged[0][1] == 0          # tensor 0 is read last in the backward pass
 
 
+def both(ops, tensors, budget):
+    """The oracle's plan, after checking that the library produces the same one."""
+    want = po.generate(ops, tensors, budget)
+    rc, actions, events, rep = api.plan_generate(ops, tensors, budget)
+    assert (actions, events, rep.peak_bytes, rep.n_over_budget) == (want[0], want[1], want[2], want[4])
+    assert abs(rep.overhead_seconds - want[3]) < 1e-12
+    return want
+
+
+def test_hand_case_skip_connection_locks_the_tensor_it_reads():
+    """Four forward ops (op k reads tensor k-1, writes tensor k; op 3 also reads tensor 0: a skip connection),
+    then backward ops 4..7 reading tensors 3, 2, 1, 0.  Every op 1 s, every tensor 100 B, budget 350.
+    Ops 0-2 fill the pool to 300.  Op 3 allocates tensor 3: 300 + 100 >= 350.  Tensors 2, 0 (inputs) and 3 are
+    locked, so tensor 1 is the only candidate -- without the skip connection it would have been tensor 0, whose
+    reader is furthest away.  Next reader of tensor 1 = op 6: FLT = 3 s;
+      MPS_compress = (100 - 25) * 3 / (0.5 + 0.5) = 225 > MPS_compute = 100 * 3 / 2 = 150  ->  compress.
+    Pool 300 - 75 + 100 = 325 (the peak).  Ops 4, 5 free tensors 3, 2 (pool 125); op 6 decompresses tensor 1
+    (125 + 100 < 350, no purge).  Overhead 0.5 + 0.5 = 1.0 s."""
+    ops = [dict(time=1.0, inputs=[], outputs=[0]), dict(time=1.0, inputs=[0], outputs=[1]),
+           dict(time=1.0, inputs=[1], outputs=[2]), dict(time=1.0, inputs=[2, 0], outputs=[3]),
+           dict(time=1.0, inputs=[3], outputs=[]), dict(time=1.0, inputs=[2], outputs=[]),
+           dict(time=1.0, inputs=[1], outputs=[]), dict(time=1.0, inputs=[0], outputs=[])]
+    tensors = [T(100, 25, 0.5, 0.5, 2.0)] * 4
+    actions, events, peak, overhead, over = both(ops, tensors, 350)
+    assert actions == [po.KEEP, po.COMPRESS, po.KEEP, po.KEEP]
+    assert events == [(3, 1, po.COMPRESS), (6, 1, po.KEEP)]
+    assert (peak, overhead, over) == (325, 1.0, 0)
+    # the same graph without the skip connection purges tensor 0 instead (FLT = 7 - 3 = 4 s, MPS 300)
+    ops[3] = dict(time=1.0, inputs=[2], outputs=[3])
+    actions, events, *_ = both(ops, tensors, 350)
+    assert actions == [po.COMPRESS, po.KEEP, po.KEEP, po.KEEP] and events[0] == (3, 0, po.COMPRESS)
+
+
+def test_hand_case_recovering_an_evicted_tensor_forces_another_purge():
+    """Ops: 0 writes t0; 1 reads t0 writes t1; 2 reads t1 writes t2; 3 reads t2 and t0, writes t3 (10 B);
+    4 reads t3 and t1.  t0, t1, t2 are 100 B; every op 1 s; budget 300.
+    Op 2 allocates t2: pool 200 + 100 >= 300; t1, t2 locked, candidate t0 (next reader op 3, FLT 1 s):
+      MPS_compute = 100 * 1 / 0.25 = 400 > MPS_compress = 75 * 1 / 1 = 75  ->  evict; pool 100 + 100 = 200.
+    Op 3 needs t0 back: 200 + 100 >= 300 while t2, t0, t3 are locked; candidate t1 (cannot be recomputed,
+    next reader op 4, FLT 1 s, MPS_compress 75) -> compressed: pool 200 - 75 = 125, then t0 is recomputed
+    (pool 225) and t3 allocated (235, the peak).  t2 and t0 die after op 3 (pool 35); op 4 decompresses t1
+    (35 + 100 < 300).  Overhead = recompute 0.25 + compress 0.5 + decompress 0.5 = 1.25 s."""
+    ops = [dict(time=1.0, inputs=[], outputs=[0]), dict(time=1.0, inputs=[0], outputs=[1]),
+           dict(time=1.0, inputs=[1], outputs=[2]), dict(time=1.0, inputs=[2, 0], outputs=[3]),
+           dict(time=1.0, inputs=[3, 1], outputs=[])]
+    tensors = [T(100, 25, 0.5, 0.5, 0.25), T(100, 25, 0.5, 0.5, -1.0), T(100, 25, 0.5, 0.5, 2.0), T(10, 10, 0.5, 0.5, 2.0)]
+    actions, events, peak, overhead, over = both(ops, tensors, 300)
+    assert actions == [po.EVICT, po.COMPRESS, po.KEEP, po.KEEP]
+    assert events == [(2, 0, po.EVICT), (3, 1, po.COMPRESS), (3, 0, po.KEEP), (4, 1, po.KEEP)]
+    assert (peak, overhead, over) == (235, 1.25, 0)
+
+
 def random_graph(rng, n):
     ops = chain(n, op_time=1.0)
     for op in ops:
