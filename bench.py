@@ -9,6 +9,11 @@ one (reverse order), salient_mode AUTO.  The headline workload is the ResNet-18-
 activations at batch 64 (17 fp32 tensors, 563.5 MiB dense).  `value` is dense GB/s: the dense bytes
 that went through compress plus those that came out of decompress, divided by the device time.
 
+Beside the headline the line carries `sweep` (the size sweep of configs[3]: single tensors of 64 MiB, 256 MiB and
+1 GiB, fp32 and bf16, compress and decompress timed separately over copies that do not fit the L2 cache),
+`schedule` (configs[4] through fh_run_schedule) and `parity_checked` (status words re-read after the timed
+region and one tensor's container per code width compared byte for byte with the CPU oracle).
+
 One JSON line goes to stdout (rank 0).  With N > 1 (launched by torchrun) every rank runs the
 same workload on its own GPU -- planes and tensors are independent, there is no exchange step --
 and the value is the sum of the dense bytes over the slowest rank's time.
@@ -32,9 +37,10 @@ sys.path.insert(0, ROOT)
 from paper_2510_11400_b200 import synth  # noqa: E402
 
 BITS = (2, 4, 8)
-# dram__bytes_read.sum + dram__bytes_write.sum per compress call (streaming + block-wise kernel), averaged over
-# the 17 tensors of the default workload at 2 bits; see profiles/compress_resnet18_b64_traffic.md
-NCU_DRAM_BYTES_PER_COMPRESS_CALL = 36165712
+# dram__bytes_read.sum + dram__bytes_write.sum per compress call (one kernel), averaged over the 51 compress calls
+# of a step of the default workload; see profiles/compress_resnet18_b64_traffic.md.  None: the kernels have
+# changed since the counters were taken.
+NCU_DRAM_BYTES_PER_COMPRESS_CALL = None
 METRIC = "compress+decompress throughput, dense activation bytes"
 UNIT = "GB/s"
 
@@ -224,6 +230,88 @@ def run_reference(args, specs, wl_desc):
 # our arm
 # ------------------------------------------------------------------------------------------------
 
+def size_sweep(api, peak, mibs=(64, 256, 1024), repeats=20):
+    """configs[3]: single tensors of 32x32 planes, ReLU(N(0,1)), 2 bits, three-sigma mode; compress and
+    decompress timed separately with CUDA events over back-to-back calls on copies that together exceed the L2
+    cache.  fraction = (dense + container bytes) / time / measured copy bandwidth."""
+    import ctypes as C
+    import torch
+    L = api.lib()
+    sp = int(torch.cuda.current_stream().cuda_stream)
+    out = {}
+    for dt, dname in ((synth.F32, "f32"), (synth.BF16, "bf16")):
+        for mib in mibs:
+            spec = synth.config4(mib, dt)[0]
+            raw = synth.make(spec)
+            base = torch.from_numpy(raw.view(np.int16) if raw.dtype == np.uint16 else raw).cuda()
+            d = api.desc(spec.shape, spec.dtype)
+            p = api.default_params(bits=2)
+            cap = api.compressed_bytes(d, p, 1)
+            ncopy = max(2, -(-(400 << 20) // spec.dense_bytes))
+            copies = [base] + [base.clone() for _ in range(ncopy - 1)]
+            packs = [torch.empty(cap, dtype=torch.uint8, device="cuda") for _ in range(ncopy)]
+            rest = torch.empty_like(base)
+            out2 = torch.zeros(2, dtype=torch.int64, device="cuda")
+            st = torch.zeros(1, dtype=torch.int64, device="cuda")
+            cargs = [(C.byref(d), C.byref(p), c.data_ptr(), k.data_ptr(), cap, out2.data_ptr(), sp) for c, k in zip(copies, packs)]
+            dargs = [(k.data_ptr(), cap, C.byref(d), rest.data_ptr(), st.data_ptr(), sp) for k in packs]
+            reps = -(-repeats // ncopy)
+            res = {}
+            for name, arglist, fn in (("compress", cargs, L.fh_compress), ("decompress", dargs, L.fh_decompress)):
+                for a in arglist * 2:       # warm-up
+                    assert fn(*a) == 0
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(reps):
+                    for a in arglist:
+                        assert fn(*a) == 0
+                e1.record()
+                torch.cuda.synchronize()
+                assert out2[1].item() == 0 and st.item() == 0
+                res[name] = e0.elapsed_time(e1) * 1e-3 / (reps * ncopy)
+            total = int(out2[0].item())
+            out[f"{mib}MiB_{dname}"] = {
+                "dense_bytes": spec.dense_bytes, "packed_bytes": total, "calls_timed": reps * ncopy,
+                "compress_gbs": spec.dense_bytes / res["compress"] / 1e9,
+                "decompress_gbs": spec.dense_bytes / res["decompress"] / 1e9,
+                "compress_frac": (spec.dense_bytes + total) / res["compress"] / 1e9 / peak,
+                "decompress_frac": (spec.dense_bytes + total) / res["decompress"] / 1e9 / peak}
+            del copies, packs, rest, base
+            torch.cuda.empty_cache()
+    return out
+
+
+def schedule_leg(api, mode, repeats=20):
+    """configs[4]: the 20 CIFAR-ResNet-shaped tensors at batch 128, every other one compressed, through
+    fh_run_schedule (forward-order compress, reverse-order decompress, one stream)."""
+    import torch
+    specs = synth.config5(128)
+    p = api.default_params(bits=2, salient_mode=mode)
+    items, need = [], 0
+    for i, s in enumerate(specs):
+        t = torch.from_numpy(synth.make(s)).cuda()
+        d = api.desc(s.shape, s.dtype, tensor_id=i)
+        items.append(api.SchedItem(d, api.FH_COMPRESS if s.compress else api.FH_KEEP, t, torch.empty_like(t)))
+        if s.compress:
+            need += (api.compressed_bytes(d, p, 1) + 255) & ~255
+    arena = torch.empty(need, dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        rep = api.fh_run_schedule(items, p, arena)
+        assert rep.status == api.FH_OK, rep.status
+    fwd = bwd = 0.0
+    for _ in range(repeats):
+        rep = api.fh_run_schedule(items, p, arena)
+        assert rep.status == api.FH_OK, rep.status
+        fwd += rep.ms_forward
+        bwd += rep.ms_backward
+    dense = int(rep.total_dense_bytes)
+    return {"tensors": len(specs), "compressed_tensors": sum(1 for s in specs if s.compress), "repeats": repeats,
+            "ms_forward": fwd / repeats, "ms_backward": bwd / repeats, "total_dense_bytes": dense,
+            "total_packed_bytes": int(rep.total_packed_bytes), "peak_packed_bytes": int(rep.peak_packed_bytes),
+            "compress_gbs": dense / (fwd / repeats) / 1e6, "decompress_gbs": dense / (bwd / repeats) / 1e6}
+
+
 def run_ours(args, specs, wl_desc):
     import torch
     import torch.distributed as dist
@@ -258,19 +346,29 @@ def run_ours(args, specs, wl_desc):
                             out2={b: torch.zeros(2, dtype=torch.int64, device=dev) for b in BITS},
                             st={b: torch.zeros(1, dtype=torch.int64, device=dev) for b in BITS}))
     dense_bytes = sum(s.dense_bytes for s in specs)
+    n_tensors = len(tensors)
     stream = torch.cuda.current_stream()
+
+    # argument tuples are marshalled once: the timed loop only makes the C calls
+    import ctypes as C
+    L = api.lib()
+    sp = int(stream.cuda_stream)
+    cargs = {b: [(C.byref(t["desc"]), C.byref(params[b]), t["dense"].data_ptr(), t["packed"].data_ptr(), t["cap"],
+                  t["out2"][b].data_ptr(), sp) for t in tensors] for b in BITS}
+    dargs = {b: [(t["packed"].data_ptr(), t["cap"], C.byref(t["desc"]), t["restored"].data_ptr(), t["st"][b].data_ptr(), sp)
+                 for t in reversed(tensors)] for b in BITS}
 
     def step(ev=None):
         for b in BITS:
             if ev is not None:
                 ev[b][0].record(stream)
-            for t in tensors:
-                rc = api.fh_compress(t["desc"], params[b], t["dense"], t["packed"], t["out2"][b], capacity=t["cap"])
+            for a in cargs[b]:
+                rc = L.fh_compress(*a)
                 assert rc == 0, rc
             if ev is not None:
                 ev[b][1].record(stream)
-            for t in reversed(tensors):
-                rc = api.fh_decompress(t["packed"], t["cap"], t["desc"], t["restored"], t["st"][b])
+            for a in dargs[b]:
+                rc = L.fh_decompress(*a)
                 assert rc == 0, rc
             if ev is not None:
                 ev[b][2].record(stream)
@@ -310,6 +408,35 @@ def run_ours(args, specs, wl_desc):
     t_comp = {b: sum(e[b][0].elapsed_time(e[b][1]) for e in evs) for b in BITS}
     t_dec = {b: sum(e[b][1].elapsed_time(e[b][2]) for e in evs) for b in BITS}
 
+    # ---- after the timed region: every status word again, and one tensor per code width against the oracle
+    for b in BITS:
+        for t in tensors:
+            total, st = t["out2"][b].tolist()
+            assert st == 0 and t["st"][b].item() == 0, f"device status after the timed region: {st}, {t['st'][b].item()}"
+    parity_checked = False
+    if rank == 0 and not args.no_cpu:
+        from oracle import fho
+        fho.set_threads(fho.max_threads())
+        k = min(len(tensors) - 1, 10)         # a tensor of small planes when the workload has one (mixed plane classes)
+        t = tensors[k]
+        raw = synth.make(t["spec"])
+        for b in BITS:
+            assert L.fh_compress(*cargs[b][k]) == 0
+            torch.cuda.synchronize()
+            total = int(t["out2"][b][0])
+            st_o, buf_o, total_o = fho.compress(raw, fho.desc(t["spec"].shape, t["spec"].dtype, tensor_id=k),
+                                                fho.params(bits=b, salient_mode=mode, rounding=args.rounding, seed=2510_11400))
+            assert st_o == 0 and total == total_o, (total, total_o)
+            assert np.array_equal(t["packed"][:total].cpu().numpy(), buf_o), "container differs from the oracle's"
+            assert L.fh_decompress(t["packed"].data_ptr(), t["cap"], C.byref(t["desc"]), t["restored"].data_ptr(),
+                                   t["st"][b].data_ptr(), sp) == 0
+            torch.cuda.synchronize()
+            got = t["restored"].cpu().numpy()
+            _, out_o = fho.decompress(buf_o, fho.desc(t["spec"].shape, t["spec"].dtype))
+            assert np.array_equal(got.view(np.uint16) if t["spec"].dtype == synth.BF16 else got.view(np.uint32),
+                                  out_o if t["spec"].dtype == synth.BF16 else out_o.view(np.uint32)), "restored values differ"
+        parity_checked = True
+
     # ---- end to end through the host-buffer entry points (pinned host memory on both sides)
     e2e = None
     if not args.no_e2e:
@@ -348,9 +475,16 @@ def run_ours(args, specs, wl_desc):
         e2e = {"value": whole_job_value(ksteps * dense_bytes * 2 * len(BITS), world, dt), "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": ksteps}
 
+    sweep = sched = None
+    if rank == 0 and world == 1 and args.workload == "resnet18_b64" and not args.no_sweep:
+        del tensors, cargs, dargs
+        torch.cuda.empty_cache()
+        sweep = size_sweep(api, peaks()[0])
+        sched = schedule_leg(api, mode)
+
     if rank == 0:
         peak, peak_kind = peaks()
-        n_comp = args.steps * len(BITS) * len(tensors)
+        n_comp = args.steps * len(BITS) * n_tensors
         alg_comp = args.steps * sum(dense_bytes + packed_bytes[b] for b in BITS)
         comp_s = sum(t_comp.values()) / 1e3
         achieved = alg_comp / comp_s / 1e9
@@ -365,15 +499,15 @@ def run_ours(args, specs, wl_desc):
             "config": {"workload": wl_desc + ("; every tensor compressed" if args.workload == "cifar_schedule" else ""),
                        "bits": list(BITS), "salient_mode": args.mode.upper(),
                        "rounding": "nearest-even" if args.rounding == 0 else "random (Philox-4x32-10)",
-                       "tensors": len(tensors), "dense_bytes_per_pass": dense_bytes,
+                       "tensors": n_tensors, "dense_bytes_per_pass": dense_bytes,
                        "packed_bytes": {str(b): packed_bytes[b] for b in BITS},
                        "l2": "inputs larger than L2: every pass streams the whole dense set",
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "compress_gbs": {str(b): args.steps * dense_bytes / t_comp[b] / 1e6 for b in BITS},
             "decompress_gbs": {str(b): args.steps * dense_bytes / t_dec[b] / 1e6 for b in BITS},
             "roofline": {"bound": "hbm",
-                         "kernel": "compress call = streaming kernel (compress_warp / compress_cta / compress_generic) "
-                                   "+ blockwise_kernel; averaged over every compress call of the timed region",
+                         "kernel": "compress call = one kernel (compress_warp / compress_cta / compress_generic by plane "
+                                   "size); averaged over every compress call of the timed region",
                          "achieved": achieved, "peak": peak,
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
                          "launches": n_comp, "avg_launch_us": comp_s / n_comp * 1e6,
@@ -381,8 +515,12 @@ def run_ours(args, specs, wl_desc):
                          "frac_of_nominal_8000": achieved / 8000.0,
                          "decompress_achieved": args.steps * sum(dense_bytes + packed_bytes[b] for b in BITS)
                          / (sum(t_dec.values()) / 1e3) / 1e9},
-            "clocks": clocks, "gpu_launches": int(launches),
+            "clocks": clocks, "gpu_launches": int(launches), "parity_checked": parity_checked,
         }
+        if sweep is not None:
+            line["sweep"] = sweep
+        if sched is not None:
+            line["schedule"] = sched
         if e2e is not None:
             line["e2e"] = e2e
         if cpu is not None:
@@ -465,6 +603,7 @@ def main():
                     help="run the workload through fh_run_schedule (forward-order compress, reverse-order decompress)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the size sweep and the schedule leg of the default workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     specs, wl_desc = workload_specs(args.workload)
