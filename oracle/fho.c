@@ -71,6 +71,8 @@ typedef struct {
   int32_t dense_bits;
   int32_t rounding;
   uint64_t seed;
+  int32_t entropy; /* 0: fixed 8-bit residual codes; 1: Huffman stage on the dense-block codes */
+  int32_t reserved;
 } fho_params;
 
 static int g_threads = 1;
@@ -116,6 +118,7 @@ static int check_args(const fho_desc* d, const fho_params* p) {
   if (p->block != 8) return FHO_ERR_UNSUPPORTED;
   if (p->dense_bits != 8) return FHO_ERR_UNSUPPORTED;
   if (p->rounding != 0 && p->rounding != 1) return FHO_ERR_UNSUPPORTED;
+  if (p->entropy != 0 && p->entropy != 1) return FHO_ERR_UNSUPPORTED;
   if (!(p->eps >= 1e-30f) || !(p->eps <= 1e30f)) return FHO_ERR_ARG; /* keeps 2*eps and 1/(2*eps) finite */
   return FHO_OK;
 }
@@ -381,6 +384,181 @@ static uint16_t get_u16(const uint8_t* p) {
   return v;
 }
 
+/* ------------------------------------------------------------------------------------------
+ * Huffman stage (Section 4.4.1: "a Huffman tree is constructed from the quantization array for
+ * encoding"; decompression "involves Huffman decoding").  The quantization array is the array of
+ * residual code bytes of an outlier-rich plane's dense blocks (64 per block; 0 marks a verbatim value).
+ * The paper gives no alphabet, scope, tie-break or stream format; here:
+ *   scope      one code per plane, built from that plane's own code bytes (a plane's payload then
+ *              depends on nothing but the plane, like everything else in the container)
+ *   tree       the classical construction: the two nodes of least weight are merged until one is left.
+ *              Nodes are ordered by (weight, id) with id = symbol for a leaf and 256 + order of creation
+ *              for a merged node; symbols that do not occur get no code; a single symbol gets length 1
+ *   code       canonical: symbols sorted by (length, symbol) take consecutive code values, first code of
+ *              a length = (last code of the previous length + 1) << (difference of the lengths)
+ *   stream     every dense block's 64 symbols form a chunk of its own that starts on a byte boundary
+ *              (chunks decode independently); a code's bits go most significant first, bytes fill from bit 7
+ *   section    u8 len(symbol 0) | u8 smin | u8 smax | u8 0 | u8 len(s) for s = smin..smax (pad to 4)
+ *              | u8 bytes of chunk b, b = 0..n_dense-1 (pad to 4) | the chunks, concatenated (pad to 4)
+ *              where [smin, smax] is the range of symbols 1..255 that occur (1, 1 if none does)
+ * The section replaces the plain 64 * n_dense code bytes only if it is smaller; word 3 of the payload
+ * header then holds the section's size in bytes, and 0 otherwise.  Code lengths stay below 25: a plane has
+ * fewer than 2^17 code bytes and a Huffman code of depth d needs at least Fibonacci(d + 2) of them; a chunk
+ * therefore has at most 64 * 24 / 8 = 192 bytes.
+ * ------------------------------------------------------------------------------------------ */
+void fho_huffman_lengths(const uint32_t hist[256], uint8_t len[256]) {
+  /* leaves sorted by (weight, symbol); merged nodes are born in non-decreasing weight order, so two queues
+   * (leaves, merged nodes) always have the least node at one of their heads */
+  int leaf[256], n = 0;
+  for (int sym = 0; sym < 256; ++sym) {
+    len[sym] = 0;
+    if (hist[sym]) leaf[n++] = sym;
+  }
+  if (n == 0) return;
+  if (n == 1) {
+    len[leaf[0]] = 1;
+    return;
+  }
+  for (int i = 1; i < n; ++i) { /* insertion sort: stable, so equal weights stay in symbol order */
+    int v = leaf[i], j = i;
+    while (j > 0 && hist[leaf[j - 1]] > hist[v]) {
+      leaf[j] = leaf[j - 1];
+      --j;
+    }
+    leaf[j] = v;
+  }
+  uint64_t w[512];   /* weight of node id: ids 0..255 leaves (by symbol), 256.. merged nodes */
+  int parent[512];
+  for (int sym = 0; sym < 256; ++sym) w[sym] = hist[sym];
+  int li = 0, mi = 256, mn = 256; /* head of the leaf queue, head and end of the merged-node queue */
+  while ((n - li) + (mn - mi) > 1) {
+    int pick[2];
+    for (int k = 0; k < 2; ++k) {
+      int take_leaf;
+      if (li >= n) take_leaf = 0;
+      else if (mi >= mn) take_leaf = 1;
+      else take_leaf = w[leaf[li]] <= w[mi]; /* equal weights: the leaf has the smaller id */
+      pick[k] = take_leaf ? leaf[li++] : mi++;
+    }
+    w[mn] = w[pick[0]] + w[pick[1]];
+    parent[pick[0]] = parent[pick[1]] = mn;
+    ++mn;
+  }
+  int root = mn - 1;
+  for (int i = 0; i < n; ++i) {
+    int d = 0;
+    for (int v = leaf[i]; v != root; v = parent[v]) ++d;
+    len[leaf[i]] = (uint8_t)d;
+  }
+}
+
+/* Canonical code values (right-aligned in `code`) from the lengths alone. */
+void fho_canonical_codes(const uint8_t len[256], uint32_t code[256]) {
+  uint32_t next = 0;
+  int prev = 0;
+  for (int l = 1; l <= 32; ++l)
+    for (int sym = 0; sym < 256; ++sym)
+      if (len[sym] == l) {
+        next <<= (l - prev);
+        prev = l;
+        code[sym] = next++;
+      }
+}
+
+/* The entropy-coded section for `n_dense` blocks of 64 code bytes; returns its size (a multiple of 4). */
+static size_t huffman_section(const uint8_t* codes, uint32_t n_dense, uint8_t** out) {
+  uint32_t hist[256] = {0};
+  for (size_t i = 0; i < (size_t)n_dense * 64; ++i) ++hist[codes[i]];
+  uint8_t len[256];
+  uint32_t code[256] = {0};
+  fho_huffman_lengths(hist, len);
+  for (int sym = 0; sym < 256; ++sym)
+    if (len[sym] > 24) { /* cannot happen for planes this library accepts (see above); then the stage is not used */
+      *out = NULL;
+      return (size_t)-1;
+    }
+  fho_canonical_codes(len, code);
+  int smin = 1, smax = 1, any = 0;
+  for (int sym = 1; sym < 256; ++sym)
+    if (len[sym]) {
+      if (!any) smin = sym;
+      smax = sym;
+      any = 1;
+    }
+  size_t nlens = (size_t)(smax - smin + 1);
+  size_t head = 4 + a4(nlens) + a4(n_dense);
+  uint8_t* buf = (uint8_t*)calloc(head + (size_t)n_dense * 64 * 4 + 8, 1);
+  buf[0] = len[0];
+  buf[1] = (uint8_t)smin;
+  buf[2] = (uint8_t)smax;
+  for (int sym = smin; sym <= smax; ++sym) buf[4 + (sym - smin)] = len[sym];
+  uint8_t* chunk_bytes = buf + 4 + a4(nlens);
+  size_t pos = head; /* byte position of the next chunk */
+  for (uint32_t b = 0; b < n_dense; ++b) {
+    size_t bit = 0; /* bits written into this chunk */
+    for (int i = 0; i < 64; ++i) {
+      uint8_t sym = codes[(size_t)b * 64 + i];
+      for (int k = len[sym] - 1; k >= 0; --k) { /* most significant bit first */
+        if ((code[sym] >> k) & 1u) buf[pos + bit / 8] |= (uint8_t)(0x80u >> (bit % 8));
+        ++bit;
+      }
+    }
+    size_t nbytes = (bit + 7) / 8;
+    chunk_bytes[b] = (uint8_t)nbytes;
+    pos += nbytes;
+  }
+  *out = buf;
+  return a4(pos);
+}
+
+/* Decodes the section at `sec` (at most `avail` readable bytes) into n_dense * 64 code bytes; returns the
+ * section's size, or 0 if it is inconsistent. */
+static size_t huffman_decode_section(const uint8_t* sec, size_t avail, uint32_t n_dense, uint8_t* codes) {
+  if (avail < 4) return 0;
+  int smin = sec[1], smax = sec[2];
+  if (smin < 1 || smax < smin) return 0;
+  size_t nlens = (size_t)(smax - smin + 1);
+  size_t head = 4 + a4(nlens) + a4(n_dense);
+  if (avail < head) return 0;
+  uint8_t len[256] = {0};
+  len[0] = sec[0];
+  for (int sym = smin; sym <= smax; ++sym) len[sym] = sec[4 + (sym - smin)];
+  uint64_t kraft = 0; /* in units of 2^-32 */
+  int nsym = 0;
+  for (int sym = 0; sym < 256; ++sym) {
+    if (len[sym] > 32) return 0;
+    if (len[sym]) {
+      kraft += 1ull << (32 - len[sym]);
+      ++nsym;
+    }
+  }
+  if (nsym == 0 || kraft > (1ull << 32) || (nsym > 1 && kraft != (1ull << 32))) return 0;
+  uint32_t code[256] = {0};
+  fho_canonical_codes(len, code);
+  const uint8_t* chunk_bytes = sec + 4 + a4(nlens);
+  size_t pos = head;
+  for (uint32_t b = 0; b < n_dense; ++b) {
+    size_t nbytes = chunk_bytes[b];
+    if (pos + nbytes > avail) return 0;
+    size_t bit = 0;
+    for (int i = 0; i < 64; ++i) {
+      uint32_t acc = 0;
+      int l = 0, found = -1;
+      while (found < 0) {
+        if (bit >= nbytes * 8 || l >= 32) return 0;
+        acc = (acc << 1) | ((sec[pos + bit / 8] >> (7 - bit % 8)) & 1u);
+        ++bit;
+        ++l;
+        for (int sym = 0; sym < 256; ++sym)
+          if (len[sym] == l && code[sym] == acc) found = sym;
+      }
+      codes[(size_t)b * 64 + i] = (uint8_t)found;
+    }
+    pos += nbytes;
+  }
+  return a4(pos);
+}
+
 typedef struct {
   uint32_t cls;
   uint32_t n_out;
@@ -474,14 +652,25 @@ static size_t encode_salient(const float* x, const uint8_t* raw, int dtype, int 
     ++di;
   }
   size_t nbm = ((size_t)nblk + 31) / 32;
-  size_t size = 16 + 4 * nbm + 4 * ((size_t)H + 1) + a4(2 * (size_t)nnz_s) + a4(e * nnz_s) +
-                64 * (size_t)n_dense + a4(e * n_out_d);
+  /* the dense blocks' code bytes as they are, or through the Huffman stage when that is smaller */
+  uint8_t* section = NULL;
+  size_t dense_bytes = 64 * (size_t)n_dense;
+  int coded = 0;
+  if (p->entropy == 1 && n_dense > 0) {
+    size_t sz = huffman_section(codes, n_dense, &section);
+    if (sz < dense_bytes) {
+      dense_bytes = sz;
+      coded = 1;
+    }
+  }
+  size_t size = 16 + 4 * nbm + 4 * ((size_t)H + 1) + a4(2 * (size_t)nnz_s) + a4(e * nnz_s) + dense_bytes +
+                a4(e * n_out_d);
   uint8_t* buf = (uint8_t*)calloc(a16(size), 1);
   uint8_t* q = buf;
   put_u32(q, nnz_s);
   put_u32(q + 4, n_dense);
   put_u32(q + 8, n_out_d);
-  put_u32(q + 12, 0);
+  put_u32(q + 12, coded ? (uint32_t)dense_bytes : 0u); /* size of the Huffman-coded section, 0: plain code bytes */
   q += 16;
   for (int blk = 0; blk < nblk; ++blk)
     if (dense[blk]) {
@@ -502,9 +691,10 @@ static size_t encode_salient(const float* x, const uint8_t* raw, int dtype, int 
         ++t;
       }
   q = valp + a4(e * nnz_s);
-  memcpy(q, codes, (size_t)n_dense * 64);
-  q += (size_t)n_dense * 64;
+  memcpy(q, coded ? section : codes, dense_bytes);
+  q += dense_bytes;
   memcpy(q, outl, (size_t)n_out_d * e);
+  free(section);
   free(dense);
   free(row_ptr);
   free(codes);
@@ -675,7 +865,7 @@ int fho_compress(const fho_desc* d, const fho_params* p, const void* src, void* 
     uint8_t* o = (uint8_t*)dst;
     memset(o, 0, 64);
     put_u32(o + 0, 0x31434846u); /* 'F','H','C','1' */
-    put_u16(o + 4, 1);
+    put_u16(o + 4, (uint16_t)(p->entropy == 1 ? 2 : 1)); /* version 2: payloads may carry Huffman-coded sections */
     o[6] = (uint8_t)d->dtype;
     o[7] = (uint8_t)p->bits;
     put_u32(o + 8, (uint32_t)d->n);
@@ -737,10 +927,10 @@ static void store_elem(uint8_t* dst, int dtype, size_t i, float v) {
 }
 
 static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, float eps, uint32_t nnz_s,
-                                  uint32_t n_dense, uint32_t n_out_d, uint8_t* out);
+                                  uint32_t n_dense, uint32_t n_out_d, uint32_t coded_bytes, uint8_t* out);
 
 static int decode_plane(const uint8_t* src, size_t src_bytes, size_t pl, size_t P, int dtype, int H,
-                        int W, int bits, float eps, uint8_t* out) {
+                        int W, int bits, float eps, int version, uint8_t* out) {
   size_t hw = (size_t)H * W, e = esize(dtype);
   const uint8_t* te = src + 64 + 16 * pl;
   size_t off = (size_t)get_u32(te) * 16;
@@ -767,7 +957,7 @@ static int decode_plane(const uint8_t* src, size_t src_bytes, size_t pl, size_t 
   const int B = 8;
   int nby = (H + B - 1) / B, nbx = (W + B - 1) / B, nblk = nby * nbx;
   size_t nbm = ((size_t)nblk + 31) / 32;
-  uint32_t nnz_s = 0, n_dense = 0, n_out_d = 0;
+  uint32_t nnz_s = 0, n_dense = 0, n_out_d = 0, coded_bytes = 0;
   size_t size;
   if (cls == CLS_RAW) {
     size = e * hw;
@@ -775,9 +965,11 @@ static int decode_plane(const uint8_t* src, size_t src_bytes, size_t pl, size_t 
     nnz_s = get_u32(slot);
     n_dense = get_u32(slot + 4);
     n_out_d = get_u32(slot + 8);
+    coded_bytes = get_u32(slot + 12);
     if (nnz_s > hw || n_dense > (uint32_t)nblk || n_out_d > hw) return FHO_ERR_CORRUPT;
+    if (coded_bytes && (version != 2 || coded_bytes % 4 != 0 || coded_bytes >= 64 * (size_t)n_dense)) return FHO_ERR_CORRUPT;
     size = 16 + 4 * nbm + 4 * ((size_t)H + 1) + a4(2 * (size_t)nnz_s) + a4(e * nnz_s) +
-           64 * (size_t)n_dense + a4(e * n_out_d);
+           (coded_bytes ? coded_bytes : 64 * (size_t)n_dense) + a4(e * n_out_d);
   }
   /* the payload runs through the slot and continues at `off` in the overflow region */
   uint8_t* pay = (uint8_t*)calloc(a16(size) + 16, 1);
@@ -794,13 +986,13 @@ static int decode_plane(const uint8_t* src, size_t src_bytes, size_t pl, size_t 
     free(pay);
     return FHO_OK;
   }
-  int rc = decode_salient_payload(pay, dtype, H, W, eps, nnz_s, n_dense, n_out_d, out);
+  int rc = decode_salient_payload(pay, dtype, H, W, eps, nnz_s, n_dense, n_out_d, coded_bytes, out);
   free(pay);
   return rc;
 }
 
 static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, float eps, uint32_t nnz_s,
-                                  uint32_t n_dense, uint32_t n_out_d, uint8_t* out) {
+                                  uint32_t n_dense, uint32_t n_out_d, uint32_t coded_bytes, uint8_t* out) {
   const int B = 8;
   size_t hw = (size_t)H * W, e = esize(dtype);
   int nby = (H + B - 1) / B, nbx = (W + B - 1) / B, nblk = nby * nbx;
@@ -810,14 +1002,23 @@ static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, f
   const uint8_t* colp = rp + 4 * ((size_t)H + 1);
   const uint8_t* valp = colp + a4(2 * (size_t)nnz_s);
   const uint8_t* codes = valp + a4(e * nnz_s);
-  const uint8_t* outl = codes + 64 * (size_t)n_dense;
+  const uint8_t* outl = codes + (coded_bytes ? coded_bytes : 64 * (size_t)n_dense);
+  uint8_t* plain = NULL;
+  if (coded_bytes) { /* Huffman decoding first (Section 4.4.1, "Decompression involves Huffman decoding") */
+    plain = (uint8_t*)malloc((size_t)n_dense * 64 + 1);
+    if (huffman_decode_section(codes, coded_bytes, n_dense, plain) != coded_bytes) {
+      free(plain);
+      return FHO_ERR_CORRUPT;
+    }
+    codes = plain;
+  }
   memset(out, 0, e * hw);
   for (int y = 0; y < H; ++y) {
     uint32_t a = get_u32(rp + 4 * y), b = get_u32(rp + 4 * (y + 1));
-    if (a > b || b > nnz_s) return FHO_ERR_CORRUPT;
+    if (a > b || b > nnz_s) { free(plain); return FHO_ERR_CORRUPT; }
     for (uint32_t t = a; t < b; ++t) {
       uint32_t col = get_u16(colp + 2 * (size_t)t);
-      if ((int)col >= W) return FHO_ERR_CORRUPT;
+      if ((int)col >= W) { free(plain); return FHO_ERR_CORRUPT; }
       memcpy(out + ((size_t)y * W + col) * e, valp + e * t, e);
     }
   }
@@ -826,7 +1027,7 @@ static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, f
   uint32_t di = 0, oi = 0;
   for (int blk = 0; blk < nblk; ++blk) {
     if (!((get_u32(bm + 4 * (blk / 32)) >> (blk % 32)) & 1u)) continue;
-    if (di >= n_dense) return FHO_ERR_CORRUPT;
+    if (di >= n_dense) { free(plain); return FHO_ERR_CORRUPT; }
     int by = blk / nbx, bx = blk % nbx;
     int64_t k[8][8];
     for (int i = 0; i < B; ++i)
@@ -843,7 +1044,7 @@ static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, f
         }
         size_t idx = (size_t)y * W + xx;
         if (code == 0) {
-          if (oi >= n_out_d) return FHO_ERR_CORRUPT;
+          if (oi >= n_out_d) { free(plain); return FHO_ERR_CORRUPT; }
           memcpy(out + idx * e, outl + (size_t)oi * e, e);
           float v;
           if (dtype == FHO_F32)
@@ -861,6 +1062,7 @@ static int decode_salient_payload(const uint8_t* pay, int dtype, int H, int W, f
       }
     ++di;
   }
+  free(plain);
   return FHO_OK;
 }
 
@@ -868,7 +1070,8 @@ int fho_decompress(const void* src, size_t src_bytes, const fho_desc* expect, vo
   if (!src || !dst || !expect) return FHO_ERR_ARG;
   const uint8_t* s = (const uint8_t*)src;
   if (src_bytes < 64) return FHO_ERR_CORRUPT;
-  if (get_u32(s) != 0x31434846u || get_u16(s + 4) != 1) return FHO_ERR_CORRUPT;
+  if (get_u32(s) != 0x31434846u || (get_u16(s + 4) != 1 && get_u16(s + 4) != 2)) return FHO_ERR_CORRUPT;
+  int version = get_u16(s + 4);
   int dtype = s[6], bits = s[7];
   uint32_t N = get_u32(s + 8), C = get_u32(s + 12), H = get_u32(s + 16), W = get_u32(s + 20);
   if ((int)N != expect->n || (int)C != expect->c || (int)H != expect->h || (int)W != expect->w ||
@@ -887,7 +1090,7 @@ int fho_decompress(const void* src, size_t src_bytes, const fho_desc* expect, vo
 #pragma omp parallel for schedule(dynamic, 8) num_threads(g_threads)
 #endif
   for (int64_t pl = 0; pl < (int64_t)P; ++pl) {
-    int r = decode_plane(s, (size_t)tb, (size_t)pl, P, dtype, (int)H, (int)W, bits, eps,
+    int r = decode_plane(s, (size_t)tb, (size_t)pl, P, dtype, (int)H, (int)W, bits, eps, version,
                          (uint8_t*)dst + (size_t)pl * hw * e);
     if (r != FHO_OK) {
 #ifdef _OPENMP

@@ -31,13 +31,13 @@ class Params(C.Structure):
     _fields_ = [("bits", C.c_int32), ("salient_mode", C.c_int32), ("rho_num", C.c_int32),
                 ("rho_den", C.c_int32), ("block", C.c_int32), ("tau_num", C.c_int32),
                 ("tau_den", C.c_int32), ("eps", C.c_float), ("dense_bits", C.c_int32),
-                ("rounding", C.c_int32), ("seed", C.c_uint64)]
+                ("rounding", C.c_int32), ("seed", C.c_uint64), ("entropy", C.c_int32), ("reserved", C.c_int32)]
 
 
 def params(bits=2, salient_mode=AUTO, rho=(1, 32), block=8, tau=(1, 4), eps=0.0625, dense_bits=8,
-           rounding=0, seed=0) -> Params:
+           rounding=0, seed=0, entropy=0) -> Params:
     return Params(bits, salient_mode, rho[0], rho[1], block, tau[0], tau[1], eps, dense_bits,
-                  rounding, seed)
+                  rounding, seed, entropy, 0)
 
 
 def desc(shape, dtype=F32, tensor_id=0) -> Desc:
@@ -88,6 +88,10 @@ def lib():
         L.fho_philox4x32_10.argtypes = [C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)]
         L.fho_quant_code_random.restype = C.c_uint32
         L.fho_quant_code_random.argtypes = [C.c_float, C.c_float, C.c_float, C.c_int, C.c_uint32]
+        L.fho_huffman_lengths.restype = None
+        L.fho_huffman_lengths.argtypes = [C.POINTER(C.c_uint32), C.POINTER(C.c_uint8)]
+        L.fho_canonical_codes.restype = None
+        L.fho_canonical_codes.argtypes = [C.POINTER(C.c_uint8), C.POINTER(C.c_uint32)]
         L.fho_set_threads.argtypes = [C.c_int]
         L.fho_max_threads.restype = C.c_int
         L.fho_get_threads.restype = C.c_int
@@ -178,6 +182,22 @@ def philox4x32_10(ctr, key):
 
 def quant_code_random(x: float, lo: float, inv: float, bits: int, word: int) -> int:
     return int(lib().fho_quant_code_random(x, lo, inv, bits, word))
+
+
+def huffman_lengths(hist):
+    """Code lengths (256 uint8) of the Huffman code of a 256-bin histogram."""
+    h = (C.c_uint32 * 256)(*[int(v) for v in hist])
+    out = (C.c_uint8 * 256)()
+    lib().fho_huffman_lengths(h, out)
+    return [int(v) for v in out]
+
+
+def canonical_codes(lengths):
+    """Canonical code values of a list of 256 code lengths (0 where the length is 0)."""
+    l = (C.c_uint8 * 256)(*[int(v) for v in lengths])
+    out = (C.c_uint32 * 256)()
+    lib().fho_canonical_codes(l, out)
+    return [int(v) for v in out]
 
 
 def dequant(q: int, lo: float, scale: float) -> float:
