@@ -31,7 +31,7 @@
  *     FH_ERR_CUDA.
  *
  * Container (little-endian; a layout of this library, the paper gives none)
- *   [0,64)   header: u32 magic "FHC1" | u16 version=1 | u8 dtype | u8 bits | u32 N | u32 C | u32 H |
+ *   [0,64)   header: u32 magic "FHC1" | u16 version (1; 2 with entropy = 1) | u8 dtype | u8 bits | u32 N | u32 C | u32 H |
  *            u32 W | u8 block | u8 dense_bits | u8 rounding | u8 salient_mode | u16 rho_num |
  *            u16 rho_den | u16 tau_num | u16 tau_den | f32 eps | u32 n_salient | u32 n_raw |
  *            u64 tensor_id | u64 total_bytes
@@ -47,10 +47,17 @@
  *   offsets, so normal planes are written and read without knowing any other plane's size.
  *     normal : ceil(HW*bits/32) u32 words, element i in bits [(i*bits)%32, +bits) of word i*bits/32
  *     raw    : HW elements verbatim
- *     salient: u32 nnz_s | u32 n_dense | u32 n_out_d | u32 0 | block bitmap ceil(nblk/32) u32
+ *     salient: u32 nnz_s | u32 n_dense | u32 n_out_d | u32 coded | block bitmap ceil(nblk/32) u32
  *              (bit = 1: dense; blocks in raster order) | row_ptr (H+1) u32 | col nnz_s u16 (pad 4) |
- *              val nnz_s elements (pad 4) | codes n_dense*64 u8 | verbatim values n_out_d elements
- *              (pad 4)
+ *              val nnz_s elements (pad 4) | codes n_dense*64 u8, or, when coded != 0 (version 2), the
+ *              Huffman-coded section of `coded` bytes | verbatim values n_out_d elements (pad 4)
+ *     Huffman-coded section (Section 4.4.1; one code per plane from the plane's own code bytes, used only when
+ *              smaller than the plain codes): u8 len(symbol 0) | u8 smin | u8 smax | u8 0 | u8 len(s),
+ *              s = smin..smax (pad 4) | u8 bytes of chunk b, b = 0..n_dense-1 (pad 4) | chunks (pad 4);
+ *              a chunk holds the 64 symbols of one dense block, starts on a byte boundary, code bits most
+ *              significant first; codes are canonical (by length, then symbol) from Huffman lengths whose
+ *              ties are settled by (weight, id), id = symbol for a leaf, 256 + order of creation for a
+ *              merged node
  */
 #ifndef FH_H_
 #define FH_H_
@@ -109,6 +116,9 @@ typedef struct {
   int32_t rounding;         /* 0 = round half to even; 1 = random rounding of normal planes
                                (see fh_compress)                                           [0]     */
   uint64_t seed;            /* key of the random draws (rounding = 1)                      [0]     */
+  int32_t entropy;          /* 1 = Huffman stage on the dense-block residual codes (see
+                               fh_compress); container version 2                           [0]     */
+  int32_t reserved;         /* 0                                                                   */
 } fh_params;
 
 typedef enum { FH_KEEP = 0, FH_COMPRESS = 1, FH_EVICT = 2 } fh_action;
@@ -170,6 +180,11 @@ size_t fh_compressed_bytes(const fh_tensor_desc* desc, const fh_params* params, 
  * thus depends on (seed, tensor id, element position) only and results are reproducible.  Dense-block codes
  * keep round-to-nearest (their error bound needs it).  This mode runs on the general-purpose kernel and is
  * slower than rounding = 0.
+ *
+ * entropy = 1 (Section 4.4.1: "a Huffman tree is constructed from the quantization array for encoding"): the
+ * residual code bytes of an outlier-rich plane's dense blocks are Huffman-coded, one code per plane (see the
+ * container description); the stage is lossless and is skipped for a plane it would not shrink.  The container
+ * carries version 2.  This mode runs on the general-purpose kernel and is not tuned.
  */
 int fh_compress(const fh_tensor_desc* desc, const fh_params* params, const void* d_src, void* d_dst,
                 size_t dst_capacity, uint64_t* d_out2, void* stream);

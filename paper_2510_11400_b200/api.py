@@ -43,7 +43,7 @@ class fh_params(C.Structure):
     _fields_ = [("bits", C.c_int32), ("salient_mode", C.c_int32), ("rho_num", C.c_int32),
                 ("rho_den", C.c_int32), ("block", C.c_int32), ("tau_num", C.c_int32),
                 ("tau_den", C.c_int32), ("eps", C.c_float), ("dense_bits", C.c_int32),
-                ("rounding", C.c_int32), ("seed", C.c_uint64)]
+                ("rounding", C.c_int32), ("seed", C.c_uint64), ("entropy", C.c_int32), ("reserved", C.c_int32)]
 
 
 class fh_sched_entry(C.Structure):

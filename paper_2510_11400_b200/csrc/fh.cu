@@ -48,6 +48,7 @@ int check_params(const fh_params* p) {
   if (p->rho_num < 0 || p->rho_den < 1 || p->rho_num > 65535 || p->rho_den > 65535) return FH_ERR_ARG;
   if (p->tau_num < 0 || p->tau_den < 1 || p->tau_num > 65535 || p->tau_den > 65535) return FH_ERR_ARG;
   if (p->block != 8 || p->dense_bits != 8 || (p->rounding != 0 && p->rounding != 1)) return FH_ERR_UNSUPPORTED;
+  if (p->entropy != 0 && p->entropy != 1) return FH_ERR_UNSUPPORTED;
   if (!(p->eps >= 1e-30f) || !(p->eps <= 1e30f)) return FH_ERR_ARG;
   return FH_OK;
 }
@@ -93,6 +94,7 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   pl.bits = p ? p->bits : 2;
   pl.mode = p ? p->salient_mode : 0;
   pl.rounding = p ? p->rounding : 0;
+  pl.entropy = p ? p->entropy : 0;
   pl.seed = p ? p->seed : 0;
   pl.rho_num = p ? p->rho_num : 1;
   pl.rho_den = p ? p->rho_den : 32;
@@ -111,7 +113,10 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   const long double worst = 64.0L + (long double)pl.P * (16.0L + (long double)A16(pl.plane_bytes));
   if (worst / 16.0L >= 4294967295.0L) return FH_ERR_UNSUPPORTED;
   if (pl.P > 0x7FFFFFFFull) return FH_ERR_UNSUPPORTED;
-  const size_t sal_words = compress ? (size_t)(pl.H + 1 + 3 * pl.nblk) : (size_t)pl.nblk;
+  // measuring scratch of the block-wise path: row pointers and three words per block; with the Huffman stage two
+  // more words per block and the encoder's tables.  Decompress: two words per block and the decoder's tables.
+  const size_t sal_words = compress ? (size_t)(pl.H + 1 + 3 * pl.nblk) + (pl.entropy ? 2 * (size_t)pl.nblk + sizeof(fh::HufEncode) / 4 + 4 : 0)
+                                    : 2 * (size_t)pl.nblk + sizeof(fh::HufDecode) / 4 + 4;
   pl.sal_words = (uint32_t)sal_words;
   const uint32_t sal_bytes = (uint32_t)A16(4 * sal_words + 16);  // one measuring area of the block-wise path
   const bool blockwise = compress && pl.mode != FH_SALIENT_OFF;
@@ -119,10 +124,10 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   Variant v;
   // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
   const bool whole16 = pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0;
-  // (random rounding runs on the generic kernel)
+  // (random rounding and the Huffman stage run on the generic kernel)
   // (a warp-team kernel keeps one measuring area per warp: planes whose area is large -- very tall, narrow
   // ones -- go to the general-purpose kernel)
-  if (compress && pl.rounding == 0 && ((pl.groups <= 256 && (!blockwise || sal_bytes <= 1024)) || (pl.groups > 256 && whole16))) {
+  if (compress && pl.rounding == 0 && pl.entropy == 0 && ((pl.groups <= 256 && (!blockwise || sal_bytes <= 1024)) || (pl.groups > 256 && whole16))) {
     v.fast = true;
     if (pl.groups <= 256) {
       uint32_t t = pow2_ceil((pl.groups + 7) / 8);
@@ -163,7 +168,8 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
     uint32_t t = pow2_ceil((pl.groups + 7) / 8);
     pl.team = t > 32 ? 32 : t;
     const uint32_t nteams = fh::kThreads / pl.team;
-    pl.sm_total = nteams * 4 * pl.nblk + 16;
+    pl.sal_stride = sal_bytes;
+    pl.sm_total = nteams * sal_bytes + 16;
     if (pl.sm_total > kSmemLimit) return FH_ERR_UNSUPPORTED;
     pl.ppt = nteams;
     {
@@ -508,8 +514,10 @@ int launch_decompress_small(const Plan& pl0, const fh::DecompressArgs& a, cudaSt
   if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
   pl.stage_bytes = (uint32_t)((pl.ppt * pl.plane_bytes + 127) & ~(uint64_t)127);
   pl.ntiles = (uint32_t)((pl.P + pl.ppt - 1) / pl.ppt);
-  // two tile buffers, then per warp: scratch for a small plane's payload, or the block-wise scratch of a larger one
-  pl.sm_total = 2u * pl.stage_bytes + (uint32_t)fh::kWarps * (uint32_t)(A16(pl.plane_bytes) + 16 + 4u * pl.nblk);
+  // two tile buffers, then per warp: scratch for a small plane's payload, or the general path's scratch
+  const uint32_t pay = (uint32_t)A16(pl.plane_bytes) + 16u;
+  if (pl.sal_stride < pay) pl.sal_stride = pay;
+  pl.sm_total = 2u * pl.stage_bytes + (uint32_t)fh::kWarps * pl.sal_stride;
   if (pl.sm_total > kSmemLimit) return FH_ERR_UNSUPPORTED;
   int grid = 0;
   int rc = grid_for(fh::decompress_small<DT>, pl.sm_total, pl.ntiles, &grid);
@@ -613,6 +621,8 @@ void fh_default_params(fh_params* p) {
   p->dense_bits = 8;
   p->rounding = 0;
   p->seed = 0;
+  p->entropy = 0;
+  p->reserved = 0;
 }
 
 int fh_version(void) { return 1; }

@@ -24,6 +24,7 @@ namespace fh {
 
 struct SalientInfo {
   uint32_t nnz_s, n_dense, n_out_d, size;
+  uint32_t coded;  // bytes of the Huffman-coded section that replaces the dense blocks' code bytes; 0: plain codes
 };
 
 struct CompressArgs {
@@ -62,6 +63,7 @@ struct SplitOut {
   __device__ __forceinline__ uint8_t* at(uint32_t o) const { return o < npay ? slot + o : ovf + (o - npay); }
   __device__ __forceinline__ void st32(uint32_t o, uint32_t v) const { *reinterpret_cast<uint32_t*>(at(o)) = v; }
   __device__ __forceinline__ void st16(uint32_t o, uint32_t v) const { *reinterpret_cast<uint16_t*>(at(o)) = (uint16_t)v; }
+  __device__ __forceinline__ void st8(uint32_t o, uint32_t v) const { *at(o) = (uint8_t)v; }
 };
 
 // One 8x8 block in the registers of a warp: lane l holds the elements (l >> 3, l & 7) and
@@ -160,9 +162,48 @@ __device__ __noinline__ SalientInfo salient_measure(const Team& t, const Plan& p
   info.n_dense = team_excl_scan(t, blk_b, nblk);
   info.nnz_s = team_excl_scan(t, rowp, (uint32_t)H + 1u);
   info.n_out_d = team_excl_scan(t, blk_c, nblk);
+  info.coded = 0;
+  if (pl.entropy && info.n_dense) {
+    // Huffman stage (Section 4.4.1): histogram of the plane's code bytes, the code, the size of every chunk
+    uint32_t* blk_d = blk_c + nblk;   // bytes of a dense block's chunk
+    uint32_t* blk_e = blk_d + nblk;   // ... and where it starts
+    HufEncode* h = reinterpret_cast<HufEncode*>(blk_e + nblk);
+    for (uint32_t i = t.lane; i < 256u; i += t.size) h->hist[i] = 0;
+    team_sync(t);
+    for (uint32_t b = wid; b < nblk; b += nw) {
+      if (!blk_a[b]) continue;
+      const uint32_t by = b / nbx, bx = b - by * nbx;
+      const BlockRegs r = block_load<DT>(plane, H, W, (int)by, (int)bx, lane32);
+      uint32_t c0, c1, m0, m1;
+      block_codes(r, inv2e, lane32, c0, c1, m0, m1);
+      atomicAdd(&h->hist[c0], 1u);
+      atomicAdd(&h->hist[c1], 1u);
+    }
+    team_sync(t);
+    if (t.lane == 0) huffman_build(h);
+    team_sync(t);
+    if (h->maxlen <= kHufMaxLen) {
+      for (uint32_t b = wid; b < nblk; b += nw) {
+        uint32_t bits = 0;
+        if (blk_a[b]) {
+          const uint32_t by = b / nbx, bx = b - by * nbx;
+          const BlockRegs r = block_load<DT>(plane, H, W, (int)by, (int)bx, lane32);
+          uint32_t c0, c1, m0, m1;
+          block_codes(r, inv2e, lane32, c0, c1, m0, m1);
+          bits = (uint32_t)h->len[c0] + (uint32_t)h->len[c1];
+          asm volatile("redux.sync.add.u32 %0, %0, %1;" : "+r"(bits) : "r"(0xFFFFFFFFu));
+        }
+        if (lane32 == 0) blk_d[b] = blk_e[b] = (bits + 7u) >> 3;
+      }
+      team_sync(t);
+      const uint32_t chunks = team_excl_scan(t, blk_e, nblk);
+      const uint32_t section = a4(4u + a4(h->nlens) + a4(info.n_dense) + chunks);
+      if (section < 64u * info.n_dense) info.coded = section;
+    }
+  }
   const uint32_t e = (uint32_t)pl.esize;
   info.size = 16u + 4u * pl.nbm + 4u * ((uint32_t)H + 1u) + a4(2u * info.nnz_s) + a4(e * info.nnz_s) +
-              64u * info.n_dense + a4(e * info.n_out_d);
+              (info.coded ? info.coded : 64u * info.n_dense) + a4(e * info.n_out_d);
   return info;
 }
 
@@ -179,12 +220,12 @@ __device__ __noinline__ void salient_write(const Team& t, const Plan& pl, const 
   const uint32_t nw = t.block ? t.nwarps : 1u, wid = t.block ? threadIdx.x >> 5 : 0u, lane32 = threadIdx.x & 31u;
   const uint32_t o_bm = 16u, o_rp = o_bm + 4u * pl.nbm, o_col = o_rp + 4u * ((uint32_t)H + 1u);
   const uint32_t o_val = o_col + a4(2u * info.nnz_s), o_codes = o_val + a4(e * info.nnz_s);
-  const uint32_t o_outl = o_codes + 64u * info.n_dense;
+  const uint32_t o_outl = o_codes + (info.coded ? info.coded : 64u * info.n_dense);
   if (t.lane == 0) {
     out.st32(0, info.nnz_s);
     out.st32(4, info.n_dense);
     out.st32(8, info.n_out_d);
-    out.st32(12, 0);
+    out.st32(12, info.coded);
     // pads the section writers leave: col (2 bytes), val / verbatim values (bf16: 2 bytes)
     if (info.nnz_s & 1u) out.st16(o_col + 2u * info.nnz_s, 0);
     if (DT == kBF16 && (info.nnz_s & 1u)) out.st16(o_val + 2u * info.nnz_s, 0);
@@ -221,9 +262,35 @@ __device__ __noinline__ void salient_write(const Team& t, const Plan& pl, const 
       }
     }
   }
-  // dense blocks: 64 code bytes each, verbatim values in raster order
+  // dense blocks: 64 code bytes each (or their Huffman-coded chunk), verbatim values in raster order
   const float inv2e = __fdiv_rn(1.0f, __fmul_rn(2.0f, pl.eps));
   const uint32_t lt = (1u << lane32) - 1u;
+  const uint32_t* blk_d = blk_c + nblk;
+  const uint32_t* blk_e = blk_d + nblk;
+  HufEncode* h = reinterpret_cast<HufEncode*>(const_cast<uint32_t*>(blk_e + nblk));  // (only looked at when info.coded)
+  uint32_t o_chunks = 0;
+  if (info.coded) {  // the section's head: code lengths, then the bytes of every chunk; pads are zero
+    const uint32_t nl = h->nlens, o_cb = o_codes + 4u + a4(nl);
+    o_chunks = o_cb + a4(info.n_dense);
+    if (t.lane == 0) {
+      out.st8(o_codes, h->len[0]);
+      out.st8(o_codes + 1u, h->smin);
+      out.st8(o_codes + 2u, h->smax);
+      out.st8(o_codes + 3u, 0);
+      for (uint32_t o = o_codes + 4u + nl; o < o_cb; ++o) out.st8(o, 0);
+      for (uint32_t o = o_cb + info.n_dense; o < o_chunks; ++o) out.st8(o, 0);
+      uint32_t last_end = 0;  // end of the chunks: the last dense block's start + bytes
+      for (uint32_t b = nblk; b-- > 0;)
+        if (blk_a[b]) {
+          last_end = blk_e[b] + blk_d[b];
+          break;
+        }
+      for (uint32_t o = o_chunks + last_end; o < o_codes + info.coded; ++o) out.st8(o, 0);
+    }
+    for (uint32_t i = t.lane; i < nl; i += t.size) out.st8(o_codes + 4u + i, h->len[h->smin + i]);
+    for (uint32_t b = t.lane; b < nblk; b += t.size)
+      if (blk_a[b]) out.st8(o_cb + blk_b[b], blk_d[b]);
+  }
   for (uint32_t b = wid; b < nblk; b += nw) {
     if (!blk_a[b]) continue;
     const uint32_t by = b / nbx, bx = b - by * nbx;
@@ -240,6 +307,39 @@ __device__ __noinline__ void salient_write(const Team& t, const Plan& pl, const 
       const uint32_t rank = __popc(m0) + __popc(m1 & lt), idx1 = r.idx0 + 4u * (uint32_t)W;
       if (DT == kF32) out.st32(oo + 4u * rank, reinterpret_cast<const uint32_t*>(plane)[idx1]);
       else out.st16(oo + 2u * rank, reinterpret_cast<const uint16_t*>(plane)[idx1]);
+    }
+    if (info.coded) {
+      // the chunk's bits are assembled in shared memory (a code goes in most significant bit first, the words
+      // hold the stream big-endian) and leave byte by byte
+      uint32_t* stg = h->stage[wid];
+      for (uint32_t i = lane32; i < kHufStageWords; i += 32u) stg[i] = 0;
+      __syncwarp();
+      const uint32_t l0 = h->len[c0], l1 = h->len[c1];
+      uint32_t i0 = l0, i1 = l1;  // inclusive prefix sums of the lengths, raster positions l and l + 32
+      for (uint32_t o = 1; o < 32u; o <<= 1) {
+        const uint32_t u0 = __shfl_up_sync(0xFFFFFFFFu, i0, o), u1 = __shfl_up_sync(0xFFFFFFFFu, i1, o);
+        if (lane32 >= o) {
+          i0 += u0;
+          i1 += u1;
+        }
+      }
+      const uint32_t first_half = __shfl_sync(0xFFFFFFFFu, i0, 31);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const uint32_t len = half ? l1 : l0, at = half ? first_half + i1 - l1 : i0 - l0, cv = h->code[half ? c1 : c0];
+        const uint32_t wi = at >> 5;
+        const int shift = 32 - (int)(at & 31u) - (int)len;
+        if (shift >= 0) {
+          atomicOr(&stg[wi], cv << shift);
+        } else {
+          atomicOr(&stg[wi], cv >> (-shift));
+          atomicOr(&stg[wi + 1u], cv << (32 + shift));
+        }
+      }
+      __syncwarp();
+      for (uint32_t j = lane32; j < blk_d[b]; j += 32u) out.st8(o_chunks + blk_e[b] + j, (stg[j >> 2] >> (24u - 8u * (j & 3u))) & 0xFFu);
+      __syncwarp();
+      continue;
     }
     uint32_t w0 = c0 | (__shfl_down_sync(0xFFFFFFFFu, c0, 1) << 8);
     w0 |= __shfl_down_sync(0xFFFFFFFFu, w0, 2) << 16;
@@ -327,6 +427,7 @@ __device__ __forceinline__ void small_blocks(const Plan& pl, const uint8_t* plan
   sb.info.nnz_s = nnz_s;
   sb.info.n_dense = n_dense;
   sb.info.n_out_d = n_out_d;
+  sb.info.coded = 0;
   sb.info.size = 16u + 4u * pl.nbm + 4u * ((uint32_t)pl.H + 1u) + a4(2u * nnz_s) + a4(e * nnz_s) + 64u * n_dense +
                  a4(e * n_out_d);
 }
@@ -513,7 +614,9 @@ __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, 
   if (d.capacity >= 64) {
     uint4* hd = reinterpret_cast<uint4*>(d.dst);
     // a failed container must not pass for a valid one: no magic
-    hd[0] = make_uint4(code == kErrNone ? kMagic : 0u, 1u | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24), pl.N, pl.C);
+    // (version 2: payloads may carry Huffman-coded sections)
+    hd[0] = make_uint4(code == kErrNone ? kMagic : 0u, (pl.entropy ? 2u : 1u) | ((uint32_t)pl.dtype << 16) | ((uint32_t)pl.bits << 24),
+                       pl.N, pl.C);
     hd[1] = make_uint4((uint32_t)pl.H, (uint32_t)pl.W, 8u | (8u << 8) | ((uint32_t)pl.rounding << 16) | ((uint32_t)pl.mode << 24),
                        pl.rho_num | (pl.rho_den << 16));
     hd[2] = make_uint4(pl.tau_num | (pl.tau_den << 16), __float_as_uint(pl.eps), nsal, nraw);

@@ -34,7 +34,35 @@ struct SplitIn {
   __device__ __forceinline__ const uint8_t* at(uint32_t o) const { return o < npay ? slot + o : ovf + (o - npay); }
   __device__ __forceinline__ uint32_t ld32(uint32_t o) const { return __ldg(reinterpret_cast<const uint32_t*>(at(o))); }
   __device__ __forceinline__ uint32_t ld16(uint32_t o) const { return __ldg(reinterpret_cast<const uint16_t*>(at(o))); }
+  __device__ __forceinline__ uint32_t ld8(uint32_t o) const { return __ldg(at(o)); }
 };
+
+// One thread decodes a dense block's chunk of the Huffman-coded section (`nbytes` bytes at payload offset
+// `o_chunk`) into the block's 64 code bytes, four to a word.  False when the chunk is inconsistent.
+template <typename In>
+__device__ __noinline__ bool huffman_decode_chunk(const In& in, uint32_t o_chunk, uint32_t nbytes, const HufDecode* hd,
+                                                  uint32_t* codes) {
+  const uint32_t nbits = nbytes * 8u;
+  uint32_t pos = 0, cur = 0;
+  for (uint32_t i = 0; i < 16u; ++i) codes[i] = 0;
+  for (uint32_t i = 0; i < 64u; ++i) {
+    uint32_t acc = 0, sym = 256;
+    for (uint32_t l = 1; l <= kHufMaxLen; ++l) {
+      if (pos >= nbits) return false;
+      if ((pos & 7u) == 0u) cur = in.ld8(o_chunk + (pos >> 3));
+      acc = (acc << 1) | ((cur >> (7u - (pos & 7u))) & 1u);
+      ++pos;
+      const uint32_t k = acc - hd->first[l];
+      if (k < (uint32_t)hd->count[l]) {
+        sym = hd->sorted[hd->base[l] + k];
+        break;
+      }
+    }
+    if (sym > 255u) return false;
+    codes[i >> 2] |= sym << (8u * (i & 3u));
+  }
+  return true;
+}
 
 template <int DT>
 __device__ __forceinline__ void store_elem(uint8_t* plane, uint32_t i, float v) {
@@ -48,21 +76,43 @@ __device__ __forceinline__ float dequant(uint32_t q, float scale, float lo) {
   return __fmaf_rn(qf, scale, lo);
 }
 
-// Outlier-rich plane.  `scr` is the team's shared scratch: nblk words.  `ovf_avail` is the number of
-// readable bytes behind in.ovf.
+// Outlier-rich plane.  `scr` is the team's shared scratch: 2 * nblk words, followed by a HufDecode.  `ovf_avail`
+// is the number of readable bytes behind in.ovf; `version` the container's (2: the dense blocks' codes may be
+// Huffman-coded, Section 4.4.1 "Decompression involves Huffman decoding").
 template <int DT>
 __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const SplitIn& in, uint64_t ovf_avail, float eps,
-                               uint8_t* out, uint32_t* scr) {
+                               uint8_t* out, uint32_t* scr, uint32_t version) {
   const int H = pl.H, W = pl.W;
   const uint32_t nblk = pl.nblk, nbx = pl.nbx, nbm = pl.nbm, e = (uint32_t)pl.esize, HW = pl.HW;
-  const uint32_t nnz_s = in.ld32(0), n_dense = in.ld32(4), n_out_d = in.ld32(8);
+  const uint32_t nnz_s = in.ld32(0), n_dense = in.ld32(4), n_out_d = in.ld32(8), coded = in.ld32(12);
   if (nnz_s > HW || n_dense > nblk || n_out_d > HW) return false;
+  if (coded && (version != 2u || (coded & 3u) || coded >= 64u * n_dense)) return false;
   const uint64_t size = 16ull + 4ull * nbm + 4ull * ((uint64_t)H + 1) + a4(2u * nnz_s) + a4(e * nnz_s) +
-                        64ull * n_dense + a4(e * n_out_d);
+                        (coded ? (uint64_t)coded : 64ull * n_dense) + a4(e * n_out_d);
   if (size > in.npay && size - in.npay > ovf_avail) return false;
   const uint32_t o_bm = 16u, o_rp = o_bm + 4u * nbm, o_col = o_rp + 4u * ((uint32_t)H + 1u);
-  const uint32_t o_val = o_col + a4(2u * nnz_s), o_codes = o_val + a4(e * nnz_s), o_outl = o_codes + 64u * n_dense;
+  const uint32_t o_val = o_col + a4(2u * nnz_s), o_codes = o_val + a4(e * nnz_s);
+  const uint32_t o_outl = o_codes + (coded ? coded : 64u * n_dense);
   bool ok = true;
+  // Huffman-coded section: decoding tables from the stored lengths, start of every chunk from the chunks' sizes
+  uint32_t* cho = scr + nblk;  // by rank among the dense blocks
+  HufDecode* hd = reinterpret_cast<HufDecode*>(scr + 2u * nblk);
+  uint32_t o_chunks = 0, o_cb = 0;
+  if (coded) {
+    const uint32_t smin = in.ld8(o_codes + 1u), smax = in.ld8(o_codes + 2u);
+    if (smin < 1u || smax < smin) return false;
+    const uint32_t nl = smax - smin + 1u;
+    o_cb = o_codes + 4u + a4(nl);
+    o_chunks = o_cb + a4(n_dense);
+    if (o_chunks - o_codes > coded) return false;
+    for (uint32_t sym = t.lane; sym < 256u; sym += t.size)
+      hd->len[sym] = sym == 0u ? (uint8_t)in.ld8(o_codes) : ((sym >= smin && sym <= smax) ? (uint8_t)in.ld8(o_codes + 4u + sym - smin) : (uint8_t)0);
+    for (uint32_t r = t.lane; r < nblk; r += t.size) cho[r] = r < n_dense ? in.ld8(o_cb + r) : 0u;
+    team_sync(t);
+    if (t.lane == 0) huffman_tables(hd);
+    const uint32_t chunks = team_excl_scan(t, cho, nblk);
+    if (!hd->ok || o_chunks - o_codes + chunks > coded) return false;  // (the same for every thread)
+  }
   // zero fill (16-bit units cover both element sizes)
   for (uint32_t i = t.lane; i < (uint32_t)(pl.plane_bytes >> 1); i += t.size) reinterpret_cast<uint16_t*>(out)[i] = 0;
   // verbatim counts of the dense blocks -> first verbatim index of each block
@@ -73,8 +123,10 @@ __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const
       for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(in.ld32(o_bm + 4u * w));
       rank += __popc(in.ld32(o_bm + 4u * (b >> 5)) & ((1u << (b & 31u)) - 1u));
       if (rank < n_dense) {
+        uint32_t cw[16];
+        if (coded && !huffman_decode_chunk(in, o_chunks + cho[rank], in.ld8(o_cb + rank), hd, cw)) ok = false;
         for (uint32_t k = 0; k < 16; ++k) {
-          const uint32_t w = in.ld32(o_codes + 64u * rank + 4u * k);
+          const uint32_t w = coded ? cw[k] : in.ld32(o_codes + 64u * rank + 4u * k);
           cnt += ((w & 0xFFu) == 0) + ((w & 0xFF00u) == 0) + ((w & 0xFF0000u) == 0) + ((w & 0xFF000000u) == 0);
         }
       } else {
@@ -108,6 +160,11 @@ __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const
       for (uint32_t w = 0; w < (b >> 5); ++w) rank += __popc(in.ld32(o_bm + 4u * w));
       rank += __popc(in.ld32(o_bm + 4u * (b >> 5)) & ((1u << (b & 31u)) - 1u));
       const uint32_t oc = o_codes + 64u * rank;
+      uint32_t cw[16];
+      if (coded && !huffman_decode_chunk(in, o_chunks + cho[rank], in.ld8(o_cb + rank), hd, cw)) {
+        ok = false;
+        continue;
+      }
       uint32_t oi = scr[b];
       const int by = (int)(b / nbx), bx = (int)(b % nbx);
       int32_t prev[8];
@@ -116,7 +173,7 @@ __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const
 #pragma unroll 1
       for (int i = 0; i < 8; ++i) {
         const int y = by * 8 + i;
-        const uint32_t w0 = in.ld32(oc + 8u * i), w1 = in.ld32(oc + 8u * i + 4u);
+        const uint32_t w0 = coded ? cw[2 * i] : in.ld32(oc + 8u * i), w1 = coded ? cw[2 * i + 1] : in.ld32(oc + 8u * i + 4u);
         int32_t left = 0, ul = 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -156,20 +213,22 @@ __device__ __noinline__ bool decode_salient(const Team& t, const Plan& pl, const
   return ok;
 }
 
-// Header of a container against what the caller expects; also returns code width, eps and total size.
+// Header of a container against what the caller expects: 0 if it does not fit, the container's version (1, 2)
+// otherwise; also returns code width, eps and total size.
 __device__ __forceinline__ uint32_t check_header(const Plan& pl, const uint8_t* src, unsigned long long src_bytes, uint32_t& bits,
                                                  float& eps, unsigned long long& total) {
   if (src_bytes < 64ull + 16ull * pl.P) return 0u;
   const uint32_t* h = reinterpret_cast<const uint32_t*>(src);
   bits = __ldg(h + 1) >> 24;
-  bool ok = __ldg(h) == kMagic && (__ldg(h + 1) & 0xFFFFu) == 1u && ((__ldg(h + 1) >> 16) & 0xFFu) == (uint32_t)pl.dtype &&
+  const uint32_t version = __ldg(h + 1) & 0xFFFFu;
+  bool ok = __ldg(h) == kMagic && (version == 1u || version == 2u) && ((__ldg(h + 1) >> 16) & 0xFFu) == (uint32_t)pl.dtype &&
             (bits == 2u || bits == 4u || bits == 8u) && __ldg(h + 2) == pl.N && __ldg(h + 3) == pl.C &&
             __ldg(h + 4) == (uint32_t)pl.H && __ldg(h + 5) == (uint32_t)pl.W && (__ldg(h + 6) & 0xFFFFu) == (8u | (8u << 8));
   total = (unsigned long long)__ldg(h + 14) | ((unsigned long long)__ldg(h + 15) << 32);
   eps = __uint_as_float(__ldg(h + 9));
   const unsigned long long npay = a16(4u * ((pl.HW * (bits & 15u) + 31u) / 32u));
   ok = ok && total <= src_bytes && total >= 64ull + 16ull * pl.P + pl.P * npay && eps >= 1e-30f && eps <= 1e30f;
-  return ok ? 1u : 0u;
+  return ok ? version : 0u;
 }
 
 // Four restored values of one group leave as one 16-byte (fp32) or 8-byte (bf16) store.
@@ -373,8 +432,8 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
               continue;
             }
           }
-          uint32_t* scr = reinterpret_cast<uint32_t*>(smem) + (uint64_t)my_team * pl.nblk;
-          if (!decode_salient<DT>(team, s_pl, in, ovf_avail, eps, out, scr)) bad = true;
+          uint32_t* scr = reinterpret_cast<uint32_t*>(smem + (uint64_t)my_team * pl.sal_stride);
+          if (!decode_salient<DT>(team, s_pl, in, ovf_avail, eps, out, scr, s_hdr_ok)) bad = true;
         }
       } else {
         bad = true;
@@ -402,7 +461,7 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
       in.ovf = src + off;
       in.npay = npay;
       if (!decode_salient<DT>(cta, s_pl, in, off ? total - off : 0ull, s_eps, a.dst + gp * pl.plane_bytes,
-                              reinterpret_cast<uint32_t*>(smem)))
+                              reinterpret_cast<uint32_t*>(smem), s_hdr_ok))
         bad = true;
       __syncthreads();  // the scratch is reused
     }
@@ -597,7 +656,7 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_small(const Plan pl, c
     const Team warp_team = make_warp_team(s_red);
     const bool vec = (pl.plane_bytes & (DT == kF32 ? 15u : 7u)) == 0u;  // planes start on vector boundaries in the tile buffer
     const uint32_t tile_bytes_max = pl.stage_bytes;
-    const uint32_t pay_stride = a16((uint32_t)pl.plane_bytes) + 16u;  // per-warp scratch for a small plane's payload
+    const uint32_t pay_stride = pl.sal_stride;  // per-warp scratch: a small plane's payload, or the general path's tables
     uint32_t buf = 0;
     for (uint32_t tile = blockIdx.x; tile < pl.ntiles; tile += gridDim.x, buf ^= 1u) {
       uint8_t* tbuf = smem + (uint64_t)buf * tile_bytes_max;
@@ -671,7 +730,7 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_small(const Plan pl, c
         const unsigned long long ovf_avail = off ? total - off : 0ull;
         __syncwarp();
         bool good;
-        if (pl.nblk <= 4u && pl.H < 32) {
+        if (pl.nblk <= 4u && pl.H < 32 && in.ld32(12) == 0u) {  // (a Huffman-coded plane takes the general path)
           // the payload (shorter than the plane, or it would have been stored raw) is fetched in one go into the
           // warp's scratch and decoded from there
           uint8_t* pay = smem + 2ull * tile_bytes_max + (uint64_t)(tid >> 5) * pay_stride;
@@ -690,7 +749,8 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_small(const Plan pl, c
           }
         } else {
           good = decode_salient<DT>(warp_team, s_pl, in, ovf_avail, eps, out,
-                                    reinterpret_cast<uint32_t*>(smem + 2ull * tile_bytes_max) + (tid >> 5) * pl.nblk);
+                                    reinterpret_cast<uint32_t*>(smem + 2ull * tile_bytes_max + (uint64_t)(tid >> 5) * pl.sal_stride),
+                                    s_hdr_ok);
         }
         if (!good) bad = true;
         __syncwarp();

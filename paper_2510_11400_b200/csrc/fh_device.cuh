@@ -37,6 +37,7 @@ struct Plan {
   double inv_hw;         // 1 / HW in fp64
   int32_t bits, mode;
   int32_t rounding;      // 0: round half to even; 1: random rounding (Philox draws)
+  int32_t entropy;       // 1: Huffman stage on the dense-block codes of outlier-rich planes (container version 2)
   uint64_t seed;
   uint32_t rho_num, rho_den, tau_num, tau_den;
   float eps;
@@ -569,6 +570,133 @@ __device__ __forceinline__ uint32_t team_excl_scan(const Team& t, uint32_t* arr,
   }
   team_sync(t);
   return total;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Huffman stage on the residual code bytes of an outlier-rich plane's dense blocks (entropy = 1)
+// ------------------------------------------------------------------------------------------------
+// One code per plane from the plane's own 256-bin histogram; classical merge of the two least nodes, nodes
+// ordered by (weight, id), a leaf's id its symbol, a merged node's 256 + its order of creation; canonical
+// code values by (length, symbol); every dense block a chunk of its own that starts on a byte boundary, bits
+// most significant first.  Section: u8 len(0) | u8 smin | u8 smax | u8 0 | u8 len(smin..smax) (pad 4) |
+// u8 bytes of each chunk (pad 4) | chunks (pad 4).  Lengths stay below 25 (a plane has fewer than 2^17 codes).
+constexpr uint32_t kHufMaxLen = 24;
+constexpr uint32_t kHufStageWords = 48;  // a chunk has at most 64 * 24 / 8 = 192 bytes
+
+// Encoder scratch of one unit (shared memory).
+struct HufEncode {
+  uint32_t hist[256];
+  uint32_t code[256];
+  uint32_t w[512];        // node weights: 0..255 leaves by symbol, 256.. merged nodes
+  uint16_t parent[512];
+  uint16_t leaf[256];     // symbols that occur, sorted by (weight, symbol)
+  uint8_t len[256];
+  uint32_t smin, smax, maxlen, nlens;
+  uint32_t stage[kMaxWarps][kHufStageWords];  // a chunk's bits while a warp assembles them
+};
+
+// One thread: code lengths and canonical codes from h->hist.
+__device__ __noinline__ void huffman_build(HufEncode* h) {
+  uint32_t n = 0;
+  for (uint32_t sym = 0; sym < 256u; ++sym) {
+    h->len[sym] = 0;
+    h->code[sym] = 0;
+    h->w[sym] = h->hist[sym];
+    if (h->hist[sym]) h->leaf[n++] = (uint16_t)sym;
+  }
+  if (n == 1) h->len[h->leaf[0]] = 1;
+  if (n > 1) {
+    for (uint32_t i = 1; i < n; ++i) {  // insertion sort: equal weights stay in symbol order
+      const uint16_t v = h->leaf[i];
+      uint32_t j = i;
+      while (j > 0 && h->hist[h->leaf[j - 1]] > h->hist[v]) {
+        h->leaf[j] = h->leaf[j - 1];
+        --j;
+      }
+      h->leaf[j] = v;
+    }
+    uint32_t li = 0, mi = 256, mn = 256;  // head of the leaf queue, head and end of the queue of merged nodes
+    while ((n - li) + (mn - mi) > 1u) {
+      uint32_t pick[2];
+      for (int k = 0; k < 2; ++k) {
+        bool take_leaf;
+        if (li >= n) take_leaf = false;
+        else if (mi >= mn) take_leaf = true;
+        else take_leaf = h->w[h->leaf[li]] <= h->w[mi];  // equal weights: the leaf has the smaller id
+        pick[k] = take_leaf ? h->leaf[li++] : mi++;
+      }
+      h->w[mn] = h->w[pick[0]] + h->w[pick[1]];
+      h->parent[pick[0]] = h->parent[pick[1]] = (uint16_t)mn;
+      ++mn;
+    }
+    const uint32_t root = mn - 1u;
+    for (uint32_t i = 0; i < n; ++i) {
+      uint32_t d = 0;
+      for (uint32_t v = h->leaf[i]; v != root; v = h->parent[v]) ++d;
+      h->len[h->leaf[i]] = (uint8_t)min(d, 255u);
+    }
+  }
+  uint32_t next = 0, prev = 0, maxlen = 0, smin = 1, smax = 1;
+  bool any = false;
+  for (uint32_t l = 1; l <= 32u; ++l)
+    for (uint32_t sym = 0; sym < 256u; ++sym)
+      if (h->len[sym] == l) {
+        next <<= (l - prev);
+        prev = l;
+        h->code[sym] = next++;
+      }
+  for (uint32_t sym = 0; sym < 256u; ++sym) {
+    maxlen = max(maxlen, (uint32_t)h->len[sym]);
+    if (sym && h->len[sym]) {
+      if (!any) smin = sym;
+      smax = sym;
+      any = true;
+    }
+  }
+  h->smin = smin;
+  h->smax = smax;
+  h->maxlen = maxlen;
+  h->nlens = smax - smin + 1u;
+}
+
+// Decoder tables of one unit (shared memory), from the lengths stored in a section.
+struct HufDecode {
+  uint32_t first[kHufMaxLen + 1];   // first code value of every length
+  uint16_t count[kHufMaxLen + 1];   // symbols of every length
+  uint16_t base[kHufMaxLen + 1];    // index of a length's first symbol in `sorted`
+  uint8_t sorted[256];              // symbols by (length, symbol)
+  uint8_t len[256];
+  uint32_t ok;
+};
+// One thread: tables from t->len; t->ok = 0 unless the lengths form a complete prefix code (or a single code of any length).
+__device__ __noinline__ void huffman_tables(HufDecode* t) {
+  for (uint32_t l = 0; l <= kHufMaxLen; ++l) t->count[l] = 0;
+  unsigned long long kraft = 0;  // in units of 2^-32
+  uint32_t nsym = 0;
+  bool bad = false;
+  for (uint32_t sym = 0; sym < 256u; ++sym) {
+    const uint32_t l = t->len[sym];
+    if (l > kHufMaxLen) bad = true;
+    else if (l) {
+      ++t->count[l];
+      kraft += 1ull << (32u - l);
+      ++nsym;
+    }
+  }
+  if (nsym == 0 || kraft > (1ull << 32) || (nsym > 1 && kraft != (1ull << 32))) bad = true;
+  uint32_t next = 0, prev = 0, idx = 0;
+  for (uint32_t l = 1; l <= kHufMaxLen; ++l) {
+    t->base[l] = (uint16_t)idx;
+    if (t->count[l]) {
+      next <<= (l - prev);
+      prev = l;
+    }
+    t->first[l] = next;
+    for (uint32_t sym = 0; sym < 256u && !bad; ++sym)
+      if (t->len[sym] == l) t->sorted[idx++] = (uint8_t)sym;
+    next += t->count[l];
+  }
+  t->ok = bad ? 0u : 1u;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -30,7 +30,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_sizes_match_header_layout():
     assert C.sizeof(api.fh_tensor_desc) == 32
-    assert C.sizeof(api.fh_params) == 48
+    assert C.sizeof(api.fh_params) == 56
     assert C.sizeof(api.fh_sched_entry) == 56
     assert C.sizeof(api.fh_sched_report) == 40
 

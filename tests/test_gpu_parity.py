@@ -122,6 +122,31 @@ def test_parity_forced_modes(shape, dtype, mode):
     full_parity(spec, bits=4, salient_mode=mode)
 
 
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_parity_huffman_stage(shape, dtype):
+    """entropy = 1: the dense-block residual codes of outlier-rich planes go through the Huffman stage (one
+    code per plane); container (version 2) identical to the oracle's byte for byte, restored values identical,
+    in the three-sigma mode on mixed planes and with every plane forced down the block-wise path."""
+    kind = "spiky_relu" if (shape[1] >= 3) else "relu"
+    buf = full_parity(synth.TensorSpec("t", shape, dtype, kind, 71), bits=4, entropy=1, eps=0.25)
+    assert fho.parse_header(buf)["version"] == 2
+    buf = full_parity(synth.TensorSpec("t", shape, dtype, "relu", 72), bits=2, entropy=1, eps=0.25, salient_mode=api.FH_SALIENT_ALL)
+    plain = fho.compress(synth.make(synth.TensorSpec("t", shape, dtype, "relu", 72)), fho.desc(shape, dtype),
+                         fho.params(bits=2, eps=0.25, salient_mode=fho.ALL))[1]
+    assert buf.size <= plain.size
+
+
+def test_huffman_stage_gain_on_the_supplementary_workload():
+    """Every 16th channel sparse-spiky (the recipe that drives planes down the block-wise path), ResNet-shaped
+    56x56 planes: the stage shrinks the container, and the GPU's bytes are the oracle's."""
+    spec = synth.supplement([synth.TensorSpec("s", (8, 64, 56, 56), synth.F32, "relu", 130)])[0]
+    plain = full_parity(spec, bits=2, eps=0.0625)
+    coded = full_parity(spec, bits=2, eps=0.0625, entropy=1)
+    assert coded.size < plain.size
+    print(f"supplement 8x64x56x56: {plain.size} B plain, {coded.size} B with the Huffman stage")
+
+
 @pytest.mark.parametrize("kind", ["relu", "normal", "laplace_ch", "laplace_iid", "spiky_normal"])
 @pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
 def test_parity_value_distributions(kind, dtype):
