@@ -24,7 +24,8 @@
  *     Dense and packed device buffers must be 16-byte aligned.
  *   - fh_compress and fh_decompress only enqueue work on `stream` (a cudaStream_t passed as
  *     void*; NULL is the legacy default stream) and never synchronise.  Per stream the library keeps
- *     one small scratch allocation (counters, and four bytes per plane of the largest tensor seen)
+ *     one small scratch allocation (counters, and about 13 bytes per tile of planes of the largest
+ *     tensor seen: the words through which tiles tell one another where their payloads go)
  *     that it creates on first use and frees in fh_shutdown(); growing it for a tensor with more
  *     planes synchronises the device once.
  *   - There is no CPU fallback: without a CUDA device every entry point that does work returns

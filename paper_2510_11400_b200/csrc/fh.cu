@@ -291,7 +291,7 @@ int next_call(uint32_t* calls, unsigned long long* scan, size_t tile_cap, cudaSt
 
 int sm_count();
 
-// Scratch of the channel-wide three-sigma mode (grown like the work list).
+// Scratch of the channel-wide three-sigma mode (grown on demand like the per-stream scratch).
 int get_channel_scratch(StreamScratch* s, size_t planes, size_t channels) {
   if (planes > s->pn_cap) {
     size_t cap = s->pn_cap ? s->pn_cap : 65536;

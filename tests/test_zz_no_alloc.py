@@ -44,7 +44,7 @@ def _compress_both(spec, bits):
 def test_static_scratch_entry_point_matches_fh_compress_on_two_calls_in_a_row():
     build.build()
     api.lib()
-    # first call: many planes of mixed classes, so the work list and the chunk sums are really used
+    # first call: many planes of mixed classes, so the placement words of the fixed scratch are really used
     a = synth.TensorSpec("za", (64, 48, 14, 14), synth.F32, "spiky_relu", 5)
     ref, got = _compress_both(a, 2)
     assert ref.size == got.size and np.array_equal(ref, got)
@@ -60,7 +60,7 @@ def test_static_scratch_entry_point_matches_fh_compress_on_two_calls_in_a_row():
 def test_static_scratch_entry_point_refuses_tensors_beyond_its_limit():
     import torch
     build.build()
-    planes = api.FH_STATIC_MAX_PLANES + 64           # one batch row more than the fixed work list holds
+    planes = api.FH_STATIC_MAX_PLANES + 64           # one batch row more than the fixed scratch holds
     d = api.desc((planes // 64, 64, 4, 4), api.FH_F32)
     p = api.default_params(bits=2)
     x = torch.zeros(planes * 16, dtype=torch.float32, device="cuda")
