@@ -553,7 +553,7 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   StreamScratch* s = nullptr;
   rc = get_scratch(stream, pl.mode == FH_SALIENT_OFF ? 0 : pl.ntiles, &s);
   if (rc != FH_OK) return rc;
-  fh::CompressArgs a;
+  fh::CompressArgs a = {};
   a.src = (const uint8_t*)d_src;
   a.dst_base = (uint8_t*)d_dst;
   a.capacity = capacity;
@@ -932,7 +932,7 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   const size_t cap = FH_STATIC_MAX_PLANES;
   if (cudaMemsetAsync(base, 0, fh::kScratchHeadBytes, stream) != cudaSuccess) return FH_ERR_CUDA;
   if (cudaMemsetAsync(scan + cap, 0, (cap / 32) * sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
-  fh::CompressArgs a;
+  fh::CompressArgs a = {};
   a.src = (const uint8_t*)d_src;
   a.dst_base = (uint8_t*)d_dst;
   a.capacity = dst_capacity;

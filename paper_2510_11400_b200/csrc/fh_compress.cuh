@@ -741,6 +741,11 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
 
   const uint32_t tid = threadIdx.x;
   if (tid == 0 && a.early_ticket) s_tile = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
+  if (tid == 0 && pl.mode != kModeOff) {  // (before the wait for the previous kernel, whose tail hides it)
+    s_ctl.pl = pl;
+    s_ctl.a = a;
+    s_ctl.head = kNoTile;
+  }
   dep_wait();     // the previous kernel on the stream has completed
   dep_trigger();  // the next kernel on the stream may become resident as this one drains
   uint8_t* tile_buf = smem + pl.sm_tile;
@@ -748,12 +753,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
   Rec* rec = reinterpret_cast<Rec*>(smem + pl.sm_rec);
   uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal);
   const Dest d = make_dest(pl, a);
-  if (tid == 0 && pl.mode != kModeOff) {
-    s_ctl.pl = pl;
-    s_ctl.a = a;
-    s_ctl.d = d;
-    s_ctl.head = kNoTile;
-  }
+  if (tid == 0 && pl.mode != kModeOff) s_ctl.d = d;
   const Team team = make_team(pl.team, s_red);
   const Team cta = make_team(kThreads, s_red);
   const uint32_t nteams = team.block ? 1u : kThreads / team.size;
@@ -1280,6 +1280,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
   const uint32_t nstage = pl.nstage;
   const bool scan_on = pl.mode != kModeOff;
   uint32_t first_ticket = 0;
+  // Everything that needs no global memory comes before the wait for the previous kernel, whose tail hides it.
   if (tid == 0) {
     for (uint32_t s = 0; s < nstage; ++s) {
       mbar_init(&s_full[s], 1);
@@ -1287,20 +1288,9 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     }
     fence_mbar_init();
     s_abort = 0;
-  }
-  // (the ticket counter of this call was returned to zero by the call before the previous one, which had
-  // completed before the previous kernel let this one start)
-  if (tid == (uint32_t)kThreads && a.early_ticket)
-    first_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
-  dep_wait();     // the previous kernel on the stream has completed; global memory may be touched from here on
-  dep_trigger();  // the next kernel on the stream may become resident as this one drains
-  const Dest d = make_dest(pl, a);
-  if (tid == 0) {
-    if (!d.fits && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
     if (scan_on) {
       s_ctl.pl = pl;
       s_ctl.a = a;
-      s_ctl.d = d;
       s_ctl.head = kNoTile;
       for (uint32_t s = 0; s < nstage; ++s) {
         s_ctl.U[s] = s_ctl.C[s] = s_ctl.arr[s] = 0;
@@ -1308,7 +1298,21 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
       }
     }
   }
+  // (the ticket counter of this call was returned to zero by the call before the previous one, which had
+  // completed before the previous kernel let this one start)
+  if (tid == (uint32_t)kThreads && a.early_ticket)
+    first_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
   __syncthreads();
+  dep_wait();     // the previous kernel on the stream has completed; global memory may be touched from here on
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
+  const Dest d = make_dest(pl, a);
+  if (warp < (uint32_t)kWarps) {  // (the producer goes straight to its first loads)
+    if (tid == 0) {
+      if (!d.fits && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+      if (scan_on) s_ctl.d = d;
+    }
+    asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");  // the consumer warps: s_ctl.d is in place
+  }
 
   if (warp == (uint32_t)kWarps) {
     // ======================= producer (all 32 lanes walk the loop, lane 0 issues) =======================
@@ -1573,10 +1577,13 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     // completed before the previous kernel let this one start)
     if (a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
   }
+  if (tid == 0 && scan_on) {  // (before the wait for the previous kernel, whose tail hides it)
+    s_ctl.pl = pl;
+    s_ctl.a = a;
+    s_ctl.head = kNoTile;
+  }
   dep_wait();     // the previous kernel on the stream has completed; global memory may be touched from here on
   dep_trigger();  // the next kernel on the stream may become resident as this one drains
-  const Dest d = make_dest(pl, a);
-  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
   auto issue = [&](uint32_t s) {
     const uint32_t t = next_ticket;
     s_tiles[s] = t;
@@ -1589,15 +1596,14 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
       next_ticket = issued < nstage ? t + 1u : (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
     }
   };
-  if (tid == 0) {
-    if (scan_on) {
-      s_ctl.pl = pl;
-      s_ctl.a = a;
-      s_ctl.d = d;
-      s_ctl.head = kNoTile;
-    }
+  if (tid == 0) {  // the first loads before anything else
     if (!a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
     for (uint32_t s = 0; s < nstage; ++s) issue(s);
+  }
+  const Dest d = make_dest(pl, a);
+  if (tid == 0) {
+    if (!d.fits && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+    if (scan_on) s_ctl.d = d;
   }
   __syncthreads();
 

@@ -150,12 +150,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// Bounded wait that also gives up when *abort becomes non-zero.
+// Bounded wait that also gives up when *abort becomes non-zero (looked at every eighth attempt: an attempt
+// ends early whenever anything arrives at the barrier, so a waiting warp makes many of them).
 __device__ __forceinline__ bool mbar_wait_abortable(uint64_t* bar, uint32_t parity, uint32_t limit,
                                                     const volatile uint32_t* abort) {
   for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (*abort) return false;
+    if ((i & 7u) == 7u && *abort) return false;
   }
   return false;
 }
