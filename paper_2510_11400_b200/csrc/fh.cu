@@ -222,6 +222,8 @@ struct StreamScratch {
   unsigned long long* scan = nullptr;    // placement scan: tile words, group sums, group prefixes; then the tile links
   size_t tile_cap = 0;                   // tiles the scan arrays hold (groups: tile_cap / 32)
   uint32_t calls = 0;                    // compress calls so far: parity of the ticket counter, epoch of the scan
+  uint32_t scan_calls = 0;               // ... those that used the placement scan: which set of group sums is next
+  uint32_t prev_groups = 0;              // groups of 32 tiles the last of them used (the next one clears that set)
   uint32_t* plane_nout = nullptr;        // channel-wide three-sigma mode: per-plane counts ...
   size_t pn_cap = 0;
   fh::ChanStat* chan = nullptr;          // ... and per-channel statistics
@@ -229,7 +231,8 @@ struct StreamScratch {
   unsigned long long* sched = nullptr;   // schedule runner: offsets, sizes, statuses
   size_t sched_cap = 0;
 };
-inline size_t scan_words(size_t tile_cap) { return tile_cap + 2 * (tile_cap / 32) + tile_cap / 2; }
+// tile words | two sets of group sums | group prefixes | tile links (32-bit)
+inline size_t scan_words(size_t tile_cap) { return tile_cap + 3 * (tile_cap / 32) + tile_cap / 2; }
 
 std::mutex g_mu;
 std::map<std::pair<int, cudaStream_t>, StreamScratch> g_scratch;
@@ -260,6 +263,7 @@ int get_scratch(cudaStream_t stream, size_t tiles, StreamScratch** out) {
       s.scan = nullptr;
       s.tile_cap = 0;
     }
+    s.prev_groups = 0;
     if (cudaMalloc(&s.scan, scan_words(cap) * sizeof(unsigned long long)) != cudaSuccess) return FH_ERR_CUDA;
     if (cudaMemsetAsync(s.scan, 0, scan_words(cap) * sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
     s.tile_cap = cap;
@@ -270,22 +274,44 @@ int get_scratch(cudaStream_t stream, size_t tiles, StreamScratch** out) {
 
 // Parity, epoch and scan pointers of the next compress call on a scratch (`scan` may be null when the call
 // places nothing).  The epoch never is 0; when the counter wraps, the tagged arrays are cleared.
-int next_call(uint32_t* calls, unsigned long long* scan, size_t tile_cap, cudaStream_t stream, fh::CompressArgs* a) {
+// `s`: the per-stream scratch, whose two sets of group sums alternate between the calls that use the scan (the
+// call returns the other set -- the one its predecessor used -- to zero); null: one set, which the caller
+// clears ahead of every call (the fixed scratch of fh_compress_static).
+int next_call(uint32_t* calls, unsigned long long* scan, size_t tile_cap, StreamScratch* s, uint32_t groups_now,
+              cudaStream_t stream, fh::CompressArgs* a) {
   ++*calls;
   if ((*calls & 0x7FFFFFFFu) == 0u) {  // 2^31 calls later an old tag could pass for a new one: start afresh
-    if (scan && cudaMemsetAsync(scan, 0, scan_words(tile_cap) * sizeof(unsigned long long), stream) != cudaSuccess)
-      return FH_ERR_CUDA;
+    const size_t words = s ? scan_words(tile_cap) : tile_cap + 2 * (tile_cap / 32);
+    unsigned long long* all = s ? s->scan : scan;  // (also when this very call places nothing)
+    if (all && cudaMemsetAsync(all, 0, words * sizeof(unsigned long long), stream) != cudaSuccess) return FH_ERR_CUDA;
+    if (s) s->prev_groups = 0;
     ++*calls;
   }
+  const size_t ngrp = tile_cap / 32;
   a->parity = *calls & 1u;
   a->scan.tile = scan;
-  a->scan.grp = scan ? scan + tile_cap : nullptr;
-  a->scan.gpre = scan ? scan + tile_cap + tile_cap / 32 : nullptr;
-  a->defer_next = scan ? reinterpret_cast<uint32_t*>(scan + tile_cap + 2 * (tile_cap / 32)) : nullptr;
+  a->scan.grp = nullptr;
+  a->scan.grp_clear = nullptr;
+  a->scan.clear_groups = 0;
+  a->scan.gpre = nullptr;
+  a->defer_next = nullptr;
+  if (scan && s) {
+    const uint32_t set = s->scan_calls++ & 1u;
+    a->scan.grp = scan + tile_cap + set * ngrp;
+    a->scan.grp_clear = scan + tile_cap + (1u - set) * ngrp;
+    a->scan.clear_groups = s->prev_groups;
+    s->prev_groups = groups_now;
+    a->scan.gpre = scan + tile_cap + 2 * ngrp;
+    a->defer_next = reinterpret_cast<uint32_t*>(scan + tile_cap + 3 * ngrp);
+  } else if (scan) {
+    a->scan.grp = scan + tile_cap;
+    a->scan.grp_clear = a->scan.grp;
+    a->scan.gpre = scan + tile_cap + ngrp;
+    a->defer_next = reinterpret_cast<uint32_t*>(scan + tile_cap + 2 * ngrp);
+  }
   a->scan.epoch = *calls & 0x7FFFFFFFu;
   a->scan.polls = g_scan_polls;
   a->scan.skip_tile = g_skip_tile;
-  a->scan.reserved = 0;
   return FH_OK;
 }
 
@@ -562,7 +588,7 @@ int enqueue_compress(const fh_tensor_desc* desc, const fh_params* params, const 
   a.out2 = d_out2;
   a.sc = s->sc;
   a.early_ticket = 1;
-  rc = next_call(&s->calls, s->scan, s->tile_cap, stream, &a);
+  rc = next_call(&s->calls, pl.mode == FH_SALIENT_OFF ? nullptr : s->scan, s->tile_cap, s, (pl.ntiles + 31u) / 32u, stream, &a);
   if (rc != FH_OK) return rc;
   a.chan_nout = nullptr;
   a.plane_nout = nullptr;
@@ -941,7 +967,7 @@ int fh_compress_static(const fh_tensor_desc* desc, const fh_params* params, cons
   a.out2 = (unsigned long long*)d_out2;
   a.sc = reinterpret_cast<fh::Scratch*>(base);
   a.early_ticket = 0;  // the counters are cleared by the memset just enqueued: nothing may touch them before it
-  rc = next_call(&g_static_calls[dev], scan, cap, stream, &a);
+  rc = next_call(&g_static_calls[dev], scan, cap, nullptr, 0, stream, &a);
   if (rc != FH_OK) return rc;
   a.chan_nout = nullptr;
   a.plane_nout = nullptr;

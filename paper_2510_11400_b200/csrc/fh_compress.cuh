@@ -54,6 +54,18 @@ __device__ __forceinline__ uint32_t channel_class(const Plan& pl, const Compress
   return total * pl.rho_den > (unsigned long long)pl.rho_num * pl.N * pl.HW ? kClsSalient : kClsNormal;
 }
 
+// A CTA whose threads change one of the call's counters (error code, overflow size, plane counts) notes it in
+// this flag; cta_exit passes it on through the exit counter, so that the last CTA of a call in which nobody did
+// -- every plane normal, no error: the usual case -- neither fences nor reads the counters back.
+__device__ __forceinline__ volatile uint32_t* cta_dirty() {
+  __shared__ uint32_t flag;
+  return &flag;
+}
+__device__ __forceinline__ void report_error(const CompressArgs& a, uint32_t code) {
+  *cta_dirty() = 1u;
+  atomicMax(&a.sc->status, (unsigned long long)code);
+}
+
 // Where the bytes of a salient / raw payload go: offsets below npay land in the plane's slot, the
 // rest in its overflow part.  Offsets and npay are multiples of the access size.
 struct SplitOut {
@@ -550,6 +562,7 @@ __device__ __forceinline__ uint32_t plane_units(const Plan& pl, const SalientInf
 
 // Per-call counters of a tile's outlier-rich planes (one thread): nsal and nraw share a word.
 __device__ __forceinline__ void count_blockwise(const CompressArgs& a, uint32_t units, uint32_t nsal, uint32_t nraw) {
+  if (units | nsal | nraw) *cta_dirty() = 1u;
   if (units) atomicAdd(&a.sc->ovf16, (unsigned long long)units);
   if (nsal | nraw) atomicAdd(&a.sc->nsal, (unsigned long long)nsal | ((unsigned long long)nraw << 32));
 }
@@ -604,11 +617,17 @@ __device__ __forceinline__ void warp_plane_write(const Team& warp_team, const Pl
 
 // One thread, after everything else of the call is done: header, result words, and every counter the
 // call touched back to zero.
-__device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, const Dest& d) {
-  const unsigned long long ovf16 = ld_relaxed(&a.sc->ovf16);
-  const unsigned long long cnt = ld_relaxed(&a.sc->nsal);
+// `touched`: some CTA of the call has changed a counter; otherwise all of them are known to be zero.
+__device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, const Dest& d, bool touched) {
+  unsigned long long ovf16 = 0, cnt = 0;
+  uint32_t code = kErrNone;
+  if (touched) {
+    __threadfence();  // the counters as the other CTAs left them before they were counted out
+    ovf16 = ld_relaxed(&a.sc->ovf16);
+    cnt = ld_relaxed(&a.sc->nsal);
+    code = (uint32_t)ld_relaxed(&a.sc->status);
+  }
   const uint32_t nsal = (uint32_t)cnt, nraw = (uint32_t)(cnt >> 32);
-  uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
   const unsigned long long total = pl.ovf_off + ovf16 * 16ull;
   if (total > d.capacity && code < kErrCapacity) code = kErrCapacity;
   if (d.capacity >= 64) {
@@ -632,21 +651,34 @@ __device__ __forceinline__ void finalize(const Plan& pl, const CompressArgs& a, 
   if (code) st_relaxed(&a.sc->status, 0ull);
 }
 
-// Last step of every CTA: the last CTA to leave returns the scan's group counters and the hand-out
-// counters to zero and finishes the container.
+// Last step of every CTA: the last CTA to leave returns the group sums of the previous call's placement scan and
+// the hand-out counters to zero and finishes the container.
+// The exit counter carries the CTAs that have left in its low half and, in its high half, how many of them had
+// changed a counter of the call (cta_dirty); only such a CTA fences -- its updates must be performed before it is
+// counted out -- so a call without outlier-rich planes and without errors ends with one atomic per CTA and no
+// read-back.  The container itself needs no fence: its readers are later kernels.
 __device__ __forceinline__ void cta_exit(const Plan& pl, const CompressArgs& a, const Dest& d, uint32_t* s_last) {
-  __threadfence();
+  __syncthreads();  // every thread's note in the flag is in
+  const bool dirty = *cta_dirty() != 0u;  // (the same for every thread)
+  if (dirty) {
+    __threadfence();
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const unsigned long long old = atomicAdd(&a.sc->exited, 1ull | (dirty ? 1ull << 32 : 0ull));
+    const bool last = (uint32_t)old == gridDim.x - 1u;
+    *s_last = last ? (((old >> 32) != 0ull || dirty) ? 3u : 1u) : 0u;
+  }
   __syncthreads();
-  if (threadIdx.x == 0) *s_last = atomicAdd(&a.sc->exited, 1ull) == (unsigned long long)gridDim.x - 1ull;
-  __syncthreads();
-  if (!*s_last) return;
+  const uint32_t last = *s_last;
+  if (!last) return;
   if (pl.mode != kModeOff)
-    for (uint32_t k = threadIdx.x; k < ((pl.ntiles + 31u) >> 5); k += blockDim.x) a.scan.grp[k] = 0ull;
+    for (uint32_t k = threadIdx.x; k < a.scan.clear_groups; k += blockDim.x) a.scan.grp_clear[k] = 0ull;
   if (threadIdx.x != 0) return;
-  __threadfence();
+  // (what follows is read by later kernels only, which start work after this one has completed: no fence)
   st_relaxed(&a.sc->ticket[a.parity], 0ull);
   st_relaxed(&a.sc->exited, 0ull);
-  finalize(pl, a, d);
+  finalize(pl, a, d, (last & 2u) != 0u);
 }
 
 __device__ __forceinline__ void store_table_entry(const Dest& d, uint64_t plane, uint32_t off16, uint32_t meta, float lo,
@@ -740,6 +772,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
   __shared__ BlockCtl s_ctl;
 
   const uint32_t tid = threadIdx.x;
+  if (tid == 0) *cta_dirty() = 0u;
   if (tid == 0 && a.early_ticket) s_tile = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
   if (tid == 0 && pl.mode != kModeOff) {  // (before the wait for the previous kernel, whose tail hides it)
     s_ctl.pl = pl;
@@ -761,7 +794,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
   constexpr uint32_t L = (1u << BITS) - 1u;
   const bool need_sigma = pl.mode == kModeAuto;
   uint32_t rp = 0;  // reduction counter (see red_half)
-  if (!d.fits && tid == 0 && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+  if (!d.fits && tid == 0 && blockIdx.x == 0) report_error(a, kErrCapacity);
 
   for (bool first = true;; first = false) {
     if (tid == 0 && !(first && a.early_ticket)) s_tile = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
@@ -797,7 +830,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
       team_minmax(team, lo, hi, rp);
       const float range = __fsub_rn(hi, lo);
       if (!(fabsf(range) <= 3.402823466e38f) && team.lane == 0)
-        atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+        report_error(a, kErrNonfinite);
 
       uint32_t cls = kClsNormal, n_out = 0;
       if (need_sigma) {
@@ -925,7 +958,7 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
       uint32_t base = 0;
       if (U) ok = scan_prefix(a.scan, tile, base);
       if (tid == 0) {
-        if (!ok) atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+        if (!ok) report_error(a, kErrTimeout);
         s_ctl.base = base;
         s_ctl.ok = ok;
       }
@@ -1046,7 +1079,7 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
   hi = max_nan(hi, hi1);
   team_minmax(team, lo, hi, rp);
   const float range = __fsub_rn(hi, lo);
-  if (!(fabsf(range) <= 3.402823466e38f) && lane == 0) atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+  if (!(fabsf(range) <= 3.402823466e38f) && lane == 0) report_error(a, kErrNonfinite);
 
   // distances from the minimum, in place (x - lo is x + (-lo): the same rounding)
   {
@@ -1247,7 +1280,7 @@ __device__ __noinline__ void warp_phase2(BlockCtl* c, uint8_t* stages, uint8_t* 
         uint32_t base = 0;
         if (run) ok = scan_prefix(c->a.scan, tile, base);
         if (lane == 0) {
-          if (!ok) atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
+          if (!ok) report_error(c->a, kErrTimeout);
           c->base = base;
           c->ok = ok;
         }
@@ -1288,6 +1321,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     }
     fence_mbar_init();
     s_abort = 0;
+    *cta_dirty() = 0u;
     if (scan_on) {
       s_ctl.pl = pl;
       s_ctl.a = a;
@@ -1308,7 +1342,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
   const Dest d = make_dest(pl, a);
   if (warp < (uint32_t)kWarps) {  // (the producer goes straight to its first loads)
     if (tid == 0) {
-      if (!d.fits && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+      if (!d.fits && blockIdx.x == 0) report_error(a, kErrCapacity);
       if (scan_on) s_ctl.d = d;
     }
     asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory");  // the consumer warps: s_ctl.d is in place
@@ -1380,7 +1414,7 @@ __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Pla
     if (aborted) {  // wait (bounded) for copies still in flight before the CTA may exit
       s_abort = 1;
       if (lane == 0) {
-        atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+        report_error(a, kErrTimeout);
         for (uint32_t k = 0; k < nstage; ++k) {
           mbar_wait(&s_full[k], 0u, 1u << 10);
           mbar_wait(&s_full[k], 1u, 1u << 10);
@@ -1478,7 +1512,7 @@ __device__ __noinline__ void cta_phase2(BlockCtl* c, double* red, uint8_t* stage
     parity ^= 1u;
     if (!ready) {  // the load timed out: report, wait (bounded) for the copy, give up
       if (tid == 0) {
-        atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
+        report_error(c->a, kErrTimeout);
         mbar_wait(bar, parity ^ 1u, 1u << 10);
       }
       return;
@@ -1491,7 +1525,7 @@ __device__ __noinline__ void cta_phase2(BlockCtl* c, double* red, uint8_t* stage
       uint32_t base = 0;
       if (units) ok = scan_prefix(c->a.scan, tile, base);
       if (tid == 0) {
-        if (!ok) atomicMax(&c->a.sc->status, (unsigned long long)kErrTimeout);
+        if (!ok) report_error(c->a, kErrTimeout);
         c->base = base;
         c->ok = ok;
       }
@@ -1573,6 +1607,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
     fence_mbar_init();
     s_abort = 0;
+    *cta_dirty() = 0u;
     // (the ticket counter of this call was returned to zero by the call before the previous one, which had
     // completed before the previous kernel let this one start)
     if (a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
@@ -1602,7 +1637,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
   }
   const Dest d = make_dest(pl, a);
   if (tid == 0) {
-    if (!d.fits && blockIdx.x == 0) atomicMax(&a.sc->status, (unsigned long long)kErrCapacity);
+    if (!d.fits && blockIdx.x == 0) report_error(a, kErrCapacity);
     if (scan_on) s_ctl.d = d;
   }
   __syncthreads();
@@ -1639,7 +1674,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     team_minmax(team, lo, hi, rp);  // one barrier: also tells every thread about an abort
     if (s_abort) break;
     const float range = __fsub_rn(hi, lo), nlo = -lo;
-    if (!(fabsf(range) <= 3.402823466e38f) && tid == 0) atomicMax(&a.sc->status, (unsigned long long)kErrNonfinite);
+    if (!(fabsf(range) <= 3.402823466e38f) && tid == 0) report_error(a, kErrNonfinite);
 
     // ---- sweep 2: integer moments of the distances from lo, thresholds
     float dlo = 0.0f, dhi = 0.0f;
@@ -1730,7 +1765,7 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
   }
 
   if (s_abort && tid == 0) {  // a load timed out: report, then wait (bounded) for copies still in flight
-    atomicMax(&a.sc->status, (unsigned long long)kErrTimeout);
+    report_error(a, kErrTimeout);
     for (uint32_t k = 0; k < nstage; ++k)
       if (s_tiles[k] < pl.ntiles) {
         mbar_wait(&s_full[k], 0u, 1u << 10);

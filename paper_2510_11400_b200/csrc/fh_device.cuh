@@ -709,8 +709,11 @@ __device__ __noinline__ void huffman_tables(HufDecode* t) {
 // it waits for anything -- and a tile with U > 0 then needs the sum over all earlier tiles.  Two levels
 // keep that look-back short (sizes in units of 16 bytes):
 //   tile[t] = epoch << 32 | U_t          written once per call; an entry of another epoch reads as "not yet"
-//   grp[g]  = count << 40 | sum of U     over the tiles of group g = t >> 5 that have published (atomic adds;
-//                                        returned to zero by the call's last CTA)
+//   grp[g]  = count << 40 | sum of U     over the tiles of group g = t >> 5 that have published (atomic adds).
+//                                        Two sets alternate between consecutive calls on a scratch; a call's last
+//                                        CTA returns the set of the call BEFORE it to zero (grp_clear): every add
+//                                        of that call was performed when its kernel completed, so no fence is
+//                                        needed between a tile's add and the clearing store.
 //   gpre[g] = epoch << 32 | sum of U     over all tiles of groups 0..g, published by whoever has worked it out
 // Progress: tiles are taken in ticket order by CTAs that are running, a CTA works through its tiles in
 // increasing order, and a tile publishes before it waits; so the smallest tile that has not published is
@@ -719,10 +722,11 @@ struct Scan {
   unsigned long long* tile;
   unsigned long long* grp;
   unsigned long long* gpre;
+  unsigned long long* grp_clear;  // group sums the call's last CTA returns to zero (see above)
+  uint32_t clear_groups;          // ... and how many
   uint32_t epoch;      // of this call (never 0)
   uint32_t polls;      // limit of every wait, in polls of about 0.1 us
   uint32_t skip_tile;  // this tile never publishes (fault injection for the time-out test; 0xFFFFFFFF: none)
-  uint32_t reserved;
 };
 
 // One thread: tile t has measured its planes.
