@@ -271,6 +271,42 @@ __device__ __forceinline__ void decode_chunk32(const uint32_t (&w)[8], uint32_t 
   }
 }
 
+// The same for bf16 planes of whole 16-byte chunks: a lane restores two neighbouring groups at a time -- groups
+// g0 + 64 k + 2 l and the one after it -- so that eight values leave as one 16-byte store (four stores of 512
+// contiguous bytes per warp and chunk instead of eight of 256).
+template <int BITS>
+__device__ __forceinline__ void decode_chunk32_bf16_pairs(const uint32_t (&w)[8], uint32_t lane, uint32_t g0, uint32_t g1,
+                                                          float scale, float lo, uint8_t* out) {
+  constexpr uint32_t L = (1u << BITS) - 1u, full = 0xFFFFFFFFu;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const uint32_t g = g0 + (uint32_t)k * 64u + 2u * lane;
+    uint32_t wa, wb;  // code words of groups g and g + 1
+    if (BITS == 2) {         // a byte per group: halfword 32 k + l of the chunk = word 16 k + (l >> 1)
+      const uint32_t src = __shfl_sync(full, w[k >> 1], (uint32_t)(k & 1) * 16u + (lane >> 1));
+      const uint32_t h = src >> ((lane & 1u) * 16u);
+      wa = h & 0xFFu;
+      wb = (h >> 8) & 0xFFu;
+    } else if (BITS == 4) {  // two bytes per group: word 32 k + l, the lane's own
+      wa = w[k] & 0xFFFFu;
+      wb = w[k] >> 16;
+    } else {                 // a word per group: words 64 k + 2 l and the next, held by lanes 2 l mod 32 and the next
+      const uint32_t sl = (2u * lane) & 31u;
+      const uint32_t a0 = __shfl_sync(full, w[2 * k], sl), a1 = __shfl_sync(full, w[2 * k + 1], sl);
+      const uint32_t b0 = __shfl_sync(full, w[2 * k], sl + 1u), b1 = __shfl_sync(full, w[2 * k + 1], sl + 1u);
+      wa = lane < 16u ? a0 : a1;
+      wb = lane < 16u ? b0 : b1;
+    }
+    uint4 v;
+    v.x = f32x2_to_bf16x2(dequant(wa & L, scale, lo), dequant((wa >> BITS) & L, scale, lo));
+    v.y = f32x2_to_bf16x2(dequant((wa >> (2 * BITS)) & L, scale, lo), dequant((wa >> (3 * BITS)) & L, scale, lo));
+    v.z = f32x2_to_bf16x2(dequant(wb & L, scale, lo), dequant((wb >> BITS) & L, scale, lo));
+    v.w = f32x2_to_bf16x2(dequant((wb >> (2 * BITS)) & L, scale, lo), dequant((wb >> (3 * BITS)) & L, scale, lo));
+    if (g + 1u < g1) reinterpret_cast<uint4*>(out)[g >> 1] = v;
+    else if (g < g1) reinterpret_cast<uint2*>(out)[g] = make_uint2(v.x, v.y);
+  }
+}
+
 // Normal plane, sub-warp team of TT lanes (planes of at most 8 * TT groups, one chunk).  cw[k] holds the
 // code word of group lane + k * TT, requested before the table entry was known.  Whole groups of planes
 // that start on a vector boundary leave as one store; everything else (planes that do not, the ragged
@@ -394,7 +430,11 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
       if (cls == kClsNormal) {
         if (off != slots_off + gp * npay) { bad = true; continue; }
         const float lo = __uint_as_float(e.z), scale = __uint_as_float(e.w);
-        if (TT == 32) {
+        if (TT == 32 && DT == kBF16 && (pl.plane_bytes & 15u) == 0u) {
+          if (bits == 2u) decode_chunk32_bf16_pairs<2>(cw, lane, g0, g1, scale, lo, out);
+          else if (bits == 4u) decode_chunk32_bf16_pairs<4>(cw, lane, g0, g1, scale, lo, out);
+          else decode_chunk32_bf16_pairs<8>(cw, lane, g0, g1, scale, lo, out);
+        } else if (TT == 32) {
           if (bits == 2u) decode_chunk32<DT, 2>(cw, lane, g0, g1, scale, lo, out);
           else if (bits == 4u) decode_chunk32<DT, 4>(cw, lane, g0, g1, scale, lo, out);
           else decode_chunk32<DT, 8>(cw, lane, g0, g1, scale, lo, out);
