@@ -140,6 +140,15 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
       // fewer, busier threads win as long as enough warps stay resident)
       pl.team = pl.plane_bytes <= 16 * 1024 ? 128 : (pl.plane_bytes <= 64 * 1024 ? 256 : 512);
       v.G = 0;
+      // planes of up to 4096 groups: the register variant, with the smallest (threads, groups per thread)
+      // that holds the plane
+      static const uint32_t kCombo[6][2] = {{128, 7}, {128, 8}, {256, 7}, {256, 8}, {448, 7}, {512, 8}};
+      for (int k = 0; k < 6; ++k)
+        if (kCombo[k][0] * kCombo[k][1] >= pl.groups) {
+          pl.team = kCombo[k][0];
+          v.G = (int)kCombo[k][1];
+          break;
+        }
       pl.ppt = 1;
     }
     if (pl.ppt > pl.P) pl.ppt = (uint32_t)pl.P;
@@ -443,6 +452,21 @@ int launch_cta_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream)
              ? FH_OK : FH_ERR_CUDA;
 }
 
+template <int DT, bool SIGMA, int NT, int G>
+int launch_cta_regs_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
+  int grid = 0;
+  if (pl.groups == (uint32_t)(NT * G)) {
+    int rc = grid_for(fh::compress_cta_regs<DT, SIGMA, NT, G, true>, pl.sm_total, pl.ntiles, &grid, NT);
+    if (rc != FH_OK) return rc;
+    return launch_dependent(fh::compress_cta_regs<DT, SIGMA, NT, G, true>, grid, NT, pl.sm_total, stream,
+                            with_first_request(pl, grid, 2), a) == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+  }
+  int rc = grid_for(fh::compress_cta_regs<DT, SIGMA, NT, G, false>, pl.sm_total, pl.ntiles, &grid, NT);
+  if (rc != FH_OK) return rc;
+  return launch_dependent(fh::compress_cta_regs<DT, SIGMA, NT, G, false>, grid, NT, pl.sm_total, stream,
+                          with_first_request(pl, grid, 2), a) == cudaSuccess ? FH_OK : FH_ERR_CUDA;
+}
+
 template <int DT, bool SIGMA, int TT, bool FULLVEC>
 int launch_warp_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
   int grid = 0;
@@ -470,6 +494,17 @@ int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, c
   if (!v.cta) {
     const bool fullvec = pl.plane_bytes % 16 == 0 && pl.HW % 4 == 0 && pl.groups == 8u * pl.team;
     return fullvec ? launch_warp_tt<DT, SIGMA, true>(pl, a, stream) : launch_warp_tt<DT, SIGMA, false>(pl, a, stream);
+  }
+  if (v.G) {
+    switch (pl.team * 16 + v.G) {
+      case 128 * 16 + 7: return launch_cta_regs_t<DT, SIGMA, 128, 7>(pl, a, stream);
+      case 128 * 16 + 8: return launch_cta_regs_t<DT, SIGMA, 128, 8>(pl, a, stream);
+      case 256 * 16 + 7: return launch_cta_regs_t<DT, SIGMA, 256, 7>(pl, a, stream);
+      case 256 * 16 + 8: return launch_cta_regs_t<DT, SIGMA, 256, 8>(pl, a, stream);
+      case 448 * 16 + 7: return launch_cta_regs_t<DT, SIGMA, 448, 7>(pl, a, stream);
+      case 512 * 16 + 8: return launch_cta_regs_t<DT, SIGMA, 512, 8>(pl, a, stream);
+    }
+    return FH_ERR_UNSUPPORTED;
   }
   switch (pl.team) {
     case 128: return launch_cta_t<DT, SIGMA, 128>(pl, a, stream);

@@ -1110,7 +1110,8 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
       long long Is, Iq;
       team_sum2(team, (int32_t)(as - (uint32_t)G * kMagicBits), (int32_t)(aq - (uint32_t)G * kMagicBits), Is, Iq, rp);
       float dlo, dhi;
-      sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, dlo, dhi);
+      if (TT > 32) sigma_thresholds(Is, Iq, sc, pl.inv_hw, dlo, dhi);  // (a CTA team's sums may pass 32 bits)
+      else sigma_thresholds((int32_t)Is, (int32_t)Iq, sc, pl.inv_hw, dlo, dhi);
       uint32_t cnt = 0;
       if (range > dhi || 0.0f < dlo) {  // otherwise no element can lie outside: the count is zero
         uint32_t c[4] = {0, 0, 0, 0};  // four counters: short dependency chains
@@ -1764,6 +1765,110 @@ __global__ void __launch_bounds__(NT) compress_cta(const Plan pl, const Compress
     // s_tiles[s] for the next iteration was written at least one barrier ago (nstage >= 2)
   }
 
+  if (s_abort && tid == 0) {  // a load timed out: report, then wait (bounded) for copies still in flight
+    report_error(a, kErrTimeout);
+    for (uint32_t k = 0; k < nstage; ++k)
+      if (s_tiles[k] < pl.ntiles) {
+        mbar_wait(&s_full[k], 0u, 1u << 10);
+        mbar_wait(&s_full[k], 1u, 1u << 10);
+      }
+  }
+  if (scan_on) {
+    __syncthreads();
+    if (s_ctl.head != kNoTile && !s_abort)
+      cta_phase2<DT, NT>(&s_ctl, s_red, smem + pl.sm_tile, sal, &s_full[0], phase & 1u);
+  }
+  cta_exit(pl, a, d, &s_last);
+}
+
+// -------------------------------------------------------------------------------------------------
+// CTA-team kernel, register variant: planes of 257 to NT * G groups (whole 16-byte chunks).  As compress_cta, but
+// every thread takes its G groups out of the stage once and keeps them in registers for the whole sweep
+// (plane_sweep with the CTA as the team): one pass over shared memory instead of three, the distances
+// computed once.  A normal plane's stage is free as soon as the sweep returns -- its last read of the stage
+// lies before the first reduction's barrier -- and takes the next load at once.
+// -------------------------------------------------------------------------------------------------
+template <int DT, bool SIGMA, int NT, int G, bool FULL>
+__global__ void __launch_bounds__(NT, NT > 256 ? 2 : (NT > 128 ? 3 : 6)) compress_cta_regs(const Plan pl, const CompressArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  __shared__ double s_red[kMaxWarps * 5];
+  __shared__ __align__(8) uint64_t s_full[kMaxStages];
+  __shared__ uint32_t s_tiles[kMaxStages];
+  __shared__ uint32_t s_abort, s_last;
+  __shared__ BlockCtl s_ctl;
+
+  const uint32_t tid = threadIdx.x;
+  const Team team = make_team(NT, s_red);
+  const uint32_t nstage = pl.nstage;
+  const bool scan_on = pl.mode != kModeOff;
+  uint32_t* sal = reinterpret_cast<uint32_t*>(smem + pl.sm_sal);
+  uint32_t rp = 0;
+  // Thread 0 requests the tiles and issues the loads: the first nstage tiles in one request, later ones one
+  // at a time, the request running one tile ahead of its use.  Tiles come in ticket order.
+  uint32_t next_ticket = 0, issued = 0;
+  if (tid == 0) {
+    for (uint32_t s = 0; s < nstage; ++s) mbar_init(&s_full[s], 1);
+    fence_mbar_init();
+    s_abort = 0;
+    *cta_dirty() = 0u;
+    if (a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
+    if (scan_on) {  // (before the wait for the previous kernel, whose tail hides it)
+      s_ctl.pl = pl;
+      s_ctl.a = a;
+      s_ctl.head = kNoTile;
+    }
+  }
+  dep_wait();     // the previous kernel on the stream has completed; global memory may be touched from here on
+  dep_trigger();  // the next kernel on the stream may become resident as this one drains
+  auto issue = [&](uint32_t s) {
+    const uint32_t t = next_ticket;
+    s_tiles[s] = t;
+    if (t < pl.ntiles) {
+      fence_proxy_async();
+      mbar_expect_tx(&s_full[s], (uint32_t)pl.plane_bytes);
+      bulk_g2s(smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes, a.src + (uint64_t)t * pl.plane_bytes,
+               (uint32_t)pl.plane_bytes, &s_full[s]);
+      ++issued;
+      next_ticket = issued < nstage ? t + 1u : (uint32_t)atomicAdd(&a.sc->ticket[a.parity], 1ull);
+    }
+  };
+  if (tid == 0) {  // the first loads before anything else
+    if (!a.early_ticket) next_ticket = (uint32_t)atomicAdd(&a.sc->ticket[a.parity], (unsigned long long)nstage);
+    for (uint32_t s = 0; s < nstage; ++s) issue(s);
+  }
+  const Dest d = make_dest(pl, a);
+  if (tid == 0) {
+    if (!d.fits && blockIdx.x == 0) report_error(a, kErrCapacity);
+    if (scan_on) s_ctl.d = d;
+  }
+  __syncthreads();
+
+  uint32_t s = 0, phase = 0;
+  for (;;) {
+    const uint32_t tile = s_tiles[s];
+    if (tile >= pl.ntiles) break;
+    bool ready = mbar_wait(&s_full[s], (phase >> s) & 1u, 1u << 20);
+    phase ^= 1u << s;
+    if (!__syncthreads_and(ready)) {  // a load timed out (the same answer for every thread)
+      if (tid == 0) s_abort = 1;
+      break;
+    }
+    const uint8_t* plane = smem + pl.sm_tile + (uint64_t)s * pl.stage_bytes;
+    const uint32_t meta = plane_sweep<DT, SIGMA, G, NT, FULL, true>(team, pl, d, a, plane, (uint64_t)tile, rp);
+    if ((meta & 3u) == kClsNormal) {  // (the same for every thread) complete; every read of the stage lies behind a barrier
+      if (tid == 0) {
+        if (scan_on) scan_publish(a.scan, tile, 0u);
+        issue(s);
+      }
+    } else {  // phase 1 of the block-wise path
+      cta_tile_measure<DT, NT>(&s_ctl, s_red, plane, sal, tile, meta);
+      __syncthreads();  // every thread is done with the stage
+      if (tid == 0) issue(s);
+    }
+    s = s + 1 == nstage ? 0 : s + 1;
+    // s_tiles[s] for the next iteration was written at least one barrier ago (nstage >= 2)
+  }
+  __syncthreads();
   if (s_abort && tid == 0) {  // a load timed out: report, then wait (bounded) for copies still in flight
     report_error(a, kErrTimeout);
     for (uint32_t k = 0; k < nstage; ++k)
