@@ -15,7 +15,7 @@ DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("fh_device.cuh", "fh_channel.c
 
 def nvcc_cmd(extra=()):
     return ["nvcc", "-std=c++17", "-O3", "-lineinfo", "-gencode", "arch=compute_100a,code=sm_100a",
-            "-Xcompiler", "-fPIC", "-shared", "--fmad=false", "-split-compile=0", "-o", LIB, *extra, *SOURCES]
+            "-Xcompiler", "-fPIC", "-shared", "--fmad=false", "-o", LIB, *extra, *SOURCES]
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

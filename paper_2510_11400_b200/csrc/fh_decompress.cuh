@@ -231,6 +231,32 @@ __device__ __forceinline__ uint32_t check_header(const Plan& pl, const uint8_t* 
   return ok ? version : 0u;
 }
 
+// Last step of every CTA.  The exit counter carries the CTAs that have left in its low half and, in its high half,
+// how many of them had found something wrong; only such a CTA reports and fences, and the last CTA reads the
+// status back only when there was one: a clean call ends with one atomic per CTA.  (The restored tensor needs no
+// fence: its readers are later kernels.)
+__device__ __forceinline__ void decompress_exit(const DecompressArgs& a, bool bad) {
+  const bool any_bad = __syncthreads_or(bad) != 0;  // (the same for every thread)
+  if (any_bad) {
+    if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
+    __threadfence();
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const unsigned long long old = atomicAdd(&a.sc->exited, 1ull | (any_bad ? 1ull << 32 : 0ull));
+    if ((uint32_t)old == gridDim.x - 1u) {
+      uint32_t code = kErrNone;
+      if ((old >> 32) != 0ull || any_bad) {
+        __threadfence();
+        code = (uint32_t)ld_relaxed(&a.sc->status);
+        st_relaxed(&a.sc->status, 0ull);
+      }
+      if (a.d_status) *a.d_status = status_word(code);
+      st_relaxed(&a.sc->exited, 0ull);
+    }
+  }
+}
+
 // Four restored values of one group leave as one 16-byte (fp32) or 8-byte (bf16) store.
 template <int DT>
 __device__ __forceinline__ void store_group(uint8_t* out, uint32_t g, float v0, float v1, float v2, float v3) {
@@ -506,19 +532,7 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_kernel(const Plan pl, 
       __syncthreads();  // the scratch is reused
     }
   }
-  if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned long long prev = atomicAdd(&a.sc->exited, 1ull);
-    if (prev == (unsigned long long)gridDim.x - 1ull) {
-      __threadfence();
-      const uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
-      if (a.d_status) *a.d_status = status_word(code);
-      st_relaxed(&a.sc->status, 0ull);
-      st_relaxed(&a.sc->exited, 0ull);
-    }
-  }
+  decompress_exit(a, bad);
 }
 
 // -------------------------------------------------------------------------------------------------
@@ -812,19 +826,7 @@ __global__ void __launch_bounds__(kThreads, 4) decompress_small(const Plan pl, c
     }
     if (tid == 0) bulk_wait<0>();  // every store of this CTA is complete
   }
-  if (bad) atomicMax(&a.sc->status, (unsigned long long)kErrCorrupt);
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const unsigned long long prev = atomicAdd(&a.sc->exited, 1ull);
-    if (prev == (unsigned long long)gridDim.x - 1ull) {
-      __threadfence();
-      const uint32_t code = (uint32_t)ld_relaxed(&a.sc->status);
-      if (a.d_status) *a.d_status = status_word(code);
-      st_relaxed(&a.sc->status, 0ull);
-      st_relaxed(&a.sc->exited, 0ull);
-    }
-  }
+  decompress_exit(a, bad);
 }
 
 }  // namespace fh
