@@ -117,6 +117,18 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append([c.strip() for c in line.split(",")])
 
+    def keep_busy(self, step, want: int, limit_s: float):
+        """Repeats `step` (untimed) until `want` samples have come in or `limit_s` seconds have passed: the
+        timed region of a short run is over before nvidia-smi has answered once, so the same load is kept up
+        on both sides of it and the samples are those of that load."""
+        if self.proc is None:
+            return
+        import torch
+        t0 = time.perf_counter()
+        while len(self.rows) < want and time.perf_counter() - t0 < limit_s:
+            step()
+            torch.cuda.synchronize()
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -389,20 +401,26 @@ def run_ours(args, specs, wl_desc):
     evs = [{b: [torch.cuda.Event(enable_timing=True) for _ in range(3)] for b in BITS} for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local)
+    sampler.start()
+    if not args.no_clock_window:
+        sampler.keep_busy(step, 2, 3.0)  # (untimed) the load is running when the first samples are taken
     if world > 1:
         dist.barrier()
     torch.cuda.synchronize()
     launches0 = api.kernel_launches()
-    sampler.start()
     e0.record(stream)
     for k in range(args.steps):
         step(evs[k])
     e1.record(stream)
     torch.cuda.synchronize()
+    launches = api.kernel_launches() - launches0
     if world > 1:
         dist.barrier()
+    if not args.no_clock_window:
+        sampler.keep_busy(step, len(sampler.rows) + 4, 1.5)  # (untimed) ... and still running for the last ones
     clocks = sampler.stop()
-    launches = api.kernel_launches() - launches0
+    if not args.no_clock_window:
+        clocks["window"] = "the same step repeated back to back, untimed, before and after the timed steps"
     ms = e0.elapsed_time(e1)
     ms = slowest_rank(ms, world, dev)
     t_comp = {b: sum(e[b][0].elapsed_time(e[b][1]) for e in evs) for b in BITS}
@@ -598,11 +616,13 @@ def main():
     ap.add_argument("--workload", default="resnet18_b64")
     ap.add_argument("--mode", default="auto", choices=["auto", "off", "all", "channel", "tensor"])
     ap.add_argument("--rounding", type=int, default=0, choices=[0, 1],
-                    help="1: random rounding of normal planes (runs on the general-purpose kernel)")
+                    help="1: random rounding of normal planes (Philox-4x32-10 draws)")
     ap.add_argument("--schedule", action="store_true",
                     help="run the workload through fh_run_schedule (forward-order compress, reverse-order decompress)")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-clock-window", action="store_true",
+                    help="do not repeat the step (untimed) around the timed region for the clock samples: for runs under a profiler")
     ap.add_argument("--no-sweep", action="store_true", help="skip the size sweep and the schedule leg of the default workload")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

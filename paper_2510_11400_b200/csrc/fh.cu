@@ -124,10 +124,12 @@ int make_plan(const fh_tensor_desc* d, const fh_params* p, bool compress, Plan* 
   Variant v;
   // ---- fast compress kernels: planes of whole 16-byte chunks whose groups fit the register budget
   const bool whole16 = pl.HW % 4 == 0 && pl.plane_bytes % 16 == 0;
-  // (random rounding and the Huffman stage run on the generic kernel)
+  // (the Huffman stage runs on the generic kernel; random rounding on the warp-team kernels in the plane-wise
+  // three-sigma mode, on the generic kernel otherwise)
   // (a warp-team kernel keeps one measuring area per warp: planes whose area is large -- very tall, narrow
   // ones -- go to the general-purpose kernel)
-  if (compress && pl.rounding == 0 && pl.entropy == 0 && ((pl.groups <= 256 && (!blockwise || sal_bytes <= 1024)) || (pl.groups > 256 && whole16))) {
+  const bool rounding_ok = pl.rounding == 0 || (pl.groups <= 256 && pl.mode == FH_SALIENT_AUTO);
+  if (compress && rounding_ok && pl.entropy == 0 && ((pl.groups <= 256 && (!blockwise || sal_bytes <= 1024)) || (pl.groups > 256 && whole16))) {
     v.fast = true;
     if (pl.groups <= 256) {
       uint32_t t = pow2_ceil((pl.groups + 7) / 8);
@@ -467,7 +469,7 @@ int launch_cta_regs_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t st
                           with_first_request(pl, grid, 2), a) == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
-template <int DT, bool SIGMA, int TT, bool FULLVEC>
+template <int DT, int SIGMA, int TT, bool FULLVEC>
 int launch_warp_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
   int grid = 0;
   int rc = grid_for(fh::compress_warp<DT, SIGMA, TT, FULLVEC>, pl.sm_total, pl.ntiles, &grid, fh::kWarpKernelThreads);
@@ -476,7 +478,7 @@ int launch_warp_t(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream
                           with_first_request(pl, grid, 1), a) == cudaSuccess ? FH_OK : FH_ERR_CUDA;
 }
 
-template <int DT, bool SIGMA, bool FULLVEC>
+template <int DT, int SIGMA, bool FULLVEC>
 int launch_warp_tt(const Plan& pl, const fh::CompressArgs& a, cudaStream_t stream) {
   switch (pl.team) {
     case 1: return launch_warp_t<DT, SIGMA, 1, FULLVEC>(pl, a, stream);
@@ -490,11 +492,20 @@ int launch_warp_tt(const Plan& pl, const fh::CompressArgs& a, cudaStream_t strea
 }
 
 template <int DT, bool SIGMA>
+int launch_cta_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream);
+
+template <int DT, int SIGMA>
 int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
   if (!v.cta) {
     const bool fullvec = pl.plane_bytes % 16 == 0 && pl.HW % 4 == 0 && pl.groups == 8u * pl.team;
     return fullvec ? launch_warp_tt<DT, SIGMA, true>(pl, a, stream) : launch_warp_tt<DT, SIGMA, false>(pl, a, stream);
   }
+  if constexpr (SIGMA == 2) return FH_ERR_UNSUPPORTED;  // (make_plan sends random rounding on large planes elsewhere)
+  else return launch_cta_g<DT, SIGMA != 0>(pl, v, a, stream);
+}
+
+template <int DT, bool SIGMA>
+int launch_cta_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
   if (v.G) {
     switch (pl.team * 16 + v.G) {
       case 128 * 16 + 7: return launch_cta_regs_t<DT, SIGMA, 128, 7>(pl, a, stream);
@@ -517,11 +528,13 @@ int launch_fast_g(const Plan& pl, const Variant& v, const fh::CompressArgs& a, c
 int launch_compress(const Plan& pl, const Variant& v, const fh::CompressArgs& a, cudaStream_t stream) {
   int rc;
   if (v.fast) {
-    const bool sigma = pl.mode == FH_SALIENT_AUTO;
+    const int sigma = pl.mode == FH_SALIENT_AUTO ? (pl.rounding ? 2 : 1) : 0;
     if (pl.dtype == FH_F32)
-      rc = sigma ? launch_fast_g<fh::kF32, true>(pl, v, a, stream) : launch_fast_g<fh::kF32, false>(pl, v, a, stream);
+      rc = sigma == 2 ? launch_fast_g<fh::kF32, 2>(pl, v, a, stream)
+           : sigma    ? launch_fast_g<fh::kF32, 1>(pl, v, a, stream) : launch_fast_g<fh::kF32, 0>(pl, v, a, stream);
     else
-      rc = sigma ? launch_fast_g<fh::kBF16, true>(pl, v, a, stream) : launch_fast_g<fh::kBF16, false>(pl, v, a, stream);
+      rc = sigma == 2 ? launch_fast_g<fh::kBF16, 2>(pl, v, a, stream)
+           : sigma    ? launch_fast_g<fh::kBF16, 1>(pl, v, a, stream) : launch_fast_g<fh::kBF16, 0>(pl, v, a, stream);
   } else if (pl.dtype == FH_F32) {
     rc = pl.bits == 2   ? launch_generic_t<fh::kF32, 2>(pl, a, stream)
          : pl.bits == 4 ? launch_generic_t<fh::kF32, 4>(pl, a, stream)

@@ -1015,7 +1015,8 @@ __global__ void __launch_bounds__(kThreads) compress_generic(const Plan pl, cons
 // TT: team size (1..32), a compile-time constant so that the strides between a thread's groups are
 // immediates.  FULL: groups == G * TT.  VEC: planes are whole 16-byte chunks (vector loads, no ragged last
 // group).  Returns class | n_out << 2; a normal plane is complete when the function returns.
-template <int DT, bool SIGMA, int G, int TT, bool FULL, bool VEC>
+// SIGMA: 0 no three-sigma statistics, 1 the plane's own, 2 the same with random rounding of the codes.
+template <int DT, int SIGMA, int G, int TT, bool FULL, bool VEC>
 __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl, const Dest& d, const CompressArgs& a,
                                                 const uint8_t* plane, uint64_t gp, uint32_t& rp) {
   // A thread's G group slots that lie past the plane, and the elements past a ragged last group, are
@@ -1148,7 +1149,26 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
   float inv, scale;
   quant_params(range, (1u << bits) - 1u, inv, scale);
   uint8_t* slot = d.dst + pl.slots_off + gp * pl.npay;
-  if (bits == 2u) FH_STORE_CODES(2)
+  if (SIGMA == 2) {
+    // random rounding: one generator call per group, counter = (group, plane, tensor id), key = seed; a padded
+    // position (distance 0) gets code 0 whatever the draw
+    const uint32_t L = (1u << bits) - 1u;
+#pragma unroll
+    for (int k = 0; k < G; ++k) {
+      const uint32_t g = lane + (uint32_t)(k * TT);
+      if (FULL || g < groups) {
+        uint32_t rnd[4];
+        philox4x32_10(g, (uint32_t)gp, (uint32_t)pl.tensor_id, (uint32_t)(pl.tensor_id >> 32), (uint32_t)pl.seed,
+                      (uint32_t)(pl.seed >> 32), rnd);
+        uint32_t word = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) word |= quant_code_random(x[k][e], inv, L, rnd[e]) << (e * bits);
+        if (bits == 2u) slot[g] = (uint8_t)word;
+        else if (bits == 4u) reinterpret_cast<uint16_t*>(slot)[g] = (uint16_t)word;
+        else reinterpret_cast<uint32_t*>(slot)[g] = word;
+      }
+    }
+  } else if (bits == 2u) FH_STORE_CODES(2)
   else if (bits == 4u) FH_STORE_CODES(4)
   else FH_STORE_CODES(8)
   // zero padding of the slot behind the codes
@@ -1164,7 +1184,7 @@ __device__ __forceinline__ uint32_t plane_sweep(const Team& team, const Plan& pl
 
 // Picks the specialisation of the sweep.  FULLVEC kernels are launched only for planes of exactly
 // G * TT whole groups, so they carry nothing but the lean variant; the others choose at run time.
-template <int DT, bool SIGMA, int G, int TT, bool FULLVEC>
+template <int DT, int SIGMA, int G, int TT, bool FULLVEC>
 __device__ __forceinline__ uint32_t plane_sweep_any(const Team& team, const Plan& pl, const Dest& d,
                                                     const CompressArgs& a, const uint8_t* plane, uint64_t gp,
                                                     bool vec, uint32_t& rp) {
@@ -1300,7 +1320,7 @@ __device__ __noinline__ void warp_phase2(BlockCtl* c, uint8_t* stages, uint8_t* 
   }
 }
 
-template <int DT, bool SIGMA, int TT, bool FULLVEC>
+template <int DT, int SIGMA, int TT, bool FULLVEC>
 __global__ void __launch_bounds__(kWarpKernelThreads, 3) compress_warp(const Plan pl, const CompressArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ double s_red[kMaxWarps * 5];
