@@ -343,8 +343,8 @@ def test_launch_counter_counts_our_kernels():
 def test_back_to_back_calls_without_host_synchronisation():
     """Several tensors with outlier-rich planes, compressed and restored back to back on one stream for
     three rounds with no host synchronisation in between: kernels of consecutive calls overlap at their
-    edges, and the block-wise kernel's barrier over its grid must still complete (every status word 0);
-    the last round is compared with the oracle."""
+    edges, share the per-stream counters and alternate between the two sets of the placement scan's group
+    sums; every wait must still end (every status word 0); the last round is compared with the oracle."""
     import torch
     specs = [synth.TensorSpec("a", (8, 96, 112, 112), synth.BF16, "laplace_ch", 21),
              synth.TensorSpec("b", (16, 144, 56, 56), synth.BF16, "laplace_ch", 22),
