@@ -114,6 +114,44 @@ def test_parity_auto_mode_mixed_planes(shape, dtype, bits):
     full_parity(spec, bits=bits)
 
 
+# Planes of 257 to 4096 groups run on the CTA-team kernel that keeps a thread's groups in registers: one shape per
+# (threads, groups per thread) it is built for, each with a plane that fills the threads exactly and one that does
+# not, and one shape beyond it (the kernel that sweeps the plane in shared memory).
+CTA_SHAPES = [
+    (1, 4, 56, 64), (1, 4, 57, 60),      # 896 groups = 128 x 7; 855
+    (1, 4, 64, 64), (1, 4, 40, 100),     # 1024 = 128 x 8; 1000
+    (1, 4, 64, 112), (1, 4, 60, 100),    # 1792 = 256 x 7; 1500
+    (1, 4, 128, 64), (1, 4, 80, 100),    # 2048 = 256 x 8; 2000
+    (1, 4, 112, 112), (1, 4, 100, 120),  # 3136 = 448 x 7; 3000
+    (1, 4, 128, 128), (1, 4, 100, 160),  # 4096 = 512 x 8; 4000
+    (1, 3, 160, 164),                    # 6560 groups: beyond the register variant
+]
+
+
+@pytest.mark.parametrize("shape", CTA_SHAPES)
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_parity_cta_team_kernels(shape, dtype):
+    full_parity(synth.TensorSpec("t", shape, dtype, "spiky_relu", 61), bits=2)
+    full_parity(synth.TensorSpec("t", shape, dtype, "normal", 62), bits=8, salient_mode=api.FH_SALIENT_OFF)
+
+
+@pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
+def test_moment_sums_of_a_cta_team_beyond_32_bits(dtype):
+    """Planes whose elements all lie near the maximum, with a single small one: every group's scaled sums are
+    near their largest, and over 3136 groups the integer moment sums pass 2^32 (a warp team's never can)."""
+    shape = (1, 6, 112, 112)
+    rng = np.random.default_rng(5)
+    x = (1000.0 + rng.random(shape, dtype=np.float32)).astype(np.float32)
+    x[0, :, 3, 5] = 0.0                                  # the minimum: distances of about the range everywhere else
+    x[0, 1::2, 60:70, 40:90] = 2000.0                    # every other plane: 500 far elements (outlier-rich or not, the oracle says)
+    raw = synth.to_bf16_bits(x).reshape(shape) if dtype == synth.BF16 else x
+    st_o, buf_o, total_o, d = oracle_compress(raw, shape, dtype, bits=4)
+    assert st_o == fho.OK
+    st_g, packed, total_g = gpu_compress(raw, shape, dtype, bits=4)
+    assert st_g == api.FH_OK and total_g == total_o
+    assert np.array_equal(packed[:total_g].cpu().numpy(), buf_o)
+
+
 @pytest.mark.parametrize("shape", SHAPES)
 @pytest.mark.parametrize("dtype", [synth.F32, synth.BF16])
 @pytest.mark.parametrize("mode", [api.FH_SALIENT_OFF, api.FH_SALIENT_ALL])
@@ -403,6 +441,37 @@ def _full_size(spec, bits_list):
         out[bits] = buf_o
         del packed, out_g
     return out
+
+
+def test_calls_with_and_without_the_placement_scan_interleaved_on_one_stream():
+    """Calls that place overflow parts alternate between two sets of group sums, and a call clears the set of
+    the last call that used the scan; calls with the three-sigma rule off use neither.  Mixed on one stream,
+    with tensors of different tile counts, every container must still equal the oracle's."""
+    import torch
+    seq = [("a", (4, 40, 14, 14), "spiky_relu", api.FH_SALIENT_AUTO), ("b", (2, 64, 7, 7), "normal", api.FH_SALIENT_OFF),
+           ("c", (16, 96, 7, 7), "spiky_relu", api.FH_SALIENT_AUTO), ("d", (1, 8, 56, 56), "spiky_relu", api.FH_SALIENT_ALL),
+           ("e", (2, 9, 14, 14), "relu", api.FH_SALIENT_OFF), ("f", (1, 300, 4, 4), "spiky_relu", api.FH_SALIENT_AUTO),
+           ("g", (4, 40, 14, 14), "spiky_relu", api.FH_SALIENT_AUTO)]
+    items = []
+    for i, (name, shape, kind, mode) in enumerate(seq):
+        sp = synth.TensorSpec(name, shape, synth.F32, kind, 70 + i)
+        raw = synth.make(sp)
+        d = api.desc(shape, synth.F32)
+        p = api.default_params(bits=4, salient_mode=mode)
+        cap = api.compressed_bytes(d, p, 1)
+        items.append(dict(sp=sp, raw=raw, d=d, p=p, cap=cap, x=to_dev(raw), mode=mode,
+                          dst=torch.empty(cap, dtype=torch.uint8, device="cuda"),
+                          o=torch.zeros(2, dtype=torch.int64, device="cuda")))
+    for rnd in range(3):
+        for t in items:
+            assert api.fh_compress(t["d"], t["p"], t["x"], t["dst"], t["o"], capacity=t["cap"]) == api.FH_OK
+    torch.cuda.synchronize()
+    for t in items:
+        assert int(t["o"][1]) == 0
+        st_o, buf_o, total_o, _ = oracle_compress(t["raw"], t["sp"].shape, synth.F32, bits=4, salient_mode=t["mode"])
+        assert st_o == fho.OK and int(t["o"][0]) == total_o
+        assert np.array_equal(t["dst"][:total_o].cpu().numpy(), buf_o), t["sp"].name
+
 
 
 @pytest.mark.parametrize("index", range(17))
