@@ -524,7 +524,7 @@ def run_ours(args, specs, wl_desc):
             "compress_gbs": {str(b): args.steps * dense_bytes / t_comp[b] / 1e6 for b in BITS},
             "decompress_gbs": {str(b): args.steps * dense_bytes / t_dec[b] / 1e6 for b in BITS},
             "roofline": {"bound": "hbm",
-                         "kernel": "compress call = one kernel (compress_warp / compress_cta / compress_generic by plane "
+                         "kernel": "compress call = one kernel (compress_warp / compress_cta_regs / compress_cta / compress_generic by plane "
                                    "size); averaged over every compress call of the timed region",
                          "achieved": achieved, "peak": peak,
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak, "traffic": traffic,
