@@ -52,6 +52,9 @@ def workload_specs(name: str):
     if name == "mobilenetv2_b128":
         return synth.config3(128), "configs[2]: MobileNetV2-shaped expanded activations, batch 128, bf16, Laplace(0,1) " \
                                    "with channel-clustered +-50 outliers"
+    if name == "mobilenetv2_b128_iid":
+        return synth.config3(128, stress=True), "configs[2]: MobileNetV2-shaped expanded activations, batch 128, bf16, " \
+                                                "Laplace(0,1) with 1 % outliers at +-50, independent per element"
     if name == "cifar_schedule":
         return synth.config5(128), "configs[4]: 20 ResNet-18/CIFAR-shaped tensors, batch 128, fp32"
     if name == "config1":
